@@ -1,0 +1,286 @@
+/*
+ * grace.h -- C ABI of the B200 decode-step library (libgrace_b200.so).
+ *
+ * One decode step of a GTM-constrained, wide-beam, short-sequence SID decoder
+ * (GRACE, Sections 3.1-3.3, 4.1-4.4, 5.1-5.4):
+ *
+ *   cross-attention  beams of a request as query rows against shared K/V   grace_cross_attn
+ *   self-attention   over a parent-addressed KV cache, fused cache write   grace_self_attn
+ *   CD + GTM mask    and score add on next-token log-probabilities          grace_gtm_mask
+ *   beam top-k       per request over beam x codebook candidates            grace_beam_topk
+ *   state update     node ids / keys of the selected children               grace_beam_update
+ *   whole step       decoder layers + the four ops above                    grace_decode_step
+ *
+ * Conventions (all functions):
+ *   - Pointers named d_* or documented "device" are device pointers; "host" are host pointers.
+ *   - Every buffer is caller-owned; the library never allocates or frees device memory and
+ *     never synchronises.  Work is enqueued on `stream` (a cudaStream_t passed as void*); the
+ *     buffers must stay alive until the stream has passed the call.
+ *   - Rows are request-major: row r = b * M + m (Appendix B).
+ *   - Return value: GRACE_OK or an error detected on the host before anything is enqueued.
+ *   - `d_status` (device int32*, may be NULL): conditions detected on the device are OR-ed
+ *     into it (GRACE_DEV_* bits).  The caller zeroes it.
+ *   - bf16 tensors are passed as uint16_t* holding bf16 bit patterns.
+ */
+#ifndef GRACE_H_
+#define GRACE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GRACE_OK = 0,
+  GRACE_INVALID_ARG = 1,        /* null pointer, misaligned pointer, negative size         */
+  GRACE_UNSUPPORTED_SHAPE = 2,  /* shape outside what the kernels are built for            */
+  GRACE_WORKSPACE_TOO_SMALL = 3,
+  GRACE_CUDA_ERROR = 4,         /* a CUDA runtime / driver call failed                     */
+  GRACE_TIMEOUT = 5
+} grace_status_t;
+
+/* bits OR-ed into *d_status by kernels */
+#define GRACE_DEV_BAD_INDEX 1   /* a gathered index was out of range; the access was skipped */
+#define GRACE_DEV_NAN 2         /* NaN among log-probs / candidates (precondition violated)   */
+#define GRACE_DEV_TIMEOUT 4     /* a bounded device-side wait ran out                        */
+#define GRACE_DEV_TOPK_EXACT_PATH 8 /* informational: top-k fell back to the multi-pass path  */
+
+const char* grace_status_string(grace_status_t s);
+/* Library version, and the compute capability the kernels were built for (100 = sm_100a). */
+int grace_version(void);
+int grace_built_for_sm(void);
+
+/* ------------------------------------------------------------------------------------------
+ * Index structures (Section 4.4, Appendix A).
+ *
+ * The trie is held in its per-node child-bitmask form: node ids are assigned level by level
+ * (root = 0) and, inside a level, in lexicographic prefix order, so the children of a node are
+ * consecutive ids in token order and
+ *     child(n, v) = child_base[n] + popcount(child_bits[n] restricted to tokens < v).
+ * CD_t[v] (Section 4.1) is bit v of child_bits[n].  Only nodes of levels 0..L-1 have rows.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t V;                    /* vocabulary size per position; multiple of 64, <= 65535 - 1 */
+  int32_t L;                    /* SID length                                             */
+  int64_t num_nodes;            /* all nodes, leaves included                             */
+  int64_t num_internal;         /* nodes of levels 0..L-1 (those with rows below)         */
+  const uint64_t* child_bits;   /* device [num_internal][V/64]; token v = bit v&63 of word v>>6 */
+  const int32_t* child_base;    /* device [num_internal]; id of the first child, -1 if none */
+} grace_trie_t;
+
+typedef enum {
+  GRACE_MATCH_NONE = 0,         /* TM = 1: constrained decoding only                      */
+  GRACE_MATCH_NODE_BITMASK = 1, /* per request, one eligibility bit per trie node         */
+  GRACE_MATCH_PREFIX_BLOOM = 2  /* per request, a Bloom filter over prefix keys           */
+} grace_matcher_kind_t;
+
+/* TM_t[v] = match(u, p || v) (Section 4.1) in its per-request forms.
+ *   NODE_BITMASK: bits = device uint64 [B][words_per_request]; node n is bit n&63 of word n>>6;
+ *                 a prefix is eligible iff its subtree holds an eligible SID.
+ *   PREFIX_BLOOM: bits = device uint64 [B][words_per_request], words_per_request = 2^log2_bits/64.
+ *                 key(p) = sum_i (token_i + 1) << 16 i;  z = splitmix64 finaliser of key;
+ *                 h1 = low 32 bits, h2 = high 32 bits | 1; probe_i = (h1 + i*h2) mod 2^32 mod 2^log2_bits,
+ *                 i = 0 .. n_hashes-1.  Member iff all probed bits are set. */
+typedef struct {
+  int32_t kind;
+  int32_t bloom_log2_bits;
+  int32_t bloom_hashes;
+  int32_t reserved;
+  int64_t words_per_request;
+  const uint64_t* bits;
+} grace_matcher_t;
+
+/* Host-side index builders (not on the timed path; host memory in, host memory out).
+ * `sids` is host int32 [n_sids][L], lexicographically sorted and distinct (else INVALID_ARG). */
+
+/* level_start: host int64 [L+2]; level_start[l] = id of the first node of level l,
+ * level_start[L+1] = num_nodes. */
+grace_status_t grace_trie_count_nodes(const int32_t* sids, int64_t n_sids, int V, int L,
+                                      int64_t* level_start);
+/* child_bits host uint64 [level_start[L]][V/64], child_base host int32 [level_start[L]]. */
+grace_status_t grace_trie_build_dense(const int32_t* sids, int64_t n_sids, int V, int L,
+                                      uint64_t* child_bits, int32_t* child_base);
+/* node_bits host uint64 [ceil(num_nodes/64)], zeroed by the callee: upward closure of the
+ * eligible SIDs (eligible: host uint8 [n_sids], non-zero = eligible). */
+grace_status_t grace_node_bitmask_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                        const uint8_t* eligible, uint64_t* node_bits);
+/* bloom_words host uint64 [2^log2_bits / 64], zeroed by the callee: keys of every prefix
+ * (length 1..L) of every eligible SID. */
+grace_status_t grace_bloom_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                 const uint8_t* eligible, int log2_bits, int n_hashes,
+                                 uint64_t* bloom_words);
+/* Node id of a prefix (host tokens[len]) in a host copy of the dense trie; *node = -1 if the
+ * prefix is not in the catalog. */
+grace_status_t grace_trie_walk(const uint64_t* child_bits, const int32_t* child_base, int V, int L,
+                               int64_t num_internal, const int32_t* tokens, int len, int32_t* node);
+
+/* ------------------------------------------------------------------------------------------
+ * Cross-attention, beam-as-query layout (Section 5.1, Appendix B).
+ *   out[b*M+m, h, :] = softmax_t( q[b*M+m, h, :] . k[b, h, t, :] * scale ) @ v[b, h, :, :]
+ * K and V are read once per (request, head) and shared by the M beams of the request.
+ *   q, out : device bf16, element (r, h, i) at r*row_stride + h*d_h + i   (strides in elements)
+ *   k, v   : device bf16, element (b, h, t, i) at b*kv_stride_b + h*kv_stride_h + t*kv_stride_t + i
+ *   lse    : device fp32 [B*M][H] or NULL; natural-log sum-exp of the scaled scores
+ * fp32 accumulation and softmax; bf16 output.  Pointers 16-byte aligned, strides multiples of 8.
+ * Supported: d_h in {32, 64, 128}; any B, M, H, T_ctx >= 1.
+ * ---------------------------------------------------------------------------------------- */
+grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
+                                const uint16_t* k, const uint16_t* v,
+                                int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                                uint16_t* out, int64_t out_row_stride, float* lse,
+                                int B, int M, int H, int d_h, int T_ctx, float scale,
+                                int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Self-attention over the parent-addressed KV cache, fused with the cache write
+ * (Sections 5.2, 5.3; the block table P of Section 5.3 in its uncomposed form).
+ * Row r = b*M_t + m at step t:
+ *   k_cache[t][r] <- k of qkv[r],  v_cache[t][r] <- v of qkv[r]
+ *   a_t = m;  a_{j-1} = parents[j][b*M_j + a_j]          (j = t .. 1)
+ *   out[r, h] = softmax_j( q[r,h] . k_cache[j][b*M_j + a_j, h] * scale ) @ v_cache[j][...],  j = 0..t
+ * The current token is part of the prefix; no KV bytes are ever copied on beam reordering.
+ *   qkv     : device bf16 [R][3][H][d_h], row stride qkv_row_stride elements
+ *   k_cache, v_cache : device bf16 [L_cache][R_max][H][d_h]
+ *   parents : device int32 [L_cache][R_max]; slab j (j >= 1) holds, for each row of step j, the
+ *             index of its parent inside the same request's step-(j-1) beam; slab 0 is unused
+ *   beam_sizes : host int32 [t+1] = M_0 .. M_t
+ *   out     : device bf16 [R][H][d_h], row stride out_row_stride elements
+ * Supported: t <= 7, d_h in {32, 64, 128}, H*d_h a multiple of 8 and <= 2048.
+ * An out-of-range parent index sets GRACE_DEV_BAD_INDEX and is treated as 0.
+ * ---------------------------------------------------------------------------------------- */
+grace_status_t grace_self_attn(const uint16_t* qkv, int64_t qkv_row_stride,
+                               uint16_t* k_cache, uint16_t* v_cache,
+                               const int32_t* parents, const int32_t* beam_sizes,
+                               uint16_t* out, int64_t out_row_stride,
+                               int B, int t, int H, int d_h, int64_t R_max, float scale,
+                               int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * CD + GTM mask and score add (Sections 3.1, 4.1; kernel role of Section 5.4).
+ *   allow[r, v] = CD(node[r], v) AND TM(b, prefix[r] || v)
+ *   cand[r, v]  = beam_score[r] + logp[r, v] (one fp32 add) if allow else -inf
+ *   logp fp32 [R][V]; beam_score fp32 [R]; beam_node int32 [R] (-1 = dead beam: nothing allowed);
+ *   beam_key uint64 [R] (prefix keys, read only by the Bloom matcher); prefix_len = tokens
+ *   already decoded (= step index).  cand fp32 [R][V] (may be NULL), allow_bits uint64 [R][V/64]
+ *   (may be NULL).  All device.  R = B*M.
+ * ---------------------------------------------------------------------------------------- */
+grace_status_t grace_gtm_mask(const float* logp, const float* beam_score, const int32_t* beam_node,
+                              const uint64_t* beam_key, const grace_trie_t* trie,
+                              const grace_matcher_t* matcher, float* cand, uint64_t* allow_bits,
+                              int B, int M, int V, int prefix_len, int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Beam x codebook top-k (Sections 3.1, 3.3).  Per request b, the K best of cand[b][0..N)
+ * under the total order (value descending, flat index ascending); -0.0 == +0.0; -inf takes
+ * part like any value.  Outputs are in that order:
+ *   out_score fp32, out_flat int32, out_parent = flat / V, out_token = flat % V, each [B][K]
+ *   (out_flat / out_parent / out_token may be NULL).
+ * Needs a device workspace of grace_beam_topk_workspace_bytes(B, N, K) bytes, 256-byte aligned;
+ * its contents on entry do not matter.  1 <= K <= min(N, 4096); N < 2^31.
+ * ---------------------------------------------------------------------------------------- */
+size_t grace_beam_topk_workspace_bytes(int B, int64_t N, int K);
+grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, int K, int V,
+                               float* out_score, int32_t* out_flat, int32_t* out_parent,
+                               int32_t* out_token, void* ws, size_t ws_bytes,
+                               int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Beam-state update after top-k ("rearrangement", Sections 3.3, 4.4).  For new row i of request b:
+ *   src = b*M_prev + parent[b][i]
+ *   new_key[b*K+i]  = prev_key[src] | (token+1) << 16*prefix_len
+ *   new_node[b*K+i] = child(prev_node[src], token)   or -1 if score = -inf or prev_node[src] < 0
+ * Only these small arrays move; KV stays where it is.  All device; parent/token/score [B][K].
+ * ---------------------------------------------------------------------------------------- */
+grace_status_t grace_beam_update(const int32_t* parent, const int32_t* token, const float* score,
+                                 const int32_t* prev_node, const uint64_t* prev_key,
+                                 const grace_trie_t* trie, int32_t* new_node, uint64_t* new_key,
+                                 int B, int K, int M_prev, int prefix_len,
+                                 int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Decoder-layer building blocks used by grace_decode_step (Section 3.2; the paper leaves these
+ * GEMMs to a vendor library, Section 5.2 "Kernel fusion").  Exported so each can be checked.
+ * ---------------------------------------------------------------------------------------- */
+
+/* y = act(x @ w^T) (+ residual).  x bf16 [M][K] (row stride ldx), w bf16 [N][K] (row stride ldw),
+ * fp32 accumulation.  Exactly one of y_bf16 / y_f32 is non-NULL ([M][N], row stride ldy).
+ * residual: fp32 [M][N] (row stride ldy) or NULL, added before the store; may alias y_f32.
+ * relu != 0 applies max(., 0) before the residual.  K multiple of 64, N multiple of 16;
+ * pointers 16-byte aligned, strides multiples of 8 elements. */
+grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                            uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
+                            int M, int N, int K, int relu, void* stream);
+
+/* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
+grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
+                                uint16_t* out, int R, int D, float eps, void* stream);
+
+/* x fp32 [R][D] = embed[token[r]] + pos (embed bf16 [V+1][D], pos bf16 [D]); token int32 [R]. */
+grace_status_t grace_embed(const int32_t* token, const uint16_t* embed, const uint16_t* pos,
+                           float* x, int R, int D, int n_rows_embed, int32_t* d_status, void* stream);
+
+/* In place: logits fp32 [R][V] -> log-probabilities (natural log), normalised over all V. */
+grace_status_t grace_log_softmax(float* logits, int R, int V, void* stream);
+
+/* Per-layer weights; every matrix is bf16 [out_features][in_features], dense rows. */
+typedef struct {
+  const float *ln1_g, *ln1_b, *ln2_g, *ln2_b, *ln3_g, *ln3_b;
+  const uint16_t *w_qkv;   /* [3*H*d_h][d_model]  rows ordered (q|k|v, head, i) */
+  const uint16_t *w_o;     /* [d_model][H*d_h] */
+  const uint16_t *w_qc;    /* [H*d_h][d_model] */
+  const uint16_t *w_oc;    /* [d_model][H*d_h] */
+  const uint16_t *w_1;     /* [d_ffn][d_model] */
+  const uint16_t *w_2;     /* [d_model][d_ffn] */
+  const uint16_t *k_cross, *v_cross;   /* [B][H][T_ctx][d_h], projected once per request */
+  uint16_t *k_cache, *v_cache;         /* [L][R_max][H][d_h] */
+} grace_layer_t;
+
+#define GRACE_MAX_LAYERS 16
+#define GRACE_MAX_STEPS 8
+
+/* Everything one decode step reads and writes.  A plain struct of caller-owned device buffers
+ * (host struct, passed by pointer, read during the call only). */
+typedef struct {
+  int32_t B, n_layers, d_model, H, d_h, d_ffn, V, L, T_ctx;
+  int32_t beam_sizes[GRACE_MAX_STEPS + 1]; /* M_0 .. M_{L-1}, then the final K at index L  */
+  int64_t R_max;                           /* B * max beam size                             */
+  float ln_eps;
+  grace_layer_t layers[GRACE_MAX_LAYERS];
+  const uint16_t *embed;      /* [V+1][d_model], row V = start token */
+  const uint16_t *pos;        /* [L][d_model]                        */
+  const float *lnf_g, *lnf_b;
+  const uint16_t *w_out;      /* [V][d_model]                        */
+  grace_trie_t trie;
+  grace_matcher_t matcher;
+  /* beam state, double-buffered by step parity: index (t & 1) is read, ((t+1) & 1) written */
+  int32_t *token[2];          /* [R_max] input token of each row                          */
+  float *score[2];            /* [R_max]                                                  */
+  int32_t *node[2];           /* [R_max]                                                  */
+  uint64_t *key[2];           /* [R_max]                                                  */
+  int32_t *parents;           /* [L+1][R_max]; slab t+1 is written by step t               */
+  int32_t *out_flat;          /* [R_max] scratch for the selected flat indices             */
+  /* activations (scratch) */
+  float *x;                   /* [R_max][d_model] residual stream                         */
+  uint16_t *h;                /* [R_max][max(d_model, d_ffn)]                             */
+  uint16_t *qkv;              /* [R_max][max(3*H*d_h, d_ffn)]: qkv, cross-q, FFN hidden     */
+  uint16_t *attn;             /* [R_max][H*d_h]                                            */
+  float *logp;                /* [R_max][V]; also receives cand in place                  */
+  void *topk_ws; size_t topk_ws_bytes;
+  int32_t *d_status;
+} grace_decoder_t;
+
+/* Host-only consistency check of a decoder struct (null pointers, shape limits). */
+grace_status_t grace_decoder_validate(const grace_decoder_t* dec);
+
+/* Step t (0-based) of the decode loop (Sections 3.1-3.3): embed the rows' input tokens, run the
+ * decoder layers (self-attention with cache write, cross-attention, feed-forward), logits,
+ * log-softmax, CD+GTM mask with score add, top-k of beam_sizes[t+1] per request, state update.
+ * Reads state buffers [t & 1], writes [(t+1) & 1] and parents slab t+1. */
+grace_status_t grace_decode_step(const grace_decoder_t* dec, int t, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRACE_H_ */

@@ -1,0 +1,282 @@
+"""ctypes binding of the C ABI declared in include/grace.h.
+
+Functions take torch CUDA tensors (device memory and the current stream come
+from torch; nothing else does) or numpy arrays for the host-side index
+builders.  Names match the C entry points.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgrace_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2608_00938_b200.build` "
+        "(there is no fallback path)")
+
+lib = C.CDLL(LIB_PATH)
+
+GRACE_OK = 0
+DEV_BAD_INDEX, DEV_NAN, DEV_TIMEOUT, DEV_TOPK_EXACT_PATH = 1, 2, 4, 8
+MATCH_NONE, MATCH_NODE_BITMASK, MATCH_PREFIX_BLOOM = 0, 1, 2
+MAX_LAYERS, MAX_STEPS = 16, 8
+
+_vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_size_t
+
+
+class TrieStruct(C.Structure):
+    _fields_ = [("V", C.c_int32), ("L", C.c_int32), ("num_nodes", C.c_int64),
+                ("num_internal", C.c_int64), ("child_bits", _vp), ("child_base", _vp)]
+
+
+class MatcherStruct(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("bloom_log2_bits", C.c_int32), ("bloom_hashes", C.c_int32),
+                ("reserved", C.c_int32), ("words_per_request", C.c_int64), ("bits", _vp)]
+
+
+class LayerStruct(C.Structure):
+    _fields_ = [(n, _vp) for n in (
+        "ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b",
+        "w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2",
+        "k_cross", "v_cross", "k_cache", "v_cache")]
+
+
+class DecoderStruct(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("n_layers", C.c_int32), ("d_model", C.c_int32), ("H", C.c_int32),
+        ("d_h", C.c_int32), ("d_ffn", C.c_int32), ("V", C.c_int32), ("L", C.c_int32),
+        ("T_ctx", C.c_int32),
+        ("beam_sizes", C.c_int32 * (MAX_STEPS + 1)),
+        ("R_max", C.c_int64),
+        ("ln_eps", C.c_float),
+        ("layers", LayerStruct * MAX_LAYERS),
+        ("embed", _vp), ("pos", _vp), ("lnf_g", _vp), ("lnf_b", _vp), ("w_out", _vp),
+        ("trie", TrieStruct), ("matcher", MatcherStruct),
+        ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
+        ("parents", _vp), ("out_flat", _vp),
+        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp),
+        ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
+        ("d_status", _vp),
+    ]
+
+
+def _sig(name, restype, argtypes):
+    fn = getattr(lib, name)
+    fn.restype = restype
+    fn.argtypes = argtypes
+    return fn
+
+
+_status_string = _sig("grace_status_string", C.c_char_p, [_i32])
+_version = _sig("grace_version", _i32, [])
+_built_for_sm = _sig("grace_built_for_sm", _i32, [])
+_trie_count_nodes = _sig("grace_trie_count_nodes", _i32, [_vp, _i64, _i32, _i32, _vp])
+_trie_build_dense = _sig("grace_trie_build_dense", _i32, [_vp, _i64, _i32, _i32, _vp, _vp])
+_node_bitmask_build = _sig("grace_node_bitmask_build", _i32, [_vp, _i64, _i32, _i32, _vp, _vp])
+_bloom_build = _sig("grace_bloom_build", _i32, [_vp, _i64, _i32, _i32, _vp, _i32, _i32, _vp])
+_trie_walk = _sig("grace_trie_walk", _i32, [_vp, _vp, _i32, _i32, _i64, _vp, _i32, _vp])
+_cross_attn = _sig("grace_cross_attn", _i32, [_vp, _i64, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _vp,
+                                             _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp])
+_self_attn = _sig("grace_self_attn", _i32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64,
+                                           _i32, _i32, _i32, _i32, _i64, _f32, _vp, _vp])
+_gtm_mask = _sig("grace_gtm_mask", _i32, [_vp, _vp, _vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct),
+                                         _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
+_topk_ws = _sig("grace_beam_topk_workspace_bytes", _sz, [_i32, _i64, _i32])
+_beam_topk = _sig("grace_beam_topk", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp])
+_beam_update = _sig("grace_beam_update", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct), _vp, _vp,
+                                               _i32, _i32, _i32, _i32, _vp, _vp])
+_linear = _sig("grace_linear", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp])
+_layer_norm = _sig("grace_layer_norm", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _f32, _vp])
+_embed = _sig("grace_embed", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp])
+_log_softmax = _sig("grace_log_softmax", _i32, [_vp, _i32, _i32, _vp])
+_decoder_validate = _sig("grace_decoder_validate", _i32, [C.POINTER(DecoderStruct)])
+_decode_step = _sig("grace_decode_step", _i32, [C.POINTER(DecoderStruct), _i32, _vp])
+
+
+class GraceError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_status_string(code).decode()} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != GRACE_OK:
+        raise GraceError(code, where)
+
+
+def _dp(t):
+    """Device pointer of a torch tensor (None -> NULL)."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "expected a contiguous CUDA tensor"
+    return t.data_ptr()
+
+
+def _hp(a, dtype):
+    assert isinstance(a, np.ndarray) and a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def version() -> int:
+    return _version()
+
+
+def built_for_sm() -> int:
+    return _built_for_sm()
+
+
+# ----------------------------------------------------------------------------
+# host-side index builders (numpy in, numpy out)
+# ----------------------------------------------------------------------------
+def grace_trie_count_nodes(sids: np.ndarray, V: int) -> np.ndarray:
+    n, L = sids.shape
+    level_start = np.zeros(L + 2, dtype=np.int64)
+    _check(_trie_count_nodes(_hp(sids, np.int32), n, V, L, level_start.ctypes.data), "grace_trie_count_nodes")
+    return level_start
+
+
+def grace_trie_build_dense(sids: np.ndarray, V: int):
+    """-> (child_bits uint64 [n_internal, V/64], child_base int32 [n_internal], level_start)."""
+    n, L = sids.shape
+    level_start = grace_trie_count_nodes(sids, V)
+    n_int = int(level_start[L])
+    bits = np.empty((n_int, V // 64), dtype=np.uint64)
+    base = np.empty(n_int, dtype=np.int32)
+    _check(_trie_build_dense(_hp(sids, np.int32), n, V, L, bits.ctypes.data, base.ctypes.data),
+           "grace_trie_build_dense")
+    return bits, base, level_start
+
+
+def grace_node_bitmask_build(sids: np.ndarray, V: int, eligible: np.ndarray, num_nodes: int) -> np.ndarray:
+    n, L = sids.shape
+    out = np.empty((num_nodes + 63) // 64, dtype=np.uint64)
+    el = np.ascontiguousarray(eligible, dtype=np.uint8)
+    _check(_node_bitmask_build(_hp(sids, np.int32), n, V, L, el.ctypes.data, out.ctypes.data),
+           "grace_node_bitmask_build")
+    return out
+
+
+def grace_bloom_build(sids: np.ndarray, V: int, eligible: np.ndarray, log2_bits: int, n_hashes: int) -> np.ndarray:
+    n, L = sids.shape
+    out = np.empty((1 << log2_bits) // 64, dtype=np.uint64)
+    el = np.ascontiguousarray(eligible, dtype=np.uint8)
+    _check(_bloom_build(_hp(sids, np.int32), n, V, L, el.ctypes.data, log2_bits, n_hashes, out.ctypes.data),
+           "grace_bloom_build")
+    return out
+
+
+def grace_trie_walk(child_bits: np.ndarray, child_base: np.ndarray, V: int, L: int, tokens) -> int:
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    node = C.c_int32(-2)
+    _check(_trie_walk(_hp(child_bits, np.uint64), _hp(child_base, np.int32), V, L, child_bits.shape[0],
+                      tok.ctypes.data, tok.shape[0], C.addressof(node)), "grace_trie_walk")
+    return node.value
+
+
+def make_trie(child_bits_dev, child_base_dev, V: int, L: int, num_nodes: int) -> TrieStruct:
+    return TrieStruct(V, L, num_nodes, child_bits_dev.shape[0], _dp(child_bits_dev), _dp(child_base_dev))
+
+
+def make_matcher(kind: int, bits_dev=None, log2_bits: int = 0, n_hashes: int = 0) -> MatcherStruct:
+    words = 0 if bits_dev is None else bits_dev.shape[-1]
+    return MatcherStruct(kind, log2_bits, n_hashes, 0, words, _dp(bits_dev))
+
+
+# ----------------------------------------------------------------------------
+# device ops (torch CUDA tensors; bf16 tensors are torch.bfloat16)
+# ----------------------------------------------------------------------------
+def grace_cross_attn(q, k, v, out, scale: float, lse=None, d_status=None):
+    """q/out [B*M, H, d] (or [B, M, H, d]) bf16; k/v [B, H, T, d] bf16 (any strides with unit last)."""
+    B, H, T, d = k.shape
+    q2 = q.reshape(-1, H, d)
+    o2 = out.reshape(-1, H, d)
+    M = q2.shape[0] // B
+    assert k.stride() == v.stride() and k.stride(3) == 1
+    _check(_cross_attn(q2.data_ptr(), q2.stride(0), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1),
+                       k.stride(2), o2.data_ptr(), o2.stride(0), _dp(lse), B, M, H, d, T, scale,
+                       _dp(d_status), _stream()), "grace_cross_attn")
+    return out
+
+
+def grace_self_attn(qkv, k_cache, v_cache, parents, beam_sizes, out, B: int, t: int, scale: float,
+                    d_status=None):
+    """qkv [R, 3, H, d]; caches [L, R_max, H, d]; parents int32 [L, R_max]; out [R, H, d]."""
+    R, three, H, d = qkv.shape
+    bs = np.ascontiguousarray(beam_sizes[: t + 1], dtype=np.int32)
+    _check(_self_attn(_dp(qkv), qkv.stride(0), _dp(k_cache), _dp(v_cache), _dp(parents), bs.ctypes.data,
+                      _dp(out), out.stride(0), B, t, H, d, k_cache.shape[1], scale, _dp(d_status), _stream()),
+           "grace_self_attn")
+    return out
+
+
+def grace_gtm_mask(logp, beam_score, beam_node, beam_key, trie: TrieStruct, matcher: MatcherStruct,
+                   cand, allow_bits, B: int, M: int, prefix_len: int, d_status=None):
+    V = logp.shape[-1]
+    _check(_gtm_mask(_dp(logp), _dp(beam_score), _dp(beam_node), _dp(beam_key), C.byref(trie), C.byref(matcher),
+                     _dp(cand), _dp(allow_bits), B, M, V, prefix_len, _dp(d_status), _stream()), "grace_gtm_mask")
+
+
+def grace_beam_topk_workspace_bytes(B: int, N: int, K: int) -> int:
+    return _topk_ws(B, N, K)
+
+
+def grace_beam_topk(cand, K: int, V: int, out_score, out_flat, out_parent, out_token, ws, d_status=None):
+    """cand fp32 [B, N]; outputs [B, K]; ws: uint8 CUDA tensor of workspace_bytes."""
+    B, N = cand.shape
+    _check(_beam_topk(_dp(cand), B, N, K, V, _dp(out_score), _dp(out_flat), _dp(out_parent), _dp(out_token),
+                      _dp(ws), ws.numel() * ws.element_size(), _dp(d_status), _stream()), "grace_beam_topk")
+
+
+def grace_beam_update(parent, token, score, prev_node, prev_key, trie: TrieStruct, new_node, new_key,
+                      B: int, K: int, M_prev: int, prefix_len: int, d_status=None):
+    _check(_beam_update(_dp(parent), _dp(token), _dp(score), _dp(prev_node), _dp(prev_key), C.byref(trie),
+                        _dp(new_node), _dp(new_key), B, K, M_prev, prefix_len, _dp(d_status), _stream()),
+           "grace_beam_update")
+
+
+def grace_linear(x, w, y, residual=None, relu: bool = False):
+    """y = act(x @ w.T) (+ residual); x [M, K] bf16, w [N, K] bf16, y [M, N] bf16 or fp32."""
+    import torch
+    M, K = x.shape
+    N = w.shape[0]
+    yb, yf = (_dp(y), None) if y.dtype == torch.bfloat16 else (None, _dp(y))
+    _check(_linear(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), yb, yf, y.stride(0),
+                   _dp(residual), M, N, K, int(relu), _stream()), "grace_linear")
+    return y
+
+
+def grace_layer_norm(x, gamma, beta, out, eps: float = 1e-5):
+    R, D = x.shape
+    _check(_layer_norm(_dp(x), _dp(gamma), _dp(beta), _dp(out), R, D, eps, _stream()), "grace_layer_norm")
+    return out
+
+
+def grace_embed(token, embed, pos, x, d_status=None):
+    R, D = x.shape
+    _check(_embed(_dp(token), _dp(embed), _dp(pos), _dp(x), R, D, embed.shape[0], _dp(d_status), _stream()),
+           "grace_embed")
+    return x
+
+
+def grace_log_softmax(logits):
+    R, V = logits.shape
+    _check(_log_softmax(_dp(logits), R, V, _stream()), "grace_log_softmax")
+    return logits
+
+
+def grace_decoder_validate(dec: DecoderStruct) -> int:
+    return _decoder_validate(C.byref(dec))
+
+
+def grace_decode_step(dec: DecoderStruct, t: int):
+    _check(_decode_step(C.byref(dec), t, _stream()), "grace_decode_step")

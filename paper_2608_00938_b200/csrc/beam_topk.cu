@@ -1,0 +1,425 @@
+// Beam x codebook top-k (Sections 3.1, 3.3): per request, the K best of N = M * |V| candidates
+// under the total order (value descending, flat index ascending), returned in that order.
+//
+// The candidates are read from HBM once.  Four launches:
+//   1. sample   : per request, 4096 sample points x 8 consecutive floats (one 32-byte sector per
+//                 point, one point per N/4096-element stratum).  The r-th largest sample, with r
+//                 a few standard deviations above K * (samples / N), becomes a threshold that
+//                 with high probability has between K and `kCap` candidates above it.
+//   2. collect  : the one full pass.  Every candidate above the threshold is appended to the
+//                 request's list (warp-aggregated atomics; hits are a fraction of a percent).
+//   3. exact    : requests whose list came out short or overflowed (and every request when N is
+//                 small) are redone by one CTA with a three-level radix select that resolves
+//                 ties by index.  Exits at once for requests that do not need it.
+//   4. finalize : bitonic sort of the list on (key, index), write the first K; if the threshold
+//                 was -inf and fewer than K finite candidates exist, the remaining slots are the
+//                 lowest-index -inf candidates.
+// The result is exact whatever the threshold; the threshold only decides which path runs.
+#include "common.cuh"
+
+namespace grace {
+
+constexpr int kCap = 8192;               // list capacity per request (entries)
+constexpr int kHeaderWords = 16;         // per-request header, 64 bytes
+constexpr int kSamplePoints = 4096;
+constexpr int kSampleSize = kSamplePoints * 8;
+constexpr int kTopkThreads = 1024;
+
+struct TopkHeader {                      // lives in the workspace, one per request
+  uint32_t count;                        // entries appended (may exceed kCap: overflow)
+  uint32_t t_excl;                       // collect keys strictly above this
+  uint32_t need_exact;
+  uint32_t pad[kHeaderWords - 3];
+};
+
+__host__ __device__ inline size_t topk_header_bytes(int B) { return (size_t)B * sizeof(TopkHeader); }
+
+// ---- block primitives (kTopkThreads threads) -------------------------------------------
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    uint32_t o = __shfl_up_sync(kFullMask, v, d);
+    if (lane >= d) v += o;
+  }
+  return v;
+}
+
+// Exclusive prefix sum over the block; *total receives the block sum.  scratch: 33 words.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratch, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t incl = warp_incl_scan(v);
+  __syncthreads();                                   // scratch may still be read from a previous call
+  if (lane == 31) scratch[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = (lane < (int)(blockDim.x >> 5)) ? scratch[lane] : 0u;
+    uint32_t wi = warp_incl_scan(w);
+    scratch[lane] = wi - w;
+    if (lane == 31) scratch[32] = wi;
+  }
+  __syncthreads();
+  *total = scratch[32];
+  return scratch[warp] + incl - v;
+}
+
+// One radix level.  hist[nbins] holds counts of digit values among the still-matching keys.
+// Finds the digit d with (#keys with larger digit) < k <= (#keys with digit >= d); returns d and
+// reduces *k by the number of keys with a larger digit.  nbins <= 4 * blockDim.x.
+__device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, int nbins, uint32_t* k,
+                                               uint32_t* scratch, uint32_t* result) {
+  // thread t owns bins [4t, 4t+4) counted from the top: bin index nbins-1-4t-j
+  uint32_t c[4];
+  uint32_t mine = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int bin = nbins - 1 - (4 * (int)threadIdx.x + j);
+    c[j] = (bin >= 0) ? hist[bin] : 0u;
+    mine += c[j];
+  }
+  uint32_t total;
+  uint32_t above = block_excl_scan(mine, scratch, &total);   // keys in bins above this thread's
+  const uint32_t want = *k;
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int bin = nbins - 1 - (4 * (int)threadIdx.x + j);
+    if (bin >= 0 && above < want && want <= above + c[j]) {
+      result[0] = (uint32_t)bin;
+      result[1] = want - above;
+    }
+    above += c[j];
+  }
+  __syncthreads();
+  *k = result[1];
+  return result[0];
+}
+
+// ---- 1. sample -------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kTopkThreads)
+topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, TopkHeader* hdr) {
+  extern __shared__ uint32_t smem_u32[];
+  uint32_t* keys = smem_u32;                     // kSampleSize
+  uint32_t* hist = keys + kSampleSize;           // 4096
+  uint32_t* scratch = hist + 4096;               // 40
+  uint32_t* result = scratch + 40;               // 2
+  const int b = blockIdx.x;
+  const float* row = cand + (int64_t)b * N;
+  const int64_t stratum = (N / kSamplePoints) & ~(int64_t)7;       // multiple of 8 elements
+  const uint32_t slots = (uint32_t)(stratum >> 3);
+  for (int p = threadIdx.x; p < kSamplePoints; p += kTopkThreads) {
+    const uint32_t h = (uint32_t)(mix64((uint64_t)p * 0x10001ull + (uint64_t)b) >> 33);
+    const int64_t at = (int64_t)p * stratum + (int64_t)(h % slots) * 8;
+    const float4 a = __ldg(reinterpret_cast<const float4*>(row + at));
+    const float4 c = __ldg(reinterpret_cast<const float4*>(row + at + 4));
+    uint32_t* dst = keys + p * 8;
+    dst[0] = ordered_key(a.x); dst[1] = ordered_key(a.y); dst[2] = ordered_key(a.z); dst[3] = ordered_key(a.w);
+    dst[4] = ordered_key(c.x); dst[5] = ordered_key(c.y); dst[6] = ordered_key(c.z); dst[7] = ordered_key(c.w);
+  }
+  uint32_t k = rank, prefix = 0;
+  // three radix levels over the sample held in shared memory: 12 + 12 + 8 bits
+  const int shifts[3] = {20, 8, 0};
+  const int bits[3] = {12, 12, 8};
+#pragma unroll 1
+  for (int level = 0; level < 3; ++level) {
+    const int nb = 1 << bits[level];
+    for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
+    __syncthreads();
+    const int hi_shift = shifts[level] + bits[level];
+    for (int i = threadIdx.x; i < kSampleSize; i += kTopkThreads) {
+      const uint32_t u = keys[i];
+      const bool match = (level == 0) || ((u >> hi_shift) == prefix);
+      if (match) atomicAdd(&hist[(u >> shifts[level]) & (nb - 1)], 1u);
+    }
+    __syncthreads();
+    const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
+    prefix = (prefix << bits[level]) | d;
+  }
+  if (threadIdx.x == 0) {
+    hdr[b].count = 0;
+    hdr[b].need_exact = 0;
+    hdr[b].t_excl = (prefix <= kKeyNegInf) ? kKeyNegInf : prefix - 1;
+  }
+}
+
+__global__ void topk_reset_kernel(TopkHeader* hdr, int B) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) { hdr[b].count = 0; hdr[b].t_excl = 0; hdr[b].need_exact = 1; }
+}
+
+// ---- 2. collect ------------------------------------------------------------------------------
+constexpr int kCollectThreads = 256;
+constexpr int kCollectUnroll = 8;                         // float4 loads in flight per thread
+
+__global__ void __launch_bounds__(kCollectThreads)
+topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, uint2* lists,
+                    int32_t* d_status) {
+  const int b = blockIdx.y;
+  const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
+  const int64_t n4 = N >> 2;
+  const uint32_t t_excl = hdr[b].t_excl;
+  uint2* list = lists + (int64_t)b * kCap;
+  const int lane = threadIdx.x & 31;
+  const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
+  bool saw_nan = false;
+  for (int64_t base = (int64_t)blockIdx.x * tile; base < n4; base += (int64_t)gridDim.x * tile) {
+    float4 v[kCollectUnroll];
+#pragma unroll
+    for (int u = 0; u < kCollectUnroll; ++u) {
+      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
+      v[u] = (i < n4) ? __ldcs(row + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int u = 0; u < kCollectUnroll; ++u) {
+      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
+      const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+      uint32_t key[4];
+      uint32_t hits = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        key[j] = ordered_key(x[j]);
+        if (x[j] != x[j]) saw_nan = true;
+        hits += (key[j] > t_excl) ? 1u : 0u;
+      }
+      if (__any_sync(kFullMask, hits != 0)) {
+        const uint32_t incl = warp_incl_scan(hits);
+        const uint32_t total = __shfl_sync(kFullMask, incl, 31);
+        uint32_t start = 0;
+        if (lane == 31) start = atomicAdd(&hdr[b].count, total);
+        start = __shfl_sync(kFullMask, start, 31) + incl - hits;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (key[j] > t_excl) {
+            if (start < (uint32_t)kCap) list[start] = make_uint2(key[j], (uint32_t)(i * 4 + j));
+            ++start;
+          }
+        }
+      }
+    }
+  }
+  if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
+}
+
+// ---- 3. exact --------------------------------------------------------------------------------
+// One CTA per request.  Three histogram passes over the row fix the K-th key exactly; a fourth
+// pass in index order writes the keys above it and the first ties.
+__global__ void __launch_bounds__(kTopkThreads)
+topk_exact_kernel(const float* __restrict__ cand, int64_t N, int K, TopkHeader* hdr, uint2* lists,
+                  int force, int32_t* d_status) {
+  __shared__ uint32_t hist[4096];
+  __shared__ uint32_t scratch[40];
+  __shared__ uint32_t result[2];
+  const int b = blockIdx.x;
+  if (!force) {
+    const uint32_t c = hdr[b].count;
+    const bool short_list = c < (uint32_t)K && hdr[b].t_excl != kKeyNegInf;
+    if (!(c > (uint32_t)kCap || short_list)) return;
+    if (threadIdx.x == 0) flag_status(d_status, GRACE_DEV_TOPK_EXACT_PATH);
+  }
+  const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
+  const int64_t n4 = N >> 2;
+  uint32_t k = (uint32_t)K, prefix = 0;
+  const int shifts[3] = {20, 8, 0};
+  const int bits[3] = {12, 12, 8};
+  bool saw_nan = false;
+#pragma unroll 1
+  for (int level = 0; level < 3; ++level) {
+    const int nb = 1 << bits[level];
+    for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
+    __syncthreads();
+    const int hi_shift = shifts[level] + bits[level];
+    uint32_t n_ninf = 0;            // -inf dominates masked rows: count it in a register
+    for (int64_t i = threadIdx.x; i < n4; i += kTopkThreads) {
+      const float4 v = __ldg(row + i);
+      const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (level == 0 && x[j] != x[j]) saw_nan = true;
+        const uint32_t u = ordered_key(x[j]);
+        if (u == kKeyNegInf) { ++n_ninf; continue; }
+        const bool match = (level == 0) || ((u >> hi_shift) == prefix);
+        if (match) atomicAdd(&hist[(u >> shifts[level]) & (nb - 1)], 1u);
+      }
+    }
+    if (n_ninf != 0 && ((level == 0) || ((kKeyNegInf >> hi_shift) == prefix)))
+      atomicAdd(&hist[(kKeyNegInf >> shifts[level]) & (nb - 1)], n_ninf);
+    __syncthreads();
+    const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
+    prefix = (prefix << bits[level]) | d;
+  }
+  if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
+  // prefix = exact K-th key; k = number of ties (key == prefix) to take, lowest indices first
+  const uint32_t kth = prefix, n_ties = k, n_above = (uint32_t)K - k;
+  uint2* list = lists + (int64_t)b * kCap;
+  uint32_t done_above = 0, done_ties = 0;
+  for (int64_t base = 0; base < n4; base += kTopkThreads) {
+    const int64_t i = base + threadIdx.x;
+    float4 v = make_float4(0, 0, 0, 0);
+    uint32_t key[4] = {0, 0, 0, 0};
+    uint32_t above = 0, ties = 0;
+    if (i < n4) {
+      v = __ldg(row + i);
+      key[0] = ordered_key(v.x); key[1] = ordered_key(v.y); key[2] = ordered_key(v.z); key[3] = ordered_key(v.w);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { above += key[j] > kth; ties += key[j] == kth; }
+    }
+    uint32_t tot_above, tot_ties;
+    uint32_t pa = block_excl_scan(above, scratch, &tot_above) + done_above;
+    uint32_t pt = block_excl_scan(ties, scratch, &tot_ties) + done_ties;
+    if (i < n4) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (key[j] > kth) {
+          if (pa < n_above) list[pa] = make_uint2(key[j], (uint32_t)(i * 4 + j));
+          ++pa;
+        } else if (key[j] == kth) {
+          if (pt < n_ties) list[n_above + pt] = make_uint2(key[j], (uint32_t)(i * 4 + j));
+          ++pt;
+        }
+      }
+    }
+    done_above += tot_above;
+    done_ties += tot_ties;
+    if (done_ties >= n_ties && done_above >= n_above) break;   // uniform across the block
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) { hdr[b].count = (uint32_t)K; hdr[b].need_exact = 0; }
+}
+
+// ---- 4. finalize -----------------------------------------------------------------------------
+__global__ void __launch_bounds__(kTopkThreads)
+topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, const TopkHeader* hdr,
+                     const uint2* lists, float* out_score, int32_t* out_flat, int32_t* out_parent,
+                     int32_t* out_token) {
+  extern __shared__ unsigned long long sort_keys[];         // up to kCap entries
+  __shared__ uint32_t scratch[40];
+  const int b = blockIdx.x;
+  const uint32_t c = min(hdr[b].count, (uint32_t)kCap);
+  uint32_t n_sort = 1;
+  while (n_sort < c) n_sort <<= 1;
+  if (n_sort < 2) n_sort = 2;
+  const uint2* list = lists + (int64_t)b * kCap;
+  for (uint32_t i = threadIdx.x; i < n_sort; i += kTopkThreads) {
+    unsigned long long comp = 0ull;
+    if (i < c) {
+      const uint2 e = list[i];
+      comp = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
+    }
+    sort_keys[i] = comp;
+  }
+  __syncthreads();
+  // bitonic sort, descending
+  for (uint32_t size = 2; size <= n_sort; size <<= 1) {
+    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+      for (uint32_t t = threadIdx.x; t < (n_sort >> 1); t += kTopkThreads) {
+        const uint32_t lo = 2 * t - (t & (stride - 1));
+        const uint32_t hi = lo + stride;
+        const bool desc = ((lo & size) == 0);
+        const unsigned long long a = sort_keys[lo], d = sort_keys[hi];
+        if ((a < d) == desc) { sort_keys[lo] = d; sort_keys[hi] = a; }
+      }
+      __syncthreads();
+    }
+  }
+  const float* row = cand + (int64_t)b * N;
+  const uint32_t n_out = min(c, (uint32_t)K);
+  for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
+    const uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
+    const int64_t o = (int64_t)b * K + i;
+    out_score[o] = row[idx];
+    if (out_flat) out_flat[o] = (int32_t)idx;
+    if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
+    if (out_token) out_token[o] = (int32_t)(idx % (uint32_t)V);
+  }
+  if (c < (uint32_t)K) {
+    // Threshold was -inf and the row has fewer than K candidates above it: the rest of the beam
+    // is the lowest-index candidates at -inf.  At most c of the first K positions are finite, so
+    // scanning K positions is enough.
+    const uint32_t need = (uint32_t)K - c;
+    uint32_t done = 0;
+    for (uint32_t base = 0; base < (uint32_t)K && done < need; base += kTopkThreads) {
+      const uint32_t i = base + threadIdx.x;
+      const bool is_low = (i < (uint32_t)K) && (ordered_key(row[i]) <= kKeyNegInf);
+      uint32_t total;
+      const uint32_t rank = block_excl_scan(is_low ? 1u : 0u, scratch, &total) + done;
+      if (is_low && rank < need) {
+        const int64_t o = (int64_t)b * K + c + rank;
+        out_score[o] = row[i];
+        if (out_flat) out_flat[o] = (int32_t)i;
+        if (out_parent) out_parent[o] = (int32_t)(i / (uint32_t)V);
+        if (out_token) out_token[o] = (int32_t)(i % (uint32_t)V);
+      }
+      done += total;
+    }
+  }
+}
+
+// Sampling plan: rank r of the sample whose value is the threshold, or 0 if sampling is not
+// worthwhile / not safe for this shape (then the exact path handles every request).
+static uint32_t sample_rank(int64_t N, int K) {
+  if (N < (int64_t)kSampleSize * 8 || (N & 7)) return 0;
+  const double frac = (double)kSampleSize / (double)N;
+  const double expect = K * frac;
+  const double r = ceil(expect + 4.0 * sqrt(expect) + 8.0);
+  if (r / frac > 0.75 * kCap || r > kSampleSize / 4) return 0;
+  return (uint32_t)r;
+}
+
+}  // namespace grace
+
+extern "C" size_t grace_beam_topk_workspace_bytes(int B, int64_t N, int K) {
+  (void)N; (void)K;
+  if (B <= 0) return 0;
+  return grace::topk_header_bytes(B) + (size_t)B * grace::kCap * sizeof(uint2);
+}
+
+namespace grace {
+// Shared by the public entry point and the variant that owns its scratch.
+grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int V, float* out_score,
+                                int32_t* out_flat, int32_t* out_parent, int32_t* out_token,
+                                void* ws, int32_t* d_status, cudaStream_t s) {
+  TopkHeader* hdr = reinterpret_cast<TopkHeader*>(ws);
+  uint2* lists = reinterpret_cast<uint2*>(reinterpret_cast<char*>(ws) + topk_header_bytes(B));
+  const uint32_t rank = sample_rank(N, K);
+  static bool attrs_set = false;
+  const size_t sample_smem = (size_t)(kSampleSize + 4096 + 40 + 2) * sizeof(uint32_t);
+  const size_t final_smem = (size_t)kCap * sizeof(unsigned long long);
+  if (!attrs_set) {
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sample_smem));
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)final_smem));
+    attrs_set = true;
+  }
+  if (rank != 0) {
+    topk_sample_kernel<<<B, kTopkThreads, sample_smem, s>>>(cand, N, rank, hdr);
+    GRACE_LAUNCH_CHECK();
+    const int64_t n4 = N >> 2;
+    const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
+    int chunks = (int)((n4 + tile - 1) / tile);
+    dim3 grid((unsigned)chunks, (unsigned)B);
+    topk_collect_kernel<<<grid, kCollectThreads, 0, s>>>(cand, N, hdr, lists, d_status);
+    GRACE_LAUNCH_CHECK();
+    topk_exact_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, K, hdr, lists, 0, d_status);
+    GRACE_LAUNCH_CHECK();
+  } else {
+    topk_exact_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, K, hdr, lists, 1, d_status);
+    GRACE_LAUNCH_CHECK();
+  }
+  topk_finalize_kernel<<<B, kTopkThreads, final_smem, s>>>(cand, N, K, V, hdr, lists, out_score, out_flat,
+                                                          out_parent, out_token);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+}  // namespace grace
+
+extern "C" grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, int K, int V,
+                                          float* out_score, int32_t* out_flat, int32_t* out_parent,
+                                          int32_t* out_token, void* ws, size_t ws_bytes,
+                                          int32_t* d_status, void* stream) {
+  if (!cand || !out_score || !ws) return GRACE_INVALID_ARG;
+  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || K > N || V <= 0) return GRACE_INVALID_ARG;
+  if (K > 4096 || (N & 3)) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(cand) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return GRACE_INVALID_ARG;
+  if (ws_bytes < grace_beam_topk_workspace_bytes(B, N, K)) return GRACE_WORKSPACE_TOO_SMALL;
+  return grace::launch_beam_topk(cand, B, N, K, V, out_score, out_flat, out_parent, out_token, ws,
+                                 d_status, (cudaStream_t)stream);
+}

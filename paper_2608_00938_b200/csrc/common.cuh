@@ -1,0 +1,56 @@
+// Shared host/device helpers for the decode-step kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <math.h>
+
+#include "../../include/grace.h"
+
+#define GRACE_CUDA_TRY(expr)                                  \
+  do {                                                        \
+    cudaError_t _e = (expr);                                  \
+    if (_e != cudaSuccess) return GRACE_CUDA_ERROR;           \
+  } while (0)
+
+#define GRACE_LAUNCH_CHECK()                                  \
+  do {                                                        \
+    if (cudaGetLastError() != cudaSuccess) return GRACE_CUDA_ERROR; \
+  } while (0)
+
+static inline bool grace_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+namespace grace {
+
+constexpr uint32_t kFullMask = 0xffffffffu;
+constexpr uint32_t kKeyNegInf = 0x007fffffu;   // ordered key of -inf
+
+// Monotone map fp32 -> uint32: larger value <=> larger key.  -0.0 maps with +0.0.
+__device__ __forceinline__ uint32_t ordered_key(float x) {
+  uint32_t b = __float_as_uint(x);
+  if (b == 0x80000000u) b = 0u;
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ void flag_status(int32_t* d_status, int bits) {
+  if (d_status != nullptr) atomicOr(d_status, bits);
+}
+
+// splitmix64 finaliser used by the prefix Bloom filter.
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t key) {
+  uint64_t z = key + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+}  // namespace grace

@@ -1,0 +1,141 @@
+// Cross-attention in the beam-as-query layout (Section 5.1, Appendix B): the M beams of a request
+// are M query rows against that request's one copy of K and V.
+//
+// Two kernels behind one entry point:
+//   * cross_attn_tc_kernel (cross_attn_tc.cuh): tcgen05 / TMEM / TMA flash attention for
+//     d_h = 64, the serving shapes.
+//   * cross_attn_small_kernel (below): a plain CUDA-core kernel for everything else (tiny
+//     configurations, d_h = 32 or 128, unaligned strides).  One warp per (row, head); lanes split
+//     the encoder positions for the scores and the head dimension for the weighted sum.
+#include "common.cuh"
+#include "cross_attn_tc.cuh"
+
+namespace grace {
+
+struct CrossSmallParams {
+  const uint16_t* q; const uint16_t* k; const uint16_t* v; uint16_t* out; float* lse;
+  int64_t q_row_stride, out_row_stride, kv_stride_b, kv_stride_h, kv_stride_t;
+  int R, M, H, T; float scale;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(128)
+cross_attn_small_kernel(const CrossSmallParams p) {
+  constexpr int kChunk = 128;                 // encoder positions per round
+  constexpr int kPerLane = DH / 32;           // output elements per lane
+  __shared__ float probs[4][kChunk];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t item = (int64_t)blockIdx.x * 4 + warp;      // (row, head)
+  if (item >= (int64_t)p.R * p.H) return;
+  const int r = (int)(item / p.H), h = (int)(item % p.H);
+  const int b = r / p.M;
+  const uint16_t* qp = p.q + (int64_t)r * p.q_row_stride + h * DH;
+  const uint16_t* kb = p.k + (int64_t)b * p.kv_stride_b + (int64_t)h * p.kv_stride_h;
+  const uint16_t* vb = p.v + (int64_t)b * p.kv_stride_b + (int64_t)h * p.kv_stride_h;
+  uint32_t qreg[DH / 2];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) {
+    const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(qp) + i);
+    qreg[4 * i] = t4.x; qreg[4 * i + 1] = t4.y; qreg[4 * i + 2] = t4.z; qreg[4 * i + 3] = t4.w;
+  }
+  float m_run = -INFINITY, l_run = 0.f;
+  float acc[kPerLane];
+#pragma unroll
+  for (int j = 0; j < kPerLane; ++j) acc[j] = 0.f;
+  for (int t0 = 0; t0 < p.T; t0 += kChunk) {
+    float s[kChunk / 32];
+    float cmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kChunk / 32; ++i) {
+      const int t = t0 + i * 32 + lane;
+      s[i] = -INFINITY;
+      if (t < p.T) {
+        const uint4* kr = reinterpret_cast<const uint4*>(kb + (int64_t)t * p.kv_stride_t);
+        float d = 0.f;
+#pragma unroll
+        for (int c = 0; c < DH / 8; ++c) {
+          const uint4 kk = __ldg(kr + c);
+          d = fmaf(bf16_lo(qreg[4 * c]), bf16_lo(kk.x), d);     d = fmaf(bf16_hi(qreg[4 * c]), bf16_hi(kk.x), d);
+          d = fmaf(bf16_lo(qreg[4 * c + 1]), bf16_lo(kk.y), d); d = fmaf(bf16_hi(qreg[4 * c + 1]), bf16_hi(kk.y), d);
+          d = fmaf(bf16_lo(qreg[4 * c + 2]), bf16_lo(kk.z), d); d = fmaf(bf16_hi(qreg[4 * c + 2]), bf16_hi(kk.z), d);
+          d = fmaf(bf16_lo(qreg[4 * c + 3]), bf16_lo(kk.w), d); d = fmaf(bf16_hi(qreg[4 * c + 3]), bf16_hi(kk.w), d);
+        }
+        s[i] = d * p.scale;
+      }
+      cmax = fmaxf(cmax, s[i]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cmax = fmaxf(cmax, __shfl_xor_sync(kFullMask, cmax, o));
+    const float m_new = fmaxf(m_run, cmax);
+    const float corr = __expf(m_run - m_new);            // 0 on the first round (m_run = -inf)
+    float csum = 0.f;
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < kChunk / 32; ++i) {
+      const float e = (t0 + i * 32 + lane < p.T) ? __expf(s[i] - m_new) : 0.f;
+      probs[warp][i * 32 + lane] = e;
+      csum += e;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(kFullMask, csum, o);
+    l_run = l_run * corr + csum;
+    m_run = m_new;
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) acc[j] *= corr;
+    const int tn = min(kChunk, p.T - t0);
+    for (int tt = 0; tt < tn; ++tt) {
+      const float w = probs[warp][tt];
+      const uint16_t* vr = vb + (int64_t)(t0 + tt) * p.kv_stride_t;
+#pragma unroll
+      for (int j = 0; j < kPerLane; ++j)
+        acc[j] = fmaf(w, __uint_as_float((uint32_t)__ldg(vr + j * 32 + lane) << 16), acc[j]);
+    }
+  }
+  const float inv = 1.f / l_run;
+  uint16_t* op = p.out + (int64_t)r * p.out_row_stride + h * DH;
+#pragma unroll
+  for (int j = 0; j < kPerLane; ++j) {
+    __nv_bfloat16 o = __float2bfloat16_rn(acc[j] * inv);
+    op[j * 32 + lane] = *reinterpret_cast<uint16_t*>(&o);
+  }
+  if (p.lse != nullptr && lane == 0) p.lse[(int64_t)r * p.H + h] = m_run + logf(l_run);
+}
+
+}  // namespace grace
+
+extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
+                                           const uint16_t* k, const uint16_t* v,
+                                           int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                                           uint16_t* out, int64_t out_row_stride, float* lse,
+                                           int B, int M, int H, int d_h, int T_ctx, float scale,
+                                           int32_t* d_status, void* stream) {
+  using namespace grace;
+  (void)d_status;
+  if (!q || !k || !v || !out) return GRACE_INVALID_ARG;
+  if (B <= 0 || M <= 0 || H <= 0 || T_ctx <= 0 || (int64_t)B * M > 0x7fffffff) return GRACE_INVALID_ARG;
+  if (d_h != 32 && d_h != 64 && d_h != 128) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(q) || !grace_aligned16(k) || !grace_aligned16(v) || !grace_aligned16(out) ||
+      (q_row_stride & 7) || (out_row_stride & 7) || (kv_stride_b & 7) || (kv_stride_h & 7) || (kv_stride_t & 7) ||
+      q_row_stride < (int64_t)H * d_h || out_row_stride < (int64_t)H * d_h || kv_stride_t < d_h)
+    return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cross_attn_tc_supported(B, M, H, d_h, T_ctx)) {
+    return launch_cross_attn_tc(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,
+                                out_row_stride, lse, B, M, H, d_h, T_ctx, scale, s);
+  }
+  CrossSmallParams p;
+  p.q = q; p.k = k; p.v = v; p.out = out; p.lse = lse;
+  p.q_row_stride = q_row_stride; p.out_row_stride = out_row_stride;
+  p.kv_stride_b = kv_stride_b; p.kv_stride_h = kv_stride_h; p.kv_stride_t = kv_stride_t;
+  p.R = B * M; p.M = M; p.H = H; p.T = T_ctx; p.scale = scale;
+  const int64_t items = (int64_t)p.R * H;
+  const unsigned blocks = (unsigned)((items + 3) / 4);
+  switch (d_h) {
+    case 32: cross_attn_small_kernel<32><<<blocks, 128, 0, s>>>(p); break;
+    case 64: cross_attn_small_kernel<64><<<blocks, 128, 0, s>>>(p); break;
+    default: cross_attn_small_kernel<128><<<blocks, 128, 0, s>>>(p); break;
+  }
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}

@@ -1,0 +1,89 @@
+// One decode step of the GTM-constrained beam search (Sections 3.1-3.3): decoder layers on the
+// current beam rows, log-probabilities, CD + GTM mask with score add, beam top-k, state update.
+// Host-side sequencing only; every stage is one of the library's own kernels on the caller's
+// stream, with no allocation and no synchronisation, so the loop can be enqueued back to back.
+#include "common.cuh"
+
+extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
+  if (!d) return GRACE_INVALID_ARG;
+  if (d->B <= 0 || d->n_layers <= 0 || d->n_layers > GRACE_MAX_LAYERS || d->L <= 0 || d->L > 4 ||
+      d->L > GRACE_MAX_STEPS || d->H <= 0 || d->T_ctx <= 0)
+    return GRACE_INVALID_ARG;
+  if ((d->d_h != 32 && d->d_h != 64 && d->d_h != 128) || d->d_model % 64 || d->d_ffn % 64 ||
+      (d->H * d->d_h) % 64 || d->V % 64 || d->V <= 0 || d->V >= 65535 || d->d_model > 4096 || d->H * d->d_h > 1024)
+    return GRACE_UNSUPPORTED_SHAPE;
+  int64_t mmax = 0;
+  for (int t = 0; t <= d->L; ++t) {
+    if (d->beam_sizes[t] <= 0) return GRACE_INVALID_ARG;
+    if (t < d->L && d->beam_sizes[t] > mmax) mmax = d->beam_sizes[t];
+    if (t > 0 && (int64_t)d->beam_sizes[t] > (int64_t)d->beam_sizes[t - 1] * d->V) return GRACE_INVALID_ARG;
+    if (d->beam_sizes[t] > 4096) return GRACE_UNSUPPORTED_SHAPE;
+  }
+  if (d->beam_sizes[d->L] > mmax) mmax = d->beam_sizes[d->L];
+  if (d->R_max < (int64_t)d->B * mmax) return GRACE_INVALID_ARG;
+  for (int l = 0; l < d->n_layers; ++l) {
+    const grace_layer_t& w = d->layers[l];
+    if (!w.ln1_g || !w.ln1_b || !w.ln2_g || !w.ln2_b || !w.ln3_g || !w.ln3_b || !w.w_qkv || !w.w_o || !w.w_qc ||
+        !w.w_oc || !w.w_1 || !w.w_2 || !w.k_cross || !w.v_cross || !w.k_cache || !w.v_cache)
+      return GRACE_INVALID_ARG;
+  }
+  if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || !d->x || !d->h || !d->qkv ||
+      !d->attn || !d->logp || !d->topk_ws || !d->out_flat)
+    return GRACE_INVALID_ARG;
+  for (int i = 0; i < 2; ++i)
+    if (!d->token[i] || !d->score[i] || !d->node[i] || !d->key[i]) return GRACE_INVALID_ARG;
+  if (d->trie.V != d->V || d->trie.L != d->L || !d->trie.child_bits || !d->trie.child_base) return GRACE_INVALID_ARG;
+  return GRACE_OK;
+}
+
+#define GRACE_TRY(expr)                         \
+  do {                                          \
+    grace_status_t _s = (expr);                 \
+    if (_s != GRACE_OK) return _s;              \
+  } while (0)
+
+extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, void* stream) {
+  GRACE_TRY(grace_decoder_validate(d));
+  if (t < 0 || t >= d->L) return GRACE_INVALID_ARG;
+  const int cur = t & 1, nxt = cur ^ 1;
+  const int B = d->B, M = d->beam_sizes[t], K = d->beam_sizes[t + 1];
+  const int R = B * M;
+  const int D = d->d_model, HD = d->H * d->d_h;
+  const float scale = 1.0f / sqrtf((float)d->d_h);
+  int32_t* st = d->d_status;
+
+  GRACE_TRY(grace_embed(d->token[cur], d->embed, d->pos + (int64_t)t * D, d->x, R, D, d->V + 1, st, stream));
+  for (int l = 0; l < d->n_layers; ++l) {
+    const grace_layer_t& w = d->layers[l];
+    // self-attention block
+    GRACE_TRY(grace_layer_norm(d->x, w.ln1_g, w.ln1_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(grace_linear(d->h, D, w.w_qkv, D, d->qkv, nullptr, 3 * HD, nullptr, R, 3 * HD, D, 0, stream));
+    GRACE_TRY(grace_self_attn(d->qkv, 3 * HD, w.k_cache, w.v_cache, d->parents, d->beam_sizes, d->attn, HD,
+                              B, t, d->H, d->d_h, d->R_max, scale, st, stream));
+    GRACE_TRY(grace_linear(d->attn, HD, w.w_o, HD, nullptr, d->x, D, d->x, R, D, HD, 0, stream));
+    // cross-attention block
+    GRACE_TRY(grace_layer_norm(d->x, w.ln2_g, w.ln2_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(grace_linear(d->h, D, w.w_qc, D, d->qkv, nullptr, HD, nullptr, R, HD, D, 0, stream));
+    GRACE_TRY(grace_cross_attn(d->qkv, HD, w.k_cross, w.v_cross, (int64_t)d->H * d->T_ctx * d->d_h,
+                               (int64_t)d->T_ctx * d->d_h, d->d_h, d->attn, HD, nullptr, B, M, d->H, d->d_h,
+                               d->T_ctx, scale, st, stream));
+    GRACE_TRY(grace_linear(d->attn, HD, w.w_oc, HD, nullptr, d->x, D, d->x, R, D, HD, 0, stream));
+    // feed-forward block
+    GRACE_TRY(grace_layer_norm(d->x, w.ln3_g, w.ln3_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(grace_linear(d->h, D, w.w_1, D, d->qkv, nullptr, d->d_ffn, nullptr, R, d->d_ffn, D, 1, stream));
+    GRACE_TRY(grace_linear(d->qkv, d->d_ffn, w.w_2, d->d_ffn, nullptr, d->x, D, d->x, R, D, d->d_ffn, 0, stream));
+  }
+  GRACE_TRY(grace_layer_norm(d->x, d->lnf_g, d->lnf_b, d->h, R, D, d->ln_eps, stream));
+  GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
+  GRACE_TRY(grace_log_softmax(d->logp, R, d->V, stream));
+  // CD + GTM mask and score add, in place over the log-probabilities
+  GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->logp,
+                           nullptr, B, M, d->V, t, st, stream));
+  // parents of step t+1 live in slab t+1; tokens become the next step's input tokens
+  int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
+  GRACE_TRY(grace_beam_topk(d->logp, B, (int64_t)M * d->V, K, d->V, d->score[nxt], d->out_flat, parent_out,
+                            d->token[nxt], d->topk_ws, d->topk_ws_bytes, st, stream));
+  GRACE_TRY(grace_beam_update(parent_out, d->token[nxt], d->score[nxt], d->node[cur], d->key[cur], &d->trie,
+                              d->node[nxt], d->key[nxt], B, K, M, t, st, stream));
+  return GRACE_OK;
+}

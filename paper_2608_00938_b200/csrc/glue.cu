@@ -1,0 +1,174 @@
+// Decoder-layer glue around the attention kernels (Section 3.2): token embedding, LayerNorm,
+// log-softmax.  All three are row-wise and HBM-bound; one warp (LayerNorm, embedding) or one
+// CTA (log-softmax over the vocabulary) per row, fp32 statistics.
+#include "common.cuh"
+
+namespace grace {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFullMask, v, o));
+  return v;
+}
+
+// x fp32 [R][D] -> out bf16 [R][D]; D % 4 == 0, D <= 4096.  Two-pass statistics in registers.
+template <int MAXV>   // float4 pieces per lane
+__global__ void __launch_bounds__(128)
+layer_norm_kernel(const float* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                  uint16_t* __restrict__ out, int R, int D, float eps) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= R) return;
+  const int n4 = D >> 2;
+  const float4* row = reinterpret_cast<const float4*>(x + (int64_t)r * D);
+  float4 v[MAXV];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 32 + lane;
+    v[i] = (c < n4) ? __ldg(row + c) : make_float4(0, 0, 0, 0);
+    sum += v[i].x + v[i].y + v[i].z + v[i].w;
+  }
+  const float mean = warp_sum(sum) / (float)D;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 32 + lane;
+    if (c < n4) {
+      const float a = v[i].x - mean, b = v[i].y - mean, cc = v[i].z - mean, d = v[i].w - mean;
+      sq += a * a + b * b + cc * cc + d * d;
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(sq) / (float)D + eps);
+  uint2* orow = reinterpret_cast<uint2*>(out + (int64_t)r * D);
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 32 + lane;
+    if (c < n4) {
+      const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + c);
+      const float4 bb = __ldg(reinterpret_cast<const float4*>(beta) + c);
+      const float a = (v[i].x - mean) * rstd * g.x + bb.x;
+      const float b = (v[i].y - mean) * rstd * g.y + bb.y;
+      const float cc = (v[i].z - mean) * rstd * g.z + bb.z;
+      const float d = (v[i].w - mean) * rstd * g.w + bb.w;
+      orow[c] = make_uint2(pack_bf16x2(a, b), pack_bf16x2(cc, d));
+    }
+  }
+}
+
+__global__ void embed_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
+                             const uint16_t* __restrict__ pos, float* __restrict__ x, int R, int D,
+                             int n_rows_embed, int32_t* d_status) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= R) return;
+  int tok = __ldg(token + r);
+  if (tok < 0 || tok >= n_rows_embed) {
+    if (lane == 0) flag_status(d_status, GRACE_DEV_BAD_INDEX);
+    tok = 0;
+  }
+  const uint2* erow = reinterpret_cast<const uint2*>(embed + (int64_t)tok * D);
+  const uint2* prow = reinterpret_cast<const uint2*>(pos);
+  float4* xrow = reinterpret_cast<float4*>(x + (int64_t)r * D);
+  for (int c = lane; c < (D >> 2); c += 32) {
+    const uint2 e = __ldg(erow + c), p = __ldg(prow + c);
+    xrow[c] = make_float4(bf16_lo(e.x) + bf16_lo(p.x), bf16_hi(e.x) + bf16_hi(p.x),
+                          bf16_lo(e.y) + bf16_lo(p.y), bf16_hi(e.y) + bf16_hi(p.y));
+  }
+}
+
+// In-place log-softmax of fp32 [R][V]; one CTA of 256 threads per row, row held in registers.
+template <int MAXV>
+__global__ void __launch_bounds__(256)
+log_softmax_kernel(float* __restrict__ logits, int R, int V) {
+  __shared__ float red[8];
+  const int r = blockIdx.x;
+  const int n4 = V >> 2;
+  float4* row = reinterpret_cast<float4*>(logits + (int64_t)r * V);
+  float4 v[MAXV];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 256 + threadIdx.x;
+    v[i] = (c < n4) ? row[c] : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    mx = fmaxf(mx, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+  }
+  mx = warp_max(mx);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+  __syncthreads();
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 256 + threadIdx.x;
+    if (c < n4) sum += expf(v[i].x - mx) + expf(v[i].y - mx) + expf(v[i].z - mx) + expf(v[i].w - mx);
+  }
+  sum = warp_sum(sum);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  sum = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) sum += red[w];
+  const float lse = mx + logf(sum);
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 256 + threadIdx.x;
+    if (c < n4) row[c] = make_float4(v[i].x - lse, v[i].y - lse, v[i].z - lse, v[i].w - lse);
+  }
+}
+
+}  // namespace grace
+
+extern "C" grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
+                                           uint16_t* out, int R, int D, float eps, void* stream) {
+  using namespace grace;
+  if (!x || !gamma || !beta || !out || R <= 0 || D <= 0) return GRACE_INVALID_ARG;
+  if ((D & 3) || D > 4096) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(x) || !grace_aligned16(gamma) || !grace_aligned16(beta) || (reinterpret_cast<uintptr_t>(out) & 7))
+    return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blocks = (R + 3) / 4;
+  const int pieces = ((D >> 2) + 31) / 32;
+  if (pieces <= 2) layer_norm_kernel<2><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 4) layer_norm_kernel<4><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 8) layer_norm_kernel<8><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 16) layer_norm_kernel<16><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else layer_norm_kernel<32><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_embed(const int32_t* token, const uint16_t* embed, const uint16_t* pos,
+                                      float* x, int R, int D, int n_rows_embed, int32_t* d_status, void* stream) {
+  if (!token || !embed || !pos || !x || R <= 0 || D <= 0 || n_rows_embed <= 0) return GRACE_INVALID_ARG;
+  if (D & 3) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(x) || (reinterpret_cast<uintptr_t>(embed) & 7) || (reinterpret_cast<uintptr_t>(pos) & 7))
+    return GRACE_INVALID_ARG;
+  grace::embed_kernel<<<(R + 3) / 4, 128, 0, (cudaStream_t)stream>>>(token, embed, pos, x, R, D, n_rows_embed, d_status);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_log_softmax(float* logits, int R, int V, void* stream) {
+  using namespace grace;
+  if (!logits || R <= 0 || V <= 0) return GRACE_INVALID_ARG;
+  if ((V & 3) || V > 16384) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(logits)) return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int pieces = ((V >> 2) + 255) / 256;
+  if (pieces <= 1) log_softmax_kernel<1><<<R, 256, 0, s>>>(logits, R, V);
+  else if (pieces <= 2) log_softmax_kernel<2><<<R, 256, 0, s>>>(logits, R, V);
+  else if (pieces <= 4) log_softmax_kernel<4><<<R, 256, 0, s>>>(logits, R, V);
+  else if (pieces <= 8) log_softmax_kernel<8><<<R, 256, 0, s>>>(logits, R, V);
+  else log_softmax_kernel<16><<<R, 256, 0, s>>>(logits, R, V);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}

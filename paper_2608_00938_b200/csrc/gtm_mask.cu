@@ -1,0 +1,231 @@
+// CD + GTM mask with score add (Sections 3.1, 4.1, 5.4) and the beam-state update after top-k
+// (Sections 3.3, 4.4).
+//
+// One warp owns one beam row.  The row's child bitmask (V/64 words) is loaded once into
+// registers, one word per lane, with a warp prefix sum of popcounts so that any lane can turn a
+// token into the id of the child node.  Each lane then streams float4 pieces of the row's
+// log-probabilities: coalesced 512-byte warp loads in, 512-byte warp stores out.  The request's
+// matcher (node-eligibility bits or Bloom filter words) is read only for catalog-valid tokens.
+// HBM-bound at the root levels (4 bytes in + 4 bytes out per candidate).
+#include "common.cuh"
+
+namespace grace {
+
+struct MaskParams {
+  const float* logp;
+  const float* beam_score;
+  const int32_t* beam_node;
+  const uint64_t* beam_key;
+  const uint64_t* child_bits;
+  const int32_t* child_base;
+  const uint64_t* matcher_bits;
+  float* cand;
+  uint64_t* allow_bits;
+  int32_t* d_status;
+  int64_t num_internal, num_nodes, words_per_request;
+  int R, M, V, prefix_len;
+  int bloom_mask_bits;     // 2^log2_bits - 1 (as uint32)
+  int bloom_hashes;
+};
+
+template <int KIND>
+__device__ __forceinline__ bool token_matches(const MaskParams& p, const uint64_t* req_bits,
+                                              int64_t child, uint64_t row_key, int v) {
+  if (KIND == GRACE_MATCH_NONE) return true;
+  if (KIND == GRACE_MATCH_NODE_BITMASK) {
+    if (child < 0 || child >= p.num_nodes) return false;
+    return (__ldg(req_bits + (child >> 6)) >> (child & 63)) & 1ull;
+  }
+  // prefix Bloom filter: all probed bits must be set; stop at the first clear bit
+  const uint64_t key = row_key | ((uint64_t)(v + 1) << (16 * p.prefix_len));
+  const uint64_t z = mix64(key);
+  const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
+  for (int i = 0; i < p.bloom_hashes; ++i) {
+    const uint32_t pos = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
+    if (!((__ldg(req_bits + (pos >> 6)) >> (pos & 63)) & 1ull)) return false;
+  }
+  return true;
+}
+
+constexpr int kMaskWarpsPerBlock = 8;
+
+template <int KIND>
+__global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
+gtm_mask_kernel(const MaskParams p) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * kMaskWarpsPerBlock + (threadIdx.x >> 5);
+  if (r >= p.R) return;
+  const int V = p.V;
+  const int W = V >> 6;
+  const int b = r / p.M;
+  int node = __ldg(p.beam_node + r);
+  bool dead = node < 0;
+  if (!dead && node >= p.num_internal) {           // leaf or garbage: nothing below it
+    if (node >= p.num_nodes && lane == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
+    dead = true;
+  }
+  const float score = __ldg(p.beam_score + r);
+  const uint64_t row_key = (KIND == GRACE_MATCH_PREFIX_BLOOM) ? __ldg(p.beam_key + r) : 0ull;
+  const uint64_t* req_bits = (KIND == GRACE_MATCH_NONE) ? nullptr : p.matcher_bits + (int64_t)b * p.words_per_request;
+  const int32_t base = dead ? -1 : __ldg(p.child_base + node);
+  const float ninf = __int_as_float(0xff800000);
+  const float* lrow = p.logp + (int64_t)r * V;
+  bool saw_nan = false;
+
+  // chunks of 2048 tokens: 32 words, one per lane
+  int rank_before_chunk = 0;
+  for (int w0 = 0; w0 < W; w0 += 32) {
+    uint64_t word = 0;
+    if (!dead && w0 + lane < W) word = __ldg(p.child_bits + (int64_t)node * W + w0 + lane);
+    int pc = __popcll(word);
+    int incl = pc;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int o = __shfl_up_sync(kFullMask, incl, d);
+      if (lane >= d) incl += o;
+    }
+    const int excl = incl - pc + rank_before_chunk;       // children before this lane's word
+    rank_before_chunk += __shfl_sync(kFullMask, incl, 31);
+
+    const int chunk_tokens = min(2048, V - (w0 << 6));
+    // 128 tokens per iteration: lane handles tokens 4*lane .. 4*lane+3 of the group
+    for (int g = 0; g < chunk_tokens; g += 128) {
+      const int tok0 = (w0 << 6) + g + 4 * lane;          // first token of this lane
+      const bool in_range = (g + 4 * lane) < chunk_tokens; // V % 64 == 0, so all 4 or none
+      const int src_lane = (g >> 6) + (lane >> 4);         // lane holding the word of these tokens
+      const uint64_t cw = __shfl_sync(kFullMask, word, src_lane);
+      const int cex = __shfl_sync(kFullMask, excl, src_lane);
+      float4 lp = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (in_range && !dead && cw != 0ull) lp = __ldg(reinterpret_cast<const float4*>(lrow + tok0));
+      float vals[4] = {lp.x, lp.y, lp.z, lp.w};
+      float outv[4];
+      uint32_t nib = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int bit = (tok0 + j) & 63;
+        bool ok = in_range && ((cw >> bit) & 1ull);
+        if (ok) {
+          const int64_t child = (int64_t)base + cex + __popcll(cw & ((1ull << bit) - 1ull));
+          ok = token_matches<KIND>(p, req_bits, child, row_key, tok0 + j);
+        }
+        outv[j] = ok ? (score + vals[j]) : ninf;
+        if (ok && vals[j] != vals[j]) saw_nan = true;
+        nib |= (ok ? 1u : 0u) << j;
+      }
+      if (in_range && p.cand != nullptr)
+        *reinterpret_cast<float4*>(p.cand + (int64_t)r * V + tok0) = make_float4(outv[0], outv[1], outv[2], outv[3]);
+      if (p.allow_bits != nullptr) {
+        // 16 lanes x 4 bits -> one 64-bit word
+        uint64_t x = (uint64_t)nib << (4 * (lane & 15));
+#pragma unroll
+        for (int d = 1; d < 16; d <<= 1) x |= __shfl_xor_sync(kFullMask, x, d);
+        if ((lane & 15) == 0 && in_range)
+          p.allow_bits[(int64_t)r * W + w0 + (g >> 6) + (lane >> 4)] = x;
+      }
+    }
+  }
+  if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
+}
+
+__global__ void beam_update_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ token,
+                                   const float* __restrict__ score, const int32_t* __restrict__ prev_node,
+                                   const uint64_t* __restrict__ prev_key, const uint64_t* __restrict__ child_bits,
+                                   const int32_t* __restrict__ child_base, int64_t num_internal,
+                                   int32_t* __restrict__ new_node, uint64_t* __restrict__ new_key,
+                                   int B, int K, int M_prev, int V, int prefix_len, int32_t* d_status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * K) return;
+  const int b = i / K;
+  int par = parent[i];
+  const int tok = token[i];
+  if (par < 0 || par >= M_prev || tok < 0 || tok >= V) {
+    flag_status(d_status, GRACE_DEV_BAD_INDEX);
+    new_node[i] = -1;
+    new_key[i] = 0;
+    return;
+  }
+  const int64_t src = (int64_t)b * M_prev + par;
+  new_key[i] = prev_key[src] | ((uint64_t)(tok + 1) << (16 * prefix_len));
+  const int node = prev_node[src];
+  int out = -1;
+  if (node >= 0 && node < num_internal && score[i] != __int_as_float(0xff800000)) {
+    const int W = V >> 6;
+    const uint64_t* row = child_bits + (int64_t)node * W;
+    const uint64_t word = row[tok >> 6];
+    if ((word >> (tok & 63)) & 1ull) {
+      int rank = __popcll(word & ((1ull << (tok & 63)) - 1ull));
+      for (int w = 0; w < (tok >> 6); ++w) rank += __popcll(row[w]);
+      out = child_base[node] + rank;
+    }
+  }
+  new_node[i] = out;
+}
+
+}  // namespace grace
+
+static bool trie_ok(const grace_trie_t* t, int V) {
+  return t && t->child_bits && t->child_base && t->V == V && V > 0 && V % 64 == 0 && V < 65535 &&
+         t->num_internal > 0 && t->num_nodes >= t->num_internal && t->L >= 1 && t->L <= 4;
+}
+
+extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_score,
+                                         const int32_t* beam_node, const uint64_t* beam_key,
+                                         const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                         float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                         int prefix_len, int32_t* d_status, void* stream) {
+  using namespace grace;
+  if (!logp || !beam_score || !beam_node || !matcher || (!cand && !allow_bits)) return GRACE_INVALID_ARG;
+  if (B <= 0 || M <= 0 || (int64_t)B * M > 0x7fffffff) return GRACE_INVALID_ARG;
+  if (!trie_ok(trie, V)) return GRACE_INVALID_ARG;
+  if (prefix_len < 0 || prefix_len >= trie->L) return GRACE_INVALID_ARG;
+  if (!grace_aligned16(logp) || (cand && !grace_aligned16(cand))) return GRACE_INVALID_ARG;
+  MaskParams p;
+  p.logp = logp; p.beam_score = beam_score; p.beam_node = beam_node; p.beam_key = beam_key;
+  p.child_bits = trie->child_bits; p.child_base = trie->child_base;
+  p.matcher_bits = matcher->bits; p.cand = cand; p.allow_bits = allow_bits; p.d_status = d_status;
+  p.num_internal = trie->num_internal; p.num_nodes = trie->num_nodes;
+  p.words_per_request = matcher->words_per_request;
+  p.R = B * M; p.M = M; p.V = V; p.prefix_len = prefix_len;
+  p.bloom_mask_bits = 0; p.bloom_hashes = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blocks = (p.R + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock;
+  const int threads = kMaskWarpsPerBlock * 32;
+  switch (matcher->kind) {
+    case GRACE_MATCH_NONE:
+      gtm_mask_kernel<GRACE_MATCH_NONE><<<blocks, threads, 0, s>>>(p);
+      break;
+    case GRACE_MATCH_NODE_BITMASK:
+      if (!matcher->bits || matcher->words_per_request * 64 < trie->num_nodes) return GRACE_INVALID_ARG;
+      gtm_mask_kernel<GRACE_MATCH_NODE_BITMASK><<<blocks, threads, 0, s>>>(p);
+      break;
+    case GRACE_MATCH_PREFIX_BLOOM:
+      if (!matcher->bits || !beam_key || matcher->bloom_log2_bits < 6 || matcher->bloom_log2_bits > 32 ||
+          matcher->bloom_hashes < 1 || matcher->bloom_hashes > 16 ||
+          matcher->words_per_request != (int64_t)((1ull << matcher->bloom_log2_bits) / 64))
+        return GRACE_INVALID_ARG;
+      p.bloom_mask_bits = (int)(uint32_t)((1ull << matcher->bloom_log2_bits) - 1ull);
+      p.bloom_hashes = matcher->bloom_hashes;
+      gtm_mask_kernel<GRACE_MATCH_PREFIX_BLOOM><<<blocks, threads, 0, s>>>(p);
+      break;
+    default:
+      return GRACE_INVALID_ARG;
+  }
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_beam_update(const int32_t* parent, const int32_t* token, const float* score,
+                                            const int32_t* prev_node, const uint64_t* prev_key,
+                                            const grace_trie_t* trie, int32_t* new_node, uint64_t* new_key,
+                                            int B, int K, int M_prev, int prefix_len,
+                                            int32_t* d_status, void* stream) {
+  if (!parent || !token || !score || !prev_node || !prev_key || !new_node || !new_key) return GRACE_INVALID_ARG;
+  if (!trie || !trie_ok(trie, trie->V)) return GRACE_INVALID_ARG;
+  if (B <= 0 || K <= 0 || M_prev <= 0 || prefix_len < 0 || prefix_len >= 4) return GRACE_INVALID_ARG;
+  const int n = B * K;
+  grace::beam_update_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
+      parent, token, score, prev_node, prev_key, trie->child_bits, trie->child_base, trie->num_internal,
+      new_node, new_key, B, K, M_prev, trie->V, prefix_len, d_status);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}

@@ -1,0 +1,165 @@
+// Host-side index builders: dense child-bitmask trie (Section 4.4, Appendix A), per-request
+// node-eligibility bitmask and prefix Bloom filter (Section 4.1's TM in per-request form).
+// Not on the timed path.
+#include <vector>
+
+#include "common.cuh"
+
+namespace {
+
+bool sids_sorted_distinct(const int32_t* sids, int64_t n, int V, int L) {
+  for (int64_t i = 0; i < n; ++i) {
+    const int32_t* cur = sids + i * L;
+    for (int j = 0; j < L; ++j)
+      if (cur[j] < 0 || cur[j] >= V) return false;
+    if (i == 0) continue;
+    const int32_t* prev = cur - L;
+    int j = 0;
+    while (j < L && prev[j] == cur[j]) ++j;
+    if (j == L || prev[j] > cur[j]) return false;
+  }
+  return true;
+}
+
+bool shape_ok(const int32_t* sids, int64_t n, int V, int L) {
+  return sids != nullptr && n > 0 && V > 0 && V % 64 == 0 && V < 65535 && L >= 1 && L <= 4;
+}
+
+// For sorted SIDs, SID i opens a new node at level l (1-based) iff it differs from SID i-1
+// somewhere in its first l tokens.  first_diff = index of the first differing token.
+inline int first_diff(const int32_t* sids, int64_t i, int L) {
+  if (i == 0) return 0;
+  const int32_t* a = sids + (i - 1) * L;
+  const int32_t* b = sids + i * L;
+  int j = 0;
+  while (j < L && a[j] == b[j]) ++j;
+  return j;
+}
+
+inline uint64_t prefix_key(const int32_t* tok, int len) {
+  uint64_t key = 0;
+  for (int i = 0; i < len; ++i) key |= (uint64_t)(tok[i] + 1) << (16 * i);
+  return key;
+}
+
+}  // namespace
+
+extern "C" grace_status_t grace_trie_count_nodes(const int32_t* sids, int64_t n_sids, int V, int L,
+                                                 int64_t* level_start) {
+  if (!shape_ok(sids, n_sids, V, L) || level_start == nullptr) return GRACE_INVALID_ARG;
+  if (!sids_sorted_distinct(sids, n_sids, V, L)) return GRACE_INVALID_ARG;
+  std::vector<int64_t> count(L + 1, 0);
+  count[0] = 1;
+  for (int64_t i = 0; i < n_sids; ++i) {
+    int d = first_diff(sids, i, L);
+    for (int l = d + 1; l <= L; ++l) ++count[l];      // new nodes at levels d+1 .. L
+  }
+  level_start[0] = 0;
+  for (int l = 0; l <= L; ++l) level_start[l + 1] = level_start[l] + count[l];
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_trie_build_dense(const int32_t* sids, int64_t n_sids, int V, int L,
+                                                 uint64_t* child_bits, int32_t* child_base) {
+  if (child_bits == nullptr || child_base == nullptr) return GRACE_INVALID_ARG;
+  std::vector<int64_t> level_start(L + 2);
+  grace_status_t st = grace_trie_count_nodes(sids, n_sids, V, L, level_start.data());
+  if (st != GRACE_OK) return st;
+  const int64_t n_internal = level_start[L];
+  const int W = V / 64;
+  for (int64_t i = 0; i < n_internal * W; ++i) child_bits[i] = 0;
+  for (int64_t i = 0; i < n_internal; ++i) child_base[i] = -1;
+  // cur[l] = id of the node holding the current SID's length-l prefix
+  std::vector<int64_t> cur(L + 1, 0), next_id(L + 1);
+  for (int l = 0; l <= L; ++l) next_id[l] = level_start[l];
+  cur[0] = 0;
+  for (int64_t i = 0; i < n_sids; ++i) {
+    const int32_t* s = sids + i * L;
+    int d = first_diff(sids, i, L);
+    for (int l = d + 1; l <= L; ++l) {
+      cur[l] = next_id[l]++;
+      const int64_t parent = cur[l - 1];
+      const int tok = s[l - 1];
+      child_bits[parent * W + (tok >> 6)] |= 1ull << (tok & 63);
+      if (child_base[parent] < 0) child_base[parent] = (int32_t)cur[l];
+    }
+  }
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_node_bitmask_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                                   const uint8_t* eligible, uint64_t* node_bits) {
+  if (eligible == nullptr || node_bits == nullptr) return GRACE_INVALID_ARG;
+  std::vector<int64_t> level_start(L + 2);
+  grace_status_t st = grace_trie_count_nodes(sids, n_sids, V, L, level_start.data());
+  if (st != GRACE_OK) return st;
+  const int64_t words = (level_start[L + 1] + 63) / 64;
+  for (int64_t i = 0; i < words; ++i) node_bits[i] = 0;
+  std::vector<int64_t> cur(L + 1, 0), next_id(L + 1);
+  for (int l = 0; l <= L; ++l) next_id[l] = level_start[l];
+  for (int64_t i = 0; i < n_sids; ++i) {
+    int d = first_diff(sids, i, L);
+    for (int l = d + 1; l <= L; ++l) cur[l] = next_id[l]++;
+    if (eligible[i]) {
+      for (int l = 0; l <= L; ++l) node_bits[cur[l] >> 6] |= 1ull << (cur[l] & 63);
+    }
+  }
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_bloom_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                            const uint8_t* eligible, int log2_bits, int n_hashes,
+                                            uint64_t* bloom_words) {
+  if (!shape_ok(sids, n_sids, V, L) || eligible == nullptr || bloom_words == nullptr)
+    return GRACE_INVALID_ARG;
+  if (log2_bits < 6 || log2_bits > 32 || n_hashes < 1 || n_hashes > 16) return GRACE_INVALID_ARG;
+  const uint64_t m_mask = (1ull << log2_bits) - 1;
+  for (uint64_t i = 0; i < (1ull << log2_bits) / 64; ++i) bloom_words[i] = 0;
+  for (int64_t i = 0; i < n_sids; ++i) {
+    if (!eligible[i]) continue;
+    for (int len = 1; len <= L; ++len) {
+      const uint64_t z = grace::mix64(prefix_key(sids + i * L, len));
+      const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
+      for (int p = 0; p < n_hashes; ++p) {
+        const uint64_t pos = (uint32_t)(h1 + (uint32_t)p * h2) & m_mask;
+        bloom_words[pos >> 6] |= 1ull << (pos & 63);
+      }
+    }
+  }
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_trie_walk(const uint64_t* child_bits, const int32_t* child_base,
+                                          int V, int L, int64_t num_internal, const int32_t* tokens,
+                                          int len, int32_t* node) {
+  if (!child_bits || !child_base || !tokens || !node || len < 0 || len > L || V % 64) return GRACE_INVALID_ARG;
+  const int W = V / 64;
+  int64_t cur = 0;
+  for (int i = 0; i < len; ++i) {
+    const int tok = tokens[i];
+    if (tok < 0 || tok >= V || cur >= num_internal) { *node = -1; return GRACE_OK; }
+    const uint64_t* row = child_bits + cur * W;
+    if (!((row[tok >> 6] >> (tok & 63)) & 1)) { *node = -1; return GRACE_OK; }
+    int rank = 0;
+    for (int w = 0; w < (tok >> 6); ++w) rank += __builtin_popcountll(row[w]);
+    rank += __builtin_popcountll(row[tok >> 6] & ((1ull << (tok & 63)) - 1));
+    cur = child_base[cur] + rank;
+  }
+  *node = (int32_t)cur;
+  return GRACE_OK;
+}
+
+extern "C" const char* grace_status_string(grace_status_t s) {
+  switch (s) {
+    case GRACE_OK: return "ok";
+    case GRACE_INVALID_ARG: return "invalid argument";
+    case GRACE_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case GRACE_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case GRACE_CUDA_ERROR: return "CUDA error";
+    case GRACE_TIMEOUT: return "timeout";
+  }
+  return "unknown";
+}
+
+extern "C" int grace_version(void) { return 1; }
+extern "C" int grace_built_for_sm(void) { return 100; }

@@ -1,0 +1,183 @@
+// y = act(x @ w^T) (+ residual): the projection / feed-forward / logits GEMMs of the decoder
+// layer (Section 3.2), on tcgen05 tensor cores.
+//
+// One CTA computes a 128 x BN output tile.  A producer thread streams 128 x 64 bf16 tiles of x
+// and BN x 64 tiles of w through a ring of shared-memory stages with TMA (128-byte swizzle,
+// out-of-range rows read as zero, so ragged M and N need no special path).  One thread issues
+// tcgen05.mma (M = 128, N = BN, K = 16 per instruction) with the fp32 accumulator in TMEM;
+// tcgen05.commit frees each stage as soon as the tensor core has consumed it.  All four warps then
+// read the accumulator back (each warp its own 32 TMEM lanes = 32 output rows), apply ReLU /
+// residual, and store bf16 or fp32.  Two CTAs fit on an SM, so one CTA's epilogue overlaps the
+// other's main loop.
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace grace {
+
+constexpr int kGemmBM = 128;
+constexpr int kGemmBK = 64;
+constexpr int kGemmStages = 3;
+
+template <int BN>
+struct GemmSmem {
+  static constexpr int kABytes = kGemmBM * kGemmBK * 2;
+  static constexpr int kBBytes = BN * kGemmBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kTotal = kGemmStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct GemmParams {
+  uint16_t* y_bf16;
+  float* y_f32;
+  const float* residual;
+  int64_t ldy;
+  int M, N, K, relu;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(128)
+linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+              const GemmParams p) {
+  using S = GemmSmem<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(tiles + kGemmStages * S::kStageBytes);
+  uint64_t* empty = full + kGemmStages;
+  uint64_t* accum_bar = empty + kGemmStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * kGemmBM, n0 = blockIdx.x * BN;
+  const int KB = p.K / kGemmBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGemmStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+    tc::mbar_init(accum_bar, 1);
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+    tc::tma_prefetch_desc(&map_x);
+    tc::tma_prefetch_desc(&map_w);
+  }
+  if (warp == 0) tc::tmem_alloc(tmem_slot, BN < 32 ? 32 : BN);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    // ---- TMA producer ----
+    for (int kb = 0; kb < KB; ++kb) {
+      const int s = kb % kGemmStages;
+      if (!tc::mbar_wait(empty + s, ((kb / kGemmStages) & 1) ^ 1, abort_flag)) break;
+      tc::mbar_expect_tx(full + s, S::kStageBytes);
+      uint8_t* a = tiles + s * S::kStageBytes;
+      tc::tma_load_2d(a, &map_x, full + s, kb * kGemmBK, m0);
+      tc::tma_load_2d(a + S::kABytes, &map_w, full + s, kb * kGemmBK, n0);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---- MMA issuer ----
+    constexpr uint32_t idesc = tc::idesc_bf16(kGemmBM, BN, 0);
+    for (int kb = 0; kb < KB; ++kb) {
+      const int s = kb % kGemmStages;
+      if (!tc::mbar_wait(full + s, (kb / kGemmStages) & 1, abort_flag)) break;
+      tc::tc_fence_after();
+      const uint32_t a_addr = tc::smem_addr(tiles + s * S::kStageBytes);
+      const uint64_t a_desc = tc::smem_desc_sw128(a_addr, 16, 1024);
+      const uint64_t b_desc = tc::smem_desc_sw128(a_addr + S::kABytes, 16, 1024);
+#pragma unroll
+      for (int k = 0; k < kGemmBK / 16; ++k)
+        tc::mma_ss(tmem_base, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+      tc::mma_commit(empty + s);
+    }
+    tc::mma_commit(accum_bar);
+  }
+  __syncwarp();
+
+  // ---- epilogue: warp w owns TMEM lanes 32w .. 32w+31 = rows m0 + 32w + lane ----
+  const bool ok = tc::mbar_wait(accum_bar, 0, abort_flag);
+  tc::tc_fence_after();
+  __syncwarp();
+  if (ok) {
+    const int m = m0 + warp * 32 + lane;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 16) {
+      uint32_t acc[16];
+      tc::tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, acc);
+      tc::tmem_ld_wait();
+      const int n = n0 + c;
+      if (m < p.M && n < p.N) {           // N % 16 == 0: the 16 columns are all in or all out
+        float v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          v[j] = __uint_as_float(acc[j]);
+          if (p.relu) v[j] = fmaxf(v[j], 0.f);
+        }
+        if (p.residual != nullptr) {
+          const float4* res = reinterpret_cast<const float4*>(p.residual + (int64_t)m * p.ldy + n);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float4 r4 = res[j];
+            v[4 * j] += r4.x; v[4 * j + 1] += r4.y; v[4 * j + 2] += r4.z; v[4 * j + 3] += r4.w;
+          }
+        }
+        if (p.y_f32 != nullptr) {
+          float4* dst = reinterpret_cast<float4*>(p.y_f32 + (int64_t)m * p.ldy + n);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(p.y_bf16 + (int64_t)m * p.ldy + n);
+          dst[0] = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+          dst[1] = make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
+        }
+      }
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem_base, BN < 32 ? 32 : BN);
+}
+
+template <int BN>
+static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw, const GemmParams& p, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmSmem<BN>::kTotal));
+    attr_set = true;
+  }
+  dim3 grid((p.N + BN - 1) / BN, (p.M + kGemmBM - 1) / kGemmBM);
+  linear_kernel<BN><<<grid, 128, GemmSmem<BN>::kTotal, s>>>(mx, mw, p);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+}  // namespace grace
+
+extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                       uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
+                                       int M, int N, int K, int relu, void* stream) {
+  using namespace grace;
+  if (!x || !w || ((y_bf16 == nullptr) == (y_f32 == nullptr))) return GRACE_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
+  if ((K % kGemmBK) || (N % 16)) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(x) || !grace_aligned16(w) || !grace_aligned16(y_bf16) || !grace_aligned16(y_f32) ||
+      !grace_aligned16(residual) || (ldx & 7) || (ldw & 7) || (ldy & 7) || ldx < K || ldw < K || ldy < N)
+    return GRACE_INVALID_ARG;
+  CUtensorMap mx, mw;
+  const int BN = (N >= 128) ? 128 : 64;
+  {
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M}, str[1] = {(uint64_t)ldx};
+    const uint32_t box[2] = {(uint32_t)kGemmBK, (uint32_t)kGemmBM};
+    if (!tc::make_tmap_bf16(&mx, x, 2, dims, str, box)) return GRACE_CUDA_ERROR;
+  }
+  {
+    const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N}, str[1] = {(uint64_t)ldw};
+    const uint32_t box[2] = {(uint32_t)kGemmBK, (uint32_t)BN};
+    if (!tc::make_tmap_bf16(&mw, w, 2, dims, str, box)) return GRACE_CUDA_ERROR;
+  }
+  GemmParams p;
+  p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.ldy = ldy;
+  p.M = M; p.N = N; p.K = K; p.relu = relu;
+  cudaStream_t s = (cudaStream_t)stream;
+  return BN == 128 ? launch_linear<128>(mx, mw, p, s) : launch_linear<64>(mx, mw, p, s);
+}

@@ -1,0 +1,40 @@
+"""Helpers shared by the GPU parity tests (tensor upload, tolerance check)."""
+import numpy as np
+import torch
+
+import synth
+
+DEV = "cuda:0"
+
+
+def dev_bf16(bits: np.ndarray) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> torch.bfloat16 CUDA tensor of the same shape."""
+    return torch.from_numpy(bits.view(np.int16).copy()).to(DEV).view(torch.bfloat16)
+
+
+def host_f64_of_bf16(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    if a.dtype == np.uint64:
+        return torch.from_numpy(a.view(np.int64).copy()).to(DEV)
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def host_u64(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint64)
+
+
+def f64(bits: np.ndarray) -> np.ndarray:
+    return synth.bf16_bits_to_f32(bits).astype(np.float64)
+
+
+def assert_attention_close(got: np.ndarray, ref: np.ndarray, what: str = ""):
+    """bf16 attention outputs vs the fp64 oracle on the same bf16-rounded inputs:
+    max |g - r| <= 2e-2 and ||g - r||_F / ||r||_F <= 1e-2."""
+    got = got.astype(np.float64)
+    err = np.abs(got - ref)
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert err.max() <= 2e-2, f"{what}: max abs err {err.max():.4g} at {np.unravel_index(err.argmax(), err.shape)}"
+    assert rel <= 1e-2, f"{what}: relative Frobenius err {rel:.4g}"

@@ -1,0 +1,370 @@
+"""GPU parity: every C-ABI op against the oracle on the same seeded inputs, at
+sizes the oracle finishes in seconds that still span several tiles and ragged
+tails.  Integer / index / mask results bit-exact; bf16 attention within
+2e-2 max-abs and 1e-2 relative of the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import attention as OA
+from oracle import gtm as OG
+from oracle import matchers as OM
+from oracle import topk as OT
+from oracle.sid_trie import SidTrie
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2608_00938_b200 import api as _api
+    return _api
+
+
+from gpu_util import DEV, assert_attention_close, dev, dev_bf16, f64, host_u64  # noqa: E402
+
+
+# ------------------------------------------------------------------------------------------
+# CD + GTM mask
+# ------------------------------------------------------------------------------------------
+def _mask_problem(seed, V, L, n_sids, B, M, depth, frac=0.3):
+    rng = synth.rng_for(4, seed)
+    sids = synth.catalog(rng, n_sids, V, L)
+    trie = SidTrie(sids, V)
+    elig = [synth.eligible_subset(rng, n_sids, frac) for _ in range(B)]
+    prefix = np.zeros((B, M, depth), dtype=np.int32)
+    node = np.full((B, M), -1, dtype=np.int32)
+    for b in range(B):
+        pr = synth.beam_prefixes_from_sids(rng, sids[elig[b]], depth, M) if depth else np.zeros((1, 0), np.int32)
+        n = pr.shape[0]
+        prefix[b, :n] = pr
+        node[b, :n] = [trie.walk(p) for p in pr]
+    key = OM.prefix_keys(prefix.reshape(B * M, depth))
+    score = np.concatenate([synth.descending_scores(rng, M, depth) for _ in range(B)])
+    logp = synth.logp_rows(rng, B * M, V)
+    return sids, trie, elig, node.reshape(-1), key, score, logp
+
+
+@pytest.mark.parametrize("kind", ["none", "node", "bloom"])
+@pytest.mark.parametrize("V,L,n_sids,B,M,depth", [
+    (64, 3, 2000, 1, 16, 1),          # config-1 sized
+    (1024, 4, 60000, 3, 37, 1),       # dense level-1 rows, ragged row count
+    (1024, 4, 60000, 2, 64, 2),       # sparse rows
+    (2048, 4, 30000, 2, 9, 1),        # one bitmask word per lane
+    (4096, 3, 30000, 2, 5, 1),        # more than one 2048-token chunk
+    (192, 3, 5000, 2, 11, 0),         # root row, V not a multiple of 128
+])
+def test_gtm_mask_matches_oracle(api, kind, V, L, n_sids, B, M, depth):
+    if depth == 0:
+        M = 1
+    sids, trie, elig, node, key, score, logp = _mask_problem(7 * V + depth, V, L, n_sids, B, M, depth)
+    node[-1] = -1                                                     # a dead beam
+    bits, base, level_start = api.grace_trie_build_dense(sids, V)
+    d_bits, d_base = dev(bits), dev(base)
+    trie_s = api.make_trie(d_bits, d_base, V, L, trie.num_nodes)
+    if kind == "none":
+        o_matcher, matcher, keep = OG.NoMatcher(), api.make_matcher(api.MATCH_NONE), None
+    elif kind == "node":
+        o_matcher = OG.NodeBitmaskMatcher(np.stack([OM.node_eligibility(trie, sids, e) for e in elig]))
+        keep = dev(np.stack([api.grace_node_bitmask_build(sids, V, e, trie.num_nodes) for e in elig]))
+        matcher = api.make_matcher(api.MATCH_NODE_BITMASK, keep)
+    else:
+        o_matcher = OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 16, 4) for e in elig])
+        keep = dev(np.stack([api.grace_bloom_build(sids, V, e, 16, 4) for e in elig]))
+        matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, keep, 16, 4)
+    cand_ref, allow_ref, child_ref = OG.gtm_mask(logp, score, node, key, depth, trie, o_matcher, B, M)
+    cand = torch.full((B * M, V), 7.0, device=DEV)
+    allow = torch.zeros((B * M, V // 64), dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_gtm_mask(dev(logp), dev(score), dev(node), dev(key), trie_s, matcher, cand, allow, B, M, depth, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(host_u64(allow), OG.pack_allow_bits(allow_ref))
+    assert np.array_equal(cand.cpu().numpy().view(np.uint32), cand_ref.view(np.uint32))      # bit-exact fp32
+    # in-place form (cand aliases logp) and the mask-only form give the same result
+    inplace = dev(logp)
+    api.grace_gtm_mask(inplace, dev(score), dev(node), dev(key), trie_s, matcher, inplace, None, B, M, depth, status)
+    assert np.array_equal(inplace.cpu().numpy().view(np.uint32), cand_ref.view(np.uint32))
+
+
+def test_gtm_mask_flags_nan_and_bad_node(api):
+    V, L = 64, 3
+    sids, trie, elig, node, key, score, logp = _mask_problem(3, V, L, 500, 1, 8, 1)
+    bits, base, _ = api.grace_trie_build_dense(sids, V)
+    trie_s = api.make_trie(dev(bits), dev(base), V, L, trie.num_nodes)
+    toks, _ = trie.lookup(int(node[0]))
+    logp[0, toks[0]] = np.nan
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    cand = torch.empty((8, V), device=DEV)
+    api.grace_gtm_mask(dev(logp), dev(score), dev(node), dev(key), trie_s, api.make_matcher(api.MATCH_NONE), cand,
+                       None, 1, 8, 1, status)
+    assert status.item() & api.DEV_NAN
+    status.zero_()
+    node2 = node.copy()
+    node2[3] = trie.num_nodes + 5
+    api.grace_gtm_mask(dev(synth.logp_rows(synth.rng_for(4, 9), 8, V)), dev(score), dev(node2), dev(key), trie_s,
+                       api.make_matcher(api.MATCH_NONE), cand, None, 1, 8, 1, status)
+    assert status.item() & api.DEV_BAD_INDEX
+    assert torch.isneginf(cand[3]).all()
+
+
+# ------------------------------------------------------------------------------------------
+# beam top-k
+# ------------------------------------------------------------------------------------------
+def _run_topk(api, cand: np.ndarray, K: int, V: int):
+    B, N = cand.shape
+    d_cand = dev(cand)
+    ws = torch.empty(api.grace_beam_topk_workspace_bytes(B, N, K), dtype=torch.uint8, device=DEV)
+    ws.fill_(0xAB)                                           # contents on entry must not matter
+    score = torch.empty((B, K), device=DEV)
+    flat = torch.empty((B, K), dtype=torch.int32, device=DEV)
+    parent = torch.empty_like(flat)
+    token = torch.empty_like(flat)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_beam_topk(d_cand, K, V, score, flat, parent, token, ws, status)
+    torch.cuda.synchronize()
+    return score.cpu().numpy(), flat.cpu().numpy(), parent.cpu().numpy(), token.cpu().numpy(), status.item()
+
+
+def _check_topk(api, cand, K, V, expect_exact_path=None):
+    s_ref, f_ref, p_ref, t_ref = OT.beam_topk(cand, K, V)
+    s, f, p, t, status = _run_topk(api, cand, K, V)
+    assert not (status & (api.DEV_NAN | api.DEV_BAD_INDEX))
+    assert np.array_equal(f, f_ref)
+    assert np.array_equal(s.view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(p, p_ref) and np.array_equal(t, t_ref)
+    if expect_exact_path is not None:
+        assert bool(status & api.DEV_TOPK_EXACT_PATH) == expect_exact_path
+    return status
+
+
+@pytest.mark.parametrize("B,M,V,K", [(1, 16, 64, 16), (3, 7, 192, 50), (2, 33, 1024, 2048), (1, 1, 64, 64)])
+def test_topk_small_shapes(api, B, M, V, K):
+    rng = synth.rng_for(4, 100 + M)
+    cand = synth.normal_f32(rng, (B, M * V), 3.0)
+    _check_topk(api, cand, K, V)
+    cand[rng.random(cand.shape) < 0.9] = -np.inf                # mostly masked: -inf takes part
+    _check_topk(api, cand, K, V)
+
+
+def test_topk_sampled_path_dense_and_masked(api):
+    """N large enough for the sampled-threshold path: dense scores, then masks of several densities."""
+    B, M, V, K = 3, 300, 1024, 2048
+    rng = synth.rng_for(4, 200)
+    logp = synth.logp_rows(rng, B * M, V)
+    score = np.concatenate([synth.descending_scores(rng, M, 2) for _ in range(B)])
+    cand = (score[:, None] + logp).astype(np.float32).reshape(B, M * V)
+    _check_topk(api, cand, K, V, expect_exact_path=False)
+    for density in (0.2, 0.01, 0.005):                          # 0.005 * 307200 = 1536 finite < K: underfull
+        masked = cand.copy()
+        masked[rng.random(cand.shape) >= density] = -np.inf
+        _check_topk(api, masked, K, V, expect_exact_path=False)
+    _check_topk(api, cand, 1, V)
+    _check_topk(api, cand, 4096, V)
+
+
+def test_topk_adversarial_inputs_take_the_exact_path_and_stay_exact(api):
+    B, N, V, K = 2, 300 * 1024, 1024, 2048
+    rng = synth.rng_for(4, 300)
+    same = np.full((B, N), -1.5, dtype=np.float32)              # all ties: lowest indices win
+    _check_topk(api, same, K, V, expect_exact_path=True)
+    ninf = np.full((B, N), -np.inf, dtype=np.float32)           # everything masked
+    _check_topk(api, ninf, K, V)
+    few = rng.integers(0, 7, size=(B, N)).astype(np.float32)    # 7 distinct values, huge tie groups
+    few[0, 5] = -0.0
+    _check_topk(api, few, K, V, expect_exact_path=True)
+    zeros = np.zeros((B, N), dtype=np.float32)
+    zeros[:, ::2] = -0.0                                        # -0.0 == +0.0
+    zeros[:, 1000:] = -1.0
+    _check_topk(api, zeros, K, V)
+    ramp = np.arange(N, dtype=np.float32)[None].repeat(B, 0)   # sorted ascending: sample is badly stratified
+    _check_topk(api, ramp, K, V)
+    _check_topk(api, -ramp, K, V)
+
+
+def test_topk_flags_nan(api):
+    cand = synth.normal_f32(synth.rng_for(4, 301), (1, 4096))
+    cand[0, 77] = np.nan
+    *_, status = _run_topk(api, cand, 16, 64)
+    assert status & api.DEV_NAN
+
+
+# ------------------------------------------------------------------------------------------
+# beam-state update
+# ------------------------------------------------------------------------------------------
+def test_beam_update_matches_oracle(api):
+    V, L, B, M, K = 1024, 4, 3, 40, 64
+    sids, trie, elig, node, key, score, logp = _mask_problem(11, V, L, 60000, B, M, 2)
+    bits, base, _ = api.grace_trie_build_dense(sids, V)
+    trie_s = api.make_trie(dev(bits), dev(base), V, L, trie.num_nodes)
+    cand, _, _ = OG.gtm_mask(logp, score, node, key, 2, trie, OG.NoMatcher(), B, M)
+    sc, flat, par, tok = OT.beam_topk(cand.reshape(B, M * V), K, V)       # includes -inf picks (underfull)
+    assert np.isneginf(sc).any() and np.isfinite(sc).any()
+    node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, node, key, 2, M)
+    new_node = torch.empty(B * K, dtype=torch.int32, device=DEV)
+    new_key = torch.empty(B * K, dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_beam_update(dev(par), dev(tok), dev(sc), dev(node), dev(key), trie_s, new_node, new_key, B, K, M, 2, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(new_node.cpu().numpy(), node_ref)
+    assert np.array_equal(host_u64(new_key), key_ref)
+
+
+# ------------------------------------------------------------------------------------------
+# self-attention
+# ------------------------------------------------------------------------------------------
+def _self_attn_problem(seed, B, beam_sizes, H, d, L):
+    rng = synth.rng_for(3, seed)
+    t = len(beam_sizes) - 1
+    R_max = B * max(beam_sizes)
+    kc = np.zeros((L, R_max, H, d), dtype=np.uint16)
+    vc = np.zeros((L, R_max, H, d), dtype=np.uint16)
+    parents = np.zeros((L, R_max), dtype=np.int32)
+    for j in range(t):
+        n = B * beam_sizes[j]
+        kc[j, :n] = synth.normal_bf16(rng, (n, H, d))
+        vc[j, :n] = synth.normal_bf16(rng, (n, H, d))
+    for j in range(1, t + 1):
+        parents[j, :B * beam_sizes[j]] = synth.uniform_parents(rng, B, beam_sizes[j - 1], beam_sizes[j])
+    qkv = synth.normal_bf16(rng, (B * beam_sizes[t], 3, H, d))
+    return qkv, kc, vc, parents
+
+
+@pytest.mark.parametrize("B,beam_sizes,H,d", [
+    (3, [1], 8, 64), (3, [1, 37], 8, 64), (2, [1, 50, 70], 8, 64), (2, [1, 64, 64, 130], 8, 64),
+    (2, [5, 64, 64, 64, 33], 8, 64), (1, [1, 16, 16], 4, 32), (2, [1, 20, 20, 20], 16, 64), (2, [1, 9, 9], 4, 128),
+    (1, [2, 3, 4, 5, 6, 7, 8, 9], 2, 64),
+])
+def test_self_attn_matches_oracle(api, B, beam_sizes, H, d):
+    L = max(5, len(beam_sizes))
+    t = len(beam_sizes) - 1
+    qkv, kc, vc, parents = _self_attn_problem(17 * t + H, B, beam_sizes, H, d, L)
+    scale = 1.0 / np.sqrt(d)
+    par_list = [None] + [parents[j] for j in range(1, t + 1)]
+    ref, kc_ref, vc_ref = OA.self_attn(f64(qkv), f64(kc), f64(vc), par_list, beam_sizes, t, B, scale)
+    d_kc, d_vc = dev_bf16(kc), dev_bf16(vc)
+    R = B * beam_sizes[t]
+    out = torch.zeros((R, H, d), dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_self_attn(dev_bf16(qkv), d_kc, d_vc, dev(parents), beam_sizes, out, B, t, scale, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert_attention_close(out.float().cpu().numpy(), ref, "self-attn out")
+    # cache write: slab t holds exactly the rows' k, v; everything else untouched (bit-exact)
+    kc_exp, vc_exp = kc.copy(), vc.copy()
+    kc_exp[t, :R], vc_exp[t, :R] = qkv[:, 1], qkv[:, 2]
+    assert np.array_equal(d_kc.view(torch.int16).cpu().numpy().view(np.uint16), kc_exp)
+    assert np.array_equal(d_vc.view(torch.int16).cpu().numpy().view(np.uint16), vc_exp)
+
+
+def test_self_attn_flags_bad_parent(api):
+    B, sizes, H, d = 1, [1, 8], 8, 64
+    qkv, kc, vc, parents = _self_attn_problem(5, B, sizes, H, d, 5)
+    parents[1, 3] = 99
+    out = torch.zeros((8, H, d), dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_self_attn(dev_bf16(qkv), dev_bf16(kc), dev_bf16(vc), dev(parents), sizes, out, B, 1, 0.125, status)
+    torch.cuda.synchronize()
+    assert status.item() & api.DEV_BAD_INDEX
+
+
+# ------------------------------------------------------------------------------------------
+# cross-attention
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,M,H,d,T", [
+    (1, 16, 4, 32, 64),            # config 1
+    (2, 5, 2, 64, 7),              # tiny, ragged
+    (2, 130, 8, 64, 128),          # tensor-core shape, ragged M tile
+    (3, 256, 8, 64, 512),          # config-2 slice
+    (2, 384, 4, 64, 1024),         # long encoder
+    (2, 70, 2, 64, 200),           # T not a multiple of the K/V block
+    (2, 33, 2, 128, 96),
+    (1, 1, 8, 64, 1024),           # step 0 of the decode loop: one row per request
+])
+def test_cross_attn_matches_oracle(api, B, M, H, d, T):
+    rng = synth.rng_for(2, B * 1000 + M + T)
+    q = synth.normal_bf16(rng, (B, M, H, d))
+    k = synth.normal_bf16(rng, (B, H, T, d))
+    v = synth.normal_bf16(rng, (B, H, T, d))
+    scale = 1.0 / np.sqrt(d)
+    ref, lse_ref = OA.cross_attn(f64(q), f64(k), f64(v), scale)
+    out = torch.zeros((B * M, H, d), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros((B * M, H), dtype=torch.float32, device=DEV)
+    api.grace_cross_attn(dev_bf16(q).reshape(B * M, H, d), dev_bf16(k), dev_bf16(v), out, scale, lse)
+    torch.cuda.synchronize()
+    assert_attention_close(out.float().cpu().numpy().reshape(B, M, H, d), ref, "cross-attn out")
+    np.testing.assert_allclose(lse.cpu().numpy().reshape(B, M, H), lse_ref, atol=2e-3, rtol=0)
+
+
+def test_cross_attn_strided_kv_layout(api):
+    """K/V stored [B, T, H, d] (projection output order) are read through strides."""
+    B, M, H, d, T = 2, 140, 8, 64, 256
+    rng = synth.rng_for(2, 77)
+    q = synth.normal_bf16(rng, (B, M, H, d))
+    k_bthd = synth.normal_bf16(rng, (B, T, H, d))
+    v_bthd = synth.normal_bf16(rng, (B, T, H, d))
+    scale = 0.125
+    ref, _ = OA.cross_attn(f64(q), f64(k_bthd).transpose(0, 2, 1, 3), f64(v_bthd).transpose(0, 2, 1, 3), scale)
+    out = torch.zeros((B * M, H, d), dtype=torch.bfloat16, device=DEV)
+    api.grace_cross_attn(dev_bf16(q).reshape(B * M, H, d), dev_bf16(k_bthd).permute(0, 2, 1, 3),
+                         dev_bf16(v_bthd).permute(0, 2, 1, 3), out, scale)
+    torch.cuda.synchronize()
+    assert_attention_close(out.float().cpu().numpy().reshape(B, M, H, d), ref, "cross-attn strided")
+
+
+# ------------------------------------------------------------------------------------------
+# decoder glue
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,N,K,relu,res,f32out", [
+    (16, 384, 128, False, False, False), (300, 512, 512, False, True, True), (257, 2048, 512, True, False, False),
+    (130, 64, 2048, False, True, True), (1, 1536, 512, False, False, False), (100, 80, 64, False, False, True),
+])
+def test_linear_matches_fp64_matmul(api, M, N, K, relu, res, f32out):
+    rng = synth.rng_for(5, M + N + K)
+    x = synth.normal_bf16(rng, (M, K))
+    w = synth.normal_bf16(rng, (N, K), 0.05)
+    r = synth.normal_f32(rng, (M, N)) if res else None
+    ref = f64(x) @ f64(w).T
+    if relu:
+        ref = np.maximum(ref, 0)
+    if res:
+        ref = ref + r
+    y = torch.zeros((M, N), dtype=torch.float32 if f32out else torch.bfloat16, device=DEV)
+    d_res = None
+    if res:
+        y.copy_(dev(r))                                           # residual aliases the output
+        d_res = y
+    api.grace_linear(dev_bf16(x), dev_bf16(w), y, d_res, relu)
+    torch.cuda.synchronize()
+    got = y.float().cpu().numpy().astype(np.float64)
+    tol = 2e-3 if f32out else 2e-2
+    assert np.abs(got - ref).max() <= tol * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
+
+
+def test_layer_norm_embed_log_softmax(api):
+    rng = synth.rng_for(5, 9)
+    R, D, V = 77, 512, 2048
+    x = synth.normal_f32(rng, (R, D), 2.0) + 0.5
+    g, b = synth.normal_f32(rng, D), synth.normal_f32(rng, D)
+    out = torch.zeros((R, D), dtype=torch.bfloat16, device=DEV)
+    api.grace_layer_norm(dev(x), dev(g), dev(b), out, 1e-5)
+    x64 = x.astype(np.float64)
+    ref = (x64 - x64.mean(1, keepdims=True)) / np.sqrt(x64.var(1, keepdims=True) + 1e-5) * g + b
+    assert np.abs(out.float().cpu().numpy() - ref).max() <= 2e-2 * max(1, np.abs(ref).max())
+    emb = synth.normal_bf16(rng, (V + 1, D))
+    pos = synth.normal_bf16(rng, (D,))
+    tok = rng.integers(0, V + 1, size=R).astype(np.int32)
+    xo = torch.zeros((R, D), device=DEV)
+    api.grace_embed(dev(tok), dev_bf16(emb), dev_bf16(pos), xo)
+    ref = synth.bf16_bits_to_f32(emb)[tok] + synth.bf16_bits_to_f32(pos)
+    assert np.array_equal(xo.cpu().numpy(), ref)
+    for Vv in (64, 1024, 2048, 4096):
+        z = synth.normal_f32(rng, (R, Vv), 3.0)
+        d_z = dev(z)
+        api.grace_log_softmax(d_z)
+        z64 = z.astype(np.float64)
+        ref = z64 - z64.max(1, keepdims=True)
+        ref = ref - np.log(np.exp(ref).sum(1, keepdims=True))
+        np.testing.assert_allclose(d_z.cpu().numpy(), ref, atol=2e-5, rtol=0)
