@@ -184,12 +184,16 @@ def grace_trie_walk(child_bits: np.ndarray, child_base: np.ndarray, V: int, L: i
 
 
 def make_trie(child_bits_dev, child_base_dev, V: int, L: int, num_nodes: int) -> TrieStruct:
-    return TrieStruct(V, L, num_nodes, child_bits_dev.shape[0], _dp(child_bits_dev), _dp(child_base_dev))
+    trie = TrieStruct(V, L, num_nodes, child_bits_dev.shape[0], _dp(child_bits_dev), _dp(child_base_dev))
+    trie._keepalive = (child_bits_dev, child_base_dev)      # the struct only holds raw pointers
+    return trie
 
 
 def make_matcher(kind: int, bits_dev=None, log2_bits: int = 0, n_hashes: int = 0) -> MatcherStruct:
     words = 0 if bits_dev is None else bits_dev.shape[-1]
-    return MatcherStruct(kind, log2_bits, n_hashes, 0, words, _dp(bits_dev))
+    matcher = MatcherStruct(kind, log2_bits, n_hashes, 0, words, _dp(bits_dev))
+    matcher._keepalive = bits_dev
+    return matcher
 
 
 # ----------------------------------------------------------------------------
