@@ -233,7 +233,8 @@ typedef struct {
   const uint16_t *w_oc;    /* [d_model][H*d_h] */
   const uint16_t *w_1;     /* [d_ffn][d_model] */
   const uint16_t *w_2;     /* [d_model][d_ffn] */
-  const uint16_t *k_cross, *v_cross;   /* [B][H][T_ctx][d_h], projected once per request */
+  const uint16_t *k_cross, *v_cross;   /* [B][T_ctx][H][d_h]: as the once-per-request projection
+                                          GEMM of the encoder output writes them (Section 3.2) */
   uint16_t *k_cache, *v_cache;         /* [L][R_max][H][d_h] */
 } grace_layer_t;
 
@@ -266,7 +267,8 @@ typedef struct {
   uint16_t *h;                /* [R_max][max(d_model, d_ffn)]                             */
   uint16_t *qkv;              /* [R_max][max(3*H*d_h, d_ffn)]: qkv, cross-q, FFN hidden     */
   uint16_t *attn;             /* [R_max][H*d_h]                                            */
-  float *logp;                /* [R_max][V]; also receives cand in place                  */
+  float *logp;                /* [R_max][V] log-probabilities                              */
+  float *cand;                /* [R_max][V] masked scores; may be the same buffer as logp  */
   void *topk_ws; size_t topk_ws_bytes;
   int32_t *d_status;
 } grace_decoder_t;

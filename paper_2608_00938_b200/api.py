@@ -59,7 +59,7 @@ class DecoderStruct(C.Structure):
         ("trie", TrieStruct), ("matcher", MatcherStruct),
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
-        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp),
+        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("cand", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]

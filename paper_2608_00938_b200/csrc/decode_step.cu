@@ -28,7 +28,7 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
       return GRACE_INVALID_ARG;
   }
   if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || !d->x || !d->h || !d->qkv ||
-      !d->attn || !d->logp || !d->topk_ws || !d->out_flat)
+      !d->attn || !d->logp || !d->cand || !d->topk_ws || !d->out_flat)
     return GRACE_INVALID_ARG;
   for (int i = 0; i < 2; ++i)
     if (!d->token[i] || !d->score[i] || !d->node[i] || !d->key[i]) return GRACE_INVALID_ARG;
@@ -64,9 +64,8 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
     // cross-attention block
     GRACE_TRY(grace_layer_norm(d->x, w.ln2_g, w.ln2_b, d->h, R, D, d->ln_eps, stream));
     GRACE_TRY(grace_linear(d->h, D, w.w_qc, D, d->qkv, nullptr, HD, nullptr, R, HD, D, 0, stream));
-    GRACE_TRY(grace_cross_attn(d->qkv, HD, w.k_cross, w.v_cross, (int64_t)d->H * d->T_ctx * d->d_h,
-                               (int64_t)d->T_ctx * d->d_h, d->d_h, d->attn, HD, nullptr, B, M, d->H, d->d_h,
-                               d->T_ctx, scale, st, stream));
+    GRACE_TRY(grace_cross_attn(d->qkv, HD, w.k_cross, w.v_cross, (int64_t)d->T_ctx * HD, d->d_h, HD, d->attn, HD,
+                               nullptr, B, M, d->H, d->d_h, d->T_ctx, scale, st, stream));
     GRACE_TRY(grace_linear(d->attn, HD, w.w_oc, HD, nullptr, d->x, D, d->x, R, D, HD, 0, stream));
     // feed-forward block
     GRACE_TRY(grace_layer_norm(d->x, w.ln3_g, w.ln3_b, d->h, R, D, d->ln_eps, stream));
@@ -76,12 +75,12 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   GRACE_TRY(grace_layer_norm(d->x, d->lnf_g, d->lnf_b, d->h, R, D, d->ln_eps, stream));
   GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
   GRACE_TRY(grace_log_softmax(d->logp, R, d->V, stream));
-  // CD + GTM mask and score add, in place over the log-probabilities
-  GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->logp,
+  // CD + GTM mask and score add (in place when cand == logp)
+  GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->cand,
                            nullptr, B, M, d->V, t, st, stream));
   // parents of step t+1 live in slab t+1; tokens become the next step's input tokens
   int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
-  GRACE_TRY(grace_beam_topk(d->logp, B, (int64_t)M * d->V, K, d->V, d->score[nxt], d->out_flat, parent_out,
+  GRACE_TRY(grace_beam_topk(d->cand, B, (int64_t)M * d->V, K, d->V, d->score[nxt], d->out_flat, parent_out,
                             d->token[nxt], d->topk_ws, d->topk_ws_bytes, st, stream));
   GRACE_TRY(grace_beam_update(parent_out, d->token[nxt], d->score[nxt], d->node[cur], d->key[cur], &d->trie,
                               d->node[nxt], d->key[nxt], B, K, M, t, st, stream));

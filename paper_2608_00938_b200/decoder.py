@@ -1,0 +1,146 @@
+"""Buffer set-up for grace_decode_step: uploads weights and index structures,
+allocates the caller-owned state / cache / activation buffers with torch and
+fills the C struct.  No arithmetic happens here; every step of the decode path
+runs in the library's kernels."""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+import torch
+
+from . import api
+
+
+def _bf16(a: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device).to(torch.bfloat16).contiguous()
+
+
+def _f32(a: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
+
+
+class Decoder:
+    """Owns the device buffers of one decode loop and the grace_decoder_t that points at them.
+
+    weights: dict as produced by `synth.decoder_weights` (fp32 arrays; matrices are rounded to
+    bf16 on upload).  beam_sizes: (M_0 .. M_{L-1}, K_final).  trie_bits / trie_base: host arrays
+    from `api.grace_trie_build_dense`.  matcher: (kind, host uint64 [B, words] or None,
+    log2_bits, n_hashes).
+    """
+
+    def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
+                 trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
+                 separate_cand=False):
+        assert len(beam_sizes) == L + 1
+        self.device = torch.device(device)
+        self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
+        self.d_model, self.d_ffn, self.n_layers = d_model, d_ffn, n_layers
+        self.beam_sizes = list(beam_sizes)
+        HD = n_heads * d_head
+        self.R_max = R_max = B * max(beam_sizes)
+        dev = self.device
+        self._keep = []
+        s = api.DecoderStruct()
+        s.B, s.n_layers, s.d_model, s.H, s.d_h, s.d_ffn, s.V, s.L, s.T_ctx = (
+            B, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx)
+        for i, m in enumerate(beam_sizes):
+            s.beam_sizes[i] = m
+        s.R_max = R_max
+        s.ln_eps = 1e-5
+        self.w_kc, self.w_vc, self.k_cross, self.v_cross, self.k_cache, self.v_cache = [], [], [], [], [], []
+        for li, lw in enumerate(weights["layers"]):
+            lay = s.layers[li]
+            for name in ("ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b"):
+                t = _f32(lw[name], dev); self._keep.append(t); setattr(lay, name, t.data_ptr())
+            for name in ("w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2"):
+                t = _bf16(lw[name], dev); self._keep.append(t); setattr(lay, name, t.data_ptr())
+            self.w_kc.append(_bf16(lw["w_kc"], dev))
+            self.w_vc.append(_bf16(lw["w_vc"], dev))
+            self.k_cross.append(torch.zeros((B, T_ctx, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+            self.v_cross.append(torch.zeros((B, T_ctx, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+            self.k_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+            self.v_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+            lay.k_cross, lay.v_cross = self.k_cross[li].data_ptr(), self.v_cross[li].data_ptr()
+            lay.k_cache, lay.v_cache = self.k_cache[li].data_ptr(), self.v_cache[li].data_ptr()
+        self.embed = _bf16(weights["embed"], dev)
+        self.pos = _bf16(weights["pos"], dev)
+        self.lnf_g, self.lnf_b = _f32(weights["lnf_g"], dev), _f32(weights["lnf_b"], dev)
+        self.w_out = _bf16(weights["w_out"], dev)
+        s.embed, s.pos, s.lnf_g, s.lnf_b, s.w_out = (self.embed.data_ptr(), self.pos.data_ptr(),
+                                                     self.lnf_g.data_ptr(), self.lnf_b.data_ptr(),
+                                                     self.w_out.data_ptr())
+        # index structures
+        self.trie_bits = torch.from_numpy(trie_bits.view(np.int64)).to(dev)
+        self.trie_base = torch.from_numpy(trie_base).to(dev)
+        self.trie = api.make_trie(self.trie_bits, self.trie_base, V, L, num_nodes)
+        kind, mbits, log2_bits, n_hashes = matcher
+        self.matcher_bits = None if mbits is None else torch.from_numpy(
+            np.ascontiguousarray(mbits).view(np.int64)).to(dev)
+        self.matcher = api.make_matcher(kind, self.matcher_bits, log2_bits, n_hashes)
+        s.trie, s.matcher = self.trie, self.matcher
+        # beam state
+        self.token = [torch.zeros(R_max, dtype=torch.int32, device=dev) for _ in range(2)]
+        self.score = [torch.zeros(R_max, dtype=torch.float32, device=dev) for _ in range(2)]
+        self.node = [torch.zeros(R_max, dtype=torch.int32, device=dev) for _ in range(2)]
+        self.key = [torch.zeros(R_max, dtype=torch.int64, device=dev) for _ in range(2)]
+        for i in range(2):
+            s.token[i], s.score[i] = self.token[i].data_ptr(), self.score[i].data_ptr()
+            s.node[i], s.key[i] = self.node[i].data_ptr(), self.key[i].data_ptr()
+        self.parents = torch.zeros((L + 1, R_max), dtype=torch.int32, device=dev)
+        self.out_flat = torch.zeros(R_max, dtype=torch.int32, device=dev)
+        s.parents, s.out_flat = self.parents.data_ptr(), self.out_flat.data_ptr()
+        # activations
+        self.x = torch.zeros((R_max, d_model), dtype=torch.float32, device=dev)
+        self.h = torch.zeros((R_max, max(d_model, d_ffn)), dtype=torch.bfloat16, device=dev)
+        self.qkv = torch.zeros((R_max, max(3 * HD, d_ffn)), dtype=torch.bfloat16, device=dev)
+        self.attn = torch.zeros((R_max, HD), dtype=torch.bfloat16, device=dev)
+        self.logp = torch.zeros((R_max, V), dtype=torch.float32, device=dev)
+        self.cand = torch.zeros((R_max, V), dtype=torch.float32, device=dev) if separate_cand else self.logp
+        max_n = max(beam_sizes[t] * V for t in range(L))
+        ws_bytes = api.grace_beam_topk_workspace_bytes(B, max_n, max(beam_sizes[1:]))
+        self.topk_ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+        self.d_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        s.x, s.h, s.qkv, s.attn, s.logp, s.cand = (self.x.data_ptr(), self.h.data_ptr(), self.qkv.data_ptr(),
+                                                   self.attn.data_ptr(), self.logp.data_ptr(), self.cand.data_ptr())
+        s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()
+        self.struct = s
+        code = api.grace_decoder_validate(s)
+        if code != api.GRACE_OK:
+            raise api.GraceError(code, "grace_decoder_validate")
+
+    # ---- once per request batch: cross-attention K/V from the encoder output (Section 3.2) ----
+    def project_cross_kv(self, enc: torch.Tensor) -> None:
+        """enc bf16 [B, T_ctx, d_enc] -> k_cross / v_cross [B, T_ctx, H, d_h] per layer."""
+        B, T, d_enc = enc.shape
+        x = enc.reshape(B * T, d_enc)
+        for li in range(self.n_layers):
+            api.grace_linear(x, self.w_kc[li], self.k_cross[li].view(B * T, -1))
+            api.grace_linear(x, self.w_vc[li], self.v_cross[li].view(B * T, -1))
+
+    def reset(self) -> None:
+        """Start state (Section 3.3: M_0 = 1): start token, score 0, root node, empty key."""
+        self.token[0][: self.B].fill_(self.V)
+        self.score[0][: self.B].zero_()
+        self.node[0][: self.B].zero_()
+        self.key[0][: self.B].zero_()
+        self.d_status.zero_()
+
+    def step(self, t: int) -> None:
+        api.grace_decode_step(self.struct, t)
+
+    def decode(self) -> None:
+        for t in range(self.L):
+            self.step(t)
+
+    def results(self):
+        """(sids int64 [B, K, L], score [B, K], node [B, K]) read back by following the parents."""
+        L, B, K = self.L, self.B, self.beam_sizes[-1]
+        fin = L & 1
+        score = self.score[fin][: B * K].view(B, K).cpu().numpy()
+        node = self.node[fin][: B * K].view(B, K).cpu().numpy()
+        key = self.key[fin][: B * K].view(B, K).cpu().numpy().view(np.uint64)
+        sids = np.zeros((B, K, L), dtype=np.int64)
+        for j in range(L):
+            sids[:, :, j] = ((key >> np.uint64(16 * j)) & np.uint64(0xFFFF)).astype(np.int64) - 1
+        return sids, score, node

@@ -1,0 +1,129 @@
+"""GPU parity of grace_decode_step against the oracle's constrained beam search
+(configuration 1: one request, beam 16, 2-layer decoder, 2,000-SID catalog,
+node-bitmask matcher), teacher-forced step by step, plus a free-running decode."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import decoder as OD
+from oracle import gtm as OG
+from oracle import matchers as OM
+from oracle import topk as OT
+from oracle.sid_trie import SidTrie
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import DEV, dev  # noqa: E402
+
+
+def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=2000, V=64, seed_variant=0,
+             std=0.02):
+    rng = synth.rng_for(1, seed_variant)
+    L = 3
+    sids = synth.catalog(rng, n_sids, V, L)
+    trie = SidTrie(sids, V)
+    elig = [synth.eligible_subset(rng, n_sids, 0.3) for _ in range(B)]
+    shp = synth.DecoderShape(2, 128, 4, 32, 512, 128, V, L)
+    w = synth.decoder_weights(rng, shp, std=std, as_bf16=True)
+    enc = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, 64, 128)))
+    return dict(sids=sids, trie=trie, elig=elig, shp=shp, w=w, enc=enc, schedule=schedule, final_k=final_k, B=B,
+                matcher_kind=matcher_kind)
+
+
+def _make_gpu_decoder(cfg, separate_cand=True):
+    from paper_2608_00938_b200 import api
+    from paper_2608_00938_b200.decoder import Decoder
+    shp, sids, trie = cfg["shp"], cfg["sids"], cfg["trie"]
+    bits, base, level_start = api.grace_trie_build_dense(sids, shp.V)
+    if cfg["matcher_kind"] == "node":
+        mb = np.stack([api.grace_node_bitmask_build(sids, shp.V, e, trie.num_nodes) for e in cfg["elig"]])
+        matcher = (api.MATCH_NODE_BITMASK, mb, 0, 0)
+    else:
+        mb = np.stack([api.grace_bloom_build(sids, shp.V, e, 14, 4) for e in cfg["elig"]])
+        matcher = (api.MATCH_PREFIX_BLOOM, mb, 14, 4)
+    dec = Decoder(n_layers=shp.n_layers, d_model=shp.d_model, n_heads=shp.n_heads, d_head=shp.d_head,
+                  d_ffn=shp.d_ffn, V=shp.V, L=shp.L, T_ctx=cfg["enc"].shape[1], B=cfg["B"],
+                  beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=cfg["w"], trie_bits=bits,
+                  trie_base=base, num_nodes=trie.num_nodes, matcher=matcher, device=DEV, separate_cand=separate_cand)
+    dec.project_cross_kv(torch.from_numpy(cfg["enc"]).to(DEV).to(torch.bfloat16))
+    return dec, api
+
+
+def _oracle_matcher(cfg):
+    sids, trie = cfg["sids"], cfg["trie"]
+    if cfg["matcher_kind"] == "node":
+        return OG.NodeBitmaskMatcher(np.stack([OM.node_eligibility(trie, sids, e) for e in cfg["elig"]]))
+    return OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 14, 4) for e in cfg["elig"]])
+
+
+@pytest.mark.parametrize("B,kind,schedule,final_k", [
+    (1, "node", (1, 16, 16), 16),            # configuration 1
+    (3, "bloom", (1, 40, 24), 32),           # several requests, dynamic per-step beam sizes, Bloom matcher
+])
+def test_decode_step_teacher_forced(B, kind, schedule, final_k):
+    cfg = _config1(B=B, matcher_kind=kind, schedule=schedule, final_k=final_k)
+    shp, trie = cfg["shp"], cfg["trie"]
+    record = []
+    OD.beam_search(cfg["w"], shp, cfg["enc"], trie, _oracle_matcher(cfg), schedule, final_k, record=record)
+    dec, api = _make_gpu_decoder(cfg)
+    dec.reset()
+    V, L = shp.V, shp.L
+    sizes = list(schedule) + [final_k]
+    for t in range(L):
+        step = record[t]
+        M, K = sizes[t], sizes[t + 1]
+        R = B * M
+        cur, nxt = t & 1, (t + 1) & 1
+        # teacher forcing: the step starts from the oracle's beam state (caches come from the GPU's own
+        # earlier steps, which ran on the same tokens and parents)
+        dec.token[cur][:R].copy_(dev(step["tokens"].astype(np.int32)))
+        dec.score[cur][:R].copy_(dev(step["score"]))
+        dec.node[cur][:R].copy_(dev(step["node"]))
+        dec.key[cur][:R].copy_(dev(step["key"]))
+        if t > 0:
+            dec.parents[t, :R].copy_(dev(record[t - 1]["out_parent"].reshape(-1)))
+        dec.step(t)
+        torch.cuda.synchronize()
+        assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+        # log-probabilities: bf16 pipeline vs the fp64 oracle on the same bf16-valued weights
+        logp = dec.logp[:R].cpu().numpy()
+        assert np.abs(logp - step["logp"]).max() <= 2e-2
+        np.testing.assert_allclose(np.exp(logp.astype(np.float64)).sum(1), 1.0, atol=1e-4)
+        # the mask is an integer decision on exact inputs: identical to the oracle's
+        cand = dec.cand[:R].cpu().numpy()
+        assert np.array_equal(np.isfinite(cand), step["allow"])
+        assert np.array_equal(cand[step["allow"]], (step["score"][:, None] + logp)[step["allow"]])
+        # selection and state update: exact against the oracle run on the GPU's own candidates
+        sc, flat, par, tok = OT.beam_topk(cand.reshape(B, M * V), K, V)
+        assert np.array_equal(dec.out_flat[:B * K].cpu().numpy().reshape(B, K), flat)
+        assert np.array_equal(dec.score[nxt][:B * K].cpu().numpy().view(np.uint32).reshape(B, K), sc.view(np.uint32))
+        assert np.array_equal(dec.parents[t + 1, :B * K].cpu().numpy().reshape(B, K), par)
+        assert np.array_equal(dec.token[nxt][:B * K].cpu().numpy().reshape(B, K), tok)
+        node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, step["node"], step["key"], t, M)
+        assert np.array_equal(dec.node[nxt][:B * K].cpu().numpy(), node_ref)
+        assert np.array_equal(dec.key[nxt][:B * K].cpu().numpy().view(np.uint64), key_ref)
+
+
+def test_free_running_decode_emits_only_eligible_catalog_sids():
+    """Wide beams on a small catalog: the search is exhaustive, so GPU and oracle must return the same
+    set of SIDs; every emitted SID is in the catalog and passes the matcher at every prefix."""
+    cfg = _config1(B=2, matcher_kind="node", schedule=(1, 64, 64), final_k=64, n_sids=60, std=0.3)
+    shp, trie, sids = cfg["shp"], cfg["trie"], cfg["sids"]
+    out = OD.beam_search(cfg["w"], shp, cfg["enc"], trie, _oracle_matcher(cfg), cfg["schedule"], cfg["final_k"])
+    dec, api = _make_gpu_decoder(cfg, separate_cand=False)
+    dec.reset()
+    dec.decode()
+    torch.cuda.synchronize()
+    assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+    g_sids, g_score, g_node = dec.results()
+    for b in range(cfg["B"]):
+        good = {tuple(s) for s, e in zip(sids.tolist(), cfg["elig"][b]) if e}
+        valid = np.isfinite(g_score[b])
+        got = [tuple(s) for s in g_sids[b][valid].tolist()]
+        want = [tuple(s) for s in out["sids"][b][out["valid"][b]].tolist()]
+        assert set(got) == set(want) == good
+        assert all(trie.walk(s) == n for s, n in zip(got, g_node[b][valid]))
+        assert (g_score[b][1:] <= g_score[b][:-1]).all()
+        # weights of std 0.3 give scores down to -35: bf16 activations carry ~1% of that
+        np.testing.assert_allclose(np.sort(g_score[b][valid]), np.sort(out["score"][b][out["valid"][b]]), atol=3e-2, rtol=2e-2)
