@@ -1,0 +1,518 @@
+#!/usr/bin/env python
+"""Benchmark of the GTM-constrained decode loop on B200.
+
+One bench "step" is one full pass of the hot path over one batch: the 4-step constrained beam
+search of the serving-scale configuration (32 requests x beam 2048, 4-layer decoder, codebook
+2048, catalog of 1M SIDs, per-request Bloom matcher).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-ops]
+
+N > 1 is launched with torch.distributed.run; every rank decodes its own 32 requests (weak
+scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+CFG5 = dict(name="cfg5_full_decoder_step", B=32, schedule=(1, 2048, 2048, 2048), final_k=2048, n_layers=4,
+            d_model=512, H=8, d_h=64, d_ffn=2048, d_enc=512, T_ctx=1024, V=2048, L=4, n_sids=1_000_000,
+            elig_frac=0.2, bloom_log2=22, bloom_hashes=4)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p["bf16_tflops_sustained"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# inputs (seeded, synthetic; shapes of the paper's serving workload)
+# ------------------------------------------------------------------------------------------------
+def make_inputs(cfg, variant=0):
+    rng = synth.rng_for(5, variant)
+    sids = synth.catalog(rng, cfg["n_sids"], cfg["V"], cfg["L"])
+    elig = [synth.eligible_subset(rng, cfg["n_sids"], cfg["elig_frac"]) for _ in range(cfg["B"])]
+    shp = synth.DecoderShape(cfg["n_layers"], cfg["d_model"], cfg["H"], cfg["d_h"], cfg["d_ffn"], cfg["d_enc"],
+                             cfg["V"], cfg["L"])
+    weights = synth.decoder_weights(rng, shp, as_bf16=True)
+    enc_bits = synth.normal_bf16(rng, (cfg["B"], cfg["T_ctx"], cfg["d_enc"]))
+    return dict(sids=sids, elig=elig, shp=shp, weights=weights, enc_bits=enc_bits)
+
+
+def build_decoder(cfg, inp, device):
+    from paper_2608_00938_b200 import api
+    from paper_2608_00938_b200.decoder import Decoder
+    bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
+    num_nodes = int(level_start[-1])
+    blooms = np.stack([api.grace_bloom_build(inp["sids"], cfg["V"], e, cfg["bloom_log2"], cfg["bloom_hashes"])
+                       for e in inp["elig"]])
+    dec = Decoder(n_layers=cfg["n_layers"], d_model=cfg["d_model"], n_heads=cfg["H"], d_head=cfg["d_h"],
+                  d_ffn=cfg["d_ffn"], V=cfg["V"], L=cfg["L"], T_ctx=cfg["T_ctx"], B=cfg["B"],
+                  beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=inp["weights"], trie_bits=bits,
+                  trie_base=base, num_nodes=num_nodes,
+                  matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device)
+    return dec
+
+
+def beam_steps(cfg):
+    return cfg["B"] * sum(cfg["schedule"])
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampler
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, power, reasons = [], [], [], set()
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w_max=max(power), samples=len(sm),
+                    reasons=sorted(reasons))
+
+
+# ------------------------------------------------------------------------------------------------
+# timing of the decode loop
+# ------------------------------------------------------------------------------------------------
+def time_decode(dec, steps, warmup, dist=None):
+    import torch
+    from paper_2608_00938_b200 import api
+    L = dec.L
+    for _ in range(warmup):
+        dec.reset(); dec.decode()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 1)] for _ in range(steps)]
+    launches0 = api.grace_kernel_launch_count()
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for it in range(steps):
+        dec.reset()
+        ev[it][0].record()
+        for t in range(L):
+            dec.step(t)
+            ev[it][t + 1].record()
+    t_end.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    launches = api.grace_kernel_launch_count() - launches0
+    total_ms = t_begin.elapsed_time(t_end)
+    per_step_us = [statistics.mean(ev[it][t].elapsed_time(ev[it][t + 1]) for it in range(steps)) * 1e3
+                   for t in range(L)]
+    return total_ms / steps, per_step_us, launches
+
+
+def time_e2e(dec, enc_bits, steps, warmup):
+    """Same loop through the public API starting from HOST memory: pinned encoder output -> device, cross-K/V
+    projection, 4 decode steps, results (scores, keys, nodes) -> host."""
+    import torch
+    B, K = dec.B, dec.beam_sizes[-1]
+    enc_host = torch.from_numpy(enc_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    enc_dev = torch.empty_like(enc_host, device=dec.device)
+    fin = dec.L & 1
+    out_score = torch.empty((B * K,), dtype=torch.float32).pin_memory()
+    out_key = torch.empty((B * K,), dtype=torch.int64).pin_memory()
+    out_node = torch.empty((B * K,), dtype=torch.int32).pin_memory()
+
+    def one():
+        enc_dev.copy_(enc_host, non_blocking=True)
+        dec.project_cross_kv(enc_dev)
+        dec.reset(); dec.decode()
+        out_score.copy_(dec.score[fin][:B * K], non_blocking=True)
+        out_key.copy_(dec.key[fin][:B * K], non_blocking=True)
+        out_node.copy_(dec.node[fin][:B * K], non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        one()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(steps):
+        one()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    h2d = enc_host.numel() * 2
+    d2h = out_score.numel() * 4 + out_key.numel() * 8 + out_node.numel() * 4
+    return ms, h2d, d2h
+
+
+# ------------------------------------------------------------------------------------------------
+# per-op breakdown of one decode loop (same C-ABI ops, same order, events around each)
+# ------------------------------------------------------------------------------------------------
+def op_breakdown(dec, cfg, reps=3):
+    import torch
+    from paper_2608_00938_b200 import api
+    D, HD, F, V, H, dh = cfg["d_model"], cfg["H"] * cfg["d_h"], cfg["d_ffn"], cfg["V"], cfg["H"], cfg["d_h"]
+    B, L = cfg["B"], cfg["L"]
+    sizes = list(cfg["schedule"]) + [cfg["final_k"]]
+    scale = 1.0 / np.sqrt(dh)
+    times, flops, counts = {}, {}, {}
+    pending = []
+
+    def timed(name, fn, fl=0.0):
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        pending.append((name, a, b))
+        flops[name] = flops.get(name, 0.0) + fl
+        counts[name] = counts.get(name, 0) + 1
+
+    s = dec.struct
+    for _ in range(reps):
+        dec.reset()
+        for t in range(L):
+            M, K = sizes[t], sizes[t + 1]
+            R = B * M
+            cur, nxt = t & 1, (t + 1) & 1
+            x, h, qkv, attn = dec.x[:R], dec.h, dec.qkv, dec.attn[:R]
+            hD = h.view(-1)[:R * D].view(R, D)
+            timed("embed", lambda: api.grace_embed(dec.token[cur][:R], dec.embed, dec.pos[t], x, dec.d_status))
+            for li in range(cfg["n_layers"]):
+                lay = dec._layer_tensors[li]
+                q3 = qkv.view(-1)[:R * 3 * HD].view(R, 3 * HD)
+                q1 = qkv.view(-1)[:R * HD].view(R, HD)
+                ff = qkv.view(-1)[:R * F].view(R, F)
+                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln1_g"], lay["ln1_b"], hD))
+                timed("linear", lambda: api.grace_linear(hD, lay["w_qkv"], q3), 2.0 * R * D * 3 * HD)
+                timed("self_attn", lambda: api.grace_self_attn(q3.view(R, 3, H, dh), dec.k_cache[li], dec.v_cache[li],
+                                                               dec.parents, sizes, attn.view(R, H, dh), B, t, scale,
+                                                               dec.d_status))
+                timed("linear", lambda: api.grace_linear(attn, lay["w_o"], x, x), 2.0 * R * HD * D)
+                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln2_g"], lay["ln2_b"], hD))
+                timed("linear", lambda: api.grace_linear(hD, lay["w_qc"], q1), 2.0 * R * D * HD)
+                timed("cross_attn", lambda: api.grace_cross_attn(
+                    q1.view(R, H, dh), dec.k_cross[li].permute(0, 2, 1, 3), dec.v_cross[li].permute(0, 2, 1, 3),
+                    attn.view(R, H, dh), scale), 4.0 * R * H * dh * cfg["T_ctx"])
+                timed("linear", lambda: api.grace_linear(attn, lay["w_oc"], x, x), 2.0 * R * HD * D)
+                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln3_g"], lay["ln3_b"], hD))
+                timed("linear", lambda: api.grace_linear(hD, lay["w_1"], ff, None, True), 2.0 * R * D * F)
+                timed("linear", lambda: api.grace_linear(ff, lay["w_2"], x, x), 2.0 * R * F * D)
+            timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
+            logp = dec.logp[:R]
+            timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
+            timed("log_softmax", lambda: api.grace_log_softmax(logp))
+            timed("gtm_mask", lambda: api.grace_gtm_mask(logp, dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R],
+                                                         dec.trie, dec.matcher, logp, None, B, M, t, dec.d_status))
+            par = dec.parents[t + 1]
+            timed("beam_topk", lambda: api.grace_beam_topk(logp.view(B, M * V), K, V, dec.score[nxt][:B * K].view(B, K),
+                                                           dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K),
+                                                           dec.token[nxt][:B * K].view(B, K), dec.topk_ws, dec.d_status))
+            timed("beam_update", lambda: api.grace_beam_update(par[:B * K], dec.token[nxt][:B * K], dec.score[nxt][:B * K],
+                                                               dec.node[cur][:R], dec.key[cur][:R], dec.trie,
+                                                               dec.node[nxt][:B * K], dec.key[nxt][:B * K], B, K, M, t,
+                                                               dec.d_status))
+    torch.cuda.synchronize()
+    for name, a, b in pending:
+        times[name] = times.get(name, 0.0) + a.elapsed_time(b)
+    total = sum(times.values())
+    return {name: dict(ms_per_loop=times[name] / reps, share=times[name] / total, calls_per_loop=counts[name] // reps,
+                       flops_per_loop=flops[name] / reps) for name in times}
+
+
+# ------------------------------------------------------------------------------------------------
+# op-level rooflines at the per-op benchmark configurations
+# ------------------------------------------------------------------------------------------------
+def _time_op(fn, n_sets, iters=30, warm=5):
+    import torch
+    for i in range(warm):
+        fn(i % n_sets)
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(iters):
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(); fn(i % n_sets); b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    ts = sorted(a.elapsed_time(b) for a, b in evs)
+    return ts[len(ts) // 2] * 1e3, ts[min(len(ts) - 1, int(len(ts) * 0.99))] * 1e3    # P50, P99 in us
+
+
+def op_rooflines(device, peaks):
+    import torch
+    from paper_2608_00938_b200 import api
+    out = {}
+    g = torch.Generator(device=device); g.manual_seed(synth.seed_for(2))
+    rnd = lambda *shape: torch.randn(*shape, device=device, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    # ---- cross-attention, configuration 2 sweep: 3 rotating buffer sets keep L2 cold ----
+    for B, M, T in ((64, 256, 512), (64, 1024, 512), (64, 256, 1024), (64, 1024, 1024), (32, 2048, 1024)):
+        H, d = 8, 64
+        sets = [(rnd(B * M, H, d), rnd(B, H, T, d), rnd(B, H, T, d), torch.empty(B * M, H, d, device=device, dtype=torch.bfloat16))
+                for _ in range(3)]
+        p50, p99 = _time_op(lambda i: api.grace_cross_attn(sets[i][0], sets[i][1], sets[i][2], sets[i][3], 0.125), 3)
+        nbytes = 2 * (2 * B * M * H * d + 2 * B * H * T * d)
+        flops = 4.0 * B * M * H * d * T
+        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+        t_tc = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
+        bound = "hbm" if t_hbm >= t_tc else "tensor"
+        out[f"cross_attn_B{B}_M{M}_T{T}"] = dict(
+            p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, tflops=flops / p50 / 1e6, bound=bound,
+            frac=max(t_hbm, t_tc) / p50, frac_hbm=t_hbm / p50, frac_tensor=t_tc / p50)
+        del sets
+    # ---- self-attention, configuration 3: T_self = 1..5 ----
+    B, M, H, d, Lc = 32, 2048, 8, 64, 5
+    R = B * M
+    kc, vc = rnd(Lc, R, H, d), rnd(Lc, R, H, d)
+    parents = torch.randint(0, M, (Lc, R), device=device, dtype=torch.int32, generator=g)
+    qkv = rnd(R, 3, H, d)
+    o = torch.empty(R, H, d, device=device, dtype=torch.bfloat16)
+    for t in range(5):
+        sizes = [M] * (t + 1)
+        p50, p99 = _time_op(lambda i: api.grace_self_attn(qkv, kc, vc, parents, sizes, o, B, t, 0.125), 1)
+        logical = R * 1024 * (6 + 2 * t)                       # q,k,v read 3 KB + k,v write 2 KB + out 1 KB + 2 KB/ancestor
+        out[f"self_attn_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, gbs=logical / p50 / 1e3, bound="hbm",
+                                          frac=logical / p50 / 1e3 / peaks["hbm_gbs"])
+    del kc, vc, qkv, o
+    # ---- top-k alone, configuration 4 (dense, all finite: worst case) ----
+    B, M, V, K = 32, 2048, 1024, 2048
+    cands = [torch.randn(B, M * V, device=device, generator=g) * 3.0 - 8.0 for _ in range(2)]
+    ws = torch.empty(api.grace_beam_topk_workspace_bytes(B, M * V, K), dtype=torch.uint8, device=device)
+    sc = torch.empty(B, K, device=device); fl = torch.empty(B, K, device=device, dtype=torch.int32)
+    pa, tk = torch.empty_like(fl), torch.empty_like(fl)
+    st = torch.zeros(1, device=device, dtype=torch.int32)
+    p50, p99 = _time_op(lambda i: api.grace_beam_topk(cands[i], K, V, sc, fl, pa, tk, ws, st), 2)
+    nbytes = B * M * V * 4
+    out["beam_topk_dense_B32_N2M_K2048"] = dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm",
+                                               frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"],
+                                               exact_path_used=bool(st.item() & api.DEV_TOPK_EXACT_PATH))
+    return out
+
+
+def mask_roofline(dec, cfg, peaks):
+    """CD+GTM mask alone at the first full-width level (depth 1: dense rows), on the bench decoder's own state."""
+    import torch
+    from paper_2608_00938_b200 import api
+    B, M, V = cfg["B"], cfg["schedule"][1], cfg["V"]
+    R = B * M
+    dec.reset(); dec.step(0)                                   # state [1] now holds the level-1 beams
+    logp = torch.log_softmax(torch.randn(R, V, device=dec.device) * 3.0, dim=1)
+    cand = torch.empty_like(logp)
+    p50, p99 = _time_op(lambda i: api.grace_gtm_mask(logp, dec.score[1][:R], dec.node[1][:R], dec.key[1][:R], dec.trie,
+                                                     dec.matcher, cand, None, B, M, 1, dec.d_status), 1)
+    live = int((dec.node[1][:R] >= 0).sum().item())
+    nbytes = 2 * R * V * 4
+    return dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm", frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"],
+                live_rows=live, rows=R, matcher="prefix_bloom", note="dense-form bytes: 4 B in + 4 B out per candidate")
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, inp, beam, request=0):
+    """One request of the workload decoded by the oracle with beam `beam`; returns (seconds, beam-steps)."""
+    from oracle import decoder as OD
+    from oracle import gtm as OG
+    from oracle import matchers as OM
+    from oracle.sid_trie import SidTrie
+    trie = oracle_sample.trie if getattr(oracle_sample, "trie", None) is not None else SidTrie(inp["sids"], cfg["V"])
+    oracle_sample.trie = trie
+    bloom = OM.build_prefix_bloom(inp["sids"], inp["elig"][request], cfg["bloom_log2"], cfg["bloom_hashes"])
+    enc = synth.bf16_bits_to_f32(inp["enc_bits"][request:request + 1])
+    schedule = (1,) + (beam,) * (cfg["L"] - 1)
+    t0 = time.perf_counter()
+    OD.beam_search(inp["weights"], inp["shp"], enc, trie, OG.PrefixBloomMatcher([bloom]), schedule, beam)
+    return time.perf_counter() - t0, sum(schedule)
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    cfg = dict(CFG5)
+    inp = make_inputs(cfg, 0)
+    beam = 2048 if (args.steps + args.warmup) <= 16 else 512     # keep the whole run within a few minutes
+    for _ in range(args.warmup):
+        oracle_sample(cfg, inp, beam)
+    secs, units = 0.0, 0
+    for _ in range(args.steps):
+        s, u = oracle_sample(cfg, inp, beam)
+        secs += s; units += u
+    value = units / secs
+    sample = f"1 of {cfg['B']} requests, beam schedule (1,{beam},{beam},{beam}), all 4 steps, per bench step"
+    line = dict(impl="reference", metric="beam_steps_per_s", value=value, unit="beam-steps/s", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=secs / args.steps * 1e3, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=cfg["name"], B=cfg["B"], schedule=list(cfg["schedule"]), V=cfg["V"], L=cfg["L"],
+                            n_layers=cfg["n_layers"], d_model=cfg["d_model"], T_ctx=cfg["T_ctx"]),
+                cpu_baseline=dict(value=value, unit="beam-steps/s", cores=cpu_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit="beam-steps/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-ops", action="store_true", help="skip the per-op roofline microbenchmarks")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_00938_b200 import api  # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    dgroup = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+        dgroup = dist
+    peaks = load_peaks()
+    cfg = dict(CFG5)
+    inp = make_inputs(cfg, variant=rank)
+    dec = build_decoder(cfg, inp, device)
+    dec._layer_tensors = _layer_tensor_views(dec, inp)
+    enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
+    dec.project_cross_kv(enc_dev)
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms_loop, per_step_us, launches = time_decode(dec, args.steps, args.warmup, dgroup)
+    clocks = sampler.stop()
+    status = int(dec.d_status.item())
+    if world > 1:
+        tmax = torch.tensor([ms_loop], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_loop = float(tmax.item())
+    units = beam_steps(cfg) * world
+    value = units / (ms_loop * 1e-3)
+
+    e2e_ms, h2d, d2h = time_e2e(dec, inp["enc_bits"], max(3, args.steps // 2), 3)
+    if world > 1:
+        tmax = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+
+    line = dict(metric="beam_steps_per_s", value=value, unit="beam-steps/s", n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms_loop, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload=cfg["name"], B=cfg["B"], schedule=list(cfg["schedule"]), final_k=cfg["final_k"],
+                            n_layers=cfg["n_layers"], d_model=cfg["d_model"], H=cfg["H"], d_h=cfg["d_h"],
+                            d_ffn=cfg["d_ffn"], T_ctx=cfg["T_ctx"], V=cfg["V"], L=cfg["L"], catalog_sids=cfg["n_sids"],
+                            matcher="prefix_bloom_2^22x4", parallelism=f"requests sharded x{world}",
+                            l2="working set ~5 GB per loop, far larger than the 126 MB L2"),
+                step_latency_us=per_step_us, clocks=clocks, gpu_launches=int(launches), device_status=status,
+                e2e=dict(value=units / (e2e_ms * 1e-3), unit="beam-steps/s", ms_per_step=e2e_ms,
+                         h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                         includes="pinned encoder output H2D, cross-K/V projection, 4 decode steps, results D2H"))
+
+    if rank == 0:
+        bd = op_breakdown(dec, cfg)
+        line["op_breakdown"] = bd
+        top = max(bd, key=lambda k: bd[k]["ms_per_loop"])
+        if top in ("linear", "cross_attn"):
+            ach = bd[top]["flops_per_loop"] / (bd[top]["ms_per_loop"] * 1e-3) / 1e12
+            peak = peaks["bf16_tflops_sustained"]
+            line["roofline"] = dict(kernel=top, bound="tensor", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
+                                    traffic=None, peak_source=f"{peaks['source']} (sustained)",
+                                    launches_per_loop=bd[top]["calls_per_loop"])
+        else:
+            line["roofline"] = dict(kernel=top, bound="hbm", achieved=None, peak=peaks["hbm_gbs"], unit="GB/s", frac=None,
+                                    traffic=None, peak_source=peaks["source"])
+        if not args.no_ops and world == 1:
+            ops = op_rooflines(device, peaks)
+            ops["gtm_mask_depth1_B32_M2048_V2048"] = mask_roofline(dec, cfg, peaks)
+            line["op_rooflines"] = ops
+        if not args.no_cpu and world == 1:
+            secs, units_cpu = oracle_sample(cfg, inp, 2048)
+            line["cpu_baseline"] = dict(value=units_cpu / secs, unit="beam-steps/s", cores=cpu_threads(), kind="oracle",
+                                        seconds=secs,
+                                        sample=f"1 of {cfg['B']} requests, full schedule (1,2048,2048,2048), all 4 steps")
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def _layer_tensor_views(dec, inp):
+    """Per-layer weight tensors for the op-breakdown pass (the decode path itself only sees raw pointers)."""
+    import torch
+    from paper_2608_00938_b200.decoder import _bf16, _f32
+    out = []
+    for lw in inp["weights"]["layers"]:
+        d = {}
+        for name in ("ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b"):
+            d[name] = _f32(lw[name], dec.device)
+        for name in ("w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2"):
+            d[name] = _bf16(lw[name], dec.device)
+        out.append(d)
+    return out
+
+
+if __name__ == "__main__":
+    main()

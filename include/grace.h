@@ -51,6 +51,8 @@ const char* grace_status_string(grace_status_t s);
 /* Library version, and the compute capability the kernels were built for (100 = sm_100a). */
 int grace_version(void);
 int grace_built_for_sm(void);
+/* Number of kernels this library has launched in this process so far (all entry points). */
+uint64_t grace_kernel_launch_count(void);
 
 /* ------------------------------------------------------------------------------------------
  * Index structures (Section 4.4, Appendix A).
@@ -275,6 +277,10 @@ typedef struct {
 
 /* Host-only consistency check of a decoder struct (null pointers, shape limits). */
 grace_status_t grace_decoder_validate(const grace_decoder_t* dec);
+
+/* Start state of a decode loop (Section 3.3: M_0 = 1): for each of the B requests, input token =
+ * start token (V), score 0, node = root, key 0, written to state buffers [0]; *d_status = 0. */
+grace_status_t grace_decode_begin(const grace_decoder_t* dec, void* stream);
 
 /* Step t (0-based) of the decode loop (Sections 3.1-3.3): embed the rows' input tokens, run the
  * decoder layers (self-attention with cache write, cross-attention, feed-forward), logits,

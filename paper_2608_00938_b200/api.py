@@ -96,6 +96,8 @@ _embed = _sig("grace_embed", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _vp, _
 _log_softmax = _sig("grace_log_softmax", _i32, [_vp, _i32, _i32, _vp])
 _decoder_validate = _sig("grace_decoder_validate", _i32, [C.POINTER(DecoderStruct)])
 _decode_step = _sig("grace_decode_step", _i32, [C.POINTER(DecoderStruct), _i32, _vp])
+_decode_begin = _sig("grace_decode_begin", _i32, [C.POINTER(DecoderStruct), _vp])
+_launch_count = _sig("grace_kernel_launch_count", C.c_uint64, [])
 
 
 class GraceError(RuntimeError):
@@ -280,6 +282,14 @@ def grace_log_softmax(logits):
 
 def grace_decoder_validate(dec: DecoderStruct) -> int:
     return _decoder_validate(C.byref(dec))
+
+
+def grace_kernel_launch_count() -> int:
+    return int(_launch_count())
+
+
+def grace_decode_begin(dec: DecoderStruct):
+    _check(_decode_begin(C.byref(dec), _stream()), "grace_decode_begin")
 
 
 def grace_decode_step(dec: DecoderStruct, t: int):

@@ -14,8 +14,11 @@
     if (_e != cudaSuccess) return GRACE_CUDA_ERROR;           \
   } while (0)
 
+// Follows every kernel launch: counts it (grace_kernel_launch_count) and checks the launch.
+extern unsigned long long g_grace_launches;
 #define GRACE_LAUNCH_CHECK()                                  \
   do {                                                        \
+    __atomic_fetch_add(&g_grace_launches, 1ull, __ATOMIC_RELAXED); \
     if (cudaGetLastError() != cudaSuccess) return GRACE_CUDA_ERROR; \
   } while (0)
 

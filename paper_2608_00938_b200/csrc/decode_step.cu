@@ -36,6 +36,25 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
   return GRACE_OK;
 }
 
+namespace grace {
+__global__ void decode_begin_kernel(int32_t* token, float* score, int32_t* node, uint64_t* key, int32_t* d_status,
+                                    int rows, int start_token) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < rows) { token[i] = start_token; score[i] = 0.f; node[i] = 0; key[i] = 0ull; }
+  if (i == 0 && d_status != nullptr) *d_status = 0;
+}
+}  // namespace grace
+
+extern "C" grace_status_t grace_decode_begin(const grace_decoder_t* d, void* stream) {
+  grace_status_t st = grace_decoder_validate(d);
+  if (st != GRACE_OK) return st;
+  const int rows = d->B * d->beam_sizes[0];
+  grace::decode_begin_kernel<<<(rows + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
+      d->token[0], d->score[0], d->node[0], d->key[0], d->d_status, rows, d->V);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
 #define GRACE_TRY(expr)                         \
   do {                                          \
     grace_status_t _s = (expr);                 \

@@ -161,5 +161,7 @@ extern "C" const char* grace_status_string(grace_status_t s) {
   return "unknown";
 }
 
+unsigned long long g_grace_launches = 0;
+extern "C" uint64_t grace_kernel_launch_count(void) { return __atomic_load_n(&g_grace_launches, __ATOMIC_RELAXED); }
 extern "C" int grace_version(void) { return 1; }
 extern "C" int grace_built_for_sm(void) { return 100; }

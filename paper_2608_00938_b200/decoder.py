@@ -120,11 +120,7 @@ class Decoder:
 
     def reset(self) -> None:
         """Start state (Section 3.3: M_0 = 1): start token, score 0, root node, empty key."""
-        self.token[0][: self.B].fill_(self.V)
-        self.score[0][: self.B].zero_()
-        self.node[0][: self.B].zero_()
-        self.key[0][: self.B].zero_()
-        self.d_status.zero_()
+        api.grace_decode_begin(self.struct)
 
     def step(self, t: int) -> None:
         api.grace_decode_step(self.struct, t)
