@@ -424,6 +424,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2608_00938_b200 import api  # fails loudly if the CUDA library is missing
+    from paper_2608_00938_b200.sharding import max_over_ranks
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
     torch.cuda.set_device(local_rank)
     device = f"cuda:{local_rank}"
@@ -445,18 +446,12 @@ def main():
     ms_loop, per_step_us, launches = time_decode(dec, args.steps, args.warmup, dgroup)
     clocks = sampler.stop()
     status = int(dec.d_status.item())
-    if world > 1:
-        tmax = torch.tensor([ms_loop], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_loop = float(tmax.item())
+    ms_loop = max_over_ranks(ms_loop, device)
     units = beam_steps(cfg) * world
     value = units / (ms_loop * 1e-3)
 
     e2e_ms, h2d, d2h = time_e2e(dec, inp["enc_bits"], max(3, args.steps // 2), 3)
-    if world > 1:
-        tmax = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = max_over_ranks(e2e_ms, device)
 
     line = dict(metric="beam_steps_per_s", value=value, unit="beam-steps/s", n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms_loop, higher_is_better=True, scaling="weak", vs_baseline=None,
