@@ -1,0 +1,90 @@
+"""Run ONE op of the library on a chosen shape a few times (CUDA-event timing).
+
+Meant for profiler captures of a single kernel on a small case and for quick shape sweeps:
+
+    python -m paper_2608_00938_b200.opbench linear --M 32768 --N 2048 --K 512 --iters 5
+    python -m paper_2608_00938_b200.opbench cross_attn --B 16 --M 2048 --T 1024 --iters 5
+    python -m paper_2608_00938_b200.opbench self_attn --B 32 --M 2048 --t 3
+    python -m paper_2608_00938_b200.opbench topk --B 32 --M 2048 --V 1024 --K 2048
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import api
+
+
+def _time(fn, iters, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3)
+    return sorted(ts)[len(ts) // 2]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "layer_norm", "log_softmax"])
+    for name, default in (("B", 32), ("M", 2048), ("N", 2048), ("K", 512), ("T", 1024), ("H", 8), ("d", 64),
+                          ("V", 1024), ("t", 3), ("iters", 5)):
+        ap.add_argument(f"--{name}", type=int, default=default)
+    ap.add_argument("--f32out", action="store_true")
+    ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--relu", action="store_true")
+    a = ap.parse_args()
+    dev = "cuda:0"
+    torch.manual_seed(0)
+    bf = lambda *s: torch.randn(*s, device=dev).to(torch.bfloat16)
+    if a.op == "linear":
+        x, w = bf(a.M, a.K), bf(a.N, a.K) * 0.05
+        y = torch.zeros(a.M, a.N, device=dev, dtype=torch.float32 if (a.f32out or a.residual) else torch.bfloat16)
+        us = _time(lambda: api.grace_linear(x, w, y, y if a.residual else None, a.relu), a.iters)
+        print(f"linear M={a.M} N={a.N} K={a.K}: {us:.1f} us, {2.0 * a.M * a.N * a.K / us / 1e6:.1f} TFLOP/s")
+    elif a.op == "cross_attn":
+        q, k, v = bf(a.B * a.M, a.H, a.d), bf(a.B, a.H, a.T, a.d), bf(a.B, a.H, a.T, a.d)
+        o = torch.empty_like(q)
+        us = _time(lambda: api.grace_cross_attn(q, k, v, o, a.d ** -0.5), a.iters)
+        fl = 4.0 * a.B * a.M * a.H * a.d * a.T
+        by = 2 * (2 * q.numel() + 2 * k.numel())
+        print(f"cross_attn B={a.B} M={a.M} T={a.T}: {us:.1f} us, {fl / us / 1e6:.1f} TFLOP/s, {by / us / 1e3:.0f} GB/s")
+    elif a.op == "self_attn":
+        R = a.B * a.M
+        Lc = a.t + 1
+        kc, vc = bf(Lc, R, a.H, a.d), bf(Lc, R, a.H, a.d)
+        par = torch.randint(0, a.M, (Lc, R), device=dev, dtype=torch.int32)
+        qkv, o = bf(R, 3, a.H, a.d), torch.empty(R, a.H, a.d, device=dev, dtype=torch.bfloat16)
+        us = _time(lambda: api.grace_self_attn(qkv, kc, vc, par, [a.M] * Lc, o, a.B, a.t, a.d ** -0.5), a.iters)
+        by = R * a.H * a.d * 2 * (6 + 2 * a.t)
+        print(f"self_attn R={R} T_self={a.t + 1}: {us:.1f} us, {by / us / 1e3:.0f} GB/s (logical bytes)")
+    elif a.op == "topk":
+        N = a.M * a.V
+        cand = torch.randn(a.B, N, device=dev) * 3 - 8
+        ws = torch.empty(api.grace_beam_topk_workspace_bytes(a.B, N, a.K), dtype=torch.uint8, device=dev)
+        sc = torch.empty(a.B, a.K, device=dev)
+        fl = torch.empty(a.B, a.K, device=dev, dtype=torch.int32)
+        pa, tk = torch.empty_like(fl), torch.empty_like(fl)
+        us = _time(lambda: api.grace_beam_topk(cand, a.K, a.V, sc, fl, pa, tk, ws), a.iters)
+        print(f"topk B={a.B} N={N} K={a.K}: {us:.1f} us, {a.B * N * 4 / us / 1e3:.0f} GB/s")
+    elif a.op == "layer_norm":
+        R = a.B * a.M
+        x = torch.randn(R, a.K, device=dev)
+        g, b = torch.ones(a.K, device=dev), torch.zeros(a.K, device=dev)
+        o = torch.empty(R, a.K, device=dev, dtype=torch.bfloat16)
+        us = _time(lambda: api.grace_layer_norm(x, g, b, o), a.iters)
+        print(f"layer_norm R={R} D={a.K}: {us:.1f} us, {R * a.K * 6 / us / 1e3:.0f} GB/s")
+    else:
+        R = a.B * a.M
+        z = torch.randn(R, a.V, device=dev)
+        us = _time(lambda: api.grace_log_softmax(z), a.iters)
+        print(f"log_softmax R={R} V={a.V}: {us:.1f} us, {R * a.V * 8 / us / 1e3:.0f} GB/s")
+
+
+if __name__ == "__main__":
+    main()
