@@ -138,6 +138,196 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
   if (warp == 0) tc::tmem_dealloc(tmem_base, BN < 32 ? 32 : BN);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent kernel for the large GEMMs of the decoder (M in the tens of thousands).
+//
+// One CTA per SM walks over 128 x 256 output tiles (n fastest, so the CTAs running at the same
+// time share an A row panel in L2).  Warp 0 streams A (128 x 64) and W (256 x 64) tiles through a
+// 4-stage ring; warp 1 issues tcgen05.mma 128 x 256 x 16 into one of TWO TMEM accumulators
+// (2 x 256 columns = all of TMEM), so the four epilogue warps drain tile i while the tensor core
+// already works on tile i+1.  The epilogue reads 64 (bf16) or 32 (fp32) columns at a time from
+// TMEM, writes them to a 128-byte-swizzled staging tile in shared memory and hands it to TMA:
+// a plain tile store, or an fp32 add-reduction straight into the residual stream (x += y), so
+// the residual is never read into the SM.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPBM = 128, kPBN = 256, kPBK = 64, kPStages = 4;
+constexpr int kPABytes = kPBM * kPBK * 2;                 // 16 KB
+constexpr int kPBBytes = kPBN * kPBK * 2;                 // 32 KB
+constexpr int kPStageBytes = kPABytes + kPBBytes;
+constexpr int kPStagingBytes = 128 * 128;                 // 128 rows x 128 bytes
+constexpr int kPSmem = kPStages * kPStageBytes + 2 * kPStagingBytes + 1024 + 256;
+
+enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2 };
+
+template <int OUT>
+__global__ void __launch_bounds__(192, 1)
+linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                         const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* staging = tiles + kPStages * kPStageBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(staging + 2 * kPStagingBytes);
+  uint64_t* empty = full + kPStages;
+  uint64_t* acc_full = empty + kPStages;       // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KB = K / kPBK;
+  const int n_tiles = (N + kPBN - 1) / kPBN, m_tiles = (M + kPBM - 1) / kPBM;
+  const int total = n_tiles * m_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 4); }
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+    tc::tma_prefetch_desc(&map_x); tc::tma_prefetch_desc(&map_w); tc::tma_prefetch_desc(&map_y);
+  }
+  if (warp == 0) tc::tmem_alloc(tmem_slot, 512);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {                                        // ---- TMA producer ----
+      int it = 0;
+      for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
+        const int m0 = (tile / n_tiles) * kPBM, n0 = (tile % n_tiles) * kPBN;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % kPStages;
+          if (!tc::mbar_wait(empty + s, ((it / kPStages) & 1) ^ 1, abort_flag)) { tile = total; break; }
+          tc::mbar_expect_tx(full + s, kPStageBytes);
+          uint8_t* a = tiles + s * kPStageBytes;
+          tc::tma_load_2d(a, &map_x, full + s, kb * kPBK, m0);
+          tc::tma_load_2d(a + kPABytes, &map_w, full + s, kb * kPBK, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {                                        // ---- MMA issuer ----
+      constexpr uint32_t idesc = tc::idesc_bf16(kPBM, kPBN, 0);
+      int it = 0, local = 0;
+      for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++local) {
+        const int ab = local & 1;
+        if (!tc::mbar_wait(acc_empty + ab, ((local >> 1) & 1) ^ 1, abort_flag)) break;
+        tc::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * kPBN);
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % kPStages;
+          if (!tc::mbar_wait(full + s, (it / kPStages) & 1, abort_flag)) { ok = false; break; }
+          tc::tc_fence_after();
+          const uint32_t a_addr = tc::smem_addr(tiles + s * kPStageBytes);
+          const uint64_t a_desc = tc::smem_desc_sw128(a_addr, 16, 1024);
+          const uint64_t b_desc = tc::smem_desc_sw128(a_addr + kPABytes, 16, 1024);
+#pragma unroll
+          for (int k = 0; k < kPBK / 16; ++k)
+            tc::mma_ss(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+          tc::mma_commit(empty + s);
+        }
+        if (!ok) break;
+        tc::mma_commit(acc_full + ab);
+      }
+    }
+  } else {
+    // ---- epilogue warps 2..5: TMEM lane quarter q, rows q*32 + lane of the tile ----
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const bool issuer = (warp == 2 && lane == 0);
+    constexpr int kColsPerChunk = (OUT == kOutBf16) ? 64 : 32;
+    int local = 0, g = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++local) {
+      const int m0 = (tile / n_tiles) * kPBM, n0 = (tile % n_tiles) * kPBN;
+      const int ab = local & 1;
+      bool ok = tc::mbar_wait(acc_full + ab, (local >> 1) & 1, abort_flag);
+      ok = __all_sync(kFullMask, ok);
+      if (!ok) break;
+      tc::tc_fence_after();
+      const uint32_t t_acc = tmem_base + (uint32_t)(ab * kPBN) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kPBN / kColsPerChunk; ++c, ++g) {
+        uint8_t* buf = staging + (g & 1) * kPStagingBytes;
+        if (issuer) tc::bulk_wait_read<1>();               // the store that last used `buf` has read it
+        tc::named_bar_sync(1, 128);
+        uint4* my_row = reinterpret_cast<uint4*>(buf + row * 128);
+        if (OUT == kOutBf16) {
+#pragma unroll
+          for (int hseg = 0; hseg < 2; ++hseg) {
+            uint32_t r[32];
+            tc::tmem_ld32(t_acc + (uint32_t)(c * 64 + hseg * 32), r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                v[e] = __uint_as_float(r[8 * j + e]);
+                if (relu) v[e] = fmaxf(v[e], 0.f);
+              }
+              const int piece = hseg * 4 + j;
+              my_row[piece ^ (row & 7)] = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]),
+                                                     pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+            }
+          }
+        } else {
+          uint32_t r[32];
+          tc::tmem_ld32(t_acc + (uint32_t)(c * 32), r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              v[e] = __uint_as_float(r[4 * j + e]);
+              if (relu) v[e] = fmaxf(v[e], 0.f);
+            }
+            my_row[j ^ (row & 7)] = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]),
+                                               __float_as_uint(v[3]));
+          }
+        }
+        if (c == kPBN / kColsPerChunk - 1) {               // accumulator fully read: hand it back
+          tc::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(acc_empty + ab);
+        }
+        tc::fence_proxy_async_smem();
+        tc::named_bar_sync(1, 128);
+        if (issuer) {
+          if (OUT == kOutF32Add) tc::tma_reduce_add_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
+          else tc::tma_store_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
+          tc::bulk_commit();
+        }
+      }
+    }
+    if (issuer) tc::bulk_wait_all();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tmem_base, 512);
+}
+
+template <int OUT>
+static grace_status_t launch_persistent(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M,
+                                        int N, int K, int relu, cudaStream_t s) {
+  static bool attr_set = false;
+  static int n_sm = 0;
+  if (!attr_set) {
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_persistent_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem));
+    int dev = 0;
+    GRACE_CUDA_TRY(cudaGetDevice(&dev));
+    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    attr_set = true;
+  }
+  const int total = ((N + kPBN - 1) / kPBN) * ((M + kPBM - 1) / kPBM);
+  const int grid = total < n_sm ? total : n_sm;
+  linear_persistent_kernel<OUT><<<grid, 192, kPSmem, s>>>(mx, mw, my, M, N, K, relu);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
 template <int BN>
 static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw, const GemmParams& p, cudaStream_t s) {
   static bool attr_set = false;
@@ -163,6 +353,25 @@ extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uin
   if (!grace_aligned16(x) || !grace_aligned16(w) || !grace_aligned16(y_bf16) || !grace_aligned16(y_f32) ||
       !grace_aligned16(residual) || (ldx & 7) || (ldw & 7) || (ldy & 7) || ldx < K || ldw < K || ldy < N)
     return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const bool aliased = (residual != nullptr) && (residual == y_f32);
+  if (M >= 1024 && N >= 256 && (residual == nullptr || aliased)) {
+    // large GEMM: persistent kernel, TMA-store epilogue (add-reduction when y is the residual stream)
+    CUtensorMap mx, mw, my;
+    const uint64_t dx[2] = {(uint64_t)K, (uint64_t)M}, sx[1] = {(uint64_t)ldx};
+    const uint32_t bx[2] = {(uint32_t)kPBK, (uint32_t)kPBM};
+    const uint64_t dw[2] = {(uint64_t)K, (uint64_t)N}, sw[1] = {(uint64_t)ldw};
+    const uint32_t bw[2] = {(uint32_t)kPBK, (uint32_t)kPBN};
+    const uint64_t dy[2] = {(uint64_t)N, (uint64_t)M}, sy[1] = {(uint64_t)ldy};
+    const bool f32 = (y_f32 != nullptr);
+    const uint32_t by[2] = {f32 ? 32u : 64u, 128u};
+    if (!tc::make_tmap_bf16(&mx, x, 2, dx, sx, bx) || !tc::make_tmap_bf16(&mw, w, 2, dw, sw, bw) ||
+        !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
+      return GRACE_CUDA_ERROR;
+    if (!f32) return launch_persistent<kOutBf16>(mx, mw, my, M, N, K, relu, s);
+    if (aliased) return launch_persistent<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
+    return launch_persistent<kOutF32>(mx, mw, my, M, N, K, relu, s);
+  }
   CUtensorMap mx, mw;
   const int BN = (N >= 128) ? 128 : 64;
   {
@@ -178,6 +387,5 @@ extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uin
   GemmParams p;
   p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.ldy = ldy;
   p.M = M; p.N = N; p.K = K; p.relu = relu;
-  cudaStream_t s = (cudaStream_t)stream;
   return BN == 128 ? launch_linear<128>(mx, mw, p, s) : launch_linear<64>(mx, mw, p, s);
 }

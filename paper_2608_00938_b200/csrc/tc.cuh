@@ -32,19 +32,24 @@ inline EncodeTiledFn encode_tiled_fn() {
 
 // bf16 tensor of `rank` dims (dims[0] innermost, contiguous), strides in elements for dims 1..,
 // box in elements.  128-byte swizzle: box[0] must be 64 elements.  Out-of-range reads give 0.
-inline bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                           const uint64_t* strides_elems, const uint32_t* box, bool swizzle128 = true) {
+inline bool make_tmap(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                      const uint64_t* strides_elems, const uint32_t* box, bool is_f32, bool swizzle128 = true) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
   cuuint64_t gdim[5], gstr[4];
   cuuint32_t gbox[5], estr[5];
+  const uint64_t esize = is_f32 ? 4 : 2;
   for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; gbox[i] = box[i]; estr[i] = 1; }
-  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_elems[i] * 2;
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
-                  gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_elems[i] * esize;
+  CUresult r = fn(map, is_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+                  const_cast<void*>(base), gdim, gstr, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+inline bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                           const uint64_t* strides_elems, const uint32_t* box, bool swizzle128 = true) {
+  return make_tmap(map, base, rank, dims, strides_elems, box, false, swizzle128);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -104,6 +109,24 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(smem_addr(dst)), "l"(map), "r"(smem_addr(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// Shared -> global tile store / fp32 add-reduction (bulk async group; rows or columns outside the
+// tensor are clipped).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(smem_addr(src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(smem_addr(src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }

@@ -320,6 +320,10 @@ def test_cross_attn_strided_kv_layout(api):
 @pytest.mark.parametrize("M,N,K,relu,res,f32out", [
     (16, 384, 128, False, False, False), (300, 512, 512, False, True, True), (257, 2048, 512, True, False, False),
     (130, 64, 2048, False, True, True), (1, 1536, 512, False, False, False), (100, 80, 64, False, False, True),
+    # persistent-kernel shapes (M >= 1024, N >= 256): ragged M and N tiles, every epilogue mode
+    (1500, 512, 512, False, True, True), (2125, 1536, 512, False, False, False), (1100, 2048, 512, True, False, False),
+    (1300, 512, 2048, False, True, True), (1024, 2048, 512, False, False, True), (1111, 320, 128, False, False, True),
+    (40000, 256, 64, True, False, False), (19000, 512, 512, False, True, True),
 ])
 def test_linear_matches_fp64_matmul(api, M, N, K, relu, res, f32out):
     rng = synth.rng_for(5, M + N + K)
