@@ -5,15 +5,16 @@
 // of 128:
 //   S   = Q K_blk^T        tcgen05.mma, A = Q (shared, K-major), B = K_blk (shared, K-major),
 //                          fp32 S[128 x 128] in TMEM
-//   P   = exp2(S*c - max)  128 softmax threads, one query row each (TMEM lane = row); P is
-//                          written back over S as packed bf16
-//   O_b = P V_blk          tcgen05.mma, A = P (TMEM), B = V_blk (shared, read MN-major, so V is
-//                          used as stored: no transpose anywhere)
-//   O  += O_b              in registers, with the usual running-max rescale
+//   P   = exp2(S*c - max)  256 softmax threads: TMEM lane = query row, two threads per row each
+//                          taking half of the block's columns; P goes to its own TMEM columns
+//                          as packed bf16
+//   O  += P V_blk          tcgen05.mma, A = P (TMEM), B = V_blk (shared, read MN-major, so V is
+//                          used as stored: no transpose anywhere); O stays in TMEM for the whole
+//                          row tile and is rescaled lazily, only when a row maximum grows by > 2^8
 // K/V blocks arrive by TMA through a two-stage ring; Q, K and V are addressed with 4-D tensor
 // maps over the caller's strides, so the beam-major Q / O layout is never permuted (the view /
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
-// and masked in the softmax.  Warp roles: 0-3 softmax + epilogue, 4 TMA producer, 5 MMA issuer.
+// and masked in the softmax.  Warp roles: 0-7 softmax + epilogue, 8 TMA producer, 9 MMA issuer.
 // Two CTAs share an SM, so one CTA's MMAs run under the other's exponentials.
 #pragma once
 #include "common.cuh"
@@ -26,8 +27,10 @@ constexpr int kCaBN = 128;        // encoder positions per block
 constexpr int kCaDH = 64;
 constexpr int kCaStages = 2;
 constexpr int kCaTileBytes = 128 * 64 * 2;                       // 16 KB: Q, K_blk or V_blk
-constexpr int kCaSmemBytes = kCaTileBytes * (1 + 2 * kCaStages) + 1024 + 256;
-constexpr uint32_t kCaTmemCols = 256;                            // S/P: 0..127, O_blk: 128..191
+constexpr int kCaSoftmaxWarps = 8;
+constexpr int kCaThreads = (kCaSoftmaxWarps + 2) * 32;
+constexpr int kCaSmemBytes = kCaTileBytes * (1 + 2 * kCaStages) + 1024 + 256 + 2 * 2 * 128 * 4 + 2 * 128 * 4;
+constexpr uint32_t kCaTmemCols = 256;                            // S: 0..127, O_blk: 128..191, P: 192..255
 
 struct CrossTcParams {
   uint16_t* out;
@@ -43,7 +46,13 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(192)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float m;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+  return m;
+}
+
+__global__ void __launch_bounds__(kCaThreads, 2)
 cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const CrossTcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -56,9 +65,11 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   uint64_t* kv_empty = kv_full + kCaStages;
   uint64_t* s_full = kv_empty + kCaStages;
   uint64_t* p_full = s_full + 1;
-  uint64_t* o_last = p_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_last + 1);
+  uint64_t* o_full = p_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* half_max = reinterpret_cast<float*>(bars + 32);         // [2 parity][2 halves][128 rows]
+  float* half_sum = half_max + 2 * 2 * 128;                      // [2 halves][128 rows]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * kCaBM, h = blockIdx.y, b = blockIdx.z;
@@ -68,20 +79,21 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     tc::mbar_init(q_full, 1);
     for (int s = 0; s < kCaStages; ++s) { tc::mbar_init(kv_full + s, 1); tc::mbar_init(kv_empty + s, 1); }
     tc::mbar_init(s_full, 1);
-    tc::mbar_init(p_full, 4);                  // one arrival per softmax warp
-    tc::mbar_init(o_last, 1);
+    tc::mbar_init(p_full, kCaSoftmaxWarps);    // one arrival per softmax warp
+    tc::mbar_init(o_full, 1);
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
-  if (warp == 4) tc::tmem_alloc(tmem_slot, kCaTmemCols);
+  if (warp == kCaSoftmaxWarps) tc::tmem_alloc(tmem_slot, kCaTmemCols);
   tc::tc_fence_before();
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base;           // S fp32 cols 0..127; P bf16x2 cols 0..63
-  const uint32_t tmem_o = tmem_base + 128;     // O_blk fp32 cols 128..191
+  const uint32_t tmem_s = tmem_base;           // S fp32, 128 columns
+  const uint32_t tmem_o = tmem_base + 128;     // O_blk fp32, 64 columns
+  const uint32_t tmem_p = tmem_base + 192;     // P bf16 pairs, 64 columns
 
-  if (warp == 4) {
+  if (warp == kCaSoftmaxWarps) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
@@ -95,7 +107,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, kv_full + s, 0, j * kCaBN, h, b);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kCaSoftmaxWarps + 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc_s = tc::idesc_bf16(kCaBM, kCaBN, 0);     // Q K^T : B K-major
@@ -114,13 +126,9 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       for (int j = 0; ok && j < NB; ++j) {
         const int s = j % kCaStages;
         if (!tc::mbar_wait(p_full, j & 1, abort_flag)) break;
-        tc::tc_fence_after();
-        const uint32_t v_addr = tc::smem_addr(kv_tiles + (2 * s + 1) * kCaTileBytes);
-#pragma unroll
-        for (int k = 0; k < kCaBN / 16; ++k)
-          tc::mma_ts(tmem_o, tmem_s + 8 * k, tc::smem_desc_sw128(v_addr + 2048 * k, 1024, 1024), idesc_o,
-                     k ? 1u : 0u);
-        tc::mma_commit(kv_empty + s);                       // K_blk, V_blk of block j are consumed
+        // p_full(j) also means every softmax thread has read S of block j: S of block j+1 goes
+        // first, so the softmax threads get their next scores while P V of block j still runs.
+        // (P has its own TMEM columns, so S(j+1) cannot clobber it.)
         if (j + 1 < NB) {
           const int s1 = (j + 1) % kCaStages;
           if (!tc::mbar_wait(kv_full + s1, ((j + 1) / kCaStages) & 1, abort_flag)) break;
@@ -130,111 +138,133 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           for (int k = 0; k < kCaDH / 16; ++k)
             tc::mma_ss(tmem_s, tc::smem_desc_sw128(q_addr + 32 * k, 16, 1024),
                        tc::smem_desc_sw128(k_addr + 32 * k, 16, 1024), idesc_s, k ? 1u : 0u);
-          tc::mma_commit(s_full);                           // also: O_blk of block j is complete
-        } else {
-          tc::mma_commit(o_last);
+          tc::mma_commit(s_full);
         }
+        tc::tc_fence_after();
+        const uint32_t v_addr = tc::smem_addr(kv_tiles + (2 * s + 1) * kCaTileBytes);
+#pragma unroll
+        for (int k = 0; k < kCaBN / 16; ++k)
+          tc::mma_ts(tmem_o, tmem_p + 8 * k, tc::smem_desc_sw128(v_addr + 2048 * k, 1024, 1024), idesc_o,
+                     (j | k) ? 1u : 0u);              // O accumulates in TMEM across blocks
+        tc::mma_commit(kv_empty + s);                       // K_blk, V_blk of block j are consumed
+        tc::mma_commit(o_full);                             // O_blk of block j is complete
       }
     }
   } else {
-    // ---------------- softmax + epilogue: thread = query row ----------------
-    const int row = warp * 32 + lane;                       // TMEM lane
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    // ---------------- softmax + epilogue ----------------
+    // Warps w and w+4 share the TMEM lanes (= query rows) 32*(w&3)..+31; each takes one half of the
+    // 128 score columns and one half of the 64 output columns of those rows.  O stays in TMEM and
+    // accumulates across blocks; it is rescaled only when a row's maximum grows by more than 2^8
+    // (probabilities may then reach 256, which bf16 and the fp32 sums hold without loss).
+    const int quarter = warp & 3, half = warp >> 2;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int col_base = 64 * half;
+    const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
     float m_run = -INFINITY, l_run = 0.f;
-    float o_acc[kCaDH];
-#pragma unroll
-    for (int i = 0; i < kCaDH; ++i) o_acc[i] = 0.f;
     bool ok = true;
     for (int j = 0; j < NB; ++j) {
       ok = ok && tc::mbar_wait(s_full, j & 1, abort_flag);
       ok = __all_sync(kFullMask, ok);
       if (!ok) break;
       tc::tc_fence_after();
-      if (j > 0) {                                          // O_blk of block j-1 is complete too
-#pragma unroll
-        for (int c = 0; c < kCaDH / 32; ++c) {
-          uint32_t r[32];
-          tc::tmem_ld32(tmem_o + lane_addr + 32 * c, r);
-          tc::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o_acc[32 * c + i] += __uint_as_float(r[i]);
-        }
-      }
-      const int valid = min(kCaBN, p.T - j * kCaBN);        // columns of this block that exist
-      // pass 1: row maximum
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < kCaBN / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(tmem_s + lane_addr + 32 * c, r);
+      uint32_t r[64];
+      {
+        uint32_t (&r0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
+        uint32_t (&r1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
+        tc::tmem_ld32(tmem_s + lane_addr + col_base, r0);
+        tc::tmem_ld32(tmem_s + lane_addr + col_base + 32, r1);
         tc::tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (32 * c + i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
       }
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float alpha = ex2(m_run - m_new);               // 0 on the first block
-      if (alpha != 1.f) {
-        l_run *= alpha;
+      const int valid = min(kCaBN, p.T - j * kCaBN) - col_base;   // this thread's columns that exist
+      if (valid < 64) {
 #pragma unroll
-        for (int i = 0; i < kCaDH; ++i) o_acc[i] *= alpha;
+        for (int i = 0; i < 64; ++i)
+          if (i >= valid) r[i] = 0xff800000u;                     // -inf: no weight, no influence on the max
       }
+      float mx = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+#pragma unroll
+      for (int i = 3; i + 1 < 64; i += 2) mx = max3(mx, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+      mx = fmaxf(mx, __uint_as_float(r[63]));
+      float* hm = half_max + (j & 1) * 256;
+      hm[half * 128 + row] = mx;
+      tc::named_bar_sync(2 + quarter, 64);                  // the two warps of this row quarter
+      const float m_blk = fmaxf(mx, hm[(half ^ 1) * 128 + row]) * p.scale_log2;
+      const bool grow = m_blk > m_run + 8.0f;               // always true on the first block
+      const float m_new = grow ? m_blk : m_run;
+      const float alpha = grow ? ex2(m_run - m_new) : 1.0f; // 0 on the first block
       m_run = m_new;
-      // pass 2: probabilities, written over S as packed bf16
-      float sum = 0.f;
+      // probabilities -> packed bf16 in the P columns; row sum
+      const float2 neg_m2 = make_float2(-m_new, -m_new);
+      float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int c = 0; c < kCaBN / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(tmem_s + lane_addr + 32 * c, r);
-        tc::tmem_ld_wait();
-        uint32_t packed[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float e0 = ex2(fmaf(__uint_as_float(r[2 * i]), p.scale_log2, -m_new));
-          float e1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), p.scale_log2, -m_new));
-          if (32 * c + 2 * i >= valid) e0 = 0.f;
-          if (32 * c + 2 * i + 1 >= valid) e1 = 0.f;
-          sum += e0 + e1;
-          packed[i] = pack_bf16x2(e0, e1);
-        }
-        tc::tmem_st16(tmem_s + lane_addr + 16 * c, packed);
+      for (int i = 0; i < 32; ++i) {
+        const float2 t = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), scale2, neg_m2);
+        const float2 e = make_float2(ex2(t.x), ex2(t.y));
+        sum2 = __fadd2_rn(sum2, e);
+        r[i] = pack_bf16x2(e.x, e.y);
       }
-      l_run += sum;
+      l_run = fmaf(l_run, alpha, sum2.x + sum2.y);
+      if (j > 0) {
+        // P V of block j-1 reads the P columns and writes O: it must be complete before P of this
+        // block is stored and before O is rescaled.  (It was issued right after S of this block,
+        // so by now it has long finished.)
+        ok = tc::mbar_wait(o_full, (j - 1) & 1, abort_flag);
+        ok = __all_sync(kFullMask, ok);
+        if (!ok) break;
+        tc::tc_fence_after();
+      }
+      {
+        uint32_t (&p0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[0]);
+        uint32_t (&p1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[16]);
+        tc::tmem_st16(tmem_p + lane_addr + 32 * half, p0);
+        tc::tmem_st16(tmem_p + lane_addr + 32 * half + 16, p1);
+      }
+      if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
+        uint32_t o[32];
+        tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
+        tc::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+        uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
+        uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
+        tc::tmem_st16(tmem_o + lane_addr + 32 * half, o0);
+        tc::tmem_st16(tmem_o + lane_addr + 32 * half + 16, o1);
+      }
       tc::tmem_st_wait();
       tc::tc_fence_before();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(p_full);
     }
-    if (ok) ok = tc::mbar_wait(o_last, 0, abort_flag);
+    if (ok) ok = tc::mbar_wait(o_full, (NB - 1) & 1, abort_flag);
     ok = __all_sync(kFullMask, ok);
     if (ok) {
       tc::tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < kCaDH / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(tmem_o + lane_addr + 32 * c, r);
-        tc::tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o_acc[32 * c + i] += __uint_as_float(r[i]);
-      }
+      uint32_t o[32];
+      tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
+      tc::tmem_ld_wait();
+      half_sum[half * 128 + row] = l_run;
+      tc::named_bar_sync(2 + quarter, 64);
+      const float l_tot = l_run + half_sum[(half ^ 1) * 128 + row];
       const int m = m0 + row;
       if (m < p.M) {
-        const float inv = 1.f / l_run;
+        const float inv = 1.f / l_tot;
         const int64_t r_out = (int64_t)b * p.M + m;
-        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * kCaDH);
+        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * kCaDH + 32 * half);
 #pragma unroll
-        for (int i = 0; i < kCaDH / 8; ++i)
-          dst[i] = make_uint4(pack_bf16x2(o_acc[8 * i] * inv, o_acc[8 * i + 1] * inv),
-                              pack_bf16x2(o_acc[8 * i + 2] * inv, o_acc[8 * i + 3] * inv),
-                              pack_bf16x2(o_acc[8 * i + 4] * inv, o_acc[8 * i + 5] * inv),
-                              pack_bf16x2(o_acc[8 * i + 6] * inv, o_acc[8 * i + 7] * inv));
-        if (p.lse != nullptr) p.lse[r_out * p.H + h] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+        for (int i = 0; i < 4; ++i)
+          dst[i] = make_uint4(
+              pack_bf16x2(__uint_as_float(o[8 * i]) * inv, __uint_as_float(o[8 * i + 1]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv));
+        if (p.lse != nullptr && half == 0) p.lse[r_out * p.H + h] = (m_run + log2f(l_tot)) * 0.6931471805599453f;
       }
     }
   }
   tc::tc_fence_before();
   __syncthreads();
-  if (warp == 4) tc::tmem_dealloc(tmem_base, kCaTmemCols);
+  if (warp == kCaSoftmaxWarps) tc::tmem_dealloc(tmem_base, kCaTmemCols);
 }
 
 inline bool cross_attn_tc_supported(int B, int M, int H, int d_h, int T_ctx) {
@@ -269,7 +299,7 @@ inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stri
   p.out = out; p.lse = lse; p.out_row_stride = out_row_stride; p.M = M; p.H = H; p.T = T_ctx;
   p.scale_log2 = scale * 1.4426950408889634f;
   dim3 grid((unsigned)((M + kCaBM - 1) / kCaBM), (unsigned)H, (unsigned)B);
-  cross_attn_tc_kernel<<<grid, 192, kCaSmemBytes, s>>>(mq, mk, mv, p);
+  cross_attn_tc_kernel<<<grid, kCaThreads, kCaSmemBytes, s>>>(mq, mk, mv, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
