@@ -1,12 +1,13 @@
 // CD + GTM mask with score add (Sections 3.1, 4.1, 5.4) and the beam-state update after top-k
 // (Sections 3.3, 4.4).
 //
-// One warp owns one beam row.  The row's child bitmask (V/64 words) is loaded once into
-// registers, one word per lane, with a warp prefix sum of popcounts so that any lane can turn a
-// token into the id of the child node.  Each lane then streams float4 pieces of the row's
-// log-probabilities: coalesced 512-byte warp loads in, 512-byte warp stores out.  The request's
-// matcher (node-eligibility bits or Bloom filter words) is read only for catalog-valid tokens.
-// HBM-bound at the root levels (4 bytes in + 4 bytes out per candidate).
+// One warp owns one beam row.  The row's child bitmask (V/64 words, one word per lane) and a warp
+// prefix sum of its popcounts give every lane the k-th catalog-valid child directly, so matcher
+// work (node-eligibility bit or Bloom probes) is done only for valid children and with all lanes
+// busy.  The row is then streamed with float4 accesses: 512-byte warp stores out, and log-prob
+// sectors in only where a token is allowed.  HBM-bound at the root levels (4 bytes out plus up to
+// 4 bytes in per candidate); with the Bloom matcher the random 8-byte probes into the request's
+// 512 KB filter (L2-resident) add a latency/L2-bandwidth term.
 #include "common.cuh"
 
 namespace grace {
@@ -28,32 +29,38 @@ struct MaskParams {
   int bloom_hashes;
 };
 
-template <int KIND>
-__device__ __forceinline__ bool token_matches(const MaskParams& p, const uint64_t* req_bits,
-                                              int64_t child, uint64_t row_key, int v) {
-  if (KIND == GRACE_MATCH_NONE) return true;
-  if (KIND == GRACE_MATCH_NODE_BITMASK) {
-    if (child < 0 || child >= p.num_nodes) return false;
-    return (__ldg(req_bits + (child >> 6)) >> (child & 63)) & 1ull;
+// Position of the n-th (0-based) set bit of a 64-bit word that has more than n bits set.
+__device__ __forceinline__ int nth_set_bit64(uint64_t word, int n) {
+  uint32_t x = (uint32_t)word;
+  int pos = 0;
+  int c = __popc(x);
+  if (n >= c) { n -= c; x = (uint32_t)(word >> 32); pos = 32; }
+#pragma unroll
+  for (int width = 16; width >= 1; width >>= 1) {
+    const uint32_t low = x & ((1u << width) - 1u);
+    c = __popc(low);
+    if (n >= c) { n -= c; x >>= width; pos += width; } else { x = low; }
   }
-  // prefix Bloom filter: all probed bits must be set; stop at the first clear bit
-  const uint64_t key = row_key | ((uint64_t)(v + 1) << (16 * p.prefix_len));
-  const uint64_t z = mix64(key);
-  const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
-  for (int i = 0; i < p.bloom_hashes; ++i) {
-    const uint32_t pos = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
-    if (!((__ldg(req_bits + (pos >> 6)) >> (pos & 63)) & 1ull)) return false;
-  }
-  return true;
+  return pos;
 }
 
 constexpr int kMaskWarpsPerBlock = 8;
 
+// One warp per beam row, two phases per chunk of 2048 tokens:
+//   1. the catalog-valid children (set bits of the node's child bitmask) are enumerated compactly,
+//      lane k takes the k-th, (k+32)-th, ... child, evaluates the request's matcher for it and ORs
+//      the result into the warp's allow words in shared memory.  Bloom probes are issued two at a
+//      time so that both loads are in flight together.
+//   2. the row is streamed: cand = score + logp where allowed, -inf elsewhere; a 32-byte sector of
+//      log-probabilities is read only if one of its tokens is allowed.
 template <int KIND>
 __global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
 gtm_mask_kernel(const MaskParams p) {
-  const int lane = threadIdx.x & 31;
-  const int r = blockIdx.x * kMaskWarpsPerBlock + (threadIdx.x >> 5);
+  __shared__ uint64_t s_words[kMaskWarpsPerBlock][32];
+  __shared__ unsigned long long s_allow[kMaskWarpsPerBlock][32];
+  __shared__ int s_incl[kMaskWarpsPerBlock][32];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int r = blockIdx.x * kMaskWarpsPerBlock + wib;
   if (r >= p.R) return;
   const int V = p.V;
   const int W = V >> 6;
@@ -71,58 +78,86 @@ gtm_mask_kernel(const MaskParams p) {
   const float ninf = __int_as_float(0xff800000);
   const float* lrow = p.logp + (int64_t)r * V;
   bool saw_nan = false;
+  uint64_t* words = s_words[wib];
+  unsigned long long* allow = s_allow[wib];
+  int* incl = s_incl[wib];
 
-  // chunks of 2048 tokens: 32 words, one per lane
   int rank_before_chunk = 0;
   for (int w0 = 0; w0 < W; w0 += 32) {
     uint64_t word = 0;
     if (!dead && w0 + lane < W) word = __ldg(p.child_bits + (int64_t)node * W + w0 + lane);
-    int pc = __popcll(word);
-    int incl = pc;
+    const int pc = __popcll(word);
+    int inc = pc;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-      int o = __shfl_up_sync(kFullMask, incl, d);
-      if (lane >= d) incl += o;
+      const int o = __shfl_up_sync(kFullMask, inc, d);
+      if (lane >= d) inc += o;
     }
-    const int excl = incl - pc + rank_before_chunk;       // children before this lane's word
-    rank_before_chunk += __shfl_sync(kFullMask, incl, 31);
+    const int total = __shfl_sync(kFullMask, inc, 31);
+    __syncwarp();
+    words[lane] = word;
+    incl[lane] = inc;
+    allow[lane] = (KIND == GRACE_MATCH_NONE) ? word : 0ull;
+    __syncwarp();
 
-    const int chunk_tokens = min(2048, V - (w0 << 6));
-    // 128 tokens per iteration: lane handles tokens 4*lane .. 4*lane+3 of the group
-    for (int g = 0; g < chunk_tokens; g += 128) {
-      const int tok0 = (w0 << 6) + g + 4 * lane;          // first token of this lane
-      const bool in_range = (g + 4 * lane) < chunk_tokens; // V % 64 == 0, so all 4 or none
-      const int src_lane = (g >> 6) + (lane >> 4);         // lane holding the word of these tokens
-      const uint64_t cw = __shfl_sync(kFullMask, word, src_lane);
-      const int cex = __shfl_sync(kFullMask, excl, src_lane);
-      float4 lp = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (in_range && !dead && cw != 0ull) lp = __ldg(reinterpret_cast<const float4*>(lrow + tok0));
-      float vals[4] = {lp.x, lp.y, lp.z, lp.w};
-      float outv[4];
-      uint32_t nib = 0;
+    if (KIND != GRACE_MATCH_NONE) {
+      for (int k0 = 0; k0 < total; k0 += 32) {
+        const int k = k0 + lane;
+        const bool have = k < total;
+        // word holding the k-th child: smallest w with incl[w] > k
+        int lo = 0;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int bit = (tok0 + j) & 63;
-        bool ok = in_range && ((cw >> bit) & 1ull);
-        if (ok) {
-          const int64_t child = (int64_t)base + cex + __popcll(cw & ((1ull << bit) - 1ull));
-          ok = token_matches<KIND>(p, req_bits, child, row_key, tok0 + j);
+        for (int step = 16; step >= 1; step >>= 1)
+          if (have && incl[lo + step - 1] <= k) lo += step;
+        const uint64_t cw = have ? words[lo] : 1ull;
+        const int within = have ? k - (incl[lo] - __popcll(cw)) : 0;
+        const int bit = nth_set_bit64(cw, within);
+        bool ok = have;
+        if (KIND == GRACE_MATCH_NODE_BITMASK) {
+          const int64_t child = (int64_t)base + rank_before_chunk + k;
+          if (ok) ok = (child >= 0 && child < p.num_nodes) && ((__ldg(req_bits + (child >> 6)) >> (child & 63)) & 1ull);
+        } else {
+          const int v = (w0 << 6) + (lo << 6) + bit;
+          const uint64_t z = mix64(row_key | ((uint64_t)(v + 1) << (16 * p.prefix_len)));
+          const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
+          for (int i = 0; i < p.bloom_hashes && ok; i += 2) {
+            const uint32_t pos_a = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
+            const uint32_t pos_b = (h1 + (uint32_t)(i + 1) * h2) & (uint32_t)p.bloom_mask_bits;
+            const uint64_t wa = __ldg(req_bits + (pos_a >> 6));
+            const uint64_t wb = (i + 1 < p.bloom_hashes) ? __ldg(req_bits + (pos_b >> 6)) : ~0ull;
+            ok = ((wa >> (pos_a & 63)) & 1ull) && ((i + 1 >= p.bloom_hashes) || ((wb >> (pos_b & 63)) & 1ull));
+          }
         }
-        outv[j] = ok ? (score + vals[j]) : ninf;
-        if (ok && vals[j] != vals[j]) saw_nan = true;
-        nib |= (ok ? 1u : 0u) << j;
+        if (ok) atomicOr(&allow[lo], 1ull << bit);
       }
-      if (in_range && p.cand != nullptr)
-        *reinterpret_cast<float4*>(p.cand + (int64_t)r * V + tok0) = make_float4(outv[0], outv[1], outv[2], outv[3]);
-      if (p.allow_bits != nullptr) {
-        // 16 lanes x 4 bits -> one 64-bit word
-        uint64_t x = (uint64_t)nib << (4 * (lane & 15));
+      __syncwarp();
+    }
+    rank_before_chunk += total;
+
+    if (p.allow_bits != nullptr && w0 + lane < W) p.allow_bits[(int64_t)r * W + w0 + lane] = allow[lane];
+    if (p.cand != nullptr) {
+      const int chunk_tokens = min(2048, V - (w0 << 6));
+      // 128 tokens per iteration: lane handles tokens 4*lane .. 4*lane+3 of the group
+      for (int g = 0; g < chunk_tokens; g += 128) {
+        const int tok_in_chunk = g + 4 * lane;
+        if (tok_in_chunk >= chunk_tokens) continue;           // V % 64 == 0, so all 4 or none
+        const uint32_t nib = (uint32_t)(allow[tok_in_chunk >> 6] >> (tok_in_chunk & 63)) & 0xfu;
+        // log-probs are read only where a token of this lane is allowed
+        float4 lp = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (nib != 0u) lp = __ldg(reinterpret_cast<const float4*>(lrow + (w0 << 6) + tok_in_chunk));
+        const float vals[4] = {lp.x, lp.y, lp.z, lp.w};
+        float outv[4];
 #pragma unroll
-        for (int d = 1; d < 16; d <<= 1) x |= __shfl_xor_sync(kFullMask, x, d);
-        if ((lane & 15) == 0 && in_range)
-          p.allow_bits[(int64_t)r * W + w0 + (g >> 6) + (lane >> 4)] = x;
+        for (int j = 0; j < 4; ++j) {
+          const bool okj = (nib >> j) & 1u;
+          outv[j] = okj ? (score + vals[j]) : ninf;
+          if (okj && vals[j] != vals[j]) saw_nan = true;
+        }
+        *reinterpret_cast<float4*>(p.cand + (int64_t)r * V + (w0 << 6) + tok_in_chunk) =
+            make_float4(outv[0], outv[1], outv[2], outv[3]);
       }
     }
+    __syncwarp();
   }
   if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
 }
