@@ -220,27 +220,41 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
         }
         const uint32_t incl = warp_incl_scan(real);
         const uint32_t total = __shfl_sync(kFullMask, incl, 31);
-        uint32_t start = 0;
-        if (lane == 31 && total != 0) start = atomicAdd(&stage_count, total);
-        start = __shfl_sync(kFullMask, start, 31) + incl - real;
+        uint32_t start = 0, gbase = 0;
+        if (lane == 31 && total != 0) {
+          start = atomicAdd(&stage_count, total);
+          // entries that land beyond the stage go straight to the request's list, with their own
+          // reservation there (a run of hits, e.g. thousands of tied candidates, can exceed it)
+          const uint32_t first_over = max(start, (uint32_t)kStage);
+          if (start + total > first_over) gbase = atomicAdd(&hdr[b].count, start + total - first_over);
+        }
+        start = __shfl_sync(kFullMask, start, 31);
+        gbase = __shfl_sync(kFullMask, gbase, 31);
+        const uint32_t first_over = max(start, (uint32_t)kStage);
+        uint32_t pos = start + incl - real;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (key[j] > t_excl) {
-            if (start < (uint32_t)kStage) stage[start] = make_uint2(key[j], (uint32_t)(i * 4 + j));
-            ++start;
+            const uint2 entry = make_uint2(key[j], (uint32_t)(i * 4 + j));
+            if (pos < (uint32_t)kStage) {
+              stage[pos] = entry;
+            } else {
+              const uint32_t g = gbase + (pos - first_over);
+              if (g < (uint32_t)kCap) list[g] = entry;
+            }
+            ++pos;
           }
         }
       }
     }
-    // flush when the stage is at least half full (a tile that overflows it outright means the
-    // request's list overflows too: the true count is kept, the entries are dropped)
+    // flush when the stage is at least half full
     __syncthreads();
-    const uint32_t staged = stage_count;
+    const uint32_t staged = min(stage_count, (uint32_t)kStage);
     if (staged >= (uint32_t)kStage / 2) {
       if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
       __syncthreads();
       const uint32_t dst = flush_base;
-      for (uint32_t e = threadIdx.x; e < min(staged, (uint32_t)kStage); e += kCollectThreads)
+      for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
         if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
       __syncthreads();
       if (threadIdx.x == 0) stage_count = 0;
@@ -248,12 +262,12 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
     }
   }
   __syncthreads();
-  const uint32_t staged = stage_count;
+  const uint32_t staged = min(stage_count, (uint32_t)kStage);
   if (staged != 0) {
     if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
     __syncthreads();
     const uint32_t dst = flush_base;
-    for (uint32_t e = threadIdx.x; e < min(staged, (uint32_t)kStage); e += kCollectThreads)
+    for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
       if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
   }
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
@@ -487,7 +501,8 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, To
   const float* row = cand + (int64_t)b * N;
   const uint32_t n_out = min(c, (uint32_t)K);
   for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
-    const uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
+    uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
+    if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
     const int64_t o = (int64_t)b * K + i;
     out_score[o] = row[idx];
     if (out_flat) out_flat[o] = (int32_t)idx;
@@ -594,3 +609,4 @@ extern "C" grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, i
   return grace::launch_beam_topk(cand, B, N, K, V, out_score, out_flat, out_parent, out_token, ws,
                                  d_status, (cudaStream_t)stream);
 }
+

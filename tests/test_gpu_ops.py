@@ -178,6 +178,11 @@ def test_topk_adversarial_inputs_take_the_exact_path_and_stay_exact(api):
     zeros[:, ::2] = -0.0                                        # -0.0 == +0.0
     zeros[:, 1000:] = -1.0
     _check_topk(api, zeros, K, V)
+    burst = np.full((B, N), -np.inf, dtype=np.float32)          # a dense run of ties above a sparse rest:
+    burst[rng.random((B, N)) < 0.003] = -3.0                    # thousands of hits inside one tile of the
+    burst[0, :5000] = 0.5                                       # collecting pass, but fewer than the list holds
+    burst[1, 70000:73000] = 0.25
+    _check_topk(api, burst, 1500, V)
     ramp = np.arange(N, dtype=np.float32)[None].repeat(B, 0)   # sorted ascending: sample is badly stratified
     _check_topk(api, ramp, K, V)
     _check_topk(api, -ramp, K, V)
