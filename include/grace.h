@@ -188,6 +188,29 @@ grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, int K, int V
                                int32_t* out_token, void* ws, size_t ws_bytes,
                                int32_t* d_status, void* stream);
 
+/* grace_beam_topk with the scratch memory built into the library (the paper has no counterpart:
+ * this exists for callers of this library, not for the method).
+ *
+ * For callers that cannot allocate device memory where they need the selection -- a plug-in that
+ * is handed input and output buffers only, a hot path on which the host framework forbids
+ * allocation, a process whose memory pool is already committed -- the per-request headers and
+ * candidate lists live in a fixed array inside the library's device image instead of a caller
+ * workspace.  Same arguments and results as grace_beam_topk, minus `ws`.
+ *   - Limit: B <= grace_beam_topk_static_max_requests() (32; the array is about 2 MB and every GPU
+ *     that loads the library holds it until the process exits).  A larger B returns
+ *     GRACE_WORKSPACE_TOO_SMALL and launches nothing; K and N limits are those of grace_beam_topk.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current); make that first call before any stream capture.
+ *   - The call itself allocates nothing and frees nothing.
+ *   - All calls on a device share the one array: calls that may overlap on the GPU (different
+ *     streams, or concurrent host threads) race and must be serialised by the caller.  The array
+ *     keeps the previous call's contents; the kernels rewrite everything they read, so no clearing
+ *     is needed between calls. */
+int grace_beam_topk_static_max_requests(void);
+grace_status_t grace_beam_topk_static(const float* cand, int B, int64_t N, int K, int V,
+                                      float* out_score, int32_t* out_flat, int32_t* out_parent,
+                                      int32_t* out_token, int32_t* d_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Beam-state update after top-k ("rearrangement", Sections 3.3, 4.4).  For new row i of request b:
  *   src = b*M_prev + parent[b][i]

@@ -88,6 +88,8 @@ _gtm_mask = _sig("grace_gtm_mask", _i32, [_vp, _vp, _vp, _vp, C.POINTER(TrieStru
                                          _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
 _topk_ws = _sig("grace_beam_topk_workspace_bytes", _sz, [_i32, _i64, _i32])
 _beam_topk = _sig("grace_beam_topk", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp])
+_beam_topk_static = _sig("grace_beam_topk_static", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp])
+_beam_topk_static_max = _sig("grace_beam_topk_static_max_requests", _i32, [])
 _beam_update = _sig("grace_beam_update", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct), _vp, _vp,
                                                _i32, _i32, _i32, _i32, _vp, _vp])
 _linear = _sig("grace_linear", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp])
@@ -241,6 +243,23 @@ def grace_beam_topk(cand, K: int, V: int, out_score, out_flat, out_parent, out_t
     B, N = cand.shape
     _check(_beam_topk(_dp(cand), B, N, K, V, _dp(out_score), _dp(out_flat), _dp(out_parent), _dp(out_token),
                       _dp(ws), ws.numel() * ws.element_size(), _dp(d_status), _stream()), "grace_beam_topk")
+
+
+def grace_beam_topk_static_max_requests() -> int:
+    return _beam_topk_static_max()
+
+
+def grace_beam_topk_static(cand, K: int, V: int, out_score, out_flat, out_parent, out_token, d_status=None):
+    """grace_beam_topk without a caller workspace: the scratch is a fixed array inside the library.
+
+    For callers that cannot allocate device memory at this point (buffers-only plug-ins, hot paths
+    on which allocation is forbidden).  At most grace_beam_topk_static_max_requests() requests per
+    call; calls on one device share the scratch and must not overlap on the GPU.  The first call on
+    a device should happen outside stream capture.
+    """
+    B, N = cand.shape
+    _check(_beam_topk_static(_dp(cand), B, N, K, V, _dp(out_score), _dp(out_flat), _dp(out_parent), _dp(out_token),
+                             _dp(d_status), _stream()), "grace_beam_topk_static")
 
 
 def grace_beam_update(parent, token, score, prev_node, prev_key, trie: TrieStruct, new_node, new_key,

@@ -610,3 +610,57 @@ extern "C" grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, i
                                  d_status, (cudaStream_t)stream);
 }
 
+
+
+// ---------------------------------------------------------------------------------------------
+// grace_beam_topk_static: the same selection with the scratch memory owned by the library.
+//
+// Some callers cannot allocate device memory at the point where they need a top-k: code running
+// inside a framework that forbids allocation on its hot path, a plug-in that is handed input and
+// output buffers and nothing else, a process whose memory pool is already fully committed.  For
+// them the per-request headers and candidate lists live in a fixed array in the library's own
+// device image.  The array is sized for kStaticMaxRequests requests (about 2 MB); every GPU that
+// loads the library holds it until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace grace {
+constexpr int kStaticMaxRequests = 32;
+constexpr size_t kStaticScratchBytes =
+    (size_t)kStaticMaxRequests * (sizeof(TopkHeader) + (size_t)kCap * sizeof(uint2));
+static __device__ __align__(256) unsigned char g_topk_static_scratch[kStaticScratchBytes];
+
+// In host code the name of a __device__ array is only a stand-in, not a device address: the address
+// has to be asked for, once per device, while that device is current.
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+static grace_status_t static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GRACE_CUDA_ERROR;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_topk_static_scratch) != cudaSuccess || ptr == nullptr) return GRACE_CUDA_ERROR;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return GRACE_OK;
+}
+}  // namespace grace
+
+extern "C" int grace_beam_topk_static_max_requests(void) { return grace::kStaticMaxRequests; }
+
+extern "C" grace_status_t grace_beam_topk_static(const float* cand, int B, int64_t N, int K, int V,
+                                                 float* out_score, int32_t* out_flat, int32_t* out_parent,
+                                                 int32_t* out_token, int32_t* d_status, void* stream) {
+  if (!cand || !out_score) return GRACE_INVALID_ARG;
+  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || K > N || V <= 0) return GRACE_INVALID_ARG;
+  if (K > grace::kMaxK || (N & 3)) return GRACE_UNSUPPORTED_SHAPE;
+  if (B > grace::kStaticMaxRequests) return GRACE_WORKSPACE_TOO_SMALL;     // beyond the built-in scratch
+  if (!grace_aligned16(cand)) return GRACE_INVALID_ARG;
+  void* scratch = nullptr;
+  grace_status_t st = grace::static_scratch_for_current_device(&scratch);
+  if (st != GRACE_OK) return st;
+  // The kernels (re)initialise every header word they read, so the previous call's contents do not
+  // matter; nothing here has to start at zero.
+  return grace::launch_beam_topk(cand, B, N, K, V, out_score, out_flat, out_parent, out_token, scratch, d_status,
+                                 (cudaStream_t)stream);
+}
