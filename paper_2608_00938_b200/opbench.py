@@ -31,10 +31,13 @@ def _time(fn, iters, warm=2):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "layer_norm", "log_softmax"])
+    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "mask", "layer_norm", "log_softmax"])
     for name, default in (("B", 32), ("M", 2048), ("N", 2048), ("K", 512), ("T", 1024), ("H", 8), ("d", 64),
                           ("V", 1024), ("t", 3), ("iters", 5)):
         ap.add_argument(f"--{name}", type=int, default=default)
+    ap.add_argument("--density", type=float, default=0.21, help="mask: fraction of tokens that are catalog children")
+    ap.add_argument("--fill", type=float, default=0.43, help="mask: fraction of Bloom bits set")
+    ap.add_argument("--matcher", default="bloom", choices=["none", "node", "bloom"])
     ap.add_argument("--f32out", action="store_true")
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--relu", action="store_true")
@@ -72,6 +75,35 @@ def main():
         pa, tk = torch.empty_like(fl), torch.empty_like(fl)
         us = _time(lambda: api.grace_beam_topk(cand, a.K, a.V, sc, fl, pa, tk, ws), a.iters)
         print(f"topk B={a.B} N={N} K={a.K}: {us:.1f} us, {a.B * N * 4 / us / 1e3:.0f} GB/s")
+    elif a.op == "mask":
+        # synthetic index with the statistics of a trie level: every row has its own node whose child
+        # bitmask has `density` of its bits set; the matcher bits are random with the given fill
+        R, W = a.B * a.M, a.V // 64
+        bits = torch.zeros(R, W, dtype=torch.int64, device=dev)
+        for bit in range(64):
+            bits |= (torch.rand(R, W, device=dev) < a.density).to(torch.int64) << bit
+        base = torch.arange(R, device=dev, dtype=torch.int32) * 8 + 1
+        num_nodes = int(R * 8 + a.V + 2)
+        trie = api.make_trie(bits, base, a.V, 4, num_nodes)
+        if a.matcher == "bloom":
+            words = (1 << 22) // 64
+            mb = torch.zeros(a.B, words, dtype=torch.int64, device=dev)
+            for bit in range(64):
+                mb |= (torch.rand(a.B, words, device=dev) < a.fill).to(torch.int64) << bit
+            matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, mb, 22, 4)
+        elif a.matcher == "node":
+            mb = torch.randint(-2 ** 62, 2 ** 62, (a.B, (num_nodes + 63) // 64), dtype=torch.int64, device=dev)
+            matcher = api.make_matcher(api.MATCH_NODE_BITMASK, mb)
+        else:
+            matcher = api.make_matcher(api.MATCH_NONE)
+        logp = torch.log_softmax(torch.randn(R, a.V, device=dev) * 3, dim=1)
+        score = -torch.rand(R, device=dev)
+        node = torch.arange(R, device=dev, dtype=torch.int32)
+        key = torch.randint(1, a.V, (R,), device=dev, dtype=torch.int64)
+        cand = torch.empty_like(logp)
+        us = _time(lambda: api.grace_gtm_mask(logp, score, node, key, trie, matcher, cand, None, a.B, a.M, 1), a.iters)
+        print(f"mask[{a.matcher}] R={R} V={a.V} density={a.density}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s "
+              f"(dense-form bytes)")
     elif a.op == "layer_norm":
         R = a.B * a.M
         x = torch.randn(R, a.K, device=dev)
