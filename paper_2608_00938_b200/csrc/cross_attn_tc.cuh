@@ -1,8 +1,8 @@
 // Cross-attention on tcgen05 tensor cores (Section 5.1: beams of a request are the M dimension of
 // a dense contraction against that request's shared K/V), head size 64.
 //
-// One CTA owns 128 query rows of one (request, head) and streams the encoder positions in blocks
-// of 128:
+// A work item is 128 query rows of one (request, head); its encoder positions are streamed in
+// blocks of 128:
 //   S   = Q K_blk^T        tcgen05.mma, A = Q (shared, K-major), B = K_blk (shared, K-major),
 //                          fp32 S[128 x 128] in TMEM
 //   P   = exp2(S*c - max)  256 softmax threads: TMEM lane = query row, two threads per row each
@@ -15,28 +15,32 @@
 // maps over the caller's strides, so the beam-major Q / O layout is never permuted (the view /
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
 // and masked in the softmax.  Warp roles: 0-7 softmax + epilogue, 8 TMA producer, 9 MMA issuer.
-// Two CTAs share an SM, so one CTA's MMAs run under the other's exponentials.
+// The kernel is persistent (two CTAs per SM, each looping over work items; Q is double-buffered),
+// so the next item's loads and first S overlap the current item's epilogue, and one CTA's MMAs
+// run under the other's exponentials.
 #pragma once
 #include "common.cuh"
 #include "tc.cuh"
 
 namespace grace {
 
-constexpr int kCaBM = 128;        // query rows per CTA
+constexpr int kCaBM = 128;        // query rows per work item
 constexpr int kCaBN = 128;        // encoder positions per block
 constexpr int kCaDH = 64;
 constexpr int kCaStages = 2;
 constexpr int kCaTileBytes = 128 * 64 * 2;                       // 16 KB: Q, K_blk or V_blk
 constexpr int kCaSoftmaxWarps = 8;
 constexpr int kCaThreads = (kCaSoftmaxWarps + 2) * 32;
-constexpr int kCaSmemBytes = kCaTileBytes * (1 + 2 * kCaStages) + 1024 + 256 + 2 * 2 * 128 * 4 + 2 * 128 * 4;
-constexpr uint32_t kCaTmemCols = 256;                            // S: 0..127, O_blk: 128..191, P: 192..255
+constexpr int kCaBarBytes = 256;
+constexpr int kCaSmemBytes = kCaTileBytes * (2 + 2 * kCaStages) + 1024 + kCaBarBytes + 2 * 2 * 128 * 4 + 2 * 2 * 128 * 4;
+constexpr uint32_t kCaTmemCols = 256;                            // S: 0..127, O: 128..191, P: 192..255
 
 struct CrossTcParams {
   uint16_t* out;
   float* lse;
   int64_t out_row_stride;
-  int M, H, T;
+  int B, M, H, T;
+  int tiles_m, total_items;
   float scale_log2;             // scale * log2(e)
 };
 
@@ -52,35 +56,40 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return m;
 }
 
+// Persistent kernel: a flat grid of two CTAs per SM; CTA g takes the work items g, g + gridDim.x,
+// ...  An item is one (request, head, 128-row tile); consecutive items are the tiles of the same
+// (request, head), so the CTAs running at the same time read the same K/V from L2.
 __global__ void __launch_bounds__(kCaThreads, 2)
 cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const CrossTcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* q_tile = tiles;
-  uint8_t* kv_tiles = tiles + kCaTileBytes;                      // stage s: K at 2s, V at 2s+1
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + kCaTileBytes * (1 + 2 * kCaStages));
-  uint64_t* q_full = bars;
-  uint64_t* kv_full = bars + 1;
-  uint64_t* kv_empty = kv_full + kCaStages;
+  uint8_t* q_tiles = tiles;                                      // two Q buffers
+  uint8_t* kv_tiles = tiles + 2 * kCaTileBytes;                  // stage s: K at 2s, V at 2s+1
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + kCaTileBytes * (2 + 2 * kCaStages));
+  uint64_t* q_full = bars;                    // [2]
+  uint64_t* q_empty = bars + 2;               // [2]
+  uint64_t* kv_full = bars + 4;               // [stages]
+  uint64_t* kv_empty = kv_full + kCaStages;   // [stages]
   uint64_t* s_full = kv_empty + kCaStages;
   uint64_t* p_full = s_full + 1;
   uint64_t* o_full = p_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 1);
+  uint64_t* s_free = o_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_free + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* half_max = reinterpret_cast<float*>(bars + 32);         // [2 parity][2 halves][128 rows]
-  float* half_sum = half_max + 2 * 2 * 128;                      // [2 halves][128 rows]
+  float* half_max = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + kCaBarBytes);   // [2][2][128]
+  float* half_sum = half_max + 2 * 2 * 128;                                                     // [2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * kCaBM, h = blockIdx.y, b = blockIdx.z;
   const int NB = (p.T + kCaBN - 1) / kCaBN;
 
   if (threadIdx.x == 0) {
-    tc::mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 1); }
     for (int s = 0; s < kCaStages; ++s) { tc::mbar_init(kv_full + s, 1); tc::mbar_init(kv_empty + s, 1); }
     tc::mbar_init(s_full, 1);
     tc::mbar_init(p_full, kCaSoftmaxWarps);    // one arrival per softmax warp
     tc::mbar_init(o_full, 1);
+    tc::mbar_init(s_free, kCaSoftmaxWarps);
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
@@ -90,21 +99,30 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base;           // S fp32, 128 columns
-  const uint32_t tmem_o = tmem_base + 128;     // O_blk fp32, 64 columns
+  const uint32_t tmem_o = tmem_base + 128;     // O fp32, 64 columns
   const uint32_t tmem_p = tmem_base + 192;     // P bf16 pairs, 64 columns
 
   if (warp == kCaSoftmaxWarps) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
-      tc::mbar_expect_tx(q_full, kCaTileBytes);
-      tc::tma_load_4d(q_tile, &map_q, q_full, 0, h, m0, b);
-      for (int j = 0; j < NB; ++j) {
-        const int s = j % kCaStages;
-        if (!tc::mbar_wait(kv_empty + s, ((j / kCaStages) & 1) ^ 1, abort_flag)) break;
-        tc::mbar_expect_tx(kv_full + s, 2 * kCaTileBytes);
-        tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes, &map_k, kv_full + s, 0, j * kCaBN, h, b);
-        tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, kv_full + s, 0, j * kCaBN, h, b);
+      int li = 0, g = 0;                                     // local item count, global block count
+      for (int item = blockIdx.x; item < p.total_items; item += gridDim.x, ++li) {
+        const int tile = item % p.tiles_m, bh = item / p.tiles_m;
+        const int h = bh % p.H, b = bh / p.H;
+        const int qb = li & 1;
+        if (!tc::mbar_wait(q_empty + qb, ((li >> 1) & 1) ^ 1, abort_flag)) break;
+        tc::mbar_expect_tx(q_full + qb, kCaTileBytes);
+        tc::tma_load_4d(q_tiles + qb * kCaTileBytes, &map_q, q_full + qb, 0, h, tile * kCaBM, b);
+        bool ok = true;
+        for (int j = 0; j < NB; ++j, ++g) {
+          const int s = g % kCaStages;
+          if (!tc::mbar_wait(kv_empty + s, ((g / kCaStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          tc::mbar_expect_tx(kv_full + s, 2 * kCaTileBytes);
+          tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes, &map_k, kv_full + s, 0, j * kCaBN, h, b);
+          tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, kv_full + s, 0, j * kCaBN, h, b);
+        }
+        if (!ok) break;
       }
     }
   } else if (warp == kCaSoftmaxWarps + 1) {
@@ -112,42 +130,43 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (lane == 0) {
       constexpr uint32_t idesc_s = tc::idesc_bf16(kCaBM, kCaBN, 0);     // Q K^T : B K-major
       constexpr uint32_t idesc_o = tc::idesc_bf16(kCaBM, kCaDH, 1);     // P V   : B MN-major
-      const uint32_t q_addr = tc::smem_addr(q_tile);
-      bool ok = tc::mbar_wait(q_full, 0, abort_flag) && tc::mbar_wait(kv_full + 0, 0, abort_flag);
-      if (ok) {
+      const int my_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+      const int total_blocks = my_items * NB;
+      // S of global block g: Q buffer of its item, K of ring stage g % stages
+      auto issue_s = [&](int g) -> bool {
+        const int li = g / NB, j = g - li * NB, qb = li & 1, s = g % kCaStages;
+        if (j == 0 && !tc::mbar_wait(q_full + qb, (li >> 1) & 1, abort_flag)) return false;
+        if (!tc::mbar_wait(kv_full + s, (g / kCaStages) & 1, abort_flag)) return false;
         tc::tc_fence_after();
-        const uint32_t k_addr = tc::smem_addr(kv_tiles);
+        const uint32_t q_addr = tc::smem_addr(q_tiles + qb * kCaTileBytes);
+        const uint32_t k_addr = tc::smem_addr(kv_tiles + (2 * s) * kCaTileBytes);
 #pragma unroll
         for (int k = 0; k < kCaDH / 16; ++k)
           tc::mma_ss(tmem_s, tc::smem_desc_sw128(q_addr + 32 * k, 16, 1024),
                      tc::smem_desc_sw128(k_addr + 32 * k, 16, 1024), idesc_s, k ? 1u : 0u);
         tc::mma_commit(s_full);
-      }
-      for (int j = 0; ok && j < NB; ++j) {
-        const int s = j % kCaStages;
-        if (!tc::mbar_wait(p_full, j & 1, abort_flag)) break;
-        // p_full(j) also means every softmax thread has read S of block j: S of block j+1 goes
-        // first, so the softmax threads get their next scores while P V of block j still runs.
-        // (P has its own TMEM columns, so S(j+1) cannot clobber it.)
-        if (j + 1 < NB) {
-          const int s1 = (j + 1) % kCaStages;
-          if (!tc::mbar_wait(kv_full + s1, ((j + 1) / kCaStages) & 1, abort_flag)) break;
-          tc::tc_fence_after();
-          const uint32_t k_addr = tc::smem_addr(kv_tiles + (2 * s1) * kCaTileBytes);
-#pragma unroll
-          for (int k = 0; k < kCaDH / 16; ++k)
-            tc::mma_ss(tmem_s, tc::smem_desc_sw128(q_addr + 32 * k, 16, 1024),
-                       tc::smem_desc_sw128(k_addr + 32 * k, 16, 1024), idesc_s, k ? 1u : 0u);
-          tc::mma_commit(s_full);
-        }
+        if (j == NB - 1) tc::mma_commit(q_empty + qb);       // last use of this item's Q tile
+        return true;
+      };
+      bool ok = total_blocks > 0 && issue_s(0);
+      for (int g = 0; ok && g < total_blocks; ++g) {
+        const int j = g % NB, s = g % kCaStages;
+        // s_free(g): every softmax thread holds its scores of block g in registers, so the S
+        // columns can be overwritten: S of block g+1 (possibly the next item's first block) runs
+        // on the tensor core while the exponentials of block g are computed.
+        if (!tc::mbar_wait(s_free, g & 1, abort_flag)) break;
+        if (g + 1 < total_blocks && !issue_s(g + 1)) break;
+        // p_full(g): P of block g is in its TMEM columns (and, on an item's first block, the
+        // previous item's epilogue has read O).
+        if (!tc::mbar_wait(p_full, g & 1, abort_flag)) break;
         tc::tc_fence_after();
         const uint32_t v_addr = tc::smem_addr(kv_tiles + (2 * s + 1) * kCaTileBytes);
 #pragma unroll
         for (int k = 0; k < kCaBN / 16; ++k)
           tc::mma_ts(tmem_o, tmem_p + 8 * k, tc::smem_desc_sw128(v_addr + 2048 * k, 1024, 1024), idesc_o,
-                     (j | k) ? 1u : 0u);              // O accumulates in TMEM across blocks
-        tc::mma_commit(kv_empty + s);                       // K_blk, V_blk of block j are consumed
-        tc::mma_commit(o_full);                             // O_blk of block j is complete
+                     (j | k) ? 1u : 0u);                     // O accumulates in TMEM across an item's blocks
+        tc::mma_commit(kv_empty + s);                        // K_blk, V_blk of block g are consumed
+        tc::mma_commit(o_full);                              // O includes block g
       }
     }
   } else {
@@ -160,93 +179,117 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int col_base = 64 * half;
-    const float2 scale2 = make_float2(p.scale_log2, p.scale_log2);
-    float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int j = 0; j < NB; ++j) {
-      ok = ok && tc::mbar_wait(s_full, j & 1, abort_flag);
-      ok = __all_sync(kFullMask, ok);
-      if (!ok) break;
-      tc::tc_fence_after();
-      uint32_t r[64];
-      {
-        uint32_t (&r0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
-        uint32_t (&r1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
-        tc::tmem_ld32(tmem_s + lane_addr + col_base, r0);
-        tc::tmem_ld32(tmem_s + lane_addr + col_base + 32, r1);
-        tc::tmem_ld_wait();
-      }
-      const int valid = min(kCaBN, p.T - j * kCaBN) - col_base;   // this thread's columns that exist
-      if (valid < 64) {
-#pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (i >= valid) r[i] = 0xff800000u;                     // -inf: no weight, no influence on the max
-      }
-      float mx = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
-#pragma unroll
-      for (int i = 3; i + 1 < 64; i += 2) mx = max3(mx, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-      mx = fmaxf(mx, __uint_as_float(r[63]));
-      float* hm = half_max + (j & 1) * 256;
-      hm[half * 128 + row] = mx;
-      tc::named_bar_sync(2 + quarter, 64);                  // the two warps of this row quarter
-      const float m_blk = fmaxf(mx, hm[(half ^ 1) * 128 + row]) * p.scale_log2;
-      const bool grow = m_blk > m_run + 8.0f;               // always true on the first block
-      const float m_new = grow ? m_blk : m_run;
-      const float alpha = grow ? ex2(m_run - m_new) : 1.0f; // 0 on the first block
-      m_run = m_new;
-      // probabilities -> packed bf16 in the P columns; row sum
-      const float2 neg_m2 = make_float2(-m_new, -m_new);
-      float2 sum2 = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float2 t = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), scale2, neg_m2);
-        const float2 e = make_float2(ex2(t.x), ex2(t.y));
-        sum2 = __fadd2_rn(sum2, e);
-        r[i] = pack_bf16x2(e.x, e.y);
-      }
-      l_run = fmaf(l_run, alpha, sum2.x + sum2.y);
-      if (j > 0) {
-        // P V of block j-1 reads the P columns and writes O: it must be complete before P of this
-        // block is stored and before O is rescaled.  (It was issued right after S of this block,
-        // so by now it has long finished.)
-        ok = tc::mbar_wait(o_full, (j - 1) & 1, abort_flag);
+    int g = 0, n_done = 0;
+    for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
+      const int tile = item % p.tiles_m, bh = item / p.tiles_m;
+      const int h = bh % p.H, b = bh / p.H;
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < NB; ++j, ++g) {
+        ok = ok && tc::mbar_wait(s_full, g & 1, abort_flag);
         ok = __all_sync(kFullMask, ok);
         if (!ok) break;
         tc::tc_fence_after();
-      }
-      {
-        uint32_t (&p0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[0]);
-        uint32_t (&p1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[16]);
-        tc::tmem_st16(tmem_p + lane_addr + 32 * half, p0);
-        tc::tmem_st16(tmem_p + lane_addr + 32 * half + 16, p1);
-      }
-      if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
-        uint32_t o[32];
-        tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
-        tc::tmem_ld_wait();
+        uint32_t r[64];
+        {
+          uint32_t (&r0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
+          uint32_t (&r1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
+          tc::tmem_ld32(tmem_s + lane_addr + col_base, r0);
+          tc::tmem_ld32(tmem_s + lane_addr + col_base + 32, r1);
+          tc::tmem_ld_wait();
+        }
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(s_free);              // the scores now live in registers
+        const int valid = min(kCaBN, p.T - j * kCaBN) - col_base;   // this thread's columns that exist
+        if (valid < 64) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-        uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
-        uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
-        tc::tmem_st16(tmem_o + lane_addr + 32 * half, o0);
-        tc::tmem_st16(tmem_o + lane_addr + 32 * half + 16, o1);
+          for (int i = 0; i < 64; ++i)
+            if (i >= valid) r[i] = 0xff800000u;                     // -inf: no weight, no influence on the max
+        }
+        // four independent chains instead of one 32-deep one
+        float mx0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+        float mx1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+        float mx2 = max3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+        float mx3 = max3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
+#pragma unroll
+        for (int i = 12; i + 7 < 64; i += 8) {
+          mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+          mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+          mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+        }
+        mx0 = max3(mx0, __uint_as_float(r[60]), __uint_as_float(r[61]));
+        mx1 = max3(mx1, __uint_as_float(r[62]), __uint_as_float(r[63]));
+        float mx = fmaxf(max3(mx0, mx1, mx2), mx3);
+        float* hm = half_max + (g & 1) * 256;
+        hm[half * 128 + row] = mx;
+        tc::named_bar_sync(2 + quarter, 64);                  // the two warps of this row quarter
+        const float m_blk = fmaxf(mx, hm[(half ^ 1) * 128 + row]) * p.scale_log2;
+        const bool grow = m_blk > m_run + 8.0f;               // always true on an item's first block
+        const float m_new = grow ? m_blk : m_run;
+        const float alpha = grow ? ex2(m_run - m_new) : 1.0f; // 0 on the first block
+        m_run = m_new;
+        // probabilities -> packed bf16 in the P columns; row sum in four independent accumulators
+        const float neg_m = -m_new;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float e0 = ex2(fmaf(__uint_as_float(r[4 * i]), p.scale_log2, neg_m));
+          const float e1 = ex2(fmaf(__uint_as_float(r[4 * i + 1]), p.scale_log2, neg_m));
+          const float e2 = ex2(fmaf(__uint_as_float(r[4 * i + 2]), p.scale_log2, neg_m));
+          const float e3 = ex2(fmaf(__uint_as_float(r[4 * i + 3]), p.scale_log2, neg_m));
+          s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+          r[2 * i] = pack_bf16x2(e0, e1);
+          r[2 * i + 1] = pack_bf16x2(e2, e3);
+        }
+        l_run = fmaf(l_run, alpha, (s0 + s1) + (s2 + s3));
+        if (j > 0) {
+          // P V of block j-1 reads the P columns and writes O: it must be complete before P of this
+          // block is stored and before O is rescaled.  (It was issued right after S of this block,
+          // so by now it has long finished.)
+          ok = tc::mbar_wait(o_full, (g - 1) & 1, abort_flag);
+          ok = __all_sync(kFullMask, ok);
+          if (!ok) break;
+          tc::tc_fence_after();
+        }
+        {
+          uint32_t (&p0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[0]);
+          uint32_t (&p1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[16]);
+          tc::tmem_st16(tmem_p + lane_addr + 32 * half, p0);
+          tc::tmem_st16(tmem_p + lane_addr + 32 * half + 16, p1);
+        }
+        if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
+          uint32_t o[32];
+          tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+          uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
+          uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
+          tc::tmem_st16(tmem_o + lane_addr + 32 * half, o0);
+          tc::tmem_st16(tmem_o + lane_addr + 32 * half + 16, o1);
+        }
+        tc::tmem_st_wait();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(p_full);
       }
-      tc::tmem_st_wait();
-      tc::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(p_full);
-    }
-    if (ok) ok = tc::mbar_wait(o_full, (NB - 1) & 1, abort_flag);
-    ok = __all_sync(kFullMask, ok);
-    if (ok) {
+      if (!ok) break;
+      // ---- epilogue of the item: O / l -> bf16 rows of out ----
+      ok = tc::mbar_wait(o_full, (g - 1) & 1, abort_flag);
+      ok = __all_sync(kFullMask, ok);
+      if (!ok) break;
       tc::tc_fence_after();
       uint32_t o[32];
       tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
       tc::tmem_ld_wait();
-      half_sum[half * 128 + row] = l_run;
+      float* hs = half_sum + (n_done & 1) * 256;              // double-buffered by item parity
+      hs[half * 128 + row] = l_run;
       tc::named_bar_sync(2 + quarter, 64);
-      const float l_tot = l_run + half_sum[(half ^ 1) * 128 + row];
-      const int m = m0 + row;
+      const float l_tot = l_run + hs[(half ^ 1) * 128 + row];
+      ++n_done;
+      const int m = tile * kCaBM + row;
       if (m < p.M) {
         const float inv = 1.f / l_tot;
         const int64_t r_out = (int64_t)b * p.M + m;
@@ -295,10 +338,20 @@ inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stri
     GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
     attr_set = true;
   }
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    GRACE_CUDA_TRY(cudaGetDevice(&dev));
+    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  }
   CrossTcParams p;
-  p.out = out; p.lse = lse; p.out_row_stride = out_row_stride; p.M = M; p.H = H; p.T = T_ctx;
+  p.out = out; p.lse = lse; p.out_row_stride = out_row_stride; p.B = B; p.M = M; p.H = H; p.T = T_ctx;
+  p.tiles_m = (M + kCaBM - 1) / kCaBM;
+  const int64_t items = (int64_t)p.tiles_m * H * B;
+  if (items > 0x7fffffff) return GRACE_UNSUPPORTED_SHAPE;
+  p.total_items = (int)items;
   p.scale_log2 = scale * 1.4426950408889634f;
-  dim3 grid((unsigned)((M + kCaBM - 1) / kCaBM), (unsigned)H, (unsigned)B);
+  const int grid = (int)(items < 2 * n_sm ? items : 2 * n_sm);
   cross_attn_tc_kernel<<<grid, kCaThreads, kCaSmemBytes, s>>>(mq, mk, mv, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
