@@ -11,7 +11,7 @@
 //   O  += P V_blk          tcgen05.mma, A = P (TMEM), B = V_blk (shared, read MN-major, so V is
 //                          used as stored: no transpose anywhere); O stays in TMEM for the whole
 //                          row tile and is rescaled lazily, only when a row maximum grows by > 2^8
-// K/V blocks arrive by TMA through a two-stage ring; Q, K and V are addressed with 4-D tensor
+// K and V blocks arrive by TMA through two separate two-slot rings; Q, K and V are addressed with 4-D tensor
 // maps over the caller's strides, so the beam-major Q / O layout is never permuted (the view /
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
 // and masked in the softmax.  Warp roles: 0-7 softmax + epilogue, 8 TMA producer, 9 MMA issuer.
@@ -69,9 +69,11 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + kCaTileBytes * (2 + 2 * kCaStages));
   uint64_t* q_full = bars;                    // [2]
   uint64_t* q_empty = bars + 2;               // [2]
-  uint64_t* kv_full = bars + 4;               // [stages]
-  uint64_t* kv_empty = kv_full + kCaStages;   // [stages]
-  uint64_t* s_full = kv_empty + kCaStages;
+  uint64_t* k_full = bars + 4;                // [stages]  K and V have separate rings: a K slot is
+  uint64_t* k_empty = k_full + kCaStages;     // [stages]  free once S of its block has run, a V
+  uint64_t* v_full = k_empty + kCaStages;     // [stages]  slot only after P V of its block
+  uint64_t* v_empty = v_full + kCaStages;     // [stages]
+  uint64_t* s_full = v_empty + kCaStages;
   uint64_t* p_full = s_full + 1;
   uint64_t* o_full = p_full + 1;
   uint64_t* s_free = o_full + 1;
@@ -85,7 +87,10 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) { tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 1); }
-    for (int s = 0; s < kCaStages; ++s) { tc::mbar_init(kv_full + s, 1); tc::mbar_init(kv_empty + s, 1); }
+    for (int s = 0; s < kCaStages; ++s) {
+      tc::mbar_init(k_full + s, 1); tc::mbar_init(k_empty + s, 1);
+      tc::mbar_init(v_full + s, 1); tc::mbar_init(v_empty + s, 1);
+    }
     tc::mbar_init(s_full, 1);
     tc::mbar_init(p_full, kCaSoftmaxWarps);    // one arrival per softmax warp
     tc::mbar_init(o_full, 1);
@@ -106,23 +111,50 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
-      int li = 0, g = 0;                                     // local item count, global block count
-      for (int item = blockIdx.x; item < p.total_items; item += gridDim.x, ++li) {
-        const int tile = item % p.tiles_m, bh = item / p.tiles_m;
-        const int h = bh % p.H, b = bh / p.H;
-        const int qb = li & 1;
-        if (!tc::mbar_wait(q_empty + qb, ((li >> 1) & 1) ^ 1, abort_flag)) break;
-        tc::mbar_expect_tx(q_full + qb, kCaTileBytes);
-        tc::tma_load_4d(q_tiles + qb * kCaTileBytes, &map_q, q_full + qb, 0, h, tile * kCaBM, b);
-        bool ok = true;
-        for (int j = 0; j < NB; ++j, ++g) {
-          const int s = g % kCaStages;
-          if (!tc::mbar_wait(kv_empty + s, ((g / kCaStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
-          tc::mbar_expect_tx(kv_full + s, 2 * kCaTileBytes);
-          tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes, &map_k, kv_full + s, 0, j * kCaBN, h, b);
-          tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, kv_full + s, 0, j * kCaBN, h, b);
+      // One thread feeds three queues (Q per item, K and V per block).  K of block g+2 can be
+      // requested as soon as S of block g has run, long before the V slot of block g frees, so the
+      // thread polls: whichever slot is free next gets its load, neither queue blocks the other.
+      const int my_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+      const int total_blocks = my_items * NB;
+      int gk = 0, gv = 0;                                    // next K block, next V block (global indices)
+      int idle = 0;
+      while ((gk < total_blocks || gv < total_blocks) && !*abort_flag) {
+        bool progressed = false;
+        if (gk < total_blocks) {
+          const int li = gk / NB, j = gk - li * NB, s = gk % kCaStages;
+          const int item = (int)blockIdx.x + li * (int)gridDim.x;
+          const int bh = item / p.tiles_m, h = bh % p.H, b = bh / p.H;
+          const bool need_q = (j == 0);
+          const int qb = li & 1;
+          if (tc::mbar_try_wait_now(k_empty + s, ((gk / kCaStages) & 1) ^ 1) &&
+              (!need_q || tc::mbar_try_wait_now(q_empty + qb, ((li >> 1) & 1) ^ 1))) {
+            if (need_q) {
+              tc::mbar_expect_tx(q_full + qb, kCaTileBytes);
+              tc::tma_load_4d(q_tiles + qb * kCaTileBytes, &map_q, q_full + qb, 0, h, (item % p.tiles_m) * kCaBM, b);
+            }
+            tc::mbar_expect_tx(k_full + s, kCaTileBytes);
+            tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes, &map_k, k_full + s, 0, j * kCaBN, h, b);
+            ++gk;
+            progressed = true;
+          }
         }
-        if (!ok) break;
+        if (gv < total_blocks && gv < gk) {
+          const int li = gv / NB, j = gv - li * NB, s = gv % kCaStages;
+          const int item = (int)blockIdx.x + li * (int)gridDim.x;
+          const int bh = item / p.tiles_m, h = bh % p.H, b = bh / p.H;
+          if (tc::mbar_try_wait_now(v_empty + s, ((gv / kCaStages) & 1) ^ 1)) {
+            tc::mbar_expect_tx(v_full + s, kCaTileBytes);
+            tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, v_full + s, 0, j * kCaBN, h, b);
+            ++gv;
+            progressed = true;
+          }
+        }
+        if (progressed) {
+          idle = 0;
+        } else {
+          __nanosleep(64);
+          if (++idle > (1 << 24)) *abort_flag = 1;           // bounded: about a second of nothing to do
+        }
       }
     }
   } else if (warp == kCaSoftmaxWarps + 1) {
@@ -136,7 +168,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       auto issue_s = [&](int g) -> bool {
         const int li = g / NB, j = g - li * NB, qb = li & 1, s = g % kCaStages;
         if (j == 0 && !tc::mbar_wait(q_full + qb, (li >> 1) & 1, abort_flag)) return false;
-        if (!tc::mbar_wait(kv_full + s, (g / kCaStages) & 1, abort_flag)) return false;
+        if (!tc::mbar_wait(k_full + s, (g / kCaStages) & 1, abort_flag)) return false;
         tc::tc_fence_after();
         const uint32_t q_addr = tc::smem_addr(q_tiles + qb * kCaTileBytes);
         const uint32_t k_addr = tc::smem_addr(kv_tiles + (2 * s) * kCaTileBytes);
@@ -145,6 +177,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tc::mma_ss(tmem_s, tc::smem_desc_sw128(q_addr + 32 * k, 16, 1024),
                      tc::smem_desc_sw128(k_addr + 32 * k, 16, 1024), idesc_s, k ? 1u : 0u);
         tc::mma_commit(s_full);
+        tc::mma_commit(k_empty + s);                         // K of block g is consumed
         if (j == NB - 1) tc::mma_commit(q_empty + qb);       // last use of this item's Q tile
         return true;
       };
@@ -159,13 +192,14 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // p_full(g): P of block g is in its TMEM columns (and, on an item's first block, the
         // previous item's epilogue has read O).
         if (!tc::mbar_wait(p_full, g & 1, abort_flag)) break;
+        if (!tc::mbar_wait(v_full + s, (g / kCaStages) & 1, abort_flag)) break;
         tc::tc_fence_after();
         const uint32_t v_addr = tc::smem_addr(kv_tiles + (2 * s + 1) * kCaTileBytes);
 #pragma unroll
         for (int k = 0; k < kCaBN / 16; ++k)
           tc::mma_ts(tmem_o, tmem_p + 8 * k, tc::smem_desc_sw128(v_addr + 2048 * k, 1024, 1024), idesc_o,
                      (j | k) ? 1u : 0u);                     // O accumulates in TMEM across an item's blocks
-        tc::mma_commit(kv_empty + s);                        // K_blk, V_blk of block g are consumed
+        tc::mma_commit(v_empty + s);                         // V of block g is consumed
         tc::mma_commit(o_full);                              // O includes block g
       }
     }

@@ -73,25 +73,38 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
+// One try_wait: the hardware may park the thread for up to `kSuspendNs` before answering, so a
+// waiting warp does not occupy issue slots.
+constexpr uint32_t kSuspendNs = 20000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
+  return ok != 0;
+}
+// Non-blocking test of a barrier phase (no suspend hint): for threads that poll several queues.
+__device__ __forceinline__ bool mbar_try_wait_now(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2^31 clock ticks (about a second) and reports it through
+// Bounded wait: gives up after 2^16 parked polls (about a second) and reports it through
 // `*abort_flag` (shared memory), which every later wait of the CTA checks first.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long start = clock64();
-  while (true) {
+  for (int polls = 0; polls < (1 << 16); ++polls) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - start > (1ll << 31)) { *abort_flag = 1; return false; }
   }
+  *abort_flag = 1;
+  return false;
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
