@@ -246,9 +246,15 @@ def op_breakdown(dec, cfg, reps=3):
             timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
             logp = dec.logp[:R]
             timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
-            timed("log_softmax", lambda: api.grace_log_softmax(logp))
-            timed("gtm_mask", lambda: api.grace_gtm_mask(logp, dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R],
-                                                         dec.trie, dec.matcher, logp, None, B, M, t, dec.d_status))
+            if dec.row_lse is not None:                 # the decode path fuses log-softmax into the mask kernel
+                timed("gtm_mask", lambda: api.grace_gtm_mask_logits(logp, dec.row_lse[:R], dec.score[cur][:R],
+                                                                    dec.node[cur][:R], dec.key[cur][:R], dec.trie,
+                                                                    dec.matcher, logp, None, B, M, t, dec.d_status))
+            else:
+                timed("log_softmax", lambda: api.grace_log_softmax(logp))
+                timed("gtm_mask", lambda: api.grace_gtm_mask(logp, dec.score[cur][:R], dec.node[cur][:R],
+                                                             dec.key[cur][:R], dec.trie, dec.matcher, logp, None, B, M,
+                                                             t, dec.d_status))
             par = dec.parents[t + 1]
             timed("beam_topk", lambda: api.grace_beam_topk(logp.view(B, M * V), K, V, dec.score[nxt][:B * K].view(B, K),
                                                            dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K),

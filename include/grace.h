@@ -173,6 +173,17 @@ grace_status_t grace_gtm_mask(const float* logp, const float* beam_score, const 
                               const grace_matcher_t* matcher, float* cand, uint64_t* allow_bits,
                               int B, int M, int V, int prefix_len, int32_t* d_status, void* stream);
 
+/* The same with the log-softmax fused in (Section 3.1: "a fused constraint kernel"): `logits` fp32
+ * [R][V] are raw decoder outputs; each live row is read once, normalised over the whole vocabulary
+ * (log-sum-exp written to row_lse fp32 [R] if not NULL, 0 for dead rows) and
+ *   cand[r, v] = beam_score[r] + (logits[r, v] - lse[r]) if allowed else -inf.
+ * cand may alias logits. */
+grace_status_t grace_gtm_mask_logits(const float* logits, float* row_lse, const float* beam_score,
+                                     const int32_t* beam_node, const uint64_t* beam_key,
+                                     const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                     float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                     int prefix_len, int32_t* d_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * Beam x codebook top-k (Sections 3.1, 3.3).  Per request b, the K best of cand[b][0..N)
  * under the total order (value descending, flat index ascending); -0.0 == +0.0; -inf takes
@@ -292,7 +303,9 @@ typedef struct {
   uint16_t *h;                /* [R_max][max(d_model, d_ffn)]                             */
   uint16_t *qkv;              /* [R_max][max(3*H*d_h, d_ffn)]: qkv, cross-q, FFN hidden     */
   uint16_t *attn;             /* [R_max][H*d_h]                                            */
-  float *logp;                /* [R_max][V] log-probabilities                              */
+  float *logp;                /* [R_max][V] log-probabilities; raw logits when row_lse is set */
+  float *row_lse;             /* NULL, or [R_max]: fuse log-softmax into the mask kernel; the
+                                 per-row log-sum-exp lands here (0 for dead rows)            */
   float *cand;                /* [R_max][V] masked scores; may be the same buffer as logp  */
   void *topk_ws; size_t topk_ws_bytes;
   int32_t *d_status;

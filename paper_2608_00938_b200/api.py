@@ -59,7 +59,7 @@ class DecoderStruct(C.Structure):
         ("trie", TrieStruct), ("matcher", MatcherStruct),
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
-        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("cand", _vp),
+        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -86,6 +86,8 @@ _self_attn = _sig("grace_self_attn", _i32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, 
                                            _i32, _i32, _i32, _i32, _i64, _f32, _vp, _vp])
 _gtm_mask = _sig("grace_gtm_mask", _i32, [_vp, _vp, _vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct),
                                          _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
+_gtm_mask_logits = _sig("grace_gtm_mask_logits", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct),
+                                                       C.POINTER(MatcherStruct), _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
 _topk_ws = _sig("grace_beam_topk_workspace_bytes", _sz, [_i32, _i64, _i32])
 _beam_topk = _sig("grace_beam_topk", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp])
 _beam_topk_static = _sig("grace_beam_topk_static", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp])
@@ -232,6 +234,15 @@ def grace_gtm_mask(logp, beam_score, beam_node, beam_key, trie: TrieStruct, matc
     V = logp.shape[-1]
     _check(_gtm_mask(_dp(logp), _dp(beam_score), _dp(beam_node), _dp(beam_key), C.byref(trie), C.byref(matcher),
                      _dp(cand), _dp(allow_bits), B, M, V, prefix_len, _dp(d_status), _stream()), "grace_gtm_mask")
+
+
+def grace_gtm_mask_logits(logits, row_lse, beam_score, beam_node, beam_key, trie: TrieStruct, matcher: MatcherStruct,
+                          cand, allow_bits, B: int, M: int, prefix_len: int, d_status=None):
+    """Fused log-softmax + CD/GTM mask + score add on raw logits [R, V] (V <= 2048)."""
+    V = logits.shape[-1]
+    _check(_gtm_mask_logits(_dp(logits), _dp(row_lse), _dp(beam_score), _dp(beam_node), _dp(beam_key), C.byref(trie),
+                            C.byref(matcher), _dp(cand), _dp(allow_bits), B, M, V, prefix_len, _dp(d_status),
+                            _stream()), "grace_gtm_mask_logits")
 
 
 def grace_beam_topk_workspace_bytes(B: int, N: int, K: int) -> int:

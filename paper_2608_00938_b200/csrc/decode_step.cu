@@ -93,10 +93,15 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   }
   GRACE_TRY(grace_layer_norm(d->x, d->lnf_g, d->lnf_b, d->h, R, D, d->ln_eps, stream));
   GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
-  GRACE_TRY(grace_log_softmax(d->logp, R, d->V, stream));
-  // CD + GTM mask and score add (in place when cand == logp)
-  GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->cand,
-                           nullptr, B, M, d->V, t, st, stream));
+  // log-softmax, CD + GTM mask and score add: one fused kernel when row_lse is provided
+  if (d->row_lse != nullptr) {
+    GRACE_TRY(grace_gtm_mask_logits(d->logp, d->row_lse, d->score[cur], d->node[cur], d->key[cur], &d->trie,
+                                    &d->matcher, d->cand, nullptr, B, M, d->V, t, st, stream));
+  } else {
+    GRACE_TRY(grace_log_softmax(d->logp, R, d->V, stream));
+    GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->cand,
+                             nullptr, B, M, d->V, t, st, stream));
+  }
   // parents of step t+1 live in slab t+1; tokens become the next step's input tokens
   int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
   GRACE_TRY(grace_beam_topk(d->cand, B, (int64_t)M * d->V, K, d->V, d->score[nxt], d->out_flat, parent_out,

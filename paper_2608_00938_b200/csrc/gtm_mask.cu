@@ -21,6 +21,7 @@ struct MaskParams {
   const int32_t* child_base;
   const uint64_t* matcher_bits;
   float* cand;
+  float* row_lse;            // LOGITS mode: receives log-sum-exp of each live row
   uint64_t* allow_bits;
   int32_t* d_status;
   int64_t num_internal, num_nodes, words_per_request;
@@ -53,7 +54,9 @@ constexpr int kMaskWarpsPerBlock = 8;
 //      time so that both loads are in flight together.
 //   2. the row is streamed: cand = score + logp where allowed, -inf elsewhere; a 32-byte sector of
 //      log-probabilities is read only if one of its tokens is allowed.
-template <int KIND>
+// LOGITS = true: `logp` holds raw logits; the row's log-sum-exp is taken in a first streaming pass
+// and cand = score + (logit - lse) for allowed tokens.
+template <int KIND, bool LOGITS>
 __global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
 gtm_mask_kernel(const MaskParams p) {
   __shared__ uint64_t s_words[kMaskWarpsPerBlock][32];
@@ -78,6 +81,41 @@ gtm_mask_kernel(const MaskParams p) {
   const float ninf = __int_as_float(0xff800000);
   const float* lrow = p.logp + (int64_t)r * V;
   bool saw_nan = false;
+  float lse = 0.f;
+  if (LOGITS && !dead) {
+    // one streaming pass over the row: per-lane running maximum and rescaled sum, merged across the
+    // warp at the end (the row is not kept: phase 2 re-reads only the allowed sectors, from L2)
+    float m_l = -INFINITY, s_l = 0.f;
+    const int n4 = V >> 2;
+    for (int c0 = 0; c0 < n4; c0 += 128) {
+      float4 x[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int c = c0 + u * 32 + lane;
+        x[u] = (c < n4) ? __ldg(reinterpret_cast<const float4*>(lrow) + c)
+                        : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      }
+      float mx = m_l;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) mx = fmaxf(mx, fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)));
+      if (mx > -INFINITY) {
+        float acc = s_l * expf(m_l - mx);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          acc += expf(x[u].x - mx) + expf(x[u].y - mx) + expf(x[u].z - mx) + expf(x[u].w - mx);
+        s_l = acc;
+        m_l = mx;
+      }
+    }
+    float m_w = m_l;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
+    float s_w = (m_l > -INFINITY) ? s_l * expf(m_l - m_w) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s_w += __shfl_xor_sync(kFullMask, s_w, o);
+    lse = m_w + logf(s_w);
+  }
+  if (LOGITS && lane == 0 && p.row_lse != nullptr) p.row_lse[r] = lse;
   uint64_t* words = s_words[wib];
   unsigned long long* allow = s_allow[wib];
   int* incl = s_incl[wib];
@@ -100,7 +138,28 @@ gtm_mask_kernel(const MaskParams p) {
     allow[lane] = (KIND == GRACE_MATCH_NONE) ? word : 0ull;
     __syncwarp();
 
-    if (KIND != GRACE_MATCH_NONE) {
+    if (KIND == GRACE_MATCH_NODE_BITMASK) {
+      // The children of a node have consecutive ids, so the eligibility bits of this lane's
+      // children are `pc` consecutive bits of the request's node bitmask; they are spread back
+      // onto the set bits of the child word (a software bit-deposit), one lane per word.
+      const int64_t first = (int64_t)base + rank_before_chunk + (inc - pc);
+      uint64_t elig = 0ull;
+      if (pc != 0 && first >= 0 && first + pc <= p.num_nodes) {
+        const uint64_t lo = __ldg(req_bits + (first >> 6));
+        const int sh = (int)(first & 63);
+        elig = lo >> sh;
+        if (sh != 0 && sh + pc > 64) elig |= __ldg(req_bits + (first >> 6) + 1) << (64 - sh);
+      }
+      uint64_t out = 0ull, rest = word;
+      while (rest != 0ull) {
+        const uint64_t low = rest & (0ull - rest);
+        if (elig & 1ull) out |= low;
+        elig >>= 1;
+        rest ^= low;
+      }
+      allow[lane] = out;
+      __syncwarp();
+    } else if (KIND != GRACE_MATCH_NONE) {
       for (int k0 = 0; k0 < total; k0 += 32) {
         const int k = k0 + lane;
         const bool have = k < total;
@@ -144,7 +203,10 @@ gtm_mask_kernel(const MaskParams p) {
         const uint32_t nib = (uint32_t)(allow[tok_in_chunk >> 6] >> (tok_in_chunk & 63)) & 0xfu;
         // log-probs are read only where a token of this lane is allowed
         float4 lp = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (nib != 0u) lp = __ldg(reinterpret_cast<const float4*>(lrow + (w0 << 6) + tok_in_chunk));
+        if (nib != 0u) {
+          lp = __ldg(reinterpret_cast<const float4*>(lrow + (w0 << 6) + tok_in_chunk));
+          if (LOGITS) lp = make_float4(lp.x - lse, lp.y - lse, lp.z - lse, lp.w - lse);
+        }
         const float vals[4] = {lp.x, lp.y, lp.z, lp.w};
         float outv[4];
 #pragma unroll
@@ -203,11 +265,10 @@ static bool trie_ok(const grace_trie_t* t, int V) {
          t->num_internal > 0 && t->num_nodes >= t->num_internal && t->L >= 1 && t->L <= 4;
 }
 
-extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_score,
-                                         const int32_t* beam_node, const uint64_t* beam_key,
-                                         const grace_trie_t* trie, const grace_matcher_t* matcher,
-                                         float* cand, uint64_t* allow_bits, int B, int M, int V,
-                                         int prefix_len, int32_t* d_status, void* stream) {
+static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse, const float* beam_score,
+                                  const int32_t* beam_node, const uint64_t* beam_key, const grace_trie_t* trie,
+                                  const grace_matcher_t* matcher, float* cand, uint64_t* allow_bits, int B, int M,
+                                  int V, int prefix_len, int32_t* d_status, void* stream) {
   using namespace grace;
   if (!logp || !beam_score || !beam_node || !matcher || (!cand && !allow_bits)) return GRACE_INVALID_ARG;
   if (B <= 0 || M <= 0 || (int64_t)B * M > 0x7fffffff) return GRACE_INVALID_ARG;
@@ -217,7 +278,7 @@ extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_sc
   MaskParams p;
   p.logp = logp; p.beam_score = beam_score; p.beam_node = beam_node; p.beam_key = beam_key;
   p.child_bits = trie->child_bits; p.child_base = trie->child_base;
-  p.matcher_bits = matcher->bits; p.cand = cand; p.allow_bits = allow_bits; p.d_status = d_status;
+  p.matcher_bits = matcher->bits; p.cand = cand; p.row_lse = row_lse; p.allow_bits = allow_bits; p.d_status = d_status;
   p.num_internal = trie->num_internal; p.num_nodes = trie->num_nodes;
   p.words_per_request = matcher->words_per_request;
   p.R = B * M; p.M = M; p.V = V; p.prefix_len = prefix_len;
@@ -225,13 +286,18 @@ extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_sc
   cudaStream_t s = (cudaStream_t)stream;
   const int blocks = (p.R + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock;
   const int threads = kMaskWarpsPerBlock * 32;
+#define GRACE_MASK_LAUNCH(K)                                                      \
+  do {                                                                            \
+    if (logits) gtm_mask_kernel<K, true><<<blocks, threads, 0, s>>>(p);           \
+    else gtm_mask_kernel<K, false><<<blocks, threads, 0, s>>>(p);                 \
+  } while (0)
   switch (matcher->kind) {
     case GRACE_MATCH_NONE:
-      gtm_mask_kernel<GRACE_MATCH_NONE><<<blocks, threads, 0, s>>>(p);
+      GRACE_MASK_LAUNCH(GRACE_MATCH_NONE);
       break;
     case GRACE_MATCH_NODE_BITMASK:
       if (!matcher->bits || matcher->words_per_request * 64 < trie->num_nodes) return GRACE_INVALID_ARG;
-      gtm_mask_kernel<GRACE_MATCH_NODE_BITMASK><<<blocks, threads, 0, s>>>(p);
+      GRACE_MASK_LAUNCH(GRACE_MATCH_NODE_BITMASK);
       break;
     case GRACE_MATCH_PREFIX_BLOOM:
       if (!matcher->bits || !beam_key || matcher->bloom_log2_bits < 6 || matcher->bloom_log2_bits > 32 ||
@@ -240,13 +306,32 @@ extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_sc
         return GRACE_INVALID_ARG;
       p.bloom_mask_bits = (int)(uint32_t)((1ull << matcher->bloom_log2_bits) - 1ull);
       p.bloom_hashes = matcher->bloom_hashes;
-      gtm_mask_kernel<GRACE_MATCH_PREFIX_BLOOM><<<blocks, threads, 0, s>>>(p);
+      GRACE_MASK_LAUNCH(GRACE_MATCH_PREFIX_BLOOM);
       break;
     default:
       return GRACE_INVALID_ARG;
   }
+#undef GRACE_MASK_LAUNCH
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_gtm_mask(const float* logp, const float* beam_score,
+                                         const int32_t* beam_node, const uint64_t* beam_key,
+                                         const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                         float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                         int prefix_len, int32_t* d_status, void* stream) {
+  return launch_mask(logp, false, nullptr, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B, M, V,
+                     prefix_len, d_status, stream);
+}
+
+extern "C" grace_status_t grace_gtm_mask_logits(const float* logits, float* row_lse, const float* beam_score,
+                                                const int32_t* beam_node, const uint64_t* beam_key,
+                                                const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                                float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                                int prefix_len, int32_t* d_status, void* stream) {
+  return launch_mask(logits, true, row_lse, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B, M, V,
+                     prefix_len, d_status, stream);
 }
 
 extern "C" grace_status_t grace_beam_update(const int32_t* parent, const int32_t* token, const float* score,

@@ -31,7 +31,7 @@ class Decoder:
 
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
-                 separate_cand=False):
+                 separate_cand=False, fuse_log_softmax=True):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -97,12 +97,15 @@ class Decoder:
         self.attn = torch.zeros((R_max, HD), dtype=torch.bfloat16, device=dev)
         self.logp = torch.zeros((R_max, V), dtype=torch.float32, device=dev)
         self.cand = torch.zeros((R_max, V), dtype=torch.float32, device=dev) if separate_cand else self.logp
+        # with row_lse set, `logp` keeps the raw logits and the mask kernel normalises them itself
+        self.row_lse = torch.zeros(R_max, dtype=torch.float32, device=dev) if fuse_log_softmax else None
         max_n = max(beam_sizes[t] * V for t in range(L))
         ws_bytes = api.grace_beam_topk_workspace_bytes(B, max_n, max(beam_sizes[1:]))
         self.topk_ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
         self.d_status = torch.zeros(1, dtype=torch.int32, device=dev)
         s.x, s.h, s.qkv, s.attn, s.logp, s.cand = (self.x.data_ptr(), self.h.data_ptr(), self.qkv.data_ptr(),
                                                    self.attn.data_ptr(), self.logp.data_ptr(), self.cand.data_ptr())
+        s.row_lse = None if self.row_lse is None else self.row_lse.data_ptr()
         s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()
         self.struct = s
         code = api.grace_decoder_validate(s)
@@ -128,6 +131,13 @@ class Decoder:
     def decode(self) -> None:
         for t in range(self.L):
             self.step(t)
+
+    def log_probs(self, rows: int) -> torch.Tensor:
+        """Log-probabilities of the last step's first `rows` rows (reconstructed from logits and the row
+        log-sum-exp when the log-softmax is fused into the mask kernel; needs separate_cand)."""
+        if self.row_lse is None:
+            return self.logp[:rows]
+        return self.logp[:rows] - self.row_lse[:rows, None]
 
     def results(self):
         """(sids int64 [B, K, L], score [B, K], node [B, K]) read back by following the parents."""

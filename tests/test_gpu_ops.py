@@ -88,6 +88,51 @@ def test_gtm_mask_matches_oracle(api, kind, V, L, n_sids, B, M, depth):
     assert np.array_equal(inplace.cpu().numpy().view(np.uint32), cand_ref.view(np.uint32))
 
 
+@pytest.mark.parametrize("kind", ["node", "bloom"])
+@pytest.mark.parametrize("V,M,depth", [(1024, 37, 1), (2048, 20, 1), (64, 16, 1), (1024, 50, 2)])
+def test_gtm_mask_logits_fused_log_softmax(api, kind, V, M, depth):
+    """Fused variant: raw logits in; same allow bits as the oracle (exact), candidates equal to
+    score + (logit - lse) in fp32, and the row log-sum-exp within fp32 rounding of the fp64 value."""
+    L, B, n_sids = (3, 2, 2000) if V == 64 else (4, 2, 60000)
+    sids, trie, elig, node, key, score, _ = _mask_problem(5 * V + depth, V, L, n_sids, B, M, depth)
+    node[-1] = -1
+    rng = synth.rng_for(4, 77)
+    logits = synth.normal_f32(rng, (B * M, V), 3.0)
+    z = logits.astype(np.float64)
+    lse_ref = z.max(1) + np.log(np.exp(z - z.max(1, keepdims=True)).sum(1))
+    logp_ref = (z - lse_ref[:, None]).astype(np.float32)
+    bits, base, _ = api.grace_trie_build_dense(sids, V)
+    trie_s = api.make_trie(dev(bits), dev(base), V, L, trie.num_nodes)
+    if kind == "node":
+        o_matcher = OG.NodeBitmaskMatcher(np.stack([OM.node_eligibility(trie, sids, e) for e in elig]))
+        matcher = api.make_matcher(api.MATCH_NODE_BITMASK,
+                                   dev(np.stack([api.grace_node_bitmask_build(sids, V, e, trie.num_nodes) for e in elig])))
+    else:
+        o_matcher = OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 16, 4) for e in elig])
+        matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, dev(np.stack([api.grace_bloom_build(sids, V, e, 16, 4) for e in elig])), 16, 4)
+    cand_ref, allow_ref, _ = OG.gtm_mask(logp_ref, score, node, key, depth, trie, o_matcher, B, M)
+    d_logits = dev(logits)
+    cand = torch.full((B * M, V), 7.0, device=DEV)
+    allow = torch.zeros((B * M, V // 64), dtype=torch.int64, device=DEV)
+    lse = torch.full((B * M,), -1.0, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_gtm_mask_logits(d_logits, lse, dev(score), dev(node), dev(key), trie_s, matcher, cand, allow, B, M, depth, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(host_u64(allow), OG.pack_allow_bits(allow_ref))
+    h_cand, h_lse = cand.cpu().numpy(), lse.cpu().numpy()
+    live = node >= 0
+    np.testing.assert_allclose(h_lse[live], lse_ref[live], atol=2e-5, rtol=0)
+    assert (h_lse[~live] == 0).all()
+    assert np.array_equal(np.isfinite(h_cand), allow_ref)
+    np.testing.assert_allclose(h_cand[allow_ref], cand_ref[allow_ref], atol=3e-5, rtol=0)
+    own = (score[:, None] + (logits - h_lse[:, None]))[allow_ref]                 # the kernel's own fp32 arithmetic
+    assert np.array_equal(h_cand[allow_ref].view(np.uint32), own.astype(np.float32).view(np.uint32))
+    # in place over the logits
+    api.grace_gtm_mask_logits(d_logits, None, dev(score), dev(node), dev(key), trie_s, matcher, d_logits, None, B, M, depth, status)
+    assert np.array_equal(d_logits.cpu().numpy().view(np.uint32), h_cand.view(np.uint32))
+
+
 def test_gtm_mask_flags_nan_and_bad_node(api):
     V, L = 64, 3
     sids, trie, elig, node, key, score, logp = _mask_problem(3, V, L, 500, 1, 8, 1)
