@@ -476,11 +476,21 @@ def main():
         bd = op_breakdown(dec, cfg)
         line["op_breakdown"] = bd
         top = max(bd, key=lambda k: bd[k]["ms_per_loop"])
+        # DRAM bytes per flop of the dominant kernels, from the committed ncu captures under profiles/
+        # (linear_persistent_kernel 32768x2048x512: 110.4 MB for 68.7 GFLOP; cross_attn_tc_kernel B16 M2048 T1024:
+        # 73.8 MB for 68.7 GFLOP); the bench's launches are larger than a capture may be, so the traffic is scaled
+        # by the flops of an average launch (it grows in proportion: every tile streams its operands once).
+        dram_bytes_per_flop = {"linear": 110.43e6 / 68.72e9, "cross_attn": 73.85e6 / 68.72e9}
         if top in ("linear", "cross_attn"):
             ach = bd[top]["flops_per_loop"] / (bd[top]["ms_per_loop"] * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
+            per_launch = bd[top]["flops_per_loop"] / bd[top]["calls_per_loop"]
             line["roofline"] = dict(kernel=top, bound="tensor", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
-                                    traffic=None, peak_source=f"{peaks['source']} (sustained)",
+                                    traffic=per_launch * dram_bytes_per_flop[top],
+                                    traffic_note="DRAM bytes of an average launch, scaled from the ncu capture in profiles/",
+                                    flops_per_launch=per_launch,
+                                    us_per_launch=bd[top]["ms_per_loop"] * 1e3 / bd[top]["calls_per_loop"],
+                                    peak_source=f"{peaks['source']} (sustained: kernel timed inside a long step)",
                                     launches_per_loop=bd[top]["calls_per_loop"])
         else:
             line["roofline"] = dict(kernel=top, bound="hbm", achieved=None, peak=peaks["hbm_gbs"], unit="GB/s", frac=None,
