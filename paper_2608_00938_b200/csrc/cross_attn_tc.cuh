@@ -164,43 +164,79 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       constexpr uint32_t idesc_o = tc::idesc_bf16(kCaBM, kCaDH, 1);     // P V   : B MN-major
       const int my_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
       const int total_blocks = my_items * NB;
-      // S of global block g: Q buffer of its item, K of ring stage g % stages
-      auto issue_s = [&](int g) -> bool {
-        const int li = g / NB, j = g - li * NB, qb = li & 1, s = g % kCaStages;
+      // Every operand descriptor is fixed by (Q buffer, ring slot, k-step): build them once.  The
+      // issuing thread shares its scheduler with busy softmax warps, so each instruction it does not
+      // execute per block shortens the hand-off to the tensor core.
+      uint64_t q_desc[2][kCaDH / 16], k_desc[kCaStages][kCaDH / 16], v_desc[kCaStages][kCaBN / 16];
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int k = 0; k < kCaDH / 16; ++k)
+          q_desc[i][k] = tc::smem_desc_sw128(tc::smem_addr(q_tiles + i * kCaTileBytes) + 32 * k, 16, 1024);
+#pragma unroll
+      for (int st = 0; st < kCaStages; ++st) {
+#pragma unroll
+        for (int k = 0; k < kCaDH / 16; ++k)
+          k_desc[st][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st) * kCaTileBytes) + 32 * k, 16, 1024);
+#pragma unroll
+        for (int k = 0; k < kCaBN / 16; ++k)
+          v_desc[st][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st + 1) * kCaTileBytes) + 2048 * k, 1024, 1024);
+      }
+      // S of global block g: Q buffer of its item, K of ring slot g % stages
+      auto issue_s = [&](int g, int j, int li) -> bool {
+        const int qb = li & 1, s = g % kCaStages;
         if (j == 0 && !tc::mbar_wait(q_full + qb, (li >> 1) & 1, abort_flag)) return false;
         if (!tc::mbar_wait(k_full + s, (g / kCaStages) & 1, abort_flag)) return false;
         tc::tc_fence_after();
-        const uint32_t q_addr = tc::smem_addr(q_tiles + qb * kCaTileBytes);
-        const uint32_t k_addr = tc::smem_addr(kv_tiles + (2 * s) * kCaTileBytes);
+        if (qb == 0) {
+          if (s == 0) {
 #pragma unroll
-        for (int k = 0; k < kCaDH / 16; ++k)
-          tc::mma_ss(tmem_s, tc::smem_desc_sw128(q_addr + 32 * k, 16, 1024),
-                     tc::smem_desc_sw128(k_addr + 32 * k, 16, 1024), idesc_s, k ? 1u : 0u);
+            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
+          } else {
+#pragma unroll
+            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
+          }
+        } else {
+          if (s == 0) {
+#pragma unroll
+            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
+          } else {
+#pragma unroll
+            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
+          }
+        }
         tc::mma_commit(s_full);
         tc::mma_commit(k_empty + s);                         // K of block g is consumed
         if (j == NB - 1) tc::mma_commit(q_empty + qb);       // last use of this item's Q tile
         return true;
       };
-      bool ok = total_blocks > 0 && issue_s(0);
+      static_assert(kCaStages == 2, "descriptor selection below is written for two ring slots");
+      bool ok = total_blocks > 0 && issue_s(0, 0, 0);
+      int j = 0, li = 0;                                     // block inside the item, local item index
       for (int g = 0; ok && g < total_blocks; ++g) {
-        const int j = g % NB, s = g % kCaStages;
+        const int s = g & 1;
+        int j1 = j + 1, li1 = li;
+        if (j1 == NB) { j1 = 0; ++li1; }
         // s_free(g): every softmax thread holds its scores of block g in registers, so the S
         // columns can be overwritten: S of block g+1 (possibly the next item's first block) runs
         // on the tensor core while the exponentials of block g are computed.
         if (!tc::mbar_wait(s_free, g & 1, abort_flag)) break;
-        if (g + 1 < total_blocks && !issue_s(g + 1)) break;
+        if (g + 1 < total_blocks && !issue_s(g + 1, j1, li1)) break;
         // p_full(g): P of block g is in its TMEM columns (and, on an item's first block, the
         // previous item's epilogue has read O).
         if (!tc::mbar_wait(p_full, g & 1, abort_flag)) break;
-        if (!tc::mbar_wait(v_full + s, (g / kCaStages) & 1, abort_flag)) break;
+        if (!tc::mbar_wait(v_full + s, (g >> 1) & 1, abort_flag)) break;
         tc::tc_fence_after();
-        const uint32_t v_addr = tc::smem_addr(kv_tiles + (2 * s + 1) * kCaTileBytes);
+        if (s == 0) {
 #pragma unroll
-        for (int k = 0; k < kCaBN / 16; ++k)
-          tc::mma_ts(tmem_o, tmem_p + 8 * k, tc::smem_desc_sw128(v_addr + 2048 * k, 1024, 1024), idesc_o,
-                     (j | k) ? 1u : 0u);                     // O accumulates in TMEM across an item's blocks
+          for (int k = 0; k < kCaBN / 16; ++k) tc::mma_ts(tmem_o, tmem_p + 8 * k, v_desc[0][k], idesc_o, (j | k) ? 1u : 0u);
+        } else {
+#pragma unroll
+          for (int k = 0; k < kCaBN / 16; ++k) tc::mma_ts(tmem_o, tmem_p + 8 * k, v_desc[1][k], idesc_o, (j | k) ? 1u : 0u);
+        }
         tc::mma_commit(v_empty + s);                         // V of block g is consumed
         tc::mma_commit(o_full);                              // O includes block g
+        j = j1; li = li1;
       }
     }
   } else {
