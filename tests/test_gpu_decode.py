@@ -128,3 +128,34 @@ def test_free_running_decode_emits_only_eligible_catalog_sids():
         assert (g_score[b][1:] <= g_score[b][:-1]).all()
         # weights of std 0.3 give scores down to -35: bf16 activations carry ~1% of that
         np.testing.assert_allclose(np.sort(g_score[b][valid]), np.sort(out["score"][b][out["valid"][b]]), atol=3e-2, rtol=5e-2)
+
+
+def test_whole_decode_loop_replays_from_a_cuda_graph():
+    """The decode loop enqueues kernels only (no allocation, no host synchronisation, tensor maps passed by
+    value), so all steps can be captured once into a CUDA graph and replayed (Section 5: the full fixed-length
+    decoding loop is captured as one graph).  The replay must reproduce the eager results bit for bit."""
+    cfg = _config1(B=3, matcher_kind="bloom", schedule=(1, 40, 24), final_k=32)
+    dec, api = _make_gpu_decoder(cfg, separate_cand=False)
+    dec.reset(); dec.decode()                                   # eager run (also warms every lazy attribute set-up)
+    torch.cuda.synchronize()
+    fin = dec.L & 1
+    n = cfg["B"] * cfg["final_k"]
+    eager = (dec.score[fin][:n].clone(), dec.key[fin][:n].clone(), dec.node[fin][:n].clone())
+    launches0 = api.grace_kernel_launch_count()
+    graph = torch.cuda.CUDAGraph()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            dec.reset(); dec.decode()
+    per_loop = api.grace_kernel_launch_count() - launches0
+    assert per_loop > 0
+    for buf in (dec.score[fin], dec.key[fin], dec.node[fin]):
+        buf.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert api.grace_kernel_launch_count() - launches0 == per_loop          # replays launch nothing from the host
+    assert torch.equal(dec.score[fin][:n].view(torch.int32), eager[0].view(torch.int32))
+    assert torch.equal(dec.key[fin][:n], eager[1]) and torch.equal(dec.node[fin][:n], eager[2])
+    assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
