@@ -176,3 +176,59 @@ def build_prefix_bloom(sids: np.ndarray, eligible: np.ndarray, log2_bits: int,
     for l in range(1, chosen.shape[1] + 1):
         bloom.add(prefix_keys(np.unique(chosen[:, :l], axis=0)))
     return bloom
+
+
+# ---------------------------------------------------------------------------
+# Per-node matcher index of the paper (Sections 4.2-4.4, Appendix A)
+# ---------------------------------------------------------------------------
+class NodeMatcherIndex:
+    """bitmask_index / bloom_index per child entry and the deduplicated row tables.
+
+    Every trie node stores the OR of the rows of the ads below it (Section 4.2, 4.3); a child entry
+    carries the ids of its child node's two rows in tables of unique rows (Section 4.4).  Built here
+    from the definition: for every node, OR the rows of every ad whose SID has the node's prefix.
+    """
+
+    def __init__(self, trie, sids: np.ndarray, ad_sid: np.ndarray, ad_bitmask: np.ndarray, ad_bloom: np.ndarray):
+        L = trie.sid_length
+        # rows of the SIDs (leaf level): OR over the SID's ads
+        order = np.argsort(ad_sid, kind="stable")
+        starts = np.searchsorted(ad_sid[order], np.arange(sids.shape[0]))
+        leaf_bm = np.bitwise_or.reduceat(ad_bitmask[order], starts, axis=0)
+        leaf_bl = np.bitwise_or.reduceat(ad_bloom[order], starts, axis=0)
+        node_bm = np.zeros((trie.num_nodes, ad_bitmask.shape[1]), dtype=U64)
+        node_bl = np.zeros((trie.num_nodes, ad_bloom.shape[1]), dtype=U64)
+        for l in range(L, -1, -1):
+            # SIDs are sorted, so the SIDs under the i-th prefix of level l are one contiguous run
+            if l == 0:
+                first = np.zeros(1, dtype=np.int64)
+            else:
+                change = np.any(sids[1:, :l] != sids[:-1, :l], axis=1)
+                first = np.concatenate([[0], np.nonzero(change)[0] + 1])
+            base = int(trie.level_start[l])
+            node_bm[base: base + first.shape[0]] = np.bitwise_or.reduceat(leaf_bm, first, axis=0)
+            node_bl[base: base + first.shape[0]] = np.bitwise_or.reduceat(leaf_bl, first, axis=0)
+        self.node_bitmask, self.node_bloom = node_bm, node_bl
+        child = trie.csr_child_nodes.astype(np.int64)
+        self.bitmask_table, self.bitmask_index = np.unique(node_bm[child], axis=0, return_inverse=True)
+        self.bloom_table, self.bloom_index = np.unique(node_bl[child], axis=0, return_inverse=True)
+        self.bitmask_index = self.bitmask_index.reshape(-1).astype(np.int32)
+        self.bloom_index = self.bloom_index.reshape(-1).astype(np.int32)
+
+
+class NodeRowsMatcher:
+    """TM of the paper's form for `oracle.gtm.gtm_mask`: attribute bitmask AND any-location Bloom."""
+
+    def __init__(self, trie, index: NodeMatcherIndex, user_bitmask: np.ndarray, user_blooms: np.ndarray):
+        self.trie, self.index = trie, index
+        self.user_bitmask, self.user_blooms = user_bitmask, user_blooms
+
+    def match(self, request, row_key, prefix_len, tokens, child_nodes):
+        out = np.zeros(tokens.shape[0], dtype=bool)
+        for i, child in enumerate(child_nodes):
+            j = int(child) - 1                       # child entry of node `child` (entries follow node order)
+            assert int(self.trie.csr_child_nodes[j]) == int(child)
+            bm = self.index.bitmask_table[self.index.bitmask_index[j]]
+            bl = self.index.bloom_table[self.index.bloom_index[j]]
+            out[i] = bitmask_match(bm, self.user_bitmask[request]) and bloom_any(bl, self.user_blooms[request])
+        return out

@@ -20,4 +20,8 @@ from .gen import (  # noqa: F401
     DecoderShape,
     beam_prefixes_from_sids,
     descending_scores,
+    TargetingLayout,
+    location_rows,
+    ads_for_sids,
+    request_attributes,
 )

@@ -185,3 +185,75 @@ def decoder_weights(rng: np.random.Generator, shp: DecoderShape, std: float = 0.
             "w_2": lin(d, shp.d_ffn),
         })
     return w
+
+
+# --------------------------------------------------------------------------
+# ads targeting rows (inputs of the per-node matcher form, Sections 4.2 / 4.3)
+# --------------------------------------------------------------------------
+@dataclass(frozen=True)
+class TargetingLayout:
+    """Bit layout of the packed attribute mask and the size of the Bloom rows.
+
+    attributes: (first_bit, n_values) per low-cardinality attribute, packed into W_bm 64-bit words.
+    Locations are the high-cardinality attribute: each of `n_locations` ids owns `bits_per_location`
+    fixed positions of a (64 * W_bl)-bit Bloom row (the positions are drawn once, here: turning a
+    location string into its row is outside the decode path, the rows arrive pre-built).
+    """
+    W_bm: int = 7
+    W_bl: int = 4
+    attributes: tuple = ((0, 200), (200, 8), (208, 3), (211, 40), (251, 12), (263, 100), (363, 60))
+    n_locations: int = 5000
+    bits_per_location: int = 3
+
+
+def _set_bits(rows: np.ndarray, row_ids: np.ndarray, bit_ids: np.ndarray) -> None:
+    np.bitwise_or.at(rows, (row_ids, bit_ids >> 6), np.uint64(1) << (bit_ids & 63).astype(np.uint64))
+
+
+def location_rows(rng: np.random.Generator, layout: TargetingLayout) -> np.ndarray:
+    """uint64 [n_locations, W_bl]: the Bloom row bloom(l) of every location id."""
+    rows = np.zeros((layout.n_locations, layout.W_bl), dtype=np.uint64)
+    pos = rng.integers(0, 64 * layout.W_bl, size=(layout.n_locations, layout.bits_per_location))
+    ids = np.repeat(np.arange(layout.n_locations), layout.bits_per_location)
+    _set_bits(rows, ids, pos.reshape(-1))
+    return rows
+
+
+def ads_for_sids(rng: np.random.Generator, n_sids: int, layout: TargetingLayout, loc_rows: np.ndarray):
+    """Synthetic ads under every SID (1 / 2 / 11 ads per SID at p50 / p90 / p99, like the paper's index).
+
+    Returns (ad_sid int64 [n_ads], ad_bitmask uint64 [n_ads, W_bm], ad_bloom uint64 [n_ads, W_bl]).
+    An ad allows, per attribute, either every value (probability 0.5) or 1-3 random values, and
+    targets 1-4 random locations.
+    """
+    u = rng.random(n_sids)
+    n_ads = np.where(u < 0.55, 1, np.where(u < 0.90, 2, np.where(u < 0.985, rng.integers(3, 9, n_sids),
+                                                                   rng.integers(9, 25, n_sids))))
+    ad_sid = np.repeat(np.arange(n_sids, dtype=np.int64), n_ads)
+    total = ad_sid.shape[0]
+    bm = np.zeros((total, layout.W_bm), dtype=np.uint64)
+    for first, n_values in layout.attributes:
+        everything = rng.random(total) < 0.5
+        ids = np.nonzero(everything)[0]
+        _set_bits(bm, np.repeat(ids, n_values), np.tile(first + np.arange(n_values), ids.shape[0]))
+        ids = np.nonzero(~everything)[0]
+        for _ in range(3):
+            keep = rng.random(ids.shape[0]) < (1.0 if _ == 0 else 0.5)
+            _set_bits(bm, ids[keep], first + rng.integers(0, n_values, size=int(keep.sum())))
+    bl = np.zeros((total, layout.W_bl), dtype=np.uint64)
+    for _ in range(4):
+        keep = rng.random(total) < (1.0 if _ == 0 else 0.4)
+        loc = rng.integers(0, layout.n_locations, size=int(keep.sum()))
+        bl[keep] |= loc_rows[loc]
+    return ad_sid, bm, bl
+
+
+def request_attributes(rng: np.random.Generator, B: int, layout: TargetingLayout, loc_rows: np.ndarray,
+                       n_loc: int = 64):
+    """Per request: one observed value per attribute -> uint64 [B, W_bm]; n_loc user locations ->
+    uint64 [B, n_loc, W_bl] (their Bloom rows) and the location ids int64 [B, n_loc]."""
+    ubm = np.zeros((B, layout.W_bm), dtype=np.uint64)
+    for first, n_values in layout.attributes:
+        _set_bits(ubm, np.arange(B), first + rng.integers(0, n_values, size=B))
+    loc = rng.integers(0, layout.n_locations, size=(B, n_loc))
+    return ubm, loc_rows[loc], loc

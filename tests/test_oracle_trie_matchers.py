@@ -202,3 +202,48 @@ def test_node_eligibility_is_existence_of_eligible_descendant(small):
     words = Mx.pack_node_bits(marks)
     for node in range(trie.num_nodes):
         assert ((int(words[node >> 6]) >> (node & 63)) & 1) == int(marks[node])
+
+
+def test_node_rows_index_is_the_union_over_descendant_ads_and_is_conservative():
+    """Per-node rows = OR over the ads below the node (Sections 4.2, 4.3): brute force; and the node-level
+    test never drops a prefix that has a truly eligible ad below it (it may keep more: OR-union and Bloom
+    collisions are false positives only)."""
+    V, L, n = 64, 3, 300
+    rng = synth.rng_for(4, 70)
+    sids = synth.catalog(rng, n, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout(W_bm=2, W_bl=4, attributes=((0, 20), (20, 4), (24, 30), (64, 40)),
+                                   n_locations=300, bits_per_location=3)
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n, layout, loc_rows)
+    assert np.bincount(ad_sid, minlength=n).min() >= 1
+    index = Mx.NodeMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl)
+    # brute-force union per node
+    for node in range(trie.num_nodes):
+        p = trie.prefix_of(node)
+        below = [a for a in range(ad_sid.shape[0]) if tuple(sids[ad_sid[a]][:len(p)]) == p]
+        assert np.array_equal(index.node_bitmask[node], Mx.union_rows(ad_bm[below]))
+        assert np.array_equal(index.node_bloom[node], Mx.union_rows(ad_bl[below]))
+    # the tables are deduplicated and the indices reproduce the child's rows
+    assert len({r.tobytes() for r in index.bitmask_table}) == index.bitmask_table.shape[0]
+    for j in range(trie.num_child_entries):
+        child = int(trie.csr_child_nodes[j])
+        assert np.array_equal(index.bitmask_table[index.bitmask_index[j]], index.node_bitmask[child])
+        assert np.array_equal(index.bloom_table[index.bloom_index[j]], index.node_bloom[child])
+    # conservativeness against exact ad-level matching
+    ubm, ubl, uloc = synth.request_attributes(rng, 4, layout, loc_rows, n_loc=8)
+    for b in range(4):
+        eligible_ads = [a for a in range(ad_sid.shape[0])
+                        if Mx.bitmask_match(ad_bm[a], ubm[b]) and Mx.bloom_any(ad_bl[a], ubl[b])]
+        for a in eligible_ads:
+            sid = sids[ad_sid[a]]
+            for l in range(1, L + 1):
+                node = trie.walk(sid[:l])
+                assert Mx.bitmask_match(index.node_bitmask[node], ubm[b])
+                assert Mx.bloom_any(index.node_bloom[node], ubl[b])
+        # Appendix A lookup from the root = the children whose rows pass
+        got = Mx.paper_lookup(trie, index.bitmask_index, index.bloom_index, index.bitmask_table, index.bloom_table,
+                              0, ubm[b], ubl[b])
+        want = [(int(t), int(c)) for t, c in zip(*trie.lookup(0))
+                if Mx.bitmask_match(index.node_bitmask[c], ubm[b]) and Mx.bloom_any(index.node_bloom[c], ubl[b])]
+        assert got == want
