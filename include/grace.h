@@ -185,6 +185,59 @@ grace_status_t grace_gtm_mask_logits(const float* logits, float* row_lse, const 
                                      int prefix_len, int32_t* d_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * The paper's own index form (Sections 4.2-4.4, 5.4, Appendix A): CSR child entries that carry
+ * ids of deduplicated per-node matcher rows, tested against per-request attribute rows.
+ *   node row   : OR of the rows of every ad below the node (bitmask: W_bm words, Bloom: W_bl words)
+ *   bitmask    : passes iff (row AND user_bitmask) == user_bitmask           (Section 4.2)
+ *   Bloom      : passes iff for ANY of the request's N_loc location rows q, (q AND row) == q
+ *                (Section 4.3); no location row -> no match
+ * Child entries follow node order (entry j leads to node j + 1), children of a node are sorted by
+ * token.  All pointers device.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t V, L, W_bm, W_bl, N_loc, reserved;
+  int64_t num_nodes, num_entries;
+  const int32_t* node_offsets;      /* [num_nodes + 1]                                   */
+  const int32_t* csr_child_nodes;   /* [num_entries]                                     */
+  const int16_t* csr_tokens;        /* [num_entries]                                     */
+  const int32_t* bitmask_index;     /* [num_entries] row of bitmask_table                */
+  const int32_t* bloom_index;       /* [num_entries] row of bloom_table                  */
+  const uint64_t* bitmask_table;    /* [n_bitmask_rows][W_bm]                            */
+  const uint64_t* bloom_table;      /* [n_bloom_rows][W_bl]                              */
+  const uint64_t* user_bitmask;     /* [B][W_bm]                                         */
+  const uint64_t* user_blooms;      /* [B][N_loc][W_bl]                                  */
+} grace_gtm_index_t;
+
+/* Host-side builder.  sids host int32 [n_sids][L] sorted and distinct; ads sorted by SID:
+ * ad_sid host int64 [n_ads] (index into sids, non-decreasing, every SID has at least one ad),
+ * ad_bitmask host uint64 [n_ads][W_bm], ad_bloom host uint64 [n_ads][W_bl].
+ * Outputs (host, caller-allocated): node_offsets [num_nodes+1], csr_child_nodes / csr_tokens /
+ * bitmask_index / bloom_index [num_nodes-1]; tables of unique rows.  Call once with both table
+ * pointers NULL to learn n_bitmask_rows / n_bloom_rows, then again with tables of that size. */
+grace_status_t grace_gtm_index_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                     const int64_t* ad_sid, int64_t n_ads, const uint64_t* ad_bitmask,
+                                     int W_bm, const uint64_t* ad_bloom, int W_bl,
+                                     int32_t* node_offsets, int32_t* csr_child_nodes, int16_t* csr_tokens,
+                                     int32_t* bitmask_index, int32_t* bloom_index,
+                                     uint64_t* bitmask_table, int64_t* n_bitmask_rows,
+                                     uint64_t* bloom_table, int64_t* n_bloom_rows);
+
+/* CD + GTM lookup and score add on the index above (the kernel of Section 5.4): for every beam the
+ * child-entry range of its node is scanned, bitmask first (stop at the first failing word), Bloom
+ * only for entries that pass it (stop at the first location that is contained); the request's rows
+ * are staged in shared memory once per thread block.  Outputs as grace_gtm_mask.  V <= 4096,
+ * W_bm <= 16, W_bl <= 8, N_loc <= 256. */
+grace_status_t grace_gtm_lookup(const float* logp, const float* beam_score, const int32_t* beam_node,
+                                const grace_gtm_index_t* index, float* cand, uint64_t* allow_bits,
+                                int B, int M, int32_t* d_status, void* stream);
+
+/* grace_beam_update on the CSR form: new_node = the child entry of prev_node[src] whose token matches. */
+grace_status_t grace_beam_update_csr(const int32_t* parent, const int32_t* token, const float* score,
+                                     const int32_t* prev_node, const uint64_t* prev_key,
+                                     const grace_gtm_index_t* index, int32_t* new_node, uint64_t* new_key,
+                                     int B, int K, int M_prev, int prefix_len, int32_t* d_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Beam x codebook top-k (Sections 3.1, 3.3).  Per request b, the K best of cand[b][0..N)
  * under the total order (value descending, flat index ascending); -0.0 == +0.0; -inf takes
  * part like any value.  Outputs are in that order:

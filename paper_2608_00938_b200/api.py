@@ -39,6 +39,14 @@ class MatcherStruct(C.Structure):
                 ("reserved", C.c_int32), ("words_per_request", C.c_int64), ("bits", _vp)]
 
 
+class GtmIndexStruct(C.Structure):
+    _fields_ = [("V", C.c_int32), ("L", C.c_int32), ("W_bm", C.c_int32), ("W_bl", C.c_int32), ("N_loc", C.c_int32),
+                ("reserved", C.c_int32), ("num_nodes", C.c_int64), ("num_entries", C.c_int64),
+                ("node_offsets", _vp), ("csr_child_nodes", _vp), ("csr_tokens", _vp), ("bitmask_index", _vp),
+                ("bloom_index", _vp), ("bitmask_table", _vp), ("bloom_table", _vp), ("user_bitmask", _vp),
+                ("user_blooms", _vp)]
+
+
 class LayerStruct(C.Structure):
     _fields_ = [(n, _vp) for n in (
         "ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b",
@@ -88,6 +96,11 @@ _gtm_mask = _sig("grace_gtm_mask", _i32, [_vp, _vp, _vp, _vp, C.POINTER(TrieStru
                                          _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
 _gtm_mask_logits = _sig("grace_gtm_mask_logits", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct),
                                                        C.POINTER(MatcherStruct), _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
+_gtm_index_build = _sig("grace_gtm_index_build", _i32, [_vp, _i64, _i32, _i32, _vp, _i64, _vp, _i32, _vp, _i32,
+                                                       _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
+_gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
+_beam_update_csr = _sig("grace_beam_update_csr", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp,
+                                                       _i32, _i32, _i32, _i32, _vp, _vp])
 _topk_ws = _sig("grace_beam_topk_workspace_bytes", _sz, [_i32, _i64, _i32])
 _beam_topk = _sig("grace_beam_topk", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp])
 _beam_topk_static = _sig("grace_beam_topk_static", _i32, [_vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp])
@@ -187,6 +200,64 @@ def grace_trie_walk(child_bits: np.ndarray, child_base: np.ndarray, V: int, L: i
     _check(_trie_walk(_hp(child_bits, np.uint64), _hp(child_base, np.int32), V, L, child_bits.shape[0],
                       tok.ctypes.data, tok.shape[0], C.addressof(node)), "grace_trie_walk")
     return node.value
+
+
+def grace_gtm_index_build(sids: np.ndarray, V: int, ad_sid: np.ndarray, ad_bitmask: np.ndarray, ad_bloom: np.ndarray):
+    """Host build of the paper-form index -> dict of numpy arrays (Appendix A field names)."""
+    n, L = sids.shape
+    num_nodes = int(grace_trie_count_nodes(sids, V)[-1])
+    E = num_nodes - 1
+    W_bm, W_bl = ad_bitmask.shape[1], ad_bloom.shape[1]
+    out = dict(node_offsets=np.empty(num_nodes + 1, np.int32), csr_child_nodes=np.empty(E, np.int32),
+               csr_tokens=np.empty(E, np.int16), bitmask_index=np.empty(E, np.int32), bloom_index=np.empty(E, np.int32))
+    ad_sid = np.ascontiguousarray(ad_sid, dtype=np.int64)
+    n_bm, n_bl = C.c_int64(0), C.c_int64(0)
+
+    def call(bm_table, bl_table):
+        return _gtm_index_build(_hp(sids, np.int32), n, V, L, ad_sid.ctypes.data, ad_sid.shape[0],
+                                _hp(ad_bitmask, np.uint64), W_bm, _hp(ad_bloom, np.uint64), W_bl,
+                                out["node_offsets"].ctypes.data, out["csr_child_nodes"].ctypes.data,
+                                out["csr_tokens"].ctypes.data, out["bitmask_index"].ctypes.data,
+                                out["bloom_index"].ctypes.data, bm_table, C.addressof(n_bm), bl_table, C.addressof(n_bl))
+    _check(call(None, None), "grace_gtm_index_build (sizes)")
+    out["bitmask_table"] = np.empty((n_bm.value, W_bm), np.uint64)
+    out["bloom_table"] = np.empty((n_bl.value, W_bl), np.uint64)
+    _check(call(out["bitmask_table"].ctypes.data, out["bloom_table"].ctypes.data), "grace_gtm_index_build")
+    out.update(num_nodes=num_nodes, V=V, L=L)
+    return out
+
+
+def make_gtm_index(host_index: dict, user_bitmask: np.ndarray, user_blooms: np.ndarray, device="cuda:0") -> GtmIndexStruct:
+    """Upload a host index (from grace_gtm_index_build) and the per-request rows; returns the C struct."""
+    import torch
+
+    def up(a):
+        if a.dtype == np.uint64:
+            a = a.view(np.int64)
+        return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    keep = {k: up(host_index[k]) for k in ("node_offsets", "csr_child_nodes", "csr_tokens", "bitmask_index",
+                                           "bloom_index", "bitmask_table", "bloom_table")}
+    keep["user_bitmask"], keep["user_blooms"] = up(user_bitmask), up(user_blooms)
+    s = GtmIndexStruct(host_index["V"], host_index["L"], user_bitmask.shape[1], host_index["bloom_table"].shape[1],
+                       user_blooms.shape[1], 0, host_index["num_nodes"], host_index["num_nodes"] - 1,
+                       *[keep[k].data_ptr() for k in ("node_offsets", "csr_child_nodes", "csr_tokens", "bitmask_index",
+                                                      "bloom_index", "bitmask_table", "bloom_table", "user_bitmask",
+                                                      "user_blooms")])
+    s._keepalive = keep
+    return s
+
+
+def grace_gtm_lookup(logp, beam_score, beam_node, index: GtmIndexStruct, cand, allow_bits, B: int, M: int,
+                     d_status=None):
+    _check(_gtm_lookup(_dp(logp), _dp(beam_score), _dp(beam_node), C.byref(index), _dp(cand), _dp(allow_bits), B, M,
+                       _dp(d_status), _stream()), "grace_gtm_lookup")
+
+
+def grace_beam_update_csr(parent, token, score, prev_node, prev_key, index: GtmIndexStruct, new_node, new_key,
+                          B: int, K: int, M_prev: int, prefix_len: int, d_status=None):
+    _check(_beam_update_csr(_dp(parent), _dp(token), _dp(score), _dp(prev_node), _dp(prev_key), C.byref(index),
+                            _dp(new_node), _dp(new_key), B, K, M_prev, prefix_len, _dp(d_status), _stream()),
+           "grace_beam_update_csr")
 
 
 def make_trie(child_bits_dev, child_base_dev, V: int, L: int, num_nodes: int) -> TrieStruct:

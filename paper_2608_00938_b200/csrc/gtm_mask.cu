@@ -224,6 +224,147 @@ gtm_mask_kernel(const MaskParams p) {
   if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
 }
 
+// ---------------------------------------------------------------------------------------------
+// CD + GTM lookup on the paper's index form (Sections 4.4, 5.4, Appendix A): CSR child entries
+// with ids of deduplicated per-node bitmask / Bloom rows, tested against the request's rows.
+// grid (ceil(M / 8), B): a CTA serves eight beams of ONE request, so the request's attribute
+// bitmask and its N_loc location rows are staged in shared memory once and reused by every
+// candidate of those beams.  One warp per beam; lanes take the child entries of the beam's node.
+// Evaluation order as in the paper: bitmask first (stop at the first failing word), Bloom only for
+// entries that pass, inner scan stops at the first word that is not contained, outer scan at the
+// first location that is.
+// ---------------------------------------------------------------------------------------------
+struct LookupParams {
+  const float* logp;
+  const float* beam_score;
+  const int32_t* beam_node;
+  grace_gtm_index_t idx;
+  float* cand;
+  uint64_t* allow_bits;
+  int32_t* d_status;
+  int M;
+};
+
+constexpr int kLookupMaxWords = 64;          // V <= 4096
+
+template <int WBM, int WBL>
+__global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
+gtm_lookup_kernel(const LookupParams p) {
+  extern __shared__ uint64_t s_user[];                         // [WBM] bitmask, then [N_loc][WBL]
+  __shared__ unsigned long long s_allow[kMaskWarpsPerBlock][kLookupMaxWords];
+  const grace_gtm_index_t& ix = p.idx;
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int b = blockIdx.y;
+  const int V = ix.V, W = V >> 6;
+  for (int i = threadIdx.x; i < WBM; i += blockDim.x) s_user[i] = ix.user_bitmask[(int64_t)b * WBM + i];
+  for (int i = threadIdx.x; i < ix.N_loc * WBL; i += blockDim.x)
+    s_user[WBM + i] = ix.user_blooms[(int64_t)b * ix.N_loc * WBL + i];
+  __syncthreads();
+  const int m = blockIdx.x * kMaskWarpsPerBlock + wib;
+  if (m >= p.M) return;
+  const int64_t r = (int64_t)b * p.M + m;
+  unsigned long long* allow = s_allow[wib];
+  for (int w = lane; w < W; w += 32) allow[w] = 0ull;
+  __syncwarp();
+  const int node = __ldg(p.beam_node + r);
+  bool dead = node < 0;
+  if (!dead && node >= ix.num_nodes) {
+    if (lane == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
+    dead = true;
+  }
+  if (!dead) {
+    const int start = __ldg(ix.node_offsets + node), end = __ldg(ix.node_offsets + node + 1);
+    for (int j = start + lane; j < end; j += 32) {
+      const int tok = (int)__ldg(ix.csr_tokens + j);
+      const uint64_t* bm = ix.bitmask_table + (int64_t)__ldg(ix.bitmask_index + j) * WBM;
+      bool ok = tok >= 0 && tok < V;
+#pragma unroll
+      for (int w = 0; w < WBM; ++w) {
+        if (!ok) break;
+        const uint64_t u = s_user[w];
+        ok = (__ldg(bm + w) & u) == u;
+      }
+      if (ok) {
+        const uint64_t* blp = ix.bloom_table + (int64_t)__ldg(ix.bloom_index + j) * WBL;
+        uint64_t bl[WBL];
+#pragma unroll
+        for (int w = 0; w < WBL; ++w) bl[w] = __ldg(blp + w);
+        bool any = false;
+        for (int q = 0; q < ix.N_loc && !any; ++q) {
+          const uint64_t* qr = s_user + WBM + q * WBL;
+          bool contained = true;
+#pragma unroll
+          for (int w = 0; w < WBL; ++w) {
+            if (!contained) break;
+            const uint64_t x = qr[w];
+            contained = (x & bl[w]) == x;
+          }
+          any = contained;
+        }
+        ok = any;
+      }
+      if (ok) atomicOr(&allow[tok >> 6], 1ull << (tok & 63));
+    }
+  }
+  __syncwarp();
+  const float score = __ldg(p.beam_score + r);
+  const float ninf = __int_as_float(0xff800000);
+  const float* lrow = p.logp + r * V;
+  bool saw_nan = false;
+  if (p.allow_bits != nullptr)
+    for (int w = lane; w < W; w += 32) p.allow_bits[r * W + w] = allow[w];
+  if (p.cand != nullptr) {
+    for (int g = 0; g < V; g += 128) {
+      const int tok0 = g + 4 * lane;
+      if (tok0 >= V) continue;
+      const uint32_t nib = (uint32_t)(allow[tok0 >> 6] >> (tok0 & 63)) & 0xfu;
+      float4 lp = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nib != 0u) lp = __ldg(reinterpret_cast<const float4*>(lrow + tok0));
+      const float vals[4] = {lp.x, lp.y, lp.z, lp.w};
+      float outv[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool okj = (nib >> j) & 1u;
+        outv[j] = okj ? (score + vals[j]) : ninf;
+        if (okj && vals[j] != vals[j]) saw_nan = true;
+      }
+      *reinterpret_cast<float4*>(p.cand + r * V + tok0) = make_float4(outv[0], outv[1], outv[2], outv[3]);
+    }
+  }
+  if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
+}
+
+__global__ void beam_update_csr_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ token,
+                                       const float* __restrict__ score, const int32_t* __restrict__ prev_node,
+                                       const uint64_t* __restrict__ prev_key, const grace_gtm_index_t ix,
+                                       int32_t* __restrict__ new_node, uint64_t* __restrict__ new_key, int B, int K,
+                                       int M_prev, int prefix_len, int32_t* d_status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * K) return;
+  const int b = i / K;
+  const int par = parent[i], tok = token[i];
+  if (par < 0 || par >= M_prev || tok < 0 || tok >= ix.V) {
+    flag_status(d_status, GRACE_DEV_BAD_INDEX);
+    new_node[i] = -1;
+    new_key[i] = 0;
+    return;
+  }
+  const int64_t src = (int64_t)b * M_prev + par;
+  new_key[i] = prev_key[src] | ((uint64_t)(tok + 1) << (16 * prefix_len));
+  const int node = prev_node[src];
+  int out = -1;
+  if (node >= 0 && node < ix.num_nodes && score[i] != __int_as_float(0xff800000)) {
+    int lo = ix.node_offsets[node], hi = ix.node_offsets[node + 1];       // tokens are sorted inside the range
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      const int t = (int)ix.csr_tokens[mid];
+      if (t < tok) lo = mid + 1; else hi = mid;
+    }
+    if (lo < ix.node_offsets[node + 1] && (int)ix.csr_tokens[lo] == tok) out = ix.csr_child_nodes[lo];
+  }
+  new_node[i] = out;
+}
+
 __global__ void beam_update_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict__ token,
                                    const float* __restrict__ score, const int32_t* __restrict__ prev_node,
                                    const uint64_t* __restrict__ prev_key, const uint64_t* __restrict__ child_bits,
@@ -346,6 +487,53 @@ extern "C" grace_status_t grace_beam_update(const int32_t* parent, const int32_t
   grace::beam_update_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
       parent, token, score, prev_node, prev_key, trie->child_bits, trie->child_base, trie->num_internal,
       new_node, new_key, B, K, M_prev, trie->V, prefix_len, d_status);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+static bool gtm_index_ok(const grace_gtm_index_t* ix) {
+  return ix && ix->node_offsets && ix->csr_child_nodes && ix->csr_tokens && ix->bitmask_index && ix->bloom_index &&
+         ix->bitmask_table && ix->bloom_table && ix->V > 0 && ix->V % 64 == 0 && ix->V <= 32767 && ix->L >= 1 &&
+         ix->L <= 4 && ix->num_nodes > 0 && ix->num_entries == ix->num_nodes - 1 && ix->W_bm >= 1 && ix->W_bl >= 1 &&
+         ix->N_loc >= 0;
+}
+
+extern "C" grace_status_t grace_gtm_lookup(const float* logp, const float* beam_score, const int32_t* beam_node,
+                                           const grace_gtm_index_t* index, float* cand, uint64_t* allow_bits,
+                                           int B, int M, int32_t* d_status, void* stream) {
+  using namespace grace;
+  if (!logp || !beam_score || !beam_node || (!cand && !allow_bits) || !gtm_index_ok(index)) return GRACE_INVALID_ARG;
+  if (!index->user_bitmask || (index->N_loc > 0 && !index->user_blooms)) return GRACE_INVALID_ARG;
+  if (B <= 0 || M <= 0 || B > 65535) return GRACE_INVALID_ARG;
+  if (index->V > 64 * kLookupMaxWords || index->N_loc > 256) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(logp) || (cand && !grace_aligned16(cand))) return GRACE_INVALID_ARG;
+  LookupParams p;
+  p.logp = logp; p.beam_score = beam_score; p.beam_node = beam_node; p.idx = *index; p.cand = cand;
+  p.allow_bits = allow_bits; p.d_status = d_status; p.M = M;
+  dim3 grid((unsigned)((M + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock), (unsigned)B);
+  const size_t smem = (size_t)(index->W_bm + (size_t)index->N_loc * index->W_bl) * sizeof(uint64_t);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int threads = kMaskWarpsPerBlock * 32;
+  if (index->W_bm == 7 && index->W_bl == 4) gtm_lookup_kernel<7, 4><<<grid, threads, smem, s>>>(p);
+  else if (index->W_bm == 2 && index->W_bl == 4) gtm_lookup_kernel<2, 4><<<grid, threads, smem, s>>>(p);
+  else if (index->W_bm == 1 && index->W_bl == 1) gtm_lookup_kernel<1, 1><<<grid, threads, smem, s>>>(p);
+  else if (index->W_bm == 4 && index->W_bl == 4) gtm_lookup_kernel<4, 4><<<grid, threads, smem, s>>>(p);
+  else return GRACE_UNSUPPORTED_SHAPE;      // row widths are compile-time: (7,4) as in the paper, plus (1,1), (2,4), (4,4)
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_beam_update_csr(const int32_t* parent, const int32_t* token, const float* score,
+                                                const int32_t* prev_node, const uint64_t* prev_key,
+                                                const grace_gtm_index_t* index, int32_t* new_node, uint64_t* new_key,
+                                                int B, int K, int M_prev, int prefix_len, int32_t* d_status,
+                                                void* stream) {
+  if (!parent || !token || !score || !prev_node || !prev_key || !new_node || !new_key || !gtm_index_ok(index))
+    return GRACE_INVALID_ARG;
+  if (B <= 0 || K <= 0 || M_prev <= 0 || prefix_len < 0 || prefix_len >= 4) return GRACE_INVALID_ARG;
+  const int n = B * K;
+  grace::beam_update_csr_kernel<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(
+      parent, token, score, prev_node, prev_key, *index, new_node, new_key, B, K, M_prev, prefix_len, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

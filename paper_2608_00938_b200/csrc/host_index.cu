@@ -1,6 +1,9 @@
 // Host-side index builders: dense child-bitmask trie (Section 4.4, Appendix A), per-request
 // node-eligibility bitmask and prefix Bloom filter (Section 4.1's TM in per-request form).
 // Not on the timed path.
+#include <string>
+#include <unordered_map>
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -146,6 +149,91 @@ extern "C" grace_status_t grace_trie_walk(const uint64_t* child_bits, const int3
     cur = child_base[cur] + rank;
   }
   *node = (int32_t)cur;
+  return GRACE_OK;
+}
+
+namespace {
+// Rows are deduplicated by content; ids are given in order of first appearance.
+struct RowTable {
+  int W;
+  std::unordered_map<std::string, int32_t> ids;
+  std::vector<uint64_t> rows;
+  explicit RowTable(int w) : W(w) {}
+  int32_t add(const uint64_t* row) {
+    std::string key(reinterpret_cast<const char*>(row), sizeof(uint64_t) * W);
+    auto it = ids.find(key);
+    if (it != ids.end()) return it->second;
+    const int32_t id = (int32_t)ids.size();
+    ids.emplace(std::move(key), id);
+    rows.insert(rows.end(), row, row + W);
+    return id;
+  }
+};
+}  // namespace
+
+extern "C" grace_status_t grace_gtm_index_build(const int32_t* sids, int64_t n_sids, int V, int L,
+                                                const int64_t* ad_sid, int64_t n_ads, const uint64_t* ad_bitmask,
+                                                int W_bm, const uint64_t* ad_bloom, int W_bl,
+                                                int32_t* node_offsets, int32_t* csr_child_nodes, int16_t* csr_tokens,
+                                                int32_t* bitmask_index, int32_t* bloom_index,
+                                                uint64_t* bitmask_table, int64_t* n_bitmask_rows,
+                                                uint64_t* bloom_table, int64_t* n_bloom_rows) {
+  if (!ad_sid || !ad_bitmask || !ad_bloom || !node_offsets || !csr_child_nodes || !csr_tokens || !bitmask_index ||
+      !bloom_index || !n_bitmask_rows || !n_bloom_rows || n_ads <= 0 || W_bm <= 0 || W_bl <= 0 || V > 32767)
+    return GRACE_INVALID_ARG;
+  if ((bitmask_table == nullptr) != (bloom_table == nullptr)) return GRACE_INVALID_ARG;
+  std::vector<int64_t> level_start(L + 2);
+  grace_status_t st = grace_trie_count_nodes(sids, n_sids, V, L, level_start.data());
+  if (st != GRACE_OK) return st;
+  const int64_t num_nodes = level_start[L + 1];
+  // ads: sorted by SID, every SID covered
+  for (int64_t a = 0; a < n_ads; ++a) {
+    if (ad_sid[a] < 0 || ad_sid[a] >= n_sids || (a > 0 && ad_sid[a] < ad_sid[a - 1])) return GRACE_INVALID_ARG;
+    if (a > 0 && ad_sid[a] > ad_sid[a - 1] + 1) return GRACE_INVALID_ARG;
+  }
+  if (ad_sid[0] != 0 || ad_sid[n_ads - 1] != n_sids - 1) return GRACE_INVALID_ARG;
+  // node rows: every node on the path of a SID receives the OR of that SID's ads
+  std::vector<uint64_t> node_bm((size_t)num_nodes * W_bm, 0), node_bl((size_t)num_nodes * W_bl, 0);
+  std::vector<int64_t> cur(L + 1, 0), next_id(L + 1), parent_of((size_t)num_nodes, -1);
+  std::vector<int16_t> token_of((size_t)num_nodes, 0);
+  for (int l = 0; l <= L; ++l) next_id[l] = level_start[l];
+  int64_t a = 0;
+  for (int64_t i = 0; i < n_sids; ++i) {
+    const int d = first_diff(sids, i, L);
+    for (int l = d + 1; l <= L; ++l) {
+      cur[l] = next_id[l]++;
+      parent_of[cur[l]] = cur[l - 1];
+      token_of[cur[l]] = (int16_t)sids[i * L + l - 1];
+    }
+    for (; a < n_ads && ad_sid[a] == i; ++a) {
+      for (int l = 0; l <= L; ++l) {
+        uint64_t* bm = &node_bm[(size_t)cur[l] * W_bm];
+        uint64_t* bl = &node_bl[(size_t)cur[l] * W_bl];
+        for (int w = 0; w < W_bm; ++w) bm[w] |= ad_bitmask[a * W_bm + w];
+        for (int w = 0; w < W_bl; ++w) bl[w] |= ad_bloom[a * W_bl + w];
+      }
+    }
+  }
+  // child entries in node order: entry j leads to node j + 1 (level order, lexicographic inside a level)
+  for (int64_t n = 0; n <= num_nodes; ++n) node_offsets[n] = 0;
+  for (int64_t c = 1; c < num_nodes; ++c) ++node_offsets[parent_of[c] + 1];
+  for (int64_t n = 0; n < num_nodes; ++n) node_offsets[n + 1] += node_offsets[n];
+  RowTable bm_rows(W_bm), bl_rows(W_bl);
+  for (int64_t c = 1; c < num_nodes; ++c) {
+    const int64_t j = c - 1;
+    csr_child_nodes[j] = (int32_t)c;
+    csr_tokens[j] = token_of[c];
+    bitmask_index[j] = bm_rows.add(&node_bm[(size_t)c * W_bm]);
+    bloom_index[j] = bl_rows.add(&node_bl[(size_t)c * W_bl]);
+  }
+  if (bitmask_table != nullptr) {
+    if (*n_bitmask_rows < (int64_t)bm_rows.ids.size() || *n_bloom_rows < (int64_t)bl_rows.ids.size())
+      return GRACE_WORKSPACE_TOO_SMALL;
+    std::copy(bm_rows.rows.begin(), bm_rows.rows.end(), bitmask_table);
+    std::copy(bl_rows.rows.begin(), bl_rows.rows.end(), bloom_table);
+  }
+  *n_bitmask_rows = (int64_t)bm_rows.ids.size();
+  *n_bloom_rows = (int64_t)bl_rows.ids.size();
   return GRACE_OK;
 }
 

@@ -155,6 +155,69 @@ def test_gtm_mask_flags_nan_and_bad_node(api):
 
 
 # ------------------------------------------------------------------------------------------
+# the paper's index form: CSR child entries + deduplicated per-node rows (Sections 4.2-4.4, 5.4)
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("V,L,n_sids,B,M,depth,n_loc", [
+    (64, 3, 2000, 2, 16, 1, 8), (1024, 4, 60000, 3, 37, 1, 64), (1024, 4, 60000, 2, 64, 2, 64),
+    (2048, 4, 30000, 2, 9, 0, 64), (1024, 4, 60000, 2, 20, 3, 0),
+])
+def test_gtm_lookup_paper_form_matches_oracle(api, V, L, n_sids, B, M, depth, n_loc):
+    if depth == 0:
+        M = 1
+    rng = synth.rng_for(4, 500 + V + depth)
+    sids = synth.catalog(rng, n_sids, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout()
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n_sids, layout, loc_rows)
+    ubm, ubl, _ = synth.request_attributes(rng, B, layout, loc_rows, n_loc=max(n_loc, 1))
+    if n_loc == 0:
+        ubl = ubl[:, :0]                                         # no location row: nothing may match
+    ubm[0] = 0                                                   # a request without attribute constraints
+    o_index = OM.NodeMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl)
+    # beams on random catalog prefixes of the given depth (+ a dead one)
+    node = np.full(B * M, -1, dtype=np.int32)
+    key = np.zeros(B * M, dtype=np.uint64)
+    for b in range(B):
+        pref = synth.beam_prefixes_from_sids(rng, sids, depth, M) if depth else np.zeros((1, 0), np.int32)
+        for i, pr in enumerate(pref):
+            node[b * M + i] = trie.walk(pr)
+        key[b * M: b * M + pref.shape[0]] = OM.prefix_keys(pref)
+    if M > 1:
+        node[-1] = -1
+    score = np.concatenate([synth.descending_scores(rng, M, max(depth, 1)) for _ in range(B)])
+    logp = synth.logp_rows(rng, B * M, V)
+    cand_ref, allow_ref, child_ref = OG.gtm_mask(logp, score, node, key, depth, trie,
+                                                 OM.NodeRowsMatcher(trie, o_index, ubm, ubl), B, M)
+    if n_loc == 0:
+        assert not allow_ref.any()
+    else:
+        assert allow_ref.any() and not allow_ref.all()
+    h_index = api.grace_gtm_index_build(sids, V, ad_sid, ad_bm, ad_bl)
+    index = api.make_gtm_index(h_index, ubm, np.ascontiguousarray(ubl), DEV)
+    cand = torch.full((B * M, V), 7.0, device=DEV)
+    allow = torch.zeros((B * M, V // 64), dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_gtm_lookup(dev(logp), dev(score), dev(node), index, cand, allow, B, M, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(host_u64(allow), OG.pack_allow_bits(allow_ref))
+    assert np.array_equal(cand.cpu().numpy().view(np.uint32), cand_ref.view(np.uint32))
+    # state update through the CSR form
+    K = min(32, M * V)
+    sc, flat, par, tok = OT.beam_topk(cand_ref.reshape(B, M * V), K, V)
+    node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, node, key, depth, M)
+    new_node = torch.empty(B * K, dtype=torch.int32, device=DEV)
+    new_key = torch.empty(B * K, dtype=torch.int64, device=DEV)
+    api.grace_beam_update_csr(dev(par), dev(tok), dev(sc), dev(node), dev(key), index, new_node, new_key, B, K, M,
+                              depth, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(new_node.cpu().numpy(), node_ref)
+    assert np.array_equal(host_u64(new_key), key_ref)
+
+
+# ------------------------------------------------------------------------------------------
 # beam top-k
 # ------------------------------------------------------------------------------------------
 def _run_topk(api, cand: np.ndarray, K: int, V: int):

@@ -90,3 +90,28 @@ def test_matcher_builders_match_oracle(api):
         assert np.array_equal(words, Mx.build_prefix_bloom(sids, elig, log2m, k).words)
     none = api.grace_node_bitmask_build(sids, V, np.zeros(n, bool), trie.num_nodes)
     assert not none.any()
+
+
+def test_gtm_index_builder_matches_oracle_rows(api):
+    """The library's host builder of the per-node matcher index (Appendix A layout) against the oracle's:
+    same CSR arrays; same row content behind every child entry's two indices; tables free of duplicates."""
+    V, L, n = 128, 4, 4000
+    rng = synth.rng_for(4, 80)
+    sids = synth.catalog(rng, n, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout()
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n, layout, loc_rows)
+    ref = Mx.NodeMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl)
+    got = api.grace_gtm_index_build(sids, V, ad_sid, ad_bm, ad_bl)
+    assert got["num_nodes"] == trie.num_nodes
+    assert np.array_equal(got["node_offsets"], trie.node_offsets)
+    assert np.array_equal(got["csr_child_nodes"], trie.csr_child_nodes)
+    assert np.array_equal(got["csr_tokens"], trie.csr_tokens)
+    assert np.array_equal(got["bitmask_table"][got["bitmask_index"]], ref.bitmask_table[ref.bitmask_index])
+    assert np.array_equal(got["bloom_table"][got["bloom_index"]], ref.bloom_table[ref.bloom_index])
+    assert got["bitmask_table"].shape == ref.bitmask_table.shape and got["bloom_table"].shape == ref.bloom_table.shape
+    assert len({r.tobytes() for r in got["bloom_table"]}) == got["bloom_table"].shape[0]
+    # unsorted ads are rejected
+    with pytest.raises(api.GraceError):
+        api.grace_gtm_index_build(sids, V, ad_sid[::-1].copy(), ad_bm, ad_bl)
