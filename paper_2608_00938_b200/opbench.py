@@ -31,7 +31,7 @@ def _time(fn, iters, warm=2):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "mask", "layer_norm", "log_softmax"])
+    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "mask", "lookup", "layer_norm", "log_softmax"])
     for name, default in (("B", 32), ("M", 2048), ("N", 2048), ("K", 512), ("T", 1024), ("H", 8), ("d", 64),
                           ("V", 1024), ("t", 3), ("iters", 5)):
         ap.add_argument(f"--{name}", type=int, default=default)
@@ -104,6 +104,34 @@ def main():
         us = _time(lambda: api.grace_gtm_mask(logp, score, node, key, trie, matcher, cand, None, a.B, a.M, 1), a.iters)
         print(f"mask[{a.matcher}] R={R} V={a.V} density={a.density}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s "
               f"(dense-form bytes)")
+    elif a.op == "lookup":
+        # the paper's index form on a synthetic catalog: --N SIDs (thousands), vocabulary --V, depth --t beams
+        import numpy as np
+        import synth
+        rng = synth.rng_for(4, 900)
+        n_sids, L, depth = a.N * 1000, 4, a.t
+        sids = synth.catalog(rng, n_sids, a.V, L)
+        layout = synth.TargetingLayout()
+        loc_rows = synth.location_rows(rng, layout)
+        ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n_sids, layout, loc_rows)
+        ubm, ubl, _ = synth.request_attributes(rng, a.B, layout, loc_rows, n_loc=64)
+        h = api.grace_gtm_index_build(sids, a.V, ad_sid, ad_bm, ad_bl)
+        index = api.make_gtm_index(h, ubm, np.ascontiguousarray(ubl), dev)
+        level = np.unique(sids[:, :depth], axis=0)                      # nodes of that depth, in id order
+        first = int(api.grace_trie_count_nodes(sids, a.V)[depth])
+        pick = rng.integers(0, level.shape[0], size=a.B * a.M)
+        node = torch.from_numpy((first + pick).astype(np.int32)).to(dev)
+        R = a.B * a.M
+        logp = torch.log_softmax(torch.randn(R, a.V, device=dev) * 3, dim=1)
+        score = -torch.rand(R, device=dev)
+        cand = torch.empty_like(logp)
+        allow = torch.zeros(R, a.V // 64, dtype=torch.int64, device=dev)
+        us = _time(lambda: api.grace_gtm_lookup(logp, score, node, index, cand, allow, a.B, a.M), a.iters)
+        deg = np.diff(h["node_offsets"])[first + pick].mean()
+        frac = float((allow != 0).any(dim=1).float().mean())
+        print(f"lookup R={R} V={a.V} depth={depth}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s (dense-form bytes); "
+              f"children/beam {deg:.1f}, rows with a survivor {frac:.2f}, tables {h['bitmask_table'].shape[0]} / "
+              f"{h['bloom_table'].shape[0]} unique rows for {h['num_nodes'] - 1} entries")
     elif a.op == "layer_norm":
         R = a.B * a.M
         x = torch.randn(R, a.K, device=dev)
