@@ -252,6 +252,7 @@ __global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
 gtm_lookup_kernel(const LookupParams p) {
   extern __shared__ uint64_t s_user[];                         // [WBM] bitmask, then [N_loc][WBL]
   __shared__ unsigned long long s_allow[kMaskWarpsPerBlock][kLookupMaxWords];
+  __shared__ int s_queue[kMaskWarpsPerBlock][64];
   const grace_gtm_index_t& ix = p.idx;
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int b = blockIdx.y;
@@ -274,36 +275,57 @@ gtm_lookup_kernel(const LookupParams p) {
   }
   if (!dead) {
     const int start = __ldg(ix.node_offsets + node), end = __ldg(ix.node_offsets + node + 1);
-    for (int j = start + lane; j < end; j += 32) {
-      const int tok = (int)__ldg(ix.csr_tokens + j);
-      const uint64_t* bm = ix.bitmask_table + (int64_t)__ldg(ix.bitmask_index + j) * WBM;
-      bool ok = tok >= 0 && tok < V;
+    int* queue = s_queue[wib];                 // child entries that passed the bitmask, waiting for Bloom
+    int queued = 0;
+    for (int j0 = start; j0 < end || queued > 0; j0 += 32) {
+      // ---- bitmask stage: one entry per lane, first failing word ends it ----
+      const int j = j0 + lane;
+      bool pass = false;
+      if (j < end) {
+        const uint64_t* bm = ix.bitmask_table + (int64_t)__ldg(ix.bitmask_index + j) * WBM;
+        pass = true;
 #pragma unroll
-      for (int w = 0; w < WBM; ++w) {
-        if (!ok) break;
-        const uint64_t u = s_user[w];
-        ok = (__ldg(bm + w) & u) == u;
-      }
-      if (ok) {
-        const uint64_t* blp = ix.bloom_table + (int64_t)__ldg(ix.bloom_index + j) * WBL;
-        uint64_t bl[WBL];
-#pragma unroll
-        for (int w = 0; w < WBL; ++w) bl[w] = __ldg(blp + w);
-        bool any = false;
-        for (int q = 0; q < ix.N_loc && !any; ++q) {
-          const uint64_t* qr = s_user + WBM + q * WBL;
-          bool contained = true;
-#pragma unroll
-          for (int w = 0; w < WBL; ++w) {
-            if (!contained) break;
-            const uint64_t x = qr[w];
-            contained = (x & bl[w]) == x;
-          }
-          any = contained;
+        for (int w = 0; w < WBM; ++w) {
+          if (!pass) break;
+          const uint64_t u = s_user[w];
+          pass = (__ldg(bm + w) & u) == u;
         }
-        ok = any;
       }
-      if (ok) atomicOr(&allow[tok >> 6], 1ull << (tok & 63));
+      // survivors are queued so that the (much longer) Bloom stage always runs with full warps
+      const uint32_t votes = __ballot_sync(kFullMask, pass);
+      if (pass) queue[queued + __popc(votes & ((1u << lane) - 1u))] = j;
+      queued += __popc(votes);
+      __syncwarp();
+      const bool last_round = (j0 + 32 >= end);
+      while (queued >= 32 || (last_round && queued > 0)) {
+        const int take = min(queued, 32);
+        const int e = (lane < take) ? queue[queued - take + lane] : -1;
+        queued -= take;
+        bool ok = false;
+        if (e >= 0) {
+          const uint64_t* blp = ix.bloom_table + (int64_t)__ldg(ix.bloom_index + e) * WBL;
+          uint64_t nbl[WBL];                   // complement of the candidate row: q is contained iff q & ~row == 0
+#pragma unroll
+          for (int w = 0; w < WBL; ++w) nbl[w] = ~__ldg(blp + w);
+          // ANY-of-N_loc, branch-free inside a group of eight locations, early exit between groups
+          for (int q0 = 0; q0 < ix.N_loc && !ok; q0 += 8) {
+            const int qn = min(8, ix.N_loc - q0);
+            for (int q = 0; q < qn; ++q) {
+              const uint64_t* qr = s_user + WBM + (q0 + q) * WBL;
+              uint64_t outside = 0ull;
+#pragma unroll
+              for (int w = 0; w < WBL; ++w) outside |= qr[w] & nbl[w];
+              ok = ok || (outside == 0ull);
+            }
+          }
+        }
+        if (ok) {
+          const int tok = (int)__ldg(ix.csr_tokens + e);
+          if (tok >= 0 && tok < V) atomicOr(&allow[tok >> 6], 1ull << (tok & 63));
+        }
+        __syncwarp();
+      }
+      if (j0 >= end) break;                    // only the final drain was left
     }
   }
   __syncwarp();
