@@ -56,7 +56,7 @@ def make_inputs(cfg, variant=0):
     return dict(sids=sids, elig=elig, shp=shp, weights=weights, enc_bits=enc_bits)
 
 
-def build_decoder(cfg, inp, device):
+def build_decoder(cfg, inp, device, residual_bf16=False):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -67,7 +67,8 @@ def build_decoder(cfg, inp, device):
                   d_ffn=cfg["d_ffn"], V=cfg["V"], L=cfg["L"], T_ctx=cfg["T_ctx"], B=cfg["B"],
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=inp["weights"], trie_bits=bits,
                   trie_base=base, num_nodes=num_nodes,
-                  matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device)
+                  matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
+                  residual_bf16=residual_bf16)
     return dec
 
 
@@ -236,7 +237,11 @@ def op_breakdown(dec, cfg, reps=3):
         flops[name] = flops.get(name, 0.0) + fl
         counts[name] = counts.get(name, 0) + 1
 
-    s = dec.struct
+    import torch as _t
+    if dec.x.dtype == _t.bfloat16:          # bf16 residual stream: y += x w^T by a bf16 add-reduction
+        add_into_x = lambda a, w, x: api.grace_linear_add_bf16(a, w, x)
+    else:
+        add_into_x = lambda a, w, x: api.grace_linear(a, w, x, x)
     for _ in range(reps):
         dec.reset()
         for t in range(L):
@@ -256,16 +261,16 @@ def op_breakdown(dec, cfg, reps=3):
                 timed("self_attn", lambda: api.grace_self_attn(q3.view(R, 3, H, dh), dec.k_cache[li], dec.v_cache[li],
                                                                dec.parents, sizes, attn.view(R, H, dh), B, t, scale,
                                                                dec.d_status))
-                timed("linear", lambda: api.grace_linear(attn, lay["w_o"], x, x), 2.0 * R * HD * D)
+                timed("linear", lambda: add_into_x(attn, lay["w_o"], x), 2.0 * R * HD * D)
                 timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln2_g"], lay["ln2_b"], hD))
                 timed("linear", lambda: api.grace_linear(hD, lay["w_qc"], q1), 2.0 * R * D * HD)
                 timed("cross_attn", lambda: api.grace_cross_attn(
                     q1.view(R, H, dh), dec.k_cross[li].permute(0, 2, 1, 3), dec.v_cross[li].permute(0, 2, 1, 3),
                     attn.view(R, H, dh), scale), 4.0 * R * H * dh * cfg["T_ctx"])
-                timed("linear", lambda: api.grace_linear(attn, lay["w_oc"], x, x), 2.0 * R * HD * D)
+                timed("linear", lambda: add_into_x(attn, lay["w_oc"], x), 2.0 * R * HD * D)
                 timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln3_g"], lay["ln3_b"], hD))
                 timed("linear", lambda: api.grace_linear(hD, lay["w_1"], ff, None, True), 2.0 * R * D * F)
-                timed("linear", lambda: api.grace_linear(ff, lay["w_2"], x, x), 2.0 * R * F * D)
+                timed("linear", lambda: add_into_x(ff, lay["w_2"], x), 2.0 * R * F * D)
             timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
             logp = dec.logp[:R]
             timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
@@ -440,6 +445,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-ops", action="store_true", help="skip the per-op roofline microbenchmarks")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--residual", default="bf16", choices=["bf16", "f32"],
+                    help="dtype of the residual stream between blocks (weights, activations and caches are bf16 either way)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -464,7 +471,7 @@ def main():
     peaks = load_peaks()
     cfg = dict(CFG5)
     inp = make_inputs(cfg, variant=rank)
-    dec = build_decoder(cfg, inp, device)
+    dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"))
     dec._layer_tensors = _layer_tensor_views(dec, inp)
     enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
     dec.project_cross_kv(enc_dev)
@@ -497,7 +504,8 @@ def main():
                             n_layers=cfg["n_layers"], d_model=cfg["d_model"], H=cfg["H"], d_h=cfg["d_h"],
                             d_ffn=cfg["d_ffn"], T_ctx=cfg["T_ctx"], V=cfg["V"], L=cfg["L"], catalog_sids=cfg["n_sids"],
                             matcher="prefix_bloom_2^22x4", parallelism=f"requests sharded x{world}",
-                            l2="working set ~5 GB per loop, far larger than the 126 MB L2", launch=launch_mode),
+                            l2="working set ~5 GB per loop, far larger than the 126 MB L2", launch=launch_mode,
+                            residual_stream=args.residual, accumulate="f32"),
                 launch_modes=dict(eager_ms_per_step=eager_ms, cuda_graph_ms_per_step=graph_ms),
                 step_latency_us=per_step_us, clocks=clocks, gpu_launches=int(launches_per_loop * args.steps),
                 device_status=status,

@@ -302,6 +302,12 @@ grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, i
                             uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
                             int M, int N, int K, int relu, void* stream);
 
+/* y += x @ w^T with a bf16 residual stream y [M][N] (row stride ldy): the product is accumulated in
+ * fp32, rounded to bf16 and added to y in bf16 (large problems: by a TMA add-reduction, y is never read
+ * into the SM).  Same shape and alignment rules as grace_linear. */
+grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                     uint16_t* y_inout, int64_t ldy, int M, int N, int K, void* stream);
+
 /* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
 grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
                                 uint16_t* out, int R, int D, float eps, void* stream);
@@ -309,6 +315,13 @@ grace_status_t grace_layer_norm(const float* x, const float* gamma, const float*
 /* x fp32 [R][D] = embed[token[r]] + pos (embed bf16 [V+1][D], pos bf16 [D]); token int32 [R]. */
 grace_status_t grace_embed(const int32_t* token, const uint16_t* embed, const uint16_t* pos,
                            float* x, int R, int D, int n_rows_embed, int32_t* d_status, void* stream);
+
+/* The same two with a bf16 residual stream (x bf16 [R][D]; statistics still in fp32; LayerNorm: D % 8 == 0,
+ * D <= 2048). */
+grace_status_t grace_layer_norm_bf16(const uint16_t* x, const float* gamma, const float* beta,
+                                     uint16_t* out, int R, int D, float eps, void* stream);
+grace_status_t grace_embed_bf16(const int32_t* token, const uint16_t* embed, const uint16_t* pos,
+                                uint16_t* x, int R, int D, int n_rows_embed, int32_t* d_status, void* stream);
 
 /* In place: logits fp32 [R][V] -> log-probabilities (natural log), normalised over all V. */
 grace_status_t grace_log_softmax(float* logits, int R, int V, void* stream);
@@ -352,7 +365,8 @@ typedef struct {
   int32_t *parents;           /* [L+1][R_max]; slab t+1 is written by step t               */
   int32_t *out_flat;          /* [R_max] scratch for the selected flat indices             */
   /* activations (scratch) */
-  float *x;                   /* [R_max][d_model] residual stream                         */
+  float *x;                   /* [R_max][d_model] fp32 residual stream, or NULL ...        */
+  uint16_t *x_bf16;           /* ... then [R_max][d_model] bf16 residual stream            */
   uint16_t *h;                /* [R_max][max(d_model, d_ffn)]                             */
   uint16_t *qkv;              /* [R_max][max(3*H*d_h, d_ffn)]: qkv, cross-q, FFN hidden     */
   uint16_t *attn;             /* [R_max][H*d_h]                                            */

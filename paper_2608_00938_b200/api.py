@@ -67,7 +67,7 @@ class DecoderStruct(C.Structure):
         ("trie", TrieStruct), ("matcher", MatcherStruct),
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
-        ("x", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp),
+        ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -108,6 +108,9 @@ _beam_topk_static_max = _sig("grace_beam_topk_static_max_requests", _i32, [])
 _beam_update = _sig("grace_beam_update", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct), _vp, _vp,
                                                _i32, _i32, _i32, _i32, _vp, _vp])
 _linear = _sig("grace_linear", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp])
+_linear_add_bf16 = _sig("grace_linear_add_bf16", _i32, [_vp, _i64, _vp, _i64, _vp, _i64, _i32, _i32, _i32, _vp])
+_layer_norm_bf16 = _sig("grace_layer_norm_bf16", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _f32, _vp])
+_embed_bf16 = _sig("grace_embed_bf16", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp])
 _layer_norm = _sig("grace_layer_norm", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _f32, _vp])
 _embed = _sig("grace_embed", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp])
 _log_softmax = _sig("grace_log_softmax", _i32, [_vp, _i32, _i32, _vp])
@@ -362,14 +365,34 @@ def grace_linear(x, w, y, residual=None, relu: bool = False):
     return y
 
 
+def grace_linear_add_bf16(x, w, y):
+    """y (bf16 [M, N], in place) += x @ w.T."""
+    M, K = x.shape
+    N = w.shape[0]
+    _check(_linear_add_bf16(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), _dp(y), y.stride(0), M, N, K, _stream()),
+           "grace_linear_add_bf16")
+    return y
+
+
 def grace_layer_norm(x, gamma, beta, out, eps: float = 1e-5):
+    """x fp32 or bf16 [R, D] -> out bf16."""
+    import torch
     R, D = x.shape
+    if x.dtype == torch.bfloat16:
+        _check(_layer_norm_bf16(_dp(x), _dp(gamma), _dp(beta), _dp(out), R, D, eps, _stream()), "grace_layer_norm_bf16")
+        return out
     _check(_layer_norm(_dp(x), _dp(gamma), _dp(beta), _dp(out), R, D, eps, _stream()), "grace_layer_norm")
     return out
 
 
 def grace_embed(token, embed, pos, x, d_status=None):
+    """x fp32 or bf16 [R, D] = embed[token] + pos."""
+    import torch
     R, D = x.shape
+    if x.dtype == torch.bfloat16:
+        _check(_embed_bf16(_dp(token), _dp(embed), _dp(pos), _dp(x), R, D, embed.shape[0], _dp(d_status), _stream()),
+               "grace_embed_bf16")
+        return x
     _check(_embed(_dp(token), _dp(embed), _dp(pos), _dp(x), R, D, embed.shape[0], _dp(d_status), _stream()),
            "grace_embed")
     return x

@@ -27,7 +27,7 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
         !w.w_oc || !w.w_1 || !w.w_2 || !w.k_cross || !w.v_cross || !w.k_cache || !w.v_cache)
       return GRACE_INVALID_ARG;
   }
-  if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || !d->x || !d->h || !d->qkv ||
+  if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || (!d->x && !d->x_bf16) || !d->h || !d->qkv ||
       !d->attn || !d->logp || !d->cand || !d->topk_ws || !d->out_flat)
     return GRACE_INVALID_ARG;
   for (int i = 0; i < 2; ++i)
@@ -71,27 +71,38 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   const float scale = 1.0f / sqrtf((float)d->d_h);
   int32_t* st = d->d_status;
 
-  GRACE_TRY(grace_embed(d->token[cur], d->embed, d->pos + (int64_t)t * D, d->x, R, D, d->V + 1, st, stream));
+  // residual stream: fp32 (x) or bf16 (x_bf16)
+  const bool xb = (d->x == nullptr);
+  auto layer_norm = [&](const float* g, const float* b) -> grace_status_t {
+    return xb ? grace_layer_norm_bf16(d->x_bf16, g, b, d->h, R, D, d->ln_eps, stream)
+              : grace_layer_norm(d->x, g, b, d->h, R, D, d->ln_eps, stream);
+  };
+  auto add_into_x = [&](const uint16_t* a, int64_t lda, const uint16_t* w, int K) -> grace_status_t {
+    return xb ? grace_linear_add_bf16(a, lda, w, K, d->x_bf16, D, R, D, K, stream)
+              : grace_linear(a, lda, w, K, nullptr, d->x, D, d->x, R, D, K, 0, stream);
+  };
+  if (xb) GRACE_TRY(grace_embed_bf16(d->token[cur], d->embed, d->pos + (int64_t)t * D, d->x_bf16, R, D, d->V + 1, st, stream));
+  else GRACE_TRY(grace_embed(d->token[cur], d->embed, d->pos + (int64_t)t * D, d->x, R, D, d->V + 1, st, stream));
   for (int l = 0; l < d->n_layers; ++l) {
     const grace_layer_t& w = d->layers[l];
     // self-attention block
-    GRACE_TRY(grace_layer_norm(d->x, w.ln1_g, w.ln1_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(layer_norm(w.ln1_g, w.ln1_b));
     GRACE_TRY(grace_linear(d->h, D, w.w_qkv, D, d->qkv, nullptr, 3 * HD, nullptr, R, 3 * HD, D, 0, stream));
     GRACE_TRY(grace_self_attn(d->qkv, 3 * HD, w.k_cache, w.v_cache, d->parents, d->beam_sizes, d->attn, HD,
                               B, t, d->H, d->d_h, d->R_max, scale, st, stream));
-    GRACE_TRY(grace_linear(d->attn, HD, w.w_o, HD, nullptr, d->x, D, d->x, R, D, HD, 0, stream));
+    GRACE_TRY(add_into_x(d->attn, HD, w.w_o, HD));
     // cross-attention block
-    GRACE_TRY(grace_layer_norm(d->x, w.ln2_g, w.ln2_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(layer_norm(w.ln2_g, w.ln2_b));
     GRACE_TRY(grace_linear(d->h, D, w.w_qc, D, d->qkv, nullptr, HD, nullptr, R, HD, D, 0, stream));
     GRACE_TRY(grace_cross_attn(d->qkv, HD, w.k_cross, w.v_cross, (int64_t)d->T_ctx * HD, d->d_h, HD, d->attn, HD,
                                nullptr, B, M, d->H, d->d_h, d->T_ctx, scale, st, stream));
-    GRACE_TRY(grace_linear(d->attn, HD, w.w_oc, HD, nullptr, d->x, D, d->x, R, D, HD, 0, stream));
+    GRACE_TRY(add_into_x(d->attn, HD, w.w_oc, HD));
     // feed-forward block
-    GRACE_TRY(grace_layer_norm(d->x, w.ln3_g, w.ln3_b, d->h, R, D, d->ln_eps, stream));
+    GRACE_TRY(layer_norm(w.ln3_g, w.ln3_b));
     GRACE_TRY(grace_linear(d->h, D, w.w_1, D, d->qkv, nullptr, d->d_ffn, nullptr, R, d->d_ffn, D, 1, stream));
-    GRACE_TRY(grace_linear(d->qkv, d->d_ffn, w.w_2, d->d_ffn, nullptr, d->x, D, d->x, R, D, d->d_ffn, 0, stream));
+    GRACE_TRY(add_into_x(d->qkv, d->d_ffn, w.w_2, d->d_ffn));
   }
-  GRACE_TRY(grace_layer_norm(d->x, d->lnf_g, d->lnf_b, d->h, R, D, d->ln_eps, stream));
+  GRACE_TRY(layer_norm(d->lnf_g, d->lnf_b));
   GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
   // log-softmax, CD + GTM mask and score add: one fused kernel when row_lse is provided
   if (d->row_lse != nullptr) {

@@ -61,6 +61,111 @@ layer_norm_kernel(const float* __restrict__ x, const float* __restrict__ gamma, 
   }
 }
 
+// bf16 residual stream: x bf16 [R][D] -> out bf16 [R][D]; D % 8 == 0, D <= 2048.  A warp takes ROWS rows at a
+// time and issues all of their 16-byte loads before the first reduction (a 1 KB row alone keeps too few bytes
+// in flight); the packed values stay in registers and are unpacked once per pass.
+template <int MAXV, int ROWS>   // MAXV: 16-byte pieces (8 bf16) per lane and row
+__global__ void __launch_bounds__(128)
+layer_norm_bf16_kernel(const uint16_t* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                       uint16_t* __restrict__ out, int R, int D, float eps) {
+  const int lane = threadIdx.x & 31;
+  const int r0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
+  if (r0 >= R) return;
+  const int n8 = D >> 3;
+  uint4 raw[ROWS][MAXV];
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    const uint4* row = reinterpret_cast<const uint4*>(x + (int64_t)(r0 + j) * D);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = i * 32 + lane;
+      raw[j][i] = (c < n8 && r0 + j < R) ? ld_stream_u4(row + c) : make_uint4(0, 0, 0, 0);
+    }
+  }
+  // statistics and normalisation on packed fp32 pairs (the kernel is issue-bound otherwise)
+  float mean[ROWS], rstd[ROWS];
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    f32x2_t acc = f2_pack(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const uint4 t = raw[j][i];
+      acc = f2_add(acc, f2_add(f2_add(f2_from_bf16x2(t.x), f2_from_bf16x2(t.y)),
+                               f2_add(f2_from_bf16x2(t.z), f2_from_bf16x2(t.w))));
+    }
+    float lo, hi;
+    f2_unpack(acc, lo, hi);
+    mean[j] = warp_sum(lo + hi) / (float)D;
+  }
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    const f32x2_t m2 = f2_pack(mean[j], mean[j]);
+    f32x2_t acc = f2_pack(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      if (i * 32 + lane < n8) {
+        const uint4 t = raw[j][i];
+        const uint32_t w4[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const f32x2_t d = f2_sub(f2_from_bf16x2(w4[e]), m2);
+          acc = f2_fma(d, d, acc);
+        }
+      }
+    }
+    float lo, hi;
+    f2_unpack(acc, lo, hi);
+    rstd[j] = rsqrtf(warp_sum(lo + hi) / (float)D + eps);
+  }
+#pragma unroll
+  for (int i = 0; i < MAXV; ++i) {
+    const int c = i * 32 + lane;
+    if (c < n8) {
+      const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c), g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * c + 1);
+      const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c), b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * c + 1);
+      const f32x2_t g[4] = {f2_pack(g0.x, g0.y), f2_pack(g0.z, g0.w), f2_pack(g1.x, g1.y), f2_pack(g1.z, g1.w)};
+      const f32x2_t bb[4] = {f2_pack(b0.x, b0.y), f2_pack(b0.z, b0.w), f2_pack(b1.x, b1.y), f2_pack(b1.z, b1.w)};
+#pragma unroll
+      for (int j = 0; j < ROWS; ++j) {
+        if (r0 + j < R) {
+          const uint4 t = raw[j][i];
+          const uint32_t w4[4] = {t.x, t.y, t.z, t.w};
+          const f32x2_t m2 = f2_pack(mean[j], mean[j]), r2 = f2_pack(rstd[j], rstd[j]);
+          uint32_t o4[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float lo, hi;
+            f2_unpack(f2_fma(f2_mul(f2_sub(f2_from_bf16x2(w4[e]), m2), r2), g[e], bb[e]), lo, hi);
+            o4[e] = pack_bf16x2(lo, hi);
+          }
+          reinterpret_cast<uint4*>(out + (int64_t)(r0 + j) * D)[c] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        }
+      }
+    }
+  }
+}
+
+__global__ void embed_bf16_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
+                                  const uint16_t* __restrict__ pos, uint16_t* __restrict__ x, int R, int D,
+                                  int n_rows_embed, int32_t* d_status) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= R) return;
+  int tok = __ldg(token + r);
+  if (tok < 0 || tok >= n_rows_embed) {
+    if (lane == 0) flag_status(d_status, GRACE_DEV_BAD_INDEX);
+    tok = 0;
+  }
+  const uint2* erow = reinterpret_cast<const uint2*>(embed + (int64_t)tok * D);
+  const uint2* prow = reinterpret_cast<const uint2*>(pos);
+  uint2* xrow = reinterpret_cast<uint2*>(x + (int64_t)r * D);
+  for (int c = lane; c < (D >> 2); c += 32) {
+    const uint2 e = __ldg(erow + c), p = __ldg(prow + c);
+    xrow[c] = make_uint2(pack_bf16x2(bf16_lo(e.x) + bf16_lo(p.x), bf16_hi(e.x) + bf16_hi(p.x)),
+                         pack_bf16x2(bf16_lo(e.y) + bf16_lo(p.y), bf16_hi(e.y) + bf16_hi(p.y)));
+  }
+}
+
 __global__ void embed_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
                              const uint16_t* __restrict__ pos, float* __restrict__ x, int R, int D,
                              int n_rows_embed, int32_t* d_status) {
@@ -169,6 +274,37 @@ extern "C" grace_status_t grace_log_softmax(float* logits, int R, int V, void* s
   else if (pieces <= 4) log_softmax_kernel<4><<<R, 256, 0, s>>>(logits, R, V);
   else if (pieces <= 8) log_softmax_kernel<8><<<R, 256, 0, s>>>(logits, R, V);
   else log_softmax_kernel<16><<<R, 256, 0, s>>>(logits, R, V);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_layer_norm_bf16(const uint16_t* x, const float* gamma, const float* beta,
+                                                uint16_t* out, int R, int D, float eps, void* stream) {
+  using namespace grace;
+  if (!x || !gamma || !beta || !out || R <= 0 || D <= 0) return GRACE_INVALID_ARG;
+  if ((D & 7) || D > 2048) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(x) || !grace_aligned16(gamma) || !grace_aligned16(beta) || !grace_aligned16(out))
+    return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int pieces = ((D >> 3) + 31) / 32;
+  auto blocks = [&](int rows) { return (R + 4 * rows - 1) / (4 * rows); };
+  if (pieces <= 1) layer_norm_bf16_kernel<1, 4><<<blocks(4), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 2) layer_norm_bf16_kernel<2, 4><<<blocks(4), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 4) layer_norm_bf16_kernel<4, 2><<<blocks(2), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 8) layer_norm_bf16_kernel<8, 1><<<blocks(1), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  else return GRACE_UNSUPPORTED_SHAPE;
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_embed_bf16(const int32_t* token, const uint16_t* embed, const uint16_t* pos,
+                                           uint16_t* x, int R, int D, int n_rows_embed, int32_t* d_status,
+                                           void* stream) {
+  if (!token || !embed || !pos || !x || R <= 0 || D <= 0 || n_rows_embed <= 0) return GRACE_INVALID_ARG;
+  if (D & 3) return GRACE_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(embed) & 7) || (reinterpret_cast<uintptr_t>(pos) & 7))
+    return GRACE_INVALID_ARG;
+  grace::embed_bf16_kernel<<<(R + 3) / 4, 128, 0, (cudaStream_t)stream>>>(token, embed, pos, x, R, D, n_rows_embed, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

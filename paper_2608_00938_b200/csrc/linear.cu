@@ -30,6 +30,7 @@ struct GemmParams {
   uint16_t* y_bf16;
   float* y_f32;
   const float* residual;
+  const uint16_t* residual_bf16;   // bf16 residual stream (added in fp32, result rounded to bf16)
   int64_t ldy;
   int M, N, K, relu;
 };
@@ -121,6 +122,15 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             v[4 * j] += r4.x; v[4 * j + 1] += r4.y; v[4 * j + 2] += r4.z; v[4 * j + 3] += r4.w;
           }
         }
+        if (p.residual_bf16 != nullptr) {
+          const uint4* res = reinterpret_cast<const uint4*>(p.residual_bf16 + (int64_t)m * p.ldy + n);
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint4 r4 = res[j];
+            v[8 * j] += bf16_lo(r4.x); v[8 * j + 1] += bf16_hi(r4.x); v[8 * j + 2] += bf16_lo(r4.y); v[8 * j + 3] += bf16_hi(r4.y);
+            v[8 * j + 4] += bf16_lo(r4.z); v[8 * j + 5] += bf16_hi(r4.z); v[8 * j + 6] += bf16_lo(r4.w); v[8 * j + 7] += bf16_hi(r4.w);
+          }
+        }
         if (p.y_f32 != nullptr) {
           float4* dst = reinterpret_cast<float4*>(p.y_f32 + (int64_t)m * p.ldy + n);
 #pragma unroll
@@ -157,7 +167,7 @@ constexpr int kPStageBytes = kPABytes + kPBBytes;
 constexpr int kPStagingBytes = 128 * 128;                 // 128 rows x 128 bytes
 constexpr int kPSmem = kPStages * kPStageBytes + 2 * kPStagingBytes + 1024 + 256;
 
-enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2 };
+enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3 };
 
 template <int OUT>
 __global__ void __launch_bounds__(192, 1)
@@ -237,7 +247,8 @@ linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
     const int q = warp & 3;
     const int row = q * 32 + lane;
     const bool issuer = (warp == 2 && lane == 0);
-    constexpr int kColsPerChunk = (OUT == kOutBf16) ? 64 : 32;
+    constexpr bool kBf16Out = (OUT == kOutBf16 || OUT == kOutBf16Add);
+    constexpr int kColsPerChunk = kBf16Out ? 64 : 32;
     int local = 0, g = 0;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++local) {
       const int m0 = (tile / n_tiles) * kPBM, n0 = (tile % n_tiles) * kPBN;
@@ -253,7 +264,7 @@ linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         if (issuer) tc::bulk_wait_read<1>();               // the store that last used `buf` has read it
         tc::named_bar_sync(1, 128);
         uint4* my_row = reinterpret_cast<uint4*>(buf + row * 128);
-        if (OUT == kOutBf16) {
+        if (kBf16Out) {
 #pragma unroll
           for (int hseg = 0; hseg < 2; ++hseg) {
             uint32_t r[32];
@@ -296,7 +307,7 @@ linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
         tc::fence_proxy_async_smem();
         tc::named_bar_sync(1, 128);
         if (issuer) {
-          if (OUT == kOutF32Add) tc::tma_reduce_add_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
+          if (OUT == kOutF32Add || OUT == kOutBf16Add) tc::tma_reduce_add_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
           else tc::tma_store_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
           tc::bulk_commit();
         }
@@ -343,9 +354,9 @@ static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw
 
 }  // namespace grace
 
-extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
-                                       uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
-                                       int M, int N, int K, int relu, void* stream) {
+static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                  uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
+                                  bool add_into_bf16, int M, int N, int K, int relu, void* stream) {
   using namespace grace;
   if (!x || !w || ((y_bf16 == nullptr) == (y_f32 == nullptr))) return GRACE_INVALID_ARG;
   if (M <= 0 || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
@@ -368,7 +379,8 @@ extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uin
     if (!tc::make_tmap_bf16(&mx, x, 2, dx, sx, bx) || !tc::make_tmap_bf16(&mw, w, 2, dw, sw, bw) ||
         !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
       return GRACE_CUDA_ERROR;
-    if (!f32) return launch_persistent<kOutBf16>(mx, mw, my, M, N, K, relu, s);
+    if (!f32) return add_into_bf16 ? launch_persistent<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
+                                   : launch_persistent<kOutBf16>(mx, mw, my, M, N, K, relu, s);
     if (aliased) return launch_persistent<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
     return launch_persistent<kOutF32>(mx, mw, my, M, N, K, relu, s);
   }
@@ -385,7 +397,18 @@ extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uin
     if (!tc::make_tmap_bf16(&mw, w, 2, dims, str, box)) return GRACE_CUDA_ERROR;
   }
   GemmParams p;
-  p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.ldy = ldy;
-  p.M = M; p.N = N; p.K = K; p.relu = relu;
+  p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.residual_bf16 = add_into_bf16 ? y_bf16 : nullptr;
+  p.ldy = ldy; p.M = M; p.N = N; p.K = K; p.relu = relu;
   return BN == 128 ? launch_linear<128>(mx, mw, p, s) : launch_linear<64>(mx, mw, p, s);
+}
+
+extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                       uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
+                                       int M, int N, int K, int relu, void* stream) {
+  return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, residual, false, M, N, K, relu, stream);
+}
+
+extern "C" grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                                uint16_t* y_inout, int64_t ldy, int M, int N, int K, void* stream) {
+  return linear_impl(x, ldx, w, ldw, y_inout, nullptr, ldy, nullptr, true, M, N, K, 0, stream);
 }

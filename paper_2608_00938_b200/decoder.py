@@ -31,7 +31,7 @@ class Decoder:
 
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
-                 separate_cand=False, fuse_log_softmax=True):
+                 separate_cand=False, fuse_log_softmax=True, residual_bf16=False):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -91,7 +91,8 @@ class Decoder:
         self.out_flat = torch.zeros(R_max, dtype=torch.int32, device=dev)
         s.parents, s.out_flat = self.parents.data_ptr(), self.out_flat.data_ptr()
         # activations
-        self.x = torch.zeros((R_max, d_model), dtype=torch.float32, device=dev)
+        # residual stream: fp32, or bf16 (half the traffic of every LayerNorm and residual projection)
+        self.x = torch.zeros((R_max, d_model), dtype=torch.bfloat16 if residual_bf16 else torch.float32, device=dev)
         self.h = torch.zeros((R_max, max(d_model, d_ffn)), dtype=torch.bfloat16, device=dev)
         self.qkv = torch.zeros((R_max, max(3 * HD, d_ffn)), dtype=torch.bfloat16, device=dev)
         self.attn = torch.zeros((R_max, HD), dtype=torch.bfloat16, device=dev)
@@ -103,7 +104,8 @@ class Decoder:
         ws_bytes = api.grace_beam_topk_workspace_bytes(B, max_n, max(beam_sizes[1:]))
         self.topk_ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
         self.d_status = torch.zeros(1, dtype=torch.int32, device=dev)
-        s.x, s.h, s.qkv, s.attn, s.logp, s.cand = (self.x.data_ptr(), self.h.data_ptr(), self.qkv.data_ptr(),
+        s.x, s.x_bf16 = (None, self.x.data_ptr()) if residual_bf16 else (self.x.data_ptr(), None)
+        s.h, s.qkv, s.attn, s.logp, s.cand = (self.h.data_ptr(), self.qkv.data_ptr(),
                                                    self.attn.data_ptr(), self.logp.data_ptr(), self.cand.data_ptr())
         s.row_lse = None if self.row_lse is None else self.row_lse.data_ptr()
         s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()

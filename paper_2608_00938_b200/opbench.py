@@ -41,14 +41,19 @@ def main():
     ap.add_argument("--f32out", action="store_true")
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--relu", action="store_true")
+    ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
     a = ap.parse_args()
     dev = "cuda:0"
     torch.manual_seed(0)
     bf = lambda *s: torch.randn(*s, device=dev).to(torch.bfloat16)
     if a.op == "linear":
         x, w = bf(a.M, a.K), bf(a.N, a.K) * 0.05
-        y = torch.zeros(a.M, a.N, device=dev, dtype=torch.float32 if (a.f32out or a.residual) else torch.bfloat16)
-        us = _time(lambda: api.grace_linear(x, w, y, y if a.residual else None, a.relu), a.iters)
+        y = torch.zeros(a.M, a.N, device=dev, dtype=torch.float32 if (a.f32out or a.residual) and not a.bf16stream
+                        else torch.bfloat16)
+        if a.bf16stream:
+            us = _time(lambda: api.grace_linear_add_bf16(x, w, y), a.iters)
+        else:
+            us = _time(lambda: api.grace_linear(x, w, y, y if a.residual else None, a.relu), a.iters)
         print(f"linear M={a.M} N={a.N} K={a.K}: {us:.1f} us, {2.0 * a.M * a.N * a.K / us / 1e6:.1f} TFLOP/s")
     elif a.op == "cross_attn":
         q, k, v = bf(a.B * a.M, a.H, a.d), bf(a.B, a.H, a.T, a.d), bf(a.B, a.H, a.T, a.d)
@@ -135,10 +140,12 @@ def main():
     elif a.op == "layer_norm":
         R = a.B * a.M
         x = torch.randn(R, a.K, device=dev)
+        if a.bf16stream:
+            x = x.to(torch.bfloat16)
         g, b = torch.ones(a.K, device=dev), torch.zeros(a.K, device=dev)
         o = torch.empty(R, a.K, device=dev, dtype=torch.bfloat16)
         us = _time(lambda: api.grace_layer_norm(x, g, b, o), a.iters)
-        print(f"layer_norm R={R} D={a.K}: {us:.1f} us, {R * a.K * 6 / us / 1e3:.0f} GB/s")
+        print(f"layer_norm R={R} D={a.K}: {us:.1f} us, {R * a.K * (x.element_size() + 2) / us / 1e3:.0f} GB/s")
     else:
         R = a.B * a.M
         z = torch.randn(R, a.V, device=dev)

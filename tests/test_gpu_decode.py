@@ -31,7 +31,7 @@ def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=
                 matcher_kind=matcher_kind)
 
 
-def _make_gpu_decoder(cfg, separate_cand=True):
+def _make_gpu_decoder(cfg, separate_cand=True, residual_bf16=False):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     shp, sids, trie = cfg["shp"], cfg["sids"], cfg["trie"]
@@ -45,7 +45,8 @@ def _make_gpu_decoder(cfg, separate_cand=True):
     dec = Decoder(n_layers=shp.n_layers, d_model=shp.d_model, n_heads=shp.n_heads, d_head=shp.d_head,
                   d_ffn=shp.d_ffn, V=shp.V, L=shp.L, T_ctx=cfg["enc"].shape[1], B=cfg["B"],
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=cfg["w"], trie_bits=bits,
-                  trie_base=base, num_nodes=trie.num_nodes, matcher=matcher, device=DEV, separate_cand=separate_cand)
+                  trie_base=base, num_nodes=trie.num_nodes, matcher=matcher, device=DEV, separate_cand=separate_cand,
+                  residual_bf16=residual_bf16)
     dec.project_cross_kv(torch.from_numpy(cfg["enc"]).to(DEV).to(torch.bfloat16))
     return dec, api
 
@@ -57,16 +58,17 @@ def _oracle_matcher(cfg):
     return OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 14, 4) for e in cfg["elig"]])
 
 
-@pytest.mark.parametrize("B,kind,schedule,final_k", [
-    (1, "node", (1, 16, 16), 16),            # configuration 1
-    (3, "bloom", (1, 40, 24), 32),           # several requests, dynamic per-step beam sizes, Bloom matcher
+@pytest.mark.parametrize("B,kind,schedule,final_k,residual_bf16", [
+    (1, "node", (1, 16, 16), 16, False),     # configuration 1
+    (3, "bloom", (1, 40, 24), 32, False),    # several requests, dynamic per-step beam sizes, Bloom matcher
+    (3, "bloom", (1, 40, 24), 32, True),     # the same with the residual stream held in bf16
 ])
-def test_decode_step_teacher_forced(B, kind, schedule, final_k):
+def test_decode_step_teacher_forced(B, kind, schedule, final_k, residual_bf16):
     cfg = _config1(B=B, matcher_kind=kind, schedule=schedule, final_k=final_k)
     shp, trie = cfg["shp"], cfg["trie"]
     record = []
     OD.beam_search(cfg["w"], shp, cfg["enc"], trie, _oracle_matcher(cfg), schedule, final_k, record=record)
-    dec, api = _make_gpu_decoder(cfg)
+    dec, api = _make_gpu_decoder(cfg, residual_bf16=residual_bf16)
     dec.reset()
     V, L = shp.V, shp.L
     sizes = list(schedule) + [final_k]

@@ -229,57 +229,60 @@ def test_decode_step_config5_teacher_forced_on_one_request():
     assert int(level_start[-1]) == trie.num_nodes
     blooms = np.stack([api.grace_bloom_build(sids, V, e, cfg["bloom_log2"], cfg["bloom_hashes"]) for e in inp["elig"]])
     assert np.array_equal(blooms[0], bloom0.words)
-    dec = Decoder(n_layers=cfg["n_layers"], d_model=cfg["d_model"], n_heads=cfg["H"], d_head=cfg["d_h"],
-                  d_ffn=cfg["d_ffn"], V=V, L=L, T_ctx=cfg["T_ctx"], B=B, beam_sizes=sizes, weights=inp["weights"],
-                  trie_bits=bits, trie_base=base, num_nodes=trie.num_nodes,
-                  matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=DEV,
-                  separate_cand=True)
-    dec.project_cross_kv(dev_bf16(inp["enc_bits"]))
-    dec.reset()
-    for t in range(L):
-        step = record[t]
-        M, K = sizes[t], sizes[t + 1]
-        cur, nxt = t & 1, (t + 1) & 1
-        # request 0 occupies rows 0..M-1 (request-major); the other 31 requests run free
-        dec.token[cur][:M].copy_(dev(step["tokens"].astype(np.int32)))
-        dec.score[cur][:M].copy_(dev(step["score"]))
-        dec.node[cur][:M].copy_(dev(step["node"]))
-        dec.key[cur][:M].copy_(dev(step["key"]))
-        if t > 0:
-            dec.parents[t, :M].copy_(dev(record[t - 1]["out_parent"].reshape(-1)))
-        dec.step(t)
-        torch.cuda.synchronize()
-        assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
-        logp = dec.log_probs(M).cpu().numpy()
-        live = step["node"] >= 0                 # dead beams are never normalised (everything is masked)
-        err = np.abs(logp - step["logp"])[live].max()
-        assert err <= 2e-2, f"step {t}: log-prob error {err}"
-        cand = dec.cand[:M].cpu().numpy()
-        assert np.array_equal(np.isfinite(cand), step["allow"])                       # same mask as the oracle
-        assert np.array_equal(cand[step["allow"]], (step["score"][:, None] + logp)[step["allow"]])
-        sc, flat, par, tok = OT.beam_topk(cand.reshape(1, M * V), K, V)               # exact on the GPU's own candidates
-        assert np.array_equal(dec.out_flat[:K].cpu().numpy(), flat[0])
-        assert np.array_equal(dec.score[nxt][:K].cpu().numpy().view(np.uint32), sc[0].view(np.uint32))
-        assert np.array_equal(dec.parents[t + 1, :K].cpu().numpy(), par[0])
-        assert np.array_equal(dec.token[nxt][:K].cpu().numpy(), tok[0])
-        node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, step["node"], step["key"], t, M)
-        assert np.array_equal(dec.node[nxt][:K].cpu().numpy(), node_ref)
-        assert np.array_equal(dec.key[nxt][:K].cpu().numpy().view(np.uint64), key_ref)
-        # every request (free-running ones too): selected scores sorted, live beams sit on catalog nodes
-        all_sc = dec.score[nxt][:B * K].view(B, K).cpu().numpy()
-        assert (all_sc[:, 1:] <= all_sc[:, :-1]).all()
-        all_node = dec.node[nxt][:B * K].cpu().numpy()
-        assert np.array_equal(all_node >= 0, np.isfinite(all_sc.reshape(-1)))
-        assert ((all_node < 0) | ((all_node >= trie.level_start[t + 1]) & (all_node < trie.level_start[t + 2]))).all()
-    # the emitted SIDs of every request are catalog SIDs whose prefixes all pass that request's Bloom filter
-    g_sids, g_score, g_node = dec.results()
-    catalog_keys = set(OM.prefix_keys(sids).tolist())
-    for b in (0, 5, 31):
-        valid = np.isfinite(g_score[b])
-        assert valid.sum() > 0
-        keys = OM.prefix_keys(g_sids[b][valid])
-        assert all(int(x) in catalog_keys for x in keys)
-        bl = OM.PrefixBloom(cfg["bloom_log2"], cfg["bloom_hashes"])
-        bl.words = blooms[b]
-        for l in range(1, L + 1):
-            assert bl.contains(OM.prefix_keys(g_sids[b][valid][:, :l])).all()
+    for residual_bf16 in (False, True):          # fp32 and bf16 residual stream, same tolerance
+        dec = Decoder(n_layers=cfg["n_layers"], d_model=cfg["d_model"], n_heads=cfg["H"], d_head=cfg["d_h"],
+                      d_ffn=cfg["d_ffn"], V=V, L=L, T_ctx=cfg["T_ctx"], B=B, beam_sizes=sizes, weights=inp["weights"],
+                      trie_bits=bits, trie_base=base, num_nodes=trie.num_nodes,
+                      matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=DEV,
+                      separate_cand=True, residual_bf16=residual_bf16)
+        dec.project_cross_kv(dev_bf16(inp["enc_bits"]))
+        dec.reset()
+        for t in range(L):
+            step = record[t]
+            M, K = sizes[t], sizes[t + 1]
+            cur, nxt = t & 1, (t + 1) & 1
+            # request 0 occupies rows 0..M-1 (request-major); the other 31 requests run free
+            dec.token[cur][:M].copy_(dev(step["tokens"].astype(np.int32)))
+            dec.score[cur][:M].copy_(dev(step["score"]))
+            dec.node[cur][:M].copy_(dev(step["node"]))
+            dec.key[cur][:M].copy_(dev(step["key"]))
+            if t > 0:
+                dec.parents[t, :M].copy_(dev(record[t - 1]["out_parent"].reshape(-1)))
+            dec.step(t)
+            torch.cuda.synchronize()
+            assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+            logp = dec.log_probs(M).cpu().numpy()
+            live = step["node"] >= 0                 # dead beams are never normalised (everything is masked)
+            err = np.abs(logp - step["logp"])[live].max()
+            assert err <= 2e-2, f"step {t}: log-prob error {err}"
+            cand = dec.cand[:M].cpu().numpy()
+            assert np.array_equal(np.isfinite(cand), step["allow"])                       # same mask as the oracle
+            assert np.array_equal(cand[step["allow"]], (step["score"][:, None] + logp)[step["allow"]])
+            sc, flat, par, tok = OT.beam_topk(cand.reshape(1, M * V), K, V)               # exact on the GPU's own candidates
+            assert np.array_equal(dec.out_flat[:K].cpu().numpy(), flat[0])
+            assert np.array_equal(dec.score[nxt][:K].cpu().numpy().view(np.uint32), sc[0].view(np.uint32))
+            assert np.array_equal(dec.parents[t + 1, :K].cpu().numpy(), par[0])
+            assert np.array_equal(dec.token[nxt][:K].cpu().numpy(), tok[0])
+            node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, step["node"], step["key"], t, M)
+            assert np.array_equal(dec.node[nxt][:K].cpu().numpy(), node_ref)
+            assert np.array_equal(dec.key[nxt][:K].cpu().numpy().view(np.uint64), key_ref)
+            # every request (free-running ones too): selected scores sorted, live beams sit on catalog nodes
+            all_sc = dec.score[nxt][:B * K].view(B, K).cpu().numpy()
+            assert (all_sc[:, 1:] <= all_sc[:, :-1]).all()
+            all_node = dec.node[nxt][:B * K].cpu().numpy()
+            assert np.array_equal(all_node >= 0, np.isfinite(all_sc.reshape(-1)))
+            assert ((all_node < 0) | ((all_node >= trie.level_start[t + 1]) & (all_node < trie.level_start[t + 2]))).all()
+        # the emitted SIDs of every request are catalog SIDs whose prefixes all pass that request's Bloom filter
+        g_sids, g_score, g_node = dec.results()
+        catalog_keys = set(OM.prefix_keys(sids).tolist())
+        for b in (0, 5, 31):
+            valid = np.isfinite(g_score[b])
+            assert valid.sum() > 0
+            keys = OM.prefix_keys(g_sids[b][valid])
+            assert all(int(x) in catalog_keys for x in keys)
+            bl = OM.PrefixBloom(cfg["bloom_log2"], cfg["bloom_hashes"])
+            bl.words = blooms[b]
+            for l in range(1, L + 1):
+                assert bl.contains(OM.prefix_keys(g_sids[b][valid][:, :l])).all()
+        del dec
+        torch.cuda.empty_cache()

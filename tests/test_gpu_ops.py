@@ -460,6 +460,46 @@ def test_linear_matches_fp64_matmul(api, M, N, K, relu, res, f32out):
     assert np.abs(got - ref).max() <= tol * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
 
 
+@pytest.mark.parametrize("M,N,K", [
+    (300, 512, 512), (130, 64, 2048), (7, 128, 64),                       # small-tile kernel
+    (1500, 512, 512), (1300, 512, 2048), (19000, 512, 512), (1111, 320, 128),   # persistent kernel, ragged tiles
+])
+def test_linear_add_into_bf16_residual_stream(api, M, N, K):
+    rng = synth.rng_for(5, 7 * M + N + K)
+    x = synth.normal_bf16(rng, (M, K))
+    w = synth.normal_bf16(rng, (N, K), 0.05)
+    r = synth.normal_bf16(rng, (M, N))
+    ref = f64(x) @ f64(w).T + f64(r)
+    y = dev_bf16(r).clone()
+    api.grace_linear_add_bf16(dev_bf16(x), dev_bf16(w), y)
+    torch.cuda.synchronize()
+    got = y.float().cpu().numpy().astype(np.float64)
+    # product rounded to bf16 (2^-9 relative), then a bf16 add: two roundings of values of size |ref|
+    assert np.abs(got - ref).max() <= 2e-2 * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
+    err = np.abs(got - ref) / np.maximum(np.abs(ref), np.abs(f64(r)))
+    assert np.median(err) <= 2.0 ** -8
+
+
+def test_layer_norm_embed_bf16_stream(api):
+    rng = synth.rng_for(5, 10)
+    for R, D in ((77, 512), (5, 128), (33, 1024), (9, 2048), (6, 72)):
+        xb = synth.normal_bf16(rng, (R, D), 2.0)
+        g, b = synth.normal_f32(rng, D), synth.normal_f32(rng, D)
+        out = torch.zeros((R, D), dtype=torch.bfloat16, device=DEV)
+        api.grace_layer_norm(dev_bf16(xb), dev(g), dev(b), out, 1e-5)
+        x64 = f64(xb)
+        ref = (x64 - x64.mean(1, keepdims=True)) / np.sqrt(x64.var(1, keepdims=True) + 1e-5) * g + b
+        assert np.abs(out.float().cpu().numpy() - ref).max() <= 2e-2 * max(1, np.abs(ref).max())
+    R, D, V = 77, 512, 2048
+    emb = synth.normal_bf16(rng, (V + 1, D))
+    pos = synth.normal_bf16(rng, (D,))
+    tok = rng.integers(0, V + 1, size=R).astype(np.int32)
+    xo = torch.zeros((R, D), dtype=torch.bfloat16, device=DEV)
+    api.grace_embed(dev(tok), dev_bf16(emb), dev_bf16(pos), xo)
+    ref = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(emb)[tok] + synth.bf16_bits_to_f32(pos))
+    assert np.array_equal(xo.view(torch.int16).cpu().numpy().view(np.uint16), ref)   # one fp32 add, one RNE rounding
+
+
 def test_layer_norm_embed_log_softmax(api):
     rng = synth.rng_for(5, 9)
     R, D, V = 77, 512, 2048
