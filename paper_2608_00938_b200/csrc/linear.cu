@@ -149,117 +149,128 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------------
-// Persistent kernel for the large GEMMs of the decoder (M in the tens of thousands).
+// Persistent CTA-pair kernel for the large GEMMs of the decoder (M in the tens of thousands).
 //
-// One CTA per SM walks over 128 x 256 output tiles (n fastest, so the CTAs running at the same
-// time share an A row panel in L2).  Warp 0 streams A (128 x 64) and W (256 x 64) tiles through a
-// 4-stage ring; warp 1 issues tcgen05.mma 128 x 256 x 16 into one of TWO TMEM accumulators
-// (2 x 256 columns = all of TMEM), so the four epilogue warps drain tile i while the tensor core
-// already works on tile i+1.  The epilogue reads 64 (bf16) or 32 (fp32) columns at a time from
-// TMEM, writes them to a 128-byte-swizzled staging tile in shared memory and hands it to TMA:
-// a plain tile store, or an fp32 add-reduction straight into the residual stream (x += y), so
-// the residual is never read into the SM.
+// A cluster of two CTAs (two SMs) walks over 256 x 256 output tiles (n fastest, so the pairs running
+// at the same time share an A row panel in L2) with one tcgen05.mma.cta_group::2 stream.  Each CTA
+// stages its own 128 rows of A and its own 128 rows of W (half of the tile's N) through a 6-stage
+// ring, so an SM fills 32 KB of shared memory per 64-wide k-block where a lone 128 x 256 tile needs
+// 48 KB: the fill rate of shared memory, not the tensor pipe, is what limits these GEMMs.  The even
+// CTA issues every MMA into one of TWO TMEM accumulators (2 x 256 columns = all of TMEM), so the
+// four epilogue warps of each CTA drain tile i while the tensor cores already work on tile i+1.
+// tcgen05.commit arrives on the barriers of both CTAs, and both CTAs' TMA loads count their bytes on
+// the even CTA's "stage full" barrier (plain one-destination loads; nothing is multicast).
+// The epilogue reads 64 (bf16) or 32 (fp32) columns at a time from TMEM, writes them to a
+// 128-byte-swizzled staging tile in shared memory and hands it to TMA: a plain tile store, or an
+// add-reduction straight into the residual stream (x += y), so the residual is never read into the SM.
 // ---------------------------------------------------------------------------------------------
-constexpr int kPBM = 128, kPBN = 256, kPBK = 64, kPStages = 4;
-constexpr int kPABytes = kPBM * kPBK * 2;                 // 16 KB
-constexpr int kPBBytes = kPBN * kPBK * 2;                 // 32 KB
-constexpr int kPStageBytes = kPABytes + kPBBytes;
+constexpr int kPBK = 64;
 constexpr int kPStagingBytes = 128 * 128;                 // 128 rows x 128 bytes
-constexpr int kPSmem = kPStages * kPStageBytes + 2 * kPStagingBytes + 1024 + 256;
 
 enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3 };
 
+constexpr int kQStages = 6;
+constexpr int kQABytes = 128 * kPBK * 2;                  // 16 KB: 128 rows of A
+constexpr int kQBBytes = 128 * kPBK * 2;                  // 16 KB: 128 of the tile's 256 rows of W
+constexpr int kQStageBytes = kQABytes + kQBBytes;
+constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 1024 + 256;
+
 template <int OUT>
 __global__ void __launch_bounds__(192, 1)
-linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                         const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu) {
+linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                   const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* staging = tiles + kPStages * kPStageBytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(staging + 2 * kPStagingBytes);
-  uint64_t* empty = full + kPStages;
-  uint64_t* acc_full = empty + kPStages;       // [2]
-  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint8_t* staging = tiles + kQStages * kQStageBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(staging + 2 * kPStagingBytes);   // even CTA only: both CTAs' bytes landed
+  uint64_t* empty = full + kQStages;           // the pair's MMAs have read the stage
+  uint64_t* acc_full = empty + kQStages;       // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2] even CTA only: 4 local + 4 remote epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = tc::cluster_cta_rank();            // 0: issues the MMAs; 1: peer
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int KB = K / kPBK;
-  const int n_tiles = (N + kPBN - 1) / kPBN, m_tiles = (M + kPBM - 1) / kPBM;
+  const int n_tiles = (N + 255) / 256, m_tiles = (M + 255) / 256;
   const int total = n_tiles * m_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
-    for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 4); }
+    for (int s = 0; s < kQStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 8); }
     *abort_flag = 0;
     tc::fence_mbar_init();
     tc::tma_prefetch_desc(&map_x); tc::tma_prefetch_desc(&map_w); tc::tma_prefetch_desc(&map_y);
   }
-  if (warp == 0) tc::tmem_alloc(tmem_slot, 512);
+  if (warp == 0) tc::tmem_alloc_pair(tmem_slot, 512);
   tc::tc_fence_before();
   __syncthreads();
+  tc::cluster_sync_all();                                  // both CTAs' barriers exist before any remote arrive
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {                                        // ---- TMA producer ----
+    if (lane == 0) {                                        // ---- TMA producer (both CTAs) ----
       int it = 0;
-      for (int tile = blockIdx.x; tile < total; tile += gridDim.x) {
-        const int m0 = (tile / n_tiles) * kPBM, n0 = (tile % n_tiles) * kPBN;
+      for (int tile = pair; tile < total; tile += n_pairs) {
+        const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256 + (int)rank * 128;
         for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % kPStages;
-          if (!tc::mbar_wait(empty + s, ((it / kPStages) & 1) ^ 1, abort_flag)) { tile = total; break; }
-          tc::mbar_expect_tx(full + s, kPStageBytes);
-          uint8_t* a = tiles + s * kPStageBytes;
-          tc::tma_load_2d(a, &map_x, full + s, kb * kPBK, m0);
-          tc::tma_load_2d(a + kPABytes, &map_w, full + s, kb * kPBK, n0);
+          const int s = it % kQStages;
+          if (!tc::mbar_wait_cluster(empty + s, ((it / kQStages) & 1) ^ 1, abort_flag)) { tile = total; break; }
+          if (rank == 0) tc::mbar_expect_tx(full + s, 2 * kQStageBytes);     // this CTA's bytes and the peer's
+          uint8_t* a = tiles + s * kQStageBytes;
+          const uint32_t bar = tc::cluster_addr_of(full + s, 0);
+          tc::tma_load_2d_pair(a, &map_x, bar, kb * kPBK, m0);
+          tc::tma_load_2d_pair(a + kQABytes, &map_w, bar, kb * kPBK, n0);
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {                                        // ---- MMA issuer ----
-      constexpr uint32_t idesc = tc::idesc_bf16(kPBM, kPBN, 0);
+    if (lane == 0 && rank == 0) {                           // ---- even CTA: MMA issuer for the pair ----
+      constexpr uint32_t idesc = tc::idesc_bf16(256, 256, 0);
       int it = 0, local = 0;
-      for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++local) {
+      for (int tile = pair; tile < total; tile += n_pairs, ++local) {
         const int ab = local & 1;
-        if (!tc::mbar_wait(acc_empty + ab, ((local >> 1) & 1) ^ 1, abort_flag)) break;
+        if (!tc::mbar_wait_cluster(acc_empty + ab, ((local >> 1) & 1) ^ 1, abort_flag)) break;
         tc::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * kPBN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(ab * 256);
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % kPStages;
-          if (!tc::mbar_wait(full + s, (it / kPStages) & 1, abort_flag)) { ok = false; break; }
+          const int s = it % kQStages;
+          const uint32_t ph = (it / kQStages) & 1;
+          if (!tc::mbar_wait_cluster(full + s, ph, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
-          const uint32_t a_addr = tc::smem_addr(tiles + s * kPStageBytes);
+          const uint32_t a_addr = tc::smem_addr(tiles + s * kQStageBytes);
           const uint64_t a_desc = tc::smem_desc_sw128(a_addr, 16, 1024);
-          const uint64_t b_desc = tc::smem_desc_sw128(a_addr + kPABytes, 16, 1024);
+          const uint64_t b_desc = tc::smem_desc_sw128(a_addr + kQABytes, 16, 1024);
 #pragma unroll
           for (int k = 0; k < kPBK / 16; ++k)
-            tc::mma_ss(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
-          tc::mma_commit(empty + s);
+            tc::mma_ss_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) ? 1u : 0u);
+          tc::mma_commit_pair(empty + s, 3);
         }
         if (!ok) break;
-        tc::mma_commit(acc_full + ab);
+        tc::mma_commit_pair(acc_full + ab, 3);
       }
     }
   } else {
-    // ---- epilogue warps 2..5: TMEM lane quarter q, rows q*32 + lane of the tile ----
+    // ---- epilogue warps 2..5 of both CTAs: TMEM lane quarter q = rows q*32 + lane of this CTA's 128 ----
     const int q = warp & 3;
     const int row = q * 32 + lane;
     const bool issuer = (warp == 2 && lane == 0);
     constexpr bool kBf16Out = (OUT == kOutBf16 || OUT == kOutBf16Add);
     constexpr int kColsPerChunk = kBf16Out ? 64 : 32;
     int local = 0, g = 0;
-    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++local) {
-      const int m0 = (tile / n_tiles) * kPBM, n0 = (tile % n_tiles) * kPBN;
+    for (int tile = pair; tile < total; tile += n_pairs, ++local) {
+      const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
       const int ab = local & 1;
-      bool ok = tc::mbar_wait(acc_full + ab, (local >> 1) & 1, abort_flag);
+      bool ok = tc::mbar_wait_cluster(acc_full + ab, (local >> 1) & 1, abort_flag);
       ok = __all_sync(kFullMask, ok);
       if (!ok) break;
       tc::tc_fence_after();
-      const uint32_t t_acc = tmem_base + (uint32_t)(ab * kPBN) + ((uint32_t)(q * 32) << 16);
+      const uint32_t t_acc = tmem_base + (uint32_t)(ab * 256) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < kPBN / kColsPerChunk; ++c, ++g) {
+      for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
         uint8_t* buf = staging + (g & 1) * kPStagingBytes;
         if (issuer) tc::bulk_wait_read<1>();               // the store that last used `buf` has read it
         tc::named_bar_sync(1, 128);
@@ -299,42 +310,56 @@ linear_persistent_kernel(const __grid_constant__ CUtensorMap map_x, const __grid
                                                __float_as_uint(v[3]));
           }
         }
-        if (c == kPBN / kColsPerChunk - 1) {               // accumulator fully read: hand it back
+        if (c == 256 / kColsPerChunk - 1) {                // accumulator fully read: hand it back to the issuer
           tc::tc_fence_before();
           __syncwarp();
-          if (lane == 0) tc::mbar_arrive(acc_empty + ab);
+          if (lane == 0) {
+            if (rank == 0) tc::mbar_arrive(acc_empty + ab);
+            else tc::mbar_arrive_remote(acc_empty + ab, 0);
+          }
         }
         tc::fence_proxy_async_smem();
         tc::named_bar_sync(1, 128);
-        if (issuer) {
+        if (issuer && m0 < M) {
           if (OUT == kOutF32Add || OUT == kOutBf16Add) tc::tma_reduce_add_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
           else tc::tma_store_2d(&map_y, buf, n0 + c * kColsPerChunk, m0);
-          tc::bulk_commit();
         }
+        if (issuer) tc::bulk_commit();
       }
     }
     if (issuer) tc::bulk_wait_all();
   }
+  // neither CTA may leave while its peer can still read its shared memory or arrive on its barriers
   tc::tc_fence_before();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tmem_base, 512);
+  tc::cluster_sync_all();
+  if (warp == 0) tc::tmem_dealloc_pair(tmem_base, 512);
 }
 
 template <int OUT>
-static grace_status_t launch_persistent(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M,
-                                        int N, int K, int relu, cudaStream_t s) {
+static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
+                                  int K, int relu, cudaStream_t s) {
   static bool attr_set = false;
-  static int n_sm = 0;
+  static int max_clusters = 0;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
   if (!attr_set) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_persistent_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem));
-    int dev = 0;
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
+    int dev = 0, n_sm = 0;
     GRACE_CUDA_TRY(cudaGetDevice(&dev));
     GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    cfg.gridDim = dim3(n_sm & ~1);
+    GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&max_clusters, linear_pair_kernel<OUT>, &cfg));
+    if (max_clusters <= 0) return GRACE_CUDA_ERROR;
+    if (max_clusters > n_sm / 2) max_clusters = n_sm / 2;
     attr_set = true;
   }
-  const int total = ((N + kPBN - 1) / kPBN) * ((M + kPBM - 1) / kPBM);
-  const int grid = total < n_sm ? total : n_sm;
-  linear_persistent_kernel<OUT><<<grid, 192, kPSmem, s>>>(mx, mw, my, M, N, K, relu);
+  const int total = ((N + 255) / 256) * ((M + 255) / 256);
+  cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
+  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu));
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -367,22 +392,22 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
   cudaStream_t s = (cudaStream_t)stream;
   const bool aliased = (residual != nullptr) && (residual == y_f32);
   if (M >= 1024 && N >= 256 && (residual == nullptr || aliased)) {
-    // large GEMM: persistent kernel, TMA-store epilogue (add-reduction when y is the residual stream)
+    // large GEMM: persistent CTA-pair kernel, TMA-store epilogue (add-reduction when y is the residual stream)
     CUtensorMap mx, mw, my;
     const uint64_t dx[2] = {(uint64_t)K, (uint64_t)M}, sx[1] = {(uint64_t)ldx};
-    const uint32_t bx[2] = {(uint32_t)kPBK, (uint32_t)kPBM};
+    const uint32_t bx[2] = {(uint32_t)kPBK, 128u};
     const uint64_t dw[2] = {(uint64_t)K, (uint64_t)N}, sw[1] = {(uint64_t)ldw};
-    const uint32_t bw[2] = {(uint32_t)kPBK, (uint32_t)kPBN};
+    const uint32_t bw[2] = {(uint32_t)kPBK, 128u};      // each CTA of a pair stages 128 of the tile's 256 rows of W
     const uint64_t dy[2] = {(uint64_t)N, (uint64_t)M}, sy[1] = {(uint64_t)ldy};
     const bool f32 = (y_f32 != nullptr);
     const uint32_t by[2] = {f32 ? 32u : 64u, 128u};
     if (!tc::make_tmap_bf16(&mx, x, 2, dx, sx, bx) || !tc::make_tmap_bf16(&mw, w, 2, dw, sw, bw) ||
         !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
       return GRACE_CUDA_ERROR;
-    if (!f32) return add_into_bf16 ? launch_persistent<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
-                                   : launch_persistent<kOutBf16>(mx, mw, my, M, N, K, relu, s);
-    if (aliased) return launch_persistent<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
-    return launch_persistent<kOutF32>(mx, mw, my, M, N, K, relu, s);
+    if (!f32) return add_into_bf16 ? launch_pair<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
+                                   : launch_pair<kOutBf16>(mx, mw, my, M, N, K, relu, s);
+    if (aliased) return launch_pair<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
+    return launch_pair<kOutF32>(mx, mw, my, M, N, K, relu, s);
   }
   CUtensorMap mx, mw;
   const int BN = (N >= 128) ? 128 : 64;
