@@ -1,5 +1,5 @@
 // Cross-attention on tcgen05 tensor cores (Section 5.1: beams of a request are the M dimension of
-// a dense contraction against that request's shared K/V), head size 64.
+// a dense contraction against that request's shared K/V), head size 64 or 128.
 //
 // A work item is 128 query rows of one (request, head); its encoder positions are streamed in
 // blocks of 128:
@@ -15,9 +15,12 @@
 // maps over the caller's strides, so the beam-major Q / O layout is never permuted (the view /
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
 // and masked in the softmax.  Warp roles: 0-7 softmax + epilogue, 8 TMA producer, 9 MMA issuer.
-// The kernel is persistent (two CTAs per SM, each looping over work items; Q is double-buffered),
-// so the next item's loads and first S overlap the current item's epilogue, and one CTA's MMAs
-// run under the other's exponentials.
+// The kernel is persistent (each CTA loops over work items; Q is double-buffered), so the next item's
+// loads and first S overlap the current item's epilogue.  Head size 64 runs two CTAs per SM (256 TMEM
+// columns each), so one CTA's MMAs run under the other's exponentials; head size 128 needs 320
+// columns (O is twice as wide) and 192 KB of tiles, so it runs one CTA per SM.  A 128-wide tile is
+// held as two 64-wide halves (the 128-byte swizzle spans 64 bf16), each with its own TMA box and its
+// own MMA k-steps (Q, K) or output-column half (V).
 #pragma once
 #include "common.cuh"
 #include "tc.cuh"
@@ -26,14 +29,18 @@ namespace grace {
 
 constexpr int kCaBM = 128;        // query rows per work item
 constexpr int kCaBN = 128;        // encoder positions per block
-constexpr int kCaDH = 64;
 constexpr int kCaStages = 2;
-constexpr int kCaTileBytes = 128 * 64 * 2;                       // 16 KB: Q, K_blk or V_blk
+constexpr int kCaHalfBytes = 128 * 64 * 2;                       // 16 KB: 128 rows x 64 bf16, one swizzle span wide
 constexpr int kCaSoftmaxWarps = 8;
 constexpr int kCaThreads = (kCaSoftmaxWarps + 2) * 32;
 constexpr int kCaBarBytes = 256;
-constexpr int kCaSmemBytes = kCaTileBytes * (2 + 2 * kCaStages) + 1024 + kCaBarBytes + 2 * 2 * 128 * 4 + 2 * 2 * 128 * 4;
-constexpr uint32_t kCaTmemCols = 256;                            // S: 0..127, O: 128..191, P: 192..255
+template <int DH> struct CaCfg {
+  static constexpr int kHalves = DH / 64;
+  static constexpr int kTileBytes = kCaHalfBytes * kHalves;      // Q, K_blk or V_blk
+  static constexpr int kSmemBytes = kTileBytes * (2 + 2 * kCaStages) + 1024 + kCaBarBytes + 2 * 2 * 128 * 4 + 2 * 2 * 128 * 4;
+  static constexpr uint32_t kTmemCols = DH == 64 ? 256 : 512;    // S: 0..127, O: 128..128+DH-1, P: the next 64
+  static constexpr int kCtasPerSm = DH == 64 ? 2 : 1;
+};
 
 struct CrossTcParams {
   uint16_t* out;
@@ -59,9 +66,12 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // Persistent kernel: a flat grid of two CTAs per SM; CTA g takes the work items g, g + gridDim.x,
 // ...  An item is one (request, head, 128-row tile); consecutive items are the tiles of the same
 // (request, head), so the CTAs running at the same time read the same K/V from L2.
-__global__ void __launch_bounds__(kCaThreads, 2)
+template <int DH>
+__global__ void __launch_bounds__(kCaThreads, CaCfg<DH>::kCtasPerSm)
 cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const CrossTcParams p) {
+  constexpr int kCaTileBytes = CaCfg<DH>::kTileBytes, kHalves = CaCfg<DH>::kHalves;
+  constexpr uint32_t kCaTmemCols = CaCfg<DH>::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_tiles = tiles;                                      // two Q buffers
@@ -104,8 +114,8 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base;           // S fp32, 128 columns
-  const uint32_t tmem_o = tmem_base + 128;     // O fp32, 64 columns
-  const uint32_t tmem_p = tmem_base + 192;     // P bf16 pairs, 64 columns
+  const uint32_t tmem_o = tmem_base + 128;     // O fp32, DH columns
+  const uint32_t tmem_p = tmem_base + 128 + DH;   // P bf16 pairs, 64 columns
 
   if (warp == kCaSoftmaxWarps) {
     // ---------------- TMA producer ----------------
@@ -130,10 +140,15 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
               (!need_q || tc::mbar_try_wait_now(q_empty + qb, ((li >> 1) & 1) ^ 1))) {
             if (need_q) {
               tc::mbar_expect_tx(q_full + qb, kCaTileBytes);
-              tc::tma_load_4d(q_tiles + qb * kCaTileBytes, &map_q, q_full + qb, 0, h, (item % p.tiles_m) * kCaBM, b);
+#pragma unroll
+              for (int hf = 0; hf < kHalves; ++hf)
+                tc::tma_load_4d(q_tiles + qb * kCaTileBytes + hf * kCaHalfBytes, &map_q, q_full + qb, 64 * hf, h,
+                                (item % p.tiles_m) * kCaBM, b);
             }
             tc::mbar_expect_tx(k_full + s, kCaTileBytes);
-            tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes, &map_k, k_full + s, 0, j * kCaBN, h, b);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf)
+              tc::tma_load_4d(kv_tiles + (2 * s) * kCaTileBytes + hf * kCaHalfBytes, &map_k, k_full + s, 64 * hf, j * kCaBN, h, b);
             ++gk;
             progressed = true;
           }
@@ -144,7 +159,9 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const int bh = item / p.tiles_m, h = bh % p.H, b = bh / p.H;
           if (tc::mbar_try_wait_now(v_empty + s, ((gv / kCaStages) & 1) ^ 1)) {
             tc::mbar_expect_tx(v_full + s, kCaTileBytes);
-            tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes, &map_v, v_full + s, 0, j * kCaBN, h, b);
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf)
+              tc::tma_load_4d(kv_tiles + (2 * s + 1) * kCaTileBytes + hf * kCaHalfBytes, &map_v, v_full + s, 64 * hf, j * kCaBN, h, b);
             ++gv;
             progressed = true;
           }
@@ -161,26 +178,29 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc_s = tc::idesc_bf16(kCaBM, kCaBN, 0);     // Q K^T : B K-major
-      constexpr uint32_t idesc_o = tc::idesc_bf16(kCaBM, kCaDH, 1);     // P V   : B MN-major
+      constexpr uint32_t idesc_o = tc::idesc_bf16(kCaBM, 64, 1);        // P V   : B MN-major, 64 output columns at a time
       const int my_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
       const int total_blocks = my_items * NB;
       // Every operand descriptor is fixed by (Q buffer, ring slot, k-step): build them once.  The
       // issuing thread shares its scheduler with busy softmax warps, so each instruction it does not
       // execute per block shortens the hand-off to the tensor core.
-      uint64_t q_desc[2][kCaDH / 16], k_desc[kCaStages][kCaDH / 16], v_desc[kCaStages][kCaBN / 16];
+      // k-step k of Q or K: 16 of the DH columns = 32 bytes inside the 64-wide half (k / 4)
+      uint64_t q_desc[2][DH / 16], k_desc[kCaStages][DH / 16], v_desc[kCaStages][kHalves][kCaBN / 16];
 #pragma unroll
       for (int i = 0; i < 2; ++i)
 #pragma unroll
-        for (int k = 0; k < kCaDH / 16; ++k)
-          q_desc[i][k] = tc::smem_desc_sw128(tc::smem_addr(q_tiles + i * kCaTileBytes) + 32 * k, 16, 1024);
+        for (int k = 0; k < DH / 16; ++k)
+          q_desc[i][k] = tc::smem_desc_sw128(tc::smem_addr(q_tiles + i * kCaTileBytes) + (k / 4) * kCaHalfBytes + 32 * (k % 4), 16, 1024);
 #pragma unroll
       for (int st = 0; st < kCaStages; ++st) {
 #pragma unroll
-        for (int k = 0; k < kCaDH / 16; ++k)
-          k_desc[st][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st) * kCaTileBytes) + 32 * k, 16, 1024);
+        for (int k = 0; k < DH / 16; ++k)
+          k_desc[st][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st) * kCaTileBytes) + (k / 4) * kCaHalfBytes + 32 * (k % 4), 16, 1024);
 #pragma unroll
-        for (int k = 0; k < kCaBN / 16; ++k)
-          v_desc[st][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st + 1) * kCaTileBytes) + 2048 * k, 1024, 1024);
+        for (int hf = 0; hf < kHalves; ++hf)
+#pragma unroll
+          for (int k = 0; k < kCaBN / 16; ++k)
+            v_desc[st][hf][k] = tc::smem_desc_sw128(tc::smem_addr(kv_tiles + (2 * st + 1) * kCaTileBytes) + hf * kCaHalfBytes + 2048 * k, 1024, 1024);
       }
       // S of global block g: Q buffer of its item, K of ring slot g % stages
       auto issue_s = [&](int g, int j, int li) -> bool {
@@ -191,18 +211,18 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (qb == 0) {
           if (s == 0) {
 #pragma unroll
-            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
+            for (int k = 0; k < DH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
           } else {
 #pragma unroll
-            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
+            for (int k = 0; k < DH / 16; ++k) tc::mma_ss(tmem_s, q_desc[0][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
           }
         } else {
           if (s == 0) {
 #pragma unroll
-            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
+            for (int k = 0; k < DH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[0][k], idesc_s, k ? 1u : 0u);
           } else {
 #pragma unroll
-            for (int k = 0; k < kCaDH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
+            for (int k = 0; k < DH / 16; ++k) tc::mma_ss(tmem_s, q_desc[1][k], k_desc[1][k], idesc_s, k ? 1u : 0u);
           }
         }
         tc::mma_commit(s_full);
@@ -229,10 +249,16 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tc::tc_fence_after();
         if (s == 0) {
 #pragma unroll
-          for (int k = 0; k < kCaBN / 16; ++k) tc::mma_ts(tmem_o, tmem_p + 8 * k, v_desc[0][k], idesc_o, (j | k) ? 1u : 0u);
+          for (int hf = 0; hf < kHalves; ++hf)
+#pragma unroll
+            for (int k = 0; k < kCaBN / 16; ++k)
+              tc::mma_ts(tmem_o + 64 * hf, tmem_p + 8 * k, v_desc[0][hf][k], idesc_o, (j | k) ? 1u : 0u);
         } else {
 #pragma unroll
-          for (int k = 0; k < kCaBN / 16; ++k) tc::mma_ts(tmem_o, tmem_p + 8 * k, v_desc[1][k], idesc_o, (j | k) ? 1u : 0u);
+          for (int hf = 0; hf < kHalves; ++hf)
+#pragma unroll
+            for (int k = 0; k < kCaBN / 16; ++k)
+              tc::mma_ts(tmem_o + 64 * hf, tmem_p + 8 * k, v_desc[1][hf][k], idesc_o, (j | k) ? 1u : 0u);
         }
         tc::mma_commit(v_empty + s);                         // V of block g is consumed
         tc::mma_commit(o_full);                              // O includes block g
@@ -242,13 +268,14 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   } else {
     // ---------------- softmax + epilogue ----------------
     // Warps w and w+4 share the TMEM lanes (= query rows) 32*(w&3)..+31; each takes one half of the
-    // 128 score columns and one half of the 64 output columns of those rows.  O stays in TMEM and
+    // 128 score columns and one half of the DH output columns of those rows.  O stays in TMEM and
     // accumulates across blocks; it is rescaled only when a row's maximum grows by more than 2^8
     // (probabilities may then reach 256, which bf16 and the fp32 sums hold without loss).
     const int quarter = warp & 3, half = warp >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int col_base = 64 * half;
+    constexpr int kOutCols = DH / 2;                       // output columns per thread
     bool ok = true;
     int g = 0, n_done = 0;
     for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
@@ -330,15 +357,18 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tc::tmem_st16(tmem_p + lane_addr + 32 * half + 16, p1);
         }
         if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
-          uint32_t o[32];
-          tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
-          tc::tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-          uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
-          uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
-          tc::tmem_st16(tmem_o + lane_addr + 32 * half, o0);
-          tc::tmem_st16(tmem_o + lane_addr + 32 * half + 16, o1);
+          for (int c = 0; c < kOutCols; c += 32) {
+            uint32_t o[32];
+            tc::tmem_ld32(tmem_o + lane_addr + kOutCols * half + c, o);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
+            uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
+            tc::tmem_st16(tmem_o + lane_addr + kOutCols * half + c, o0);
+            tc::tmem_st16(tmem_o + lane_addr + kOutCols * half + c + 16, o1);
+          }
         }
         tc::tmem_st_wait();
         tc::tc_fence_before();
@@ -351,8 +381,10 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       ok = __all_sync(kFullMask, ok);
       if (!ok) break;
       tc::tc_fence_after();
-      uint32_t o[32];
-      tc::tmem_ld32(tmem_o + lane_addr + 32 * half, o);
+      uint32_t o[kOutCols];
+#pragma unroll
+      for (int c = 0; c < kOutCols; c += 32)
+        tc::tmem_ld32(tmem_o + lane_addr + kOutCols * half + c, *reinterpret_cast<uint32_t(*)[32]>(&o[c]));
       tc::tmem_ld_wait();
       float* hs = half_sum + (n_done & 1) * 256;              // double-buffered by item parity
       hs[half * 128 + row] = l_run;
@@ -363,9 +395,9 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (m < p.M) {
         const float inv = 1.f / l_tot;
         const int64_t r_out = (int64_t)b * p.M + m;
-        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * kCaDH + 32 * half);
+        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * DH + kOutCols * half);
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < kOutCols / 8; ++i)
           dst[i] = make_uint4(
               pack_bf16x2(__uint_as_float(o[8 * i]) * inv, __uint_as_float(o[8 * i + 1]) * inv),
               pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv),
@@ -381,31 +413,32 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 }
 
 inline bool cross_attn_tc_supported(int B, int M, int H, int d_h, int T_ctx) {
-  return d_h == kCaDH && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;
+  return (d_h == 64 || d_h == 128) && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;
 }
 
-inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stride, const uint16_t* k,
-                                           const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
-                                           int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
-                                           int B, int M, int H, int d_h, int T_ctx, float scale, cudaStream_t s) {
-  (void)d_h;
+template <int DH>
+inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_stride, const uint16_t* k,
+                                              const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
+                                              int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
+                                              int B, int M, int H, int T_ctx, float scale, cudaStream_t s) {
+  constexpr int kCaSmemBytes = CaCfg<DH>::kSmemBytes;
   CUtensorMap mq, mk, mv;
   {
-    const uint64_t dims[4] = {(uint64_t)kCaDH, (uint64_t)H, (uint64_t)M, (uint64_t)B};
-    const uint64_t str[3] = {(uint64_t)kCaDH, (uint64_t)q_row_stride, (uint64_t)M * (uint64_t)q_row_stride};
-    const uint32_t box[4] = {(uint32_t)kCaDH, 1u, (uint32_t)kCaBM, 1u};
+    const uint64_t dims[4] = {(uint64_t)DH, (uint64_t)H, (uint64_t)M, (uint64_t)B};
+    const uint64_t str[3] = {(uint64_t)DH, (uint64_t)q_row_stride, (uint64_t)M * (uint64_t)q_row_stride};
+    const uint32_t box[4] = {64u, 1u, (uint32_t)kCaBM, 1u};
     if (!tc::make_tmap_bf16(&mq, q, 4, dims, str, box)) return GRACE_CUDA_ERROR;
   }
   {
-    const uint64_t dims[4] = {(uint64_t)kCaDH, (uint64_t)T_ctx, (uint64_t)H, (uint64_t)B};
+    const uint64_t dims[4] = {(uint64_t)DH, (uint64_t)T_ctx, (uint64_t)H, (uint64_t)B};
     const uint64_t str[3] = {(uint64_t)kv_stride_t, (uint64_t)kv_stride_h, (uint64_t)kv_stride_b};
-    const uint32_t box[4] = {(uint32_t)kCaDH, (uint32_t)kCaBN, 1u, 1u};
+    const uint32_t box[4] = {64u, (uint32_t)kCaBN, 1u, 1u};
     if (!tc::make_tmap_bf16(&mk, k, 4, dims, str, box)) return GRACE_CUDA_ERROR;
     if (!tc::make_tmap_bf16(&mv, v, 4, dims, str, box)) return GRACE_CUDA_ERROR;
   }
   static bool attr_set = false;
   if (!attr_set) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
     attr_set = true;
   }
   static int n_sm = 0;
@@ -421,10 +454,22 @@ inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stri
   if (items > 0x7fffffff) return GRACE_UNSUPPORTED_SHAPE;
   p.total_items = (int)items;
   p.scale_log2 = scale * 1.4426950408889634f;
-  const int grid = (int)(items < 2 * n_sm ? items : 2 * n_sm);
-  cross_attn_tc_kernel<<<grid, kCaThreads, kCaSmemBytes, s>>>(mq, mk, mv, p);
+  const int ctas = CaCfg<DH>::kCtasPerSm * n_sm;
+  const int grid = (int)(items < ctas ? items : ctas);
+  cross_attn_tc_kernel<DH><<<grid, kCaThreads, kCaSmemBytes, s>>>(mq, mk, mv, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
+}
+
+inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stride, const uint16_t* k,
+                                           const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
+                                           int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
+                                           int B, int M, int H, int d_h, int T_ctx, float scale, cudaStream_t s) {
+  if (d_h == 128)
+    return launch_cross_attn_tc_dh<128>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
+                                        lse, B, M, H, T_ctx, scale, s);
+  return launch_cross_attn_tc_dh<64>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
+                                     lse, B, M, H, T_ctx, scale, s);
 }
 
 }  // namespace grace

@@ -8,7 +8,8 @@
 // 4-byte loads, warp-uniform, served by L2), then issues all K and V loads of the prefix at
 // once, and only then does the arithmetic: dot products reduced over the d_h / 8 lanes of a
 // head, fp32 softmax over the <= 8 positions, weighted sum of V.  Beam reordering never moves
-// KV: the parent arrays are the block table.
+// KV: the parent arrays are the block table.  Rows wider than 1024 elements (e.g. 16 heads of 128)
+// are cut into 1024-element segments, one warp each (blockIdx.y): heads never interact.
 #include "common.cuh"
 
 namespace grace {
@@ -52,13 +53,14 @@ self_attn_kernel(const SelfAttnParams p) {
   const int M_t = p.beam[t];
   const int b = r / M_t;
   const int pieces = p.HD >> 3;
+  const int seg_base = blockIdx.y * (NP * 32);             // first 16-byte piece of this warp's segment
 
   // own q, k, v
   const uint4* qrow = reinterpret_cast<const uint4*>(p.qkv + (int64_t)r * p.qkv_row_stride);
   uint4 q[NP], kk[T][NP], vv[T][NP];
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
-    const int pc = i * 32 + lane;
+    const int pc = seg_base + i * 32 + lane;
     if (pc < pieces) {
       q[i] = __ldg(qrow + pc);
       kk[t][i] = __ldg(qrow + pieces + pc);
@@ -80,7 +82,7 @@ self_attn_kernel(const SelfAttnParams p) {
       local = par;
     }
     rows[0] = (int64_t)b * p.beam[0] + local;
-    if (bad && lane == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
+    if (bad && lane == 0 && blockIdx.y == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
   }
   // all prefix loads in flight together
 #pragma unroll
@@ -90,7 +92,7 @@ self_attn_kernel(const SelfAttnParams p) {
     const uint4* vr = reinterpret_cast<const uint4*>(p.v_cache + off);
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
-      const int pc = i * 32 + lane;
+      const int pc = seg_base + i * 32 + lane;
       if (pc < pieces) { kk[j][i] = __ldg(kr + pc); vv[j][i] = __ldg(vr + pc); }
       else { kk[j][i] = vv[j][i] = make_uint4(0, 0, 0, 0); }
     }
@@ -102,7 +104,7 @@ self_attn_kernel(const SelfAttnParams p) {
     uint4* vw = reinterpret_cast<uint4*>(p.v_cache + off);
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
-      const int pc = i * 32 + lane;
+      const int pc = seg_base + i * 32 + lane;
       if (pc < pieces) { kw[pc] = kk[t][i]; vw[pc] = vv[t][i]; }
     }
   }
@@ -133,7 +135,7 @@ self_attn_kernel(const SelfAttnParams p) {
       acc[4] = fmaf(w, bf16_lo(v.z), acc[4]); acc[5] = fmaf(w, bf16_hi(v.z), acc[5]);
       acc[6] = fmaf(w, bf16_lo(v.w), acc[6]); acc[7] = fmaf(w, bf16_hi(v.w), acc[7]);
     }
-    const int pc = i * 32 + lane;
+    const int pc = seg_base + i * 32 + lane;
     if (pc < pieces)
       orow[pc] = make_uint4(pack_bf16x2(acc[0], acc[1]), pack_bf16x2(acc[2], acc[3]),
                             pack_bf16x2(acc[4], acc[5]), pack_bf16x2(acc[6], acc[7]));
@@ -143,7 +145,7 @@ self_attn_kernel(const SelfAttnParams p) {
 template <int T, int NP>
 static grace_status_t launch_dh(const SelfAttnParams& p, int d_h, cudaStream_t s) {
   const int warps = 4;
-  const int blocks = (p.R + warps - 1) / warps;
+  const dim3 blocks((p.R + warps - 1) / warps, (p.HD / 8 + NP * 32 - 1) / (NP * 32));
   switch (d_h) {
     case 32: self_attn_kernel<T, NP, 32><<<blocks, warps * 32, 0, s>>>(p); break;
     case 64: self_attn_kernel<T, NP, 64><<<blocks, warps * 32, 0, s>>>(p); break;
@@ -161,7 +163,7 @@ static grace_status_t launch_np(const SelfAttnParams& p, int d_h, cudaStream_t s
     case 1: return launch_dh<T, 1>(p, d_h, s);
     case 2: return launch_dh<T, 2>(p, d_h, s);
     case 3: case 4: return launch_dh<T, 4>(p, d_h, s);
-    default: return GRACE_UNSUPPORTED_SHAPE;
+    default: return launch_dh<T, 4>(p, d_h, s);            // wider rows: segments of 4 x 32 pieces
   }
 }
 
@@ -178,7 +180,7 @@ extern "C" grace_status_t grace_self_attn(const uint16_t* qkv, int64_t qkv_row_s
   if (B <= 0 || H <= 0 || t < 0) return GRACE_INVALID_ARG;
   if (t >= kMaxSelfSteps || (d_h != 32 && d_h != 64 && d_h != 128)) return GRACE_UNSUPPORTED_SHAPE;
   const int HD = H * d_h;
-  if (HD > 1024) return GRACE_UNSUPPORTED_SHAPE;
+  if (HD > 8192) return GRACE_UNSUPPORTED_SHAPE;
   if (!grace_aligned16(qkv) || !grace_aligned16(k_cache) || !grace_aligned16(v_cache) || !grace_aligned16(out) ||
       (qkv_row_stride & 7) || (out_row_stride & 7) || qkv_row_stride < 3 * HD || out_row_stride < HD)
     return GRACE_INVALID_ARG;

@@ -349,6 +349,8 @@ def _self_attn_problem(seed, B, beam_sizes, H, d, L):
     (3, [1], 8, 64), (3, [1, 37], 8, 64), (2, [1, 50, 70], 8, 64), (2, [1, 64, 64, 130], 8, 64),
     (2, [5, 64, 64, 64, 33], 8, 64), (1, [1, 16, 16], 4, 32), (2, [1, 20, 20, 20], 16, 64), (2, [1, 9, 9], 4, 128),
     (1, [2, 3, 4, 5, 6, 7, 8, 9], 2, 64),
+    (2, [1, 24, 40, 40], 16, 128),          # the paper's decoder width: rows of 2048 = two 1024-element segments
+    (1, [1, 10, 10], 20, 64),               # 1280-wide rows: ragged second segment
 ])
 def test_self_attn_matches_oracle(api, B, beam_sizes, H, d):
     L = max(5, len(beam_sizes))
@@ -393,7 +395,9 @@ def test_self_attn_flags_bad_parent(api):
     (3, 256, 8, 64, 512),          # config-2 slice
     (2, 384, 4, 64, 1024),         # long encoder
     (2, 70, 2, 64, 200),           # T not a multiple of the K/V block
-    (2, 33, 2, 128, 96),
+    (2, 33, 2, 128, 96),           # head size 128 (two 64-wide halves per tile): one ragged block
+    (2, 300, 16, 128, 128),        # the paper's decoder shape: 16 heads of 128, 128 context tokens
+    (1, 130, 4, 128, 333),         # head size 128 over several K/V blocks, ragged M and T
     (1, 1, 8, 64, 1024),           # step 0 of the decode loop: one row per request
 ])
 def test_cross_attn_matches_oracle(api, B, M, H, d, T):
