@@ -10,7 +10,7 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
       d->L > GRACE_MAX_STEPS || d->H <= 0 || d->T_ctx <= 0)
     return GRACE_INVALID_ARG;
   if ((d->d_h != 32 && d->d_h != 64 && d->d_h != 128) || d->d_model % 64 || d->d_ffn % 64 ||
-      (d->H * d->d_h) % 64 || d->V % 64 || d->V <= 0 || d->V >= 65535 || d->d_model > 4096 || d->H * d->d_h > 1024)
+      (d->H * d->d_h) % 64 || d->V % 64 || d->V <= 0 || d->V >= 65535 || d->d_model > (d->x ? 4096 : 2048) || d->H * d->d_h > 8192)
     return GRACE_UNSUPPORTED_SHAPE;
   int64_t mmax = 0;
   for (int t = 0; t <= d->L; ++t) {
