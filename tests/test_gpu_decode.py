@@ -18,15 +18,16 @@ from gpu_util import DEV, dev  # noqa: E402
 
 
 def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=2000, V=64, seed_variant=0,
-             std=0.02):
+             std=0.02, shape=(2, 128, 4, 32, 512, 128), T_ctx=64):
+    """shape = (layers, d_model, heads, head size, FFN width, encoder width)."""
     rng = synth.rng_for(1, seed_variant)
-    L = 3
+    L = len(schedule)
     sids = synth.catalog(rng, n_sids, V, L)
     trie = SidTrie(sids, V)
     elig = [synth.eligible_subset(rng, n_sids, 0.3) for _ in range(B)]
-    shp = synth.DecoderShape(2, 128, 4, 32, 512, 128, V, L)
+    shp = synth.DecoderShape(*shape, V, L)
     w = synth.decoder_weights(rng, shp, std=std, as_bf16=True)
-    enc = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, 64, 128)))
+    enc = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, T_ctx, shape[5])))
     return dict(sids=sids, trie=trie, elig=elig, shp=shp, w=w, enc=enc, schedule=schedule, final_k=final_k, B=B,
                 matcher_kind=matcher_kind)
 
@@ -58,13 +59,18 @@ def _oracle_matcher(cfg):
     return OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 14, 4) for e in cfg["elig"]])
 
 
-@pytest.mark.parametrize("B,kind,schedule,final_k,residual_bf16", [
-    (1, "node", (1, 16, 16), 16, False),     # configuration 1
-    (3, "bloom", (1, 40, 24), 32, False),    # several requests, dynamic per-step beam sizes, Bloom matcher
-    (3, "bloom", (1, 40, 24), 32, True),     # the same with the residual stream held in bf16
+# the paper's decoder geometry, narrowed: 16 heads of 128 (rows of 2048), 128 context tokens, 4 levels
+_PAPER_LIKE = dict(shape=(2, 256, 16, 128, 512, 256), T_ctx=128, n_sids=4000)
+
+
+@pytest.mark.parametrize("B,kind,schedule,final_k,residual_bf16,extra", [
+    (1, "node", (1, 16, 16), 16, False, {}),     # configuration 1
+    (3, "bloom", (1, 40, 24), 32, False, {}),    # several requests, dynamic per-step beam sizes, Bloom matcher
+    (3, "bloom", (1, 40, 24), 32, True, {}),     # the same with the residual stream held in bf16
+    (2, "bloom", (1, 24, 48, 48), 48, True, _PAPER_LIKE),   # dynamic schedule over 4 levels, head size 128
 ])
-def test_decode_step_teacher_forced(B, kind, schedule, final_k, residual_bf16):
-    cfg = _config1(B=B, matcher_kind=kind, schedule=schedule, final_k=final_k)
+def test_decode_step_teacher_forced(B, kind, schedule, final_k, residual_bf16, extra):
+    cfg = _config1(B=B, matcher_kind=kind, schedule=schedule, final_k=final_k, **extra)
     shp, trie = cfg["shp"], cfg["trie"]
     record = []
     OD.beam_search(cfg["w"], shp, cfg["enc"], trie, _oracle_matcher(cfg), schedule, final_k, record=record)
