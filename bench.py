@@ -558,10 +558,10 @@ def main():
         line["op_breakdown"] = bd
         top = max(bd, key=lambda k: bd[k]["ms_per_loop"])
         # DRAM bytes per flop of the dominant kernels, from the committed ncu captures under profiles/
-        # (linear_persistent_kernel 32768x2048x512: 110.4 MB for 68.7 GFLOP; cross_attn_tc_kernel B16 M2048 T1024:
+        # (linear_pair_kernel 32768x2048x512: 111.2 MB for 68.7 GFLOP; cross_attn_tc_kernel B16 M2048 T1024:
         # 73.8 MB for 68.7 GFLOP); the bench's launches are larger than a capture may be, so the traffic is scaled
         # by the flops of an average launch (it grows in proportion: every tile streams its operands once).
-        dram_bytes_per_flop = {"linear": 110.43e6 / 68.72e9, "cross_attn": 73.85e6 / 68.72e9}
+        dram_bytes_per_flop = {"linear": 111.23e6 / 68.72e9, "cross_attn": 73.85e6 / 68.72e9}
         if top in ("linear", "cross_attn") and not default_workload:
             ach = bd[top]["flops_per_loop"] / (bd[top]["ms_per_loop"] * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
