@@ -16,6 +16,11 @@ Pin status (what each function is checked against, besides itself):
                                     no-false-negative property of OR-unions.
   matchers.PrefixBloom, node_eligibility  pinned: brute-force membership,
                                     analytic false-positive rate.
+  kway.* (k-way partitioned rows)   pinned: k = 1 equals the union index, the
+                                    Section 4.2 example is filtered with two
+                                    groups, ad-level eligibility never lost,
+                                    one group per SID is exact, greedy rule by
+                                    hand.
   gtm.gtm_mask                      pinned: brute force over all (row, token).
   topk.beam_topk                    pinned: python sorted() with the same key.
   decoder.beam_search               pinned: exhaustive enumeration on tiny

@@ -169,7 +169,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (progressed) {
           idle = 0;
         } else {
-          __nanosleep(64);
+          __nanosleep(512);                                 // polling costs issue slots the softmax warps of this scheduler need
           if (++idle > (1 << 24)) *abort_flag = 1;           // bounded: about a second of nothing to do
         }
       }

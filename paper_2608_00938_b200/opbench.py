@@ -42,6 +42,7 @@ def main():
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--relu", action="store_true")
     ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
+    ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
     a = ap.parse_args()
     dev = "cuda:0"
     torch.manual_seed(0)
@@ -106,8 +107,13 @@ def main():
         node = torch.arange(R, device=dev, dtype=torch.int32)
         key = torch.randint(1, a.V, (R,), device=dev, dtype=torch.int64)
         cand = torch.empty_like(logp)
-        us = _time(lambda: api.grace_gtm_mask(logp, score, node, key, trie, matcher, cand, None, a.B, a.M, 1), a.iters)
-        print(f"mask[{a.matcher}] R={R} V={a.V} density={a.density}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s "
+        if a.logits:
+            lse = torch.empty(R, device=dev)
+            us = _time(lambda: api.grace_gtm_mask_logits(logp, lse, score, node, key, trie, matcher, cand, None, a.B, a.M, 1),
+                       a.iters)
+        else:
+            us = _time(lambda: api.grace_gtm_mask(logp, score, node, key, trie, matcher, cand, None, a.B, a.M, 1), a.iters)
+        print(f"mask[{a.matcher}{', fused log-softmax' if a.logits else ''}] R={R} V={a.V} density={a.density}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s "
               f"(dense-form bytes)")
     elif a.op == "lookup":
         # the paper's index form on a synthetic catalog: --N SIDs (thousands), vocabulary --V, depth --t beams
