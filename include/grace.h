@@ -206,6 +206,11 @@ typedef struct {
   const uint64_t* bloom_table;      /* [n_bloom_rows][W_bl]                              */
   const uint64_t* user_bitmask;     /* [B][W_bm]                                         */
   const uint64_t* user_blooms;      /* [B][N_loc][W_bl]                                  */
+  /* k-way partitioned rows (Section 4.2 "k-way partition", Section 4.4): NULL = one pair of rows per
+   * child entry.  Otherwise [num_entries + 1]: entry j owns the partition slots part_offsets[j] ..
+   * part_offsets[j+1]-1, bitmask_index / bloom_index are indexed by SLOT (length part_offsets[num_entries]),
+   * and an entry is kept iff ANY of its slots passes the bitmask test and the Bloom test. */
+  const int32_t* part_offsets;
 } grace_gtm_index_t;
 
 /* Host-side builder.  sids host int32 [n_sids][L] sorted and distinct; ads sorted by SID:
@@ -221,6 +226,26 @@ grace_status_t grace_gtm_index_build(const int32_t* sids, int64_t n_sids, int V,
                                      int32_t* bitmask_index, int32_t* bloom_index,
                                      uint64_t* bitmask_table, int64_t* n_bitmask_rows,
                                      uint64_t* bloom_table, int64_t* n_bloom_rows);
+
+/* The same index with k-way partitioned rows (Section 4.2, "k-way partition"): the SIDs below a node are
+ * split into groups and one (bitmask, Bloom) pair of union rows is stored per group, in the jagged
+ * layout of Section 4.4 (the fixed-width layout of static k-way is the case of equal row lengths).
+ *   static  : k_level host int32 [L + 1], k_level[l] = k of the entries that lead to nodes of level l
+ *   dynamic : k_level NULL; per node the smallest k in 1..min(k_max, #SIDs below) whose fullest group
+ *             has fill (set bits of the pair / its width) <= fill_target, else that upper bound
+ * Construction is greedy in SID order: a SID joins the group whose pair has the fewest set bits after
+ * OR-ing the SID's rows in (ties: lowest group); empty groups are not stored.
+ * part_offsets host [num_nodes] (= entries + 1).  Call once with part_bitmask_index, part_bloom_index and
+ * both tables NULL to learn *n_parts and the table sizes, then again with arrays of those sizes. */
+grace_status_t grace_gtm_index_build_kway(const int32_t* sids, int64_t n_sids, int V, int L,
+                                          const int64_t* ad_sid, int64_t n_ads, const uint64_t* ad_bitmask,
+                                          int W_bm, const uint64_t* ad_bloom, int W_bl,
+                                          const int32_t* k_level, double fill_target, int k_max,
+                                          int32_t* node_offsets, int32_t* csr_child_nodes, int16_t* csr_tokens,
+                                          int32_t* part_offsets, int32_t* part_bitmask_index,
+                                          int32_t* part_bloom_index, int64_t* n_parts,
+                                          uint64_t* bitmask_table, int64_t* n_bitmask_rows,
+                                          uint64_t* bloom_table, int64_t* n_bloom_rows);
 
 /* CD + GTM lookup and score add on the index above (the kernel of Section 5.4): for every beam the
  * child-entry range of its node is scanned, bitmask first (stop at the first failing word), Bloom

@@ -44,7 +44,7 @@ class GtmIndexStruct(C.Structure):
                 ("reserved", C.c_int32), ("num_nodes", C.c_int64), ("num_entries", C.c_int64),
                 ("node_offsets", _vp), ("csr_child_nodes", _vp), ("csr_tokens", _vp), ("bitmask_index", _vp),
                 ("bloom_index", _vp), ("bitmask_table", _vp), ("bloom_table", _vp), ("user_bitmask", _vp),
-                ("user_blooms", _vp)]
+                ("user_blooms", _vp), ("part_offsets", _vp)]
 
 
 class LayerStruct(C.Structure):
@@ -98,6 +98,9 @@ _gtm_mask_logits = _sig("grace_gtm_mask_logits", _i32, [_vp, _vp, _vp, _vp, _vp,
                                                        C.POINTER(MatcherStruct), _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
 _gtm_index_build = _sig("grace_gtm_index_build", _i32, [_vp, _i64, _i32, _i32, _vp, _i64, _vp, _i32, _vp, _i32,
                                                        _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
+_gtm_index_build_kway = _sig("grace_gtm_index_build_kway", _i32,
+                             [_vp, _i64, _i32, _i32, _vp, _i64, _vp, _i32, _vp, _i32, _vp, C.c_double, _i32,
+                              _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
 _beam_update_csr = _sig("grace_beam_update_csr", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp,
                                                        _i32, _i32, _i32, _i32, _vp, _vp])
@@ -230,6 +233,40 @@ def grace_gtm_index_build(sids: np.ndarray, V: int, ad_sid: np.ndarray, ad_bitma
     return out
 
 
+def grace_gtm_index_build_kway(sids: np.ndarray, V: int, ad_sid: np.ndarray, ad_bitmask: np.ndarray, ad_bloom: np.ndarray,
+                               k_level=None, fill_target: float = 0.0, k_max: int = 1):
+    """Host build of the index with k-way partitioned rows: static (k_level[l] per node level) or dynamic
+    (fill_target, k_max).  Returns the dict of grace_gtm_index_build plus part_offsets; bitmask_index and
+    bloom_index are per partition slot."""
+    n, L = sids.shape
+    num_nodes = int(grace_trie_count_nodes(sids, V)[-1])
+    E = num_nodes - 1
+    W_bm, W_bl = ad_bitmask.shape[1], ad_bloom.shape[1]
+    out = dict(node_offsets=np.empty(num_nodes + 1, np.int32), csr_child_nodes=np.empty(E, np.int32),
+               csr_tokens=np.empty(E, np.int16), part_offsets=np.empty(E + 1, np.int32))
+    ad_sid = np.ascontiguousarray(ad_sid, dtype=np.int64)
+    kl = None if k_level is None else np.ascontiguousarray(k_level, dtype=np.int32)
+    assert kl is None or kl.shape[0] == L + 1
+    n_parts, n_bm, n_bl = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+
+    def call(pbm, pbl, bm_table, bl_table):
+        return _gtm_index_build_kway(_hp(sids, np.int32), n, V, L, ad_sid.ctypes.data, ad_sid.shape[0],
+                                     _hp(ad_bitmask, np.uint64), W_bm, _hp(ad_bloom, np.uint64), W_bl,
+                                     None if kl is None else kl.ctypes.data, float(fill_target), int(k_max),
+                                     out["node_offsets"].ctypes.data, out["csr_child_nodes"].ctypes.data,
+                                     out["csr_tokens"].ctypes.data, out["part_offsets"].ctypes.data, pbm, pbl,
+                                     C.addressof(n_parts), bm_table, C.addressof(n_bm), bl_table, C.addressof(n_bl))
+    _check(call(None, None, None, None), "grace_gtm_index_build_kway (sizes)")
+    out["bitmask_index"] = np.empty(n_parts.value, np.int32)
+    out["bloom_index"] = np.empty(n_parts.value, np.int32)
+    out["bitmask_table"] = np.empty((n_bm.value, W_bm), np.uint64)
+    out["bloom_table"] = np.empty((n_bl.value, W_bl), np.uint64)
+    _check(call(out["bitmask_index"].ctypes.data, out["bloom_index"].ctypes.data, out["bitmask_table"].ctypes.data,
+                out["bloom_table"].ctypes.data), "grace_gtm_index_build_kway")
+    out.update(num_nodes=num_nodes, V=V, L=L)
+    return out
+
+
 def make_gtm_index(host_index: dict, user_bitmask: np.ndarray, user_blooms: np.ndarray, device="cuda:0") -> GtmIndexStruct:
     """Upload a host index (from grace_gtm_index_build) and the per-request rows; returns the C struct."""
     import torch
@@ -241,11 +278,14 @@ def make_gtm_index(host_index: dict, user_bitmask: np.ndarray, user_blooms: np.n
     keep = {k: up(host_index[k]) for k in ("node_offsets", "csr_child_nodes", "csr_tokens", "bitmask_index",
                                            "bloom_index", "bitmask_table", "bloom_table")}
     keep["user_bitmask"], keep["user_blooms"] = up(user_bitmask), up(user_blooms)
+    if host_index.get("part_offsets") is not None:          # k-way partitioned rows: the index arrays are per slot
+        keep["part_offsets"] = up(host_index["part_offsets"])
     s = GtmIndexStruct(host_index["V"], host_index["L"], user_bitmask.shape[1], host_index["bloom_table"].shape[1],
                        user_blooms.shape[1], 0, host_index["num_nodes"], host_index["num_nodes"] - 1,
                        *[keep[k].data_ptr() for k in ("node_offsets", "csr_child_nodes", "csr_tokens", "bitmask_index",
                                                       "bloom_index", "bitmask_table", "bloom_table", "user_bitmask",
-                                                      "user_blooms")])
+                                                      "user_blooms")],
+                       keep["part_offsets"].data_ptr() if "part_offsets" in keep else None)
     s._keepalive = keep
     return s
 

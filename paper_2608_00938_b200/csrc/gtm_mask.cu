@@ -274,8 +274,13 @@ gtm_lookup_kernel(const LookupParams p) {
     dead = true;
   }
   if (!dead) {
-    const int start = __ldg(ix.node_offsets + node), end = __ldg(ix.node_offsets + node + 1);
-    int* queue = s_queue[wib];                 // child entries that passed the bitmask, waiting for Bloom
+    const int e_start = __ldg(ix.node_offsets + node), e_end = __ldg(ix.node_offsets + node + 1);
+    // With k-way partitioned rows the scan runs over the partition slots of the node's entries (one
+    // contiguous range, since slots follow entry order); a slot that passes both tests keeps its entry.
+    const bool kway = (ix.part_offsets != nullptr);
+    const int start = kway ? __ldg(ix.part_offsets + e_start) : e_start;
+    const int end = kway ? __ldg(ix.part_offsets + e_end) : e_end;
+    int* queue = s_queue[wib];                 // slots that passed the bitmask, waiting for Bloom
     int queued = 0;
     for (int j0 = start; j0 < end || queued > 0; j0 += 32) {
       // ---- bitmask stage: one entry per lane, first failing word ends it ----
@@ -320,7 +325,16 @@ gtm_lookup_kernel(const LookupParams p) {
           }
         }
         if (ok) {
-          const int tok = (int)__ldg(ix.csr_tokens + e);
+          int entry = e;
+          if (kway) {                          // the entry that owns slot e: last one whose first slot is <= e
+            int lo = e_start, hi = e_end - 1;
+            while (lo < hi) {
+              const int mid = (lo + hi + 1) >> 1;
+              if (__ldg(ix.part_offsets + mid) <= e) lo = mid; else hi = mid - 1;
+            }
+            entry = lo;
+          }
+          const int tok = (int)__ldg(ix.csr_tokens + entry);
           if (tok >= 0 && tok < V) atomicOr(&allow[tok >> 6], 1ull << (tok & 63));
         }
         __syncwarp();

@@ -237,6 +237,143 @@ extern "C" grace_status_t grace_gtm_index_build(const int32_t* sids, int64_t n_s
   return GRACE_OK;
 }
 
+namespace {
+inline int popcount_row(const uint64_t* a, const uint64_t* b, int W) {   // set bits of a | b
+  int n = 0;
+  for (int w = 0; w < W; ++w) n += __builtin_popcountll(a[w] | b[w]);
+  return n;
+}
+// Greedy split of the SIDs [lo, hi) into at most k groups (smallest fill after the OR, lowest group on
+// ties).  Group rows are written to g_bm / g_bl ([k][W]); returns the largest group popcount and marks
+// the groups that received a SID.
+int greedy_groups(const uint64_t* leaf_bm, const uint64_t* leaf_bl, int64_t lo, int64_t hi, int k, int W_bm, int W_bl,
+                  std::vector<uint64_t>& g_bm, std::vector<uint64_t>& g_bl, std::vector<char>& used) {
+  g_bm.assign((size_t)k * W_bm, 0);
+  g_bl.assign((size_t)k * W_bl, 0);
+  used.assign(k, 0);
+  for (int64_t i = lo; i < hi; ++i) {
+    int best = 0, best_pc = 1 << 30;
+    for (int g = 0; g < k; ++g) {
+      const int pc = popcount_row(&g_bm[(size_t)g * W_bm], leaf_bm + i * W_bm, W_bm) +
+                     popcount_row(&g_bl[(size_t)g * W_bl], leaf_bl + i * W_bl, W_bl);
+      if (pc < best_pc) { best_pc = pc; best = g; }
+    }
+    for (int w = 0; w < W_bm; ++w) g_bm[(size_t)best * W_bm + w] |= leaf_bm[i * W_bm + w];
+    for (int w = 0; w < W_bl; ++w) g_bl[(size_t)best * W_bl + w] |= leaf_bl[i * W_bl + w];
+    used[best] = 1;
+  }
+  int max_pc = 0;
+  for (int g = 0; g < k; ++g) {
+    if (!used[g]) continue;
+    int pc = 0;
+    for (int w = 0; w < W_bm; ++w) pc += __builtin_popcountll(g_bm[(size_t)g * W_bm + w]);
+    for (int w = 0; w < W_bl; ++w) pc += __builtin_popcountll(g_bl[(size_t)g * W_bl + w]);
+    if (pc > max_pc) max_pc = pc;
+  }
+  return max_pc;
+}
+}  // namespace
+
+extern "C" grace_status_t grace_gtm_index_build_kway(const int32_t* sids, int64_t n_sids, int V, int L,
+                                                     const int64_t* ad_sid, int64_t n_ads, const uint64_t* ad_bitmask,
+                                                     int W_bm, const uint64_t* ad_bloom, int W_bl,
+                                                     const int32_t* k_level, double fill_target, int k_max,
+                                                     int32_t* node_offsets, int32_t* csr_child_nodes,
+                                                     int16_t* csr_tokens, int32_t* part_offsets,
+                                                     int32_t* part_bitmask_index, int32_t* part_bloom_index,
+                                                     int64_t* n_parts, uint64_t* bitmask_table, int64_t* n_bitmask_rows,
+                                                     uint64_t* bloom_table, int64_t* n_bloom_rows) {
+  if (!ad_sid || !ad_bitmask || !ad_bloom || !node_offsets || !csr_child_nodes || !csr_tokens || !part_offsets ||
+      !n_parts || !n_bitmask_rows || !n_bloom_rows || n_ads <= 0 || W_bm <= 0 || W_bl <= 0 || V > 32767)
+    return GRACE_INVALID_ARG;
+  const bool sizing = (part_bitmask_index == nullptr);
+  if ((part_bloom_index == nullptr) != sizing || (bitmask_table == nullptr) != sizing || (bloom_table == nullptr) != sizing)
+    return GRACE_INVALID_ARG;
+  if (k_level == nullptr && k_max < 1) return GRACE_INVALID_ARG;
+  if (k_level != nullptr)
+    for (int l = 1; l <= L; ++l)
+      if (k_level[l] < 1) return GRACE_INVALID_ARG;
+  std::vector<int64_t> level_start(L + 2);
+  grace_status_t st = grace_trie_count_nodes(sids, n_sids, V, L, level_start.data());
+  if (st != GRACE_OK) return st;
+  const int64_t num_nodes = level_start[L + 1];
+  for (int64_t a = 0; a < n_ads; ++a) {
+    if (ad_sid[a] < 0 || ad_sid[a] >= n_sids || (a > 0 && ad_sid[a] < ad_sid[a - 1])) return GRACE_INVALID_ARG;
+    if (a > 0 && ad_sid[a] > ad_sid[a - 1] + 1) return GRACE_INVALID_ARG;
+  }
+  if (ad_sid[0] != 0 || ad_sid[n_ads - 1] != n_sids - 1) return GRACE_INVALID_ARG;
+  // rows of a SID: OR over its ads
+  std::vector<uint64_t> leaf_bm((size_t)n_sids * W_bm, 0), leaf_bl((size_t)n_sids * W_bl, 0);
+  for (int64_t a = 0; a < n_ads; ++a) {
+    for (int w = 0; w < W_bm; ++w) leaf_bm[(size_t)ad_sid[a] * W_bm + w] |= ad_bitmask[a * W_bm + w];
+    for (int w = 0; w < W_bl; ++w) leaf_bl[(size_t)ad_sid[a] * W_bl + w] |= ad_bloom[a * W_bl + w];
+  }
+  // trie structure (as in grace_gtm_index_build) and, per node, the run of SIDs below it
+  std::vector<int64_t> cur(L + 1, 0), next_id(L + 1), parent_of((size_t)num_nodes, -1);
+  std::vector<int64_t> sid_lo((size_t)num_nodes, 0), sid_hi((size_t)num_nodes, 0);
+  std::vector<int16_t> token_of((size_t)num_nodes, 0);
+  std::vector<int8_t> level_of((size_t)num_nodes, 0);
+  for (int l = 0; l <= L; ++l) next_id[l] = level_start[l];
+  for (int64_t i = 0; i < n_sids; ++i) {
+    const int d = first_diff(sids, i, L);
+    for (int l = d + 1; l <= L; ++l) {
+      cur[l] = next_id[l]++;
+      parent_of[cur[l]] = cur[l - 1];
+      token_of[cur[l]] = (int16_t)sids[i * L + l - 1];
+      level_of[cur[l]] = (int8_t)l;
+      sid_lo[cur[l]] = i;
+    }
+    for (int l = 1; l <= L; ++l) sid_hi[cur[l]] = i + 1;
+  }
+  for (int64_t n = 0; n <= num_nodes; ++n) node_offsets[n] = 0;
+  for (int64_t c = 1; c < num_nodes; ++c) ++node_offsets[parent_of[c] + 1];
+  for (int64_t n = 0; n < num_nodes; ++n) node_offsets[n + 1] += node_offsets[n];
+  RowTable bm_rows(W_bm), bl_rows(W_bl);
+  std::vector<uint64_t> g_bm, g_bl;
+  std::vector<char> used;
+  const int bits = 64 * (W_bm + W_bl);
+  int64_t slot = 0;
+  part_offsets[0] = 0;
+  for (int64_t c = 1; c < num_nodes; ++c) {
+    const int64_t j = c - 1, lo = sid_lo[c], hi = sid_hi[c];
+    csr_child_nodes[j] = (int32_t)c;
+    csr_tokens[j] = token_of[c];
+    int k;
+    if (k_level != nullptr) {
+      k = (int)std::max<int64_t>(1, std::min<int64_t>(k_level[level_of[c]], hi - lo));
+      greedy_groups(leaf_bm.data(), leaf_bl.data(), lo, hi, k, W_bm, W_bl, g_bm, g_bl, used);
+    } else {
+      const int k_top = (int)std::max<int64_t>(1, std::min<int64_t>(k_max, hi - lo));
+      for (k = 1; k <= k_top; ++k) {
+        const int max_pc = greedy_groups(leaf_bm.data(), leaf_bl.data(), lo, hi, k, W_bm, W_bl, g_bm, g_bl, used);
+        if ((double)max_pc / (double)bits <= fill_target || k == k_top) break;
+      }
+    }
+    for (int g = 0; g < k; ++g) {
+      if (!used[g]) continue;
+      const int32_t ib = bm_rows.add(&g_bm[(size_t)g * W_bm]), il = bl_rows.add(&g_bl[(size_t)g * W_bl]);
+      if (!sizing) {
+        if (slot >= *n_parts) return GRACE_WORKSPACE_TOO_SMALL;
+        part_bitmask_index[slot] = ib;
+        part_bloom_index[slot] = il;
+      }
+      ++slot;
+    }
+    if (slot > 0x7fffffff) return GRACE_UNSUPPORTED_SHAPE;
+    part_offsets[j + 1] = (int32_t)slot;
+  }
+  if (!sizing) {
+    if (*n_bitmask_rows < (int64_t)bm_rows.ids.size() || *n_bloom_rows < (int64_t)bl_rows.ids.size())
+      return GRACE_WORKSPACE_TOO_SMALL;
+    std::copy(bm_rows.rows.begin(), bm_rows.rows.end(), bitmask_table);
+    std::copy(bl_rows.rows.begin(), bl_rows.rows.end(), bloom_table);
+  }
+  *n_parts = slot;
+  *n_bitmask_rows = (int64_t)bm_rows.ids.size();
+  *n_bloom_rows = (int64_t)bl_rows.ids.size();
+  return GRACE_OK;
+}
+
 extern "C" const char* grace_status_string(grace_status_t s) {
   switch (s) {
     case GRACE_OK: return "ok";

@@ -42,6 +42,7 @@ def main():
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--relu", action="store_true")
     ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
+    ap.add_argument("--kway", type=int, default=1, help="lookup: static k-way partitioned rows with this k at every level")
     ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
     a = ap.parse_args()
     dev = "cuda:0"
@@ -126,7 +127,10 @@ def main():
         loc_rows = synth.location_rows(rng, layout)
         ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n_sids, layout, loc_rows)
         ubm, ubl, _ = synth.request_attributes(rng, a.B, layout, loc_rows, n_loc=64)
-        h = api.grace_gtm_index_build(sids, a.V, ad_sid, ad_bm, ad_bl)
+        if a.kway > 1:
+            h = api.grace_gtm_index_build_kway(sids, a.V, ad_sid, ad_bm, ad_bl, k_level=[a.kway] * (L + 1))
+        else:
+            h = api.grace_gtm_index_build(sids, a.V, ad_sid, ad_bm, ad_bl)
         index = api.make_gtm_index(h, ubm, np.ascontiguousarray(ubl), dev)
         level = np.unique(sids[:, :depth], axis=0)                      # nodes of that depth, in id order
         first = int(api.grace_trie_count_nodes(sids, a.V)[depth])
@@ -140,6 +144,10 @@ def main():
         us = _time(lambda: api.grace_gtm_lookup(logp, score, node, index, cand, allow, a.B, a.M), a.iters)
         deg = np.diff(h["node_offsets"])[first + pick].mean()
         frac = float((allow != 0).any(dim=1).float().mean())
+        kept = float(torch.isfinite(cand).float().sum()) / R
+        slots = h["bitmask_index"].shape[0]
+        print(f"lookup R={R} V={a.V} depth={depth} k={a.kway}: kept {kept:.1f} of {deg:.1f} children per beam, "
+              f"{slots} matcher slots")
         print(f"lookup R={R} V={a.V} depth={depth}: {us:.1f} us, {2 * R * a.V * 4 / us / 1e3:.0f} GB/s (dense-form bytes); "
               f"children/beam {deg:.1f}, rows with a survivor {frac:.2f}, tables {h['bitmask_table'].shape[0]} / "
               f"{h['bloom_table'].shape[0]} unique rows for {h['num_nodes'] - 1} entries")

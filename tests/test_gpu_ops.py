@@ -217,6 +217,54 @@ def test_gtm_lookup_paper_form_matches_oracle(api, V, L, n_sids, B, M, depth, n_
     assert np.array_equal(host_u64(new_key), key_ref)
 
 
+@pytest.mark.parametrize("policy,depth,M", [(("static", [0, 4, 3, 2, 1]), 1, 33), (("static", [0, 4, 3, 2, 1]), 0, 1),
+                                            (("dynamic", 0.35, 6), 2, 40), (("dynamic", 0.0, 16), 1, 20)])
+def test_gtm_lookup_kway_partitions_match_oracle(api, policy, depth, M):
+    """k-way partitioned rows (Section 4.2 "k-way partition"): a child is kept iff ANY of its groups passes the
+    bitmask and the Bloom test; the kernel scans the partition slots of the beam's node."""
+    from oracle import kway as KW
+    V, L, n_sids, B = 256, 4, 6000, 3
+    rng = synth.rng_for(4, 700 + depth)
+    sids = synth.catalog(rng, n_sids, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout()
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n_sids, layout, loc_rows)
+    ubm, ubl, _ = synth.request_attributes(rng, B, layout, loc_rows, n_loc=64)
+    ubm[0] = 0
+    o_index = KW.KWayMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl, policy)
+    node = np.full(B * M, -1, dtype=np.int32)
+    key = np.zeros(B * M, dtype=np.uint64)
+    for b in range(B):
+        pref = synth.beam_prefixes_from_sids(rng, sids, depth, M) if depth else np.zeros((1, 0), np.int32)
+        for i, pr in enumerate(pref):
+            node[b * M + i] = trie.walk(pr)
+        key[b * M: b * M + pref.shape[0]] = OM.prefix_keys(pref)
+    score = np.concatenate([synth.descending_scores(rng, M, max(depth, 1)) for _ in range(B)])
+    logp = synth.logp_rows(rng, B * M, V)
+    cand_ref, allow_ref, _ = OG.gtm_mask(logp, score, node, key, depth, trie,
+                                         KW.KWayRowsMatcher(trie, o_index, ubm, ubl), B, M)
+    # partitioning only removes candidates of the union form, and does remove some
+    plain_ref = OG.gtm_mask(logp, score, node, key, depth, trie,
+                            OM.NodeRowsMatcher(trie, OM.NodeMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl), ubm, ubl), B, M)[1]
+    assert not (allow_ref & ~plain_ref).any() and allow_ref.any()
+    if policy[0] == "static":
+        h_index = api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, k_level=policy[1])
+    else:
+        h_index = api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, fill_target=policy[1], k_max=policy[2])
+    assert np.array_equal(h_index["part_offsets"], o_index.part_offsets)
+    index = api.make_gtm_index(h_index, ubm, np.ascontiguousarray(ubl), DEV)
+    cand = torch.full((B * M, V), 7.0, device=DEV)
+    allow = torch.zeros((B * M, V // 64), dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_gtm_lookup(dev(logp), dev(score), dev(node), index, cand, allow, B, M, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(host_u64(allow), OG.pack_allow_bits(allow_ref))
+    assert np.array_equal(cand.cpu().numpy().view(np.uint32), cand_ref.view(np.uint32))
+
+
+
 # ------------------------------------------------------------------------------------------
 # beam top-k
 # ------------------------------------------------------------------------------------------

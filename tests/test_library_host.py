@@ -115,3 +115,35 @@ def test_gtm_index_builder_matches_oracle_rows(api):
     # unsorted ads are rejected
     with pytest.raises(api.GraceError):
         api.grace_gtm_index_build(sids, V, ad_sid[::-1].copy(), ad_bm, ad_bl)
+
+
+@pytest.mark.parametrize("policy", [("static", [0, 4, 2, 2, 1]), ("dynamic", 0.35, 6)])
+def test_kway_index_builder_matches_oracle(api, policy):
+    """k-way partitioned rows (Section 4.2): the library's host builder against the oracle's, slot by slot."""
+    from oracle import kway as KW
+    V, L, n = 64, 4, 1500
+    rng = synth.rng_for(4, 81)
+    sids = synth.catalog(rng, n, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout()
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n, layout, loc_rows)
+    ref = KW.KWayMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl, policy)
+    if policy[0] == "static":
+        got = api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, k_level=policy[1])
+    else:
+        got = api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, fill_target=policy[1], k_max=policy[2])
+    assert np.array_equal(got["node_offsets"], trie.node_offsets)
+    assert np.array_equal(got["csr_tokens"], trie.csr_tokens)
+    assert np.array_equal(got["part_offsets"], ref.part_offsets)
+    assert (np.diff(got["part_offsets"]) > 1).any()                  # some node really is partitioned
+    assert np.array_equal(got["bitmask_table"][got["bitmask_index"]], ref.part_bitmask_rows)
+    assert np.array_equal(got["bloom_table"][got["bloom_index"]], ref.part_bloom_rows)
+    assert got["bitmask_table"].shape == ref.bitmask_table.shape and got["bloom_table"].shape == ref.bloom_table.shape
+    # k = 1 everywhere is the unpartitioned index
+    one = api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, k_level=[1] * (L + 1))
+    plain = api.grace_gtm_index_build(sids, V, ad_sid, ad_bm, ad_bl)
+    assert np.array_equal(one["part_offsets"], np.arange(trie.num_nodes))
+    assert np.array_equal(one["bitmask_table"][one["bitmask_index"]], plain["bitmask_table"][plain["bitmask_index"]])
+    with pytest.raises(api.GraceError):
+        api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, k_level=[0] * (L + 1))
