@@ -56,15 +56,22 @@ constexpr int kMaskWarpsPerBlock = 8;
 //      log-probabilities is read only if one of its tokens is allowed.
 // LOGITS = true: `logp` holds raw logits; the row's log-sum-exp is taken in a first streaming pass
 // and cand = score + (logit - lse) for allowed tokens.
-template <int KIND, bool LOGITS>
+// SPLIT = true (few rows, e.g. step 0 with one beam per request): the eight warps of a CTA share ONE
+// row: each takes every eighth group of 32 children in phase 1 and every eighth group of 128 tokens in
+// the streaming passes; the warp-level synchronisation points become CTA barriers.
+template <int KIND, bool LOGITS, bool SPLIT>
 __global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
 gtm_mask_kernel(const MaskParams p) {
   __shared__ uint64_t s_words[kMaskWarpsPerBlock][32];
   __shared__ unsigned long long s_allow[kMaskWarpsPerBlock][32];
   __shared__ int s_incl[kMaskWarpsPerBlock][32];
+  __shared__ float s_lse[2][kMaskWarpsPerBlock];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-  const int r = blockIdx.x * kMaskWarpsPerBlock + wib;
+  const int r = SPLIT ? (int)blockIdx.x : (int)blockIdx.x * kMaskWarpsPerBlock + wib;
   if (r >= p.R) return;
+  const int part = SPLIT ? wib : 0;                      // this warp's share of the row's work
+  constexpr int kParts = SPLIT ? kMaskWarpsPerBlock : 1;
+  auto sync_row = [&]() { if (SPLIT) __syncthreads(); else __syncwarp(); };
   const int V = p.V;
   const int W = V >> 6;
   const int b = r / p.M;
@@ -87,7 +94,7 @@ gtm_mask_kernel(const MaskParams p) {
     // warp at the end (the row is not kept: phase 2 re-reads only the allowed sectors, from L2)
     float m_l = -INFINITY, s_l = 0.f;
     const int n4 = V >> 2;
-    for (int c0 = 0; c0 < n4; c0 += 128) {
+    for (int c0 = part * 128; c0 < n4; c0 += kParts * 128) {
       float4 x[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -113,12 +120,24 @@ gtm_mask_kernel(const MaskParams p) {
     float s_w = (m_l > -INFINITY) ? s_l * expf(m_l - m_w) : 0.f;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s_w += __shfl_xor_sync(kFullMask, s_w, o);
-    lse = m_w + logf(s_w);
+    if (!SPLIT) lse = m_w + logf(s_w);
+    else if (lane == 0) { s_lse[0][wib] = m_w; s_lse[1][wib] = s_w; }
   }
-  if (LOGITS && lane == 0 && p.row_lse != nullptr) p.row_lse[r] = lse;
-  uint64_t* words = s_words[wib];
-  unsigned long long* allow = s_allow[wib];
-  int* incl = s_incl[wib];
+  if (SPLIT && LOGITS) {                                 // merge the warps' (maximum, rescaled sum) pairs
+    __syncthreads();
+    if (!dead) {
+      float m_c = -INFINITY;
+      for (int w = 0; w < kMaskWarpsPerBlock; ++w) m_c = fmaxf(m_c, s_lse[0][w]);
+      float s_c = 0.f;
+      for (int w = 0; w < kMaskWarpsPerBlock; ++w)
+        if (s_lse[0][w] > -INFINITY) s_c += s_lse[1][w] * expf(s_lse[0][w] - m_c);
+      lse = m_c + logf(s_c);
+    }
+  }
+  if (LOGITS && lane == 0 && part == 0 && p.row_lse != nullptr) p.row_lse[r] = lse;
+  uint64_t* words = s_words[SPLIT ? 0 : wib];
+  unsigned long long* allow = s_allow[SPLIT ? 0 : wib];
+  int* incl = s_incl[SPLIT ? 0 : wib];
 
   int rank_before_chunk = 0;
   for (int w0 = 0; w0 < W; w0 += 32) {
@@ -132,11 +151,13 @@ gtm_mask_kernel(const MaskParams p) {
       if (lane >= d) inc += o;
     }
     const int total = __shfl_sync(kFullMask, inc, 31);
-    __syncwarp();
-    words[lane] = word;
-    incl[lane] = inc;
-    allow[lane] = (KIND == GRACE_MATCH_NONE) ? word : 0ull;
-    __syncwarp();
+    sync_row();
+    if (part == 0) {
+      words[lane] = word;
+      incl[lane] = inc;
+      allow[lane] = (KIND == GRACE_MATCH_NONE) ? word : 0ull;
+    }
+    sync_row();
 
     if (KIND == GRACE_MATCH_NODE_BITMASK) {
       // The children of a node have consecutive ids, so the eligibility bits of this lane's
@@ -157,10 +178,10 @@ gtm_mask_kernel(const MaskParams p) {
         elig >>= 1;
         rest ^= low;
       }
-      allow[lane] = out;
-      __syncwarp();
+      if (part == 0) allow[lane] = out;
+      sync_row();
     } else if (KIND != GRACE_MATCH_NONE) {
-      for (int k0 = 0; k0 < total; k0 += 32) {
+      for (int k0 = part * 32; k0 < total; k0 += kParts * 32) {
         const int k = k0 + lane;
         const bool have = k < total;
         // word holding the k-th child: smallest w with incl[w] > k
@@ -189,15 +210,15 @@ gtm_mask_kernel(const MaskParams p) {
         }
         if (ok) atomicOr(&allow[lo], 1ull << bit);
       }
-      __syncwarp();
+      sync_row();
     }
     rank_before_chunk += total;
 
-    if (p.allow_bits != nullptr && w0 + lane < W) p.allow_bits[(int64_t)r * W + w0 + lane] = allow[lane];
+    if (p.allow_bits != nullptr && part == 0 && w0 + lane < W) p.allow_bits[(int64_t)r * W + w0 + lane] = allow[lane];
     if (p.cand != nullptr) {
       const int chunk_tokens = min(2048, V - (w0 << 6));
       // 128 tokens per iteration: lane handles tokens 4*lane .. 4*lane+3 of the group
-      for (int g = 0; g < chunk_tokens; g += 128) {
+      for (int g = part * 128; g < chunk_tokens; g += kParts * 128) {
         const int tok_in_chunk = g + 4 * lane;
         if (tok_in_chunk >= chunk_tokens) continue;           // V % 64 == 0, so all 4 or none
         const uint32_t nib = (uint32_t)(allow[tok_in_chunk >> 6] >> (tok_in_chunk & 63)) & 0xfu;
@@ -219,7 +240,7 @@ gtm_mask_kernel(const MaskParams p) {
             make_float4(outv[0], outv[1], outv[2], outv[3]);
       }
     }
-    __syncwarp();
+    sync_row();
   }
   if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
 }
@@ -461,12 +482,16 @@ static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse
   p.R = B * M; p.M = M; p.V = V; p.prefix_len = prefix_len;
   p.bloom_mask_bits = 0; p.bloom_hashes = 0;
   cudaStream_t s = (cudaStream_t)stream;
-  const int blocks = (p.R + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock;
+  // few rows: a CTA per row, so that the row's matcher look-ups and its streaming passes use eight warps
+  const bool split = p.R <= 2048;
+  const int blocks = split ? p.R : (p.R + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock;
   const int threads = kMaskWarpsPerBlock * 32;
 #define GRACE_MASK_LAUNCH(K)                                                      \
   do {                                                                            \
-    if (logits) gtm_mask_kernel<K, true><<<blocks, threads, 0, s>>>(p);           \
-    else gtm_mask_kernel<K, false><<<blocks, threads, 0, s>>>(p);                 \
+    if (logits && split) gtm_mask_kernel<K, true, true><<<blocks, threads, 0, s>>>(p);        \
+    else if (logits) gtm_mask_kernel<K, true, false><<<blocks, threads, 0, s>>>(p);           \
+    else if (split) gtm_mask_kernel<K, false, true><<<blocks, threads, 0, s>>>(p);            \
+    else gtm_mask_kernel<K, false, false><<<blocks, threads, 0, s>>>(p);                      \
   } while (0)
   switch (matcher->kind) {
     case GRACE_MATCH_NONE:

@@ -54,6 +54,8 @@ def _mask_problem(seed, V, L, n_sids, B, M, depth, frac=0.3):
     (2048, 4, 30000, 2, 9, 1),        # one bitmask word per lane
     (4096, 3, 30000, 2, 5, 1),        # more than one 2048-token chunk
     (192, 3, 5000, 2, 11, 0),         # root row, V not a multiple of 128
+    # more than 2048 rows: warp-per-row kernel (fewer rows run a CTA per row)
+    (192, 3, 5000, 3, 700, 1), (4096, 3, 30000, 2, 1030, 1), (64, 3, 2000, 5, 500, 2),
 ])
 def test_gtm_mask_matches_oracle(api, kind, V, L, n_sids, B, M, depth):
     if depth == 0:
@@ -89,7 +91,8 @@ def test_gtm_mask_matches_oracle(api, kind, V, L, n_sids, B, M, depth):
 
 
 @pytest.mark.parametrize("kind", ["node", "bloom"])
-@pytest.mark.parametrize("V,M,depth", [(1024, 37, 1), (2048, 20, 1), (64, 16, 1), (1024, 50, 2)])
+@pytest.mark.parametrize("V,M,depth", [(1024, 37, 1), (2048, 20, 1), (64, 16, 1), (1024, 50, 2), (192, 1100, 1),
+                                       (1024, 1050, 2)])
 def test_gtm_mask_logits_fused_log_softmax(api, kind, V, M, depth):
     """Fused variant: raw logits in; same allow bits as the oracle (exact), candidates equal to
     score + (logit - lse) in fp32, and the row log-sum-exp within fp32 rounding of the fp64 value."""
