@@ -102,6 +102,8 @@ __device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, int nbins, 
 // threshold with high probability" is kept while the selection works on 2048 keys instead of 32768.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, TopkHeader* hdr) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ uint32_t keys[2 * kTopkThreads];
   __shared__ uint32_t hist[4096];
   __shared__ uint32_t scratch[40];
@@ -158,6 +160,8 @@ topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, Top
 }
 
 __global__ void topk_reset_kernel(TopkHeader* hdr, int B) {
+  pdl_wait();
+  pdl_trigger();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) { hdr[b].count = 0; hdr[b].t_excl = 0; hdr[b].need_exact = 1; }
 }
@@ -171,6 +175,8 @@ constexpr int kStage = 1024;                              // hits staged per CTA
 __global__ void __launch_bounds__(kCollectThreads, 5)
 topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, uint2* lists,
                     int32_t* d_status) {
+  pdl_wait();
+  pdl_trigger();
   // grid (x, B): the CTAs of column b share request b's tiles round-robin.  Hits are rare (a
   // fraction of a percent), so they are staged in shared memory and appended to the request's
   // list with ONE global atomic per flush; a per-hit or per-warp atomic on the single per-request
@@ -423,6 +429,8 @@ __global__ void __launch_bounds__(kTopkThreads)
 topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, TopkHeader* hdr,
                      uint2* lists, int force_exact, float* out_score, int32_t* out_flat, int32_t* out_parent,
                      int32_t* out_token, int32_t* d_status) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ unsigned long long sort_keys_raw[];     // kCap + kMaxK keys, then a 4096-bin histogram
   unsigned long long* sort_keys = sort_keys_raw;
   __shared__ uint32_t scratch[40];
@@ -567,7 +575,7 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
   }
   int force_exact = 1;
   if (rank != 0) {
-    topk_sample_kernel<<<B, kTopkThreads, 0, s>>>(cand, N, rank, hdr);
+    launch_pdl(topk_sample_kernel, dim3(B), dim3(kTopkThreads), 0, s, cand, N, rank, hdr);
     GRACE_LAUNCH_CHECK();
     static int collect_grid = 0;
     if (collect_grid == 0) {
@@ -583,14 +591,14 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
     if (per_request < 1) per_request = 1;
     if (per_request > tiles_per_request) per_request = tiles_per_request;
     dim3 grid((unsigned)per_request, (unsigned)B);
-    topk_collect_kernel<<<grid, kCollectThreads, 0, s>>>(cand, N, hdr, lists, d_status);
+    launch_pdl(topk_collect_kernel, dim3(grid), dim3(kCollectThreads), 0, s, cand, N, hdr, lists, d_status);
     GRACE_LAUNCH_CHECK();
     force_exact = 0;
   } else {
-    topk_reset_kernel<<<(B + 255) / 256, 256, 0, s>>>(hdr, B);
+    launch_pdl(topk_reset_kernel, dim3((B + 255) / 256), dim3(256), 0, s, hdr, B);
     GRACE_LAUNCH_CHECK();
   }
-  topk_finalize_kernel<<<B, kTopkThreads, final_smem, s>>>(cand, N, K, V, hdr, lists, force_exact, out_score, out_flat,
+  launch_pdl(topk_finalize_kernel, dim3(B), dim3(kTopkThreads), final_smem, s, cand, N, K, V, hdr, lists, force_exact, out_score, out_flat,
                                                           out_parent, out_token, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;

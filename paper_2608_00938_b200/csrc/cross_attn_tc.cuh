@@ -113,6 +113,8 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                  // barrier set-up and TMEM allocation overlapped the previous kernel's tail
+  pdl_trigger();
   const uint32_t tmem_s = tmem_base;           // S fp32, 128 columns
   const uint32_t tmem_o = tmem_base + 128;     // O fp32, DH columns
   const uint32_t tmem_p = tmem_base + 128 + DH;   // P bf16 pairs, 64 columns
@@ -456,7 +458,7 @@ inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_s
   p.scale_log2 = scale * 1.4426950408889634f;
   const int ctas = CaCfg<DH>::kCtasPerSm * n_sm;
   const int grid = (int)(items < ctas ? items : ctas);
-  cross_attn_tc_kernel<DH><<<grid, kCaThreads, kCaSmemBytes, s>>>(mq, mk, mv, p);
+  launch_pdl(cross_attn_tc_kernel<DH>, dim3(grid), dim3(kCaThreads), kCaSmemBytes, s, mq, mk, mv, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

@@ -21,6 +21,8 @@ template <int MAXV>   // float4 pieces per lane
 __global__ void __launch_bounds__(128)
 layer_norm_kernel(const float* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
                   uint16_t* __restrict__ out, int R, int D, float eps) {
+  pdl_wait();
+  pdl_trigger();
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= R) return;
@@ -68,6 +70,8 @@ template <int MAXV, int ROWS>   // MAXV: 16-byte pieces (8 bf16) per lane and ro
 __global__ void __launch_bounds__(128)
 layer_norm_bf16_kernel(const uint16_t* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
                        uint16_t* __restrict__ out, int R, int D, float eps) {
+  pdl_wait();
+  pdl_trigger();
   const int lane = threadIdx.x & 31;
   const int r0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
   if (r0 >= R) return;
@@ -148,6 +152,8 @@ layer_norm_bf16_kernel(const uint16_t* __restrict__ x, const float* __restrict__
 __global__ void embed_bf16_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
                                   const uint16_t* __restrict__ pos, uint16_t* __restrict__ x, int R, int D,
                                   int n_rows_embed, int32_t* d_status) {
+  pdl_wait();
+  pdl_trigger();
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= R) return;
@@ -169,6 +175,8 @@ __global__ void embed_bf16_kernel(const int32_t* __restrict__ token, const uint1
 __global__ void embed_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
                              const uint16_t* __restrict__ pos, float* __restrict__ x, int R, int D,
                              int n_rows_embed, int32_t* d_status) {
+  pdl_wait();
+  pdl_trigger();
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= R) return;
@@ -191,6 +199,8 @@ __global__ void embed_kernel(const int32_t* __restrict__ token, const uint16_t* 
 template <int MAXV>
 __global__ void __launch_bounds__(256)
 log_softmax_kernel(float* __restrict__ logits, int R, int V) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[8];
   const int r = blockIdx.x;
   const int n4 = V >> 2;
@@ -242,11 +252,11 @@ extern "C" grace_status_t grace_layer_norm(const float* x, const float* gamma, c
   cudaStream_t s = (cudaStream_t)stream;
   const int blocks = (R + 3) / 4;
   const int pieces = ((D >> 2) + 31) / 32;
-  if (pieces <= 2) layer_norm_kernel<2><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 4) layer_norm_kernel<4><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 8) layer_norm_kernel<8><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 16) layer_norm_kernel<16><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else layer_norm_kernel<32><<<blocks, 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  if (pieces <= 2) launch_pdl(layer_norm_kernel<2>, dim3(blocks), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 4) launch_pdl(layer_norm_kernel<4>, dim3(blocks), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 8) launch_pdl(layer_norm_kernel<8>, dim3(blocks), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 16) launch_pdl(layer_norm_kernel<16>, dim3(blocks), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else launch_pdl(layer_norm_kernel<32>, dim3(blocks), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -257,7 +267,7 @@ extern "C" grace_status_t grace_embed(const int32_t* token, const uint16_t* embe
   if (D & 3) return GRACE_UNSUPPORTED_SHAPE;
   if (!grace_aligned16(x) || (reinterpret_cast<uintptr_t>(embed) & 7) || (reinterpret_cast<uintptr_t>(pos) & 7))
     return GRACE_INVALID_ARG;
-  grace::embed_kernel<<<(R + 3) / 4, 128, 0, (cudaStream_t)stream>>>(token, embed, pos, x, R, D, n_rows_embed, d_status);
+  grace::launch_pdl(grace::embed_kernel, dim3((R + 3) / 4), dim3(128), 0, (cudaStream_t)stream, token, embed, pos, x, R, D, n_rows_embed, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -269,11 +279,11 @@ extern "C" grace_status_t grace_log_softmax(float* logits, int R, int V, void* s
   if (!grace_aligned16(logits)) return GRACE_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   const int pieces = ((V >> 2) + 255) / 256;
-  if (pieces <= 1) log_softmax_kernel<1><<<R, 256, 0, s>>>(logits, R, V);
-  else if (pieces <= 2) log_softmax_kernel<2><<<R, 256, 0, s>>>(logits, R, V);
-  else if (pieces <= 4) log_softmax_kernel<4><<<R, 256, 0, s>>>(logits, R, V);
-  else if (pieces <= 8) log_softmax_kernel<8><<<R, 256, 0, s>>>(logits, R, V);
-  else log_softmax_kernel<16><<<R, 256, 0, s>>>(logits, R, V);
+  if (pieces <= 1) launch_pdl(log_softmax_kernel<1>, dim3(R), dim3(256), 0, s, logits, R, V);
+  else if (pieces <= 2) launch_pdl(log_softmax_kernel<2>, dim3(R), dim3(256), 0, s, logits, R, V);
+  else if (pieces <= 4) launch_pdl(log_softmax_kernel<4>, dim3(R), dim3(256), 0, s, logits, R, V);
+  else if (pieces <= 8) launch_pdl(log_softmax_kernel<8>, dim3(R), dim3(256), 0, s, logits, R, V);
+  else launch_pdl(log_softmax_kernel<16>, dim3(R), dim3(256), 0, s, logits, R, V);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -288,10 +298,10 @@ extern "C" grace_status_t grace_layer_norm_bf16(const uint16_t* x, const float* 
   cudaStream_t s = (cudaStream_t)stream;
   const int pieces = ((D >> 3) + 31) / 32;
   auto blocks = [&](int rows) { return (R + 4 * rows - 1) / (4 * rows); };
-  if (pieces <= 1) layer_norm_bf16_kernel<1, 4><<<blocks(4), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 2) layer_norm_bf16_kernel<2, 4><<<blocks(4), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 4) layer_norm_bf16_kernel<4, 2><<<blocks(2), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
-  else if (pieces <= 8) layer_norm_bf16_kernel<8, 1><<<blocks(1), 128, 0, s>>>(x, gamma, beta, out, R, D, eps);
+  if (pieces <= 1) launch_pdl(layer_norm_bf16_kernel<1, 4>, dim3(blocks(4)), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 2) launch_pdl(layer_norm_bf16_kernel<2, 4>, dim3(blocks(4)), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 4) launch_pdl(layer_norm_bf16_kernel<4, 2>, dim3(blocks(2)), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
+  else if (pieces <= 8) launch_pdl(layer_norm_bf16_kernel<8, 1>, dim3(blocks(1)), dim3(128), 0, s, x, gamma, beta, out, R, D, eps);
   else return GRACE_UNSUPPORTED_SHAPE;
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
@@ -304,7 +314,7 @@ extern "C" grace_status_t grace_embed_bf16(const int32_t* token, const uint16_t*
   if (D & 3) return GRACE_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(embed) & 7) || (reinterpret_cast<uintptr_t>(pos) & 7))
     return GRACE_INVALID_ARG;
-  grace::embed_bf16_kernel<<<(R + 3) / 4, 128, 0, (cudaStream_t)stream>>>(token, embed, pos, x, R, D, n_rows_embed, d_status);
+  grace::launch_pdl(grace::embed_bf16_kernel, dim3((R + 3) / 4), dim3(128), 0, (cudaStream_t)stream, token, embed, pos, x, R, D, n_rows_embed, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

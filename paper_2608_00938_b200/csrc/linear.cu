@@ -39,6 +39,8 @@ template <int BN>
 __global__ void __launch_bounds__(128)
 linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const GemmParams p) {
+  pdl_wait();
+  pdl_trigger();
   using S = GemmSmem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -209,6 +211,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   tc::cluster_sync_all();                                  // both CTAs' barriers exist before any remote arrive
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                              // everything above overlapped the previous kernel's tail
+  pdl_trigger();
 
   if (warp == 0) {
     if (lane == 0) {                                        // ---- TMA producer (both CTAs) ----
@@ -342,10 +346,12 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   static bool attr_set = false;
   static int max_clusters = 0;
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   if (!attr_set) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
     int dev = 0, n_sm = 0;
@@ -372,7 +378,7 @@ static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw
     attr_set = true;
   }
   dim3 grid((p.N + BN - 1) / BN, (p.M + kGemmBM - 1) / kGemmBM);
-  linear_kernel<BN><<<grid, 128, GemmSmem<BN>::kTotal, s>>>(mx, mw, p);
+  launch_pdl(linear_kernel<BN>, grid, dim3(128), GemmSmem<BN>::kTotal, s, mx, mw, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

@@ -45,6 +45,8 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b) {
 template <int T, int NP, int DH>
 __global__ void __launch_bounds__(128)
 self_attn_kernel(const SelfAttnParams p) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int kLanesPerHead = DH / 8;
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -147,9 +149,9 @@ static grace_status_t launch_dh(const SelfAttnParams& p, int d_h, cudaStream_t s
   const int warps = 4;
   const dim3 blocks((p.R + warps - 1) / warps, (p.HD / 8 + NP * 32 - 1) / (NP * 32));
   switch (d_h) {
-    case 32: self_attn_kernel<T, NP, 32><<<blocks, warps * 32, 0, s>>>(p); break;
-    case 64: self_attn_kernel<T, NP, 64><<<blocks, warps * 32, 0, s>>>(p); break;
-    case 128: self_attn_kernel<T, NP, 128><<<blocks, warps * 32, 0, s>>>(p); break;
+    case 32: launch_pdl(self_attn_kernel<T, NP, 32>, blocks, dim3(warps * 32), 0, s, p); break;
+    case 64: launch_pdl(self_attn_kernel<T, NP, 64>, blocks, dim3(warps * 32), 0, s, p); break;
+    case 128: launch_pdl(self_attn_kernel<T, NP, 128>, blocks, dim3(warps * 32), 0, s, p); break;
     default: return GRACE_UNSUPPORTED_SHAPE;
   }
   GRACE_LAUNCH_CHECK();
