@@ -161,7 +161,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 // CTA issues every MMA into one of TWO TMEM accumulators (2 x 256 columns = all of TMEM), so the
 // four epilogue warps of each CTA drain tile i while the tensor cores already work on tile i+1.
 // tcgen05.commit arrives on the barriers of both CTAs, and both CTAs' TMA loads count their bytes on
-// the even CTA's "stage full" barrier (plain one-destination loads; nothing is multicast).
+// the even CTA's "stage full" barrier (plain loads, each with one destination).
 // The epilogue reads 64 (bf16) or 32 (fp32) columns at a time from TMEM, writes them to a
 // 128-byte-swizzled staging tile in shared memory and hands it to TMA: a plain tile store, or an
 // add-reduction straight into the residual stream (x += y), so the residual is never read into the SM.

@@ -166,7 +166,7 @@ __device__ __forceinline__ uint32_t cluster_addr_of(const void* p, uint32_t rank
   return ra;
 }
 // TMA tile load inside a CTA pair: the bytes land in this CTA's shared memory and are counted on the
-// barrier `bar_cluster_addr`, which may live in the pair's other CTA (no multicast: one destination).
+// barrier `bar_cluster_addr`, which may live in the pair's other CTA (a plain load with a single destination).
 __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
