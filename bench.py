@@ -35,9 +35,8 @@ CFG5 = dict(name="cfg5_full_decoder_step", B=32, schedule=(1, 2048, 2048, 2048),
 
 # The paper's own decoder shape (Section 3.2 / 6.1): 16 requests, 3 layers, 16 heads of 128, codebook 512,
 # 128 context tokens, dynamic beam schedule (1, 512, 1024, 1024).  The paper does not print d_model or
-# the FFN width; 2048 / 8192 reproduce its operation count (see decoder_macs).  Its fixed schedule
-# (1, 1024, 1024, 1024) asks step 0 for 1024 beams out of 512 candidates; the library rejects a beam
-# larger than the candidate count (M * V), so only the dynamic schedule runs at this codebook size.
+# the FFN width; 2048 / 8192 reproduce its operation count (see decoder_macs).  Its fixed schedule is
+# --schedule 1,1024,1024,1024 (step 0 then asks for 1024 beams out of 512 candidates: 512 dead beams).
 PAPER_SHAPE = dict(name="paper_decoder_shape", B=16, schedule=(1, 512, 1024, 1024), final_k=1024, n_layers=3,
                    d_model=2048, H=16, d_h=128, d_ffn=8192, d_enc=2048, T_ctx=128, V=512, L=4, n_sids=1_000_000,
                    elig_frac=0.2, bloom_log2=22, bloom_hashes=4)

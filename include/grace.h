@@ -269,7 +269,9 @@ grace_status_t grace_beam_update_csr(const int32_t* parent, const int32_t* token
  *   out_score fp32, out_flat int32, out_parent = flat / V, out_token = flat % V, each [B][K]
  *   (out_flat / out_parent / out_token may be NULL).
  * Needs a device workspace of grace_beam_topk_workspace_bytes(B, N, K) bytes, 256-byte aligned;
- * its contents on entry do not matter.  1 <= K <= min(N, 4096); N < 2^31.
+ * its contents on entry do not matter.  1 <= K <= 4096; N < 2^31.  K > N (a beam wider than the
+ * candidate set, as step 0 of the paper's fixed schedule (1, 1024, ...) with 512 tokens): all N
+ * candidates in order, then K - N dead entries (score -inf, flat = parent = token = 0).
  * ---------------------------------------------------------------------------------------- */
 size_t grace_beam_topk_workspace_bytes(int B, int64_t N, int K);
 grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, int K, int V,

@@ -20,15 +20,18 @@ def beam_topk(cand: np.ndarray, K: int, V: int):
     """cand fp32 [B, N] -> (score f32, flat i32, parent i32, token i32), each [B, K]."""
     cand = np.asarray(cand, dtype=np.float32)
     B, N = cand.shape
-    assert 0 < K <= N
+    assert K > 0
     assert not np.isnan(cand).any(), "NaN candidates violate the precondition"
-    score = np.empty((B, K), dtype=np.float32)
-    flat = np.empty((B, K), dtype=np.int32)
+    # A beam wider than the candidate set (Section 3.3: the fixed schedule asks for 1024 beams where at
+    # most |V| = 512 prefixes exist): every candidate in order, then dead entries (-inf on candidate 0).
+    score = np.full((B, K), -np.inf, dtype=np.float32)
+    flat = np.zeros((B, K), dtype=np.int32)
+    k = min(K, N)
     for b in range(B):
         row = cand[b] + np.float32(0.0)               # -0.0 -> +0.0
         order = np.argsort(-row, kind="stable")       # stable: ties keep index order
-        flat[b] = order[:K]
-        score[b] = cand[b, order[:K]]
+        flat[b, :k] = order[:k]
+        score[b, :k] = cand[b, order[:k]]
     return score, flat, (flat // V).astype(np.int32), (flat % V).astype(np.int32)
 
 

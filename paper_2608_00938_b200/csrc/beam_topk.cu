@@ -426,9 +426,10 @@ __device__ void block_bitonic_sort_desc(unsigned long long* keys) {
 }
 
 __global__ void __launch_bounds__(kTopkThreads)
-topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, TopkHeader* hdr,
+topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int K_out, int V, TopkHeader* hdr,
                      uint2* lists, int force_exact, float* out_score, int32_t* out_flat, int32_t* out_parent,
                      int32_t* out_token, int32_t* d_status) {
+  // K = min(requested, N) entries are selected; rows of the outputs are K_out = requested wide.
   pdl_wait();
   pdl_trigger();
   extern __shared__ unsigned long long sort_keys_raw[];     // kCap + kMaxK keys, then a 4096-bin histogram
@@ -511,7 +512,7 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, To
   for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
     uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
     if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
-    const int64_t o = (int64_t)b * K + i;
+    const int64_t o = (int64_t)b * K_out + i;
     out_score[o] = row[idx];
     if (out_flat) out_flat[o] = (int32_t)idx;
     if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
@@ -529,7 +530,7 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, To
       uint32_t total;
       const uint32_t rank = block_excl_scan(is_low ? 1u : 0u, scratch, &total) + done;
       if (is_low && rank < need) {
-        const int64_t o = (int64_t)b * K + c + rank;
+        const int64_t o = (int64_t)b * K_out + c + rank;
         out_score[o] = row[i];
         if (out_flat) out_flat[o] = (int32_t)i;
         if (out_parent) out_parent[o] = (int32_t)(i / (uint32_t)V);
@@ -537,6 +538,14 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int V, To
       }
       done += total;
     }
+  }
+  // A beam wider than the candidate set (K_out > N): the rest are dead beams, score -inf on candidate 0.
+  for (int i = K + (int)threadIdx.x; i < K_out; i += kTopkThreads) {
+    const int64_t o = (int64_t)b * K_out + i;
+    out_score[o] = __int_as_float(0xff800000);
+    if (out_flat) out_flat[o] = 0;
+    if (out_parent) out_parent[o] = 0;
+    if (out_token) out_token[o] = 0;
   }
 }
 
@@ -566,6 +575,8 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
                                 void* ws, int32_t* d_status, cudaStream_t s) {
   TopkHeader* hdr = reinterpret_cast<TopkHeader*>(ws);
   uint2* lists = reinterpret_cast<uint2*>(reinterpret_cast<char*>(ws) + topk_header_bytes(B));
+  const int K_out = K;
+  if ((int64_t)K > N) K = (int)N;                            // every candidate is selected, the rest is padding
   const uint32_t rank = sample_rank(N, K);
   static bool attrs_set = false;
   const size_t final_smem = (size_t)(kCap + kMaxK) * sizeof(unsigned long long) + 4096 * sizeof(uint32_t);
@@ -598,7 +609,7 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
     launch_pdl(topk_reset_kernel, dim3((B + 255) / 256), dim3(256), 0, s, hdr, B);
     GRACE_LAUNCH_CHECK();
   }
-  launch_pdl(topk_finalize_kernel, dim3(B), dim3(kTopkThreads), final_smem, s, cand, N, K, V, hdr, lists, force_exact, out_score, out_flat,
+  launch_pdl(topk_finalize_kernel, dim3(B), dim3(kTopkThreads), final_smem, s, cand, N, K, K_out, V, hdr, lists, force_exact, out_score, out_flat,
                                                           out_parent, out_token, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
@@ -610,7 +621,7 @@ extern "C" grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, i
                                           int32_t* out_token, void* ws, size_t ws_bytes,
                                           int32_t* d_status, void* stream) {
   if (!cand || !out_score || !ws) return GRACE_INVALID_ARG;
-  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || K > N || V <= 0) return GRACE_INVALID_ARG;
+  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || V <= 0) return GRACE_INVALID_ARG;
   if (K > 4096 || (N & 3)) return GRACE_UNSUPPORTED_SHAPE;
   if (!grace_aligned16(cand) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return GRACE_INVALID_ARG;
   if (ws_bytes < grace_beam_topk_workspace_bytes(B, N, K)) return GRACE_WORKSPACE_TOO_SMALL;
@@ -660,7 +671,7 @@ extern "C" grace_status_t grace_beam_topk_static(const float* cand, int B, int64
                                                  float* out_score, int32_t* out_flat, int32_t* out_parent,
                                                  int32_t* out_token, int32_t* d_status, void* stream) {
   if (!cand || !out_score) return GRACE_INVALID_ARG;
-  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || K > N || V <= 0) return GRACE_INVALID_ARG;
+  if (B <= 0 || N <= 0 || N >= (1ll << 31) || K < 1 || V <= 0) return GRACE_INVALID_ARG;
   if (K > grace::kMaxK || (N & 3)) return GRACE_UNSUPPORTED_SHAPE;
   if (B > grace::kStaticMaxRequests) return GRACE_WORKSPACE_TOO_SMALL;     // beyond the built-in scratch
   if (!grace_aligned16(cand)) return GRACE_INVALID_ARG;

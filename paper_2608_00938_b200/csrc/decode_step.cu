@@ -16,7 +16,6 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
   for (int t = 0; t <= d->L; ++t) {
     if (d->beam_sizes[t] <= 0) return GRACE_INVALID_ARG;
     if (t < d->L && d->beam_sizes[t] > mmax) mmax = d->beam_sizes[t];
-    if (t > 0 && (int64_t)d->beam_sizes[t] > (int64_t)d->beam_sizes[t - 1] * d->V) return GRACE_INVALID_ARG;
     if (d->beam_sizes[t] > 4096) return GRACE_UNSUPPORTED_SHAPE;
   }
   if (d->beam_sizes[d->L] > mmax) mmax = d->beam_sizes[d->L];

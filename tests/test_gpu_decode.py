@@ -68,6 +68,7 @@ _PAPER_LIKE = dict(shape=(2, 256, 16, 128, 512, 256), T_ctx=128, n_sids=4000)
     (3, "bloom", (1, 40, 24), 32, False, {}),    # several requests, dynamic per-step beam sizes, Bloom matcher
     (3, "bloom", (1, 40, 24), 32, True, {}),     # the same with the residual stream held in bf16
     (2, "bloom", (1, 24, 48, 48), 48, True, _PAPER_LIKE),   # dynamic schedule over 4 levels, head size 128
+    (2, "node", (1, 100, 80), 80, True, {}),      # step 0 asks for more beams than there are tokens (fixed-schedule shape)
 ])
 def test_decode_step_teacher_forced(B, kind, schedule, final_k, residual_bf16, extra):
     cfg = _config1(B=B, matcher_kind=kind, schedule=schedule, final_k=final_k, **extra)

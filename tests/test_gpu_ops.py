@@ -298,7 +298,8 @@ def _check_topk(api, cand, K, V, expect_exact_path=None):
     return status
 
 
-@pytest.mark.parametrize("B,M,V,K", [(1, 16, 64, 16), (3, 7, 192, 50), (2, 33, 1024, 2048), (1, 1, 64, 64)])
+@pytest.mark.parametrize("B,M,V,K", [(1, 16, 64, 16), (3, 7, 192, 50), (2, 33, 1024, 2048), (1, 1, 64, 64),
+                                     (2, 1, 64, 100), (3, 1, 512, 1024), (1, 3, 64, 1000)])   # beams wider than M * V
 def test_topk_small_shapes(api, B, M, V, K):
     rng = synth.rng_for(4, 100 + M)
     cand = synth.normal_f32(rng, (B, M * V), 3.0)

@@ -94,6 +94,12 @@ def test_topk_equals_python_sorted():
     assert same[1][0].tolist() == list(range(9))
     with pytest.raises(AssertionError):
         T.beam_topk(np.array([[np.nan, 1.0]], np.float32), 1, 2)
+    # a beam wider than the candidate set: every candidate in order, then dead entries on candidate 0
+    small = np.array([[0.5, -np.inf, 2.0, 0.5, -1.0, -np.inf]], np.float32)
+    sc, fl, pa, tk = T.beam_topk(small, 9, 3)
+    assert fl[0].tolist() == [2, 0, 3, 4, 1, 5, 0, 0, 0]
+    assert sc[0, :4].tolist() == [2.0, 0.5, 0.5, -1.0] and np.isneginf(sc[0, 4:]).all()
+    assert pa[0, 6:].tolist() == [0, 0, 0] and tk[0, 6:].tolist() == [0, 0, 0]
 
 
 def _exhaustive(weights, shp, enc, trie, sids, passes):
@@ -154,6 +160,11 @@ def test_beam_search_is_exhaustive_when_beams_are_wide_enough(kind):
         assert (sc[0][live] <= par_score[live]).all()                        # child = parent + logp <= parent
         np.testing.assert_allclose(np.exp(step["logp"].astype(np.float64)).sum(axis=1), 1.0, atol=1e-5)
     assert (~np.isneginf(record[0]["out_score"])).sum() <= V                 # at most |V| prefixes after step 0
+    # a schedule wider than the codebook at step 0 (the paper's fixed schedule has this shape) only adds dead beams
+    wide = D.beam_search(w, shp, enc, trie, matcher, (1, 100, 100), 100)
+    assert int(wide["valid"][0].sum()) == n_valid
+    assert [tuple(s_) for s_ in wide["sids"][0, :n_valid].tolist()] == got
+    assert np.array_equal(wide["score"][0, :n_valid], out["score"][0, :n_valid])
     dead = record[-1]["new_node"] < 0
     assert np.array_equal(dead, np.isneginf(record[-1]["out_score"].reshape(-1)))
 
