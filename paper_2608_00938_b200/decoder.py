@@ -134,6 +134,56 @@ class Decoder:
         for t in range(self.L):
             self.step(t)
 
+    def serve(self, enc_hosts, outputs) -> None:
+        """Decode a sequence of batches whose encoder outputs sit in PINNED host memory.
+
+        enc_hosts: sequence of pinned bf16 tensors [B, T_ctx, d_enc]; outputs: sequence (same length) of dicts
+        with pinned host tensors 'score' fp32 [B*K], 'key' int64 [B*K], 'node' int32 [B*K] that receive the final
+        beam of that batch.  Host copies run on a second stream: the input of batch i+1 travels while batch i
+        computes (two device buffers), results leave while the next cross-K/V projection runs.  Returns after a
+        device-wide synchronize, when every output is complete.
+        """
+        n = len(enc_hosts)
+        if n == 0:
+            return
+        K, fin = self.beam_sizes[-1], self.L & 1
+        rows = self.B * K
+        comp = torch.cuda.current_stream()
+        copy = torch.cuda.Stream()
+        enc_dev = [torch.empty_like(enc_hosts[0], device=self.device) for _ in range(2)]
+        ev_in = [torch.cuda.Event() for _ in range(2)]       # input buffer filled
+        ev_free = [torch.cuda.Event() for _ in range(2)]     # input buffer consumed by the projection
+        ev_done, ev_out = torch.cuda.Event(), torch.cuda.Event()
+        for ev in ev_free:
+            ev.record(comp)
+        ev_out.record(copy)
+
+        def send(i):
+            if i >= n:
+                return
+            with torch.cuda.stream(copy):
+                copy.wait_event(ev_free[i & 1])
+                enc_dev[i & 1].copy_(enc_hosts[i], non_blocking=True)
+                ev_in[i & 1].record(copy)
+
+        send(0)
+        for i in range(n):
+            comp.wait_event(ev_in[i & 1])
+            self.project_cross_kv(enc_dev[i & 1])
+            ev_free[i & 1].record(comp)
+            send(i + 1)                                       # the next input travels under this batch's compute
+            comp.wait_event(ev_out)                           # the previous results have left the state buffers
+            self.reset()
+            self.decode()
+            ev_done.record(comp)
+            with torch.cuda.stream(copy):
+                copy.wait_event(ev_done)
+                outputs[i]["score"].copy_(self.score[fin][:rows], non_blocking=True)
+                outputs[i]["key"].copy_(self.key[fin][:rows], non_blocking=True)
+                outputs[i]["node"].copy_(self.node[fin][:rows], non_blocking=True)
+                ev_out.record(copy)
+        torch.cuda.synchronize()
+
     def log_probs(self, rows: int) -> torch.Tensor:
         """Log-probabilities of the last step's first `rows` rows (reconstructed from logits and the row
         log-sum-exp when the log-softmax is fused into the mask kernel; needs separate_cand)."""

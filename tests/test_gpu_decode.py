@@ -168,3 +168,29 @@ def test_whole_decode_loop_replays_from_a_cuda_graph():
     assert torch.equal(dec.score[fin][:n].view(torch.int32), eager[0].view(torch.int32))
     assert torch.equal(dec.key[fin][:n], eager[1]) and torch.equal(dec.node[fin][:n], eager[2])
     assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+
+
+def test_serving_loop_with_overlapped_host_copies_matches_one_batch_at_a_time():
+    """Decoder.serve: inputs arrive from pinned host memory on a copy stream (batch i+1 under batch i's compute),
+    results leave on it.  Every batch must come out exactly as when it is decoded alone."""
+    cfg = _config1(B=3, matcher_kind="bloom", schedule=(1, 40, 24), final_k=32)
+    dec, api = _make_gpu_decoder(cfg, separate_cand=False, residual_bf16=True)
+    rng = synth.rng_for(1, 77)
+    n_batches, n = 5, cfg["B"] * cfg["final_k"]
+    fin = dec.L & 1
+    encs = [synth.normal_bf16(rng, cfg["enc"].shape) for _ in range(n_batches)]
+    alone = []
+    for e in encs:
+        dec.project_cross_kv(torch.from_numpy(e.view(np.int16)).to(DEV).view(torch.bfloat16))
+        dec.reset(); dec.decode()
+        torch.cuda.synchronize()
+        alone.append((dec.score[fin][:n].cpu(), dec.key[fin][:n].cpu(), dec.node[fin][:n].cpu()))
+    assert not torch.equal(alone[0][1], alone[1][1])                       # the batches really differ
+    hosts = [torch.from_numpy(e.view(np.int16).copy()).view(torch.bfloat16).pin_memory() for e in encs]
+    outs = [dict(score=torch.empty(n, dtype=torch.float32).pin_memory(), key=torch.empty(n, dtype=torch.int64).pin_memory(),
+                 node=torch.empty(n, dtype=torch.int32).pin_memory()) for _ in range(n_batches)]
+    dec.serve(hosts, outs)
+    for i in range(n_batches):
+        assert torch.equal(outs[i]["score"].view(torch.int32), alone[i][0].view(torch.int32)), i
+        assert torch.equal(outs[i]["key"], alone[i][1]) and torch.equal(outs[i]["node"], alone[i][2]), i
+    assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
