@@ -536,7 +536,7 @@ def main():
                             macs_per_request=decoder_macs(cfg)),
                 launch_modes=dict(eager_ms_per_step=eager_ms, cuda_graph_ms_per_step=graph_ms),
                 step_latency_us=per_step_us, clocks=clocks, gpu_launches=int(launches_per_loop * args.steps),
-                device_status=status,
+                device_status=status, wait_timeouts=api.grace_wait_timeouts(),
                 e2e=dict(value=units / (e2e_ms * 1e-3), unit="beam-steps/s", ms_per_step=e2e_ms,
                          h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                          includes="per step: pinned encoder output H2D, cross-K/V projection, 4 decode steps, results D2H; copies on a second stream (step i+1's input overlaps step i)"))

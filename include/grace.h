@@ -51,6 +51,17 @@ const char* grace_status_string(grace_status_t s);
 /* Library version, and the compute capability the kernels were built for (100 = sm_100a). */
 int grace_version(void);
 int grace_built_for_sm(void);
+/* Every device-side wait of the tensor-core kernels (on an mbarrier that TMA, the tensor cores or a peer
+ * CTA completes) is bounded: after about a second it gives up, the kernel's remaining waits return at
+ * once, the kernel frees its TMEM and exits, and the output of that launch is undefined.
+ * grace_wait_timeouts: number of waits that gave up on the current device since the previous call
+ * (0 in normal operation; -1 if the counter cannot be read).  Synchronize the streams first.
+ * grace_selftest_bounded_wait: runs a one-block kernel that waits (limit: about a millisecond) on a
+ * barrier nothing arrives on, synchronizes `stream`, and returns GRACE_TIMEOUT when the wait gave up as
+ * designed (grace_wait_timeouts then reports it); the context stays usable. */
+int grace_wait_timeouts(void);
+grace_status_t grace_selftest_bounded_wait(void* stream);
+
 /* Number of kernels this library has launched in this process so far (all entry points). */
 uint64_t grace_kernel_launch_count(void);
 

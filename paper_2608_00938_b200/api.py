@@ -101,6 +101,8 @@ _gtm_index_build = _sig("grace_gtm_index_build", _i32, [_vp, _i64, _i32, _i32, _
 _gtm_index_build_kway = _sig("grace_gtm_index_build_kway", _i32,
                              [_vp, _i64, _i32, _i32, _vp, _i64, _vp, _i32, _vp, _i32, _vp, C.c_double, _i32,
                               _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
+_wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
+_selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
 _beam_update_csr = _sig("grace_beam_update_csr", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp,
                                                        _i32, _i32, _i32, _i32, _vp, _vp])
@@ -288,6 +290,16 @@ def make_gtm_index(host_index: dict, user_bitmask: np.ndarray, user_blooms: np.n
                        keep["part_offsets"].data_ptr() if "part_offsets" in keep else None)
     s._keepalive = keep
     return s
+
+
+def grace_wait_timeouts() -> int:
+    """Bounded device waits that gave up since the previous call (0 in normal operation)."""
+    return int(_wait_timeouts())
+
+
+def grace_selftest_bounded_wait() -> int:
+    """Runs the bounded-wait self-test; returns the status code (TIMEOUT = the wait gave up as designed)."""
+    return int(_selftest_bounded_wait(_stream()))
 
 
 def grace_gtm_lookup(logp, beam_score, beam_node, index: GtmIndexStruct, cand, allow_bits, B: int, M: int,

@@ -104,6 +104,10 @@ cross_attn_small_kernel(const CrossSmallParams p) {
 
 }  // namespace grace
 
+namespace grace {
+int cross_attn_tc_timeouts() { return tc::tc_timeouts_read_and_clear(); }
+}  // namespace grace
+
 extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
                                            const uint16_t* k, const uint16_t* v,
                                            int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,

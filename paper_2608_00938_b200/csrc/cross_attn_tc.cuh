@@ -172,7 +172,10 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           idle = 0;
         } else {
           __nanosleep(512);                                 // polling costs issue slots the softmax warps of this scheduler need
-          if (++idle > (1 << 24)) *abort_flag = 1;           // bounded: about a second of nothing to do
+          if (++idle > (1 << 24)) {                          // bounded: about a second of nothing to do
+            if (*abort_flag == 0) atomicAdd(&tc::g_tc_timeouts, 1);
+            *abort_flag = 1;
+          }
         }
       }
     }

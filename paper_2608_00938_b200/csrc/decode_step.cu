@@ -120,3 +120,13 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
                               d->node[nxt], d->key[nxt], B, K, M, t, st, stream));
   return GRACE_OK;
 }
+
+namespace grace {
+int linear_tc_timeouts();
+int cross_attn_tc_timeouts();
+}  // namespace grace
+
+extern "C" int grace_wait_timeouts(void) {
+  const int a = grace::linear_tc_timeouts(), b = grace::cross_attn_tc_timeouts();
+  return (a < 0 || b < 0) ? -1 : a + b;
+}

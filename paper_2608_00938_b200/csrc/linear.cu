@@ -443,3 +443,34 @@ extern "C" grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, 
                                                 uint16_t* y_inout, int64_t ldy, int M, int N, int K, void* stream) {
   return linear_impl(x, ldx, w, ldw, y_inout, nullptr, ldy, nullptr, true, M, N, K, 0, stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Bounded waits, checked without hanging anything: a one-block kernel waits on a barrier that
+// nothing ever arrives on, with a limit of 64 parked polls (about a millisecond).
+// ---------------------------------------------------------------------------------------------
+namespace grace {
+__global__ void bounded_wait_selftest_kernel(int* result) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    abort_flag = 0;
+    tc::fence_mbar_init();
+    const bool arrived = tc::mbar_wait<64>(&bar, 0, &abort_flag);
+    *result = arrived ? 1 : (abort_flag ? 2 : 3);          // 2: gave up and raised the CTA's abort flag
+  }
+}
+int linear_tc_timeouts() { return tc::tc_timeouts_read_and_clear(); }
+static __device__ int g_selftest_result;
+}  // namespace grace
+
+extern "C" grace_status_t grace_selftest_bounded_wait(void* stream) {
+  int* d_result = nullptr;
+  GRACE_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&d_result), grace::g_selftest_result));
+  grace::bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_result);
+  GRACE_LAUNCH_CHECK();
+  GRACE_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+  int h = 0;
+  GRACE_CUDA_TRY(cudaMemcpy(&h, d_result, sizeof(int), cudaMemcpyDeviceToHost));
+  return h == 2 ? GRACE_TIMEOUT : GRACE_CUDA_ERROR;
+}

@@ -95,14 +95,21 @@ __device__ __forceinline__ bool mbar_try_wait_now(uint64_t* bar, uint32_t parity
       : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after 2^16 parked polls (about a second) and reports it through
-// `*abort_flag` (shared memory), which every later wait of the CTA checks first.
+// Waits that gave up, counted per translation unit (every .cu that includes this header has its own
+// counter; tc_timeouts_read_and_clear() below reads it from the host).
+static __device__ int g_tc_timeouts = 0;
+
+// Bounded wait: gives up after `kMaxPolls` parked polls (2^16: about a second) and reports it through
+// `*abort_flag` (shared memory), which every later wait of the CTA checks first, and through the
+// timeout counter, which the host can read.
+template <int kMaxPolls = (1 << 16)>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (int polls = 0; polls < (1 << 16); ++polls) {
+  for (int polls = 0; polls < kMaxPolls; ++polls) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
   }
+  if (*abort_flag == 0) atomicAdd(&g_tc_timeouts, 1);
   *abort_flag = 1;
   return false;
 }
@@ -188,6 +195,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if (*abort_flag) return false;
   }
+  if (*abort_flag == 0) atomicAdd(&g_tc_timeouts, 1);
   *abort_flag = 1;
   return false;
 }
@@ -304,6 +312,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
 }
 
 #endif  // __CUDACC__
+
+#ifdef __CUDACC__
+// Host: number of bounded waits that gave up in this translation unit's kernels since the last call.
+inline int tc_timeouts_read_and_clear() {
+  int n = 0;
+  const int zero = 0;
+  if (cudaMemcpyFromSymbol(&n, g_tc_timeouts, sizeof(int)) != cudaSuccess) return -1;
+  if (n != 0) cudaMemcpyToSymbol(g_tc_timeouts, &zero, sizeof(int));
+  return n;
+}
+#endif
 
 }  // namespace tc
 }  // namespace grace

@@ -581,3 +581,22 @@ def test_layer_norm_embed_log_softmax(api):
         ref = z64 - z64.max(1, keepdims=True)
         ref = ref - np.log(np.exp(ref).sum(1, keepdims=True))
         np.testing.assert_allclose(d_z.cpu().numpy(), ref, atol=2e-5, rtol=0)
+
+
+def test_bounded_device_wait_gives_up_and_is_reported(api):
+    """A wait on a barrier that nothing completes must end by itself (here after about a millisecond), be
+    counted, and leave the context usable: no kernel of this library can hang the GPU on a lost signal."""
+    torch.cuda.synchronize()
+    api.grace_wait_timeouts()                                   # clear
+    assert api.grace_selftest_bounded_wait() == 5               # GRACE_TIMEOUT: the wait gave up as designed
+    assert api.grace_wait_timeouts() == 1
+    assert api.grace_wait_timeouts() == 0                       # read-and-clear
+    # the context is intact: a tensor-core GEMM right after it is still exact to tolerance
+    rng = synth.rng_for(5, 4242)
+    x, w = synth.normal_bf16(rng, (1100, 256)), synth.normal_bf16(rng, (512, 256), 0.05)
+    y = torch.zeros((1100, 512), dtype=torch.bfloat16, device=DEV)
+    api.grace_linear(dev_bf16(x), dev_bf16(w), y, None, False)
+    torch.cuda.synchronize()
+    ref = f64(x) @ f64(w).T
+    assert np.abs(y.float().cpu().numpy() - ref).max() <= 2e-2 * max(1.0, np.abs(ref).max())
+    assert api.grace_wait_timeouts() == 0
