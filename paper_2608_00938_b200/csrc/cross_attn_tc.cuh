@@ -5,16 +5,17 @@
 // blocks of 128:
 //   S   = Q K_blk^T        tcgen05.mma, A = Q (shared, K-major), B = K_blk (shared, K-major),
 //                          fp32 S[128 x 128] in TMEM
-//   P   = exp2(S*c - max)  256 softmax threads: TMEM lane = query row, two threads per row each
-//                          taking half of the block's columns; P goes to its own TMEM columns
-//                          as packed bf16
+//   P   = exp2(S*c - max)  softmax threads: TMEM lane = query row; head size 64: one thread per row
+//                          (128 threads); head size 128: two threads per row, half of the block's
+//                          columns each (256 threads); P goes to its own TMEM columns as packed bf16
 //   O  += P V_blk          tcgen05.mma, A = P (TMEM), B = V_blk (shared, read MN-major, so V is
 //                          used as stored: no transpose anywhere); O stays in TMEM for the whole
 //                          row tile and is rescaled lazily, only when a row maximum grows by > 2^8
 // K and V blocks arrive by TMA through two separate two-slot rings; Q, K and V are addressed with 4-D tensor
 // maps over the caller's strides, so the beam-major Q / O layout is never permuted (the view /
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
-// and masked in the softmax.  Warp roles: 0-7 softmax + epilogue, 8 TMA producer, 9 MMA issuer.
+// and masked in the softmax.  Warp roles: softmax + epilogue warps first, then the TMA producer warp, then
+// the MMA issuer warp.
 // The kernel is persistent (each CTA loops over work items; Q is double-buffered), so the next item's
 // loads and first S overlap the current item's epilogue.  Head size 64 runs two CTAs per SM (256 TMEM
 // columns each), so one CTA's MMAs run under the other's exponentials; head size 128 needs 320
@@ -31,8 +32,10 @@ constexpr int kCaBM = 128;        // query rows per work item
 constexpr int kCaBN = 128;        // encoder positions per block
 constexpr int kCaStages = 2;
 constexpr int kCaHalfBytes = 128 * 64 * 2;                       // 16 KB: 128 rows x 64 bf16, one swizzle span wide
-constexpr int kCaSoftmaxWarps = 8;
-constexpr int kCaThreads = (kCaSoftmaxWarps + 2) * 32;
+// TPR = softmax threads per query row: 2 (eight softmax warps, each thread half of a block's columns) or
+// 1 (four softmax warps, a thread owns the whole row: no exchange between threads, half as many trips
+// through the TMEM load / barrier / TMEM store sequence per exponential; 168 registers).  Head size 64
+// runs TPR = 1 (4 % faster at 32 x 2048 x 1024); head size 128 keeps TPR = 2 for its wider output rows.
 constexpr int kCaBarBytes = 256;
 template <int DH> struct CaCfg {
   static constexpr int kHalves = DH / 64;
@@ -66,10 +69,12 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // Persistent kernel: a flat grid of two CTAs per SM; CTA g takes the work items g, g + gridDim.x,
 // ...  An item is one (request, head, 128-row tile); consecutive items are the tiles of the same
 // (request, head), so the CTAs running at the same time read the same K/V from L2.
-template <int DH>
-__global__ void __launch_bounds__(kCaThreads, CaCfg<DH>::kCtasPerSm)
+template <int DH, int TPR>
+__global__ void __launch_bounds__((4 * TPR + 2) * 32, CaCfg<DH>::kCtasPerSm)
 cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const CrossTcParams p) {
+  constexpr int kCaSoftmaxWarps = 4 * TPR;
+  constexpr int kCols = kCaBN / TPR;                       // score columns per softmax thread and block
   constexpr int kCaTileBytes = CaCfg<DH>::kTileBytes, kHalves = CaCfg<DH>::kHalves;
   constexpr uint32_t kCaTmemCols = CaCfg<DH>::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
@@ -279,8 +284,8 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int quarter = warp & 3, half = warp >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    const int col_base = 64 * half;
-    constexpr int kOutCols = DH / 2;                       // output columns per thread
+    const int col_base = kCols * half;
+    constexpr int kOutCols = DH / TPR;                     // output columns per thread
     bool ok = true;
     int g = 0, n_done = 0;
     for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
@@ -292,21 +297,20 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         ok = __all_sync(kFullMask, ok);
         if (!ok) break;
         tc::tc_fence_after();
-        uint32_t r[64];
+        uint32_t r[kCols];
         {
-          uint32_t (&r0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
-          uint32_t (&r1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
-          tc::tmem_ld32(tmem_s + lane_addr + col_base, r0);
-          tc::tmem_ld32(tmem_s + lane_addr + col_base + 32, r1);
+#pragma unroll
+          for (int c = 0; c < kCols; c += 32)
+            tc::tmem_ld32(tmem_s + lane_addr + col_base + c, *reinterpret_cast<uint32_t(*)[32]>(&r[c]));
           tc::tmem_ld_wait();
         }
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(s_free);              // the scores now live in registers
         const int valid = min(kCaBN, p.T - j * kCaBN) - col_base;   // this thread's columns that exist
-        if (valid < 64) {
+        if (valid < kCols) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i)
+          for (int i = 0; i < kCols; ++i)
             if (i >= valid) r[i] = 0xff800000u;                     // -inf: no weight, no influence on the max
         }
         // four independent chains instead of one 32-deep one
@@ -315,19 +319,22 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         float mx2 = max3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
         float mx3 = max3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
 #pragma unroll
-        for (int i = 12; i + 7 < 64; i += 8) {
+        for (int i = 12; i + 7 < kCols; i += 8) {
           mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
           mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
           mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
           mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
         }
-        mx0 = max3(mx0, __uint_as_float(r[60]), __uint_as_float(r[61]));
-        mx1 = max3(mx1, __uint_as_float(r[62]), __uint_as_float(r[63]));
+        mx0 = max3(mx0, __uint_as_float(r[kCols - 4]), __uint_as_float(r[kCols - 3]));
+        mx1 = max3(mx1, __uint_as_float(r[kCols - 2]), __uint_as_float(r[kCols - 1]));
         float mx = fmaxf(max3(mx0, mx1, mx2), mx3);
-        float* hm = half_max + (g & 1) * 256;
-        hm[half * 128 + row] = mx;
-        tc::named_bar_sync(2 + quarter, 64);                  // the two warps of this row quarter
-        const float m_blk = fmaxf(mx, hm[(half ^ 1) * 128 + row]) * p.scale_log2;
+        if (TPR == 2) {
+          float* hm = half_max + (g & 1) * 256;
+          hm[half * 128 + row] = mx;
+          tc::named_bar_sync(2 + quarter, 64);                // the two warps of this row quarter
+          mx = fmaxf(mx, hm[(half ^ 1) * 128 + row]);
+        }
+        const float m_blk = mx * p.scale_log2;
         const bool grow = m_blk > m_run + 8.0f;               // always true on an item's first block
         const float m_new = grow ? m_blk : m_run;
         const float alpha = grow ? ex2(m_run - m_new) : 1.0f; // 0 on the first block
@@ -336,7 +343,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const float neg_m = -m_new;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < kCols / 4; ++i) {
           const float e0 = ex2(fmaf(__uint_as_float(r[4 * i]), p.scale_log2, neg_m));
           const float e1 = ex2(fmaf(__uint_as_float(r[4 * i + 1]), p.scale_log2, neg_m));
           const float e2 = ex2(fmaf(__uint_as_float(r[4 * i + 2]), p.scale_log2, neg_m));
@@ -356,10 +363,9 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tc::tc_fence_after();
         }
         {
-          uint32_t (&p0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[0]);
-          uint32_t (&p1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&r[16]);
-          tc::tmem_st16(tmem_p + lane_addr + 32 * half, p0);
-          tc::tmem_st16(tmem_p + lane_addr + 32 * half + 16, p1);
+#pragma unroll
+          for (int c = 0; c < kCols / 2; c += 16)
+            tc::tmem_st16(tmem_p + lane_addr + (kCols / 2) * half + c, *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
         }
         if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
 #pragma unroll
@@ -391,10 +397,13 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       for (int c = 0; c < kOutCols; c += 32)
         tc::tmem_ld32(tmem_o + lane_addr + kOutCols * half + c, *reinterpret_cast<uint32_t(*)[32]>(&o[c]));
       tc::tmem_ld_wait();
-      float* hs = half_sum + (n_done & 1) * 256;              // double-buffered by item parity
-      hs[half * 128 + row] = l_run;
-      tc::named_bar_sync(2 + quarter, 64);
-      const float l_tot = l_run + hs[(half ^ 1) * 128 + row];
+      float l_tot = l_run;
+      if (TPR == 2) {
+        float* hs = half_sum + (n_done & 1) * 256;            // double-buffered by item parity
+        hs[half * 128 + row] = l_run;
+        tc::named_bar_sync(2 + quarter, 64);
+        l_tot += hs[(half ^ 1) * 128 + row];
+      }
       ++n_done;
       const int m = tile * kCaBM + row;
       if (m < p.M) {
@@ -421,7 +430,7 @@ inline bool cross_attn_tc_supported(int B, int M, int H, int d_h, int T_ctx) {
   return (d_h == 64 || d_h == 128) && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;
 }
 
-template <int DH>
+template <int DH, int TPR>
 inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_stride, const uint16_t* k,
                                               const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
                                               int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
@@ -443,7 +452,7 @@ inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_s
   }
   static bool attr_set = false;
   if (!attr_set) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel<DH, TPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
     attr_set = true;
   }
   static int n_sm = 0;
@@ -461,7 +470,7 @@ inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_s
   p.scale_log2 = scale * 1.4426950408889634f;
   const int ctas = CaCfg<DH>::kCtasPerSm * n_sm;
   const int grid = (int)(items < ctas ? items : ctas);
-  launch_pdl(cross_attn_tc_kernel<DH>, dim3(grid), dim3(kCaThreads), kCaSmemBytes, s, mq, mk, mv, p);
+  launch_pdl(cross_attn_tc_kernel<DH, TPR>, dim3(grid), dim3((4 * TPR + 2) * 32), kCaSmemBytes, s, mq, mk, mv, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -471,9 +480,9 @@ inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stri
                                            int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
                                            int B, int M, int H, int d_h, int T_ctx, float scale, cudaStream_t s) {
   if (d_h == 128)
-    return launch_cross_attn_tc_dh<128>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
+    return launch_cross_attn_tc_dh<128, 2>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
                                         lse, B, M, H, T_ctx, scale, s);
-  return launch_cross_attn_tc_dh<64>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
+  return launch_cross_attn_tc_dh<64, 1>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
                                      lse, B, M, H, T_ctx, scale, s);
 }
 
