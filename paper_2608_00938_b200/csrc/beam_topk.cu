@@ -578,11 +578,10 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
   const int K_out = K;
   if ((int64_t)K > N) K = (int)N;                            // every candidate is selected, the rest is padding
   const uint32_t rank = sample_rank(N, K);
-  static bool attrs_set = false;
+  static unsigned long long attrs_set_devices = 0;
   const size_t final_smem = (size_t)(kCap + kMaxK) * sizeof(unsigned long long) + 4096 * sizeof(uint32_t);
-  if (!attrs_set) {
+  if (first_use_on_device(&attrs_set_devices)) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)final_smem));
-    attrs_set = true;
   }
   int force_exact = 1;
   if (rank != 0) {

@@ -108,4 +108,16 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// One-time per-device set-up (kernel attributes are per device): true the first time the calling
+// thread's current device is seen for this `mask` (one static mask per set-up site).  Two host threads
+// racing here both do the set-up, which is idempotent.
+inline bool first_use_on_device(unsigned long long* mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return true;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (__atomic_load_n(mask, __ATOMIC_ACQUIRE) & bit) return false;
+  __atomic_fetch_or(mask, bit, __ATOMIC_RELEASE);
+  return true;
+}
+
 }  // namespace grace

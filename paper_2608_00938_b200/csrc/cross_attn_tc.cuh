@@ -450,10 +450,9 @@ inline grace_status_t launch_cross_attn_tc_dh(const uint16_t* q, int64_t q_row_s
     if (!tc::make_tmap_bf16(&mk, k, 4, dims, str, box)) return GRACE_CUDA_ERROR;
     if (!tc::make_tmap_bf16(&mv, v, 4, dims, str, box)) return GRACE_CUDA_ERROR;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_set_devices = 0;
+  if (first_use_on_device(&attr_set_devices)) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_tc_kernel<DH, TPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCaSmemBytes));
-    attr_set = true;
   }
   static int n_sm = 0;
   if (n_sm == 0) {

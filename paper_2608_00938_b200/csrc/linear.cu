@@ -343,7 +343,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 template <int OUT>
 static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
                                   int K, int relu, cudaStream_t s) {
-  static bool attr_set = false;
+  static unsigned long long attr_set_devices = 0;
   static int max_clusters = 0;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
@@ -352,7 +352,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
-  if (!attr_set) {
+  if (first_use_on_device(&attr_set_devices)) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
     int dev = 0, n_sm = 0;
     GRACE_CUDA_TRY(cudaGetDevice(&dev));
@@ -361,7 +361,6 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
     GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&max_clusters, linear_pair_kernel<OUT>, &cfg));
     if (max_clusters <= 0) return GRACE_CUDA_ERROR;
     if (max_clusters > n_sm / 2) max_clusters = n_sm / 2;
-    attr_set = true;
   }
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
@@ -372,10 +371,9 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
 
 template <int BN>
 static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw, const GemmParams& p, cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_set_devices = 0;
+  if (first_use_on_device(&attr_set_devices)) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmSmem<BN>::kTotal));
-    attr_set = true;
   }
   dim3 grid((p.N + BN - 1) / BN, (p.M + kGemmBM - 1) / kGemmBM);
   launch_pdl(linear_kernel<BN>, grid, dim3(128), GemmSmem<BN>::kTotal, s, mx, mw, p);
