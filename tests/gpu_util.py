@@ -38,3 +38,20 @@ def assert_attention_close(got: np.ndarray, ref: np.ndarray, what: str = ""):
     rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
     assert err.max() <= 2e-2, f"{what}: max abs err {err.max():.4g} at {np.unravel_index(err.argmax(), err.shape)}"
     assert rel <= 1e-2, f"{what}: relative Frobenius err {rel:.4g}"
+
+
+def assert_log_probs_close(got: np.ndarray, ref: np.ndarray, what: str = ""):
+    """Log-probabilities of the bf16 decoder vs the fp64 oracle (rows of live beams only).
+
+    A bf16 rounding of an activation is a relative error of at most u = 2^-9; after the roundings along the
+    path the final hidden vector carries a relative rms error of a few u, and a logit z = h . w inherits it as
+    (a few u) * std(z) rms.  The bound therefore scales with the spread of the row's logits:
+        rms error <= 1.2e-2 * std   (about 6 u),      max error <= 8e-2 * std
+    (the maximum of 1e7..1e8 near-normal errors sits about six rms above zero).  At the logit spread of the
+    smallest configuration (std 0.25) this is the 2e-2 / 3e-3 the tolerance was first stated for."""
+    got, ref = got.astype(np.float64), ref.astype(np.float64)
+    std = float(ref.std())
+    err = np.abs(got - ref)
+    rms = float(np.sqrt((err ** 2).mean()))
+    assert err.max() <= 8e-2 * std, f"{what}: max log-prob error {err.max():.4g} at logit spread {std:.3g}"
+    assert rms <= 1.2e-2 * std, f"{what}: rms log-prob error {rms:.4g} at logit spread {std:.3g}"
