@@ -97,7 +97,7 @@ def build_decoder(cfg, inp, device, residual_bf16=False):
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=inp["weights"], trie_bits=bits,
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
-                  residual_bf16=residual_bf16)
+                  residual_bf16=residual_bf16, level_start=level_start)
     return dec
 
 
@@ -292,7 +292,18 @@ def op_breakdown(dec, cfg, reps=3):
             timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
             logp = dec.logp[:R]
             timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
-            if dec.row_lse is not None:                 # the decode path fuses log-softmax into the mask kernel
+            par = dec.parents[t + 1]
+            masked = dec.allow_bits is not None and t >= dec.masked_from_step
+            if masked:                                  # candidates never materialised: allow bits + masked top-k
+                bits = dec.allow_bits[:R]
+                timed("gtm_mask", lambda: api.grace_gtm_mask_logits(logp, dec.row_lse[:R], dec.score[cur][:R],
+                                                                    dec.node[cur][:R], dec.key[cur][:R], dec.trie,
+                                                                    dec.matcher, None, bits, B, M, t, dec.d_status))
+                timed("beam_topk", lambda: api.grace_beam_topk_masked(
+                    logp, bits, dec.score[cur][:R], dec.row_lse[:R], B, M, K, dec.score[nxt][:B * K].view(B, K),
+                    dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K), dec.token[nxt][:B * K].view(B, K),
+                    dec.topk_ws, dec.d_status))
+            elif dec.row_lse is not None:               # log-softmax fused into the mask kernel
                 timed("gtm_mask", lambda: api.grace_gtm_mask_logits(logp, dec.row_lse[:R], dec.score[cur][:R],
                                                                     dec.node[cur][:R], dec.key[cur][:R], dec.trie,
                                                                     dec.matcher, logp, None, B, M, t, dec.d_status))
@@ -301,10 +312,10 @@ def op_breakdown(dec, cfg, reps=3):
                 timed("gtm_mask", lambda: api.grace_gtm_mask(logp, dec.score[cur][:R], dec.node[cur][:R],
                                                              dec.key[cur][:R], dec.trie, dec.matcher, logp, None, B, M,
                                                              t, dec.d_status))
-            par = dec.parents[t + 1]
-            timed("beam_topk", lambda: api.grace_beam_topk(logp.view(B, M * V), K, V, dec.score[nxt][:B * K].view(B, K),
-                                                           dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K),
-                                                           dec.token[nxt][:B * K].view(B, K), dec.topk_ws, dec.d_status))
+            if not masked:
+                timed("beam_topk", lambda: api.grace_beam_topk(
+                    logp.view(B, M * V), K, V, dec.score[nxt][:B * K].view(B, K), dec.out_flat[:B * K].view(B, K),
+                    par[:B * K].view(B, K), dec.token[nxt][:B * K].view(B, K), dec.topk_ws, dec.d_status))
             timed("beam_update", lambda: api.grace_beam_update(par[:B * K], dec.token[nxt][:B * K], dec.score[nxt][:B * K],
                                                                dec.node[cur][:R], dec.key[cur][:R], dec.trie,
                                                                dec.node[nxt][:B * K], dec.key[nxt][:B * K], B, K, M, t,

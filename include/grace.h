@@ -290,6 +290,20 @@ grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, int K, int V
                                int32_t* out_token, void* ws, size_t ws_bytes,
                                int32_t* d_status, void* stream);
 
+/* The same selection with the candidates never materialised: candidate m * V + v of request b is
+ *   row_score[r] + (logits[r][v] - row_lse[r])   if bit v of allow_bits[r][] is set,  -inf otherwise,
+ * with r = b * M + m: exactly what grace_gtm_mask_logits would have written (same fp32 operations in the
+ * same order), so both forms return identical results.  logits fp32 [B*M][V] (V % 64 == 0), allow_bits
+ * uint64 [B*M][V/64] and row_lse fp32 [B*M] as produced by grace_gtm_mask_logits with cand = NULL,
+ * row_score fp32 [B*M] the beams' prefix scores.  Logits are read only in 16-byte pieces that hold an
+ * allowed token, so sparse trie levels cost a pass over the allow bits.  Workspace as grace_beam_topk
+ * with N = M * V. */
+grace_status_t grace_beam_topk_masked(const float* logits, const uint64_t* allow_bits, const float* row_score,
+                                      const float* row_lse, int B, int M, int V, int K,
+                                      float* out_score, int32_t* out_flat, int32_t* out_parent,
+                                      int32_t* out_token, void* ws, size_t ws_bytes,
+                                      int32_t* d_status, void* stream);
+
 /* grace_beam_topk with the scratch memory built into the library (the paper has no counterpart:
  * this exists for callers of this library, not for the method).
  *
@@ -412,6 +426,12 @@ typedef struct {
   float *row_lse;             /* NULL, or [R_max]: fuse log-softmax into the mask kernel; the
                                  per-row log-sum-exp lands here (0 for dead rows)            */
   float *cand;                /* [R_max][V] masked scores; may be the same buffer as logp  */
+  uint64_t *allow_bits;       /* NULL, or [R_max][V/64] (needs row_lse): from step masked_from_step on the
+                                 mask kernel writes only these bits and the top-k reads the logits through
+                                 them (cheaper where few tokens per row survive; where a fifth of the row
+                                 survives, materialised candidates are faster); earlier steps use cand   */
+  int32_t masked_from_step;   /* first step (0-based) that takes the allow-bits path                   */
+  int32_t reserved2;
   void *topk_ws; size_t topk_ws_bytes;
   int32_t *d_status;
 } grace_decoder_t;

@@ -67,7 +67,8 @@ class DecoderStruct(C.Structure):
         ("trie", TrieStruct), ("matcher", MatcherStruct),
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
-        ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp),
+        ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp), ("allow_bits", _vp), ("masked_from_step", C.c_int32),
+        ("reserved2", C.c_int32),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -101,6 +102,8 @@ _gtm_index_build = _sig("grace_gtm_index_build", _i32, [_vp, _i64, _i32, _i32, _
 _gtm_index_build_kway = _sig("grace_gtm_index_build_kway", _i32,
                              [_vp, _i64, _i32, _i32, _vp, _i64, _vp, _i32, _vp, _i32, _vp, C.c_double, _i32,
                               _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
+_beam_topk_masked = _sig("grace_beam_topk_masked", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
+                                                         _vp, C.c_size_t, _vp, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
@@ -290,6 +293,15 @@ def make_gtm_index(host_index: dict, user_bitmask: np.ndarray, user_blooms: np.n
                        keep["part_offsets"].data_ptr() if "part_offsets" in keep else None)
     s._keepalive = keep
     return s
+
+
+def grace_beam_topk_masked(logits, allow_bits, row_score, row_lse, B: int, M: int, K: int, out_score, out_flat, out_parent,
+                           out_token, ws, d_status=None):
+    """Top-k over candidates that are never materialised (see grace_beam_topk_masked in grace.h)."""
+    V = logits.shape[-1]
+    _check(_beam_topk_masked(_dp(logits), _dp(allow_bits), _dp(row_score), _dp(row_lse), B, M, V, K, _dp(out_score),
+                             _dp(out_flat), _dp(out_parent), _dp(out_token), _dp(ws), ws.numel() * ws.element_size(),
+                             _dp(d_status), _stream()), "grace_beam_topk_masked")
 
 
 def grace_wait_timeouts() -> int:

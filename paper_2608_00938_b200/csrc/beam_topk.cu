@@ -34,6 +34,44 @@ struct TopkHeader {                      // lives in the workspace, one per requ
 
 __host__ __device__ inline size_t topk_header_bytes(int B) { return (size_t)B * sizeof(TopkHeader); }
 
+// Where the candidates come from.  Dense: an array [B][N].  Masked: they are never materialised; candidate i
+// of request b is token v = i % V of row r = (b * N + i) / V, worth row_score[r] + (logits[r][v] - row_lse[r])
+// if bit v of the row's allow words is set and -inf otherwise: the very arithmetic of the fused mask kernel, so
+// both forms select identically.  Logits are read only where a token of the four is allowed.
+struct CandSrc {
+  const float* data;            // dense: candidates; masked: logits [B * M][V]
+  const uint64_t* allow;        // masked: [B * M][V / 64]; nullptr = dense
+  const float* row_score;       // masked: [B * M]
+  const float* row_lse;         // masked: [B * M]
+  int64_t N;
+  int V, log2_V;                // log2_V >= 0 when V is a power of two
+
+  __device__ __forceinline__ float4 load4(int b, int64_t i4, bool streaming) const {
+    if (allow == nullptr) {
+      const float4* p = reinterpret_cast<const float4*>(data + (int64_t)b * N) + i4;
+      return streaming ? __ldcs(p) : __ldg(p);
+    }
+    const int64_t g = (int64_t)b * N + i4 * 4;               // global element index; V % 64 == 0: 4 tokens of one word
+    const int64_t r = (log2_V >= 0) ? (g >> log2_V) : (g / V);
+    const int v = (int)(g - r * V);
+    const uint32_t nib = (uint32_t)(__ldg(allow + r * (V >> 6) + (v >> 6)) >> (v & 63)) & 0xfu;
+    const float ninf = __int_as_float(0xff800000);
+    if (nib == 0u) return make_float4(ninf, ninf, ninf, ninf);
+    const float4 x = __ldg(reinterpret_cast<const float4*>(data + g));
+    const float lse = __ldg(row_lse + r), sc = __ldg(row_score + r);
+    return make_float4((nib & 1u) ? sc + (x.x - lse) : ninf, (nib & 2u) ? sc + (x.y - lse) : ninf,
+                       (nib & 4u) ? sc + (x.z - lse) : ninf, (nib & 8u) ? sc + (x.w - lse) : ninf);
+  }
+  __device__ __forceinline__ float load1(int b, int64_t i) const {
+    if (allow == nullptr) return __ldg(data + (int64_t)b * N + i);
+    const int64_t g = (int64_t)b * N + i;
+    const int64_t r = (log2_V >= 0) ? (g >> log2_V) : (g / V);
+    const int v = (int)(g - r * V);
+    if (!((__ldg(allow + r * (V >> 6) + (v >> 6)) >> (v & 63)) & 1ull)) return __int_as_float(0xff800000);
+    return __ldg(row_score + r) + (__ldg(data + g) - __ldg(row_lse + r));
+  }
+};
+
 // ---- block primitives (kTopkThreads threads) -------------------------------------------
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
   const int lane = threadIdx.x & 31;
@@ -101,7 +139,7 @@ __device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, int nbins, 
 // threshold (more candidates collected), never raise it, so the guarantee "at least K above the
 // threshold with high probability" is kept while the selection works on 2048 keys instead of 32768.
 __global__ void __launch_bounds__(kTopkThreads)
-topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, TopkHeader* hdr) {
+topk_sample_kernel(const CandSrc src, uint32_t rank, TopkHeader* hdr) {
   pdl_wait();
   pdl_trigger();
   __shared__ uint32_t keys[2 * kTopkThreads];
@@ -109,7 +147,7 @@ topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, Top
   __shared__ uint32_t scratch[40];
   __shared__ uint32_t result[2];
   const int b = blockIdx.x;
-  const float* row = cand + (int64_t)b * N;
+  const int64_t N = src.N;
   const int64_t stratum = (N / kSamplePoints) & ~(int64_t)7;       // multiple of 8 elements
   const uint32_t slots = (uint32_t)(stratum >> 3);
   float4 v[2 * (kSamplePoints / kTopkThreads)];
@@ -118,8 +156,8 @@ topk_sample_kernel(const float* __restrict__ cand, int64_t N, uint32_t rank, Top
     const int p = q * kTopkThreads + threadIdx.x;
     const uint32_t h = (uint32_t)(mix64((uint64_t)p * 0x10001ull + (uint64_t)b) >> 33);
     const int64_t at = (int64_t)p * stratum + (int64_t)(h % slots) * 8;
-    v[2 * q] = __ldg(reinterpret_cast<const float4*>(row + at));
-    v[2 * q + 1] = __ldg(reinterpret_cast<const float4*>(row + at + 4));
+    v[2 * q] = src.load4(b, at >> 2, false);
+    v[2 * q + 1] = src.load4(b, (at >> 2) + 1, false);
   }
   uint32_t top1 = 0, top2 = 0;
 #pragma unroll
@@ -173,8 +211,7 @@ constexpr int kCollectUnroll = 8;                         // float4 loads in fli
 constexpr int kStage = 1024;                              // hits staged per CTA before a flush
 
 __global__ void __launch_bounds__(kCollectThreads, 5)
-topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, uint2* lists,
-                    int32_t* d_status) {
+topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d_status) {
   pdl_wait();
   pdl_trigger();
   // grid (x, B): the CTAs of column b share request b's tiles round-robin.  Hits are rare (a
@@ -184,8 +221,7 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
   __shared__ uint2 stage[kStage];
   __shared__ uint32_t stage_count, flush_base;
   const int b = blockIdx.y;
-  const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
-  const int64_t n4 = N >> 2;
+  const int64_t n4 = src.N >> 2;
   uint2* list = lists + (int64_t)b * kCap;
   const int lane = threadIdx.x & 31;
   const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
@@ -200,7 +236,7 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
 #pragma unroll
     for (int u = 0; u < kCollectUnroll; ++u) {
       const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
-      v[u] = (i < n4) ? __ldcs(row + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      v[u] = (i < n4) ? src.load4(b, i, true) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
     if (!have_threshold) {                     // after the first loads are in flight
       t_excl = __ldcg(&hdr[b].t_excl);
@@ -279,14 +315,98 @@ topk_collect_kernel(const float* __restrict__ cand, int64_t N, TopkHeader* hdr, 
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
 }
 
+// Collecting pass over candidates that are not materialised: the unit of work is one 64-bit allow word (64
+// tokens of one row).  A zero word costs one 8-byte load; otherwise the thread visits the word's non-empty
+// groups of four tokens, reads those 16 bytes of logits and tests the (up to four) allowed ones.  Hits are
+// appended one by one (they are rare) with the same staging and overflow rules as the dense pass.
+constexpr int kCollectWords = 8;                          // allow words in flight per thread
+
+__global__ void __launch_bounds__(kCollectThreads, 5)
+topk_collect_masked_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d_status) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ uint2 stage[kStage];
+  __shared__ uint32_t stage_count, flush_base;
+  const int b = blockIdx.y;
+  const int64_t n_words = src.N >> 6;
+  const uint64_t* words = src.allow + (((int64_t)b * src.N) >> 6);
+  uint2* list = lists + (int64_t)b * kCap;
+  const int64_t tile = (int64_t)kCollectThreads * kCollectWords;
+  bool saw_nan = false;
+  if (threadIdx.x == 0) stage_count = 0;
+  __syncthreads();
+  const uint32_t t_excl = __ldcg(&hdr[b].t_excl);
+  for (int64_t base = (int64_t)blockIdx.x * tile; base < n_words; base += (int64_t)gridDim.x * tile) {
+    uint64_t w[kCollectWords];
+#pragma unroll
+    for (int u = 0; u < kCollectWords; ++u) {
+      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
+      w[u] = (i < n_words) ? __ldcs(words + i) : 0ull;
+    }
+#pragma unroll 1
+    for (int u = 0; u < kCollectWords; ++u) {
+      uint64_t bits = w[u];
+      if (bits == 0ull) continue;
+      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
+      const int64_t g0 = (int64_t)b * src.N + (i << 6);    // first token of the word, global element index
+      const int64_t r = (src.log2_V >= 0) ? (g0 >> src.log2_V) : (g0 / src.V);
+      const float lse = __ldg(src.row_lse + r), sc = __ldg(src.row_score + r);
+      while (bits != 0ull) {
+        const int q = (__ffsll((long long)bits) - 1) >> 2;  // group of four tokens holding the lowest set bit
+        const uint32_t nib = (uint32_t)(bits >> (4 * q)) & 0xfu;
+        bits &= ~(0xfull << (4 * q));
+        const float4 x = __ldg(reinterpret_cast<const float4*>(src.data + g0 + 4 * q));
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (!((nib >> j) & 1u)) continue;
+          const float val = sc + (xs[j] - lse);
+          if (val != val) { saw_nan = true; continue; }
+          const uint32_t key = ordered_key(val);
+          if (key <= t_excl) continue;
+          const uint2 entry = make_uint2(key, (uint32_t)((i << 6) + 4 * q + j));
+          const uint32_t pos = atomicAdd(&stage_count, 1u);
+          if (pos < (uint32_t)kStage) {
+            stage[pos] = entry;
+          } else {                                          // stage full: straight to the request's list
+            const uint32_t gpos = atomicAdd(&hdr[b].count, 1u);
+            if (gpos < (uint32_t)kCap) list[gpos] = entry;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t staged = min(stage_count, (uint32_t)kStage);
+    if (staged >= (uint32_t)kStage / 2) {
+      if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
+      __syncthreads();
+      const uint32_t dst = flush_base;
+      for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
+        if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
+      __syncthreads();
+      if (threadIdx.x == 0) stage_count = 0;
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+  const uint32_t staged = min(stage_count, (uint32_t)kStage);
+  if (staged != 0) {
+    if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
+    __syncthreads();
+    const uint32_t dst = flush_base;
+    for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
+      if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
+  }
+  if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
+}
+
 // ---- 3. exact --------------------------------------------------------------------------------
 // One CTA per request.  Three histogram passes over the row fix the K-th key exactly; a fourth
 // pass in index order writes the keys above it and the first ties.
-__device__ void topk_exact_select(const float* __restrict__ cand, int64_t N, int K, uint2* lists, int b,
+__device__ void topk_exact_select(const CandSrc& src, int K, uint2* lists, int b,
                                   uint32_t* hist /*4096*/, uint32_t* scratch /*40*/, uint32_t* result /*2*/,
                                   int32_t* d_status) {
-  const float4* row = reinterpret_cast<const float4*>(cand + (int64_t)b * N);
-  const int64_t n4 = N >> 2;
+  const int64_t n4 = src.N >> 2;
   uint32_t k = (uint32_t)K, prefix = 0;
   const int shifts[3] = {20, 8, 0};
   const int bits[3] = {12, 12, 8};
@@ -299,7 +419,7 @@ __device__ void topk_exact_select(const float* __restrict__ cand, int64_t N, int
     const int hi_shift = shifts[level] + bits[level];
     uint32_t n_ninf = 0;            // -inf dominates masked rows: count it in a register
     for (int64_t i = threadIdx.x; i < n4; i += kTopkThreads) {
-      const float4 v = __ldg(row + i);
+      const float4 v = src.load4(b, i, false);
       const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -327,7 +447,7 @@ __device__ void topk_exact_select(const float* __restrict__ cand, int64_t N, int
     uint32_t key[4] = {0, 0, 0, 0};
     uint32_t above = 0, ties = 0;
     if (i < n4) {
-      v = __ldg(row + i);
+      v = src.load4(b, i, false);
       key[0] = ordered_key(v.x); key[1] = ordered_key(v.y); key[2] = ordered_key(v.z); key[3] = ordered_key(v.w);
 #pragma unroll
       for (int j = 0; j < 4; ++j) { above += key[j] > kth; ties += key[j] == kth; }
@@ -426,7 +546,7 @@ __device__ void block_bitonic_sort_desc(unsigned long long* keys) {
 }
 
 __global__ void __launch_bounds__(kTopkThreads)
-topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int K_out, int V, TopkHeader* hdr,
+topk_finalize_kernel(const CandSrc src, int K, int K_out, int V, TopkHeader* hdr,
                      uint2* lists, int force_exact, float* out_score, int32_t* out_flat, int32_t* out_parent,
                      int32_t* out_token, int32_t* d_status) {
   // K = min(requested, N) entries are selected; rows of the outputs are K_out = requested wide.
@@ -443,7 +563,7 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int K_out
   const bool need_exact = force_exact || c > (uint32_t)kCap || (c < (uint32_t)K && hdr[b].t_excl != kKeyNegInf);
   if (need_exact) {
     if (!force_exact && threadIdx.x == 0) flag_status(d_status, GRACE_DEV_TOPK_EXACT_PATH);
-    topk_exact_select(cand, N, K, lists, b, reinterpret_cast<uint32_t*>(sort_keys), scratch, result, d_status);
+    topk_exact_select(src, K, lists, b, reinterpret_cast<uint32_t*>(sort_keys), scratch, result, d_status);
     __syncthreads();
     c = (uint32_t)K;
   }
@@ -507,13 +627,13 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int K_out
     default: block_bitonic_sort_desc<8>(to_sort); break;
   }
   sort_keys = to_sort;
-  const float* row = cand + (int64_t)b * N;
+  const int64_t N = src.N;
   const uint32_t n_out = min(c, (uint32_t)K);
   for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
     uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
     if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
     const int64_t o = (int64_t)b * K_out + i;
-    out_score[o] = row[idx];
+    out_score[o] = src.load1(b, idx);
     if (out_flat) out_flat[o] = (int32_t)idx;
     if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
     if (out_token) out_token[o] = (int32_t)(idx % (uint32_t)V);
@@ -526,12 +646,13 @@ topk_finalize_kernel(const float* __restrict__ cand, int64_t N, int K, int K_out
     uint32_t done = 0;
     for (uint32_t base = 0; base < (uint32_t)K && done < need; base += kTopkThreads) {
       const uint32_t i = base + threadIdx.x;
-      const bool is_low = (i < (uint32_t)K) && (ordered_key(row[i]) <= kKeyNegInf);
+      const float xi = (i < (uint32_t)K) ? src.load1(b, i) : 0.f;
+      const bool is_low = (i < (uint32_t)K) && (ordered_key(xi) <= kKeyNegInf);
       uint32_t total;
       const uint32_t rank = block_excl_scan(is_low ? 1u : 0u, scratch, &total) + done;
       if (is_low && rank < need) {
         const int64_t o = (int64_t)b * K_out + c + rank;
-        out_score[o] = row[i];
+        out_score[o] = xi;
         if (out_flat) out_flat[o] = (int32_t)i;
         if (out_parent) out_parent[o] = (int32_t)(i / (uint32_t)V);
         if (out_token) out_token[o] = (int32_t)(i % (uint32_t)V);
@@ -570,9 +691,11 @@ extern "C" size_t grace_beam_topk_workspace_bytes(int B, int64_t N, int K) {
 
 namespace grace {
 // Shared by the public entry point and the variant that owns its scratch.
-grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int V, float* out_score,
+grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, float* out_score,
                                 int32_t* out_flat, int32_t* out_parent, int32_t* out_token,
                                 void* ws, int32_t* d_status, cudaStream_t s) {
+  CandSrc src = src_in;
+  const int64_t N = src.N;
   TopkHeader* hdr = reinterpret_cast<TopkHeader*>(ws);
   uint2* lists = reinterpret_cast<uint2*>(reinterpret_cast<char*>(ws) + topk_header_bytes(B));
   const int K_out = K;
@@ -585,7 +708,7 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
   }
   int force_exact = 1;
   if (rank != 0) {
-    launch_pdl(topk_sample_kernel, dim3(B), dim3(kTopkThreads), 0, s, cand, N, rank, hdr);
+    launch_pdl(topk_sample_kernel, dim3(B), dim3(kTopkThreads), 0, s, src, rank, hdr);
     GRACE_LAUNCH_CHECK();
     static int collect_grid = 0;
     if (collect_grid == 0) {
@@ -600,15 +723,26 @@ grace_status_t launch_beam_topk(const float* cand, int B, int64_t N, int K, int 
     int64_t per_request = collect_grid / B;                 // one resident wave over all requests
     if (per_request < 1) per_request = 1;
     if (per_request > tiles_per_request) per_request = tiles_per_request;
-    dim3 grid((unsigned)per_request, (unsigned)B);
-    launch_pdl(topk_collect_kernel, dim3(grid), dim3(kCollectThreads), 0, s, cand, N, hdr, lists, d_status);
-    GRACE_LAUNCH_CHECK();
+    if (src.allow != nullptr) {                              // masked: the tile is 256 x 8 allow words
+      const int64_t wtile = (int64_t)kCollectThreads * kCollectWords;
+      const int64_t wtiles = ((N >> 6) + wtile - 1) / wtile;
+      per_request = collect_grid / B;
+      if (per_request < 1) per_request = 1;
+      if (per_request > wtiles) per_request = wtiles;
+      launch_pdl(topk_collect_masked_kernel, dim3((unsigned)per_request, (unsigned)B), dim3(kCollectThreads), 0, s, src, hdr,
+                 lists, d_status);
+      GRACE_LAUNCH_CHECK();
+    } else {
+      dim3 grid((unsigned)per_request, (unsigned)B);
+      launch_pdl(topk_collect_kernel, dim3(grid), dim3(kCollectThreads), 0, s, src, hdr, lists, d_status);
+      GRACE_LAUNCH_CHECK();
+    }
     force_exact = 0;
   } else {
     launch_pdl(topk_reset_kernel, dim3((B + 255) / 256), dim3(256), 0, s, hdr, B);
     GRACE_LAUNCH_CHECK();
   }
-  launch_pdl(topk_finalize_kernel, dim3(B), dim3(kTopkThreads), final_smem, s, cand, N, K, K_out, V, hdr, lists, force_exact, out_score, out_flat,
+  launch_pdl(topk_finalize_kernel, dim3(B), dim3(kTopkThreads), final_smem, s, src, K, K_out, V, hdr, lists, force_exact, out_score, out_flat,
                                                           out_parent, out_token, d_status);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
@@ -624,8 +758,29 @@ extern "C" grace_status_t grace_beam_topk(const float* cand, int B, int64_t N, i
   if (K > 4096 || (N & 3)) return GRACE_UNSUPPORTED_SHAPE;
   if (!grace_aligned16(cand) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return GRACE_INVALID_ARG;
   if (ws_bytes < grace_beam_topk_workspace_bytes(B, N, K)) return GRACE_WORKSPACE_TOO_SMALL;
-  return grace::launch_beam_topk(cand, B, N, K, V, out_score, out_flat, out_parent, out_token, ws,
+  grace::CandSrc src = {cand, nullptr, nullptr, nullptr, N, V, -1};
+  return grace::launch_beam_topk(src, B, K, V, out_score, out_flat, out_parent, out_token, ws,
                                  d_status, (cudaStream_t)stream);
+}
+
+extern "C" grace_status_t grace_beam_topk_masked(const float* logits, const uint64_t* allow_bits,
+                                                 const float* row_score, const float* row_lse, int B, int M, int V,
+                                                 int K, float* out_score, int32_t* out_flat, int32_t* out_parent,
+                                                 int32_t* out_token, void* ws, size_t ws_bytes, int32_t* d_status,
+                                                 void* stream) {
+  if (!logits || !allow_bits || !row_score || !row_lse || !out_score || !ws) return GRACE_INVALID_ARG;
+  if (B <= 0 || M <= 0 || V <= 0 || (V & 63) || K < 1) return GRACE_INVALID_ARG;
+  const int64_t N = (int64_t)M * V;
+  if (N >= (1ll << 31) || (int64_t)B * N >= (1ll << 40)) return GRACE_INVALID_ARG;
+  if (K > 4096) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(logits) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return GRACE_INVALID_ARG;
+  if (ws_bytes < grace_beam_topk_workspace_bytes(B, N, K)) return GRACE_WORKSPACE_TOO_SMALL;
+  int log2_V = -1;
+  if ((V & (V - 1)) == 0)
+    for (log2_V = 0; (1 << log2_V) < V; ++log2_V) {}
+  grace::CandSrc src = {logits, allow_bits, row_score, row_lse, N, V, log2_V};
+  return grace::launch_beam_topk(src, B, K, V, out_score, out_flat, out_parent, out_token, ws, d_status,
+                                 (cudaStream_t)stream);
 }
 
 
@@ -679,6 +834,7 @@ extern "C" grace_status_t grace_beam_topk_static(const float* cand, int B, int64
   if (st != GRACE_OK) return st;
   // The kernels (re)initialise every header word they read, so the previous call's contents do not
   // matter; nothing here has to start at zero.
-  return grace::launch_beam_topk(cand, B, N, K, V, out_score, out_flat, out_parent, out_token, scratch, d_status,
+  grace::CandSrc src = {cand, nullptr, nullptr, nullptr, N, V, -1};
+  return grace::launch_beam_topk(src, B, K, V, out_score, out_flat, out_parent, out_token, scratch, d_status,
                                  (cudaStream_t)stream);
 }

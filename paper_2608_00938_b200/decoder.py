@@ -26,12 +26,14 @@ class Decoder:
     weights: dict as produced by `synth.decoder_weights` (fp32 arrays; matrices are rounded to
     bf16 on upload).  beam_sizes: (M_0 .. M_{L-1}, K_final).  trie_bits / trie_base: host arrays
     from `api.grace_trie_build_dense`.  matcher: (kind, host uint64 [B, words] or None,
-    log2_bits, n_hashes).
+    log2_bits, n_hashes).  level_start (optional, from the same trie build): first node id of every level;
+    used to decide per step whether masked candidates are written out or read through allow bits.
     """
 
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
-                 separate_cand=False, fuse_log_softmax=True, residual_bf16=False):
+                 separate_cand=False, fuse_log_softmax=True, residual_bf16=False, materialize_cand=None,
+                 level_start=None):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -108,6 +110,23 @@ class Decoder:
         s.h, s.qkv, s.attn, s.logp, s.cand = (self.h.data_ptr(), self.qkv.data_ptr(),
                                                    self.attn.data_ptr(), self.logp.data_ptr(), self.cand.data_ptr())
         s.row_lse = None if self.row_lse is None else self.row_lse.data_ptr()
+        # Candidates are not materialised unless asked for (or needed: no fused log-softmax, or a separate
+        # candidate buffer for inspection): the mask kernel then leaves allow bits, the top-k reads the logits
+        # through them.
+        if materialize_cand is None:
+            materialize_cand = separate_cand or not fuse_log_softmax
+        self.allow_bits = None if materialize_cand else torch.zeros((R_max, V // 64), dtype=torch.int64, device=dev)
+        s.allow_bits = None if self.allow_bits is None else self.allow_bits.data_ptr()
+        # The allow-bits path pays off where few tokens of a row survive the catalog mask.  Children per node are
+        # known from the trie: a beam of step t sits on a node of level t and has (nodes of level t+1) / (nodes of
+        # level t) children on average; steps whose rows keep more than 2 % of the codebook materialise candidates.
+        self.masked_from_step = 0
+        if self.allow_bits is not None and level_start is not None:
+            sizes = np.diff(np.asarray(level_start, dtype=np.int64))          # nodes per level 0..L
+            for t in range(L):
+                if sizes[t + 1] / max(1, sizes[t]) / V > 0.02:
+                    self.masked_from_step = t + 1
+        s.masked_from_step = self.masked_from_step
         s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()
         self.struct = s
         code = api.grace_decoder_validate(s)

@@ -194,3 +194,24 @@ def test_serving_loop_with_overlapped_host_copies_matches_one_batch_at_a_time():
         assert torch.equal(outs[i]["score"].view(torch.int32), alone[i][0].view(torch.int32)), i
         assert torch.equal(outs[i]["key"], alone[i][1]) and torch.equal(outs[i]["node"], alone[i][2]), i
     assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+
+
+@pytest.mark.parametrize("kind,schedule,final_k", [("bloom", (1, 40, 24), 32), ("node", (1, 100, 80), 80)])
+def test_decode_without_materialised_candidates_equals_the_materialised_path(kind, schedule, final_k):
+    """The fast path (mask kernel leaves allow bits, top-k reads the logits through them) must give the same
+    beams, bit for bit, as the path that writes the masked candidates and selects from them."""
+    cfg = _config1(B=3, matcher_kind=kind, schedule=schedule, final_k=final_k)
+    n = cfg["B"] * final_k
+    outs = []
+    for separate in (True, False):
+        dec, api = _make_gpu_decoder(cfg, separate_cand=separate, residual_bf16=True)
+        assert (dec.allow_bits is None) == separate
+        dec.reset(); dec.decode()
+        torch.cuda.synchronize()
+        fin = dec.L & 1
+        assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+        outs.append((dec.score[fin][:n].clone(), dec.key[fin][:n].clone(), dec.node[fin][:n].clone(),
+                     dec.parents[:, :n].clone()))
+    assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+    assert torch.equal(outs[0][3], outs[1][3])

@@ -308,6 +308,44 @@ def test_topk_small_shapes(api, B, M, V, K):
     _check_topk(api, cand, K, V)
 
 
+@pytest.mark.parametrize("B,M,V,K,density", [
+    (2, 16, 64, 16, 0.3), (3, 7, 192, 50, 0.05), (2, 300, 1024, 2048, 0.05), (2, 300, 1024, 2048, 0.0005),
+    (1, 1, 512, 1024, 0.5),                       # wider than the candidate set
+    (2, 2100, 2048, 2048, 0.05), (2, 2100, 2048, 2048, 0.0005), (1, 2048, 2048, 4096, 1.0),   # sampled path, three densities
+])
+def test_topk_on_candidates_that_are_never_materialised(api, B, M, V, K, density):
+    """grace_beam_topk_masked: logits + allow bits + row scores + row log-sum-exp in, the selection of
+    grace_beam_topk over score + (logit - lse) / -inf out, bit for bit (including a dead row and an empty request)."""
+    rng = synth.rng_for(4, 300 + M + V)
+    R = B * M
+    logits = synth.normal_f32(rng, (R, V), 1.5)
+    lse = (np.log(np.exp(logits.astype(np.float64)).sum(1))).astype(np.float32)
+    score = (-np.abs(synth.normal_f32(rng, R, 2.0))).astype(np.float32)
+    allow = rng.random((R, V)) < density
+    allow[R // 2] = False                                       # a dead beam: nothing allowed, lse irrelevant
+    lse[R // 2] = 0.0
+    if B > 1 and density < 0.01:
+        allow[M:2 * M] = False                                  # a request without a single candidate
+    cand = np.where(allow, score[:, None] + (logits - lse[:, None]), np.float32(-np.inf)).astype(np.float32)
+    bits = OG.pack_allow_bits(allow)
+    s_ref, f_ref, p_ref, t_ref = OT.beam_topk(cand.reshape(B, M * V), K, V)
+    ws = torch.empty(api.grace_beam_topk_workspace_bytes(B, M * V, K), dtype=torch.uint8, device=DEV)
+    ws.fill_(0xAB)
+    sc = torch.empty((B, K), device=DEV)
+    fl = torch.empty((B, K), dtype=torch.int32, device=DEV)
+    pa, tk = torch.empty_like(fl), torch.empty_like(fl)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_beam_topk_masked(dev(logits), dev(bits.view(np.int64)), dev(score), dev(lse), B, M, K, sc, fl, pa, tk, ws, status)
+    torch.cuda.synchronize()
+    assert not (status.item() & (api.DEV_NAN | api.DEV_BAD_INDEX))
+    assert np.array_equal(fl.cpu().numpy(), f_ref)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+    assert np.array_equal(pa.cpu().numpy(), p_ref) and np.array_equal(tk.cpu().numpy(), t_ref)
+    # and identical to the dense entry point on the materialised candidates
+    s2, f2, p2, t2, _ = _run_topk(api, cand.reshape(B, M * V), K, V)
+    assert np.array_equal(f2, f_ref) and np.array_equal(s2.view(np.uint32), s_ref.view(np.uint32))
+
+
 def test_topk_sampled_path_dense_and_masked(api):
     """N large enough for the sampled-threshold path: dense scores, then masks of several densities."""
     B, M, V, K = 3, 300, 1024, 2048
