@@ -85,7 +85,7 @@ def make_inputs(cfg, variant=0):
     return dict(sids=sids, elig=elig, shp=shp, weights=weights, enc_bits=enc_bits)
 
 
-def build_decoder(cfg, inp, device, residual_bf16=False):
+def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -97,7 +97,7 @@ def build_decoder(cfg, inp, device, residual_bf16=False):
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=inp["weights"], trie_bits=bits,
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
-                  residual_bf16=residual_bf16, level_start=level_start)
+                  residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand)
     return dec
 
 

@@ -293,3 +293,30 @@ def test_decode_step_full_size_teacher_forced_on_one_request(workload, schedule,
                 assert bl.contains(OM.prefix_keys(g_sids[b][valid][:, :l])).all()
         del dec
         torch.cuda.empty_cache()
+
+
+def test_bench_decode_path_equals_the_materialised_path_at_config5():
+    """The decoder exactly as bench.py builds it (bf16 residual stream; candidates written out on the dense trie
+    level, read through allow bits on the sparse ones) against the same decoder with every step materialised:
+    free-running over all 32 requests, the final beams must agree bit for bit."""
+    import bench
+    cfg = dict(bench.CFG5)
+    inp = bench.make_inputs(cfg, 0)
+    enc = dev_bf16(inp["enc_bits"])
+    B, K = cfg["B"], cfg["final_k"]
+    outs = []
+    for materialize in (False, True):
+        dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True, materialize_cand=materialize)
+        if not materialize:
+            assert dec.allow_bits is not None and 0 < dec.masked_from_step < cfg["L"]      # a mixed schedule
+        dec.project_cross_kv(enc)
+        dec.reset(); dec.decode()
+        torch.cuda.synchronize()
+        fin = dec.L & 1
+        assert dec.d_status.item() & ~8 == 0                                              # 8: informational
+        outs.append((dec.score[fin][:B * K].clone(), dec.key[fin][:B * K].clone(), dec.node[fin][:B * K].clone()))
+        del dec
+        torch.cuda.empty_cache()
+    assert torch.isfinite(outs[0][0]).sum() > B * K // 2
+    assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
