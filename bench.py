@@ -291,22 +291,37 @@ def op_breakdown(dec, cfg, reps=3):
                 timed("linear", lambda: add_into_x(ff, lay["w_2"], x), 2.0 * R * F * D)
             timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
             logp = dec.logp[:R]
-            timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
+            parts = dec.lse_part is not None and R >= 1024
+            if parts:                                   # the logits GEMM also leaves the rows' log-sum-exp partials
+                lsep = dec.lse_part[:R]
+                timed("linear", lambda: api.grace_linear_f32_lse(hD, dec.w_out, logp, lsep), 2.0 * R * D * V)
+            else:
+                timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
             par = dec.parents[t + 1]
             masked = dec.allow_bits is not None and t >= dec.masked_from_step
             if masked:                                  # candidates never materialised: allow bits + masked top-k
                 bits = dec.allow_bits[:R]
-                timed("gtm_mask", lambda: api.grace_gtm_mask_logits(logp, dec.row_lse[:R], dec.score[cur][:R],
-                                                                    dec.node[cur][:R], dec.key[cur][:R], dec.trie,
-                                                                    dec.matcher, None, bits, B, M, t, dec.d_status))
+                if parts:
+                    timed("gtm_mask", lambda: api.grace_gtm_mask_logits_parts(
+                        logp, dec.row_lse[:R], dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
+                        None, bits, B, M, t, lsep, dec.d_status))
+                else:
+                    timed("gtm_mask", lambda: api.grace_gtm_mask_logits(
+                        logp, dec.row_lse[:R], dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
+                        None, bits, B, M, t, dec.d_status))
                 timed("beam_topk", lambda: api.grace_beam_topk_masked(
                     logp, bits, dec.score[cur][:R], dec.row_lse[:R], B, M, K, dec.score[nxt][:B * K].view(B, K),
                     dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K), dec.token[nxt][:B * K].view(B, K),
                     dec.topk_ws, dec.d_status))
             elif dec.row_lse is not None:               # log-softmax fused into the mask kernel
-                timed("gtm_mask", lambda: api.grace_gtm_mask_logits(logp, dec.row_lse[:R], dec.score[cur][:R],
-                                                                    dec.node[cur][:R], dec.key[cur][:R], dec.trie,
-                                                                    dec.matcher, logp, None, B, M, t, dec.d_status))
+                if parts:
+                    timed("gtm_mask", lambda: api.grace_gtm_mask_logits_parts(
+                        logp, dec.row_lse[:R], dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
+                        logp, None, B, M, t, lsep, dec.d_status))
+                else:
+                    timed("gtm_mask", lambda: api.grace_gtm_mask_logits(
+                        logp, dec.row_lse[:R], dec.score[cur][:R], dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
+                        logp, None, B, M, t, dec.d_status))
             else:
                 timed("log_softmax", lambda: api.grace_log_softmax(logp))
                 timed("gtm_mask", lambda: api.grace_gtm_mask(logp, dec.score[cur][:R], dec.node[cur][:R],

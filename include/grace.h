@@ -195,6 +195,17 @@ grace_status_t grace_gtm_mask_logits(const float* logits, float* row_lse, const 
                                      float* cand, uint64_t* allow_bits, int B, int M, int V,
                                      int prefix_len, int32_t* d_status, void* stream);
 
+/* grace_gtm_mask_logits with the rows' sums already started by the producer of the logits: lse_part fp32
+ * [B*M][n_parts][2] holds, per row and column tile, (maximum, sum of e^(x - maximum)) as written by
+ * grace_linear_f32_lse (n_parts = V / 256 <= 32).  The kernel merges them instead of reading the row, so with
+ * cand = NULL it does not touch the logits at all. */
+grace_status_t grace_gtm_mask_logits_parts(const float* logits, float* row_lse, const float* beam_score,
+                                           const int32_t* beam_node, const uint64_t* beam_key,
+                                           const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                           float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                           int prefix_len, const float* lse_part, int n_parts,
+                                           int32_t* d_status, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * The paper's own index form (Sections 4.2-4.4, 5.4, Appendix A): CSR child entries that carry
  * ids of deduplicated per-node matcher rows, tested against per-request attribute rows.
@@ -360,6 +371,12 @@ grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, i
 grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
                                      uint16_t* y_inout, int64_t ldy, int M, int N, int K, void* stream);
 
+/* y_f32 = x @ w^T (fp32 output) and, from the same accumulators, the start of every row's log-sum-exp:
+ * lse_part fp32 [M][N / 256][2] receives (maximum, sum of e^(y - maximum)) over each 256-column tile of the
+ * row.  Large problems only (M >= 1024, N % 256 == 0); otherwise GRACE_UNSUPPORTED_SHAPE. */
+grace_status_t grace_linear_f32_lse(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                    float* y_f32, int64_t ldy, float* lse_part, int M, int N, int K, void* stream);
+
 /* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
 grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
                                 uint16_t* out, int R, int D, float eps, void* stream);
@@ -432,6 +449,8 @@ typedef struct {
                                  survives, materialised candidates are faster); earlier steps use cand   */
   int32_t masked_from_step;   /* first step (0-based) that takes the allow-bits path                   */
   int32_t reserved2;
+  float *lse_part;            /* NULL, or [R_max][V/256][2] (needs row_lse, V % 256 == 0): the logits GEMM
+                                 leaves per-tile log-sum-exp partials and the mask kernel merges them     */
   void *topk_ws; size_t topk_ws_bytes;
   int32_t *d_status;
 } grace_decoder_t;

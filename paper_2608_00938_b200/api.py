@@ -68,7 +68,7 @@ class DecoderStruct(C.Structure):
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
         ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp), ("allow_bits", _vp), ("masked_from_step", C.c_int32),
-        ("reserved2", C.c_int32),
+        ("reserved2", C.c_int32), ("lse_part", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -104,6 +104,10 @@ _gtm_index_build_kway = _sig("grace_gtm_index_build_kway", _i32,
                               _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp])
 _beam_topk_masked = _sig("grace_beam_topk_masked", _i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
                                                          _vp, C.c_size_t, _vp, _vp])
+_linear_f32_lse = _sig("grace_linear_f32_lse", _i32, [_vp, _i64, _vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _vp])
+_gtm_mask_logits_parts = _sig("grace_gtm_mask_logits_parts", _i32,
+                              [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct), _vp, _vp,
+                               _i32, _i32, _i32, _i32, _vp, _i32, _vp, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
@@ -302,6 +306,24 @@ def grace_beam_topk_masked(logits, allow_bits, row_score, row_lse, B: int, M: in
     _check(_beam_topk_masked(_dp(logits), _dp(allow_bits), _dp(row_score), _dp(row_lse), B, M, V, K, _dp(out_score),
                              _dp(out_flat), _dp(out_parent), _dp(out_token), _dp(ws), ws.numel() * ws.element_size(),
                              _dp(d_status), _stream()), "grace_beam_topk_masked")
+
+
+def grace_linear_f32_lse(x, w, y, lse_part):
+    """y fp32 [M, N] = x @ w.T and lse_part fp32 [M, N // 256, 2] = per-tile (maximum, sum of e^(y - maximum))."""
+    M, K = x.shape
+    N = w.shape[0]
+    _check(_linear_f32_lse(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), _dp(y), y.stride(0), _dp(lse_part), M, N, K,
+                           _stream()), "grace_linear_f32_lse")
+    return y, lse_part
+
+
+def grace_gtm_mask_logits_parts(logits, row_lse, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B: int,
+                                M: int, prefix_len: int, lse_part, d_status=None):
+    """grace_gtm_mask_logits with the per-tile log-sum-exp partials of grace_linear_f32_lse."""
+    V = logits.shape[-1]
+    _check(_gtm_mask_logits_parts(_dp(logits), _dp(row_lse), _dp(beam_score), _dp(beam_node), _dp(beam_key), C.byref(trie),
+                                  C.byref(matcher), _dp(cand), _dp(allow_bits), B, M, V, prefix_len, _dp(lse_part),
+                                  lse_part.shape[1], _dp(d_status), _stream()), "grace_gtm_mask_logits_parts")
 
 
 def grace_wait_timeouts() -> int:

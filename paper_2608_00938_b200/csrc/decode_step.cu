@@ -102,14 +102,19 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
     GRACE_TRY(add_into_x(d->qkv, d->d_ffn, w.w_2, d->d_ffn));
   }
   GRACE_TRY(layer_norm(d->lnf_g, d->lnf_b));
-  GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
+  // the logits GEMM can leave the rows' log-sum-exp partials (large steps), the mask kernel then merges them
+  const int n_parts = d->V / 256;
+  const bool parts = d->lse_part != nullptr && d->row_lse != nullptr && R >= 1024 && (d->V % 256) == 0 && n_parts <= 32;
+  if (parts) GRACE_TRY(grace_linear_f32_lse(d->h, D, d->w_out, D, d->logp, d->V, d->lse_part, R, d->V, D, stream));
+  else GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
   // log-softmax, CD + GTM mask and score add: one fused kernel when row_lse is provided
   int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
   if (d->row_lse != nullptr && d->allow_bits != nullptr && t >= d->masked_from_step) {
     // candidates never materialised: the mask kernel leaves the allow bits and the rows' log-sum-exp, the
     // selection reads the logits through them (and only where a token is allowed)
-    GRACE_TRY(grace_gtm_mask_logits(d->logp, d->row_lse, d->score[cur], d->node[cur], d->key[cur], &d->trie,
-                                    &d->matcher, nullptr, d->allow_bits, B, M, d->V, t, st, stream));
+    GRACE_TRY(grace_gtm_mask_logits_parts(d->logp, d->row_lse, d->score[cur], d->node[cur], d->key[cur], &d->trie,
+                                          &d->matcher, nullptr, d->allow_bits, B, M, d->V, t,
+                                          parts ? d->lse_part : nullptr, n_parts, st, stream));
     GRACE_TRY(grace_beam_topk_masked(d->logp, d->allow_bits, d->score[cur], d->row_lse, B, M, d->V, K, d->score[nxt],
                                      d->out_flat, parent_out, d->token[nxt], d->topk_ws, d->topk_ws_bytes, st, stream));
     GRACE_TRY(grace_beam_update(parent_out, d->token[nxt], d->score[nxt], d->node[cur], d->key[cur], &d->trie,
@@ -117,8 +122,9 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
     return GRACE_OK;
   }
   if (d->row_lse != nullptr) {
-    GRACE_TRY(grace_gtm_mask_logits(d->logp, d->row_lse, d->score[cur], d->node[cur], d->key[cur], &d->trie,
-                                    &d->matcher, d->cand, nullptr, B, M, d->V, t, st, stream));
+    GRACE_TRY(grace_gtm_mask_logits_parts(d->logp, d->row_lse, d->score[cur], d->node[cur], d->key[cur], &d->trie,
+                                          &d->matcher, d->cand, nullptr, B, M, d->V, t,
+                                          parts ? d->lse_part : nullptr, n_parts, st, stream));
   } else {
     GRACE_TRY(grace_log_softmax(d->logp, R, d->V, stream));
     GRACE_TRY(grace_gtm_mask(d->logp, d->score[cur], d->node[cur], d->key[cur], &d->trie, &d->matcher, d->cand,

@@ -22,6 +22,8 @@ struct MaskParams {
   const uint64_t* matcher_bits;
   float* cand;
   float* row_lse;            // LOGITS mode: receives log-sum-exp of each live row
+  const float2* lse_part;    // LOGITS mode, optional: [R][n_parts] (maximum, sum of e^(x - maximum)) per column tile,
+  int n_parts;               //   left by the GEMM that produced the logits; the row is then not read for its sum
   uint64_t* allow_bits;
   int32_t* d_status;
   int64_t num_internal, num_nodes, words_per_request;
@@ -96,6 +98,13 @@ gtm_mask_kernel(const MaskParams p) {
     // warp at the end (the row is not kept: phase 2 re-reads only the allowed sectors, from L2)
     float m_l = -INFINITY, s_l = 0.f;
     const int n4 = V >> 2;
+    if (p.lse_part != nullptr) {                           // the producer of the logits already summed each column tile
+      if (part == 0 && lane < p.n_parts) {
+        const float2 pr = __ldg(p.lse_part + (int64_t)r * p.n_parts + lane);
+        m_l = pr.x;
+        s_l = pr.y;
+      }
+    } else
     for (int c0 = part * 128; c0 < n4; c0 += kParts * 128) {
       float4 x[4];
 #pragma unroll
@@ -470,7 +479,8 @@ static bool trie_ok(const grace_trie_t* t, int V) {
 static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse, const float* beam_score,
                                   const int32_t* beam_node, const uint64_t* beam_key, const grace_trie_t* trie,
                                   const grace_matcher_t* matcher, float* cand, uint64_t* allow_bits, int B, int M,
-                                  int V, int prefix_len, int32_t* d_status, void* stream) {
+                                  int V, int prefix_len, int32_t* d_status, void* stream,
+                                  const float* lse_part = nullptr, int n_parts = 0) {
   using namespace grace;
   if (!logp || !beam_score || !beam_node || !matcher || (!cand && !allow_bits)) return GRACE_INVALID_ARG;
   if (B <= 0 || M <= 0 || (int64_t)B * M > 0x7fffffff) return GRACE_INVALID_ARG;
@@ -481,6 +491,9 @@ static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse
   p.logp = logp; p.beam_score = beam_score; p.beam_node = beam_node; p.beam_key = beam_key;
   p.child_bits = trie->child_bits; p.child_base = trie->child_base;
   p.matcher_bits = matcher->bits; p.cand = cand; p.row_lse = row_lse; p.allow_bits = allow_bits; p.d_status = d_status;
+  if (lse_part != nullptr && (!logits || n_parts < 1 || n_parts > 32 || (reinterpret_cast<uintptr_t>(lse_part) & 7)))
+    return GRACE_INVALID_ARG;
+  p.lse_part = reinterpret_cast<const float2*>(lse_part); p.n_parts = n_parts;
   p.num_internal = trie->num_internal; p.num_nodes = trie->num_nodes;
   p.words_per_request = matcher->words_per_request;
   p.R = B * M; p.M = M; p.V = V; p.prefix_len = prefix_len;
@@ -540,6 +553,16 @@ extern "C" grace_status_t grace_gtm_mask_logits(const float* logits, float* row_
                                                 int prefix_len, int32_t* d_status, void* stream) {
   return launch_mask(logits, true, row_lse, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B, M, V,
                      prefix_len, d_status, stream);
+}
+
+extern "C" grace_status_t grace_gtm_mask_logits_parts(const float* logits, float* row_lse, const float* beam_score,
+                                                const int32_t* beam_node, const uint64_t* beam_key,
+                                                const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                                float* cand, uint64_t* allow_bits, int B, int M, int V,
+                                                int prefix_len, const float* lse_part, int n_parts, int32_t* d_status,
+                                                      void* stream) {
+  return launch_mask(logits, true, row_lse, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B, M, V,
+                     prefix_len, d_status, stream, lse_part, n_parts);
 }
 
 extern "C" grace_status_t grace_beam_update(const int32_t* parent, const int32_t* token, const float* score,

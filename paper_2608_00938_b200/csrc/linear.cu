@@ -13,6 +13,12 @@
 #include "tc.cuh"
 
 namespace grace {
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 
 constexpr int kGemmBM = 128;
 constexpr int kGemmBK = 64;
@@ -169,7 +175,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 constexpr int kPBK = 64;
 constexpr int kPStagingBytes = 128 * 128;                 // 128 rows x 128 bytes
 
-enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3 };
+enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3, kOutF32Lse = 4 };
 
 constexpr int kQStages = 6;
 constexpr int kQABytes = 128 * kPBK * 2;                  // 16 KB: 128 rows of A
@@ -180,7 +186,7 @@ constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 1024 + 256
 template <int OUT>
 __global__ void __launch_bounds__(192, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                   const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu) {
+                   const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* staging = tiles + kQStages * kQStageBytes;
@@ -273,6 +279,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       if (!ok) break;
       tc::tc_fence_after();
       const uint32_t t_acc = tmem_base + (uint32_t)(ab * 256) + ((uint32_t)(q * 32) << 16);
+      float lse_m = -INFINITY, lse_s = 0.f;                // kOutF32Lse: running maximum and sum of 2^((v - max) log2 e)
 #pragma unroll 1
       for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
         uint8_t* buf = staging + (g & 1) * kPStagingBytes;
@@ -302,6 +309,26 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           uint32_t r[32];
           tc::tmem_ld32(t_acc + (uint32_t)(c * 32), r);
           tc::tmem_ld_wait();
+          if (OUT == kOutF32Lse) {
+            // the row's log-sum-exp over this tile's 256 columns, 32 at a time (the tiles of a row are merged later)
+            float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
+#pragma unroll
+            for (int i = 4; i < 32; i += 4) {
+              m0c = fmaxf(m0c, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+              m1c = fmaxf(m1c, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
+            }
+            const float m_new = fmaxf(lse_m, fmaxf(m0c, m1c));
+            const float kLog2e = 1.4426950408889634f;
+            const float neg = -m_new * kLog2e;
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              s0 += fast_ex2(fmaf(__uint_as_float(r[i]), kLog2e, neg));
+              s1 += fast_ex2(fmaf(__uint_as_float(r[i + 1]), kLog2e, neg));
+            }
+            lse_s = lse_s * fast_ex2((lse_m - m_new) * kLog2e) + (s0 + s1);     // first chunk: lse_s = 0, factor 0
+            lse_m = m_new;
+          }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             float v[4];
@@ -315,6 +342,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           }
         }
         if (c == 256 / kColsPerChunk - 1) {                // accumulator fully read: hand it back to the issuer
+          if (OUT == kOutF32Lse && m0 + row < M)
+            lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = make_float2(lse_m, lse_s);
           tc::tc_fence_before();
           __syncwarp();
           if (lane == 0) {
@@ -342,7 +371,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 
 template <int OUT>
 static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
-                                  int K, int relu, cudaStream_t s) {
+                                  int K, int relu, cudaStream_t s, float2* lse_part = nullptr) {
   static unsigned long long attr_set_devices = 0;
   static int max_clusters = 0;
   cudaLaunchConfig_t cfg = {};
@@ -364,7 +393,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   }
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
-  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu));
+  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu, lse_part));
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -385,7 +414,8 @@ static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw
 
 static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
                                   uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
-                                  bool add_into_bf16, int M, int N, int K, int relu, void* stream) {
+                                  bool add_into_bf16, int M, int N, int K, int relu, void* stream,
+                                  float* lse_part = nullptr) {
   using namespace grace;
   if (!x || !w || ((y_bf16 == nullptr) == (y_f32 == nullptr))) return GRACE_INVALID_ARG;
   if (M <= 0 || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
@@ -395,6 +425,8 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
     return GRACE_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   const bool aliased = (residual != nullptr) && (residual == y_f32);
+  if (lse_part != nullptr && !(M >= 1024 && N >= 256 && (N % 256) == 0 && y_f32 != nullptr && residual == nullptr && !relu))
+    return GRACE_UNSUPPORTED_SHAPE;
   if (M >= 1024 && N >= 256 && (residual == nullptr || aliased)) {
     // large GEMM: persistent CTA-pair kernel, TMA-store epilogue (add-reduction when y is the residual stream)
     CUtensorMap mx, mw, my;
@@ -410,6 +442,7 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
       return GRACE_CUDA_ERROR;
     if (!f32) return add_into_bf16 ? launch_pair<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
                                    : launch_pair<kOutBf16>(mx, mw, my, M, N, K, relu, s);
+    if (lse_part != nullptr) return launch_pair<kOutF32Lse>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part));
     if (aliased) return launch_pair<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
     return launch_pair<kOutF32>(mx, mw, my, M, N, K, relu, s);
   }
@@ -435,6 +468,13 @@ extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uin
                                        uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
                                        int M, int N, int K, int relu, void* stream) {
   return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, residual, false, M, N, K, relu, stream);
+}
+
+extern "C" grace_status_t grace_linear_f32_lse(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                               float* y_f32, int64_t ldy, float* lse_part, int M, int N, int K,
+                                               void* stream) {
+  if (!lse_part || (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
+  return linear_impl(x, ldx, w, ldw, nullptr, y_f32, ldy, nullptr, false, M, N, K, 0, stream, lse_part);
 }
 
 extern "C" grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,

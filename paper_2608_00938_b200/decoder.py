@@ -33,7 +33,7 @@ class Decoder:
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
                  separate_cand=False, fuse_log_softmax=True, residual_bf16=False, materialize_cand=None,
-                 level_start=None):
+                 level_start=None, lse_from_gemm=True):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -127,6 +127,10 @@ class Decoder:
                 if sizes[t + 1] / max(1, sizes[t]) / V > 0.02:
                     self.masked_from_step = t + 1
         s.masked_from_step = self.masked_from_step
+        # log-sum-exp partials from the logits GEMM's epilogue (one pair per row and 256-column tile)
+        self.lse_part = (torch.zeros((R_max, V // 256, 2), dtype=torch.float32, device=dev)
+                         if (fuse_log_softmax and lse_from_gemm and V % 256 == 0 and V // 256 <= 32) else None)
+        s.lse_part = None if self.lse_part is None else self.lse_part.data_ptr()
         s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()
         self.struct = s
         code = api.grace_decoder_validate(s)

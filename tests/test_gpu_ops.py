@@ -638,3 +638,73 @@ def test_bounded_device_wait_gives_up_and_is_reported(api):
     ref = f64(x) @ f64(w).T
     assert np.abs(y.float().cpu().numpy() - ref).max() <= 2e-2 * max(1.0, np.abs(ref).max())
     assert api.grace_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("M,N,K", [(1024, 256, 64), (1500, 2048, 512), (2100, 512, 2048), (33000, 2048, 512)])
+def test_logits_gemm_leaves_log_sum_exp_partials(api, M, N, K):
+    """grace_linear_f32_lse: the same fp32 product as grace_linear, plus per row and 256-column tile the pair
+    (maximum, sum of e^(y - maximum)); merged, they are the row's log-sum-exp."""
+    rng = synth.rng_for(5, 13 * M + N + K)
+    x = synth.normal_bf16(rng, (M, K))
+    w = synth.normal_bf16(rng, (N, K), 0.08)
+    y0 = torch.zeros((M, N), dtype=torch.float32, device=DEV)
+    api.grace_linear(dev_bf16(x), dev_bf16(w), y0, None, False)
+    y = torch.zeros_like(y0)
+    part = torch.full((M, N // 256, 2), 7.0, device=DEV)
+    api.grace_linear_f32_lse(dev_bf16(x), dev_bf16(w), y, part)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int32), y0.view(torch.int32))
+    p = part.cpu().numpy().astype(np.float64)
+    yt = y.cpu().numpy().astype(np.float64).reshape(M, N // 256, 256)
+    assert np.array_equal(p[:, :, 0], yt.max(2))                                        # the tile maximum, exactly
+    np.testing.assert_allclose(p[:, :, 1], np.exp(yt - yt.max(2, keepdims=True)).sum(2), rtol=2e-6)
+    lse = p[:, :, 0].max(1) + np.log((p[:, :, 1] * np.exp(p[:, :, 0] - p[:, :, 0].max(1, keepdims=True))).sum(1))
+    ref = np.log(np.exp(yt.reshape(M, N) - yt.max((1, 2))[:, None]).sum(1)) + yt.max((1, 2))
+    np.testing.assert_allclose(lse, ref, atol=1e-5, rtol=0)
+    with pytest.raises(api.GraceError):                                                 # small problems: not offered
+        api.grace_linear_f32_lse(dev_bf16(x[:100]), dev_bf16(w), y[:100], part[:100])
+
+
+@pytest.mark.parametrize("kind,M", [("bloom", 600), ("node", 37)])
+def test_mask_kernel_merges_log_sum_exp_partials(api, kind, M):
+    """grace_gtm_mask_logits_parts against grace_gtm_mask_logits on the same logits: identical allow bits, the same
+    log-sum-exp to fp32 rounding, candidates equal to score + (logit - its own lse)."""
+    V, L, B, n_sids, depth = 1024, 4, 2, 60000, 1
+    sids, trie, elig, node, key, score, _ = _mask_problem(5 * V + depth + M, V, L, n_sids, B, M, depth)
+    rng = synth.rng_for(4, 950 + M)
+    logits = synth.normal_f32(rng, (B * M, V), 2.0)
+    bits, base, level_start = api.grace_trie_build_dense(sids, V)
+    d_bits, d_base = dev(bits), dev(base)
+    trie_s = api.make_trie(d_bits, d_base, V, L, trie.num_nodes)
+    if kind == "node":
+        keep = dev(np.stack([api.grace_node_bitmask_build(sids, V, e, trie.num_nodes) for e in elig]))
+        matcher = api.make_matcher(api.MATCH_NODE_BITMASK, keep)
+    else:
+        keep = dev(np.stack([api.grace_bloom_build(sids, V, e, 14, 4) for e in elig]))
+        matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, keep, 14, 4)
+    R, W = B * M, V // 64
+    # partials as the GEMM writes them, made here from the logits themselves
+    lt = logits.astype(np.float64).reshape(R, V // 256, 256)
+    part = np.stack([lt.max(2), np.exp(lt - lt.max(2, keepdims=True)).sum(2)], axis=2).astype(np.float32)
+    out = {}
+    for name in ("stream", "parts"):
+        cand = torch.full((R, V), 3.0, device=DEV)
+        allow = torch.zeros((R, W), dtype=torch.int64, device=DEV)
+        lse = torch.zeros(R, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        if name == "stream":
+            api.grace_gtm_mask_logits(dev(logits), lse, dev(score), dev(node), dev(key), trie_s, matcher, cand, allow, B, M, depth, status)
+        else:
+            api.grace_gtm_mask_logits_parts(dev(logits), lse, dev(score), dev(node), dev(key), trie_s, matcher, cand, allow, B, M,
+                                            depth, dev(part), status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        out[name] = (cand.cpu().numpy(), host_u64(allow), lse.cpu().numpy())
+    assert np.array_equal(out["stream"][1], out["parts"][1]) and out["parts"][1].any()
+    np.testing.assert_allclose(out["parts"][2], out["stream"][2], atol=2e-5, rtol=0)
+    live = node >= 0
+    cand, lse = out["parts"][0], out["parts"][2]
+    allowed = np.isfinite(cand)
+    want = (score[:, None] + (logits - lse[:, None])).astype(np.float32)
+    assert np.array_equal(cand[allowed].view(np.uint32), want[allowed].view(np.uint32))
+    assert not allowed[~live].any()
