@@ -85,7 +85,7 @@ def make_inputs(cfg, variant=0):
     return dict(sids=sids, elig=elig, shp=shp, weights=weights, enc_bits=enc_bits)
 
 
-def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None):
+def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, fold_layer_norm=None):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -97,7 +97,8 @@ def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None):
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=inp["weights"], trie_bits=bits,
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
-                  residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand)
+                  residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand,
+                  fold_layer_norm=fold_layer_norm)
     return dec
 
 
@@ -256,6 +257,22 @@ def op_breakdown(dec, cfg, reps=3):
         counts[name] = counts.get(name, 0) + 1
 
     import torch as _t
+    folded = getattr(dec, "fold_layer_norm", False)
+
+    def ln_linear(x, g, b, hbuf, w, fold, y, fl, relu=False, lse_part=None):
+        """LayerNorm + the GEMM behind it, as the decode path runs them (two kernels, or folded)."""
+        if folded:
+            wf, cs, cb = fold
+            timed("row_stats", lambda: api.grace_row_stats_bf16(x, dec.row_affine[:x.shape[0]]))
+            timed("linear", lambda: api.grace_linear_folded_ln(x, wf, dec.row_affine[:x.shape[0]],
+                                                               None if dec.centre_stream else cs, cb, y, relu, lse_part), fl)
+        else:
+            timed("layer_norm", lambda: api.grace_layer_norm(x, g, b, hbuf))
+            if lse_part is not None:
+                timed("linear", lambda: api.grace_linear_f32_lse(hbuf, w, y, lse_part), fl)
+            else:
+                timed("linear", lambda: api.grace_linear(hbuf, w, y, None, relu), fl)
+
     if dec.x.dtype == _t.bfloat16:          # bf16 residual stream: y += x w^T by a bf16 add-reduction
         add_into_x = lambda a, w, x: api.grace_linear_add_bf16(a, w, x)
     else:
@@ -274,29 +291,24 @@ def op_breakdown(dec, cfg, reps=3):
                 q3 = qkv.view(-1)[:R * 3 * HD].view(R, 3 * HD)
                 q1 = qkv.view(-1)[:R * HD].view(R, HD)
                 ff = qkv.view(-1)[:R * F].view(R, F)
-                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln1_g"], lay["ln1_b"], hD))
-                timed("linear", lambda: api.grace_linear(hD, lay["w_qkv"], q3), 2.0 * R * D * 3 * HD)
+                fo = dec.folded[li] if folded else {}
+                ln_linear(x, lay["ln1_g"], lay["ln1_b"], hD, lay["w_qkv"], fo.get("w_qkv"), q3, 2.0 * R * D * 3 * HD)
                 timed("self_attn", lambda: api.grace_self_attn(q3.view(R, 3, H, dh), dec.k_cache[li], dec.v_cache[li],
                                                                dec.parents, sizes, attn.view(R, H, dh), B, t, scale,
                                                                dec.d_status))
                 timed("linear", lambda: add_into_x(attn, lay["w_o"], x), 2.0 * R * HD * D)
-                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln2_g"], lay["ln2_b"], hD))
-                timed("linear", lambda: api.grace_linear(hD, lay["w_qc"], q1), 2.0 * R * D * HD)
+                ln_linear(x, lay["ln2_g"], lay["ln2_b"], hD, lay["w_qc"], fo.get("w_qc"), q1, 2.0 * R * D * HD)
                 timed("cross_attn", lambda: api.grace_cross_attn(
                     q1.view(R, H, dh), dec.k_cross[li].permute(0, 2, 1, 3), dec.v_cross[li].permute(0, 2, 1, 3),
                     attn.view(R, H, dh), scale), 4.0 * R * H * dh * cfg["T_ctx"])
                 timed("linear", lambda: add_into_x(attn, lay["w_oc"], x), 2.0 * R * HD * D)
-                timed("layer_norm", lambda: api.grace_layer_norm(x, lay["ln3_g"], lay["ln3_b"], hD))
-                timed("linear", lambda: api.grace_linear(hD, lay["w_1"], ff, None, True), 2.0 * R * D * F)
+                ln_linear(x, lay["ln3_g"], lay["ln3_b"], hD, lay["w_1"], fo.get("w_1"), ff, 2.0 * R * D * F, relu=True)
                 timed("linear", lambda: add_into_x(ff, lay["w_2"], x), 2.0 * R * F * D)
-            timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
             logp = dec.logp[:R]
-            parts = dec.lse_part is not None and R >= 1024
-            if parts:                                   # the logits GEMM also leaves the rows' log-sum-exp partials
-                lsep = dec.lse_part[:R]
-                timed("linear", lambda: api.grace_linear_f32_lse(hD, dec.w_out, logp, lsep), 2.0 * R * D * V)
-            else:
-                timed("linear", lambda: api.grace_linear(hD, dec.w_out, logp), 2.0 * R * D * V)
+            parts = dec.lse_part is not None and R >= 1024   # the logits GEMM also leaves the rows' log-sum-exp partials
+            lsep = dec.lse_part[:R] if parts else None
+            ln_linear(x, dec.lnf_g, dec.lnf_b, hD, dec.w_out, (dec.w_out, dec.cs_out, dec.cb_out) if folded else None,
+                      logp, 2.0 * R * D * V, lse_part=lsep)
             par = dec.parents[t + 1]
             masked = dec.allow_bits is not None and t >= dec.masked_from_step
             if masked:                                  # candidates never materialised: allow bits + masked top-k
@@ -495,6 +507,8 @@ def main():
                     help="beam sizes per step, e.g. 1,512,1024,1024 (dynamic beam schedule, Section 3.3)")
     ap.add_argument("--residual", default="bf16", choices=["bf16", "f32"],
                     help="dtype of the residual stream between blocks (weights, activations and caches are bf16 either way)")
+    ap.add_argument("--layer-norm", default="folded", choices=["folded", "kernel"],
+                    help="LayerNorms folded into the GEMMs behind them (bf16 stream), or run as kernels of their own")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -524,7 +538,8 @@ def main():
         cfg["final_k"] = cfg["schedule"][-1]
     default_workload = (args.workload == "cfg5" and not args.schedule)
     inp = make_inputs(cfg, variant=rank)
-    dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"))
+    dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"),
+                        fold_layer_norm=(None if args.layer_norm == "folded" else False))
     dec._layer_tensors = _layer_tensor_views(dec, inp)
     enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
     dec.project_cross_kv(enc_dev)
@@ -559,6 +574,7 @@ def main():
                             matcher="prefix_bloom_2^22x4", parallelism=f"requests sharded x{world}",
                             l2="working set ~5 GB per loop, far larger than the 126 MB L2", launch=launch_mode,
                             residual_stream=args.residual, accumulate="f32",
+                            layer_norm=("folded into the GEMMs, centred stream" if dec.fold_layer_norm else "kernel"),
                             macs_per_request=decoder_macs(cfg)),
                 launch_modes=dict(eager_ms_per_step=eager_ms, cuda_graph_ms_per_step=graph_ms),
                 step_latency_us=per_step_us, clocks=clocks, gpu_launches=int(launches_per_loop * args.steps),

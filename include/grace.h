@@ -377,6 +377,25 @@ grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint1
 grace_status_t grace_linear_f32_lse(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
                                     float* y_f32, int64_t ldy, float* lse_part, int M, int N, int K, void* stream);
 
+/* A LayerNorm folded into the GEMM that consumes it.  With w' = w * gamma (per input feature),
+ *   LayerNorm(x) @ w^T  =  rstd * (x @ w'^T)  -  rstd * mean * colsum(w')  +  beta @ w^T,
+ * so the GEMM can read the raw bf16 residual stream (no normalised copy is written or read) and finish in its
+ * epilogue with two numbers per row and two per column.
+ * grace_row_stats_bf16: row_affine fp32 [R][2] = (rstd, -rstd * mean) of x bf16 [R][D] (D % 8 == 0, D <= 2048).
+ * grace_linear_folded_ln: y = row_affine[m][0] * (x @ w^T)[m][n] + row_affine[m][1] * col_sum[n] + col_bias[n],
+ *   then ReLU if relu; output bf16 (y_bf16) or fp32 (y_f32; with lse_part also the log-sum-exp partials of
+ *   grace_linear_f32_lse).  Shapes as grace_linear; col_sum / col_bias fp32 [N], 16-byte aligned.
+ *   col_sum may be NULL: the middle term is dropped.  That is exact when every row of x has zero mean, which a
+ *   pre-LayerNorm residual stream keeps if everything added into it is centred over the feature axis (embedding
+ *   rows minus their mean; output projections minus their mean over the output index): LayerNorm does not see
+ *   a per-row shift, so the model computes the same function, and the epilogue then costs one shared-memory
+ *   word per column instead of two (the difference between hiding under the next tile's MMAs and not). */
+grace_status_t grace_row_stats_bf16(const uint16_t* x, int R, int D, float eps, float* row_affine, void* stream);
+grace_status_t grace_linear_folded_ln(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                      const float* row_affine, const float* col_sum, const float* col_bias,
+                                      uint16_t* y_bf16, float* y_f32, int64_t ldy, float* lse_part,
+                                      int M, int N, int K, int relu, void* stream);
+
 /* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
 grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
                                 uint16_t* out, int R, int D, float eps, void* stream);
@@ -407,6 +426,10 @@ typedef struct {
   const uint16_t *k_cross, *v_cross;   /* [B][T_ctx][H][d_h]: as the once-per-request projection
                                           GEMM of the encoder output writes them (Section 3.2) */
   uint16_t *k_cache, *v_cache;         /* [L][R_max][H][d_h] */
+  /* With grace_decoder_t.ln_folded: w_qkv, w_qc, w_1 already carry the gain of the LayerNorm in front of
+   * them (w[n][k] * gamma[k], rounded to bf16) and these hold, per output feature n, the sum over k of that
+   * matrix (cs_*) and the sum over k of beta[k] * (unfolded) w[n][k] (cb_*), fp32 [out_features]. */
+  const float *cs_qkv, *cb_qkv, *cs_qc, *cb_qc, *cs_1, *cb_1;
 } grace_layer_t;
 
 #define GRACE_MAX_LAYERS 16
@@ -451,6 +474,11 @@ typedef struct {
   int32_t reserved2;
   float *lse_part;            /* NULL, or [R_max][V/256][2] (needs row_lse, V % 256 == 0): the logits GEMM
                                  leaves per-tile log-sum-exp partials and the mask kernel merges them     */
+  /* LayerNorms folded into the GEMMs behind them (bf16 residual stream only): NULL, or [R_max][2] scratch
+     for the row statistics; then w_qkv / w_qc / w_1 / w_out carry the gains and cb_* are set; cs_* are set
+     too unless the caller keeps the stream's rows at zero mean (see grace_linear_folded_ln). */
+  float *row_affine;
+  const float *cs_out, *cb_out;   /* [V] for the output head (final LayerNorm)                         */
   void *topk_ws; size_t topk_ws_bytes;
   int32_t *d_status;
 } grace_decoder_t;

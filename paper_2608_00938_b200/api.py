@@ -51,7 +51,8 @@ class LayerStruct(C.Structure):
     _fields_ = [(n, _vp) for n in (
         "ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b",
         "w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2",
-        "k_cross", "v_cross", "k_cache", "v_cache")]
+        "k_cross", "v_cross", "k_cache", "v_cache",
+        "cs_qkv", "cb_qkv", "cs_qc", "cb_qc", "cs_1", "cb_1")]
 
 
 class DecoderStruct(C.Structure):
@@ -68,7 +69,7 @@ class DecoderStruct(C.Structure):
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
         ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp), ("allow_bits", _vp), ("masked_from_step", C.c_int32),
-        ("reserved2", C.c_int32), ("lse_part", _vp),
+        ("reserved2", C.c_int32), ("lse_part", _vp), ("row_affine", _vp), ("cs_out", _vp), ("cb_out", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -108,6 +109,9 @@ _linear_f32_lse = _sig("grace_linear_f32_lse", _i32, [_vp, _i64, _vp, _i64, _vp,
 _gtm_mask_logits_parts = _sig("grace_gtm_mask_logits_parts", _i32,
                               [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct), _vp, _vp,
                                _i32, _i32, _i32, _i32, _vp, _i32, _vp, _vp])
+_row_stats_bf16 = _sig("grace_row_stats_bf16", _i32, [_vp, _i32, _i32, _f32, _vp, _vp])
+_linear_folded_ln = _sig("grace_linear_folded_ln", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
+                                                         _i32, _i32, _i32, _i32, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
@@ -324,6 +328,26 @@ def grace_gtm_mask_logits_parts(logits, row_lse, beam_score, beam_node, beam_key
     _check(_gtm_mask_logits_parts(_dp(logits), _dp(row_lse), _dp(beam_score), _dp(beam_node), _dp(beam_key), C.byref(trie),
                                   C.byref(matcher), _dp(cand), _dp(allow_bits), B, M, V, prefix_len, _dp(lse_part),
                                   lse_part.shape[1], _dp(d_status), _stream()), "grace_gtm_mask_logits_parts")
+
+
+def grace_row_stats_bf16(x, row_affine, eps: float = 1e-5):
+    """row_affine fp32 [R, 2] = (rstd, -rstd * mean) of the bf16 rows of x."""
+    R, D = x.shape
+    _check(_row_stats_bf16(_dp(x), R, D, eps, _dp(row_affine), _stream()), "grace_row_stats_bf16")
+    return row_affine
+
+
+def grace_linear_folded_ln(x, w_folded, row_affine, col_sum, col_bias, y, relu: bool = False, lse_part=None):
+    """y = row_affine[:, :1] * (x @ w_folded.T) + row_affine[:, 1:] * col_sum + col_bias  (LayerNorm folded into
+    the GEMM); y bf16 or fp32.  col_sum None: the rows of x have zero mean and the middle term is dropped."""
+    import torch
+    M, K = x.shape
+    N = w_folded.shape[0]
+    f32 = y.dtype == torch.float32
+    _check(_linear_folded_ln(x.data_ptr(), x.stride(0), w_folded.data_ptr(), w_folded.stride(0), _dp(row_affine),
+                             _dp(col_sum), _dp(col_bias), None if f32 else _dp(y), _dp(y) if f32 else None, y.stride(0),
+                             _dp(lse_part), M, N, K, int(relu), _stream()), "grace_linear_folded_ln")
+    return y
 
 
 def grace_wait_timeouts() -> int:

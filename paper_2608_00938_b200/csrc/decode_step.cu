@@ -29,6 +29,13 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
   if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || (!d->x && !d->x_bf16) || !d->h || !d->qkv ||
       !d->attn || !d->logp || !d->cand || !d->topk_ws || !d->out_flat)
     return GRACE_INVALID_ARG;
+  if (d->row_affine != nullptr) {                          // folded LayerNorms: bf16 stream and every bias vector
+    if (!d->x_bf16 || d->x || !d->cb_out) return GRACE_INVALID_ARG;        // (column sums: none = centred stream)
+    for (int l = 0; l < d->n_layers; ++l) {
+      const grace_layer_t& w = d->layers[l];
+      if (!w.cb_qkv || !w.cb_qc || !w.cb_1) return GRACE_INVALID_ARG;
+    }
+  }
   for (int i = 0; i < 2; ++i)
     if (!d->token[i] || !d->score[i] || !d->node[i] || !d->key[i]) return GRACE_INVALID_ARG;
   if (d->trie.V != d->V || d->trie.L != d->L || !d->trie.child_bits || !d->trie.child_base) return GRACE_INVALID_ARG;
@@ -76,6 +83,22 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
     return xb ? grace_layer_norm_bf16(d->x_bf16, g, b, d->h, R, D, d->ln_eps, stream)
               : grace_layer_norm(d->x, g, b, d->h, R, D, d->ln_eps, stream);
   };
+  // LayerNorm + the GEMM that consumes it: either the two kernels, or (folded) row statistics + a GEMM on the
+  // raw stream whose epilogue applies them
+  const bool folded = xb && d->row_affine != nullptr;
+  auto ln_linear = [&](const float* g, const float* b, const uint16_t* w, const float* cs, const float* cb,
+                       uint16_t* y_bf16, float* y_f32, int64_t ldy, int N, int relu, float* lse_part) -> grace_status_t {
+    if (folded) {
+      grace_status_t s1 = grace_row_stats_bf16(d->x_bf16, R, D, d->ln_eps, d->row_affine, stream);
+      if (s1 != GRACE_OK) return s1;
+      return grace_linear_folded_ln(d->x_bf16, D, w, D, d->row_affine, cs, cb, y_bf16, y_f32, ldy, lse_part, R, N, D, relu,
+                                    stream);
+    }
+    grace_status_t s1 = layer_norm(g, b);
+    if (s1 != GRACE_OK) return s1;
+    if (lse_part != nullptr) return grace_linear_f32_lse(d->h, D, w, D, y_f32, ldy, lse_part, R, N, D, stream);
+    return grace_linear(d->h, D, w, D, y_bf16, y_f32, ldy, nullptr, R, N, D, relu, stream);
+  };
   auto add_into_x = [&](const uint16_t* a, int64_t lda, const uint16_t* w, int K) -> grace_status_t {
     return xb ? grace_linear_add_bf16(a, lda, w, K, d->x_bf16, D, R, D, K, stream)
               : grace_linear(a, lda, w, K, nullptr, d->x, D, d->x, R, D, K, 0, stream);
@@ -85,28 +108,24 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   for (int l = 0; l < d->n_layers; ++l) {
     const grace_layer_t& w = d->layers[l];
     // self-attention block
-    GRACE_TRY(layer_norm(w.ln1_g, w.ln1_b));
-    GRACE_TRY(grace_linear(d->h, D, w.w_qkv, D, d->qkv, nullptr, 3 * HD, nullptr, R, 3 * HD, D, 0, stream));
+    GRACE_TRY(ln_linear(w.ln1_g, w.ln1_b, w.w_qkv, w.cs_qkv, w.cb_qkv, d->qkv, nullptr, 3 * HD, 3 * HD, 0, nullptr));
     GRACE_TRY(grace_self_attn(d->qkv, 3 * HD, w.k_cache, w.v_cache, d->parents, d->beam_sizes, d->attn, HD,
                               B, t, d->H, d->d_h, d->R_max, scale, st, stream));
     GRACE_TRY(add_into_x(d->attn, HD, w.w_o, HD));
     // cross-attention block
-    GRACE_TRY(layer_norm(w.ln2_g, w.ln2_b));
-    GRACE_TRY(grace_linear(d->h, D, w.w_qc, D, d->qkv, nullptr, HD, nullptr, R, HD, D, 0, stream));
+    GRACE_TRY(ln_linear(w.ln2_g, w.ln2_b, w.w_qc, w.cs_qc, w.cb_qc, d->qkv, nullptr, HD, HD, 0, nullptr));
     GRACE_TRY(grace_cross_attn(d->qkv, HD, w.k_cross, w.v_cross, (int64_t)d->T_ctx * HD, d->d_h, HD, d->attn, HD,
                                nullptr, B, M, d->H, d->d_h, d->T_ctx, scale, st, stream));
     GRACE_TRY(add_into_x(d->attn, HD, w.w_oc, HD));
     // feed-forward block
-    GRACE_TRY(layer_norm(w.ln3_g, w.ln3_b));
-    GRACE_TRY(grace_linear(d->h, D, w.w_1, D, d->qkv, nullptr, d->d_ffn, nullptr, R, d->d_ffn, D, 1, stream));
+    GRACE_TRY(ln_linear(w.ln3_g, w.ln3_b, w.w_1, w.cs_1, w.cb_1, d->qkv, nullptr, d->d_ffn, d->d_ffn, 1, nullptr));
     GRACE_TRY(add_into_x(d->qkv, d->d_ffn, w.w_2, d->d_ffn));
   }
-  GRACE_TRY(layer_norm(d->lnf_g, d->lnf_b));
   // the logits GEMM can leave the rows' log-sum-exp partials (large steps), the mask kernel then merges them
   const int n_parts = d->V / 256;
   const bool parts = d->lse_part != nullptr && d->row_lse != nullptr && R >= 1024 && (d->V % 256) == 0 && n_parts <= 32;
-  if (parts) GRACE_TRY(grace_linear_f32_lse(d->h, D, d->w_out, D, d->logp, d->V, d->lse_part, R, d->V, D, stream));
-  else GRACE_TRY(grace_linear(d->h, D, d->w_out, D, nullptr, d->logp, d->V, nullptr, R, d->V, D, 0, stream));
+  GRACE_TRY(ln_linear(d->lnf_g, d->lnf_b, d->w_out, d->cs_out, d->cb_out, nullptr, d->logp, d->V, d->V, 0,
+                      parts ? d->lse_part : nullptr));
   // log-softmax, CD + GTM mask and score add: one fused kernel when row_lse is provided
   int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
   if (d->row_lse != nullptr && d->allow_bits != nullptr && t >= d->masked_from_step) {

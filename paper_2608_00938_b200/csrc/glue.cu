@@ -149,6 +149,59 @@ layer_norm_bf16_kernel(const uint16_t* __restrict__ x, const float* __restrict__
   }
 }
 
+// Row statistics of the bf16 residual stream for a LayerNorm that is folded into the next GEMM:
+// out[r] = (rstd, -rstd * mean).  Same load and reduction structure as layer_norm_bf16_kernel.
+template <int MAXV, int ROWS>
+__global__ void __launch_bounds__(128)
+row_stats_bf16_kernel(const uint16_t* __restrict__ x, float2* __restrict__ out, int R, int D, float eps) {
+  pdl_wait();
+  pdl_trigger();
+  const int lane = threadIdx.x & 31;
+  const int r0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
+  if (r0 >= R) return;
+  const int n8 = D >> 3;
+  uint4 raw[ROWS][MAXV];
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    const uint4* row = reinterpret_cast<const uint4*>(x + (int64_t)(r0 + j) * D);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const int c = i * 32 + lane;
+      raw[j][i] = (c < n8 && r0 + j < R) ? ld_stream_u4(row + c) : make_uint4(0, 0, 0, 0);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < ROWS; ++j) {
+    f32x2_t acc = f2_pack(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      const uint4 t = raw[j][i];
+      acc = f2_add(acc, f2_add(f2_add(f2_from_bf16x2(t.x), f2_from_bf16x2(t.y)),
+                               f2_add(f2_from_bf16x2(t.z), f2_from_bf16x2(t.w))));
+    }
+    float lo, hi;
+    f2_unpack(acc, lo, hi);
+    const float mean = warp_sum(lo + hi) / (float)D;
+    const f32x2_t m2 = f2_pack(mean, mean);
+    f32x2_t sq = f2_pack(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < MAXV; ++i) {
+      if (i * 32 + lane < n8) {
+        const uint4 t = raw[j][i];
+        const uint32_t w4[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const f32x2_t d = f2_sub(f2_from_bf16x2(w4[e]), m2);
+          sq = f2_fma(d, d, sq);
+        }
+      }
+    }
+    f2_unpack(sq, lo, hi);
+    const float rstd = rsqrtf(warp_sum(lo + hi) / (float)D + eps);
+    if (lane == 0 && r0 + j < R) out[r0 + j] = make_float2(rstd, -rstd * mean);
+  }
+}
+
 __global__ void embed_bf16_kernel(const int32_t* __restrict__ token, const uint16_t* __restrict__ embed,
                                   const uint16_t* __restrict__ pos, uint16_t* __restrict__ x, int R, int D,
                                   int n_rows_embed, int32_t* d_status) {
@@ -315,6 +368,24 @@ extern "C" grace_status_t grace_embed_bf16(const int32_t* token, const uint16_t*
   if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(embed) & 7) || (reinterpret_cast<uintptr_t>(pos) & 7))
     return GRACE_INVALID_ARG;
   grace::launch_pdl(grace::embed_bf16_kernel, dim3((R + 3) / 4), dim3(128), 0, (cudaStream_t)stream, token, embed, pos, x, R, D, n_rows_embed, d_status);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_row_stats_bf16(const uint16_t* x, int R, int D, float eps, float* row_affine,
+                                               void* stream) {
+  using namespace grace;
+  if (!x || !row_affine || R <= 0 || D <= 0 || (reinterpret_cast<uintptr_t>(row_affine) & 7)) return GRACE_INVALID_ARG;
+  if ((D & 7) || D > 2048) return GRACE_UNSUPPORTED_SHAPE;
+  if (!grace_aligned16(x)) return GRACE_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  float2* out = reinterpret_cast<float2*>(row_affine);
+  const int pieces = ((D >> 3) + 31) / 32;
+  auto blocks = [&](int rows) { return (R + 4 * rows - 1) / (4 * rows); };
+  if (pieces <= 1) launch_pdl(row_stats_bf16_kernel<1, 4>, dim3(blocks(4)), dim3(128), 0, s, x, out, R, D, eps);
+  else if (pieces <= 2) launch_pdl(row_stats_bf16_kernel<2, 4>, dim3(blocks(4)), dim3(128), 0, s, x, out, R, D, eps);
+  else if (pieces <= 4) launch_pdl(row_stats_bf16_kernel<4, 2>, dim3(blocks(2)), dim3(128), 0, s, x, out, R, D, eps);
+  else launch_pdl(row_stats_bf16_kernel<8, 1>, dim3(blocks(1)), dim3(128), 0, s, x, out, R, D, eps);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

@@ -37,6 +37,10 @@ struct GemmParams {
   float* y_f32;
   const float* residual;
   const uint16_t* residual_bf16;   // bf16 residual stream (added in fp32, result rounded to bf16)
+  // LayerNorm folded into the GEMM (x is the raw stream, w carries the gain): y = row.x * acc + row.y * col_sum + col_bias
+  const float2* aff_row;           // [M]: (rstd, -rstd * mean) of the row; nullptr = plain GEMM
+  const float* aff_cs;             // [N]: sum over k of w[n][k]
+  const float* aff_cb;             // [N]: sum over k of beta[k] * w0[n][k]
   int64_t ldy;
   int M, N, K, relu;
 };
@@ -104,6 +108,23 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
   __syncwarp();
 
   // ---- epilogue: warp w owns TMEM lanes 32w .. 32w+31 = rows m0 + 32w + lane ----
+  // Folded LayerNorm: the row's pair and the column vectors of a chunk are fetched (from clamped addresses,
+  // unconditionally) one chunk ahead of their use, the first while the accumulator is still filling.
+  const bool folded = p.aff_row != nullptr;
+  const float* cs_or_cb = p.aff_cs != nullptr ? p.aff_cs : p.aff_cb;
+  float2 ar = make_float2(1.f, 0.f);
+  float4 cs_next[4], cb_next[4];
+  auto fetch_cols = [&](int c) {
+    if (!folded) return;
+    const int n = min(n0 + c, p.N - 16);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      cb_next[j] = __ldg(reinterpret_cast<const float4*>(p.aff_cb + n) + j);
+      cs_next[j] = __ldg(reinterpret_cast<const float4*>(cs_or_cb + n) + j);
+    }
+  };
+  if (folded) ar = __ldg(p.aff_row + min(m0 + warp * 32 + lane, p.M - 1));
+  fetch_cols(0);
   const bool ok = tc::mbar_wait(accum_bar, 0, abort_flag);
   tc::tc_fence_after();
   __syncwarp();
@@ -113,6 +134,15 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     for (int c = 0; c < BN; c += 16) {
       uint32_t acc[16];
       tc::tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, acc);
+      float cs[16], cb[16];
+      if (folded) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          cs[4 * j] = cs_next[j].x; cs[4 * j + 1] = cs_next[j].y; cs[4 * j + 2] = cs_next[j].z; cs[4 * j + 3] = cs_next[j].w;
+          cb[4 * j] = cb_next[j].x; cb[4 * j + 1] = cb_next[j].y; cb[4 * j + 2] = cb_next[j].z; cb[4 * j + 3] = cb_next[j].w;
+        }
+        if (c + 16 < BN) fetch_cols(c + 16);
+      }
       tc::tmem_ld_wait();
       const int n = n0 + c;
       if (m < p.M && n < p.N) {           // N % 16 == 0: the 16 columns are all in or all out
@@ -120,6 +150,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           v[j] = __uint_as_float(acc[j]);
+          if (folded) v[j] = fmaf(ar.x, v[j], p.aff_cs != nullptr ? fmaf(ar.y, cs[j], cb[j]) : cb[j]);
           if (p.relu) v[j] = fmaxf(v[j], 0.f);
         }
         if (p.residual != nullptr) {
@@ -181,14 +212,23 @@ constexpr int kQStages = 6;
 constexpr int kQABytes = 128 * kPBK * 2;                  // 16 KB: 128 rows of A
 constexpr int kQBBytes = 128 * kPBK * 2;                  // 16 KB: 128 of the tile's 256 rows of W
 constexpr int kQStageBytes = kQABytes + kQBBytes;
-constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 1024 + 256;
+constexpr int kQAffBytes = 256 * 2 * 4;                   // the tile's 256 (col_sum, col_bias) pairs
+// no slack for rounding the base up: the dynamic shared memory is declared 1024-byte aligned and the kernel
+// checks it (six stages, the staging buffers and the column vectors leave less than 1 KB of the 227 KB)
+constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 256 + kQAffBytes;
 
 template <int OUT>
 __global__ void __launch_bounds__(192, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                   const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+                   const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part,
+                   const float2* __restrict__ aff_row, const float* __restrict__ aff_cs,
+                   const float* __restrict__ aff_cb) {
+  extern __shared__ __align__(1024) uint8_t smem_pair[];
+  uint8_t* tiles = smem_pair;
+  if ((tc::smem_addr(tiles) & 1023u) != 0) {               // the swizzled tiles need it; same answer in every thread
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(&tc::g_tc_timeouts, 1);
+    return;
+  }
   uint8_t* staging = tiles + kQStages * kQStageBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(staging + 2 * kPStagingBytes);   // even CTA only: both CTAs' bytes landed
   uint64_t* empty = full + kQStages;           // the pair's MMAs have read the stage
@@ -196,6 +236,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   uint64_t* acc_empty = acc_full + 2;          // [2] even CTA only: 4 local + 4 remote epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float4* aff_s = reinterpret_cast<float4*>(staging + 2 * kPStagingBytes + 256);   // [128]: (cs, cs, cb, cb) of 2 columns
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = tc::cluster_cta_rank();            // 0: issues the MMAs; 1: peer
@@ -271,27 +312,91 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     constexpr bool kBf16Out = (OUT == kOutBf16 || OUT == kOutBf16Add);
     constexpr int kColsPerChunk = kBf16Out ? 64 : 32;
     int local = 0, g = 0;
+    // LayerNorm folded into the GEMM: y = ar.x * acc + (ar.y * col_sum + col_bias).  The tile's column vectors go
+    // through shared memory (every thread needs all 256 of them); they and the row's pair are fetched one tile
+    // ahead, so their latency never sits between two tiles of an epilogue that is the pair's critical path.
+    // (The loads are unconditional, from clamped addresses, so that nothing waits for them before their use.)
+    float2 ar_next = make_float2(1.f, 0.f), cs_next = make_float2(0.f, 0.f), cb_next = make_float2(0.f, 0.f);
+    const float* cs_or_cb = aff_cs != nullptr ? aff_cs : aff_cb;
+    auto fetch_affine = [&](int tile) {
+      if (aff_row == nullptr) return;
+      tile = min(tile, total - 1);
+      const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
+      const int col = min(n0 + 2 * row, N - 2);
+      ar_next = __ldg(aff_row + min(m0 + row, M - 1));
+      cb_next = __ldg(reinterpret_cast<const float2*>(aff_cb + col));
+      cs_next = __ldg(reinterpret_cast<const float2*>(cs_or_cb + col));
+    };
+    fetch_affine(pair);
     for (int tile = pair; tile < total; tile += n_pairs, ++local) {
       const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
       const int ab = local & 1;
+      const float2 ar = ar_next;                           // rows and columns past the edge: values never stored
+      const float4 cv = aff_cs != nullptr ? make_float4(cs_next.x, cs_next.y, cb_next.x, cb_next.y)
+                                          : make_float4(cb_next.x, cb_next.y, 0.f, 0.f);
       bool ok = tc::mbar_wait_cluster(acc_full + ab, (local >> 1) & 1, abort_flag);
       ok = __all_sync(kFullMask, ok);
       if (!ok) break;
       tc::tc_fence_after();
       const uint32_t t_acc = tmem_base + (uint32_t)(ab * 256) + ((uint32_t)(q * 32) << 16);
       float lse_m = -INFINITY, lse_s = 0.f;                // kOutF32Lse: running maximum and sum of 2^((v - max) log2 e)
+      // read after the first chunk's barrier; the previous tile's readers are past its last barrier.
+      // With col_sum: [128] x (cs, cs, cb, cb) of two columns; without: col_bias alone, [256] floats.
+      if (aff_row != nullptr) {
+        if (aff_cs != nullptr) aff_s[row] = cv;
+        else reinterpret_cast<float2*>(aff_s)[row] = make_float2(cv.x, cv.y);
+      }
+      fetch_affine(tile + n_pairs);
+      const f32x2_t ar_x = f2_pack(ar.x, ar.x), ar_y = f2_pack(ar.y, ar.y);
+      auto fold = [&](uint32_t (&r)[32], int col0) {        // col0: first of the 32 columns, within the tile
+        if (aff_row == nullptr) return;
+        if (aff_cs == nullptr) {                            // centred rows: y = ar.x * acc + col_bias
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const float4 c = aff_s[(col0 + i) >> 2];
+            float a0, a1, a2, a3;
+            f2_unpack(f2_fma(ar_x, f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), f2_pack(c.x, c.y)), a0, a1);
+            f2_unpack(f2_fma(ar_x, f2_pack(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), f2_pack(c.z, c.w)), a2, a3);
+            r[i] = __float_as_uint(a0); r[i + 1] = __float_as_uint(a1);
+            r[i + 2] = __float_as_uint(a2); r[i + 3] = __float_as_uint(a3);
+          }
+          return;
+        }
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float4 c = aff_s[(col0 + i) >> 1];
+#ifdef GRACE_FOLD_SCALAR
+          r[i] = __float_as_uint(fmaf(ar.x, __uint_as_float(r[i]), fmaf(ar.y, c.x, c.z)));
+          r[i + 1] = __float_as_uint(fmaf(ar.x, __uint_as_float(r[i + 1]), fmaf(ar.y, c.y, c.w)));
+          continue;
+#endif
+          const f32x2_t v = f2_fma(ar_x, f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])),
+                                   f2_fma(ar_y, f2_pack(c.x, c.y), f2_pack(c.z, c.w)));
+          float lo, hi;
+          f2_unpack(v, lo, hi);
+          r[i] = __float_as_uint(lo);
+          r[i + 1] = __float_as_uint(hi);
+        }
+      };
 #pragma unroll 1
       for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
         uint8_t* buf = staging + (g & 1) * kPStagingBytes;
+        uint32_t rr[kBf16Out ? 2 : 1][32];
+        if (kBf16Out) {                                    // the chunk's loads fly while the staging buffer frees up
+          tc::tmem_ld32(t_acc + (uint32_t)(c * 64), rr[0]);
+          tc::tmem_ld32(t_acc + (uint32_t)(c * 64 + 32), rr[kBf16Out ? 1 : 0]);
+        } else {
+          tc::tmem_ld32(t_acc + (uint32_t)(c * 32), rr[0]);
+        }
         if (issuer) tc::bulk_wait_read<1>();               // the store that last used `buf` has read it
         tc::named_bar_sync(1, 128);
+        tc::tmem_ld_wait();
         uint4* my_row = reinterpret_cast<uint4*>(buf + row * 128);
         if (kBf16Out) {
 #pragma unroll
           for (int hseg = 0; hseg < 2; ++hseg) {
-            uint32_t r[32];
-            tc::tmem_ld32(t_acc + (uint32_t)(c * 64 + hseg * 32), r);
-            tc::tmem_ld_wait();
+            uint32_t (&r)[32] = rr[kBf16Out ? hseg : 0];
+            fold(r, c * 64 + hseg * 32);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               float v[8];
@@ -306,9 +411,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             }
           }
         } else {
-          uint32_t r[32];
-          tc::tmem_ld32(t_acc + (uint32_t)(c * 32), r);
-          tc::tmem_ld_wait();
+          uint32_t (&r)[32] = rr[0];
+          fold(r, c * 32);
           if (OUT == kOutF32Lse) {
             // the row's log-sum-exp over this tile's 256 columns, 32 at a time (the tiles of a row are merged later)
             float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
@@ -369,9 +473,16 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   if (warp == 0) tc::tmem_dealloc_pair(tmem_base, 512);
 }
 
+struct Affine {                                            // LayerNorm folded into the GEMM; row == nullptr: off
+  const float2* row;
+  const float* cs;
+  const float* cb;
+};
+
 template <int OUT>
 static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
-                                  int K, int relu, cudaStream_t s, float2* lse_part = nullptr) {
+                                  int K, int relu, cudaStream_t s, float2* lse_part = nullptr,
+                                  Affine aff = Affine{nullptr, nullptr, nullptr}) {
   static unsigned long long attr_set_devices = 0;
   static int max_clusters = 0;
   cudaLaunchConfig_t cfg = {};
@@ -393,7 +504,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   }
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
-  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu, lse_part));
+  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb));
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -415,7 +526,8 @@ static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw
 static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
                                   uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
                                   bool add_into_bf16, int M, int N, int K, int relu, void* stream,
-                                  float* lse_part = nullptr) {
+                                  float* lse_part = nullptr,
+                                  grace::Affine aff = grace::Affine{nullptr, nullptr, nullptr}) {
   using namespace grace;
   if (!x || !w || ((y_bf16 == nullptr) == (y_f32 == nullptr))) return GRACE_INVALID_ARG;
   if (M <= 0 || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
@@ -440,11 +552,13 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
     if (!tc::make_tmap_bf16(&mx, x, 2, dx, sx, bx) || !tc::make_tmap_bf16(&mw, w, 2, dw, sw, bw) ||
         !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
       return GRACE_CUDA_ERROR;
+    if (aff.row != nullptr && (add_into_bf16 || aliased)) return GRACE_INVALID_ARG;
     if (!f32) return add_into_bf16 ? launch_pair<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
-                                   : launch_pair<kOutBf16>(mx, mw, my, M, N, K, relu, s);
-    if (lse_part != nullptr) return launch_pair<kOutF32Lse>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part));
+                                   : launch_pair<kOutBf16>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
+    if (lse_part != nullptr)
+      return launch_pair<kOutF32Lse>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part), aff);
     if (aliased) return launch_pair<kOutF32Add>(mx, mw, my, M, N, K, relu, s);
-    return launch_pair<kOutF32>(mx, mw, my, M, N, K, relu, s);
+    return launch_pair<kOutF32>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
   }
   CUtensorMap mx, mw;
   const int BN = (N >= 128) ? 128 : 64;
@@ -460,6 +574,7 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
   }
   GemmParams p;
   p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.residual_bf16 = add_into_bf16 ? y_bf16 : nullptr;
+  p.aff_row = aff.row; p.aff_cs = aff.cs; p.aff_cb = aff.cb;
   p.ldy = ldy; p.M = M; p.N = N; p.K = K; p.relu = relu;
   return BN == 128 ? launch_linear<128>(mx, mw, p, s) : launch_linear<64>(mx, mw, p, s);
 }
@@ -475,6 +590,18 @@ extern "C" grace_status_t grace_linear_f32_lse(const uint16_t* x, int64_t ldx, c
                                                void* stream) {
   if (!lse_part || (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
   return linear_impl(x, ldx, w, ldw, nullptr, y_f32, ldy, nullptr, false, M, N, K, 0, stream, lse_part);
+}
+
+extern "C" grace_status_t grace_linear_folded_ln(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                                 const float* row_affine, const float* col_sum, const float* col_bias,
+                                                 uint16_t* y_bf16, float* y_f32, int64_t ldy, float* lse_part,
+                                                 int M, int N, int K, int relu, void* stream) {
+  if (!row_affine || !col_bias || (reinterpret_cast<uintptr_t>(row_affine) & 7) ||
+      !grace_aligned16(col_sum) || !grace_aligned16(col_bias))
+    return GRACE_INVALID_ARG;
+  if (lse_part != nullptr && (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
+  grace::Affine aff = {reinterpret_cast<const float2*>(row_affine), col_sum, col_bias};
+  return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, nullptr, false, M, N, K, relu, stream, lse_part, aff);
 }
 
 extern "C" grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,

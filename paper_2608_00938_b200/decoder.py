@@ -33,7 +33,7 @@ class Decoder:
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
                  separate_cand=False, fuse_log_softmax=True, residual_bf16=False, materialize_cand=None,
-                 level_start=None, lse_from_gemm=True):
+                 level_start=None, lse_from_gemm=True, fold_layer_norm=None, centre_stream=None):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -51,12 +51,51 @@ class Decoder:
         s.R_max = R_max
         s.ln_eps = 1e-5
         self.w_kc, self.w_vc, self.k_cross, self.v_cross, self.k_cache, self.v_cache = [], [], [], [], [], []
+        # LayerNorms folded into the GEMMs behind them (bf16 residual stream): the GEMM reads the raw stream, its
+        # weights carry the gain, and its epilogue applies the row statistics (see grace_linear_folded_ln)
+        if fold_layer_norm is None:
+            fold_layer_norm = residual_bf16 and d_model <= 2048
+        assert not fold_layer_norm or residual_bf16
+        self.fold_layer_norm = fold_layer_norm
+        # Centred stream: every consumer of the residual stream is a LayerNorm, which does not see a per-row
+        # shift, so the embedding rows and the projections that add into the stream are centred over the feature
+        # axis once, here; the rows then keep zero mean and the folded GEMMs drop their column-sum term.
+        if centre_stream is None:
+            centre_stream = fold_layer_norm
+        assert not centre_stream or fold_layer_norm
+        self.centre_stream = centre_stream
+
+        def centred_rows(a):                               # [n, d_model]: each row minus its mean
+            a = np.asarray(a, np.float64)
+            return (a - a.mean(axis=1, keepdims=True)).astype(np.float32) if centre_stream else a
+
+        def centred_outputs(w):                            # [d_model, K]: minus the mean over the output index
+            w = np.asarray(w, np.float64)
+            return (w - w.mean(axis=0, keepdims=True)).astype(np.float32) if centre_stream else w
+
+        def fold(w, gamma, beta):
+            """(w * gamma as the bf16 the GEMM will use, column sums of that, beta @ w^T)."""
+            wf = _bf16(np.asarray(w, np.float32) * np.asarray(gamma, np.float32)[None, :], dev)
+            cs = wf.to(torch.float64).sum(dim=1).to(torch.float32).contiguous()
+            cb = torch.from_numpy((np.asarray(w, np.float64) @ np.asarray(beta, np.float64)).astype(np.float32)).to(dev)
+            return wf, cs, cb
+
+        self.folded = []                                   # per layer: {weight name: (folded weight, column sums, bias)}
         for li, lw in enumerate(weights["layers"]):
             lay = s.layers[li]
+            self.folded.append({})
             for name in ("ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b"):
                 t = _f32(lw[name], dev); self._keep.append(t); setattr(lay, name, t.data_ptr())
             for name in ("w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2"):
-                t = _bf16(lw[name], dev); self._keep.append(t); setattr(lay, name, t.data_ptr())
+                t = _bf16(centred_outputs(lw[name]) if name in ("w_o", "w_oc", "w_2") else lw[name], dev)
+                self._keep.append(t); setattr(lay, name, t.data_ptr())
+            if fold_layer_norm:
+                for wname, ln, short in (("w_qkv", "ln1", "qkv"), ("w_qc", "ln2", "qc"), ("w_1", "ln3", "1")):
+                    wf, cs, cb = fold(lw[wname], lw[ln + "_g"], lw[ln + "_b"])
+                    self.folded[li][wname] = (wf, cs, cb)
+                    setattr(lay, wname, wf.data_ptr())
+                    setattr(lay, "cs_" + short, None if centre_stream else cs.data_ptr())
+                    setattr(lay, "cb_" + short, cb.data_ptr())
             self.w_kc.append(_bf16(lw["w_kc"], dev))
             self.w_vc.append(_bf16(lw["w_vc"], dev))
             self.k_cross.append(torch.zeros((B, T_ctx, n_heads, d_head), dtype=torch.bfloat16, device=dev))
@@ -65,10 +104,13 @@ class Decoder:
             self.v_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
             lay.k_cross, lay.v_cross = self.k_cross[li].data_ptr(), self.v_cross[li].data_ptr()
             lay.k_cache, lay.v_cache = self.k_cache[li].data_ptr(), self.v_cache[li].data_ptr()
-        self.embed = _bf16(weights["embed"], dev)
-        self.pos = _bf16(weights["pos"], dev)
+        self.embed = _bf16(centred_rows(weights["embed"]), dev)
+        self.pos = _bf16(centred_rows(weights["pos"]), dev)
         self.lnf_g, self.lnf_b = _f32(weights["lnf_g"], dev), _f32(weights["lnf_b"], dev)
         self.w_out = _bf16(weights["w_out"], dev)
+        if fold_layer_norm:
+            self.w_out, self.cs_out, self.cb_out = fold(weights["w_out"], weights["lnf_g"], weights["lnf_b"])
+            s.cs_out, s.cb_out = None if centre_stream else self.cs_out.data_ptr(), self.cb_out.data_ptr()
         s.embed, s.pos, s.lnf_g, s.lnf_b, s.w_out = (self.embed.data_ptr(), self.pos.data_ptr(),
                                                      self.lnf_g.data_ptr(), self.lnf_b.data_ptr(),
                                                      self.w_out.data_ptr())
@@ -131,6 +173,8 @@ class Decoder:
         self.lse_part = (torch.zeros((R_max, V // 256, 2), dtype=torch.float32, device=dev)
                          if (fuse_log_softmax and lse_from_gemm and V % 256 == 0 and V // 256 <= 32) else None)
         s.lse_part = None if self.lse_part is None else self.lse_part.data_ptr()
+        self.row_affine = torch.zeros((R_max, 2), dtype=torch.float32, device=dev) if fold_layer_norm else None
+        s.row_affine = None if self.row_affine is None else self.row_affine.data_ptr()
         s.topk_ws, s.topk_ws_bytes, s.d_status = self.topk_ws.data_ptr(), ws_bytes, self.d_status.data_ptr()
         self.struct = s
         code = api.grace_decoder_validate(s)

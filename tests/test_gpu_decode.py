@@ -33,6 +33,11 @@ def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=
 
 
 def _make_gpu_decoder(cfg, separate_cand=True, residual_bf16=False):
+    # residual_bf16: False, True (the default bf16 path: LayerNorms folded into the GEMMs over a centred stream),
+    # "uncentred" (folded, column sums carry the row means) or "kernel" (LayerNorm kernels of their own)
+    fold = {"uncentred": dict(fold_layer_norm=True, centre_stream=False),
+            "kernel": dict(fold_layer_norm=False)}.get(residual_bf16, {})
+    residual_bf16 = bool(residual_bf16)
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     shp, sids, trie = cfg["shp"], cfg["sids"], cfg["trie"]
@@ -47,7 +52,7 @@ def _make_gpu_decoder(cfg, separate_cand=True, residual_bf16=False):
                   d_ffn=shp.d_ffn, V=shp.V, L=shp.L, T_ctx=cfg["enc"].shape[1], B=cfg["B"],
                   beam_sizes=list(cfg["schedule"]) + [cfg["final_k"]], weights=cfg["w"], trie_bits=bits,
                   trie_base=base, num_nodes=trie.num_nodes, matcher=matcher, device=DEV, separate_cand=separate_cand,
-                  residual_bf16=residual_bf16)
+                  residual_bf16=residual_bf16, **fold)
     dec.project_cross_kv(torch.from_numpy(cfg["enc"]).to(DEV).to(torch.bfloat16))
     return dec, api
 
@@ -67,6 +72,8 @@ _PAPER_LIKE = dict(shape=(2, 256, 16, 128, 512, 256), T_ctx=128, n_sids=4000)
     (1, "node", (1, 16, 16), 16, False, {}),     # configuration 1
     (3, "bloom", (1, 40, 24), 32, False, {}),    # several requests, dynamic per-step beam sizes, Bloom matcher
     (3, "bloom", (1, 40, 24), 32, True, {}),     # the same with the residual stream held in bf16
+    (3, "bloom", (1, 40, 24), 32, "uncentred", {}),
+    (3, "bloom", (1, 40, 24), 32, "kernel", {}),
     (2, "bloom", (1, 24, 48, 48), 48, True, _PAPER_LIKE),   # dynamic schedule over 4 levels, head size 128
     (2, "node", (1, 100, 80), 80, True, {}),      # step 0 asks for more beams than there are tokens (fixed-schedule shape)
 ])

@@ -708,3 +708,52 @@ def test_mask_kernel_merges_log_sum_exp_partials(api, kind, M):
     want = (score[:, None] + (logits - lse[:, None])).astype(np.float32)
     assert np.array_equal(cand[allowed].view(np.uint32), want[allowed].view(np.uint32))
     assert not allowed[~live].any()
+
+
+@pytest.mark.parametrize("M,N,K,relu,f32out", [(300, 384, 128, False, False), (130, 2048, 512, True, False),
+                                               (2100, 1536, 512, False, False), (1500, 2048, 512, True, False),
+                                               (1100, 512, 512, False, True), (33000, 2048, 512, False, True)])
+@pytest.mark.parametrize("centred", [False, True])
+def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
+    """grace_row_stats_bf16 + grace_linear_folded_ln against LayerNorm(x) @ w^T in fp64: the GEMM reads the raw
+    bf16 stream, its weights carry the gain, the epilogue applies (rstd, -rstd * mean) and the column vectors.
+    centred: the rows of x have zero mean (up to their bf16 rounding) and no column sums are passed."""
+    rng = synth.rng_for(5, 17 * M + N + K)
+    x = synth.normal_bf16(rng, (M, K), 1.5)
+    if centred:
+        xc = synth.bf16_bits_to_f32(x).astype(np.float64)
+        x = synth.f32_to_bf16_bits((xc - xc.mean(1, keepdims=True)).astype(np.float32))
+    else:                                   # a mean the column-sum term has to carry
+        x = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(x) + np.float32(0.75))
+    x64 = f64(x) + 0.0
+    w = synth.normal_bf16(rng, (N, K), 0.05)
+    g = (synth.normal_f32(rng, K) * 0.2 + 1.0).astype(np.float32)
+    b = (synth.normal_f32(rng, K) * 0.3).astype(np.float32)
+    ln = (x64 - x64.mean(1, keepdims=True)) / np.sqrt(x64.var(1, keepdims=True) + 1e-5) * g + b
+    ref = ln @ f64(w).T
+    if relu:
+        ref = np.maximum(ref, 0)
+    wf_bits = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(w) * g[None, :])
+    cs = f64(wf_bits).sum(1).astype(np.float32)
+    cb = (f64(w) @ b.astype(np.float64)).astype(np.float32)
+    aff = torch.zeros((M, 2), device=DEV)
+    api.grace_row_stats_bf16(dev_bf16(x), aff, 1e-5)
+    torch.cuda.synchronize()
+    a = aff.cpu().numpy().astype(np.float64)
+    rstd = 1.0 / np.sqrt(x64.var(1) + 1e-5)
+    np.testing.assert_allclose(a[:, 0], rstd, rtol=2e-6)
+    np.testing.assert_allclose(a[:, 1], -rstd * x64.mean(1), rtol=0, atol=2e-6 * (1 + np.abs(rstd * x64.mean(1)).max()))
+    y = torch.zeros((M, N), dtype=torch.float32 if f32out else torch.bfloat16, device=DEV)
+    part = torch.zeros((M, N // 256, 2), device=DEV) if (f32out and M >= 1024 and N % 256 == 0) else None
+    api.grace_linear_folded_ln(dev_bf16(x), dev_bf16(wf_bits), aff, None if centred else dev(cs), dev(cb), y, relu, part)
+    torch.cuda.synchronize()
+    got = y.float().cpu().numpy().astype(np.float64)
+    # folding rounds w * gamma to bf16 once (2^-9 relative per weight, averaging out over K terms)
+    tol = 1.2e-2 if f32out else 2e-2
+    assert np.abs(got - ref).max() <= tol * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
+    assert np.sqrt(((got - ref) ** 2).sum() / (ref ** 2).sum()) <= 5e-3
+    if part is not None:
+        p = part.cpu().numpy().astype(np.float64)
+        lse = p[:, :, 0].max(1) + np.log((p[:, :, 1] * np.exp(p[:, :, 0] - p[:, :, 0].max(1, keepdims=True))).sum(1))
+        want = np.log(np.exp(got - got.max(1, keepdims=True)).sum(1)) + got.max(1)
+        np.testing.assert_allclose(lse, want, atol=1e-5, rtol=0)
