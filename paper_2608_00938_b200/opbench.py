@@ -31,7 +31,7 @@ def _time(fn, iters, warm=2):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "mask", "lookup", "layer_norm", "log_softmax"])
+    ap.add_argument("op", choices=["linear", "cross_attn", "self_attn", "topk", "mask", "lookup", "layer_norm", "log_softmax", "row_stats"])
     for name, default in (("B", 32), ("M", 2048), ("N", 2048), ("K", 512), ("T", 1024), ("H", 8), ("d", 64),
                           ("V", 1024), ("t", 3), ("iters", 5)):
         ap.add_argument(f"--{name}", type=int, default=default)
@@ -44,6 +44,8 @@ def main():
     ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
     ap.add_argument("--kway", type=int, default=1, help="lookup: static k-way partitioned rows with this k at every level")
     ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
+    ap.add_argument("--folded", action="store_true",
+                    help="linear: LayerNorm folded into the epilogue (row pair + column bias; centred rows)")
     a = ap.parse_args()
     dev = "cuda:0"
     torch.manual_seed(0)
@@ -52,11 +54,24 @@ def main():
         x, w = bf(a.M, a.K), bf(a.N, a.K) * 0.05
         y = torch.zeros(a.M, a.N, device=dev, dtype=torch.float32 if (a.f32out or a.residual) and not a.bf16stream
                         else torch.bfloat16)
-        if a.bf16stream:
+        if a.folded:
+            aff, cb = torch.ones(a.M, 2, device=dev), torch.zeros(a.N, device=dev)
+            us = _time(lambda: api.grace_linear_folded_ln(x, w, aff, None, cb, y, a.relu), a.iters)
+        elif a.bf16stream:
             us = _time(lambda: api.grace_linear_add_bf16(x, w, y), a.iters)
         else:
             us = _time(lambda: api.grace_linear(x, w, y, y if a.residual else None, a.relu), a.iters)
         print(f"linear M={a.M} N={a.N} K={a.K}: {us:.1f} us, {2.0 * a.M * a.N * a.K / us / 1e6:.1f} TFLOP/s")
+    elif a.op == "row_stats":
+        R = a.B * a.M
+        xs = [bf(R, a.K) for _ in range(3)]                # rotated: 3 x R x K x 2 bytes, larger than L2 at R = 65536
+        aff = torch.zeros(R, 2, device=dev)
+        i = [0]
+        def run():
+            i[0] += 1
+            api.grace_row_stats_bf16(xs[i[0] % 3], aff)
+        us = _time(run, a.iters)
+        print(f"row_stats R={R} D={a.K}: {us:.1f} us, {R * (a.K * 2 + 8) / us / 1e3:.0f} GB/s")
     elif a.op == "cross_attn":
         q, k, v = bf(a.B * a.M, a.H, a.d), bf(a.B, a.H, a.T, a.d), bf(a.B, a.H, a.T, a.d)
         o = torch.empty_like(q)
