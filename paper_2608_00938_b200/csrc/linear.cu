@@ -365,11 +365,6 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
           const float4 c = aff_s[(col0 + i) >> 1];
-#ifdef GRACE_FOLD_SCALAR
-          r[i] = __float_as_uint(fmaf(ar.x, __uint_as_float(r[i]), fmaf(ar.y, c.x, c.z)));
-          r[i + 1] = __float_as_uint(fmaf(ar.x, __uint_as_float(r[i + 1]), fmaf(ar.y, c.y, c.w)));
-          continue;
-#endif
           const f32x2_t v = f2_fma(ar_x, f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])),
                                    f2_fma(ar_y, f2_pack(c.x, c.y), f2_pack(c.z, c.w)));
           float lo, hi;
