@@ -85,7 +85,8 @@ def make_inputs(cfg, variant=0):
     return dict(sids=sids, elig=elig, shp=shp, weights=weights, enc_bits=enc_bits)
 
 
-def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, fold_layer_norm=None):
+def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, fold_layer_norm=None,
+                  persist_stream_l2=None):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -98,7 +99,7 @@ def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, 
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
                   residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand,
-                  fold_layer_norm=fold_layer_norm)
+                  fold_layer_norm=fold_layer_norm, persist_stream_l2=persist_stream_l2)
     return dec
 
 
@@ -196,6 +197,7 @@ def time_decode_graph(dec, steps, warmup):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
+        dec.prepare_stream()                     # stream attributes (L2 residency of the residual stream) before capture
         with torch.cuda.graph(graph, stream=side):
             dec.reset(); dec.decode()
     torch.cuda.current_stream().wait_stream(side)
@@ -507,6 +509,8 @@ def main():
                     help="beam sizes per step, e.g. 1,512,1024,1024 (dynamic beam schedule, Section 3.3)")
     ap.add_argument("--residual", default="bf16", choices=["bf16", "f32"],
                     help="dtype of the residual stream between blocks (weights, activations and caches are bf16 either way)")
+    ap.add_argument("--l2-persist", default="on", choices=["on", "off"],
+                    help="keep the residual stream resident in L2 (access-policy window on the stream)")
     ap.add_argument("--layer-norm", default="folded", choices=["folded", "kernel"],
                     help="LayerNorms folded into the GEMMs behind them (bf16 stream), or run as kernels of their own")
     args = ap.parse_args()
@@ -539,7 +543,8 @@ def main():
     default_workload = (args.workload == "cfg5" and not args.schedule)
     inp = make_inputs(cfg, variant=rank)
     dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"),
-                        fold_layer_norm=(None if args.layer_norm == "folded" else False))
+                        fold_layer_norm=(None if args.layer_norm == "folded" else False),
+                        persist_stream_l2=(None if args.l2_persist == "on" else False))
     dec._layer_tensors = _layer_tensor_views(dec, inp)
     enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
     dec.project_cross_kv(enc_dev)

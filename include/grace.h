@@ -62,6 +62,16 @@ int grace_built_for_sm(void);
 int grace_wait_timeouts(void);
 grace_status_t grace_selftest_bounded_wait(void* stream);
 
+/* Asks the device to keep `fraction` (0 < fraction <= 1) of the lines of [ptr, ptr + bytes) resident in L2 for
+ * the kernels launched on `stream` from now on: an access-policy window on the stream (hit ratio = fraction,
+ * other lines of the window cached normally), backed by this context's persisting-L2 carve-out, both clipped
+ * to the device's limits.  Meant for the residual stream of the decoder, which every block of a step re-reads
+ * several times while far larger tensors stream past it; keeping all of a buffer half the size of the L2
+ * starves everything else (measured: slower), half of it pays.  ptr NULL or bytes 0 clears the window.
+ * Host call; nothing is enqueued; the setting belongs to this process's context and ends with it.
+ * GRACE_UNSUPPORTED_SHAPE if the device has no persisting L2. */
+grace_status_t grace_stream_l2_persist(void* stream, const void* ptr, size_t bytes, float fraction);
+
 /* Number of kernels this library has launched in this process so far (all entry points). */
 uint64_t grace_kernel_launch_count(void);
 

@@ -113,6 +113,7 @@ _row_stats_bf16 = _sig("grace_row_stats_bf16", _i32, [_vp, _i32, _i32, _f32, _vp
 _linear_folded_ln = _sig("grace_linear_folded_ln", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
                                                          _i32, _i32, _i32, _i32, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
+_stream_l2_persist = _sig("grace_stream_l2_persist", _i32, [_vp, _vp, C.c_size_t, C.c_float])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
 _gtm_lookup = _sig("grace_gtm_lookup", _i32, [_vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp, _i32, _i32, _vp, _vp])
 _beam_update_csr = _sig("grace_beam_update_csr", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(GtmIndexStruct), _vp, _vp,
@@ -348,6 +349,16 @@ def grace_linear_folded_ln(x, w_folded, row_affine, col_sum, col_bias, y, relu: 
                              _dp(col_sum), _dp(col_bias), None if f32 else _dp(y), _dp(y) if f32 else None, y.stride(0),
                              _dp(lse_part), M, N, K, int(relu), _stream()), "grace_linear_folded_ln")
     return y
+
+
+def grace_stream_l2_persist(t=None, fraction: float = 0.5) -> None:
+    """Keep `fraction` of tensor `t` resident in L2 for kernels launched on the current stream from now on
+    (None clears the window)."""
+    if t is None:
+        _check(_stream_l2_persist(_stream(), None, 0, 0.0), "grace_stream_l2_persist")
+    else:
+        _check(_stream_l2_persist(_stream(), t.data_ptr(), t.numel() * t.element_size(), fraction),
+               "grace_stream_l2_persist")
 
 
 def grace_wait_timeouts() -> int:

@@ -166,3 +166,35 @@ extern "C" int grace_wait_timeouts(void) {
   const int a = grace::linear_tc_timeouts(), b = grace::cross_attn_tc_timeouts();
   return (a < 0 || b < 0) ? -1 : a + b;
 }
+
+// Keeps part of a buffer that many kernels of a step re-read (the residual stream: three add-reductions,
+// three statistics passes and three GEMM operand reads per layer) resident in L2 across the large tensors
+// that stream past it: an access-policy window on the stream, backed by this context's persisting carve-out.
+extern "C" grace_status_t grace_stream_l2_persist(void* stream, const void* ptr, size_t bytes, float fraction) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaStreamAttrValue v;
+  memset(&v, 0, sizeof(v));
+  if (ptr == nullptr || bytes == 0) {                       // clear the window
+    v.accessPolicyWindow.hitProp = cudaAccessPropertyNormal;
+    v.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
+    GRACE_CUDA_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
+    return GRACE_OK;
+  }
+  if (!(fraction > 0.f && fraction <= 1.f)) return GRACE_INVALID_ARG;
+  int dev = 0, max_persist = 0, max_window = 0;
+  GRACE_CUDA_TRY(cudaGetDevice(&dev));
+  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev));
+  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev));
+  if (max_persist <= 0 || max_window <= 0) return GRACE_UNSUPPORTED_SHAPE;
+  const size_t window = bytes < (size_t)max_window ? bytes : (size_t)max_window;
+  size_t carve = (size_t)((double)window * fraction);
+  if (carve > (size_t)max_persist) carve = (size_t)max_persist;
+  GRACE_CUDA_TRY(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve));
+  v.accessPolicyWindow.base_ptr = const_cast<void*>(ptr);
+  v.accessPolicyWindow.num_bytes = window;
+  v.accessPolicyWindow.hitRatio = (float)((double)carve / (double)window);   // the share of the window's lines kept
+  v.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+  v.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
+  GRACE_CUDA_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
+  return GRACE_OK;
+}

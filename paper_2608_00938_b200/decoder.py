@@ -33,7 +33,8 @@ class Decoder:
     def __init__(self, *, n_layers, d_model, n_heads, d_head, d_ffn, V, L, T_ctx, B, beam_sizes, weights,
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
                  separate_cand=False, fuse_log_softmax=True, residual_bf16=False, materialize_cand=None,
-                 level_start=None, lse_from_gemm=True, fold_layer_norm=None, centre_stream=None):
+                 level_start=None, lse_from_gemm=True, fold_layer_norm=None, centre_stream=None,
+                 persist_stream_l2=None):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -149,6 +150,11 @@ class Decoder:
         self.topk_ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
         self.d_status = torch.zeros(1, dtype=torch.int32, device=dev)
         s.x, s.x_bf16 = (None, self.x.data_ptr()) if residual_bf16 else (self.x.data_ptr(), None)
+        # the bf16 stream of the large configurations (tens of MB) fits the persisting part of the L2
+        if persist_stream_l2 is None:
+            persist_stream_l2 = residual_bf16 and self.x.numel() * 2 >= (8 << 20)
+        self.persist_stream_l2 = persist_stream_l2
+        self._prepared_streams = set()
         s.h, s.qkv, s.attn, s.logp, s.cand = (self.h.data_ptr(), self.qkv.data_ptr(),
                                                    self.attn.data_ptr(), self.logp.data_ptr(), self.cand.data_ptr())
         s.row_lse = None if self.row_lse is None else self.row_lse.data_ptr()
@@ -194,7 +200,17 @@ class Decoder:
         """Start state (Section 3.3: M_0 = 1): start token, score 0, root node, empty key."""
         api.grace_decode_begin(self.struct)
 
+    def prepare_stream(self) -> None:
+        """Once per CUDA stream the decoder is used on (before any graph capture on it): asks for the residual
+        stream to stay resident in L2 (it is re-read nine times per layer while larger tensors stream past)."""
+        sid = torch.cuda.current_stream(self.device).cuda_stream
+        if self.persist_stream_l2 and sid not in self._prepared_streams:
+            api.grace_stream_l2_persist(self.x)
+            self._prepared_streams.add(sid)
+
     def step(self, t: int) -> None:
+        if self.persist_stream_l2 and not torch.cuda.is_current_stream_capturing():
+            self.prepare_stream()
         api.grace_decode_step(self.struct, t)
 
     def decode(self) -> None:

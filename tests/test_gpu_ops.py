@@ -757,3 +757,31 @@ def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
         lse = p[:, :, 0].max(1) + np.log((p[:, :, 1] * np.exp(p[:, :, 0] - p[:, :, 0].max(1, keepdims=True))).sum(1))
         want = np.log(np.exp(got - got.max(1, keepdims=True)).sum(1)) + got.max(1)
         np.testing.assert_allclose(lse, want, atol=1e-5, rtol=0)
+
+
+def test_l2_residency_window_is_a_hint_only(api):
+    """grace_stream_l2_persist changes where lines live, never what a kernel computes: the same GEMM into the
+    same residual stream gives the same bits with the window set, with it cleared, and on another stream."""
+    rng = synth.rng_for(5, 4242)
+    M, N, K = 4096, 512, 512
+    x, w = dev_bf16(synth.normal_bf16(rng, (M, K))), dev_bf16(synth.normal_bf16(rng, (N, K), 0.05))
+    base = dev_bf16(synth.normal_bf16(rng, (M, N)))
+    outs = []
+    for mode in ("plain", "window", "cleared"):
+        y = base.clone()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            if mode == "window":
+                api.grace_stream_l2_persist(y, 0.5)
+            elif mode == "cleared":
+                api.grace_stream_l2_persist(y, 1.0)
+                api.grace_stream_l2_persist(None)
+            api.grace_linear_add_bf16(x, w, y)
+        side.synchronize()
+        outs.append(y)
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    with pytest.raises(Exception):
+        api.grace_stream_l2_persist(base, 0.0)
+    with pytest.raises(Exception):
+        api.grace_stream_l2_persist(base, 1.5)
