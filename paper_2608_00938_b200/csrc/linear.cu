@@ -22,14 +22,15 @@ __device__ __forceinline__ float fast_ex2(float x) {
 
 constexpr int kGemmBM = 128;
 constexpr int kGemmBK = 64;
-constexpr int kGemmStages = 3;
 
-template <int BN>
+// STAGES = 3: throughput form (several CTAs per SM).  STAGES = 8 with BN = 64: latency form for launches whose grid
+// does not fill the GPU (step 0 of a decode: 32 rows): the whole K = 512 of a tile is in flight at once.
+template <int BN, int STAGES>
 struct GemmSmem {
   static constexpr int kABytes = kGemmBM * kGemmBK * 2;
   static constexpr int kBBytes = BN * kGemmBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kTotal = kGemmStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kTotal = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct GemmParams {
@@ -45,13 +46,16 @@ struct GemmParams {
   int M, N, K, relu;
 };
 
-template <int BN>
+template <int BN, int STAGES>
 __global__ void __launch_bounds__(128)
 linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const GemmParams p) {
-  pdl_wait();
+  // The weights do not depend on the kernel before this one: their first tiles are requested before the wait
+  // on that kernel, so their trip from HBM overlaps its tail; every thread waits before its first access to
+  // anything an earlier kernel wrote (activations, row statistics, the residual).
   pdl_trigger();
-  using S = GemmSmem<BN>;
+  constexpr int kGemmStages = STAGES;
+  using S = GemmSmem<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(tiles + kGemmStages * S::kStageBytes);
@@ -80,7 +84,15 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----
-    for (int kb = 0; kb < KB; ++kb) {
+    const int first = KB < kGemmStages ? KB : kGemmStages;  // the ring's first pass needs no empty-slot wait
+    for (int kb = 0; kb < first; ++kb) {
+      tc::mbar_expect_tx(full + kb, S::kStageBytes);
+      tc::tma_load_2d(tiles + kb * S::kStageBytes + S::kABytes, &map_w, full + kb, kb * kGemmBK, n0);
+    }
+    pdl_wait();
+    for (int kb = 0; kb < first; ++kb)
+      tc::tma_load_2d(tiles + kb * S::kStageBytes, &map_x, full + kb, kb * kGemmBK, m0);
+    for (int kb = first; kb < KB; ++kb) {
       const int s = kb % kGemmStages;
       if (!tc::mbar_wait(empty + s, ((kb / kGemmStages) & 1) ^ 1, abort_flag)) break;
       tc::mbar_expect_tx(full + s, S::kStageBytes);
@@ -106,6 +118,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     tc::mma_commit(accum_bar);
   }
   __syncwarp();
+  pdl_wait();
 
   // ---- epilogue: warp w owns TMEM lanes 32w .. 32w+31 = rows m0 + 32w + lane ----
   // Folded LayerNorm: the row's pair and the column vectors of a chunk are fetched (from clamped addresses,
@@ -504,14 +517,15 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   return GRACE_OK;
 }
 
-template <int BN>
+template <int BN, int STAGES>
 static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw, const GemmParams& p, cudaStream_t s) {
   static unsigned long long attr_set_devices = 0;
   if (first_use_on_device(&attr_set_devices)) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmSmem<BN>::kTotal));
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        GemmSmem<BN, STAGES>::kTotal));
   }
   dim3 grid((p.N + BN - 1) / BN, (p.M + kGemmBM - 1) / kGemmBM);
-  launch_pdl(linear_kernel<BN>, grid, dim3(128), GemmSmem<BN>::kTotal, s, mx, mw, p);
+  launch_pdl(linear_kernel<BN, STAGES>, grid, dim3(128), GemmSmem<BN, STAGES>::kTotal, s, mx, mw, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -556,7 +570,9 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
     return launch_pair<kOutF32>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
   }
   CUtensorMap mx, mw;
-  const int BN = (N >= 128) ? 128 : 64;
+  // a grid that leaves most SMs idle is latency-bound: narrower tiles (more CTAs) and the whole K in flight
+  const bool latency_form = (int64_t)((M + kGemmBM - 1) / kGemmBM) * ((N + 127) / 128) < 74;
+  const int BN = (N >= 128 && !latency_form) ? 128 : 64;
   {
     const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M}, str[1] = {(uint64_t)ldx};
     const uint32_t box[2] = {(uint32_t)kGemmBK, (uint32_t)kGemmBM};
@@ -571,7 +587,8 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
   p.y_bf16 = y_bf16; p.y_f32 = y_f32; p.residual = residual; p.residual_bf16 = add_into_bf16 ? y_bf16 : nullptr;
   p.aff_row = aff.row; p.aff_cs = aff.cs; p.aff_cb = aff.cb;
   p.ldy = ldy; p.M = M; p.N = N; p.K = K; p.relu = relu;
-  return BN == 128 ? launch_linear<128>(mx, mw, p, s) : launch_linear<64>(mx, mw, p, s);
+  if (BN == 128) return launch_linear<128, 3>(mx, mw, p, s);
+  return latency_form ? launch_linear<64, 8>(mx, mw, p, s) : launch_linear<64, 3>(mx, mw, p, s);
 }
 
 extern "C" grace_status_t grace_linear(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
