@@ -86,7 +86,7 @@ def make_inputs(cfg, variant=0):
 
 
 def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, fold_layer_norm=None,
-                  persist_stream_l2=None):
+                  persist_stream_l2=None, kv_in_place=True):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -99,7 +99,7 @@ def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, 
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
                   residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand,
-                  fold_layer_norm=fold_layer_norm, persist_stream_l2=persist_stream_l2)
+                  fold_layer_norm=fold_layer_norm, persist_stream_l2=persist_stream_l2, kv_in_place=kv_in_place)
     return dec
 
 
@@ -294,10 +294,16 @@ def op_breakdown(dec, cfg, reps=3):
                 q1 = qkv.view(-1)[:R * HD].view(R, HD)
                 ff = qkv.view(-1)[:R * F].view(R, F)
                 fo = dec.folded[li] if folded else {}
+                if dec.kv_in_place:                  # the projection lands in the cache slab of this step
+                    q3 = dec.qkv_slabs[li][t].view(-1)[:R * 3 * HD].view(R, 3 * HD)
                 ln_linear(x, lay["ln1_g"], lay["ln1_b"], hD, lay["w_qkv"], fo.get("w_qkv"), q3, 2.0 * R * D * 3 * HD)
-                timed("self_attn", lambda: api.grace_self_attn(q3.view(R, 3, H, dh), dec.k_cache[li], dec.v_cache[li],
-                                                               dec.parents, sizes, attn.view(R, H, dh), B, t, scale,
-                                                               dec.d_status))
+                if dec.kv_in_place:
+                    timed("self_attn", lambda: api.grace_self_attn_inplace(dec.qkv_slabs[li], dec.parents, sizes,
+                                                                           attn.view(R, H, dh), B, t, scale, dec.d_status))
+                else:
+                    timed("self_attn", lambda: api.grace_self_attn(q3.view(R, 3, H, dh), dec.k_cache[li], dec.v_cache[li],
+                                                                   dec.parents, sizes, attn.view(R, H, dh), B, t, scale,
+                                                                   dec.d_status))
                 timed("linear", lambda: add_into_x(attn, lay["w_o"], x), 2.0 * R * HD * D)
                 ln_linear(x, lay["ln2_g"], lay["ln2_b"], hD, lay["w_qc"], fo.get("w_qc"), q1, 2.0 * R * D * HD)
                 timed("cross_attn", lambda: api.grace_cross_attn(
@@ -509,6 +515,8 @@ def main():
                     help="beam sizes per step, e.g. 1,512,1024,1024 (dynamic beam schedule, Section 3.3)")
     ap.add_argument("--residual", default="bf16", choices=["bf16", "f32"],
                     help="dtype of the residual stream between blocks (weights, activations and caches are bf16 either way)")
+    ap.add_argument("--kv-cache", default="inplace", choices=["inplace", "copy"],
+                    help="self-attention cache: the steps' QKV projections kept in place, or separate K/V slabs written per step")
     ap.add_argument("--l2-persist", default="on", choices=["on", "off"],
                     help="keep the residual stream resident in L2 (access-policy window on the stream)")
     ap.add_argument("--layer-norm", default="folded", choices=["folded", "kernel"],
@@ -544,7 +552,8 @@ def main():
     inp = make_inputs(cfg, variant=rank)
     dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"),
                         fold_layer_norm=(None if args.layer_norm == "folded" else False),
-                        persist_stream_l2=(None if args.l2_persist == "on" else False))
+                        persist_stream_l2=(None if args.l2_persist == "on" else False),
+                        kv_in_place=(args.kv_cache == "inplace"))
     dec._layer_tensors = _layer_tensor_views(dec, inp)
     enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
     dec.project_cross_kv(enc_dev)

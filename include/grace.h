@@ -179,6 +179,16 @@ grace_status_t grace_self_attn(const uint16_t* qkv, int64_t qkv_row_stride,
                                uint16_t* out, int64_t out_row_stride,
                                int B, int t, int H, int d_h, int64_t R_max, float scale,
                                int32_t* d_status, void* stream);
+/* The same with the cache held in place: qkv_slabs is device bf16 [L_cache][R_max][3][H][d_h] (row stride
+ * row_stride >= 3*H*d_h elements, slab stride slab_stride >= R_max*row_stride elements), slab j being the QKV
+ * projection of step j exactly as the GEMM left it.  Slab t is this step's input; the K and V thirds of slabs
+ * 0..t are the cache, so nothing is copied and the kernel writes only `out` (Section 5.3 removes the reorder
+ * copy; this also removes the append copy).  Other arguments, limits and errors as grace_self_attn. */
+grace_status_t grace_self_attn_inplace(uint16_t* qkv_slabs, int64_t row_stride, int64_t slab_stride,
+                                       const int32_t* parents, const int32_t* beam_sizes,
+                                       uint16_t* out, int64_t out_row_stride,
+                                       int B, int t, int H, int d_h, int64_t R_max, float scale,
+                                       int32_t* d_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * CD + GTM mask and score add (Sections 3.1, 4.1; kernel role of Section 5.4).
@@ -435,11 +445,14 @@ typedef struct {
   const uint16_t *w_2;     /* [d_model][d_ffn] */
   const uint16_t *k_cross, *v_cross;   /* [B][T_ctx][H][d_h]: as the once-per-request projection
                                           GEMM of the encoder output writes them (Section 3.2) */
-  uint16_t *k_cache, *v_cache;         /* [L][R_max][H][d_h] */
+  uint16_t *k_cache, *v_cache;         /* [L][R_max][H][d_h]; unused (may be NULL) when qkv_slabs is set */
   /* With grace_decoder_t.ln_folded: w_qkv, w_qc, w_1 already carry the gain of the LayerNorm in front of
    * them (w[n][k] * gamma[k], rounded to bf16) and these hold, per output feature n, the sum over k of that
    * matrix (cs_*) and the sum over k of beta[k] * (unfolded) w[n][k] (cb_*), fp32 [out_features]. */
   const float *cs_qkv, *cb_qkv, *cs_qc, *cb_qc, *cs_1, *cb_1;
+  /* NULL, or [L][R_max][3*H*d_h]: the QKV projection of step t is written into slab t and kept, and the
+   * self-attention reads its cache from the K and V thirds of the slabs (grace_self_attn_inplace). */
+  uint16_t *qkv_slabs;
 } grace_layer_t;
 
 #define GRACE_MAX_LAYERS 16

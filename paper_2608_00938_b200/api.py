@@ -52,7 +52,7 @@ class LayerStruct(C.Structure):
         "ln1_g", "ln1_b", "ln2_g", "ln2_b", "ln3_g", "ln3_b",
         "w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2",
         "k_cross", "v_cross", "k_cache", "v_cache",
-        "cs_qkv", "cb_qkv", "cs_qc", "cb_qc", "cs_1", "cb_1")]
+        "cs_qkv", "cb_qkv", "cs_qc", "cb_qc", "cs_1", "cb_1", "qkv_slabs")]
 
 
 class DecoderStruct(C.Structure):
@@ -94,6 +94,8 @@ _cross_attn = _sig("grace_cross_attn", _i32, [_vp, _i64, _vp, _vp, _i64, _i64, _
                                              _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp])
 _self_attn = _sig("grace_self_attn", _i32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64,
                                            _i32, _i32, _i32, _i32, _i64, _f32, _vp, _vp])
+_self_attn_inplace = _sig("grace_self_attn_inplace", _i32, [_vp, _i64, _i64, _vp, _vp, _vp, _i64,
+                                                           _i32, _i32, _i32, _i32, _i64, _f32, _vp, _vp])
 _gtm_mask = _sig("grace_gtm_mask", _i32, [_vp, _vp, _vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct),
                                          _vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp])
 _gtm_mask_logits = _sig("grace_gtm_mask_logits", _i32, [_vp, _vp, _vp, _vp, _vp, C.POINTER(TrieStruct),
@@ -421,6 +423,17 @@ def grace_self_attn(qkv, k_cache, v_cache, parents, beam_sizes, out, B: int, t: 
     _check(_self_attn(_dp(qkv), qkv.stride(0), _dp(k_cache), _dp(v_cache), _dp(parents), bs.ctypes.data,
                       _dp(out), out.stride(0), B, t, H, d, k_cache.shape[1], scale, _dp(d_status), _stream()),
            "grace_self_attn")
+    return out
+
+
+def grace_self_attn_inplace(qkv_slabs, parents, beam_sizes, out, B: int, t: int, scale: float, d_status=None):
+    """qkv_slabs [L, R_max, 3, H, d]: slab j is the QKV projection of step j and, in its K and V thirds, the
+    cache; parents int32 [L, R_max]; out [R, H, d].  Nothing but `out` is written."""
+    L, R_max, three, H, d = qkv_slabs.shape
+    bs = np.ascontiguousarray(beam_sizes[: t + 1], dtype=np.int32)
+    _check(_self_attn_inplace(_dp(qkv_slabs), qkv_slabs.stride(1), qkv_slabs.stride(0), _dp(parents), bs.ctypes.data,
+                              _dp(out), out.stride(0), B, t, H, d, R_max, scale, _dp(d_status), _stream()),
+           "grace_self_attn_inplace")
     return out
 
 

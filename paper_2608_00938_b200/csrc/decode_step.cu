@@ -23,7 +23,7 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
   for (int l = 0; l < d->n_layers; ++l) {
     const grace_layer_t& w = d->layers[l];
     if (!w.ln1_g || !w.ln1_b || !w.ln2_g || !w.ln2_b || !w.ln3_g || !w.ln3_b || !w.w_qkv || !w.w_o || !w.w_qc ||
-        !w.w_oc || !w.w_1 || !w.w_2 || !w.k_cross || !w.v_cross || !w.k_cache || !w.v_cache)
+        !w.w_oc || !w.w_1 || !w.w_2 || !w.k_cross || !w.v_cross || (!w.qkv_slabs && (!w.k_cache || !w.v_cache)))
       return GRACE_INVALID_ARG;
   }
   if (!d->embed || !d->pos || !d->lnf_g || !d->lnf_b || !d->w_out || !d->parents || (!d->x && !d->x_bf16) || !d->h || !d->qkv ||
@@ -108,9 +108,17 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   for (int l = 0; l < d->n_layers; ++l) {
     const grace_layer_t& w = d->layers[l];
     // self-attention block
-    GRACE_TRY(ln_linear(w.ln1_g, w.ln1_b, w.w_qkv, w.cs_qkv, w.cb_qkv, d->qkv, nullptr, 3 * HD, 3 * HD, 0, nullptr));
-    GRACE_TRY(grace_self_attn(d->qkv, 3 * HD, w.k_cache, w.v_cache, d->parents, d->beam_sizes, d->attn, HD,
-                              B, t, d->H, d->d_h, d->R_max, scale, st, stream));
+    if (w.qkv_slabs != nullptr) {                          // the projection lands in the cache slab of this step
+      const int64_t slab = d->R_max * 3 * (int64_t)HD;
+      GRACE_TRY(ln_linear(w.ln1_g, w.ln1_b, w.w_qkv, w.cs_qkv, w.cb_qkv, w.qkv_slabs + t * slab, nullptr, 3 * HD, 3 * HD,
+                          0, nullptr));
+      GRACE_TRY(grace_self_attn_inplace(w.qkv_slabs, 3 * HD, slab, d->parents, d->beam_sizes, d->attn, HD, B, t,
+                                        d->H, d->d_h, d->R_max, scale, st, stream));
+    } else {
+      GRACE_TRY(ln_linear(w.ln1_g, w.ln1_b, w.w_qkv, w.cs_qkv, w.cb_qkv, d->qkv, nullptr, 3 * HD, 3 * HD, 0, nullptr));
+      GRACE_TRY(grace_self_attn(d->qkv, 3 * HD, w.k_cache, w.v_cache, d->parents, d->beam_sizes, d->attn, HD,
+                                B, t, d->H, d->d_h, d->R_max, scale, st, stream));
+    }
     GRACE_TRY(add_into_x(d->attn, HD, w.w_o, HD));
     // cross-attention block
     GRACE_TRY(ln_linear(w.ln2_g, w.ln2_b, w.w_qc, w.cs_qc, w.cb_qc, d->qkv, nullptr, HD, HD, 0, nullptr));

@@ -34,7 +34,7 @@ class Decoder:
                  trie_bits, trie_base, num_nodes, matcher=(api.MATCH_NONE, None, 0, 0), device="cuda:0",
                  separate_cand=False, fuse_log_softmax=True, residual_bf16=False, materialize_cand=None,
                  level_start=None, lse_from_gemm=True, fold_layer_norm=None, centre_stream=None,
-                 persist_stream_l2=None):
+                 persist_stream_l2=None, kv_in_place=True):
         assert len(beam_sizes) == L + 1
         self.device = torch.device(device)
         self.B, self.L, self.V, self.H, self.d_h, self.T_ctx = B, L, V, n_heads, d_head, T_ctx
@@ -52,6 +52,7 @@ class Decoder:
         s.R_max = R_max
         s.ln_eps = 1e-5
         self.w_kc, self.w_vc, self.k_cross, self.v_cross, self.k_cache, self.v_cache = [], [], [], [], [], []
+        self.kv_in_place, self.qkv_slabs = kv_in_place, []
         # LayerNorms folded into the GEMMs behind them (bf16 residual stream): the GEMM reads the raw stream, its
         # weights carry the gain, and its epilogue applies the row statistics (see grace_linear_folded_ln)
         if fold_layer_norm is None:
@@ -101,10 +102,15 @@ class Decoder:
             self.w_vc.append(_bf16(lw["w_vc"], dev))
             self.k_cross.append(torch.zeros((B, T_ctx, n_heads, d_head), dtype=torch.bfloat16, device=dev))
             self.v_cross.append(torch.zeros((B, T_ctx, n_heads, d_head), dtype=torch.bfloat16, device=dev))
-            self.k_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
-            self.v_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
             lay.k_cross, lay.v_cross = self.k_cross[li].data_ptr(), self.v_cross[li].data_ptr()
-            lay.k_cache, lay.v_cache = self.k_cache[li].data_ptr(), self.v_cache[li].data_ptr()
+            if kv_in_place:
+                # the cache is the steps' own QKV projections, kept: nothing is copied into a cache
+                self.qkv_slabs.append(torch.zeros((L, R_max, 3, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+                lay.qkv_slabs = self.qkv_slabs[li].data_ptr()
+            else:
+                self.k_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+                self.v_cache.append(torch.zeros((L, R_max, n_heads, d_head), dtype=torch.bfloat16, device=dev))
+                lay.k_cache, lay.v_cache = self.k_cache[li].data_ptr(), self.v_cache[li].data_ptr()
         self.embed = _bf16(centred_rows(weights["embed"]), dev)
         self.pos = _bf16(centred_rows(weights["pos"]), dev)
         self.lnf_g, self.lnf_b = _f32(weights["lnf_g"], dev), _f32(weights["lnf_b"], dev)

@@ -464,6 +464,35 @@ def test_self_attn_matches_oracle(api, B, beam_sizes, H, d):
     assert np.array_equal(d_vc.view(torch.int16).cpu().numpy().view(np.uint16), vc_exp)
 
 
+@pytest.mark.parametrize("B,beam_sizes,H,d", [
+    (3, [1], 8, 64), (2, [1, 50, 70], 8, 64), (2, [1, 64, 64, 130], 8, 64), (2, [5, 64, 64, 64, 33], 8, 64),
+    (1, [1, 16, 16], 4, 32), (2, [1, 24, 40, 40], 16, 128), (1, [1, 10, 10], 20, 64),
+])
+def test_self_attn_in_place_matches_oracle(api, B, beam_sizes, H, d):
+    """The cache held in place: slab j = the QKV projection of step j; the kernel reads the K and V thirds of the
+    slabs and writes nothing but its output (the slabs must come back bit for bit)."""
+    L = max(5, len(beam_sizes))
+    t = len(beam_sizes) - 1
+    qkv, kc, vc, parents = _self_attn_problem(17 * t + H, B, beam_sizes, H, d, L)
+    scale = 1.0 / np.sqrt(d)
+    par_list = [None] + [parents[j] for j in range(1, t + 1)]
+    ref, _, _ = OA.self_attn(f64(qkv), f64(kc), f64(vc), par_list, beam_sizes, t, B, scale)
+    R_max = kc.shape[1]
+    rng = synth.rng_for(3, 991 + t)
+    slabs = synth.normal_bf16(rng, (L, R_max, 3, H, d))         # q thirds of older slabs: noise nobody may read
+    slabs[:, :, 1], slabs[:, :, 2] = kc, vc
+    R = B * beam_sizes[t]
+    slabs[t, :R] = qkv
+    d_slabs = dev_bf16(slabs)
+    out = torch.zeros((R, H, d), dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.grace_self_attn_inplace(d_slabs, dev(parents), beam_sizes, out, B, t, scale, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert_attention_close(out.float().cpu().numpy(), ref, "self-attn (in place) out")
+    assert np.array_equal(d_slabs.view(torch.int16).cpu().numpy().view(np.uint16), slabs)
+
+
 def test_self_attn_flags_bad_parent(api):
     B, sizes, H, d = 1, [1, 8], 8, 64
     qkv, kc, vc, parents = _self_attn_problem(5, B, sizes, H, d, 5)

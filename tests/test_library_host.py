@@ -38,7 +38,7 @@ def test_struct_layouts_match_the_header(api):
     # sizes computed from the C declarations: a drift between grace.h and the binding shows here
     assert ctypes.sizeof(api.TrieStruct) == 4 + 4 + 8 + 8 + 8 + 8
     assert ctypes.sizeof(api.MatcherStruct) == 4 * 4 + 8 + 8
-    assert ctypes.sizeof(api.LayerStruct) == 22 * 8
+    assert ctypes.sizeof(api.LayerStruct) == 23 * 8
 
 
 def test_host_argument_validation(api):
