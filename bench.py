@@ -415,7 +415,16 @@ def op_rooflines(device, peaks):
         logical = R * 1024 * (6 + 2 * t)                       # q,k,v read 3 KB + k,v write 2 KB + out 1 KB + 2 KB/ancestor
         out[f"self_attn_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, gbs=logical / p50 / 1e3, bound="hbm",
                                           frac=logical / p50 / 1e3 / peaks["hbm_gbs"])
-    del kc, vc, qkv, o
+    del kc, vc, qkv
+    # the form the decode loop runs: the cache is the steps' QKV projections, kept in place (nothing written but out)
+    slabs = rnd(Lc, R, 3, H, d)
+    for t in (1, 3):
+        sizes = [M] * (t + 1)
+        p50, p99 = _time_op(lambda i: api.grace_self_attn_inplace(slabs, parents, sizes, o, B, t, 0.125), 1)
+        logical = R * 1024 * (4 + 2 * t)                       # q,k,v read 3 KB + out 1 KB + 2 KB/ancestor
+        out[f"self_attn_inplace_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, gbs=logical / p50 / 1e3, bound="hbm",
+                                                  frac=logical / p50 / 1e3 / peaks["hbm_gbs"])
+    del slabs, o
     # ---- top-k alone, configuration 4 (dense, all finite: worst case) ----
     B, M, V, K = 32, 2048, 1024, 2048
     cands = [torch.randn(B, M * V, device=device, generator=g) * 3.0 - 8.0 for _ in range(2)]
