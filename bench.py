@@ -437,11 +437,25 @@ def op_rooflines(device, peaks):
     out["beam_topk_dense_B32_N2M_K2048"] = dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm",
                                                frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"],
                                                exact_path_used=bool(st.item() & api.DEV_TOPK_EXACT_PATH))
+    del cands, ws
+    # ---- the same at the decode loop's own shape (configuration 5, step 1: 2048 beams x 2048 tokens per request) ----
+    V = 2048
+    cands = [torch.randn(B, M * V, device=device, generator=g) * 3.0 - 8.0 for _ in range(2)]
+    ws = torch.empty(api.grace_beam_topk_workspace_bytes(B, M * V, K), dtype=torch.uint8, device=device)
+    st.zero_()
+    p50, p99 = _time_op(lambda i: api.grace_beam_topk(cands[i], K, V, sc, fl, pa, tk, ws, st), 2)
+    nbytes = B * M * V * 4
+    out["beam_topk_dense_B32_N4M_K2048"] = dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm",
+                                               frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"],
+                                               exact_path_used=bool(st.item() & api.DEV_TOPK_EXACT_PATH))
+    del cands, ws
     return out
 
 
-def mask_roofline(dec, cfg, peaks):
-    """CD+GTM mask alone at the first full-width level (depth 1: dense rows), on the bench decoder's own state."""
+def mask_roofline(dec, cfg, inp, peaks):
+    """CD+GTM mask alone at the first full-width level (depth 1: dense rows), on the bench decoder's own state:
+    with the loop's prefix-Bloom matcher (random probes into a 512 KB filter per request: bound by L2 sector
+    fetches, not by HBM) and with the node-bitmask matcher over the same catalog and eligible sets (HBM-bound)."""
     import torch
     from paper_2608_00938_b200 import api
     B, M, V = cfg["B"], cfg["schedule"][1], cfg["V"]
@@ -449,12 +463,21 @@ def mask_roofline(dec, cfg, peaks):
     dec.reset(); dec.step(0)                                   # state [1] now holds the level-1 beams
     logp = torch.log_softmax(torch.randn(R, V, device=dec.device) * 3.0, dim=1)
     cand = torch.empty_like(logp)
-    p50, p99 = _time_op(lambda i: api.grace_gtm_mask(logp, dec.score[1][:R], dec.node[1][:R], dec.key[1][:R], dec.trie,
-                                                     dec.matcher, cand, None, B, M, 1, dec.d_status), 1)
     live = int((dec.node[1][:R] >= 0).sum().item())
     nbytes = 2 * R * V * 4
-    return dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm", frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"],
-                live_rows=live, rows=R, matcher="prefix_bloom", note="dense-form bytes: 4 B in + 4 B out per candidate")
+    num_nodes = int(api.grace_trie_build_dense(inp["sids"], V)[2][-1])
+    nb = np.stack([api.grace_node_bitmask_build(inp["sids"], V, e, num_nodes) for e in inp["elig"]])
+    nb_dev = torch.from_numpy(nb.view(np.int64)).to(dec.device)
+    out = {}
+    for name, matcher, note in (
+            ("gtm_mask_depth1_B32_M2048_V2048", dec.matcher, "prefix Bloom 2^22 x 4; dense-form bytes: 4 B in + 4 B out per candidate"),
+            ("gtm_mask_node_bitmask_depth1_B32_M2048_V2048", api.make_matcher(api.MATCH_NODE_BITMASK, nb_dev),
+             "node bitmask; dense-form bytes")):
+        p50, p99 = _time_op(lambda i: api.grace_gtm_mask(logp, dec.score[1][:R], dec.node[1][:R], dec.key[1][:R], dec.trie,
+                                                         matcher, cand, None, B, M, 1, dec.d_status), 1)
+        out[name] = dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm",
+                         frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"], live_rows=live, rows=R, note=note)
+    return out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -645,7 +668,7 @@ def main():
                                          note="B=16; another machine and another implementation: context, not a target")
         if not args.no_ops and world == 1 and default_workload:
             ops = op_rooflines(device, peaks)
-            ops["gtm_mask_depth1_B32_M2048_V2048"] = mask_roofline(dec, cfg, peaks)
+            ops.update(mask_roofline(dec, cfg, inp, peaks))
             line["op_rooflines"] = ops
         if not args.no_cpu and world == 1 and default_workload:
             secs, units_cpu = oracle_sample(cfg, inp, 2048)
