@@ -18,8 +18,9 @@ from gpu_util import DEV, assert_log_probs_close, dev  # noqa: E402
 
 
 def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=2000, V=64, seed_variant=0,
-             std=0.02, shape=(2, 128, 4, 32, 512, 128), T_ctx=64):
-    """shape = (layers, d_model, heads, head size, FFN width, encoder width)."""
+             std=0.02, shape=(2, 128, 4, 32, 512, 128), T_ctx=64, ln_affine=False):
+    """shape = (layers, d_model, heads, head size, FFN width, encoder width).  ln_affine: LayerNorm gains and
+    biases away from (1, 0), so that a folded LayerNorm has something to fold."""
     rng = synth.rng_for(1, seed_variant)
     L = len(schedule)
     sids = synth.catalog(rng, n_sids, V, L)
@@ -27,6 +28,12 @@ def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=
     elig = [synth.eligible_subset(rng, n_sids, 0.3) for _ in range(B)]
     shp = synth.DecoderShape(*shape, V, L)
     w = synth.decoder_weights(rng, shp, std=std, as_bf16=True)
+    if ln_affine:
+        d = shape[1]
+        for holder, names in [(w, ("lnf",))] + [(lw, ("ln1", "ln2", "ln3")) for lw in w["layers"]]:
+            for n in names:
+                holder[n + "_g"] = (1.0 + 0.25 * synth.normal_f32(rng, d)).astype(np.float32)
+                holder[n + "_b"] = (0.3 * synth.normal_f32(rng, d)).astype(np.float32)
     enc = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, T_ctx, shape[5])))
     return dict(sids=sids, trie=trie, elig=elig, shp=shp, w=w, enc=enc, schedule=schedule, final_k=final_k, B=B,
                 matcher_kind=matcher_kind)
@@ -74,6 +81,10 @@ _PAPER_LIKE = dict(shape=(2, 256, 16, 128, 512, 256), T_ctx=128, n_sids=4000)
     (3, "bloom", (1, 40, 24), 32, True, {}),     # the same with the residual stream held in bf16
     (3, "bloom", (1, 40, 24), 32, "uncentred", {}),
     (3, "bloom", (1, 40, 24), 32, "kernel", {}),
+    (3, "bloom", (1, 40, 24), 32, True, dict(ln_affine=True)),          # gains and biases that the fold must carry
+    (3, "bloom", (1, 40, 24), 32, "uncentred", dict(ln_affine=True)),
+    (3, "bloom", (1, 40, 24), 32, "kernel", dict(ln_affine=True)),
+    (3, "bloom", (1, 40, 24), 32, False, dict(ln_affine=True)),          # fp32 stream
     (2, "bloom", (1, 24, 48, 48), 48, True, _PAPER_LIKE),   # dynamic schedule over 4 levels, head size 128
     (2, "node", (1, 100, 80), 80, True, {}),      # step 0 asks for more beams than there are tokens (fixed-schedule shape)
 ])
