@@ -518,6 +518,10 @@ def test_self_attn_flags_bad_parent(api):
     (2, 300, 16, 128, 128),        # the paper's decoder shape: 16 heads of 128, 128 context tokens
     (1, 130, 4, 128, 333),         # head size 128 over several K/V blocks, ragged M and T
     (1, 1, 8, 64, 1024),           # step 0 of the decode loop: one row per request
+    (32, 1, 8, 64, 1024),          # the same at the serving batch size (row-per-CTA kernel)
+    (2, 3, 4, 128, 200),           # a few rows, head size 128, ragged split of the positions over the warps
+    (4, 8, 2, 64, 130),            # the widest beam the row-per-CTA kernel takes
+    (3, 2, 4, 64, 5),              # fewer positions than warps
 ])
 def test_cross_attn_matches_oracle(api, B, M, H, d, T):
     rng = synth.rng_for(2, B * 1000 + M + T)
