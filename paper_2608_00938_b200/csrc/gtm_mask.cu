@@ -52,8 +52,8 @@ constexpr int kMaskWarpsPerBlock = 8;
 // One warp per beam row, two phases per chunk of 2048 tokens:
 //   1. the catalog-valid children (set bits of the node's child bitmask) are enumerated compactly,
 //      lane k takes the k-th, (k+32)-th, ... child, evaluates the request's matcher for it and ORs
-//      the result into the warp's allow words in shared memory.  Bloom probes are issued two at a
-//      time so that both loads are in flight together.
+//      the result into the warp's allow words in shared memory.  Bloom probes are issued one at a
+//      time and stop at the first clear bit (fewest L2 sectors; other rows' warps cover the latency).
 //   2. the row is streamed: cand = score + logp where allowed, -inf elsewhere; a 32-byte sector of
 //      log-probabilities is read only if one of its tokens is allowed.
 // LOGITS = true: `logp` holds raw logits; the row's log-sum-exp is taken in a first streaming pass
@@ -211,12 +211,12 @@ gtm_mask_kernel(const MaskParams p) {
           const int v = (w0 << 6) + (lo << 6) + bit;
           const uint64_t z = mix64(row_key | ((uint64_t)(v + 1) << (16 * p.prefix_len)));
           const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
-          for (int i = 0; i < p.bloom_hashes && ok; i += 2) {
-            const uint32_t pos_a = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
-            const uint32_t pos_b = (h1 + (uint32_t)(i + 1) * h2) & (uint32_t)p.bloom_mask_bits;
-            const uint64_t wa = __ldg(req_bits + (pos_a >> 6));
-            const uint64_t wb = (i + 1 < p.bloom_hashes) ? __ldg(req_bits + (pos_b >> 6)) : ~0ull;
-            ok = ((wa >> (pos_a & 63)) & 1ull) && ((i + 1 >= p.bloom_hashes) || ((wb >> (pos_b & 63)) & 1ull));
+          // One probe at a time, stopping at the first clear bit: the kernel is bound by the number of 32-byte
+          // sectors it pulls out of L2 (probes are random within a 512 KB filter), not by their latency: probing
+          // in pairs fetched 2.7 sectors per candidate instead of 2.25 and ran 10 % slower, all four at once 40 %.
+          for (int i = 0; i < p.bloom_hashes && ok; ++i) {
+            const uint32_t pos = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
+            ok = (__ldg(req_bits + (pos >> 6)) >> (pos & 63)) & 1ull;
           }
         }
         if (ok) atomicOr(&allow[lo], 1ull << bit);
