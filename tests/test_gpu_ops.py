@@ -522,6 +522,9 @@ def test_self_attn_flags_bad_parent(api):
     (2, 3, 4, 128, 200),           # a few rows, head size 128, ragged split of the positions over the warps
     (4, 8, 2, 64, 130),            # the widest beam the row-per-CTA kernel takes
     (3, 2, 4, 64, 5),              # fewer positions than warps
+    (2, 1, 2, 64, 1),              # a single encoder position: the softmax is the identity (row-per-CTA kernel)
+    (1, 200, 2, 64, 1),            # the same through the tensor-core kernel (one valid column in a 128-wide block)
+    (1, 40, 2, 128, 1),
 ])
 def test_cross_attn_matches_oracle(api, B, M, H, d, T):
     rng = synth.rng_for(2, B * 1000 + M + T)
