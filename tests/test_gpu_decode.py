@@ -18,9 +18,10 @@ from gpu_util import DEV, assert_log_probs_close, dev  # noqa: E402
 
 
 def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=2000, V=64, seed_variant=0,
-             std=0.02, shape=(2, 128, 4, 32, 512, 128), T_ctx=64, ln_affine=False):
+             std=0.02, shape=(2, 128, 4, 32, 512, 128), T_ctx=64, ln_affine=False, embed_offset=0.0):
     """shape = (layers, d_model, heads, head size, FFN width, encoder width).  ln_affine: LayerNorm gains and
-    biases away from (1, 0), so that a folded LayerNorm has something to fold."""
+    biases away from (1, 0), so that a folded LayerNorm has something to fold.  embed_offset: a constant added to
+    every embedding row (a per-row shift of the residual stream, which no LayerNorm sees)."""
     rng = synth.rng_for(1, seed_variant)
     L = len(schedule)
     sids = synth.catalog(rng, n_sids, V, L)
@@ -34,6 +35,9 @@ def _config1(B=1, matcher_kind="node", schedule=(1, 16, 16), final_k=16, n_sids=
             for n in names:
                 holder[n + "_g"] = (1.0 + 0.25 * synth.normal_f32(rng, d)).astype(np.float32)
                 holder[n + "_b"] = (0.3 * synth.normal_f32(rng, d)).astype(np.float32)
+    if embed_offset:
+        w["embed"] = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(
+            (np.asarray(w["embed"], np.float32) + np.float32(embed_offset)).astype(np.float32)))
     enc = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, T_ctx, shape[5])))
     return dict(sids=sids, trie=trie, elig=elig, shp=shp, w=w, enc=enc, schedule=schedule, final_k=final_k, B=B,
                 matcher_kind=matcher_kind)
@@ -85,6 +89,11 @@ _PAPER_LIKE = dict(shape=(2, 256, 16, 128, 512, 256), T_ctx=128, n_sids=4000)
     (3, "bloom", (1, 40, 24), 32, "uncentred", dict(ln_affine=True)),
     (3, "bloom", (1, 40, 24), 32, "kernel", dict(ln_affine=True)),
     (3, "bloom", (1, 40, 24), 32, False, dict(ln_affine=True)),          # fp32 stream
+    # a stream whose rows sit at a mean of 0.5 with a spread of a few hundredths: a bf16 stream that holds the mean
+    # loses most of the signal (measured: rms error 0.04 x the logit spread for the uncentred bf16 variants); the
+    # centred stream never sees the mean (0.006 x), the fp32 stream can hold it (0.004 x)
+    (3, "bloom", (1, 40, 24), 32, True, dict(ln_affine=True, embed_offset=0.5)),
+    (3, "bloom", (1, 40, 24), 32, False, dict(ln_affine=True, embed_offset=0.5)),
     (2, "bloom", (1, 24, 48, 48), 48, True, _PAPER_LIKE),   # dynamic schedule over 4 levels, head size 128
     (2, "node", (1, 100, 80), 80, True, {}),      # step 0 asks for more beams than there are tokens (fixed-schedule shape)
 ])
