@@ -172,32 +172,29 @@ row_stats_bf16_kernel(const uint16_t* __restrict__ x, float2* __restrict__ out, 
   }
 #pragma unroll
   for (int j = 0; j < ROWS; ++j) {
-    f32x2_t acc = f2_pack(0.f, 0.f);
+    // one pass: sum and sum of squares in fp32 (inputs are bf16: eight mantissa bits, rows of at most 2048
+    // elements; the subtraction E[x^2] - mean^2 loses log2(1 + mean^2 / var) of fp32's 24 bits, nothing at all
+    // on a centred stream)
+    f32x2_t acc = f2_pack(0.f, 0.f), sq = f2_pack(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < MAXV; ++i) {
       const uint4 t = raw[j][i];
-      acc = f2_add(acc, f2_add(f2_add(f2_from_bf16x2(t.x), f2_from_bf16x2(t.y)),
-                               f2_add(f2_from_bf16x2(t.z), f2_from_bf16x2(t.w))));
+      const f32x2_t a = f2_from_bf16x2(t.x), b = f2_from_bf16x2(t.y), c = f2_from_bf16x2(t.z), d = f2_from_bf16x2(t.w);
+      acc = f2_add(acc, f2_add(f2_add(a, b), f2_add(c, d)));
+      sq = f2_fma(a, a, sq); sq = f2_fma(b, b, sq); sq = f2_fma(c, c, sq); sq = f2_fma(d, d, sq);
     }
-    float lo, hi;
+    float lo, hi, qlo, qhi;
     f2_unpack(acc, lo, hi);
-    const float mean = warp_sum(lo + hi) / (float)D;
-    const f32x2_t m2 = f2_pack(mean, mean);
-    f32x2_t sq = f2_pack(0.f, 0.f);
+    f2_unpack(sq, qlo, qhi);
+    float s1 = lo + hi, s2 = qlo + qhi;
 #pragma unroll
-    for (int i = 0; i < MAXV; ++i) {
-      if (i * 32 + lane < n8) {
-        const uint4 t = raw[j][i];
-        const uint32_t w4[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const f32x2_t d = f2_sub(f2_from_bf16x2(w4[e]), m2);
-          sq = f2_fma(d, d, sq);
-        }
-      }
+    for (int o = 16; o > 0; o >>= 1) {
+      s1 += __shfl_xor_sync(kFullMask, s1, o);
+      s2 += __shfl_xor_sync(kFullMask, s2, o);
     }
-    f2_unpack(sq, lo, hi);
-    const float rstd = rsqrtf(warp_sum(lo + hi) / (float)D + eps);
+    const float mean = s1 / (float)D;
+    const float var = fmaxf(s2 / (float)D - mean * mean, 0.f);
+    const float rstd = rsqrtf(var + eps);
     if (lane == 0 && r0 + j < R) out[r0 + j] = make_float2(rstd, -rstd * mean);
   }
 }
