@@ -206,8 +206,10 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 // A cluster of two CTAs (two SMs) walks over 256 x 256 output tiles (n fastest, so the pairs running
 // at the same time share an A row panel in L2) with one tcgen05.mma.cta_group::2 stream.  Each CTA
 // stages its own 128 rows of A and its own 128 rows of W (half of the tile's N) through a 6-stage
-// ring, so an SM fills 32 KB of shared memory per 64-wide k-block where a lone 128 x 256 tile needs
-// 48 KB: the fill rate of shared memory, not the tensor pipe, is what limits these GEMMs.  The even
+// ring, so an SM pulls 32 KB per 64-wide k-block through its port to the L2 where a lone 128 x 256 tile
+// needs 48 KB: that port (about 64 bytes per clock for loads and stores together), not the tensor pipe, is
+// what limits these GEMMs at K = 512 (256 KB of operands in, 64 KB of bf16 results out per tile and CTA
+// against 4096 clocks of MMAs).  The even
 // CTA issues every MMA into one of TWO TMEM accumulators (2 x 256 columns = all of TMEM), so the
 // four epilogue warps of each CTA drain tile i while the tensor cores already work on tile i+1.
 // tcgen05.commit arrives on the barriers of both CTAs, and both CTAs' TMA loads count their bytes on
