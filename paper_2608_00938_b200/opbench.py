@@ -44,6 +44,8 @@ def main():
     ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
     ap.add_argument("--kway", type=int, default=1, help="lookup: static k-way partitioned rows with this k at every level")
     ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
+    ap.add_argument("--inplace", action="store_true",
+                    help="self_attn: the cache slabs are the steps' QKV projections (nothing written but the output)")
     ap.add_argument("--folded", action="store_true",
                     help="linear: LayerNorm folded into the epilogue (row pair + column bias; centred rows)")
     a = ap.parse_args()
@@ -85,8 +87,12 @@ def main():
         kc, vc = bf(Lc, R, a.H, a.d), bf(Lc, R, a.H, a.d)
         par = torch.randint(0, a.M, (Lc, R), device=dev, dtype=torch.int32)
         qkv, o = bf(R, 3, a.H, a.d), torch.empty(R, a.H, a.d, device=dev, dtype=torch.bfloat16)
-        us = _time(lambda: api.grace_self_attn(qkv, kc, vc, par, [a.M] * Lc, o, a.B, a.t, a.d ** -0.5), a.iters)
-        by = R * a.H * a.d * 2 * (6 + 2 * a.t)
+        if a.inplace:
+            slabs = bf(Lc, R, 3, a.H, a.d)
+            us = _time(lambda: api.grace_self_attn_inplace(slabs, par, [a.M] * Lc, o, a.B, a.t, a.d ** -0.5), a.iters)
+        else:
+            us = _time(lambda: api.grace_self_attn(qkv, kc, vc, par, [a.M] * Lc, o, a.B, a.t, a.d ** -0.5), a.iters)
+        by = R * a.H * a.d * 2 * ((4 if a.inplace else 6) + 2 * a.t)
         print(f"self_attn R={R} T_self={a.t + 1}: {us:.1f} us, {by / us / 1e3:.0f} GB/s (logical bytes)")
     elif a.op == "topk":
         N = a.M * a.V
