@@ -178,6 +178,14 @@ extern "C" int grace_wait_timeouts(void) {
 // Keeps part of a buffer that many kernels of a step re-read (the residual stream: three add-reductions,
 // three statistics passes and three GEMM operand reads per layer) resident in L2 across the large tensors
 // that stream past it: an access-policy window on the stream, backed by this context's persisting carve-out.
+// A refused hint must not leave a stale "last error" behind for the next launch check to find.
+#define L2_TRY(expr)                                          \
+  do {                                                        \
+    if ((expr) != cudaSuccess) {                              \
+      (void)cudaGetLastError();                               \
+      return GRACE_CUDA_ERROR;                                \
+    }                                                         \
+  } while (0)
 extern "C" grace_status_t grace_stream_l2_persist(void* stream, const void* ptr, size_t bytes, float fraction) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaStreamAttrValue v;
@@ -185,24 +193,25 @@ extern "C" grace_status_t grace_stream_l2_persist(void* stream, const void* ptr,
   if (ptr == nullptr || bytes == 0) {                       // clear the window
     v.accessPolicyWindow.hitProp = cudaAccessPropertyNormal;
     v.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
-    GRACE_CUDA_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
+    L2_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
     return GRACE_OK;
   }
   if (!(fraction > 0.f && fraction <= 1.f)) return GRACE_INVALID_ARG;
   int dev = 0, max_persist = 0, max_window = 0;
-  GRACE_CUDA_TRY(cudaGetDevice(&dev));
-  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev));
-  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev));
+  L2_TRY(cudaGetDevice(&dev));
+  L2_TRY(cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev));
+  L2_TRY(cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev));
   if (max_persist <= 0 || max_window <= 0) return GRACE_UNSUPPORTED_SHAPE;
   const size_t window = bytes < (size_t)max_window ? bytes : (size_t)max_window;
   size_t carve = (size_t)((double)window * fraction);
   if (carve > (size_t)max_persist) carve = (size_t)max_persist;
-  GRACE_CUDA_TRY(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve));
+  L2_TRY(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve));
   v.accessPolicyWindow.base_ptr = const_cast<void*>(ptr);
   v.accessPolicyWindow.num_bytes = window;
   v.accessPolicyWindow.hitRatio = (float)((double)carve / (double)window);   // the share of the window's lines kept
   v.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
   v.accessPolicyWindow.missProp = cudaAccessPropertyNormal;
-  GRACE_CUDA_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
+  L2_TRY(cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v));
   return GRACE_OK;
 }
+#undef L2_TRY

@@ -211,7 +211,10 @@ class Decoder:
         stream to stay resident in L2 (it is re-read nine times per layer while larger tensors stream past)."""
         sid = torch.cuda.current_stream(self.device).cuda_stream
         if self.persist_stream_l2 and sid not in self._prepared_streams:
-            api.grace_stream_l2_persist(self.x)
+            try:
+                api.grace_stream_l2_persist(self.x)
+            except api.GraceError:                         # a residency hint the device refuses is not an error
+                self.persist_stream_l2 = False
             self._prepared_streams.add(sid)
 
     def step(self, t: int) -> None:
