@@ -441,6 +441,7 @@ def _self_attn_problem(seed, B, beam_sizes, H, d, L):
     (1, [2, 3, 4, 5, 6, 7, 8, 9], 2, 64),
     (2, [1, 24, 40, 40], 16, 128),          # the paper's decoder width: rows of 2048 = two 1024-element segments
     (1, [1, 10, 10], 20, 64),               # 1280-wide rows: ragged second segment
+    (1, [1, 6, 6], 64, 128),                # the widest row the kernel takes: 8192 elements, eight segments
 ])
 def test_self_attn_matches_oracle(api, B, beam_sizes, H, d):
     L = max(5, len(beam_sizes))
@@ -466,7 +467,8 @@ def test_self_attn_matches_oracle(api, B, beam_sizes, H, d):
 
 @pytest.mark.parametrize("B,beam_sizes,H,d", [
     (3, [1], 8, 64), (2, [1, 50, 70], 8, 64), (2, [1, 64, 64, 130], 8, 64), (2, [5, 64, 64, 64, 33], 8, 64),
-    (1, [1, 16, 16], 4, 32), (2, [1, 24, 40, 40], 16, 128), (1, [1, 10, 10], 20, 64),
+    (1, [1, 16, 16], 4, 32), (2, [1, 24, 40, 40], 16, 128), (1, [1, 10, 10], 20, 64), (1, [1, 6, 6], 64, 128),
+    (1, [2, 3, 4, 5, 6, 7, 8, 9], 2, 64),   # the longest prefix the kernel takes (T_self = 8)
 ])
 def test_self_attn_in_place_matches_oracle(api, B, beam_sizes, H, d):
     """The cache held in place: slab j = the QKV projection of step j; the kernel reads the K and V thirds of the
