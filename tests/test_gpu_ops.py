@@ -750,7 +750,9 @@ def test_mask_kernel_merges_log_sum_exp_partials(api, kind, M):
 
 @pytest.mark.parametrize("M,N,K,relu,f32out", [(300, 384, 128, False, False), (130, 2048, 512, True, False),
                                                (2100, 1536, 512, False, False), (1500, 2048, 512, True, False),
-                                               (1100, 512, 512, False, True), (33000, 2048, 512, False, True)])
+                                               (1100, 512, 512, False, True), (33000, 2048, 512, False, True),
+                                               # ragged last column tile in the pair kernel (clamped vector fetches)
+                                               (1500, 784, 512, True, False), (1300, 336, 512, False, True)])
 @pytest.mark.parametrize("centred", [False, True])
 def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
     """grace_row_stats_bf16 + grace_linear_folded_ln against LayerNorm(x) @ w^T in fp64: the GEMM reads the raw
