@@ -618,7 +618,7 @@ def main():
                             n_layers=cfg["n_layers"], d_model=cfg["d_model"], H=cfg["H"], d_h=cfg["d_h"],
                             d_ffn=cfg["d_ffn"], T_ctx=cfg["T_ctx"], V=cfg["V"], L=cfg["L"], catalog_sids=cfg["n_sids"],
                             matcher="prefix_bloom_2^22x4", parallelism=f"requests sharded x{world}",
-                            l2="working set ~5 GB per loop, far larger than the 126 MB L2", launch=launch_mode,
+                            l2="no flush needed: a loop moves ~30 GB of activations (67-540 MB per kernel) through the 126 MB L2", launch=launch_mode,
                             residual_stream=args.residual, accumulate="f32",
                             layer_norm=("folded into the GEMMs, centred stream" if dec.fold_layer_norm else "kernel"),
                             macs_per_request=decoder_macs(cfg)),
