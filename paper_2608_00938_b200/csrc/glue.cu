@@ -380,7 +380,7 @@ extern "C" grace_status_t grace_row_stats_bf16(const uint16_t* x, int R, int D, 
   const int pieces = ((D >> 3) + 31) / 32;
   auto blocks = [&](int rows) { return (R + 4 * rows - 1) / (4 * rows); };
   if (pieces <= 1) launch_pdl(row_stats_bf16_kernel<1, 4>, dim3(blocks(4)), dim3(128), 0, s, x, out, R, D, eps);
-  else if (pieces <= 2) launch_pdl(row_stats_bf16_kernel<2, 4>, dim3(blocks(4)), dim3(128), 0, s, x, out, R, D, eps);
+  else if (pieces <= 2) launch_pdl(row_stats_bf16_kernel<2, 2>, dim3(blocks(2)), dim3(128), 0, s, x, out, R, D, eps);   // measured: 2 rows per warp 12.3 us, 4: 13.2, 8: 15.2, 1: 18.4 at 65536 x 512
   else if (pieces <= 4) launch_pdl(row_stats_bf16_kernel<4, 2>, dim3(blocks(2)), dim3(128), 0, s, x, out, R, D, eps);
   else launch_pdl(row_stats_bf16_kernel<8, 1>, dim3(blocks(1)), dim3(128), 0, s, x, out, R, D, eps);
   GRACE_LAUNCH_CHECK();
