@@ -9,6 +9,10 @@
 //     the encoder positions for the scores and the head dimension for the weighted sum.
 #include "common.cuh"
 #include "cross_attn_tc.cuh"
+#include "cross_attn_ms.cuh"
+
+// The four-stream kernel is selected here once it beats the two-CTA kernel on every benchmark shape.
+static constexpr bool kUseMultiStream = true;
 
 namespace grace {
 
@@ -227,6 +231,10 @@ extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stri
     else launch_pdl(cross_attn_row_kernel<128>, dim3(B * M * H), dim3(256), 0, s, p);
     GRACE_LAUNCH_CHECK();
     return GRACE_OK;
+  }
+  if (kUseMultiStream && cross_attn_ms_supported(B, M, H, d_h, T_ctx)) {
+    return launch_cross_attn_ms(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,
+                                out_row_stride, lse, nullptr, B, M, H, T_ctx, scale, s);
   }
   if (cross_attn_tc_supported(B, M, H, d_h, T_ctx)) {
     return launch_cross_attn_tc(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,

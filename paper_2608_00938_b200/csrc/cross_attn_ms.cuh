@@ -1,0 +1,496 @@
+// Cross-attention on tcgen05 tensor cores, head size 64: four independent softmax streams per SM
+// (Section 5.1: the beams of a request are the M dimension of a dense contraction against that
+// request's shared K/V).
+//
+// At head size 64 a 128 x 128 score block costs 512 tensor-core clocks but 16384 exponentials, and
+// the special-function unit takes one warp instruction per 8 clocks and scheduler: the exponentials
+// set the pace (1024 clocks per block and SM).  A single warp can issue an exponential only every
+// ~14 clocks, and every hand-off between warps or to the tensor core (mbarrier arrive -> wake,
+// MMA issue, commit -> wake) costs 150-250 clocks, so the unit stays busy only if several warps per
+// scheduler are in DIFFERENT phases of their blocks and never wait for one another.  Hence:
+//
+//   * one CTA per SM owns all 512 TMEM columns and runs four streams.  A stream is one 128-row
+//     query tile of one (request, head) with its own 64 score columns (S, fp32; the packed bf16
+//     probabilities P overwrite the first 32 of them) and 64 output columns (O, fp32) in TMEM, its
+//     own Q tile in shared memory and its own barriers;
+//   * streams 0/1 are the two tiles of one 256-row item and share that item's K/V ring, streams
+//     2/3 those of another item with a second ring: two independent halves, so a request needs
+//     only 256 beams to fill an SM;
+//   * a stream is served by four warps (one per TMEM lane quarter, one thread per query row):
+//     16 softmax warps, four per scheduler.  The stream's first warp also issues the stream's own
+//     MMAs: after the four warps have stored P of block j it issues O += P V_j and then S of block
+//     j + 1 (the in-order tensor pipe guarantees that S never overwrites a P still to be read).
+//     Nothing is exchanged between streams; their chains  S -> softmax -> P -> P V -> next S
+//     interleave freely, each running under the other three streams' exponentials;
+//   * encoder positions are cut in blocks of 64; K and V blocks arrive by TMA through four-slot
+//     rings per half; Q, K and V are addressed with 4-D tensor maps over the caller's strides, so
+//     the beam-major Q / O layout is never permuted.  A stream's Q tile is reloaded as soon as the
+//     last S of its item has run, i.e. under the item's last softmax and epilogue.
+//
+// Ragged M and T are zero-filled by TMA and masked in the softmax; `enc_len` (optional) gives a
+// per-request number of valid encoder positions (0: the output rows are zero).  Every wait is
+// bounded (tc::mbar_wait); a wait that gives up sets the CTA's abort flag, every role leaves its
+// loops, TMEM is freed and the kernel returns.
+#pragma once
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace grace {
+
+constexpr int kMsBM = 128;                 // query rows per tile (stream)
+constexpr int kMsBN = 64;                  // encoder positions per K / V block in shared memory
+constexpr int kMsSub = 32;                 // encoder positions per softmax sub-block (two per block)
+constexpr float kMsGrowLog2 = 16.0f;       // the running reference maximum moves only when exceeded by this much
+constexpr int kMsDH = 64;
+constexpr int kMsStages = 4;               // K ring and V ring slots per half
+constexpr int kMsQBytes = kMsBM * kMsDH * 2;       // 16 KB
+constexpr int kMsKVBytes = kMsBN * kMsDH * 2;      // 8 KB
+constexpr int kMsSoftmaxWarps = 16;
+constexpr int kMsThreads = (kMsSoftmaxWarps + 1 + 4) * 32;   // + producer + one MMA issuer per stream
+constexpr int kMsBarBytes = 1024;
+constexpr int kMsSmemBytes = 1024 + 4 * kMsQBytes + 2 * 2 * kMsStages * kMsKVBytes + kMsBarBytes;
+
+struct CrossMsParams {
+  uint16_t* out;
+  float* lse;
+  const int32_t* enc_len;       // nullable: valid encoder positions per request (<= T)
+  int64_t out_row_stride;
+  int B, M, H, T;
+  int pairs_m, total_items;     // 256-row items per (request, head); items = B * H * pairs_m
+  float scale_log2;             // scale * log2(e)
+};
+
+__device__ __forceinline__ float ms_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float ms_max3(float a, float b, float c) {
+  float m;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+  return m;
+}
+
+// One 256-row item: request, head, first query row, encoder positions, blocks, live tiles.
+struct MsItem { int b, h, row0, T, nb, ntiles; };
+__device__ __forceinline__ MsItem ms_item(const CrossMsParams& p, int item) {
+  MsItem it;
+  const int bh = item / p.pairs_m;
+  const int pair = item - bh * p.pairs_m;
+  it.b = bh / p.H;
+  it.h = bh - it.b * p.H;
+  it.row0 = pair * 2 * kMsBM;
+  int t = p.T;
+  if (p.enc_len != nullptr) { const int e = __ldg(p.enc_len + it.b); t = e < 0 ? 0 : (e < t ? e : t); }
+  it.T = t;
+  it.nb = (t + kMsBN - 1) / kMsBN;
+  it.ntiles = p.M - it.row0 > kMsBM ? 2 : 1;
+  return it;
+}
+
+__global__ void __launch_bounds__(kMsThreads, 1)
+cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_v, const CrossMsParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_tiles = tiles;                                      // [stream] x 16 KB
+  uint8_t* k_tiles = tiles + 4 * kMsQBytes;                      // [half][slot] x 8 KB
+  uint8_t* v_tiles = k_tiles + 2 * kMsStages * kMsKVBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(v_tiles + 2 * kMsStages * kMsKVBytes);
+  uint64_t* q_full = bars;                          // [4] per stream
+  uint64_t* q_empty = q_full + 4;                   // [4]
+  uint64_t* k_full = q_empty + 4;                   // [2][kMsStages]
+  uint64_t* k_empty = k_full + 2 * kMsStages;       //        two arrivals: both streams of the half
+  uint64_t* v_full = k_empty + 2 * kMsStages;
+  uint64_t* v_empty = v_full + 2 * kMsStages;
+  uint64_t* s_full = v_empty + 2 * kMsStages;       // [4][2] S of a sub-block is in the stream's TMEM buffer
+  uint64_t* p_full = s_full + 8;                    // [4][2] the stream's four warps have stored P there
+  uint64_t* o_full = p_full + 8;                    // [4] the stream's last P V of the item is done
+  uint64_t* r_full = o_full + 4;                    // [4] the stream's last but one P V of the item is done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(r_full + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 4; ++i) {
+      tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 1);
+      tc::mbar_init(s_full + 2 * i, 1); tc::mbar_init(s_full + 2 * i + 1, 1);
+      tc::mbar_init(p_full + 2 * i, 4); tc::mbar_init(p_full + 2 * i + 1, 4);
+      tc::mbar_init(o_full + i, 1); tc::mbar_init(r_full + i, 1);
+    }
+    for (int i = 0; i < 2 * kMsStages; ++i) {
+      tc::mbar_init(k_full + i, 1); tc::mbar_init(k_empty + i, 2);
+      tc::mbar_init(v_full + i, 1); tc::mbar_init(v_empty + i, 2);
+    }
+    *abort_flag = 0;
+    tc::fence_mbar_init();
+  }
+  if (warp == kMsSoftmaxWarps) tc::tmem_alloc(tmem_slot, 512);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                  // barrier set-up and TMEM allocation overlapped the previous kernel's tail
+  pdl_trigger();
+  // Half `hf` of CTA c works on the items 2 (c + k gridDim) + hf, k = 0, 1, ...: the two halves of a
+  // CTA and neighbouring CTAs run neighbouring items, which share K/V in L2.
+  const int item_step = 2 * (int)gridDim.x;
+
+  if (warp == kMsSoftmaxWarps) {
+    // ---------------- TMA producer ----------------
+    // Eight queues (Q per stream, K and V per half), fed by polling: whichever slot frees next gets
+    // its load, no queue blocks another.
+    if (lane == 0) {
+      tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
+      // A queue's item is decoded when the queue moves on to it, not on every poll.
+      int q_item[4], q_cnt[4];                      // item whose Q tile comes next; loads done
+      int k_item[2], k_j[2], k_cnt[2], v_item[2], v_j[2], v_cnt[2];
+      MsItem q_it[4], k_it[2], v_it[2];
+      const MsItem none = {0, 0, 0, 0, 0, 0};
+      for (int s = 0; s < 4; ++s) {
+        q_item[s] = 2 * (int)blockIdx.x + (s >> 1); q_cnt[s] = 0;
+        q_it[s] = q_item[s] < p.total_items ? ms_item(p, q_item[s]) : none;
+      }
+      for (int hf = 0; hf < 2; ++hf) {
+        k_item[hf] = v_item[hf] = 2 * (int)blockIdx.x + hf;
+        k_j[hf] = v_j[hf] = 0; k_cnt[hf] = v_cnt[hf] = 0;
+        k_it[hf] = v_it[hf] = k_item[hf] < p.total_items ? ms_item(p, k_item[hf]) : none;
+      }
+      int idle = 0;
+      bool more = true;
+      while (more && !*abort_flag) {
+        bool progressed = false;
+        more = false;
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+          if (q_item[s] >= p.total_items) continue;
+          more = true;
+          bool advance = (s & 1) >= q_it[s].ntiles || q_it[s].nb == 0;      // nothing to load for this stream
+          if (!advance && tc::mbar_try_wait_now(q_empty + s, (q_cnt[s] & 1) ^ 1)) {
+            tc::mbar_expect_tx(q_full + s, kMsQBytes);
+            tc::tma_load_4d(q_tiles + s * kMsQBytes, &map_q, q_full + s, 0, q_it[s].h, q_it[s].row0 + (s & 1) * kMsBM, q_it[s].b);
+            ++q_cnt[s];
+            advance = true;
+          }
+          if (advance) {
+            q_item[s] += item_step;
+            if (q_item[s] < p.total_items) q_it[s] = ms_item(p, q_item[s]);
+            progressed = true;
+          }
+        }
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          if (k_item[hf] < p.total_items) {
+            more = true;
+            if (k_j[hf] >= k_it[hf].nb) {
+              k_item[hf] += item_step; k_j[hf] = 0; progressed = true;
+              if (k_item[hf] < p.total_items) k_it[hf] = ms_item(p, k_item[hf]);
+            } else {
+              const int slot = hf * kMsStages + k_cnt[hf] % kMsStages;
+              if (tc::mbar_try_wait_now(k_empty + slot, ((k_cnt[hf] / kMsStages) & 1) ^ 1)) {
+                tc::mbar_expect_tx(k_full + slot, kMsKVBytes);
+                tc::tma_load_4d(k_tiles + slot * kMsKVBytes, &map_k, k_full + slot, 0, k_j[hf] * kMsBN, k_it[hf].h, k_it[hf].b);
+                ++k_cnt[hf]; ++k_j[hf];
+                progressed = true;
+              }
+            }
+          }
+          if (v_item[hf] < p.total_items) {
+            more = true;
+            if (v_j[hf] >= v_it[hf].nb) {
+              v_item[hf] += item_step; v_j[hf] = 0; progressed = true;
+              if (v_item[hf] < p.total_items) v_it[hf] = ms_item(p, v_item[hf]);
+            } else if (v_cnt[hf] < k_cnt[hf]) {                  // K of a block is wanted before its V
+              const int slot = hf * kMsStages + v_cnt[hf] % kMsStages;
+              if (tc::mbar_try_wait_now(v_empty + slot, ((v_cnt[hf] / kMsStages) & 1) ^ 1)) {
+                tc::mbar_expect_tx(v_full + slot, kMsKVBytes);
+                tc::tma_load_4d(v_tiles + slot * kMsKVBytes, &map_v, v_full + slot, 0, v_j[hf] * kMsBN, v_it[hf].h, v_it[hf].b);
+                ++v_cnt[hf]; ++v_j[hf];
+                progressed = true;
+              }
+            }
+          }
+        }
+        if (progressed) {
+          idle = 0;
+        } else {
+          __nanosleep(400);
+          if (++idle > (1 << 24)) {                          // bounded: seconds of nothing to do
+            if (*abort_flag == 0) atomicAdd(&tc::g_tc_timeouts, 1);
+            *abort_flag = 1;
+          }
+        }
+      }
+    }
+  } else if (warp >= kMsSoftmaxWarps + 1) {
+    // ---------------- MMA issuers, one warp per stream ----------------
+    // The whole warp walks the loops and waits on the barriers; one elected lane issues (warp-uniform
+    // control flow keeps the descriptors in uniform registers).  Sequence per item with n sub-blocks:
+    //   S(0), S(1);  then for u = 0 .. n-1:  O += P(u) V(u);  S(u + 2)
+    // S(u + 2) overwrites the buffer P(u) was read from: the in-order tensor pipe makes that safe.
+    const int s = warp - (kMsSoftmaxWarps + 1);
+    const int hf = s >> 1, tile = s & 1;
+    const uint32_t tmem_s = tmem_base + 64 * s;             // two S / P buffers of 32 columns
+    const uint32_t tmem_o = tmem_base + 256 + 64 * s;
+    constexpr uint32_t idesc_s = tc::idesc_bf16(kMsBM, kMsSub, 0);    // Q K^T : B K-major, 32 score columns
+    constexpr uint32_t idesc_o = tc::idesc_bf16(kMsBM, kMsDH, 1);     // P V   : B MN-major, 64 output columns
+    // Operand descriptors differ only in their start address (bits 0..13, in 16-byte units).
+    const uint64_t q_desc = tc::smem_desc_sw128(tc::smem_addr(q_tiles + s * kMsQBytes), 16, 1024);
+    const uint64_t k_desc0 = tc::smem_desc_sw128(tc::smem_addr(k_tiles + hf * kMsStages * kMsKVBytes), 16, 1024);
+    const uint64_t v_desc0 = tc::smem_desc_sw128(tc::smem_addr(v_tiles + hf * kMsStages * kMsKVBytes), 1024, 1024);
+    uint64_t* const kf = k_full + hf * kMsStages;
+    uint64_t* const ke = k_empty + hf * kMsStages;
+    uint64_t* const vf = v_full + hf * kMsStages;
+    uint64_t* const ve = v_empty + hf * kMsStages;
+    uint32_t g_s = 0, g_p = 0;                    // sub-blocks whose S / whose P V has been issued (buffer = index & 1)
+    uint32_t qc = 0, kc = 0, vc = 0;              // Q tiles, K blocks, V blocks consumed
+    bool ok = true;
+    for (int item = 2 * (int)blockIdx.x + hf; ok && item < p.total_items; item += item_step) {
+      const MsItem it = ms_item(p, item);
+      if (tile >= it.ntiles) {
+        // No rows for this stream in the item: the half's other stream uses the K/V blocks alone,
+        // this one only hands them back (the slots count two arrivals).
+        for (int j = 0; ok && j < it.nb; ++j) {
+          ok = tc::mbar_wait(kf + kc % kMsStages, (kc / kMsStages) & 1, abort_flag);
+          if (ok && lane == 0) tc::mbar_arrive(ke + kc % kMsStages);
+          ++kc;
+          ok = ok && tc::mbar_wait(vf + vc % kMsStages, (vc / kMsStages) & 1, abort_flag);
+          if (ok && lane == 0) tc::mbar_arrive(ve + vc % kMsStages);
+          ++vc;
+        }
+        continue;
+      }
+      if (it.nb == 0) continue;
+      const int nsub = (it.T + kMsSub - 1) / kMsSub;
+      // S of sub-block u: K rows 32 (u & 1) .. + 31 of K block u >> 1
+      auto issue_s = [&](int u) -> bool {
+        if (u == 0 && !tc::mbar_wait(q_full + s, qc & 1, abort_flag)) return false;
+        const int slot = kc % kMsStages;
+        if ((u & 1) == 0 && !tc::mbar_wait(kf + slot, (kc / kMsStages) & 1, abort_flag)) return false;
+        tc::tc_fence_after();
+        const bool block_done = (u & 1) || u == nsub - 1;
+        if (tc::elect_one()) {
+          const uint64_t kd = k_desc0 + (uint64_t)((slot * kMsKVBytes + (u & 1) * (kMsSub * 128)) >> 4);
+          const uint32_t d = tmem_s + kMsSub * (g_s & 1);
+#pragma unroll
+          for (int k = 0; k < kMsDH / 16; ++k)
+            tc::mma_ss(d, q_desc + (uint64_t)((32 * k) >> 4), kd + (uint64_t)((32 * k) >> 4), idesc_s, k ? 1u : 0u);
+          tc::mma_commit(s_full + 2 * s + (g_s & 1));
+          if (block_done) tc::mma_commit(ke + slot);
+          if (u == nsub - 1) tc::mma_commit(q_empty + s);
+        }
+        __syncwarp();
+        ++g_s;
+        if (block_done) ++kc;
+        if (u == nsub - 1) ++qc;
+        return true;
+      };
+      ok = issue_s(0);
+      if (ok && nsub > 1) ok = issue_s(1);
+      for (int u = 0; ok && u < nsub; ++u) {
+        const int slot = vc % kMsStages;
+        if ((u & 1) == 0) ok = tc::mbar_wait(vf + slot, (vc / kMsStages) & 1, abort_flag);
+        ok = ok && tc::mbar_wait(p_full + 2 * s + (g_p & 1), (g_p >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc::tc_fence_after();
+        const bool block_done = (u & 1) || u == nsub - 1;
+        if (tc::elect_one()) {
+          const uint64_t vd = v_desc0 + (uint64_t)((slot * kMsKVBytes + (u & 1) * (kMsSub * 128)) >> 4);
+          const uint32_t a = tmem_s + kMsSub * (g_p & 1);
+#pragma unroll
+          for (int k = 0; k < kMsSub / 16; ++k)
+            tc::mma_ts(tmem_o, a + 8 * k, vd + (uint64_t)((2048 * k) >> 4), idesc_o, (u > 0 || k > 0) ? 1u : 0u);
+          if (block_done) tc::mma_commit(ve + slot);
+          if (u == nsub - 2) tc::mma_commit(r_full + s);       // for a late rescale of O in the last sub-block
+          if (u == nsub - 1) tc::mma_commit(o_full + s);
+        }
+        __syncwarp();
+        ++g_p;
+        if (block_done) ++vc;
+        if (u + 2 < nsub) ok = issue_s(u + 2);
+      }
+    }
+  } else {
+    // ---------------- softmax: four warps per stream ----------------
+    const int q = warp & 3;                       // TMEM lane quarter = query rows 32 q .. 32 q + 31 of the tile
+    const int s = warp >> 2;                      // stream
+    const int hf = s >> 1, tile = s & 1;
+    const int row = q * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const uint32_t tmem_s = tmem_base + 64 * s + lane_addr;
+    const uint32_t tmem_o = tmem_base + 256 + 64 * s + lane_addr;
+    uint32_t g = 0;                               // sub-blocks done (buffer = g & 1)
+    uint32_t ow = 0, rw = 0;                      // o_full / r_full phases passed
+    bool ok = true;
+    for (int item = 2 * (int)blockIdx.x + hf; ok && item < p.total_items; item += item_step) {
+      const MsItem it = ms_item(p, item);
+      if (tile >= it.ntiles) continue;
+      const int m = it.row0 + tile * kMsBM + row;
+      const bool row_live = m < p.M;
+      const int64_t r_out = (int64_t)it.b * p.M + (row_live ? m : 0);
+      uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + it.h * kMsDH);
+      if (it.nb == 0) {
+        // no encoder position: the attention output is defined as zero
+        if (row_live) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+          if (p.lse != nullptr) p.lse[r_out * p.H + it.h] = -INFINITY;
+        }
+        continue;
+      }
+      const int nsub = (it.T + kMsSub - 1) / kMsSub;
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int u = 0; u < nsub; ++u, ++g) {
+        const uint32_t buf = g & 1;
+        ok = tc::mbar_wait(s_full + 2 * s + buf, (g >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc::tc_fence_after();
+        uint32_t r[kMsSub];
+        tc::tmem_ld32(tmem_s + kMsSub * buf, r);
+        tc::tmem_ld_wait();
+        const int valid = it.T - u * kMsSub;                        // positions of this sub-block that exist (>= 1)
+        if (valid < kMsSub) {
+#pragma unroll
+          for (int c = 0; c < kMsSub; ++c)
+            if (c >= valid) r[c] = 0xff800000u;                     // -inf: no weight, no influence on the maximum
+        }
+        float mx0 = ms_max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+        float mx1 = ms_max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+        float mx2 = ms_max3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
+        float mx3 = ms_max3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
+#pragma unroll
+        for (int c = 12; c + 7 < kMsSub; c += 8) {
+          mx0 = ms_max3(mx0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+          mx1 = ms_max3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+          mx2 = ms_max3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+          mx3 = ms_max3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
+        }
+        mx0 = ms_max3(mx0, __uint_as_float(r[kMsSub - 4]), __uint_as_float(r[kMsSub - 3]));
+        mx1 = ms_max3(mx1, __uint_as_float(r[kMsSub - 2]), __uint_as_float(r[kMsSub - 1]));
+        const float m_blk = fmaxf(ms_max3(mx0, mx1, mx2), mx3) * p.scale_log2;
+        // The accumulator is rescaled only when the row maximum grows by more than 2^16 over the
+        // reference in use (probabilities may then reach 65536, which bf16 and the fp32 sums hold
+        // without loss of precision); with scores of ordinary spread that never happens after the
+        // first sub-block.
+        const bool grow = m_blk > m_run + kMsGrowLog2;              // always true on the first sub-block
+        const float m_new = grow ? m_blk : m_run;
+        const float alpha = grow ? ms_ex2(m_run - m_new) : 1.0f;    // 0 on the first sub-block
+        m_run = m_new;
+        if (u > 0 && __any_sync(kFullMask, grow)) {
+          // O is about to change under the tensor core: P V of sub-block u - 1 must be complete.  It was
+          // issued before S of sub-block u + 1 (peeked here, consumed in the next iteration) or, in the
+          // item's last sub-block, before the commit on r_full.
+          if (u + 1 < nsub) ok = tc::mbar_wait(s_full + 2 * s + (buf ^ 1), ((g + 1) >> 1) & 1, abort_flag);
+          else ok = tc::mbar_wait(r_full + s, rw & 1, abort_flag);
+          if (!ok) break;
+          tc::tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < kMsDH; c += 16) {
+            uint32_t o[16];
+            tc::tmem_ld16(tmem_o + c, o);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tc::tmem_st16(tmem_o + c, o);
+          }
+        }
+        const float neg_m = -m_new;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMsSub / 4; ++c) {
+          const float e0 = ms_ex2(fmaf(__uint_as_float(r[4 * c]), p.scale_log2, neg_m));
+          const float e1 = ms_ex2(fmaf(__uint_as_float(r[4 * c + 1]), p.scale_log2, neg_m));
+          const float e2 = ms_ex2(fmaf(__uint_as_float(r[4 * c + 2]), p.scale_log2, neg_m));
+          const float e3 = ms_ex2(fmaf(__uint_as_float(r[4 * c + 3]), p.scale_log2, neg_m));
+          s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+          r[2 * c] = pack_bf16x2(e0, e1);
+          r[2 * c + 1] = pack_bf16x2(e2, e3);
+        }
+        l_run = fmaf(l_run, alpha, (s0 + s1) + (s2 + s3));
+        tc::tmem_st16(tmem_s + kMsSub * buf, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
+        tc::tmem_st_wait();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(p_full + 2 * s + buf);
+      }
+      if (!ok) break;
+      if (nsub >= 2) ++rw;
+      // ---- end of the item: O / l -> bf16 rows of out ----
+      ok = tc::mbar_wait(o_full + s, ow & 1, abort_flag);
+      if (!ok) break;
+      ++ow;
+      tc::tc_fence_after();
+      const float inv = 1.f / l_run;
+#pragma unroll
+      for (int c = 0; c < kMsDH; c += 32) {
+        uint32_t o[32];
+        tc::tmem_ld32(tmem_o + c, o);
+        tc::tmem_ld_wait();
+        if (row_live) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            dst[c / 8 + e] = make_uint4(
+                pack_bf16x2(__uint_as_float(o[8 * e]) * inv, __uint_as_float(o[8 * e + 1]) * inv),
+                pack_bf16x2(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv),
+                pack_bf16x2(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv),
+                pack_bf16x2(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv));
+        }
+      }
+      if (row_live && p.lse != nullptr) p.lse[r_out * p.H + it.h] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+      // The next item's first P V overwrites O; it is issued only after this stream's four warps have
+      // arrived on p_full, i.e. after these loads.
+      tc::tc_fence_before();
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == kMsSoftmaxWarps) tc::tmem_dealloc(tmem_base, 512);
+}
+
+inline bool cross_attn_ms_supported(int B, int M, int H, int d_h, int T_ctx) {
+  return d_h == 64 && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;
+}
+
+inline grace_status_t launch_cross_attn_ms(const uint16_t* q, int64_t q_row_stride, const uint16_t* k,
+                                           const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
+                                           int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
+                                           const int32_t* enc_len, int B, int M, int H, int T_ctx, float scale,
+                                           cudaStream_t s) {
+  CUtensorMap mq, mk, mv;
+  {
+    const uint64_t dims[4] = {(uint64_t)kMsDH, (uint64_t)H, (uint64_t)M, (uint64_t)B};
+    const uint64_t str[3] = {(uint64_t)kMsDH, (uint64_t)q_row_stride, (uint64_t)M * (uint64_t)q_row_stride};
+    const uint32_t box[4] = {64u, 1u, (uint32_t)kMsBM, 1u};
+    if (!tc::make_tmap_bf16(&mq, q, 4, dims, str, box)) return GRACE_CUDA_ERROR;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)kMsDH, (uint64_t)T_ctx, (uint64_t)H, (uint64_t)B};
+    const uint64_t str[3] = {(uint64_t)kv_stride_t, (uint64_t)kv_stride_h, (uint64_t)kv_stride_b};
+    const uint32_t box[4] = {64u, (uint32_t)kMsBN, 1u, 1u};
+    if (!tc::make_tmap_bf16(&mk, k, 4, dims, str, box)) return GRACE_CUDA_ERROR;
+    if (!tc::make_tmap_bf16(&mv, v, 4, dims, str, box)) return GRACE_CUDA_ERROR;
+  }
+  static unsigned long long attr_set_devices = 0;
+  if (first_use_on_device(&attr_set_devices)) {
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_ms_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMsSmemBytes));
+  }
+  int dev = 0, n_sm = 0;
+  GRACE_CUDA_TRY(cudaGetDevice(&dev));
+  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  CrossMsParams p;
+  p.out = out; p.lse = lse; p.enc_len = enc_len; p.out_row_stride = out_row_stride;
+  p.B = B; p.M = M; p.H = H; p.T = T_ctx;
+  p.pairs_m = (M + 2 * kMsBM - 1) / (2 * kMsBM);
+  const int64_t items = (int64_t)p.pairs_m * H * B;
+  if (items > 0x3fffffff) return GRACE_UNSUPPORTED_SHAPE;
+  p.total_items = (int)items;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  const int64_t ctas = (items + 1) / 2;
+  const int grid = (int)(ctas < n_sm ? ctas : n_sm);
+  launch_pdl(cross_attn_ms_kernel, dim3(grid), dim3(kMsThreads), kMsSmemBytes, s, mq, mk, mv, p);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
+}
+
+}  // namespace grace
