@@ -2,30 +2,37 @@
 // (Section 5.1: the beams of a request are the M dimension of a dense contraction against that
 // request's shared K/V).
 //
-// At head size 64 a 128 x 128 score block costs 512 tensor-core clocks but 16384 exponentials, and
-// the special-function unit takes one warp instruction per 8 clocks and scheduler: the exponentials
-// set the pace (1024 clocks per block and SM).  A single warp can issue an exponential only every
-// ~14 clocks, and every hand-off between warps or to the tensor core (mbarrier arrive -> wake,
-// MMA issue, commit -> wake) costs 150-250 clocks, so the unit stays busy only if several warps per
-// scheduler are in DIFFERENT phases of their blocks and never wait for one another.  Hence:
-//
+// What sets the pace at head size 64 (measured on B200, see the profiles directory):
+//   * a 128 x 128 score block costs 512 tensor-core clocks but 16384 exponentials; the special-function
+//     unit takes one warp instruction per 8 clocks and scheduler (1024 clocks per block and SM), and a
+//     single warp can issue an exponential only every ~14 clocks: several warps per scheduler have to
+//     be in the exponentials at any time;
+//   * every tcgen05.mma / tcgen05.commit costs 32-48 clocks to ISSUE, and issue is serialised over the
+//     whole SM whichever warp it comes from: the instruction count per block matters, not only the
+//     flops (score sub-blocks of 32 columns needed 36 instructions per block and were issue-bound);
+//   * every hand-off between warps or to the tensor core (mbarrier arrive -> wake, commit -> wake)
+//     costs 150-250 clocks.
+// Hence this layout:
 //   * one CTA per SM owns all 512 TMEM columns and runs four streams.  A stream is one 128-row
-//     query tile of one (request, head) with its own 64 score columns (S, fp32; the packed bf16
+//     query tile of one (request, head) with 64 score columns (S, fp32; the packed bf16
 //     probabilities P overwrite the first 32 of them) and 64 output columns (O, fp32) in TMEM, its
-//     own Q tile in shared memory and its own barriers;
+//     own Q tiles in shared memory and its own barriers;
 //   * streams 0/1 are the two tiles of one 256-row item and share that item's K/V ring, streams
 //     2/3 those of another item with a second ring: two independent halves, so a request needs
 //     only 256 beams to fill an SM;
-//   * a stream is served by four warps (one per TMEM lane quarter, one thread per query row):
-//     16 softmax warps, four per scheduler.  The stream's first warp also issues the stream's own
-//     MMAs: after the four warps have stored P of block j it issues O += P V_j and then S of block
-//     j + 1 (the in-order tensor pipe guarantees that S never overwrites a P still to be read).
-//     Nothing is exchanged between streams; their chains  S -> softmax -> P -> P V -> next S
-//     interleave freely, each running under the other three streams' exponentials;
-//   * encoder positions are cut in blocks of 64; K and V blocks arrive by TMA through four-slot
-//     rings per half; Q, K and V are addressed with 4-D tensor maps over the caller's strides, so
-//     the beam-major Q / O layout is never permuted.  A stream's Q tile is reloaded as soon as the
-//     last S of its item has run, i.e. under the item's last softmax and epilogue.
+//   * the encoder positions are walked in blocks of 64.  Four softmax warps per stream (one per
+//     TMEM lane quarter, one thread per query row: 16 warps, four per scheduler) turn S of a block
+//     into P; a fifth warp per stream issues the stream's MMAs in the order
+//         S(0);   O += P(u) V(u),  S(u + 1)   for u = 0, 1, ...
+//     running on into the next item (S(u + 1) overwrites the columns P(u) was read from; the
+//     in-order tensor pipe makes that safe).  A stream's chain  S -> softmax -> P -> P V, next S
+//     runs under the other three streams' exponentials; nothing is exchanged between streams;
+//   * K and V arrive by TMA in blocks of 64 positions through three-slot rings per half; Q tiles
+//     are double-buffered per stream, so the next item's first scores are computed under the
+//     current item's epilogue.  Q, K, V and the output are addressed with 4-D tensor maps over the
+//     caller's strides: the beam-major Q / O layout is never permuted;
+//   * the epilogue stages the bf16 output rows in the Q tile the item no longer needs and writes
+//     them with a TMA store per warp (rows beyond M are clipped by the tensor map).
 //
 // Ragged M and T are zero-filled by TMA and masked in the softmax; `enc_len` (optional) gives a
 // per-request number of valid encoder positions (0: the output rows are zero).  Every wait is
@@ -39,21 +46,23 @@ namespace grace {
 
 constexpr int kMsBM = 128;                 // query rows per tile (stream)
 constexpr int kMsBN = 64;                  // encoder positions per K / V block in shared memory
-constexpr int kMsSub = 32;                 // encoder positions per softmax sub-block (two per block)
+constexpr int kMsSub = 64;                 // encoder positions per softmax sub-block
+constexpr int kMsBufs = 64 / kMsSub;       // score buffers per stream (64 TMEM columns)
+constexpr int kMsSubPer = kMsBN / kMsSub;  // sub-blocks per K / V block
 constexpr float kMsGrowLog2 = 16.0f;       // the running reference maximum moves only when exceeded by this much
 constexpr int kMsDH = 64;
-constexpr int kMsStages = 4;               // K ring and V ring slots per half
+constexpr int kMsStages = 3;               // K ring and V ring slots per half
 constexpr int kMsQBytes = kMsBM * kMsDH * 2;       // 16 KB
 constexpr int kMsKVBytes = kMsBN * kMsDH * 2;      // 8 KB
 constexpr int kMsSoftmaxWarps = 16;
 constexpr int kMsThreads = (kMsSoftmaxWarps + 1 + 4) * 32;   // + producer + one MMA issuer per stream
 constexpr int kMsBarBytes = 1024;
-constexpr int kMsSmemBytes = 1024 + 4 * kMsQBytes + 2 * 2 * kMsStages * kMsKVBytes + kMsBarBytes;
+constexpr int kMsSmemBytes = 1024 + 8 * kMsQBytes + 2 * 2 * kMsStages * kMsKVBytes + kMsBarBytes;
 
 struct CrossMsParams {
-  uint16_t* out;
   float* lse;
   const int32_t* enc_len;       // nullable: valid encoder positions per request (<= T)
+  uint16_t* out;                // only for rows without any encoder position (written as zeros)
   int64_t out_row_stride;
   int B, M, H, T;
   int pairs_m, total_items;     // 256-row items per (request, head); items = B * H * pairs_m
@@ -90,16 +99,17 @@ __device__ __forceinline__ MsItem ms_item(const CrossMsParams& p, int item) {
 
 __global__ void __launch_bounds__(kMsThreads, 1)
 cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                     const __grid_constant__ CUtensorMap map_v, const CrossMsParams p) {
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o,
+                     const CrossMsParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* q_tiles = tiles;                                      // [stream] x 16 KB
-  uint8_t* k_tiles = tiles + 4 * kMsQBytes;                      // [half][slot] x 8 KB
+  uint8_t* q_tiles = tiles;                                      // [stream][buffer] x 16 KB
+  uint8_t* k_tiles = tiles + 8 * kMsQBytes;                      // [half][slot] x 8 KB
   uint8_t* v_tiles = k_tiles + 2 * kMsStages * kMsKVBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(v_tiles + 2 * kMsStages * kMsKVBytes);
-  uint64_t* q_full = bars;                          // [4] per stream
-  uint64_t* q_empty = q_full + 4;                   // [4]
-  uint64_t* k_full = q_empty + 4;                   // [2][kMsStages]
+  uint64_t* q_full = bars;                          // [4][2] per stream and buffer
+  uint64_t* q_empty = q_full + 8;                   // [4][2]  four arrivals: the stream's softmax warps, after their output stores
+  uint64_t* k_full = q_empty + 8;                   // [2][kMsStages]
   uint64_t* k_empty = k_full + 2 * kMsStages;       //        two arrivals: both streams of the half
   uint64_t* v_full = k_empty + 2 * kMsStages;
   uint64_t* v_empty = v_full + 2 * kMsStages;
@@ -113,12 +123,11 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 4; ++i) {
-      tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 1);
-      tc::mbar_init(s_full + 2 * i, 1); tc::mbar_init(s_full + 2 * i + 1, 1);
-      tc::mbar_init(p_full + 2 * i, 4); tc::mbar_init(p_full + 2 * i + 1, 4);
-      tc::mbar_init(o_full + i, 1); tc::mbar_init(r_full + i, 1);
+    for (int i = 0; i < 8; ++i) {
+      tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 4);
+      tc::mbar_init(s_full + i, 1); tc::mbar_init(p_full + i, 4);
     }
+    for (int i = 0; i < 4; ++i) { tc::mbar_init(o_full + i, 1); tc::mbar_init(r_full + i, 1); }
     for (int i = 0; i < 2 * kMsStages; ++i) {
       tc::mbar_init(k_full + i, 1); tc::mbar_init(k_empty + i, 2);
       tc::mbar_init(v_full + i, 1); tc::mbar_init(v_empty + i, 2);
@@ -140,10 +149,9 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (warp == kMsSoftmaxWarps) {
     // ---------------- TMA producer ----------------
     // Eight queues (Q per stream, K and V per half), fed by polling: whichever slot frees next gets
-    // its load, no queue blocks another.
+    // its load, no queue blocks another.  A queue's item is decoded when the queue moves on to it.
     if (lane == 0) {
       tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
-      // A queue's item is decoded when the queue moves on to it, not on every poll.
       int q_item[4], q_cnt[4];                      // item whose Q tile comes next; loads done
       int k_item[2], k_j[2], k_cnt[2], v_item[2], v_j[2], v_cnt[2];
       MsItem q_it[4], k_it[2], v_it[2];
@@ -167,11 +175,14 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (q_item[s] >= p.total_items) continue;
           more = true;
           bool advance = (s & 1) >= q_it[s].ntiles || q_it[s].nb == 0;      // nothing to load for this stream
-          if (!advance && tc::mbar_try_wait_now(q_empty + s, (q_cnt[s] & 1) ^ 1)) {
-            tc::mbar_expect_tx(q_full + s, kMsQBytes);
-            tc::tma_load_4d(q_tiles + s * kMsQBytes, &map_q, q_full + s, 0, q_it[s].h, q_it[s].row0 + (s & 1) * kMsBM, q_it[s].b);
-            ++q_cnt[s];
-            advance = true;
+          if (!advance) {
+            const int buf = 2 * s + (q_cnt[s] & 1);
+            if (tc::mbar_try_wait_now(q_empty + buf, ((q_cnt[s] >> 1) & 1) ^ 1)) {
+              tc::mbar_expect_tx(q_full + buf, kMsQBytes);
+              tc::tma_load_4d(q_tiles + buf * kMsQBytes, &map_q, q_full + buf, 0, q_it[s].h, q_it[s].row0 + (s & 1) * kMsBM, q_it[s].b);
+              ++q_cnt[s];
+              advance = true;
+            }
           }
           if (advance) {
             q_item[s] += item_step;
@@ -191,6 +202,7 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
               if (tc::mbar_try_wait_now(k_empty + slot, ((k_cnt[hf] / kMsStages) & 1) ^ 1)) {
                 tc::mbar_expect_tx(k_full + slot, kMsKVBytes);
                 tc::tma_load_4d(k_tiles + slot * kMsKVBytes, &map_k, k_full + slot, 0, k_j[hf] * kMsBN, k_it[hf].h, k_it[hf].b);
+                if (k_it[hf].ntiles == 1) tc::mbar_arrive(k_empty + slot);   // the half's second stream has no rows in this item
                 ++k_cnt[hf]; ++k_j[hf];
                 progressed = true;
               }
@@ -206,6 +218,7 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
               if (tc::mbar_try_wait_now(v_empty + slot, ((v_cnt[hf] / kMsStages) & 1) ^ 1)) {
                 tc::mbar_expect_tx(v_full + slot, kMsKVBytes);
                 tc::tma_load_4d(v_tiles + slot * kMsKVBytes, &map_v, v_full + slot, 0, v_j[hf] * kMsBN, v_it[hf].h, v_it[hf].b);
+                if (v_it[hf].ntiles == 1) tc::mbar_arrive(v_empty + slot);
                 ++v_cnt[hf]; ++v_j[hf];
                 progressed = true;
               }
@@ -215,7 +228,7 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (progressed) {
           idle = 0;
         } else {
-          __nanosleep(400);
+          __nanosleep(2000);
           if (++idle > (1 << 24)) {                          // bounded: seconds of nothing to do
             if (*abort_flag == 0) atomicAdd(&tc::g_tc_timeouts, 1);
             *abort_flag = 1;
@@ -226,9 +239,8 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   } else if (warp >= kMsSoftmaxWarps + 1) {
     // ---------------- MMA issuers, one warp per stream ----------------
     // The whole warp walks the loops and waits on the barriers; one elected lane issues (warp-uniform
-    // control flow keeps the descriptors in uniform registers).  Sequence per item with n sub-blocks:
-    //   S(0), S(1);  then for u = 0 .. n-1:  O += P(u) V(u);  S(u + 2)
-    // S(u + 2) overwrites the buffer P(u) was read from: the in-order tensor pipe makes that safe.
+    // control flow keeps the descriptors in uniform registers).  Two cursors run over the stream's
+    // sub-blocks, across items: the S cursor two sub-blocks ahead of the P V cursor.
     const int s = warp - (kMsSoftmaxWarps + 1);
     const int hf = s >> 1, tile = s & 1;
     const uint32_t tmem_s = tmem_base + 64 * s;             // two S / P buffers of 32 columns
@@ -236,80 +248,91 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     constexpr uint32_t idesc_s = tc::idesc_bf16(kMsBM, kMsSub, 0);    // Q K^T : B K-major, 32 score columns
     constexpr uint32_t idesc_o = tc::idesc_bf16(kMsBM, kMsDH, 1);     // P V   : B MN-major, 64 output columns
     // Operand descriptors differ only in their start address (bits 0..13, in 16-byte units).
-    const uint64_t q_desc = tc::smem_desc_sw128(tc::smem_addr(q_tiles + s * kMsQBytes), 16, 1024);
+    const uint64_t q_desc0 = tc::smem_desc_sw128(tc::smem_addr(q_tiles + 2 * s * kMsQBytes), 16, 1024);
     const uint64_t k_desc0 = tc::smem_desc_sw128(tc::smem_addr(k_tiles + hf * kMsStages * kMsKVBytes), 16, 1024);
     const uint64_t v_desc0 = tc::smem_desc_sw128(tc::smem_addr(v_tiles + hf * kMsStages * kMsKVBytes), 1024, 1024);
     uint64_t* const kf = k_full + hf * kMsStages;
     uint64_t* const ke = k_empty + hf * kMsStages;
     uint64_t* const vf = v_full + hf * kMsStages;
     uint64_t* const ve = v_empty + hf * kMsStages;
-    uint32_t g_s = 0, g_p = 0;                    // sub-blocks whose S / whose P V has been issued (buffer = index & 1)
-    uint32_t qc = 0, kc = 0, vc = 0;              // Q tiles, K blocks, V blocks consumed
     bool ok = true;
-    for (int item = 2 * (int)blockIdx.x + hf; ok && item < p.total_items; item += item_step) {
-      const MsItem it = ms_item(p, item);
-      if (tile >= it.ntiles) {
-        // No rows for this stream in the item: the half's other stream uses the K/V blocks alone,
-        // this one only hands them back (the slots count two arrivals).
-        for (int j = 0; ok && j < it.nb; ++j) {
-          ok = tc::mbar_wait(kf + kc % kMsStages, (kc / kMsStages) & 1, abort_flag);
-          if (ok && lane == 0) tc::mbar_arrive(ke + kc % kMsStages);
-          ++kc;
-          ok = ok && tc::mbar_wait(vf + vc % kMsStages, (vc / kMsStages) & 1, abort_flag);
-          if (ok && lane == 0) tc::mbar_arrive(ve + vc % kMsStages);
-          ++vc;
-        }
-        continue;
+    struct Cursor { int item, u, nsub; };
+    // Moves a cursor to the stream's next item that has work (rows for this tile and encoder positions).
+    uint32_t kc = 0, vc = 0;                      // K / V blocks consumed
+    auto seek = [&](Cursor& c) {
+      c.u = 0; c.nsub = 0;
+      while (c.item < p.total_items) {
+        const MsItem it = ms_item(p, c.item);
+        if (tile < it.ntiles && it.nb > 0) { c.nsub = (it.T + kMsSub - 1) / kMsSub; return; }
+        c.item += item_step;
       }
-      if (it.nb == 0) continue;
-      const int nsub = (it.T + kMsSub - 1) / kMsSub;
-      // S of sub-block u: K rows 32 (u & 1) .. + 31 of K block u >> 1
-      auto issue_s = [&](int u) -> bool {
-        if (u == 0 && !tc::mbar_wait(q_full + s, qc & 1, abort_flag)) return false;
-        const int slot = kc % kMsStages;
-        if ((u & 1) == 0 && !tc::mbar_wait(kf + slot, (kc / kMsStages) & 1, abort_flag)) return false;
-        tc::tc_fence_after();
-        const bool block_done = (u & 1) || u == nsub - 1;
-        if (tc::elect_one()) {
-          const uint64_t kd = k_desc0 + (uint64_t)((slot * kMsKVBytes + (u & 1) * (kMsSub * 128)) >> 4);
-          const uint32_t d = tmem_s + kMsSub * (g_s & 1);
+    };
+    Cursor cs = {2 * (int)blockIdx.x + hf, 0, 0}, cp = cs;
+    uint32_t g_s = 0, g_p = 0;                    // sub-blocks whose S / whose P V has been issued (buffer = index & 1)
+    uint32_t qs = 0;                              // Q tiles started by the S cursor (buffer = qs & 1)
+    seek(cs);
+    seek(cp);
+    // Everything an S needs besides its TMEM buffer: the item's Q tile (first sub-block) and the K block.
+    auto wait_s_operands = [&]() {
+      if (cs.u == 0) ok = ok && tc::mbar_wait_likely_done(q_full + 2 * s + (qs & 1), (qs >> 1) & 1, abort_flag);
+      if (cs.u % kMsSubPer == 0) ok = ok && tc::mbar_wait_likely_done(kf + kc % kMsStages, (kc / kMsStages) & 1, abort_flag);
+    };
+    // S of the S cursor's sub-block (elected lane)
+    auto fire_s = [&]() {
+      const int u = cs.u;
+      const int slot = kc % kMsStages;
+      const uint64_t qd = q_desc0 + (uint64_t)(((qs & 1) * kMsQBytes) >> 4);
+      const uint64_t kd = k_desc0 + (uint64_t)((slot * kMsKVBytes + (u % kMsSubPer) * (kMsSub * 128)) >> 4);
+      const uint32_t d = tmem_s + kMsSub * (g_s % kMsBufs);
+      tc::mma_ss_c<false>(d, qd, kd, idesc_s);
+      tc::mma_ss_c<true>(d, qd + 2, kd + 2, idesc_s);
+      tc::mma_ss_c<true>(d, qd + 4, kd + 4, idesc_s);
+      tc::mma_ss_c<true>(d, qd + 6, kd + 6, idesc_s);
+      tc::mma_commit(s_full + 2 * s + (g_s % kMsBufs));
+      if (u % kMsSubPer == kMsSubPer - 1 || u == cs.nsub - 1) tc::mma_commit(ke + slot);
+    };
+    auto advance_s = [&]() {
+      ++g_s;
+      if (cs.u % kMsSubPer == kMsSubPer - 1 || cs.u == cs.nsub - 1) ++kc;
+      if (++cs.u == cs.nsub) { ++qs; cs.item += item_step; seek(cs); }
+    };
+    for (int i = 0; i < kMsBufs && ok && cs.nsub; ++i) {
+      wait_s_operands();
+      if (!ok) break;
+      tc::tc_fence_after();
+      if (tc::elect_one()) fire_s();
+      __syncwarp();
+      advance_s();
+    }
+    while (ok && cp.nsub) {
+      // Operand waits first (normally long satisfied), so that nothing but the MMAs themselves stands
+      // between the arrival of P(u) and the completion of S(u + 2).
+      const int u = cp.u;
+      const int slot = vc % kMsStages;
+      if (u % kMsSubPer == 0) ok = tc::mbar_wait_likely_done(vf + slot, (vc / kMsStages) & 1, abort_flag);
+      const bool with_s = cs.nsub != 0;
+      if (with_s) wait_s_operands();
+      ok = ok && tc::mbar_wait(p_full + 2 * s + (g_p % kMsBufs), (g_p / kMsBufs) & 1, abort_flag);
+      if (!ok) break;
+      tc::tc_fence_after();
+      const bool block_done = u % kMsSubPer == kMsSubPer - 1 || u == cp.nsub - 1;
+      if (tc::elect_one()) {
+        const uint64_t vd = v_desc0 + (uint64_t)((slot * kMsKVBytes + (u % kMsSubPer) * (kMsSub * 128)) >> 4);
+        const uint32_t a = tmem_s + kMsSub * (g_p % kMsBufs);
+        if (u == 0) tc::mma_ts_c<false>(tmem_o, a, vd, idesc_o);
+        else tc::mma_ts_c<true>(tmem_o, a, vd, idesc_o);
 #pragma unroll
-          for (int k = 0; k < kMsDH / 16; ++k)
-            tc::mma_ss(d, q_desc + (uint64_t)((32 * k) >> 4), kd + (uint64_t)((32 * k) >> 4), idesc_s, k ? 1u : 0u);
-          tc::mma_commit(s_full + 2 * s + (g_s & 1));
-          if (block_done) tc::mma_commit(ke + slot);
-          if (u == nsub - 1) tc::mma_commit(q_empty + s);
-        }
-        __syncwarp();
-        ++g_s;
-        if (block_done) ++kc;
-        if (u == nsub - 1) ++qc;
-        return true;
-      };
-      ok = issue_s(0);
-      if (ok && nsub > 1) ok = issue_s(1);
-      for (int u = 0; ok && u < nsub; ++u) {
-        const int slot = vc % kMsStages;
-        if ((u & 1) == 0) ok = tc::mbar_wait(vf + slot, (vc / kMsStages) & 1, abort_flag);
-        ok = ok && tc::mbar_wait(p_full + 2 * s + (g_p & 1), (g_p >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc::tc_fence_after();
-        const bool block_done = (u & 1) || u == nsub - 1;
-        if (tc::elect_one()) {
-          const uint64_t vd = v_desc0 + (uint64_t)((slot * kMsKVBytes + (u & 1) * (kMsSub * 128)) >> 4);
-          const uint32_t a = tmem_s + kMsSub * (g_p & 1);
-#pragma unroll
-          for (int k = 0; k < kMsSub / 16; ++k)
-            tc::mma_ts(tmem_o, a + 8 * k, vd + (uint64_t)((2048 * k) >> 4), idesc_o, (u > 0 || k > 0) ? 1u : 0u);
-          if (block_done) tc::mma_commit(ve + slot);
-          if (u == nsub - 2) tc::mma_commit(r_full + s);       // for a late rescale of O in the last sub-block
-          if (u == nsub - 1) tc::mma_commit(o_full + s);
-        }
-        __syncwarp();
-        ++g_p;
-        if (block_done) ++vc;
-        if (u + 2 < nsub) ok = issue_s(u + 2);
+        for (int k = 1; k < kMsSub / 16; ++k) tc::mma_ts_c<true>(tmem_o, a + 8 * k, vd + 128 * k, idesc_o);
+        if (with_s) fire_s();
+        if (block_done) tc::mma_commit(ve + slot);
+        if (kMsBufs == 2 && u == cp.nsub - 2) tc::mma_commit(r_full + s);   // for a late rescale of O in the last sub-block
+        if (u == cp.nsub - 1) tc::mma_commit(o_full + s);
       }
+      __syncwarp();
+      ++g_p;
+      if (block_done) ++vc;
+      if (++cp.u == cp.nsub) { cp.item += item_step; seek(cp); }
+      if (with_s) advance_s();
     }
   } else {
     // ---------------- softmax: four warps per stream ----------------
@@ -322,17 +345,27 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t tmem_o = tmem_base + 256 + 64 * s + lane_addr;
     uint32_t g = 0;                               // sub-blocks done (buffer = g & 1)
     uint32_t ow = 0, rw = 0;                      // o_full / r_full phases passed
+    uint32_t qn = 0;                              // items with work so far (Q buffer = qn & 1)
+    int release = -1;                             // Q buffer whose output stores are still to be waited for
     bool ok = true;
+    // Once the output rows staged in a Q buffer have been read by the TMA store, the buffer goes back
+    // to the producer (one arrival per softmax warp).
+    auto release_q = [&]() {
+      if (release >= 0) {
+        if (lane == 0) { tc::bulk_wait_read<0>(); tc::mbar_arrive(q_empty + 2 * s + release); }
+        release = -1;
+      }
+    };
     for (int item = 2 * (int)blockIdx.x + hf; ok && item < p.total_items; item += item_step) {
       const MsItem it = ms_item(p, item);
       if (tile >= it.ntiles) continue;
       const int m = it.row0 + tile * kMsBM + row;
       const bool row_live = m < p.M;
       const int64_t r_out = (int64_t)it.b * p.M + (row_live ? m : 0);
-      uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + it.h * kMsDH);
       if (it.nb == 0) {
         // no encoder position: the attention output is defined as zero
         if (row_live) {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + it.h * kMsDH);
 #pragma unroll
           for (int e = 0; e < 8; ++e) dst[e] = make_uint4(0u, 0u, 0u, 0u);
           if (p.lse != nullptr) p.lse[r_out * p.H + it.h] = -INFINITY;
@@ -342,12 +375,13 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       const int nsub = (it.T + kMsSub - 1) / kMsSub;
       float m_run = -INFINITY, l_run = 0.f;
       for (int u = 0; u < nsub; ++u, ++g) {
-        const uint32_t buf = g & 1;
-        ok = tc::mbar_wait(s_full + 2 * s + buf, (g >> 1) & 1, abort_flag);
+        const uint32_t buf = g % kMsBufs;
+        ok = tc::mbar_wait_likely_done(s_full + 2 * s + buf, (g / kMsBufs) & 1, abort_flag);
         if (!ok) break;
         tc::tc_fence_after();
         uint32_t r[kMsSub];
-        tc::tmem_ld32(tmem_s + kMsSub * buf, r);
+#pragma unroll
+        for (int c = 0; c < kMsSub; c += 32) tc::tmem_ld32(tmem_s + kMsSub * buf + c, *reinterpret_cast<uint32_t(*)[32]>(&r[c]));
         tc::tmem_ld_wait();
         const int valid = it.T - u * kMsSub;                        // positions of this sub-block that exist (>= 1)
         if (valid < kMsSub) {
@@ -381,9 +415,11 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // O is about to change under the tensor core: P V of sub-block u - 1 must be complete.  It was
           // issued before S of sub-block u + 1 (peeked here, consumed in the next iteration) or, in the
           // item's last sub-block, before the commit on r_full.
-          if (u + 1 < nsub) ok = tc::mbar_wait(s_full + 2 * s + (buf ^ 1), ((g + 1) >> 1) & 1, abort_flag);
-          else ok = tc::mbar_wait(r_full + s, rw & 1, abort_flag);
-          if (!ok) break;
+          if (kMsBufs == 2) {                     // (with one buffer this sub-block's S was itself issued after that P V)
+            if (u + 1 < nsub) ok = tc::mbar_wait(s_full + 2 * s + (buf ^ 1), ((g + 1) >> 1) & 1, abort_flag);
+            else ok = tc::mbar_wait(r_full + s, rw & 1, abort_flag);
+            if (!ok) break;
+          }
           tc::tc_fence_after();
 #pragma unroll
           for (int c = 0; c < kMsDH; c += 16) {
@@ -408,40 +444,53 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           r[2 * c + 1] = pack_bf16x2(e2, e3);
         }
         l_run = fmaf(l_run, alpha, (s0 + s1) + (s2 + s3));
-        tc::tmem_st16(tmem_s + kMsSub * buf, *reinterpret_cast<uint32_t(*)[16]>(&r[0]));
+#pragma unroll
+        for (int c = 0; c < kMsSub / 2; c += 16) tc::tmem_st16(tmem_s + kMsSub * buf + c, *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
         tc::tmem_st_wait();
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(p_full + 2 * s + buf);
+        if (u == 0) release_q();                  // the previous item's output stores have long been read
       }
       if (!ok) break;
       if (nsub >= 2) ++rw;
-      // ---- end of the item: O / l -> bf16 rows of out ----
+      // ---- end of the item: O / l -> bf16 rows, staged in the item's Q tile, TMA store per warp ----
       ok = tc::mbar_wait(o_full + s, ow & 1, abort_flag);
       if (!ok) break;
       ++ow;
       tc::tc_fence_after();
+      const uint32_t qb = qn & 1;
+      ++qn;
       const float inv = 1.f / l_run;
+      uint8_t* stage_row = q_tiles + (2 * s + qb) * kMsQBytes + row * 128;     // 128-byte swizzle: chunk j of row r at j ^ (r & 7)
 #pragma unroll
       for (int c = 0; c < kMsDH; c += 32) {
         uint32_t o[32];
         tc::tmem_ld32(tmem_o + c, o);
         tc::tmem_ld_wait();
-        if (row_live) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            dst[c / 8 + e] = make_uint4(
-                pack_bf16x2(__uint_as_float(o[8 * e]) * inv, __uint_as_float(o[8 * e + 1]) * inv),
-                pack_bf16x2(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv),
-                pack_bf16x2(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv),
-                pack_bf16x2(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv));
+        for (int e = 0; e < 4; ++e) {
+          const uint4 w = make_uint4(
+              pack_bf16x2(__uint_as_float(o[8 * e]) * inv, __uint_as_float(o[8 * e + 1]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv));
+          *reinterpret_cast<uint4*>(stage_row + (((c / 8 + e) ^ (row & 7)) << 4)) = w;
         }
       }
-      if (row_live && p.lse != nullptr) p.lse[r_out * p.H + it.h] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       // The next item's first P V overwrites O; it is issued only after this stream's four warps have
       // arrived on p_full, i.e. after these loads.
       tc::tc_fence_before();
+      tc::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0 && it.row0 + tile * kMsBM + q * 32 < p.M) {
+        tc::tma_store_4d(&map_o, q_tiles + (2 * s + qb) * kMsQBytes + q * 32 * 128, 0, it.h, it.row0 + tile * kMsBM + q * 32, it.b);
+        tc::bulk_commit();
+      }
+      release = (int)qb;
+      if (row_live && p.lse != nullptr) p.lse[r_out * p.H + it.h] = (m_run + log2f(l_run)) * 0.6931471805599453f;
     }
+    if (lane == 0) tc::bulk_wait_all();           // shared memory stays valid until the last stores have read it
   }
   tc::tc_fence_before();
   __syncthreads();
@@ -457,12 +506,15 @@ inline grace_status_t launch_cross_attn_ms(const uint16_t* q, int64_t q_row_stri
                                            int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
                                            const int32_t* enc_len, int B, int M, int H, int T_ctx, float scale,
                                            cudaStream_t s) {
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mk, mv, mo;
   {
     const uint64_t dims[4] = {(uint64_t)kMsDH, (uint64_t)H, (uint64_t)M, (uint64_t)B};
     const uint64_t str[3] = {(uint64_t)kMsDH, (uint64_t)q_row_stride, (uint64_t)M * (uint64_t)q_row_stride};
     const uint32_t box[4] = {64u, 1u, (uint32_t)kMsBM, 1u};
     if (!tc::make_tmap_bf16(&mq, q, 4, dims, str, box)) return GRACE_CUDA_ERROR;
+    const uint64_t ostr[3] = {(uint64_t)kMsDH, (uint64_t)out_row_stride, (uint64_t)M * (uint64_t)out_row_stride};
+    const uint32_t obox[4] = {64u, 1u, 32u, 1u};                       // one softmax warp's rows
+    if (!tc::make_tmap_bf16(&mo, out, 4, dims, ostr, obox)) return GRACE_CUDA_ERROR;
   }
   {
     const uint64_t dims[4] = {(uint64_t)kMsDH, (uint64_t)T_ctx, (uint64_t)H, (uint64_t)B};
@@ -488,7 +540,7 @@ inline grace_status_t launch_cross_attn_ms(const uint16_t* q, int64_t q_row_stri
   p.scale_log2 = scale * 1.4426950408889634f;
   const int64_t ctas = (items + 1) / 2;
   const int grid = (int)(ctas < n_sm ? ctas : n_sm);
-  launch_pdl(cross_attn_ms_kernel, dim3(grid), dim3(kMsThreads), kMsSmemBytes, s, mq, mk, mv, p);
+  launch_pdl(cross_attn_ms_kernel, dim3(grid), dim3(kMsThreads), kMsSmemBytes, s, mq, mk, mv, mo, p);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
