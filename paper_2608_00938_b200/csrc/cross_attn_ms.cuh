@@ -46,18 +46,15 @@ namespace grace {
 
 constexpr int kMsBM = 128;                 // query rows per tile (stream)
 constexpr int kMsBN = 64;                  // encoder positions per K / V block in shared memory
-constexpr int kMsSub = 64;                 // encoder positions per softmax sub-block
-constexpr int kMsBufs = 64 / kMsSub;       // score buffers per stream (64 TMEM columns)
-constexpr int kMsSubPer = kMsBN / kMsSub;  // sub-blocks per K / V block
 constexpr float kMsGrowLog2 = 16.0f;       // the running reference maximum moves only when exceeded by this much
 constexpr int kMsDH = 64;
-constexpr int kMsStages = 3;               // K ring and V ring slots per half
+constexpr int kMsStages = 3;               // K/V ring slots per half; a slot holds K and V of one block
 constexpr int kMsQBytes = kMsBM * kMsDH * 2;       // 16 KB
 constexpr int kMsKVBytes = kMsBN * kMsDH * 2;      // 8 KB
 constexpr int kMsSoftmaxWarps = 16;
-constexpr int kMsThreads = (kMsSoftmaxWarps + 1 + 4) * 32;   // + producer + one MMA issuer per stream
+constexpr int kMsThreads = (kMsSoftmaxWarps + 4) * 32;   // + one MMA issuer / TMA producer warp per stream
 constexpr int kMsBarBytes = 1024;
-constexpr int kMsSmemBytes = 1024 + 8 * kMsQBytes + 2 * 2 * kMsStages * kMsKVBytes + kMsBarBytes;
+constexpr int kMsSmemBytes = 1024 + 8 * kMsQBytes + 2 * kMsStages * 2 * kMsKVBytes + kMsBarBytes;
 
 struct CrossMsParams {
   float* lse;
@@ -104,34 +101,24 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_tiles = tiles;                                      // [stream][buffer] x 16 KB
-  uint8_t* k_tiles = tiles + 8 * kMsQBytes;                      // [half][slot] x 8 KB
-  uint8_t* v_tiles = k_tiles + 2 * kMsStages * kMsKVBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(v_tiles + 2 * kMsStages * kMsKVBytes);
+  uint8_t* kv_tiles = tiles + 8 * kMsQBytes;                     // [half][slot] x (K 8 KB, V 8 KB)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(kv_tiles + 2 * kMsStages * 2 * kMsKVBytes);
   uint64_t* q_full = bars;                          // [4][2] per stream and buffer
   uint64_t* q_empty = q_full + 8;                   // [4][2]  four arrivals: the stream's softmax warps, after their output stores
-  uint64_t* k_full = q_empty + 8;                   // [2][kMsStages]
-  uint64_t* k_empty = k_full + 2 * kMsStages;       //        two arrivals: both streams of the half
-  uint64_t* v_full = k_empty + 2 * kMsStages;
-  uint64_t* v_empty = v_full + 2 * kMsStages;
-  uint64_t* s_full = v_empty + 2 * kMsStages;       // [4][2] S of a sub-block is in the stream's TMEM buffer
-  uint64_t* p_full = s_full + 8;                    // [4][2] the stream's four warps have stored P there
-  uint64_t* o_full = p_full + 8;                    // [4] the stream's last P V of the item is done
-  uint64_t* r_full = o_full + 4;                    // [4] the stream's last but one P V of the item is done
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(r_full + 4);
+  uint64_t* kv_full = q_empty + 8;                  // [2][kMsStages]
+  uint64_t* kv_empty = kv_full + 2 * kMsStages;     //        two arrivals: both streams of the half
+  uint64_t* s_full = kv_empty + 2 * kMsStages;      // [4] S of the stream's next block is in TMEM
+  uint64_t* p_full = s_full + 4;                    // [4] the stream's four warps have stored P
+  uint64_t* o_full = p_full + 4;                    // [4] the stream's last P V of the item is done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 8; ++i) {
-      tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 4);
-      tc::mbar_init(s_full + i, 1); tc::mbar_init(p_full + i, 4);
-    }
-    for (int i = 0; i < 4; ++i) { tc::mbar_init(o_full + i, 1); tc::mbar_init(r_full + i, 1); }
-    for (int i = 0; i < 2 * kMsStages; ++i) {
-      tc::mbar_init(k_full + i, 1); tc::mbar_init(k_empty + i, 2);
-      tc::mbar_init(v_full + i, 1); tc::mbar_init(v_empty + i, 2);
-    }
+    for (int i = 0; i < 8; ++i) { tc::mbar_init(q_full + i, 1); tc::mbar_init(q_empty + i, 4); }
+    for (int i = 0; i < 4; ++i) { tc::mbar_init(s_full + i, 1); tc::mbar_init(p_full + i, 4); tc::mbar_init(o_full + i, 1); }
+    for (int i = 0; i < 2 * kMsStages; ++i) { tc::mbar_init(kv_full + i, 1); tc::mbar_init(kv_empty + i, 2); }
     *abort_flag = 0;
     tc::fence_mbar_init();
   }
@@ -146,193 +133,173 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   // CTA and neighbouring CTAs run neighbouring items, which share K/V in L2.
   const int item_step = 2 * (int)gridDim.x;
 
-  if (warp == kMsSoftmaxWarps) {
-    // ---------------- TMA producer ----------------
-    // Eight queues (Q per stream, K and V per half), fed by polling: whichever slot frees next gets
-    // its load, no queue blocks another.  A queue's item is decoded when the queue moves on to it.
-    if (lane == 0) {
-      tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v);
-      int q_item[4], q_cnt[4];                      // item whose Q tile comes next; loads done
-      int k_item[2], k_j[2], k_cnt[2], v_item[2], v_j[2], v_cnt[2];
-      MsItem q_it[4], k_it[2], v_it[2];
-      const MsItem none = {0, 0, 0, 0, 0, 0};
-      for (int s = 0; s < 4; ++s) {
-        q_item[s] = 2 * (int)blockIdx.x + (s >> 1); q_cnt[s] = 0;
-        q_it[s] = q_item[s] < p.total_items ? ms_item(p, q_item[s]) : none;
-      }
-      for (int hf = 0; hf < 2; ++hf) {
-        k_item[hf] = v_item[hf] = 2 * (int)blockIdx.x + hf;
-        k_j[hf] = v_j[hf] = 0; k_cnt[hf] = v_cnt[hf] = 0;
-        k_it[hf] = v_it[hf] = k_item[hf] < p.total_items ? ms_item(p, k_item[hf]) : none;
-      }
-      int idle = 0;
-      bool more = true;
-      while (more && !*abort_flag) {
-        bool progressed = false;
-        more = false;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          if (q_item[s] >= p.total_items) continue;
-          more = true;
-          bool advance = (s & 1) >= q_it[s].ntiles || q_it[s].nb == 0;      // nothing to load for this stream
-          if (!advance) {
-            const int buf = 2 * s + (q_cnt[s] & 1);
-            if (tc::mbar_try_wait_now(q_empty + buf, ((q_cnt[s] >> 1) & 1) ^ 1)) {
-              tc::mbar_expect_tx(q_full + buf, kMsQBytes);
-              tc::tma_load_4d(q_tiles + buf * kMsQBytes, &map_q, q_full + buf, 0, q_it[s].h, q_it[s].row0 + (s & 1) * kMsBM, q_it[s].b);
-              ++q_cnt[s];
-              advance = true;
-            }
-          }
-          if (advance) {
-            q_item[s] += item_step;
-            if (q_item[s] < p.total_items) q_it[s] = ms_item(p, q_item[s]);
-            progressed = true;
-          }
-        }
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          if (k_item[hf] < p.total_items) {
-            more = true;
-            if (k_j[hf] >= k_it[hf].nb) {
-              k_item[hf] += item_step; k_j[hf] = 0; progressed = true;
-              if (k_item[hf] < p.total_items) k_it[hf] = ms_item(p, k_item[hf]);
-            } else {
-              const int slot = hf * kMsStages + k_cnt[hf] % kMsStages;
-              if (tc::mbar_try_wait_now(k_empty + slot, ((k_cnt[hf] / kMsStages) & 1) ^ 1)) {
-                tc::mbar_expect_tx(k_full + slot, kMsKVBytes);
-                tc::tma_load_4d(k_tiles + slot * kMsKVBytes, &map_k, k_full + slot, 0, k_j[hf] * kMsBN, k_it[hf].h, k_it[hf].b);
-                if (k_it[hf].ntiles == 1) tc::mbar_arrive(k_empty + slot);   // the half's second stream has no rows in this item
-                ++k_cnt[hf]; ++k_j[hf];
-                progressed = true;
-              }
-            }
-          }
-          if (v_item[hf] < p.total_items) {
-            more = true;
-            if (v_j[hf] >= v_it[hf].nb) {
-              v_item[hf] += item_step; v_j[hf] = 0; progressed = true;
-              if (v_item[hf] < p.total_items) v_it[hf] = ms_item(p, v_item[hf]);
-            } else if (v_cnt[hf] < k_cnt[hf]) {                  // K of a block is wanted before its V
-              const int slot = hf * kMsStages + v_cnt[hf] % kMsStages;
-              if (tc::mbar_try_wait_now(v_empty + slot, ((v_cnt[hf] / kMsStages) & 1) ^ 1)) {
-                tc::mbar_expect_tx(v_full + slot, kMsKVBytes);
-                tc::tma_load_4d(v_tiles + slot * kMsKVBytes, &map_v, v_full + slot, 0, v_j[hf] * kMsBN, v_it[hf].h, v_it[hf].b);
-                if (v_it[hf].ntiles == 1) tc::mbar_arrive(v_empty + slot);
-                ++v_cnt[hf]; ++v_j[hf];
-                progressed = true;
-              }
-            }
-          }
-        }
-        if (progressed) {
-          idle = 0;
-        } else {
-          __nanosleep(2000);
-          if (++idle > (1 << 24)) {                          // bounded: seconds of nothing to do
-            if (*abort_flag == 0) atomicAdd(&tc::g_tc_timeouts, 1);
-            *abort_flag = 1;
-          }
-        }
-      }
-    }
-  } else if (warp >= kMsSoftmaxWarps + 1) {
-    // ---------------- MMA issuers, one warp per stream ----------------
-    // The whole warp walks the loops and waits on the barriers; one elected lane issues (warp-uniform
-    // control flow keeps the descriptors in uniform registers).  Two cursors run over the stream's
-    // sub-blocks, across items: the S cursor two sub-blocks ahead of the P V cursor.
-    const int s = warp - (kMsSoftmaxWarps + 1);
+  if (warp >= kMsSoftmaxWarps) {
+    // ---------------- MMA issuer and TMA producer, one warp per stream ----------------
+    // The whole warp walks the loops and tests the barriers; one elected lane issues (warp-uniform
+    // control flow keeps the descriptors in uniform registers).  MMA order per stream, across items:
+    //     S(0);   O += P(u) V(u),  S(u + 1)   for u = 0, 1, ...
+    // The warp also requests the stream's Q tiles and, for the first stream of a half, the half's
+    // K/V blocks: whenever it has to wait it first looks for a free slot to fill (refill), so loads
+    // run ahead of the MMAs without a polling warp of their own.
+    const int s = warp - kMsSoftmaxWarps;
     const int hf = s >> 1, tile = s & 1;
-    const uint32_t tmem_s = tmem_base + 64 * s;             // two S / P buffers of 32 columns
+    const uint32_t tmem_s = tmem_base + 64 * s;
     const uint32_t tmem_o = tmem_base + 256 + 64 * s;
-    constexpr uint32_t idesc_s = tc::idesc_bf16(kMsBM, kMsSub, 0);    // Q K^T : B K-major, 32 score columns
+    constexpr uint32_t idesc_s = tc::idesc_bf16(kMsBM, kMsBN, 0);     // Q K^T : B K-major, 64 score columns
     constexpr uint32_t idesc_o = tc::idesc_bf16(kMsBM, kMsDH, 1);     // P V   : B MN-major, 64 output columns
     // Operand descriptors differ only in their start address (bits 0..13, in 16-byte units).
     const uint64_t q_desc0 = tc::smem_desc_sw128(tc::smem_addr(q_tiles + 2 * s * kMsQBytes), 16, 1024);
-    const uint64_t k_desc0 = tc::smem_desc_sw128(tc::smem_addr(k_tiles + hf * kMsStages * kMsKVBytes), 16, 1024);
-    const uint64_t v_desc0 = tc::smem_desc_sw128(tc::smem_addr(v_tiles + hf * kMsStages * kMsKVBytes), 1024, 1024);
-    uint64_t* const kf = k_full + hf * kMsStages;
-    uint64_t* const ke = k_empty + hf * kMsStages;
-    uint64_t* const vf = v_full + hf * kMsStages;
-    uint64_t* const ve = v_empty + hf * kMsStages;
+    uint8_t* const kv_half = kv_tiles + hf * kMsStages * 2 * kMsKVBytes;
+    const uint64_t k_desc0 = tc::smem_desc_sw128(tc::smem_addr(kv_half), 16, 1024);
+    const uint64_t v_desc0 = tc::smem_desc_sw128(tc::smem_addr(kv_half + kMsKVBytes), 1024, 1024);
+    uint64_t* const kvf = kv_full + hf * kMsStages;
+    uint64_t* const kve = kv_empty + hf * kMsStages;
     bool ok = true;
-    struct Cursor { int item, u, nsub; };
+    if (lane == 0) { tc::tma_prefetch_desc(&map_q); tc::tma_prefetch_desc(&map_k); tc::tma_prefetch_desc(&map_v); }
+
+    // ---- loads ----
+    int lq_item = 2 * (int)blockIdx.x + hf, lq_cnt = 0;           // Q: next item to look at; tiles requested
+    int lk_item = lq_item, lk_j = 0, lk_cnt = 0;                  // K/V (first stream of the half only): item, block, blocks requested
+    MsItem lk_it = lk_item < p.total_items ? ms_item(p, lk_item) : MsItem{0, 0, 0, 0, 0, 0};
+    MsItem lq_it = lk_it;                                          // an item is decoded when a queue moves on to it
+    auto refill = [&]() -> bool {
+      bool progressed = false;
+      if (lq_item < p.total_items) {
+        const MsItem& it = lq_it;
+        bool advance = tile >= it.ntiles || it.nb == 0;             // nothing to load for this stream
+        if (!advance) {
+          const int buf = 2 * s + (lq_cnt & 1);
+          if (tc::mbar_try_wait_now(q_empty + buf, ((lq_cnt >> 1) & 1) ^ 1)) {
+            if (tc::elect_one()) {
+              tc::mbar_expect_tx(q_full + buf, kMsQBytes);
+              tc::tma_load_4d(q_tiles + buf * kMsQBytes, &map_q, q_full + buf, 0, it.h, it.row0 + tile * kMsBM, it.b);
+            }
+            __syncwarp();
+            ++lq_cnt;
+            advance = true;
+          }
+        }
+        if (advance) {
+          lq_item += item_step; progressed = true;
+          if (lq_item < p.total_items) lq_it = ms_item(p, lq_item);
+        }
+      }
+      if (tile == 0 && lk_item < p.total_items) {
+        if (lk_j >= lk_it.nb) {
+          lk_item += item_step; lk_j = 0; progressed = true;
+          if (lk_item < p.total_items) lk_it = ms_item(p, lk_item);
+        } else {
+          const int slot = lk_cnt % kMsStages;
+          if (tc::mbar_try_wait_now(kve + slot, ((lk_cnt / kMsStages) & 1) ^ 1)) {
+            if (tc::elect_one()) {
+              uint8_t* dst = kv_half + slot * 2 * kMsKVBytes;
+              tc::mbar_expect_tx(kvf + slot, 2 * kMsKVBytes);
+              tc::tma_load_4d(dst, &map_k, kvf + slot, 0, lk_j * kMsBN, lk_it.h, lk_it.b);
+              tc::tma_load_4d(dst + kMsKVBytes, &map_v, kvf + slot, 0, lk_j * kMsBN, lk_it.h, lk_it.b);
+              if (lk_it.ntiles == 1) tc::mbar_arrive(kve + slot);     // the half's second stream has no rows in this item
+            }
+            __syncwarp();
+            ++lk_cnt; ++lk_j;
+            progressed = true;
+          }
+        }
+      }
+      return progressed;
+    };
+    // A wait that keeps the loads going: test, refill, and only then park for a short while.
+    auto wait_refilling = [&](uint64_t* bar, uint32_t parity) {
+      int polls = 0;
+      while (ok && !tc::mbar_try_wait_now(bar, parity)) {
+        if (refill()) continue;
+        if (tc::mbar_try_wait_ns(bar, parity, 1000)) break;
+        if (*abort_flag) ok = false;
+        else if (++polls > (1 << 21)) {                             // bounded: seconds
+          if (lane == 0) atomicAdd(&tc::g_tc_timeouts, 1);
+          *abort_flag = 1;
+          ok = false;
+        }
+      }
+    };
+    while (refill()) {}
+
+    // ---- MMAs ----
+    struct Cursor { int item, u, nb; };
     // Moves a cursor to the stream's next item that has work (rows for this tile and encoder positions).
-    uint32_t kc = 0, vc = 0;                      // K / V blocks consumed
     auto seek = [&](Cursor& c) {
-      c.u = 0; c.nsub = 0;
+      c.u = 0; c.nb = 0;
       while (c.item < p.total_items) {
         const MsItem it = ms_item(p, c.item);
-        if (tile < it.ntiles && it.nb > 0) { c.nsub = (it.T + kMsSub - 1) / kMsSub; return; }
+        if (tile < it.ntiles && it.nb > 0) { c.nb = it.nb; return; }
         c.item += item_step;
       }
     };
     Cursor cs = {2 * (int)blockIdx.x + hf, 0, 0}, cp = cs;
-    uint32_t g_s = 0, g_p = 0;                    // sub-blocks whose S / whose P V has been issued (buffer = index & 1)
+    uint32_t kc = 0, vc = 0;                      // blocks whose S / whose P V has been issued (ring slot = count % stages)
     uint32_t qs = 0;                              // Q tiles started by the S cursor (buffer = qs & 1)
+    uint32_t pw = 0;                              // p_full phases consumed
     seek(cs);
     seek(cp);
-    // Everything an S needs besides its TMEM buffer: the item's Q tile (first sub-block) and the K block.
     auto wait_s_operands = [&]() {
-      if (cs.u == 0) ok = ok && tc::mbar_wait_likely_done(q_full + 2 * s + (qs & 1), (qs >> 1) & 1, abort_flag);
-      if (cs.u % kMsSubPer == 0) ok = ok && tc::mbar_wait_likely_done(kf + kc % kMsStages, (kc / kMsStages) & 1, abort_flag);
+      if (cs.u == 0) wait_refilling(q_full + 2 * s + (qs & 1), (qs >> 1) & 1);
+      wait_refilling(kvf + kc % kMsStages, (kc / kMsStages) & 1);
     };
-    // S of the S cursor's sub-block (elected lane)
-    auto fire_s = [&]() {
-      const int u = cs.u;
-      const int slot = kc % kMsStages;
+    auto fire_s = [&]() {                         // elected lane
       const uint64_t qd = q_desc0 + (uint64_t)(((qs & 1) * kMsQBytes) >> 4);
-      const uint64_t kd = k_desc0 + (uint64_t)((slot * kMsKVBytes + (u % kMsSubPer) * (kMsSub * 128)) >> 4);
-      const uint32_t d = tmem_s + kMsSub * (g_s % kMsBufs);
-      tc::mma_ss_c<false>(d, qd, kd, idesc_s);
-      tc::mma_ss_c<true>(d, qd + 2, kd + 2, idesc_s);
-      tc::mma_ss_c<true>(d, qd + 4, kd + 4, idesc_s);
-      tc::mma_ss_c<true>(d, qd + 6, kd + 6, idesc_s);
-      tc::mma_commit(s_full + 2 * s + (g_s % kMsBufs));
-      if (u % kMsSubPer == kMsSubPer - 1 || u == cs.nsub - 1) tc::mma_commit(ke + slot);
+      const uint64_t kd = k_desc0 + (uint64_t)(((kc % kMsStages) * 2 * kMsKVBytes) >> 4);
+      tc::mma_ss_c<false>(tmem_s, qd, kd, idesc_s);
+      tc::mma_ss_c<true>(tmem_s, qd + 2, kd + 2, idesc_s);
+      tc::mma_ss_c<true>(tmem_s, qd + 4, kd + 4, idesc_s);
+      tc::mma_ss_c<true>(tmem_s, qd + 6, kd + 6, idesc_s);
+      tc::mma_commit(s_full + s);
     };
     auto advance_s = [&]() {
-      ++g_s;
-      if (cs.u % kMsSubPer == kMsSubPer - 1 || cs.u == cs.nsub - 1) ++kc;
-      if (++cs.u == cs.nsub) { ++qs; cs.item += item_step; seek(cs); }
+      ++kc;
+      if (++cs.u == cs.nb) { ++qs; cs.item += item_step; seek(cs); }
     };
-    for (int i = 0; i < kMsBufs && ok && cs.nsub; ++i) {
+    if (cs.nb) {
       wait_s_operands();
-      if (!ok) break;
-      tc::tc_fence_after();
-      if (tc::elect_one()) fire_s();
-      __syncwarp();
-      advance_s();
+      if (ok) {
+        tc::tc_fence_after();
+        if (tc::elect_one()) fire_s();
+        __syncwarp();
+        advance_s();
+      }
     }
-    while (ok && cp.nsub) {
+    while (ok && cp.nb) {
       // Operand waits first (normally long satisfied), so that nothing but the MMAs themselves stands
-      // between the arrival of P(u) and the completion of S(u + 2).
+      // between the arrival of P(u) and the completion of S(u + 1).
       const int u = cp.u;
-      const int slot = vc % kMsStages;
-      if (u % kMsSubPer == 0) ok = tc::mbar_wait_likely_done(vf + slot, (vc / kMsStages) & 1, abort_flag);
-      const bool with_s = cs.nsub != 0;
+      const bool with_s = cs.nb != 0;
       if (with_s) wait_s_operands();
-      ok = ok && tc::mbar_wait(p_full + 2 * s + (g_p % kMsBufs), (g_p / kMsBufs) & 1, abort_flag);
+      wait_refilling(p_full + s, pw & 1);
       if (!ok) break;
+      ++pw;
       tc::tc_fence_after();
-      const bool block_done = u % kMsSubPer == kMsSubPer - 1 || u == cp.nsub - 1;
+      const uint32_t slot = vc % kMsStages;
       if (tc::elect_one()) {
-        const uint64_t vd = v_desc0 + (uint64_t)((slot * kMsKVBytes + (u % kMsSubPer) * (kMsSub * 128)) >> 4);
-        const uint32_t a = tmem_s + kMsSub * (g_p % kMsBufs);
-        if (u == 0) tc::mma_ts_c<false>(tmem_o, a, vd, idesc_o);
-        else tc::mma_ts_c<true>(tmem_o, a, vd, idesc_o);
-#pragma unroll
-        for (int k = 1; k < kMsSub / 16; ++k) tc::mma_ts_c<true>(tmem_o, a + 8 * k, vd + 128 * k, idesc_o);
+        const uint64_t vd = v_desc0 + (uint64_t)((slot * 2 * kMsKVBytes) >> 4);
+        if (u == 0) tc::mma_ts_c<false>(tmem_o, tmem_s, vd, idesc_o);
+        else tc::mma_ts_c<true>(tmem_o, tmem_s, vd, idesc_o);
+        tc::mma_ts_c<true>(tmem_o, tmem_s + 8, vd + 128, idesc_o);
+        tc::mma_ts_c<true>(tmem_o, tmem_s + 16, vd + 256, idesc_o);
+        tc::mma_ts_c<true>(tmem_o, tmem_s + 24, vd + 384, idesc_o);
+        tc::mma_commit(kve + slot);                              // K (read by S(u)) and V of the block are done with
+        if (u == cp.nb - 1) tc::mma_commit(o_full + s);
         if (with_s) fire_s();
-        if (block_done) tc::mma_commit(ve + slot);
-        if (kMsBufs == 2 && u == cp.nsub - 2) tc::mma_commit(r_full + s);   // for a late rescale of O in the last sub-block
-        if (u == cp.nsub - 1) tc::mma_commit(o_full + s);
       }
       __syncwarp();
-      ++g_p;
-      if (block_done) ++vc;
-      if (++cp.u == cp.nsub) { cp.item += item_step; seek(cp); }
+      ++vc;
+      if (++cp.u == cp.nb) { cp.item += item_step; seek(cp); }
       if (with_s) advance_s();
+    }
+    // loads still outstanding for the half's other stream (it may lag behind this one)
+    {
+      int polls = 0;
+      while (ok && (lq_item < p.total_items || (tile == 0 && lk_item < p.total_items))) {
+        if (refill()) { polls = 0; continue; }
+        __nanosleep(500);
+        if (*abort_flag || ++polls > (1 << 22)) ok = false;
+      }
     }
   } else {
     // ---------------- softmax: four warps per stream ----------------
@@ -343,8 +310,8 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     const uint32_t tmem_s = tmem_base + 64 * s + lane_addr;
     const uint32_t tmem_o = tmem_base + 256 + 64 * s + lane_addr;
-    uint32_t g = 0;                               // sub-blocks done (buffer = g & 1)
-    uint32_t ow = 0, rw = 0;                      // o_full / r_full phases passed
+    uint32_t g = 0;                               // blocks done
+    uint32_t ow = 0;                              // o_full phases passed
     uint32_t qn = 0;                              // items with work so far (Q buffer = qn & 1)
     int release = -1;                             // Q buffer whose output stores are still to be waited for
     bool ok = true;
@@ -372,21 +339,19 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         continue;
       }
-      const int nsub = (it.T + kMsSub - 1) / kMsSub;
       float m_run = -INFINITY, l_run = 0.f;
-      for (int u = 0; u < nsub; ++u, ++g) {
-        const uint32_t buf = g % kMsBufs;
-        ok = tc::mbar_wait_likely_done(s_full + 2 * s + buf, (g / kMsBufs) & 1, abort_flag);
+      for (int u = 0; u < it.nb; ++u, ++g) {
+        ok = tc::mbar_wait_likely_done(s_full + s, g & 1, abort_flag);
         if (!ok) break;
         tc::tc_fence_after();
-        uint32_t r[kMsSub];
+        uint32_t r[kMsBN];
 #pragma unroll
-        for (int c = 0; c < kMsSub; c += 32) tc::tmem_ld32(tmem_s + kMsSub * buf + c, *reinterpret_cast<uint32_t(*)[32]>(&r[c]));
+        for (int c = 0; c < kMsBN; c += 32) tc::tmem_ld32(tmem_s + c, *reinterpret_cast<uint32_t(*)[32]>(&r[c]));
         tc::tmem_ld_wait();
-        const int valid = it.T - u * kMsSub;                        // positions of this sub-block that exist (>= 1)
-        if (valid < kMsSub) {
+        const int valid = it.T - u * kMsBN;                         // positions of this block that exist (>= 1)
+        if (valid < kMsBN) {
 #pragma unroll
-          for (int c = 0; c < kMsSub; ++c)
+          for (int c = 0; c < kMsBN; ++c)
             if (c >= valid) r[c] = 0xff800000u;                     // -inf: no weight, no influence on the maximum
         }
         float mx0 = ms_max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
@@ -394,14 +359,14 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         float mx2 = ms_max3(__uint_as_float(r[6]), __uint_as_float(r[7]), __uint_as_float(r[8]));
         float mx3 = ms_max3(__uint_as_float(r[9]), __uint_as_float(r[10]), __uint_as_float(r[11]));
 #pragma unroll
-        for (int c = 12; c + 7 < kMsSub; c += 8) {
+        for (int c = 12; c + 7 < kMsBN; c += 8) {
           mx0 = ms_max3(mx0, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
           mx1 = ms_max3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
           mx2 = ms_max3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
           mx3 = ms_max3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
         }
-        mx0 = ms_max3(mx0, __uint_as_float(r[kMsSub - 4]), __uint_as_float(r[kMsSub - 3]));
-        mx1 = ms_max3(mx1, __uint_as_float(r[kMsSub - 2]), __uint_as_float(r[kMsSub - 1]));
+        mx0 = ms_max3(mx0, __uint_as_float(r[kMsBN - 4]), __uint_as_float(r[kMsBN - 3]));
+        mx1 = ms_max3(mx1, __uint_as_float(r[kMsBN - 2]), __uint_as_float(r[kMsBN - 1]));
         const float m_blk = fmaxf(ms_max3(mx0, mx1, mx2), mx3) * p.scale_log2;
         // The accumulator is rescaled only when the row maximum grows by more than 2^16 over the
         // reference in use (probabilities may then reach 65536, which bf16 and the fp32 sums hold
@@ -412,15 +377,8 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const float alpha = grow ? ms_ex2(m_run - m_new) : 1.0f;    // 0 on the first sub-block
         m_run = m_new;
         if (u > 0 && __any_sync(kFullMask, grow)) {
-          // O is about to change under the tensor core: P V of sub-block u - 1 must be complete.  It was
-          // issued before S of sub-block u + 1 (peeked here, consumed in the next iteration) or, in the
-          // item's last sub-block, before the commit on r_full.
-          if (kMsBufs == 2) {                     // (with one buffer this sub-block's S was itself issued after that P V)
-            if (u + 1 < nsub) ok = tc::mbar_wait(s_full + 2 * s + (buf ^ 1), ((g + 1) >> 1) & 1, abort_flag);
-            else ok = tc::mbar_wait(r_full + s, rw & 1, abort_flag);
-            if (!ok) break;
-          }
-          tc::tc_fence_after();
+          // O changes under the tensor core only here; P V of block u - 1 is complete, because this
+          // block's S was issued after it and has been waited for.
 #pragma unroll
           for (int c = 0; c < kMsDH; c += 16) {
             uint32_t o[16];
@@ -434,7 +392,7 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const float neg_m = -m_new;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-        for (int c = 0; c < kMsSub / 4; ++c) {
+        for (int c = 0; c < kMsBN / 4; ++c) {
           const float e0 = ms_ex2(fmaf(__uint_as_float(r[4 * c]), p.scale_log2, neg_m));
           const float e1 = ms_ex2(fmaf(__uint_as_float(r[4 * c + 1]), p.scale_log2, neg_m));
           const float e2 = ms_ex2(fmaf(__uint_as_float(r[4 * c + 2]), p.scale_log2, neg_m));
@@ -445,15 +403,14 @@ cross_attn_ms_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         l_run = fmaf(l_run, alpha, (s0 + s1) + (s2 + s3));
 #pragma unroll
-        for (int c = 0; c < kMsSub / 2; c += 16) tc::tmem_st16(tmem_s + kMsSub * buf + c, *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
+        for (int c = 0; c < kMsBN / 2; c += 16) tc::tmem_st16(tmem_s + c, *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
         tc::tmem_st_wait();
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(p_full + 2 * s + buf);
+        if (lane == 0) tc::mbar_arrive(p_full + s);
         if (u == 0) release_q();                  // the previous item's output stores have long been read
       }
       if (!ok) break;
-      if (nsub >= 2) ++rw;
       // ---- end of the item: O / l -> bf16 rows, staged in the item's Q tile, TMA store per warp ----
       ok = tc::mbar_wait(o_full + s, ow & 1, abort_flag);
       if (!ok) break;

@@ -85,6 +85,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
+// One try_wait with the given suspend hint in nanoseconds.
+__device__ __forceinline__ bool mbar_try_wait_ns(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 // Non-blocking test of a barrier phase (no suspend hint): for threads that poll several queues.
 __device__ __forceinline__ bool mbar_try_wait_now(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
