@@ -138,3 +138,40 @@ def test_more_groups_keep_fewer_prefixes_on_average():
         kept.append(sum(kw.entry_passes(j, s["ubm"][b], s["ubl"][b])
                         for b in range(8) for j in range(s["trie"].num_nodes - 1)))
     assert kept[0] >= kept[1] >= kept[2] and kept[0] > kept[2]
+
+
+def test_gtm_mask_with_kway_matcher_keeps_a_child_iff_one_of_its_groups_passes():
+    """`KWayRowsMatcher` plugged into `gtm_mask`: a child is allowed iff at least one group of its node
+    passes the bitmask test and the any-location Bloom test on its own row pair (Section 4.2, k-way
+    partition), written out here directly on the index arrays."""
+    from oracle.gtm import gtm_mask
+    s = _setup()
+    trie, sids = s["trie"], s["sids"]
+    kw = KW.KWayMatcherIndex(trie, sids, s["ad_sid"], s["ad_bm"], s["ad_bl"], ("static", [0, 4, 2, 1]))
+    B = s["ubm"].shape[0]
+    M = 4
+    matcher = KW.KWayRowsMatcher(trie, kw, s["ubm"], s["ubl"])
+    internal = [node for node in range(trie.num_nodes) if trie.lookup(node)[0].size > 0]
+    beam_node = np.array((internal * (B * M))[:B * M], dtype=np.int64)
+    V = trie.vocab_size
+    logp = -0.01 * np.arange(B * M * V, dtype=np.float32).reshape(B * M, V)
+    score = -np.arange(B * M, dtype=np.float32)
+    cand, allow, child = gtm_mask(logp, score, beam_node, np.zeros(B * M, dtype=np.uint64), 0, trie, matcher, B, M)
+    kept = dropped = 0
+    for r in range(B * M):
+        b = r // M
+        tokens, kids = trie.lookup(int(beam_node[r]))
+        for v, c in zip(tokens, kids):
+            groups = range(int(kw.part_offsets[int(c) - 1]), int(kw.part_offsets[int(c)]))
+            want = any(np.array_equal(kw.bitmask_table[kw.bitmask_index[g]] & s["ubm"][b], s["ubm"][b]) and
+                       any(np.array_equal(kw.bloom_table[kw.bloom_index[g]] & row, row) for row in s["ubl"][b])
+                       for g in groups)
+            assert bool(allow[r, v]) == want
+            if want:
+                assert int(child[r, v]) == int(c) and cand[r, v] == np.float32(score[r]) + logp[r, v]
+            kept += want
+            dropped += not want
+        others = np.ones(V, dtype=bool)
+        others[tokens] = False
+        assert not allow[r][others].any()
+    assert kept > 0 and dropped > 0

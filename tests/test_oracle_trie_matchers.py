@@ -247,3 +247,46 @@ def test_node_rows_index_is_the_union_over_descendant_ads_and_is_conservative():
         want = [(int(t), int(c)) for t, c in zip(*trie.lookup(0))
                 if Mx.bitmask_match(index.node_bitmask[c], ubm[b]) and Mx.bloom_any(index.node_bloom[c], ubl[b])]
         assert got == want
+
+
+def test_gtm_mask_with_node_rows_matcher_equals_the_appendix_a_lookup():
+    """`NodeRowsMatcher` plugged into `gtm_mask` must allow, for every beam, exactly the (token, child)
+    pairs the Appendix A lookup emits for that beam's node and that beam's request; and the candidate
+    score of such a pair is the beam's score plus the token's log-probability (Section 4.1)."""
+    V, L, n = 64, 3, 300
+    rng = synth.rng_for(4, 71)
+    sids = synth.catalog(rng, n, V, L)
+    trie = SidTrie(sids, V)
+    layout = synth.TargetingLayout(W_bm=2, W_bl=4, attributes=((0, 20), (20, 4), (24, 30), (64, 40)),
+                                   n_locations=300, bits_per_location=3)
+    loc_rows = synth.location_rows(rng, layout)
+    ad_sid, ad_bm, ad_bl = synth.ads_for_sids(rng, n, layout, loc_rows)
+    index = Mx.NodeMatcherIndex(trie, sids, ad_sid, ad_bm, ad_bl)
+    B, M = 3, 5
+    ubm, ubl, _ = synth.request_attributes(rng, B, layout, loc_rows, n_loc=8)
+    matcher = Mx.NodeRowsMatcher(trie, index, ubm, ubl)
+    from oracle.gtm import gtm_mask
+    internal = [node for node in range(trie.num_nodes) if trie.lookup(node)[0].size > 0]
+    some_kept = some_dropped = False
+    for depth_nodes in (internal[:1] * (B * M), internal[1:1 + B * M], internal[-B * M:]):
+        beam_node = np.array(depth_nodes, dtype=np.int64)
+        beam_node[2] = -1                                         # a dead beam allows nothing
+        score = -np.arange(B * M, dtype=np.float32)
+        logp = np.log(np.full((B * M, V), 1.0 / V, dtype=np.float32)) - 0.01 * np.arange(V, dtype=np.float32)
+        cand, allow, child = gtm_mask(logp, score, beam_node, np.zeros(B * M, dtype=np.uint64), 0, trie, matcher, B, M)
+        for r in range(B * M):
+            if beam_node[r] < 0:
+                assert not allow[r].any() and np.isneginf(cand[r]).all()
+                continue
+            b = r // M
+            want = Mx.paper_lookup(trie, index.bitmask_index, index.bloom_index, index.bitmask_table,
+                                   index.bloom_table, int(beam_node[r]), ubm[b], ubl[b])
+            got = [(int(v), int(child[r, v])) for v in np.flatnonzero(allow[r])]
+            assert got == want
+            for v, _ in want:
+                assert cand[r, v] == np.float32(score[r]) + logp[r, v]
+            assert np.isneginf(cand[r][~allow[r]]).all()
+            n_children = trie.lookup(int(beam_node[r]))[0].size
+            some_kept |= len(want) > 0
+            some_dropped |= len(want) < n_children
+    assert some_kept and some_dropped                             # the comparison saw both outcomes
