@@ -25,7 +25,7 @@ def api():
 
 
 # ---- configuration 2: cross-attention op sweep ----------------------------------------------------
-@pytest.mark.parametrize("B,M,T", [(64, 256, 512), (64, 1024, 512), (64, 256, 1024)])
+@pytest.mark.parametrize("B,M,T", [(64, 256, 512), (64, 1024, 512), (64, 256, 1024), (64, 1024, 1024)])
 def test_cross_attn_config2_sampled_rows(api, B, M, T):
     H, d = 8, 64
     rng = synth.rng_for(2, M + T)
@@ -320,3 +320,65 @@ def test_bench_decode_path_equals_the_materialised_path_at_config5():
     assert torch.isfinite(outs[0][0]).sum() > B * K // 2
     assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
     assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+
+
+def test_bench_decoder_teacher_forced_against_the_oracle_at_config5():
+    """The decoder exactly as bench.py builds it (bf16 residual stream, LayerNorm folded into the GEMMs over a
+    centred stream, cache held in place, candidates materialised on the dense trie level and read through
+    allow bits on the sparse ones), teacher-forced on request 0 against the oracle's decode of that request:
+    at every step the allow bits / finite candidates equal the oracle's mask, the log-probabilities agree
+    within the decoder tolerance, and the selection, parents, tokens, nodes and keys equal the oracle's
+    top-k and state update run on the GPU's own candidates, bit for bit."""
+    import bench
+    from oracle import decoder as OD
+    from paper_2608_00938_b200 import api
+    cfg = dict(bench.CFG5)
+    inp = bench.make_inputs(cfg, 0)
+    sids, V, L, B = inp["sids"], cfg["V"], cfg["L"], cfg["B"]
+    sizes = list(cfg["schedule"]) + [cfg["final_k"]]
+    trie = SidTrie(sids, V)
+    bloom0 = OM.build_prefix_bloom(sids, inp["elig"][0], cfg["bloom_log2"], cfg["bloom_hashes"])
+    record = []
+    OD.beam_search(inp["weights"], inp["shp"], synth.bf16_bits_to_f32(inp["enc_bits"][:1]), trie,
+                   OG.PrefixBloomMatcher([bloom0]), cfg["schedule"], cfg["final_k"], record=record)
+    dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True)
+    assert dec.allow_bits is not None and 0 < dec.masked_from_step < L          # both candidate paths are exercised
+    dec.project_cross_kv(dev_bf16(inp["enc_bits"]))
+    dec.reset()
+    for t in range(L):
+        step = record[t]
+        M, K = sizes[t], sizes[t + 1]
+        cur, nxt = t & 1, (t + 1) & 1
+        dec.token[cur][:M].copy_(dev(step["tokens"].astype(np.int32)))
+        dec.score[cur][:M].copy_(dev(step["score"]))
+        dec.node[cur][:M].copy_(dev(step["node"]))
+        dec.key[cur][:M].copy_(dev(step["key"]))
+        if t > 0:
+            dec.parents[t, :M].copy_(dev(record[t - 1]["out_parent"].reshape(-1)))
+        dec.step(t)
+        torch.cuda.synchronize()
+        assert dec.d_status.item() & ~api.DEV_TOPK_EXACT_PATH == 0
+        live = step["node"] >= 0
+        score = step["score"].astype(np.float32)
+        if t < dec.masked_from_step:
+            cand = dec.cand[:M].cpu().numpy()                                    # written in place of the logits
+            assert np.array_equal(np.isfinite(cand), step["allow"])
+            got_logp = (cand - score[:, None])[step["allow"]]
+            ref_logp = step["logp"][step["allow"]]
+        else:
+            bits = dec.allow_bits[:M].cpu().numpy().view(np.uint64)
+            assert np.array_equal(bits, OG.pack_allow_bits(step["allow"]))
+            logits = dec.logp[:M].cpu().numpy()
+            lse = dec.row_lse[:M].cpu().numpy()
+            logp = logits - lse[:, None]
+            cand = np.where(step["allow"], score[:, None] + logp, np.float32(-np.inf)).astype(np.float32)
+            got_logp, ref_logp = logp[live], step["logp"][live]
+        assert_log_probs_close(got_logp, ref_logp, f"bench decoder step {t}")
+        sc, flat, par, tok = OT.beam_topk(cand.reshape(1, M * V), K, V)           # exact, on the GPU's own candidates
+        assert np.array_equal(dec.out_flat[:K].cpu().numpy(), flat[0])
+        assert np.array_equal(dec.score[nxt][:K].cpu().numpy().view(np.uint32), sc[0].view(np.uint32))
+        assert np.array_equal(dec.parents[t + 1, :K].cpu().numpy(), par[0])
+        assert np.array_equal(dec.token[nxt][:K].cpu().numpy(), tok[0])
+        node_ref, key_ref = OT.update_beam_state(trie, par, tok, sc, step["node"], step["key"], t, M)
+        assert np.array_equal(dec.node[nxt][:K].cpu().numpy(), node_ref)
+        assert np.array_equal(dec.key[nxt][:K].cpu().numpy().view(np.uint64), key_ref)

@@ -22,7 +22,7 @@ def api():
     return _api
 
 
-from gpu_util import DEV, assert_attention_close, dev, dev_bf16, f64, host_u64  # noqa: E402
+from gpu_util import DEV, assert_attention_close, assert_gemm_close, dev, dev_bf16, f64, host_u64  # noqa: E402
 
 
 # ------------------------------------------------------------------------------------------
@@ -588,8 +588,8 @@ def test_linear_matches_fp64_matmul(api, M, N, K, relu, res, f32out):
     api.grace_linear(dev_bf16(x), dev_bf16(w), y, d_res, relu)
     torch.cuda.synchronize()
     got = y.float().cpu().numpy().astype(np.float64)
-    tol = 2e-3 if f32out else 2e-2
-    assert np.abs(got - ref).max() <= tol * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
+    abs_sum = np.abs(f64(x)) @ np.abs(f64(w)).T + (np.abs(r) if res else 0.0)
+    assert_gemm_close(got, ref, abs_sum, 0 if f32out else 1, f"linear {M}x{N}x{K}")
 
 
 @pytest.mark.parametrize("M,N,K", [
@@ -606,8 +606,11 @@ def test_linear_add_into_bf16_residual_stream(api, M, N, K):
     api.grace_linear_add_bf16(dev_bf16(x), dev_bf16(w), y)
     torch.cuda.synchronize()
     got = y.float().cpu().numpy().astype(np.float64)
-    # product rounded to bf16 (2^-9 relative), then a bf16 add: two roundings of values of size |ref|
-    assert np.abs(got - ref).max() <= 2e-2 * max(1.0, np.abs(ref).max()), np.abs(got - ref).max()
+    # product rounded to bf16 (2^-9 of |x w^T|), then a bf16 add (2^-9 of the sum): the abs-sum term carries
+    # the first rounding when product and residual cancel
+    abs_sum = np.abs(f64(x)) @ np.abs(f64(w)).T + np.abs(f64(r))
+    prod = np.abs(f64(x) @ f64(w).T)
+    assert_gemm_close(got, ref + 0.0, abs_sum + 2.0 ** 11 * prod, 1, f"linear_add_bf16 {M}x{N}x{K}")
     err = np.abs(got - ref) / np.maximum(np.abs(ref), np.abs(f64(r)))
     assert np.median(err) <= 2.0 ** -8
 
