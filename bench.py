@@ -366,15 +366,30 @@ def op_breakdown(dec, cfg, reps=3):
 # ------------------------------------------------------------------------------------------------
 # op-level rooflines at the per-op benchmark configurations
 # ------------------------------------------------------------------------------------------------
-def _time_op(fn, n_sets, iters=30, warm=5):
+def _time_op(fn, n_sets, iters=200, warm=20):
+    """P50 / P99 (us) of one C-ABI call over `iters` launches after `warm` warm-up launches.  Each call is
+    captured once per buffer set into a CUDA graph and the graph is replayed between a pair of events: the
+    host-side cost of a launch (tensor-map encoding, Python) would otherwise leave the GPU idle inside the
+    timed interval of kernels that take tens of microseconds.  The buffer sets rotate (cold L2)."""
     import torch
+    fn(0)                                                     # per-device set-up outside any capture
+    torch.cuda.synchronize()
+    graphs = []
+    side = torch.cuda.Stream()
+    for i in range(n_sets):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                fn(i)
+        graphs.append(g)
+    torch.cuda.synchronize()
     for i in range(warm):
-        fn(i % n_sets)
+        graphs[i % n_sets].replay()
     torch.cuda.synchronize()
     evs = []
     for i in range(iters):
         a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
-        a.record(); fn(i % n_sets); b.record()
+        a.record(); graphs[i % n_sets].replay(); b.record()
         evs.append((a, b))
     torch.cuda.synchronize()
     ts = sorted(a.elapsed_time(b) for a, b in evs)
@@ -409,12 +424,27 @@ def op_rooflines(device, peaks):
     parents = torch.randint(0, M, (Lc, R), device=device, dtype=torch.int32, generator=g)
     qkv = rnd(R, 3, H, d)
     o = torch.empty(R, H, d, device=device, dtype=torch.bfloat16)
+    # Rows share ancestors (parents are drawn uniformly from the previous beam), so the cache blocks a step
+    # must fetch from HBM are the UNIQUE ancestor blocks; the logical count charges every row all its ancestors.
+    par_host = parents.cpu().numpy().astype(np.int64)
+    base = (np.arange(R, dtype=np.int64) // M) * M
+
+    def unique_ancestor_blocks(t):
+        idx, total = np.arange(R, dtype=np.int64), 0
+        for j in range(t, 0, -1):                               # a_{j-1} = parent_j[a_j] inside the request
+            idx = base + par_host[j][idx]
+            total += np.unique(idx).size
+        return total
+
     for t in range(5):
         sizes = [M] * (t + 1)
         p50, p99 = _time_op(lambda i: api.grace_self_attn(qkv, kc, vc, parents, sizes, o, B, t, 0.125), 1)
         logical = R * 1024 * (6 + 2 * t)                       # q,k,v read 3 KB + k,v write 2 KB + out 1 KB + 2 KB/ancestor
-        out[f"self_attn_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, gbs=logical / p50 / 1e3, bound="hbm",
-                                          frac=logical / p50 / 1e3 / peaks["hbm_gbs"])
+        unique = R * 1024 * 6 + unique_ancestor_blocks(t) * 2048
+        out[f"self_attn_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, bound="hbm", gbs_unique=unique / p50 / 1e3,
+                                          gbs_logical=logical / p50 / 1e3, frac=unique / p50 / 1e3 / peaks["hbm_gbs"],
+                                          frac_logical=logical / p50 / 1e3 / peaks["hbm_gbs"],
+                                          bytes_unique=unique, bytes_logical=logical)
     del kc, vc, qkv
     # the form the decode loop runs: the cache is the steps' QKV projections, kept in place (nothing written but out)
     slabs = rnd(Lc, R, 3, H, d)
@@ -422,8 +452,11 @@ def op_rooflines(device, peaks):
         sizes = [M] * (t + 1)
         p50, p99 = _time_op(lambda i: api.grace_self_attn_inplace(slabs, parents, sizes, o, B, t, 0.125), 1)
         logical = R * 1024 * (4 + 2 * t)                       # q,k,v read 3 KB + out 1 KB + 2 KB/ancestor
-        out[f"self_attn_inplace_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, gbs=logical / p50 / 1e3, bound="hbm",
-                                                  frac=logical / p50 / 1e3 / peaks["hbm_gbs"])
+        unique = R * 1024 * 4 + unique_ancestor_blocks(t) * 2048
+        out[f"self_attn_inplace_T{t + 1}"] = dict(p50_us=p50, p99_us=p99, bound="hbm", gbs_unique=unique / p50 / 1e3,
+                                                  gbs_logical=logical / p50 / 1e3, frac=unique / p50 / 1e3 / peaks["hbm_gbs"],
+                                                  frac_logical=logical / p50 / 1e3 / peaks["hbm_gbs"],
+                                                  bytes_unique=unique, bytes_logical=logical)
     del slabs, o
     # ---- top-k alone, configuration 4 (dense, all finite: worst case) ----
     B, M, V, K = 32, 2048, 1024, 2048
@@ -470,7 +503,10 @@ def mask_roofline(dec, cfg, inp, peaks):
     nb_dev = torch.from_numpy(nb.view(np.int64)).to(dec.device)
     out = {}
     for name, matcher, note in (
-            ("gtm_mask_depth1_B32_M2048_V2048", dec.matcher, "prefix Bloom 2^22 x 4; dense-form bytes: 4 B in + 4 B out per candidate"),
+            ("gtm_mask_depth1_B32_M2048_V2048", dec.matcher,
+             "prefix Bloom 2^22 x 4; frac is on dense-form bytes (4 B in + 4 B out per candidate); the kernel reads only the "
+             "sectors that hold an allowed token: ncu saw 73 MB read + 210 MB written for 32768 rows (profiles/), i.e. "
+             "about 566 MB of DRAM traffic at this size against 1074 MB dense-form"),
             ("gtm_mask_node_bitmask_depth1_B32_M2048_V2048", api.make_matcher(api.MATCH_NODE_BITMASK, nb_dev),
              "node bitmask; dense-form bytes")):
         p50, p99 = _time_op(lambda i: api.grace_gtm_mask(logp, dec.score[1][:R], dec.node[1][:R], dec.key[1][:R], dec.trie,
@@ -499,6 +535,16 @@ def oracle_sample(cfg, inp, beam, request=0):
     return time.perf_counter() - t0, sum(schedule)
 
 
+def oracle_sample_one_thread(cfg, inp, beam, request=0):
+    """The same sample with the numerical libraries held to one thread."""
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return oracle_sample(cfg, inp, beam, request)
+    with threadpool_limits(limits=1):
+        return oracle_sample(cfg, inp, beam, request)
+
+
 def cpu_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -513,21 +559,26 @@ def run_reference(args, rank):
         return
     cfg = dict(CFG5)
     inp = make_inputs(cfg, 0)
-    beam = 2048 if (args.steps + args.warmup) <= 16 else 512     # keep the whole run within a few minutes
-    for _ in range(args.warmup):
+    beam = cfg["schedule"][1]                                    # the GPU arm's own schedule, whatever the step count
+    for _ in range(min(args.warmup, 1)):                         # a CPU program has nothing to warm beyond its first pass
         oracle_sample(cfg, inp, beam)
     secs, units = 0.0, 0
     for _ in range(args.steps):
         s, u = oracle_sample(cfg, inp, beam)
         secs += s; units += u
     value = units / secs
-    sample = f"1 of {cfg['B']} requests, beam schedule (1,{beam},{beam},{beam}), all 4 steps, per bench step"
+    secs1, units1 = oracle_sample_one_thread(cfg, inp, beam)
+    sample = (f"1 of {cfg['B']} requests, beam schedule (1,{beam},{beam},{beam}), all 4 steps, per bench step "
+              f"(one untimed pass first; {args.warmup} warm-up steps asked for)")
     line = dict(impl="reference", metric="beam_steps_per_s", value=value, unit="beam-steps/s", n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=secs / args.steps * 1e3, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
                 config=dict(workload=cfg["name"], B=cfg["B"], schedule=list(cfg["schedule"]), V=cfg["V"], L=cfg["L"],
                             n_layers=cfg["n_layers"], d_model=cfg["d_model"], T_ctx=cfg["T_ctx"]),
-                cpu_baseline=dict(value=value, unit="beam-steps/s", cores=cpu_threads(), kind="oracle", sample=sample),
+                same_config=True,
+                cpu_baseline=dict(value=value, unit="beam-steps/s", cores=cpu_threads(), kind="oracle", sample=sample,
+                                  value_threads_1=units1 / secs1,
+                                  parallelism="numpy fp64; only its BLAS calls use the thread pool"),
                 e2e=dict(value=value, unit="beam-steps/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line), flush=True)
 
@@ -638,6 +689,7 @@ def main():
         # 73.8 MB for 68.7 GFLOP); the bench's launches are larger than a capture may be, so the traffic is scaled
         # by the flops of an average launch (it grows in proportion: every tile streams its operands once).
         dram_bytes_per_flop = {"linear": 111.23e6 / 68.72e9, "cross_attn": 73.85e6 / 68.72e9}
+        line["whole_loop_tflops"] = sum(v["flops_per_loop"] for v in bd.values()) / (ms_loop * 1e-3) / 1e12
         if top in ("linear", "cross_attn") and not default_workload:
             ach = bd[top]["flops_per_loop"] / (bd[top]["ms_per_loop"] * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
@@ -649,6 +701,10 @@ def main():
             peak = peaks["bf16_tflops_sustained"]
             per_launch = bd[top]["flops_per_loop"] / bd[top]["calls_per_loop"]
             line["roofline"] = dict(kernel=top, bound="tensor", achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
+                                    frac_burst=ach / peaks["bf16_tflops"], peak_burst=peaks["bf16_tflops"],
+                                    frac_note=("frac is against the sustained cuBLAS figure (measured at a median 1372 MHz "
+                                               "under the power cap), frac_burst against the burst figure; this run's "
+                                               f"median SM clock was {clocks.get('sm_mhz')} MHz, so the truth lies between"),
                                     traffic=per_launch * dram_bytes_per_flop[top],
                                     traffic_note="DRAM bytes of an average launch, scaled from the ncu capture in profiles/",
                                     flops_per_launch=per_launch,
@@ -672,8 +728,11 @@ def main():
             line["op_rooflines"] = ops
         if not args.no_cpu and world == 1 and default_workload:
             secs, units_cpu = oracle_sample(cfg, inp, 2048)
+            secs1, _ = oracle_sample_one_thread(cfg, inp, 2048)
             line["cpu_baseline"] = dict(value=units_cpu / secs, unit="beam-steps/s", cores=cpu_threads(), kind="oracle",
-                                        seconds=secs,
+                                        seconds=secs, value_threads_1=units_cpu / secs1, seconds_threads_1=secs1,
+                                        parallelism="numpy fp64; only its BLAS calls (projections, attention products) use "
+                                                    "the thread pool, the trie walk, matcher and top-k are single-threaded",
                                         sample=f"1 of {cfg['B']} requests, full schedule (1,2048,2048,2048), all 4 steps")
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -140,6 +140,35 @@ grace_status_t grace_trie_walk(const uint64_t* child_bits, const int32_t* child_
                                int64_t num_internal, const int32_t* tokens, int len, int32_t* node);
 
 /* ------------------------------------------------------------------------------------------
+ * Weight preparation for the folded-LayerNorm decode path (host memory in, host memory out; not
+ * on the timed path).  No passage of the paper defines these: Section 3.2 fixes neither the
+ * normalisation nor its placement; the decoder here is pre-LayerNorm, and two identities of a
+ * pre-LayerNorm block are used to take the LayerNorm kernels off the path:
+ *   (fold)    LN(x; gamma, beta) W^T = rstd (x W'^T) - rstd mean colsum(W') + W beta,
+ *             W' = W * gamma (column-wise), rstd = 1 / sqrt(var(x) + eps)  (per row of x);
+ *   (centre)  LayerNorm does not see a per-row shift of its input, so everything ADDED into the
+ *             residual stream may be centred over the feature axis; the stream's rows then keep
+ *             zero mean and the colsum term vanishes.
+ * grace_decode_step with row_affine set expects weights prepared by these helpers.
+ *
+ * grace_fold_layer_norm:  w host fp32 [N, K] (row n = output feature n), gamma, beta host fp32 [K].
+ *   w_folded  host bf16 [N, K] = round-to-nearest-even(w[n,k] * gamma[k])   (the GEMM's operand)
+ *   col_sum   host fp32 [N]    = sum_k of the ROUNDED w_folded[n,k]           (fp64 accumulation)
+ *   col_bias  host fp32 [N]    = sum_k w[n,k] * beta[k]                       (fp64 accumulation)
+ * grace_centre_rows:     a host fp32 [n, d] -> out[i, :] = a[i, :] - mean(a[i, :])   (embedding, position rows)
+ * grace_centre_outputs:  w host fp32 [d_out, K] (a projection INTO the stream: row i = stream
+ *   feature i) -> out[i, k] = w[i, k] - mean_i(w[i, k]): every output row of x W^T then has zero mean.
+ * grace_f32_to_bf16:     round-to-nearest-even conversion, host fp32 [n] -> host bf16 [n].
+ * out may alias the input in the two centring calls.  Errors: GRACE_INVALID_ARG for null pointers
+ * or non-positive sizes; nothing else can fail.
+ * ---------------------------------------------------------------------------------------- */
+grace_status_t grace_fold_layer_norm(const float* w, const float* gamma, const float* beta, int64_t N, int64_t K,
+                                     uint16_t* w_folded, float* col_sum, float* col_bias);
+grace_status_t grace_centre_rows(const float* a, int64_t n, int64_t d, float* out);
+grace_status_t grace_centre_outputs(const float* w, int64_t d_out, int64_t K, float* out);
+grace_status_t grace_f32_to_bf16(const float* a, int64_t n, uint16_t* out);
+
+/* ------------------------------------------------------------------------------------------
  * Cross-attention, beam-as-query layout (Section 5.1, Appendix B).
  *   out[b*M+m, h, :] = softmax_t( q[b*M+m, h, :] . k[b, h, t, :] * scale ) @ v[b, h, :, :]
  * K and V are read once per (request, head) and shared by the M beams of the request.
@@ -155,6 +184,19 @@ grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
                                 uint16_t* out, int64_t out_row_stride, float* lse,
                                 int B, int M, int H, int d_h, int T_ctx, float scale,
                                 int32_t* d_status, void* stream);
+
+/* The same with padded encoder outputs (an extension; the paper fixes T_ctx per batch, Section 3.2):
+ *   enc_len : device int32 [B] or NULL; request b attends to positions 0 .. enc_len[b]-1 only
+ *             (values are clamped to [0, T_ctx]); NULL = all T_ctx positions.
+ * A request with enc_len 0 gets zero output rows and lse = -inf (the softmax over an empty set is
+ * left undefined by the paper).  grace_cross_attn is this call with enc_len = NULL. */
+grace_status_t grace_cross_attn_varlen(const uint16_t* q, int64_t q_row_stride,
+                                       const uint16_t* k, const uint16_t* v,
+                                       int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                                       uint16_t* out, int64_t out_row_stride, float* lse,
+                                       const int32_t* enc_len,
+                                       int B, int M, int H, int d_h, int T_ctx, float scale,
+                                       int32_t* d_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Self-attention over the parent-addressed KV cache, fused with the cache write

@@ -49,6 +49,23 @@ def cross_attn(q, k, v, scale, return_probs: bool = False):
     return out, lse
 
 
+def cross_attn_varlen(q, k, v, enc_len, scale):
+    """Cross-attention over padded encoder outputs: request b attends to its first enc_len[b] positions only
+    (an extension: Section 3.2 fixes the encoder length per batch).  A request without any position gets
+    zero output and lse = -inf.  Written as the definition: the plain cross-attention of every request on
+    its own, truncated K / V."""
+    q = np.asarray(q, dtype=np.float64)
+    B, M, H, d = q.shape
+    out = np.zeros((B, M, H, d), dtype=np.float64)
+    lse = np.full((B, M, H), -np.inf, dtype=np.float64)
+    for b in range(B):
+        n = int(enc_len[b])
+        if n > 0:
+            o, l = cross_attn(q[b:b + 1], np.asarray(k)[b:b + 1, :, :n], np.asarray(v)[b:b + 1, :, :n], scale)
+            out[b], lse[b] = o[0], l[0]
+    return out, lse
+
+
 def cross_attn_row(q_row, k_bh, v_bh, scale):
     """One (beam row, head): q_row [d], k_bh/v_bh [T, d] -> [d]."""
     s = (np.asarray(k_bh, np.float64) @ np.asarray(q_row, np.float64)) * scale

@@ -88,10 +88,16 @@ _built_for_sm = _sig("grace_built_for_sm", _i32, [])
 _trie_count_nodes = _sig("grace_trie_count_nodes", _i32, [_vp, _i64, _i32, _i32, _vp])
 _trie_build_dense = _sig("grace_trie_build_dense", _i32, [_vp, _i64, _i32, _i32, _vp, _vp])
 _node_bitmask_build = _sig("grace_node_bitmask_build", _i32, [_vp, _i64, _i32, _i32, _vp, _vp])
+_fold_layer_norm = _sig("grace_fold_layer_norm", _i32, [_vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp])
+_centre_rows = _sig("grace_centre_rows", _i32, [_vp, _i64, _i64, _vp])
+_centre_outputs = _sig("grace_centre_outputs", _i32, [_vp, _i64, _i64, _vp])
+_f32_to_bf16 = _sig("grace_f32_to_bf16", _i32, [_vp, _i64, _vp])
 _bloom_build = _sig("grace_bloom_build", _i32, [_vp, _i64, _i32, _i32, _vp, _i32, _i32, _vp])
 _trie_walk = _sig("grace_trie_walk", _i32, [_vp, _vp, _i32, _i32, _i64, _vp, _i32, _vp])
 _cross_attn = _sig("grace_cross_attn", _i32, [_vp, _i64, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _vp,
                                              _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp])
+_cross_attn_varlen = _sig("grace_cross_attn_varlen", _i32, [_vp, _i64, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _vp, _vp,
+                                                           _i32, _i32, _i32, _i32, _i32, _f32, _vp, _vp])
 _self_attn = _sig("grace_self_attn", _i32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64,
                                            _i32, _i32, _i32, _i32, _i64, _f32, _vp, _vp])
 _self_attn_inplace = _sig("grace_self_attn_inplace", _i32, [_vp, _i64, _i64, _vp, _vp, _vp, _i64,
@@ -213,6 +219,41 @@ def grace_bloom_build(sids: np.ndarray, V: int, eligible: np.ndarray, log2_bits:
     el = np.ascontiguousarray(eligible, dtype=np.uint8)
     _check(_bloom_build(_hp(sids, np.int32), n, V, L, el.ctypes.data, log2_bits, n_hashes, out.ctypes.data),
            "grace_bloom_build")
+    return out
+
+
+def grace_fold_layer_norm(w: np.ndarray, gamma: np.ndarray, beta: np.ndarray):
+    """Host: (w * gamma as bf16 bits uint16 [N, K], column sums fp32 [N], w @ beta fp32 [N])."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    g = np.ascontiguousarray(gamma, dtype=np.float32)
+    b = np.ascontiguousarray(beta, dtype=np.float32)
+    N, K = w.shape
+    assert g.shape == (K,) and b.shape == (K,)
+    wf, cs, cb = np.empty((N, K), np.uint16), np.empty(N, np.float32), np.empty(N, np.float32)
+    _check(_fold_layer_norm(w.ctypes.data, g.ctypes.data, b.ctypes.data, N, K, wf.ctypes.data, cs.ctypes.data,
+                            cb.ctypes.data), "grace_fold_layer_norm")
+    return wf, cs, cb
+
+
+def grace_centre_rows(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty_like(a)
+    _check(_centre_rows(a.ctypes.data, a.shape[0], a.shape[1], out.ctypes.data), "grace_centre_rows")
+    return out
+
+
+def grace_centre_outputs(w: np.ndarray) -> np.ndarray:
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    out = np.empty_like(w)
+    _check(_centre_outputs(w.ctypes.data, w.shape[0], w.shape[1], out.ctypes.data), "grace_centre_outputs")
+    return out
+
+
+def grace_f32_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Host: fp32 array -> bf16 bit patterns (uint16, same shape), round to nearest even."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty(a.shape, np.uint16)
+    _check(_f32_to_bf16(a.ctypes.data, a.size, out.ctypes.data), "grace_f32_to_bf16")
     return out
 
 
@@ -412,6 +453,19 @@ def grace_cross_attn(q, k, v, out, scale: float, lse=None, d_status=None):
     _check(_cross_attn(q2.data_ptr(), q2.stride(0), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1),
                        k.stride(2), o2.data_ptr(), o2.stride(0), _dp(lse), B, M, H, d, T, scale,
                        _dp(d_status), _stream()), "grace_cross_attn")
+    return out
+
+
+def grace_cross_attn_varlen(q, k, v, out, enc_len, scale: float, lse=None, d_status=None):
+    """grace_cross_attn with a per-request number of valid encoder positions: enc_len int32 [B] on the device."""
+    B, H, T, d = k.shape
+    q2 = q.reshape(-1, H, d)
+    o2 = out.reshape(-1, H, d)
+    M = q2.shape[0] // B
+    assert k.stride() == v.stride() and k.stride(3) == 1 and enc_len.element_size() == 4 and enc_len.numel() == B
+    _check(_cross_attn_varlen(q2.data_ptr(), q2.stride(0), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1),
+                              k.stride(2), o2.data_ptr(), o2.stride(0), _dp(lse), _dp(enc_len), B, M, H, d, T, scale,
+                              _dp(d_status), _stream()), "grace_cross_attn_varlen")
     return out
 
 

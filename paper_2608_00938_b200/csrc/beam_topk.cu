@@ -703,21 +703,21 @@ grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, floa
   const uint32_t rank = sample_rank(N, K);
   static unsigned long long attrs_set_devices = 0;
   const size_t final_smem = (size_t)(kCap + kMaxK) * sizeof(unsigned long long) + 4096 * sizeof(uint32_t);
-  if (first_use_on_device(&attrs_set_devices)) {
+  static int collect_grid_of[kMaxDevices] = {0};
+  DeviceSetup su(&attrs_set_devices);
+  if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)final_smem));
+    int n_sm = 0, per_sm = 0;
+    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, su.dev));
+    GRACE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_collect_kernel, kCollectThreads, 0));
+    collect_grid_of[su.dev] = n_sm * (per_sm > 0 ? per_sm : 1);
+    su.done();
   }
+  const int collect_grid = collect_grid_of[su.dev];
   int force_exact = 1;
   if (rank != 0) {
     launch_pdl(topk_sample_kernel, dim3(B), dim3(kTopkThreads), 0, s, src, rank, hdr);
     GRACE_LAUNCH_CHECK();
-    static int collect_grid = 0;
-    if (collect_grid == 0) {
-      int dev = 0, n_sm = 0, per_sm = 0;
-      GRACE_CUDA_TRY(cudaGetDevice(&dev));
-      GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-      GRACE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_collect_kernel, kCollectThreads, 0));
-      collect_grid = n_sm * (per_sm > 0 ? per_sm : 1);
-    }
     const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
     const int64_t tiles_per_request = ((N >> 2) + tile - 1) / tile;
     int64_t per_request = collect_grid / B;                 // one resident wave over all requests
@@ -803,16 +803,18 @@ static __device__ __align__(256) unsigned char g_topk_static_scratch[kStaticScra
 
 // In host code the name of a __device__ array is only a stand-in, not a device address: the address
 // has to be asked for, once per device, while that device is current.
-constexpr int kMaxDevices = 64;
 static void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+static unsigned long long g_static_scratch_devices = 0;
 
 static grace_status_t static_scratch_for_current_device(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GRACE_CUDA_ERROR;
-  if (g_static_scratch_ptr[dev] == nullptr) {
+  DeviceSetup su(&g_static_scratch_devices);                // two host threads: the second waits for the first's look-up
+  if (su) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_topk_static_scratch) != cudaSuccess || ptr == nullptr) return GRACE_CUDA_ERROR;
     g_static_scratch_ptr[dev] = ptr;
+    su.done();
   }
   *out = g_static_scratch_ptr[dev];
   return GRACE_OK;

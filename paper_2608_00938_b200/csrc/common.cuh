@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <math.h>
+#include <mutex>
 
 #include "../../include/grace.h"
 
@@ -108,16 +109,35 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// One-time per-device set-up (kernel attributes are per device): true the first time the calling
-// thread's current device is seen for this `mask` (one static mask per set-up site).  Two host threads
-// racing here both do the set-up, which is idempotent.
-inline bool first_use_on_device(unsigned long long* mask) {
+// One-time per-device set-up (kernel attributes, occupancy figures and symbol addresses are per device).
+//     static unsigned long long done_devices = 0;
+//     DeviceSetup su(&done_devices);
+//     if (su) { ...set-up for the calling thread's current device...; su.done(); }
+// The first caller on a device runs the set-up under a process-wide mutex and publishes the device's
+// bit only after it has completed; a second host thread arriving meanwhile waits for the mutex and then
+// finds the bit set.  A set-up that returns early (an error) leaves the bit clear and is retried.
+constexpr int kMaxDevices = 64;
+inline std::mutex& device_setup_mutex() { static std::mutex m; return m; }
+struct DeviceSetup {
+  unsigned long long* mask;
+  unsigned long long bit;
+  int dev;
+  bool needed;
+  std::unique_lock<std::mutex> lock;
+  explicit DeviceSetup(unsigned long long* m) : mask(m), bit(0), dev(0), needed(true) {
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { dev = 0; return; }   // set up, never cached
+    bit = 1ull << dev;
+    if (__atomic_load_n(mask, __ATOMIC_ACQUIRE) & bit) { needed = false; return; }
+    lock = std::unique_lock<std::mutex>(device_setup_mutex());
+    needed = !(__atomic_load_n(mask, __ATOMIC_ACQUIRE) & bit);
+  }
+  explicit operator bool() const { return needed; }
+  void done() { if (bit) __atomic_fetch_or(mask, bit, __ATOMIC_RELEASE); }
+};
+inline int current_device_index() {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return true;
-  const unsigned long long bit = 1ull << (dev & 63);
-  if (__atomic_load_n(mask, __ATOMIC_ACQUIRE) & bit) return false;
-  __atomic_fetch_or(mask, bit, __ATOMIC_RELEASE);
-  return true;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  return dev;
 }
 
 }  // namespace grace

@@ -19,7 +19,8 @@ namespace grace {
 struct CrossSmallParams {
   const uint16_t* q; const uint16_t* k; const uint16_t* v; uint16_t* out; float* lse;
   int64_t q_row_stride, out_row_stride, kv_stride_b, kv_stride_h, kv_stride_t;
-  int R, M, H, T; float scale;
+  int R, M, H, T_ctx; float scale;
+  const int32_t* enc_len;        // nullable: valid encoder positions per request (small kernel only)
 };
 
 template <int DH>
@@ -33,6 +34,8 @@ cross_attn_small_kernel(const CrossSmallParams p) {
   if (item >= (int64_t)p.R * p.H) return;
   const int r = (int)(item / p.H), h = (int)(item % p.H);
   const int b = r / p.M;
+  int T = p.T_ctx;                             // valid encoder positions of this request
+  if (p.enc_len != nullptr) { const int e = __ldg(p.enc_len + b); T = e < 0 ? 0 : (e < T ? e : T); }
   const uint16_t* qp = p.q + (int64_t)r * p.q_row_stride + h * DH;
   const uint16_t* kb = p.k + (int64_t)b * p.kv_stride_b + (int64_t)h * p.kv_stride_h;
   const uint16_t* vb = p.v + (int64_t)b * p.kv_stride_b + (int64_t)h * p.kv_stride_h;
@@ -46,14 +49,14 @@ cross_attn_small_kernel(const CrossSmallParams p) {
   float acc[kPerLane];
 #pragma unroll
   for (int j = 0; j < kPerLane; ++j) acc[j] = 0.f;
-  for (int t0 = 0; t0 < p.T; t0 += kChunk) {
+  for (int t0 = 0; t0 < T; t0 += kChunk) {
     float s[kChunk / 32];
     float cmax = -INFINITY;
 #pragma unroll
     for (int i = 0; i < kChunk / 32; ++i) {
       const int t = t0 + i * 32 + lane;
       s[i] = -INFINITY;
-      if (t < p.T) {
+      if (t < T) {
         const uint4* kr = reinterpret_cast<const uint4*>(kb + (int64_t)t * p.kv_stride_t);
         float d = 0.f;
 #pragma unroll
@@ -76,7 +79,7 @@ cross_attn_small_kernel(const CrossSmallParams p) {
     __syncwarp();
 #pragma unroll
     for (int i = 0; i < kChunk / 32; ++i) {
-      const float e = (t0 + i * 32 + lane < p.T) ? __expf(s[i] - m_new) : 0.f;
+      const float e = (t0 + i * 32 + lane < T) ? __expf(s[i] - m_new) : 0.f;
       probs[warp][i * 32 + lane] = e;
       csum += e;
     }
@@ -87,7 +90,7 @@ cross_attn_small_kernel(const CrossSmallParams p) {
     __syncwarp();
 #pragma unroll
     for (int j = 0; j < kPerLane; ++j) acc[j] *= corr;
-    const int tn = min(kChunk, p.T - t0);
+    const int tn = min(kChunk, T - t0);
     for (int tt = 0; tt < tn; ++tt) {
       const float w = probs[warp][tt];
       const uint16_t* vr = vb + (int64_t)(t0 + tt) * p.kv_stride_t;
@@ -96,14 +99,14 @@ cross_attn_small_kernel(const CrossSmallParams p) {
         acc[j] = fmaf(w, __uint_as_float((uint32_t)__ldg(vr + j * 32 + lane) << 16), acc[j]);
     }
   }
-  const float inv = 1.f / l_run;
+  const float inv = l_run > 0.f ? 1.f / l_run : 0.f;          // no encoder position: the output is defined as zero
   uint16_t* op = p.out + (int64_t)r * p.out_row_stride + h * DH;
 #pragma unroll
   for (int j = 0; j < kPerLane; ++j) {
     __nv_bfloat16 o = __float2bfloat16_rn(acc[j] * inv);
     op[j * 32 + lane] = *reinterpret_cast<uint16_t*>(&o);
   }
-  if (p.lse != nullptr && lane == 0) p.lse[(int64_t)r * p.H + h] = m_run + logf(l_run);
+  if (p.lse != nullptr && lane == 0) p.lse[(int64_t)r * p.H + h] = l_run > 0.f ? m_run + logf(l_run) : -INFINITY;
 }
 
 // A handful of query rows per request (step 0 of a decode: one beam per request): the tensor-core kernel would
@@ -134,8 +137,8 @@ cross_attn_row_kernel(const CrossSmallParams p) {
     q[4] = bf16_lo(t4.z) * p.scale; q[5] = bf16_hi(t4.z) * p.scale; q[6] = bf16_lo(t4.w) * p.scale; q[7] = bf16_hi(t4.w) * p.scale;
   }
   // this warp's contiguous slice of the encoder positions, RP at a time
-  const int per_warp = (p.T + kWarps - 1) / kWarps;
-  const int t_begin = warp * per_warp, t_end = min(p.T, t_begin + per_warp);
+  const int per_warp = (p.T_ctx + kWarps - 1) / kWarps;
+  const int t_begin = warp * per_warp, t_end = min(p.T_ctx, t_begin + per_warp);
   float m_run = -INFINITY, l_run = 0.f;
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   // The op is bound by reading K and V once (a row per request: nothing is reused), so loads never stop: the
@@ -204,12 +207,13 @@ namespace grace {
 int cross_attn_tc_timeouts() { return tc::tc_timeouts_read_and_clear(); }
 }  // namespace grace
 
-extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
-                                           const uint16_t* k, const uint16_t* v,
-                                           int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
-                                           uint16_t* out, int64_t out_row_stride, float* lse,
-                                           int B, int M, int H, int d_h, int T_ctx, float scale,
-                                           int32_t* d_status, void* stream) {
+extern "C" grace_status_t grace_cross_attn_varlen(const uint16_t* q, int64_t q_row_stride,
+                                                  const uint16_t* k, const uint16_t* v,
+                                                  int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                                                  uint16_t* out, int64_t out_row_stride, float* lse,
+                                                  const int32_t* enc_len,
+                                                  int B, int M, int H, int d_h, int T_ctx, float scale,
+                                                  int32_t* d_status, void* stream) {
   using namespace grace;
   (void)d_status;
   if (!q || !k || !v || !out) return GRACE_INVALID_ARG;
@@ -220,31 +224,26 @@ extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stri
       q_row_stride < (int64_t)H * d_h || out_row_stride < (int64_t)H * d_h || kv_stride_t < d_h)
     return GRACE_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  if ((d_h == 64 || d_h == 128) && M <= 8 && (int64_t)B * M * H <= 1184) {
+  CrossSmallParams p;
+  p.q = q; p.k = k; p.v = v; p.out = out; p.lse = lse;
+  p.q_row_stride = q_row_stride; p.out_row_stride = out_row_stride;
+  p.kv_stride_b = kv_stride_b; p.kv_stride_h = kv_stride_h; p.kv_stride_t = kv_stride_t;
+  p.R = B * M; p.M = M; p.H = H; p.T_ctx = T_ctx; p.scale = scale; p.enc_len = enc_len;
+  if (enc_len == nullptr && (d_h == 64 || d_h == 128) && M <= 8 && (int64_t)B * M * H <= 1184) {
     // a few rows per request (step 0 of a decode): one CTA per (row, head), all resident at once
-    CrossSmallParams p;
-    p.q = q; p.k = k; p.v = v; p.out = out; p.lse = lse;
-    p.q_row_stride = q_row_stride; p.out_row_stride = out_row_stride;
-    p.kv_stride_b = kv_stride_b; p.kv_stride_h = kv_stride_h; p.kv_stride_t = kv_stride_t;
-    p.R = B * M; p.M = M; p.H = H; p.T = T_ctx; p.scale = scale;
     if (d_h == 64) launch_pdl(cross_attn_row_kernel<64>, dim3(B * M * H), dim3(256), 0, s, p);
     else launch_pdl(cross_attn_row_kernel<128>, dim3(B * M * H), dim3(256), 0, s, p);
     GRACE_LAUNCH_CHECK();
     return GRACE_OK;
   }
-  if (kUseMultiStream && cross_attn_ms_supported(B, M, H, d_h, T_ctx)) {
+  if (kUseMultiStream && cross_attn_ms_supported(B, M, H, d_h, T_ctx) && (enc_len == nullptr || M > 8)) {
     return launch_cross_attn_ms(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,
-                                out_row_stride, lse, nullptr, B, M, H, T_ctx, scale, s);
+                                out_row_stride, lse, enc_len, B, M, H, T_ctx, scale, s);
   }
-  if (cross_attn_tc_supported(B, M, H, d_h, T_ctx)) {
+  if (enc_len == nullptr && cross_attn_tc_supported(B, M, H, d_h, T_ctx)) {
     return launch_cross_attn_tc(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,
                                 out_row_stride, lse, B, M, H, d_h, T_ctx, scale, s);
   }
-  CrossSmallParams p;
-  p.q = q; p.k = k; p.v = v; p.out = out; p.lse = lse;
-  p.q_row_stride = q_row_stride; p.out_row_stride = out_row_stride;
-  p.kv_stride_b = kv_stride_b; p.kv_stride_h = kv_stride_h; p.kv_stride_t = kv_stride_t;
-  p.R = B * M; p.M = M; p.H = H; p.T = T_ctx; p.scale = scale;
   const int64_t items = (int64_t)p.R * H;
   const unsigned blocks = (unsigned)((items + 3) / 4);
   switch (d_h) {
@@ -254,4 +253,14 @@ extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stri
   }
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_cross_attn(const uint16_t* q, int64_t q_row_stride,
+                                           const uint16_t* k, const uint16_t* v,
+                                           int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                                           uint16_t* out, int64_t out_row_stride, float* lse,
+                                           int B, int M, int H, int d_h, int T_ctx, float scale,
+                                           int32_t* d_status, void* stream) {
+  return grace_cross_attn_varlen(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride, lse,
+                                 nullptr, B, M, H, d_h, T_ctx, scale, d_status, stream);
 }

@@ -481,12 +481,14 @@ inline grace_status_t launch_cross_attn_ms(const uint16_t* q, int64_t q_row_stri
     if (!tc::make_tmap_bf16(&mv, v, 4, dims, str, box)) return GRACE_CUDA_ERROR;
   }
   static unsigned long long attr_set_devices = 0;
-  if (first_use_on_device(&attr_set_devices)) {
+  static int n_sm_of[kMaxDevices] = {0};
+  DeviceSetup su(&attr_set_devices);
+  if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(cross_attn_ms_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMsSmemBytes));
+    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm_of[su.dev], cudaDevAttrMultiProcessorCount, su.dev));
+    su.done();
   }
-  int dev = 0, n_sm = 0;
-  GRACE_CUDA_TRY(cudaGetDevice(&dev));
-  GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  const int n_sm = n_sm_of[su.dev];
   CrossMsParams p;
   p.out = out; p.lse = lse; p.enc_len = enc_len; p.out_row_stride = out_row_stride;
   p.B = B; p.M = M; p.H = H; p.T = T_ctx;

@@ -390,3 +390,69 @@ unsigned long long g_grace_launches = 0;
 extern "C" uint64_t grace_kernel_launch_count(void) { return __atomic_load_n(&g_grace_launches, __ATOMIC_RELAXED); }
 extern "C" int grace_version(void) { return 1; }
 extern "C" int grace_built_for_sm(void) { return 100; }
+
+// ------------------------------------------------------------------------------------------------
+// Weight preparation for the folded-LayerNorm decode path (host memory in, host memory out)
+// ------------------------------------------------------------------------------------------------
+namespace {
+inline uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);   // NaN stays NaN
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+inline float bf16_to_f32(uint16_t b) {
+  const uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+}  // namespace
+
+extern "C" grace_status_t grace_f32_to_bf16(const float* a, int64_t n, uint16_t* out) {
+  if (!a || !out || n < 0) return GRACE_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) out[i] = f32_to_bf16_rne(a[i]);
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_fold_layer_norm(const float* w, const float* gamma, const float* beta,
+                                                int64_t N, int64_t K, uint16_t* w_folded, float* col_sum,
+                                                float* col_bias) {
+  if (!w || !gamma || !beta || !w_folded || !col_sum || !col_bias || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
+  for (int64_t n = 0; n < N; ++n) {
+    double cs = 0.0, cb = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+      const float wv = w[n * K + k];
+      const uint16_t b = f32_to_bf16_rne(wv * gamma[k]);       // the operand the GEMM will multiply with
+      w_folded[n * K + k] = b;
+      cs += (double)bf16_to_f32(b);                              // column sums of exactly those operands
+      cb += (double)wv * (double)beta[k];
+    }
+    col_sum[n] = (float)cs;
+    col_bias[n] = (float)cb;
+  }
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_centre_rows(const float* a, int64_t n, int64_t d, float* out) {
+  if (!a || !out || n <= 0 || d <= 0) return GRACE_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) {
+    double m = 0.0;
+    for (int64_t j = 0; j < d; ++j) m += (double)a[i * d + j];
+    m /= (double)d;
+    for (int64_t j = 0; j < d; ++j) out[i * d + j] = (float)((double)a[i * d + j] - m);
+  }
+  return GRACE_OK;
+}
+
+extern "C" grace_status_t grace_centre_outputs(const float* w, int64_t d_out, int64_t K, float* out) {
+  if (!w || !out || d_out <= 0 || K <= 0) return GRACE_INVALID_ARG;
+  std::vector<double> m((size_t)K, 0.0);
+  for (int64_t i = 0; i < d_out; ++i)
+    for (int64_t k = 0; k < K; ++k) m[(size_t)k] += (double)w[i * K + k];
+  for (int64_t k = 0; k < K; ++k) m[(size_t)k] /= (double)d_out;
+  for (int64_t i = 0; i < d_out; ++i)
+    for (int64_t k = 0; k < K; ++k) out[i * K + k] = (float)((double)w[i * K + k] - m[(size_t)k]);
+  return GRACE_OK;
+}

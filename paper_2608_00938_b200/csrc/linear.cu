@@ -494,7 +494,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
                                   int K, int relu, cudaStream_t s, float2* lse_part = nullptr,
                                   Affine aff = Affine{nullptr, nullptr, nullptr}) {
   static unsigned long long attr_set_devices = 0;
-  static int max_clusters = 0;
+  static int max_clusters_of[kMaxDevices] = {0};
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -502,16 +502,19 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
-  if (first_use_on_device(&attr_set_devices)) {
+  DeviceSetup su(&attr_set_devices);
+  if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
-    int dev = 0, n_sm = 0;
-    GRACE_CUDA_TRY(cudaGetDevice(&dev));
-    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    int n_sm = 0, clusters = 0;
+    GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, su.dev));
     cfg.gridDim = dim3(n_sm & ~1);
-    GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&max_clusters, linear_pair_kernel<OUT>, &cfg));
-    if (max_clusters <= 0) return GRACE_CUDA_ERROR;
-    if (max_clusters > n_sm / 2) max_clusters = n_sm / 2;
+    GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, linear_pair_kernel<OUT>, &cfg));
+    if (clusters <= 0) return GRACE_CUDA_ERROR;
+    if (clusters > n_sm / 2) clusters = n_sm / 2;
+    max_clusters_of[su.dev] = clusters;
+    su.done();
   }
+  const int max_clusters = max_clusters_of[su.dev];
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
   GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb));
@@ -522,9 +525,11 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
 template <int BN, int STAGES>
 static grace_status_t launch_linear(const CUtensorMap& mx, const CUtensorMap& mw, const GemmParams& p, cudaStream_t s) {
   static unsigned long long attr_set_devices = 0;
-  if (first_use_on_device(&attr_set_devices)) {
+  DeviceSetup su(&attr_set_devices);
+  if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         GemmSmem<BN, STAGES>::kTotal));
+    su.done();
   }
   dim3 grid((p.N + BN - 1) / BN, (p.M + kGemmBM - 1) / kGemmBM);
   launch_pdl(linear_kernel<BN, STAGES>, grid, dim3(128), GemmSmem<BN, STAGES>::kTotal, s, mx, mw, p);

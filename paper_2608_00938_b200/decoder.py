@@ -1,7 +1,11 @@
 """Buffer set-up for grace_decode_step: uploads weights and index structures,
 allocates the caller-owned state / cache / activation buffers with torch and
-fills the C struct.  No arithmetic happens here; every step of the decode path
-runs in the library's kernels."""
+fills the C struct.  No arithmetic happens here: every step of the decode path
+runs in the library's kernels, and the one-time weight preparation of the
+folded-LayerNorm configuration (gain folded into the weights, producers of the
+residual stream centred, bf16 conversion) is done by the library's host-side
+helpers (grace_fold_layer_norm, grace_centre_rows, grace_centre_outputs,
+grace_f32_to_bf16), so a caller of the C ABI gets the same operands."""
 from __future__ import annotations
 
 import ctypes as C
@@ -12,8 +16,13 @@ import torch
 from . import api
 
 
+def _bf16_bits(bits: np.ndarray, device) -> torch.Tensor:
+    """bf16 bit patterns (uint16) -> device bf16 tensor of the same shape."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
 def _bf16(a: np.ndarray, device) -> torch.Tensor:
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device).to(torch.bfloat16).contiguous()
+    return _bf16_bits(api.grace_f32_to_bf16(a), device)
 
 
 def _f32(a: np.ndarray, device) -> torch.Tensor:
@@ -68,19 +77,15 @@ class Decoder:
         self.centre_stream = centre_stream
 
         def centred_rows(a):                               # [n, d_model]: each row minus its mean
-            a = np.asarray(a, np.float64)
-            return (a - a.mean(axis=1, keepdims=True)).astype(np.float32) if centre_stream else a
+            return api.grace_centre_rows(a) if centre_stream else a
 
         def centred_outputs(w):                            # [d_model, K]: minus the mean over the output index
-            w = np.asarray(w, np.float64)
-            return (w - w.mean(axis=0, keepdims=True)).astype(np.float32) if centre_stream else w
+            return api.grace_centre_outputs(w) if centre_stream else w
 
         def fold(w, gamma, beta):
-            """(w * gamma as the bf16 the GEMM will use, column sums of that, beta @ w^T)."""
-            wf = _bf16(np.asarray(w, np.float32) * np.asarray(gamma, np.float32)[None, :], dev)
-            cs = wf.to(torch.float64).sum(dim=1).to(torch.float32).contiguous()
-            cb = torch.from_numpy((np.asarray(w, np.float64) @ np.asarray(beta, np.float64)).astype(np.float32)).to(dev)
-            return wf, cs, cb
+            """(w * gamma as the bf16 the GEMM will use, column sums of that, beta @ w^T), uploaded."""
+            wf, cs, cb = api.grace_fold_layer_norm(w, gamma, beta)
+            return _bf16_bits(wf, dev), torch.from_numpy(cs).to(dev), torch.from_numpy(cb).to(dev)
 
         self.folded = []                                   # per layer: {weight name: (folded weight, column sums, bias)}
         for li, lw in enumerate(weights["layers"]):

@@ -559,6 +559,58 @@ def test_cross_attn_strided_kv_layout(api):
     assert_attention_close(out.float().cpu().numpy().reshape(B, M, H, d), ref, "cross-attn strided")
 
 
+@pytest.mark.parametrize("B,M,H,d,T", [(5, 300, 4, 64, 200), (3, 520, 2, 64, 330), (4, 20, 2, 32, 70), (3, 40, 2, 128, 150)])
+def test_cross_attn_with_per_request_encoder_lengths(api, B, M, H, d, T):
+    """grace_cross_attn_varlen: every request attends to its own number of encoder positions (full, a block
+    boundary, one, none, ragged); positions beyond it must have no influence, whatever they hold."""
+    rng = synth.rng_for(2, 900 + M + T)
+    q = synth.normal_bf16(rng, (B, M, H, d))
+    k = synth.normal_bf16(rng, (B, H, T, d))
+    v = synth.normal_bf16(rng, (B, H, T, d))
+    enc_len = np.array([T, 64, 1, 0, T - 37][:B], dtype=np.int32)
+    scale = d ** -0.5
+    ref, lse_ref = OA.cross_attn_varlen(f64(q), f64(k), f64(v), enc_len, scale)
+    # poison the padding: huge keys and values beyond each request's length
+    kf, vf = synth.bf16_bits_to_f32(k).copy(), synth.bf16_bits_to_f32(v).copy()
+    for b in range(B):
+        kf[b, :, enc_len[b]:] = 50.0
+        vf[b, :, enc_len[b]:] = -1000.0
+    out = torch.full((B * M, H, d), 7.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros((B * M, H), dtype=torch.float32, device=DEV)
+    api.grace_cross_attn_varlen(dev_bf16(q).reshape(B * M, H, d), dev(kf).to(torch.bfloat16), dev(vf).to(torch.bfloat16),
+                                out, dev(enc_len), scale, lse)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().reshape(B, M, H, d)
+    assert_attention_close(got, ref, "cross-attn varlen")
+    empty = enc_len == 0
+    assert (got[empty] == 0).all()
+    got_lse = lse.cpu().numpy().reshape(B, M, H)
+    assert np.isneginf(got_lse[empty]).all()
+    np.testing.assert_allclose(got_lse[~empty], lse_ref[~empty], atol=2e-3, rtol=0)
+
+
+def test_cross_attn_with_scores_that_keep_growing(api):
+    """Keys whose scores rise along the encoder positions by far more than the lazy-rescaling threshold
+    (2^16 between neighbouring blocks): the running maximum moves in almost every block and the output
+    accumulator is rescaled under way; and rows whose maximum sits in the first block, where it never is."""
+    B, M, H, d, T = 2, 300, 2, 64, 640
+    rng = synth.rng_for(2, 950)
+    q = np.abs(synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, M, H, d)))) + 0.5     # positive queries
+    q[:, ::2] *= -1.0                                                                  # every second row: scores fall instead
+    ramp = np.linspace(0.0, 9.0, T, dtype=np.float32)[None, None, :, None]
+    k = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, H, T, d))) * 0.1 + ramp
+    v = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, H, T, d)))
+    qb, kb, vb = synth.f32_to_bf16_bits(q), synth.f32_to_bf16_bits(k), synth.f32_to_bf16_bits(v)
+    scale = 0.125
+    ref, _ = OA.cross_attn(f64(qb), f64(kb), f64(vb), scale)
+    s_first = (f64(qb)[0, 1, 0] @ f64(kb)[0, 0].T) * scale * np.log2(np.e)
+    assert s_first[-1] - s_first[63] > 100.0                    # several thresholds of growth for the rising rows
+    out = torch.zeros((B * M, H, d), dtype=torch.bfloat16, device=DEV)
+    api.grace_cross_attn(dev_bf16(qb).reshape(B * M, H, d), dev_bf16(kb), dev_bf16(vb), out, scale)
+    torch.cuda.synchronize()
+    assert_attention_close(out.float().cpu().numpy().reshape(B, M, H, d), ref, "cross-attn growing scores")
+
+
 # ------------------------------------------------------------------------------------------
 # decoder glue
 # ------------------------------------------------------------------------------------------

@@ -147,3 +147,63 @@ def test_kway_index_builder_matches_oracle(api, policy):
     assert np.array_equal(one["bitmask_table"][one["bitmask_index"]], plain["bitmask_table"][plain["bitmask_index"]])
     with pytest.raises(api.GraceError):
         api.grace_gtm_index_build_kway(sids, V, ad_sid, ad_bm, ad_bl, k_level=[0] * (L + 1))
+
+
+def test_layer_norm_fold_and_centring_helpers(api):
+    """The host-side weight preparation of the folded-LayerNorm path against its definition in fp64:
+    with the helper's outputs, rstd * (x @ w'^T) - rstd * mean * col_sum + col_bias equals LayerNorm(x) @ w^T up
+    to the one bf16 rounding of w * gamma; centred rows / outputs have zero mean along the stream's feature
+    axis and differ from the input by exactly that mean; and running the oracle's decoder on weights centred
+    by the helpers changes no log-probability (the identity the product path relies on)."""
+    rng = synth.rng_for(1, 901)
+    N, K, R = 96, 160, 40
+    w = synth.normal_f32(rng, (N, K)) * 0.3
+    gamma = (1.0 + 0.3 * synth.normal_f32(rng, K)).astype(np.float32)
+    beta = (0.4 * synth.normal_f32(rng, K)).astype(np.float32)
+    x = (synth.normal_f32(rng, (R, K)) * 2.0 + 0.7).astype(np.float64)
+    wf_bits, cs, cb = api.grace_fold_layer_norm(w, gamma, beta)
+    wf = synth.bf16_bits_to_f32(wf_bits).astype(np.float64)
+    exact = w.astype(np.float64) * gamma.astype(np.float64)[None, :]
+    assert (np.abs(wf - exact) <= 2.0 ** -8 * np.abs(exact)).all()               # one rounding to bf16 (half an ulp of 8 bits)
+    assert np.array_equal(wf_bits, synth.f32_to_bf16_bits((w * gamma[None, :]).astype(np.float32)))
+    np.testing.assert_allclose(cs, wf.sum(axis=1), rtol=1e-6, atol=1e-6)         # sums of the ROUNDED operands
+    np.testing.assert_allclose(cb, w.astype(np.float64) @ beta.astype(np.float64), rtol=1e-6, atol=1e-6)
+    mean, var = x.mean(axis=1, keepdims=True), x.var(axis=1, keepdims=True)
+    rstd = 1.0 / np.sqrt(var + 1e-5)
+    ln = (x - mean) * rstd * gamma[None, :] + beta[None, :]
+    folded = rstd * (x @ wf.T) - rstd * mean * cs[None, :].astype(np.float64) + cb[None, :].astype(np.float64)
+    ref_rounded = ((x - mean) * rstd) @ wf.T + beta.astype(np.float64) @ w.astype(np.float64).T
+    np.testing.assert_allclose(folded, ref_rounded, rtol=0, atol=2e-5)           # the identity itself (same operands)
+    # and the cost of rounding w * gamma to bf16: at most 2^-8 of every product, element by element
+    assert (np.abs(folded - ln @ w.astype(np.float64).T) <= 2.0 ** -8 * (np.abs((x - mean) * rstd) @ np.abs(exact).T) + 1e-6).all()
+    # centring
+    a = (synth.normal_f32(rng, (50, K)) + 1.5).astype(np.float32)
+    ca = api.grace_centre_rows(a)
+    np.testing.assert_allclose(ca.astype(np.float64).mean(axis=1), 0.0, atol=1e-6)
+    np.testing.assert_allclose(ca, a.astype(np.float64) - a.astype(np.float64).mean(axis=1, keepdims=True), rtol=0, atol=1e-6)
+    wo = (synth.normal_f32(rng, (K, 70)) + 0.3).astype(np.float32)               # [stream features, inputs]
+    co = api.grace_centre_outputs(wo)
+    np.testing.assert_allclose(co.astype(np.float64).mean(axis=0), 0.0, atol=1e-6)
+    np.testing.assert_allclose(co, wo.astype(np.float64) - wo.astype(np.float64).mean(axis=0, keepdims=True), rtol=0, atol=1e-6)
+    h = synth.normal_f32(rng, (9, 70)).astype(np.float64)
+    np.testing.assert_allclose((h @ co.astype(np.float64).T).mean(axis=1), 0.0, atol=1e-5)   # outputs have zero mean
+    bits = api.grace_f32_to_bf16(a)
+    assert np.array_equal(bits, synth.f32_to_bf16_bits(a))
+    # the oracle's decoder on helper-centred weights: no log-probability moves
+    import copy
+    from oracle import decoder as D
+    shp = synth.DecoderShape(2, 64, 4, 16, 128, 48, 32, 3)
+    wts = synth.decoder_weights(synth.rng_for(1, 902), shp, std=0.2, as_bf16=False)
+    wts["embed"] = np.asarray(wts["embed"], np.float64) + 1.5
+    enc = synth.normal_f32(rng, (2, 10, 48)).astype(np.float64)
+
+    def log_probs(wd):
+        state = D.DecoderState(shp, 2, [1, 1])
+        return D.decoder_forward(wd, shp, state, D.cross_kv(wd, shp, enc), np.full(2, shp.V), 0, 2)
+    c = copy.deepcopy(wts)
+    c["embed"] = api.grace_centre_rows(c["embed"]).astype(np.float64)
+    c["pos"] = api.grace_centre_rows(c["pos"]).astype(np.float64)
+    for lw in c["layers"]:
+        for name in ("w_o", "w_oc", "w_2"):
+            lw[name] = api.grace_centre_outputs(lw[name]).astype(np.float64)
+    np.testing.assert_allclose(log_probs(c), log_probs(wts), rtol=0, atol=2e-5)  # fp32 storage of the centred weights

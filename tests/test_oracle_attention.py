@@ -186,3 +186,33 @@ def test_bf16_round_trip_is_rne():
     assert abs(back[6] - 0.1) <= 0.1 * 2 ** -8
     import torch
     assert torch.equal(torch.from_numpy(x).to(torch.bfloat16).float(), torch.from_numpy(back))
+
+
+def test_cross_attn_with_encoder_lengths_is_attention_over_the_truncated_encoder():
+    """`cross_attn_varlen`: pure-Python softmax over each request's first enc_len positions; padding beyond
+    them has no influence; a request without positions gets zeros."""
+    rng = np.random.default_rng(11)
+    B, M, H, d, T = 3, 4, 2, 5, 9
+    q, k, v = rng.normal(size=(B, M, H, d)), rng.normal(size=(B, H, T, d)), rng.normal(size=(B, H, T, d))
+    enc_len = [9, 4, 0]
+    out, lse = A.cross_attn_varlen(q, k, v, enc_len, 0.3)
+    k2, v2 = k.copy(), v.copy()
+    for b in range(B):
+        k2[b, :, enc_len[b]:] = 1e3
+        v2[b, :, enc_len[b]:] = -1e3
+    out2, _ = A.cross_attn_varlen(q, k2, v2, enc_len, 0.3)
+    assert np.array_equal(out, out2)
+    for b in range(B):
+        for m in range(M):
+            for h in range(H):
+                n = enc_len[b]
+                if n == 0:
+                    assert (out[b, m, h] == 0).all() and lse[b, m, h] == -np.inf
+                    continue
+                s = [0.3 * sum(q[b, m, h, i] * k[b, h, t, i] for i in range(d)) for t in range(n)]
+                mx = max(s)
+                w = [np.exp(x - mx) for x in s]
+                z = sum(w)
+                want = [sum(w[t] * v[b, h, t, i] for t in range(n)) / z for i in range(d)]
+                np.testing.assert_allclose(out[b, m, h], want, rtol=1e-12, atol=1e-12)
+                np.testing.assert_allclose(lse[b, m, h], mx + np.log(z), rtol=1e-12)
