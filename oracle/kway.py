@@ -36,7 +36,7 @@ def _popcount_rows(rows: np.ndarray) -> np.ndarray:
 
 
 def sid_rows(n_sids: int, ad_sid: np.ndarray, ad_bitmask: np.ndarray, ad_bloom: np.ndarray):
-    """Rows of a SID = OR of the rows of its ads (Section 4.2: 'the bitwise OR over all ads under it')."""
+    """Rows of a SID = OR of the rows of its ads (the union rule of Section 4.2 applied at the leaf)."""
     order = np.argsort(ad_sid, kind="stable")
     starts = np.searchsorted(ad_sid[order], np.arange(n_sids))
     return (np.bitwise_or.reduceat(ad_bitmask[order], starts, axis=0),

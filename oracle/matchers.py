@@ -52,16 +52,23 @@ def bloom_any(stored: np.ndarray, user_location_rows) -> bool:
 
 def paper_lookup(trie, bitmask_index, bloom_index, bitmask_table, bloom_table,
                  node_id: int, user_bitmask, user_blooms):
-    """Appendix A lookup: the (token, child node) pairs a request may extend to."""
-    start = int(trie.node_offsets[node_id])
-    end = int(trie.node_offsets[node_id + 1])
-    emitted = []
-    for j in range(start, end):
-        ok_bm = bitmask_match(bitmask_table[bitmask_index[j]], user_bitmask)
-        ok_bl = bloom_any(bloom_table[bloom_index[j]], user_blooms)
-        if ok_bm and ok_bl:
-            emitted.append((int(trie.csr_tokens[j]), int(trie.csr_child_nodes[j])))
-    return emitted
+    """The index lookup of Appendix A for one node and one request: the (token, child node) pairs the
+    request may extend the node's prefix with.
+
+    Stated as a filter over the node's child entries (the CSR range of the node): an entry survives iff its
+    attribute row contains the request's attribute row (Section 4.2) and its Bloom row contains at least one
+    of the request's location rows (Section 4.3; none at all if the request has no location)."""
+    entries = np.arange(int(trie.node_offsets[node_id]), int(trie.node_offsets[node_id + 1]))
+    if entries.size == 0:
+        return []
+    attr_rows = np.asarray(bitmask_table)[np.asarray(bitmask_index)[entries]]           # [n, W_bm]
+    bloom_rows = np.asarray(bloom_table)[np.asarray(bloom_index)[entries]]              # [n, W_bl]
+    want = np.asarray(user_bitmask, dtype=U64)
+    attr_ok = ((attr_rows & want[None, :]) == want[None, :]).all(axis=1)
+    locs = np.asarray(user_blooms, dtype=U64).reshape(-1, bloom_rows.shape[1])          # [N_loc, W_bl]
+    loc_ok = ((bloom_rows[:, None, :] & locs[None, :, :]) == locs[None, :, :]).all(axis=2).any(axis=1)
+    keep = entries[attr_ok & loc_ok]
+    return [(int(trie.csr_tokens[j]), int(trie.csr_child_nodes[j])) for j in keep]
 
 
 # ---------------------------------------------------------------------------
