@@ -1,18 +1,18 @@
 // Cross-attention in the beam-as-query layout (Section 5.1, Appendix B): the M beams of a request
 // are M query rows against that request's one copy of K and V.
 //
-// Two kernels behind one entry point:
-//   * cross_attn_tc_kernel (cross_attn_tc.cuh): tcgen05 / TMEM / TMA flash attention for
-//     d_h = 64, the serving shapes.
+// Four kernels behind one entry point:
+//   * cross_attn_ms_kernel (cross_attn_ms.cuh): tcgen05 / TMEM / TMA, four softmax streams per SM,
+//     head size 64: the serving shapes.
+//   * cross_attn_tc_kernel (cross_attn_tc.cuh): tcgen05 / TMEM / TMA flash attention, head size 128.
+//   * cross_attn_row_kernel (below): a handful of query rows per request (step 0 of a decode).
 //   * cross_attn_small_kernel (below): a plain CUDA-core kernel for everything else (tiny
-//     configurations, d_h = 32 or 128, unaligned strides).  One warp per (row, head); lanes split
-//     the encoder positions for the scores and the head dimension for the weighted sum.
+//     configurations, d_h = 32, per-request encoder lengths at head size 128).  One warp per (row,
+//     head); lanes split the encoder positions for the scores and the head dimension for the sum.
 #include "common.cuh"
 #include "cross_attn_tc.cuh"
 #include "cross_attn_ms.cuh"
 
-// The four-stream kernel is selected here once it beats the two-CTA kernel on every benchmark shape.
-static constexpr bool kUseMultiStream = true;
 
 namespace grace {
 
@@ -236,7 +236,7 @@ extern "C" grace_status_t grace_cross_attn_varlen(const uint16_t* q, int64_t q_r
     GRACE_LAUNCH_CHECK();
     return GRACE_OK;
   }
-  if (kUseMultiStream && cross_attn_ms_supported(B, M, H, d_h, T_ctx) && (enc_len == nullptr || M > 8)) {
+  if (cross_attn_ms_supported(B, M, H, d_h, T_ctx) && (enc_len == nullptr || M > 8)) {
     return launch_cross_attn_ms(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out,
                                 out_row_stride, lse, enc_len, B, M, H, T_ctx, scale, s);
   }

@@ -1,5 +1,6 @@
 // Cross-attention on tcgen05 tensor cores (Section 5.1: beams of a request are the M dimension of
-// a dense contraction against that request's shared K/V), head size 64 or 128.
+// a dense contraction against that request's shared K/V).  Written for head size 64 or 128; the library
+// uses it for head size 128 (head size 64 runs the four-stream kernel of cross_attn_ms.cuh).
 //
 // A work item is 128 query rows of one (request, head); its encoder positions are streamed in
 // blocks of 128:
@@ -427,7 +428,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 }
 
 inline bool cross_attn_tc_supported(int B, int M, int H, int d_h, int T_ctx) {
-  return (d_h == 64 || d_h == 128) && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;
+  return d_h == 128 && H <= 65535 && B <= 65535 && T_ctx >= 1 && M >= 1;      // head size 64: cross_attn_ms.cuh
 }
 
 template <int DH, int TPR>
@@ -477,11 +478,9 @@ inline grace_status_t launch_cross_attn_tc(const uint16_t* q, int64_t q_row_stri
                                            const uint16_t* v, int64_t kv_stride_b, int64_t kv_stride_h,
                                            int64_t kv_stride_t, uint16_t* out, int64_t out_row_stride, float* lse,
                                            int B, int M, int H, int d_h, int T_ctx, float scale, cudaStream_t s) {
-  if (d_h == 128)
-    return launch_cross_attn_tc_dh<128, 2>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
+  (void)d_h;                                                // 128 (cross_attn_tc_supported)
+  return launch_cross_attn_tc_dh<128, 2>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
                                         lse, B, M, H, T_ctx, scale, s);
-  return launch_cross_attn_tc_dh<64, 1>(q, q_row_stride, k, v, kv_stride_b, kv_stride_h, kv_stride_t, out, out_row_stride,
-                                     lse, B, M, H, T_ctx, scale, s);
 }
 
 }  // namespace grace
