@@ -24,6 +24,7 @@ constexpr int kSamplePoints = 4096;
 constexpr int kSampleSize = kSamplePoints * 8;
 constexpr int kTopkThreads = 1024;
 constexpr int kMaxK = 4096;              // largest K supported
+constexpr int kBucketMax = 128;          // finalize: largest bucket the counting sort ranks by comparison
 
 struct TopkHeader {                      // lives in the workspace, one per request
   uint32_t count;                        // entries appended (may exceed kCap: overflow)
@@ -134,18 +135,18 @@ __device__ __forceinline__ uint32_t pick_digit(const uint32_t* hist, int nbins, 
 }
 
 // ---- 1. sample -------------------------------------------------------------------------------
-// Each thread reads 4 sample points (32 keys) and keeps its two largest; the threshold is the
-// r-th largest of those 2 * 1024 keys.  Dropping a thread's third-largest key can only lower the
+// Each thread reads 4 sample points (32 keys) and keeps its two largest; the threshold is at (or a few
+// keys below) the r-th largest of those 2 * 1024 keys.  Dropping a thread's third-largest key can only lower the
 // threshold (more candidates collected), never raise it, so the guarantee "at least K above the
 // threshold with high probability" is kept while the selection works on 2048 keys instead of 32768.
 __global__ void __launch_bounds__(kTopkThreads)
 topk_sample_kernel(const CandSrc src, uint32_t rank, TopkHeader* hdr) {
   pdl_wait();
   pdl_trigger();
-  __shared__ uint32_t keys[2 * kTopkThreads];
   __shared__ uint32_t hist[4096];
   __shared__ uint32_t scratch[40];
   __shared__ uint32_t result[2];
+  __shared__ uint32_t red[64];
   const int b = blockIdx.x;
   const int64_t N = src.N;
   const int64_t stratum = (N / kSamplePoints) & ~(int64_t)7;       // multiple of 8 elements
@@ -170,25 +171,42 @@ topk_sample_kernel(const CandSrc src, uint32_t rank, TopkHeader* hdr) {
       else if (u > top2) top2 = u;
     }
   }
-  keys[2 * threadIdx.x] = top1;
-  keys[2 * threadIdx.x + 1] = top2;
-  uint32_t k = rank, prefix = 0;
-  const int shifts[3] = {20, 8, 0};
-  const int bits[3] = {12, 12, 8};
+  // The threshold need not be the r-th largest key itself: any value at or below it with few keys in
+  // between will do.  So instead of a full radix selection, histogram the keys over 4096 equal ranges
+  // between the smallest and the largest, take the lower edge of the range that holds rank r, and look
+  // closer (the same again inside that range) only while the range holds more than a few keys, which
+  // happens when an outlier stretches the span.
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t kmin = top2, kmax = top1;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(kFullMask, kmin, d));
+    kmax = max(kmax, __shfl_xor_sync(kFullMask, kmax, d));
+  }
+  if (lane == 0) { red[warp] = kmin; red[32 + warp] = kmax; }
+  __syncthreads();
+  kmin = red[lane];
+  kmax = red[32 + lane];
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(kFullMask, kmin, d));
+    kmax = max(kmax, __shfl_xor_sync(kFullMask, kmax, d));
+  }
+  uint32_t k = rank, lo = kmin, span = kmax - kmin, prefix = kmin;
 #pragma unroll 1
-  for (int level = 0; level < 3; ++level) {
-    const int nb = 1 << bits[level];
+  for (int level = 0; level < 4; ++level) {
+    const int sh = max(0, 20 - __clz(span));                 // span >> sh < 4096
     for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
     __syncthreads();
-    const int hi_shift = shifts[level] + bits[level];
-    for (int i = threadIdx.x; i < 2 * kTopkThreads; i += kTopkThreads) {
-      const uint32_t u = keys[i];
-      const bool match = (level == 0) || ((u >> hi_shift) == prefix);
-      if (match) atomicAdd(&hist[(u >> shifts[level]) & (nb - 1)], 1u);
-    }
+    if (top1 - lo <= span) atomicAdd(&hist[(top1 - lo) >> sh], 1u);
+    if (top2 - lo <= span) atomicAdd(&hist[(top2 - lo) >> sh], 1u);
     __syncthreads();
-    const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
-    prefix = (prefix << bits[level]) | d;
+    const uint32_t d = pick_digit(hist, 4096, &k, scratch, result);
+    const uint32_t in_range = hist[d];
+    prefix = lo + (d << sh);                                 // at least `rank` keys are >= prefix
+    if (sh == 0 || in_range <= 4u) break;
+    lo = prefix;
+    span = (1u << sh) - 1u;
   }
   if (threadIdx.x == 0) {
     hdr[b].count = 0;
@@ -207,111 +225,101 @@ __global__ void topk_reset_kernel(TopkHeader* hdr, int B) {
 // ---- 2. collect ------------------------------------------------------------------------------
 constexpr int kCollectThreads = 256;
 constexpr int kCollectUnroll = 8;                         // float4 loads in flight per thread
+constexpr int kCollectWarps = kCollectThreads / 32;
 
-constexpr int kStage = 1024;                              // hits staged per CTA before a flush
+constexpr int kStage = 1024;                              // hits staged per CTA before a flush (masked pass)
+constexpr int kWarpStage = 256;                           // hits staged per warp before a flush (dense pass)
+
+// Appends the warp's staged hits to the request's list with one global atomic; returns true once the list
+// has overflowed (the exact path will redo the request, so the caller may stop scanning).
+__device__ __forceinline__ bool warp_flush(uint2* wstage, uint32_t* wcount, uint32_t* list_count, uint2* list) {
+  __syncwarp();
+  const int lane = threadIdx.x & 31;
+  const uint32_t n = *reinterpret_cast<volatile uint32_t*>(wcount);
+  if (n == 0) return false;
+  uint32_t dst = 0;
+  if (lane == 0) dst = atomicAdd(list_count, n);
+  dst = __shfl_sync(kFullMask, dst, 0);
+  for (uint32_t e = lane; e < n; e += 32)
+    if (dst + e < (uint32_t)kCap) list[dst + e] = wstage[e];
+  __syncwarp();
+  if (lane == 0) *reinterpret_cast<volatile uint32_t*>(wcount) = 0;
+  __syncwarp();
+  return dst + n > (uint32_t)kCap;
+}
+
+// One float4 of candidates with at least one lane of the warp above the threshold (entered warp-uniformly).
+__device__ __forceinline__ bool collect_hits(const float4 v, bool mine, uint32_t i4, float thr, uint2* wstage,
+                                             uint32_t* wcount, uint32_t* list_count, uint2* list, bool* saw_nan) {
+  bool dead = false;
+  if (*reinterpret_cast<volatile uint32_t*>(wcount) > (uint32_t)(kWarpStage - 128))
+    dead = warp_flush(wstage, wcount, list_count, list);
+  if (mine) {
+    const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (!(x[j] <= thr)) {
+        if (x[j] != x[j]) { *saw_nan = true; continue; }
+        const uint32_t pos = atomicAdd(wcount, 1u);
+        wstage[pos] = make_uint2(ordered_key(x[j]), i4 * 4u + (uint32_t)j);
+      }
+    }
+  }
+  __syncwarp();
+  return dead;
+}
 
 __global__ void __launch_bounds__(kCollectThreads, 5)
 topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d_status) {
   pdl_wait();
   pdl_trigger();
-  // grid (x, B): the CTAs of column b share request b's tiles round-robin.  Hits are rare (a
-  // fraction of a percent), so they are staged in shared memory and appended to the request's
-  // list with ONE global atomic per flush; a per-hit or per-warp atomic on the single per-request
-  // counter serialises in L2.
-  __shared__ uint2 stage[kStage];
-  __shared__ uint32_t stage_count, flush_base;
+  // grid (x, B): the CTAs of column b split request b's candidates into contiguous, equal chunks of whole
+  // 256-float4 rows.  Hits are a fraction of a percent; each warp stages its own in shared memory (a
+  // shared-memory atomic per hit, no scan) and appends them to the request's list with ONE global atomic
+  // per flush, so the loop has no block-wide barrier and the per-request counter sees a few hundred atomics.
+  __shared__ uint2 stage[kCollectWarps][kWarpStage];
+  __shared__ uint32_t stage_count[kCollectWarps];
   const int b = blockIdx.y;
-  const int64_t n4 = src.N >> 2;
+  const int warp = threadIdx.x >> 5;
+  uint2* wstage = stage[warp];
+  uint32_t* wcount = &stage_count[warp];
+  if ((threadIdx.x & 31) == 0) *wcount = 0;
+  __syncwarp();
+  const uint32_t n4 = (uint32_t)(src.N >> 2);
+  const float4* row = reinterpret_cast<const float4*>(src.data + (int64_t)b * src.N);
   uint2* list = lists + (int64_t)b * kCap;
-  const int lane = threadIdx.x & 31;
-  const int64_t tile = (int64_t)kCollectThreads * kCollectUnroll;
-  bool saw_nan = false;
-  uint32_t t_excl = 0;
-  float thr = 0.f;
-  bool have_threshold = false;
-  if (threadIdx.x == 0) stage_count = 0;
-  __syncthreads();
-  for (int64_t base = (int64_t)blockIdx.x * tile; base < n4; base += (int64_t)gridDim.x * tile) {
+  uint32_t* list_count = &hdr[b].count;
+  const uint32_t rows_total = (n4 + kCollectThreads - 1) / kCollectThreads;
+  const uint32_t rows_per_cta = (rows_total + gridDim.x - 1) / gridDim.x;
+  uint32_t r = blockIdx.x * rows_per_cta;
+  const uint32_t r_end = min(rows_total, r + rows_per_cta);
+  const uint32_t r_full = min(r_end, n4 / kCollectThreads);      // rows below this one are wholly in bounds
+  const uint32_t t_excl = __ldcg(&hdr[b].t_excl);
+  // the same threshold as a float: key(x) > t_excl  <=>  x > thr for every non-NaN x
+  const float thr = __uint_as_float((t_excl & 0x80000000u) ? (t_excl ^ 0x80000000u) : ~t_excl);
+  bool saw_nan = false, dead = false;
+  for (; r + kCollectUnroll <= r_full && !dead; r += kCollectUnroll) {
+    const uint32_t i0 = r * kCollectThreads + threadIdx.x;
     float4 v[kCollectUnroll];
 #pragma unroll
-    for (int u = 0; u < kCollectUnroll; ++u) {
-      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
-      v[u] = (i < n4) ? src.load4(b, i, true) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    }
-    if (!have_threshold) {                     // after the first loads are in flight
-      t_excl = __ldcg(&hdr[b].t_excl);
-      // the same threshold as a float: key(x) > t_excl  <=>  x > thr for every non-NaN x
-      thr = __uint_as_float((t_excl & 0x80000000u) ? (t_excl ^ 0x80000000u) : ~t_excl);
-      have_threshold = true;
-    }
+    for (int u = 0; u < kCollectUnroll; ++u) v[u] = __ldcs(row + i0 + u * kCollectThreads);
 #pragma unroll
     for (int u = 0; u < kCollectUnroll; ++u) {
-      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
-      const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-      // !(x <= thr): above the threshold, or NaN (sorted out below)
-      const uint32_t hits = (uint32_t)!(x[0] <= thr) + (uint32_t)!(x[1] <= thr) + (uint32_t)!(x[2] <= thr) +
-                            (uint32_t)!(x[3] <= thr);
-      if (__any_sync(kFullMask, hits != 0)) {
-        uint32_t key[4];
-        uint32_t real = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          key[j] = ordered_key(x[j]);
-          if (x[j] != x[j]) { saw_nan = true; key[j] = 0; }
-          real += (key[j] > t_excl) ? 1u : 0u;
-        }
-        const uint32_t incl = warp_incl_scan(real);
-        const uint32_t total = __shfl_sync(kFullMask, incl, 31);
-        uint32_t start = 0, gbase = 0;
-        if (lane == 31 && total != 0) {
-          start = atomicAdd(&stage_count, total);
-          // entries that land beyond the stage go straight to the request's list, with their own
-          // reservation there (a run of hits, e.g. thousands of tied candidates, can exceed it)
-          const uint32_t first_over = max(start, (uint32_t)kStage);
-          if (start + total > first_over) gbase = atomicAdd(&hdr[b].count, start + total - first_over);
-        }
-        start = __shfl_sync(kFullMask, start, 31);
-        gbase = __shfl_sync(kFullMask, gbase, 31);
-        const uint32_t first_over = max(start, (uint32_t)kStage);
-        uint32_t pos = start + incl - real;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if (key[j] > t_excl) {
-            const uint2 entry = make_uint2(key[j], (uint32_t)(i * 4 + j));
-            if (pos < (uint32_t)kStage) {
-              stage[pos] = entry;
-            } else {
-              const uint32_t g = gbase + (pos - first_over);
-              if (g < (uint32_t)kCap) list[g] = entry;
-            }
-            ++pos;
-          }
-        }
-      }
-    }
-    // flush when the stage is at least half full
-    __syncthreads();
-    const uint32_t staged = min(stage_count, (uint32_t)kStage);
-    if (staged >= (uint32_t)kStage / 2) {
-      if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
-      __syncthreads();
-      const uint32_t dst = flush_base;
-      for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
-        if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
-      __syncthreads();
-      if (threadIdx.x == 0) stage_count = 0;
-      __syncthreads();
+      // !(x <= thr): above the threshold, or NaN
+      const bool mine = !(v[u].x <= thr) || !(v[u].y <= thr) || !(v[u].z <= thr) || !(v[u].w <= thr);
+      if (__any_sync(kFullMask, mine))
+        dead |= collect_hits(v[u], mine, i0 + u * kCollectThreads, thr, wstage, wcount, list_count, list, &saw_nan);
     }
   }
-  __syncthreads();
-  const uint32_t staged = min(stage_count, (uint32_t)kStage);
-  if (staged != 0) {
-    if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
-    __syncthreads();
-    const uint32_t dst = flush_base;
-    for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
-      if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
+  for (; r < r_end && !dead; ++r) {
+    const uint32_t i = r * kCollectThreads + threadIdx.x;
+    const float ninf = __int_as_float(0xff800000);
+    const float4 v = (i < n4) ? __ldcs(row + i) : make_float4(ninf, ninf, ninf, ninf);
+    const bool mine = !(v.x <= thr) || !(v.y <= thr) || !(v.z <= thr) || !(v.w <= thr);
+    if (__any_sync(kFullMask, mine))
+      dead |= collect_hits(v, mine, i, thr, wstage, wcount, list_count, list, &saw_nan);
   }
+  warp_flush(wstage, wcount, list_count, list);
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
 }
 
@@ -556,6 +564,7 @@ topk_finalize_kernel(const CandSrc src, int K, int K_out, int V, TopkHeader* hdr
   unsigned long long* sort_keys = sort_keys_raw;
   __shared__ uint32_t scratch[40];
   __shared__ uint32_t result[2];
+  __shared__ uint32_t red[64];
   const int b = blockIdx.x;
   uint32_t c = hdr[b].count;
   // Exact multi-pass selection when the sampled threshold did not deliver (list short although the
@@ -570,73 +579,162 @@ topk_finalize_kernel(const CandSrc src, int K, int K_out, int V, TopkHeader* hdr
   c = min(c, (uint32_t)kCap);
   const uint2* list = lists + (int64_t)b * kCap;
   unsigned long long* all_keys = sort_keys;                 // c composite keys (value key, ~index)
-  unsigned long long* top_keys = sort_keys + kCap;          // the K winners, sorted in place
-  uint32_t* hist = reinterpret_cast<uint32_t*>(top_keys + kMaxK);
+  unsigned long long* top_keys = sort_keys + kCap;          // the K winners (fast path: plus one bucket's overhang)
+  uint32_t* hist = reinterpret_cast<uint32_t*>(top_keys + kMaxK + kBucketMax);
+  uint32_t* offs = hist + 4096;
+  const int64_t N = src.N;
+  const uint32_t n_out = min(c, (uint32_t)K);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
   for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads) {
     const uint2 e = list[i];
     all_keys[i] = ((unsigned long long)e.x << 32) | (unsigned long long)(0xffffffffu - e.y);
+    kmin = min(kmin, e.x);
+    kmax = max(kmax, e.x);
   }
+  for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(kFullMask, kmin, d));
+    kmax = max(kmax, __shfl_xor_sync(kFullMask, kmax, d));
+  }
+  if (lane == 0) { red[warp] = kmin; red[32 + warp] = kmax; }
   __syncthreads();
-  unsigned long long* to_sort = all_keys;
-  uint32_t n_keep = c;
-  if (c > (uint32_t)K) {
-    // Composite keys are distinct, so the K-th largest is well defined: six radix levels over
-    // the 64 bits (value key first, then the index part that breaks ties towards low indices).
-    uint32_t k = (uint32_t)K;
-    unsigned long long prefix = 0ull;
-    const int shifts[6] = {52, 40, 32, 20, 8, 0};
-    const int bits[6] = {12, 12, 8, 12, 12, 8};
-#pragma unroll 1
-    for (int level = 0; level < 6; ++level) {
-      const int nb = 1 << bits[level];
-      for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
-      __syncthreads();
-      const int hi_shift = shifts[level] + bits[level];
+  kmin = red[lane];
+  kmax = red[32 + lane];
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(kFullMask, kmin, d));
+    kmax = max(kmax, __shfl_xor_sync(kFullMask, kmax, d));
+  }
+  // Fast path: a counting sort.  The value keys are spread over up to 4096 buckets by a monotone map
+  // (equal-width ranges of the key between the smallest and largest collected key), a scan from the top
+  // gives every bucket its first rank, the buckets that start below rank K are scattered to their rank
+  // ranges, and a key's rank is its bucket's first rank plus the keys of the same bucket that beat it
+  // under the total order.  Buckets hold a handful of keys unless the keys are clustered or tied in
+  // thousands; then the radix selection and bitonic sort below do the job.
+  bool fast = (c != 0);
+  if (fast) {
+    const uint32_t span = kmax - kmin;
+    const int sh = max(0, 20 - __clz(span));                // span >> sh < 4096
+    for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads)
+      atomicAdd(&hist[((uint32_t)(all_keys[i] >> 32) - kmin) >> sh], 1u);
+    __syncthreads();
+    uint32_t c4[4];
+    uint32_t mine = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      c4[j] = hist[4095 - (4 * (int)threadIdx.x + j)];
+      mine += c4[j];
+    }
+    uint32_t total;
+    uint32_t above = block_excl_scan(mine, scratch, &total);
+    bool big = false;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int bin = 4095 - (4 * (int)threadIdx.x + j);
+      offs[bin] = above;
+      if (above < n_out) {
+        if (c4[j] > (uint32_t)kBucketMax) big = true;
+        if (n_out <= above + c4[j]) result[0] = above + c4[j];   // keys in the buckets that start below rank K
+      }
+      above += c4[j];
+    }
+    fast = (__syncthreads_or(big ? 1 : 0) == 0);
+    if (fast) {
       for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads) {
         const unsigned long long u = all_keys[i];
-        const bool match = (level == 0) || ((u >> hi_shift) == prefix);
-        if (match) atomicAdd(&hist[(uint32_t)(u >> shifts[level]) & (nb - 1)], 1u);
+        const uint32_t bk = ((uint32_t)(u >> 32) - kmin) >> sh;
+        const uint32_t first = offs[bk];
+        if (first < n_out) top_keys[first + atomicSub(&hist[bk], 1u) - 1u] = u;
       }
       __syncthreads();
-      const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
-      prefix = (prefix << bits[level]) | (unsigned long long)d;
+      const uint32_t n_placed = result[0];
+      for (uint32_t p = threadIdx.x; p < n_placed; p += kTopkThreads) {
+        const unsigned long long u = top_keys[p];
+        const uint32_t key = (uint32_t)(u >> 32);
+        const uint32_t bk = (key - kmin) >> sh;
+        const uint32_t first = offs[bk];
+        const uint32_t last = (bk != 0) ? offs[bk - 1] : c;   // the next lower bucket starts where this one ends
+        uint32_t rank = first;
+        for (uint32_t q = first; q < last; ++q) rank += (top_keys[q] > u) ? 1u : 0u;
+        if (rank < n_out) {
+          uint32_t idx = 0xffffffffu - (uint32_t)(u & 0xffffffffull);
+          if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
+          const int64_t o = (int64_t)b * K_out + rank;
+          // the key maps back to the candidate's own bits, except that it does not tell -0 from +0
+          out_score[o] = (key == 0x80000000u) ? src.load1(b, idx)
+                                              : __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+          if (out_flat) out_flat[o] = (int32_t)idx;
+          if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
+          if (out_token) out_token[o] = (int32_t)(idx % (uint32_t)V);
+        }
+      }
+    } else {
+      for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
     }
-    const unsigned long long kth = prefix;                  // exactly K keys are >= kth
-    uint32_t done = 0;
-    for (uint32_t base = 0; base < c; base += kTopkThreads) {
-      const uint32_t i = base + threadIdx.x;
-      const unsigned long long u = (i < c) ? all_keys[i] : 0ull;
-      const bool win = (i < c) && (u >= kth);
-      uint32_t total;
-      const uint32_t pos = block_excl_scan(win ? 1u : 0u, scratch, &total) + done;
-      if (win) top_keys[pos] = u;
-      done += total;
+  }
+  __syncthreads();
+  if (!fast && c != 0) {
+    unsigned long long* to_sort = all_keys;
+    uint32_t n_keep = c;
+    if (c > (uint32_t)K) {
+      // Composite keys are distinct, so the K-th largest is well defined: six radix levels over
+      // the 64 bits (value key first, then the index part that breaks ties towards low indices).
+      uint32_t k = (uint32_t)K;
+      unsigned long long prefix = 0ull;
+      const int shifts[6] = {52, 40, 32, 20, 8, 0};
+      const int bits[6] = {12, 12, 8, 12, 12, 8};
+  #pragma unroll 1
+      for (int level = 0; level < 6; ++level) {
+        const int nb = 1 << bits[level];
+        for (int i = threadIdx.x; i < 4096; i += kTopkThreads) hist[i] = 0;
+        __syncthreads();
+        const int hi_shift = shifts[level] + bits[level];
+        for (uint32_t i = threadIdx.x; i < c; i += kTopkThreads) {
+          const unsigned long long u = all_keys[i];
+          const bool match = (level == 0) || ((u >> hi_shift) == prefix);
+          if (match) atomicAdd(&hist[(uint32_t)(u >> shifts[level]) & (nb - 1)], 1u);
+        }
+        __syncthreads();
+        const uint32_t d = pick_digit(hist, nb, &k, scratch, result);
+        prefix = (prefix << bits[level]) | (unsigned long long)d;
+      }
+      const unsigned long long kth = prefix;                  // exactly K keys are >= kth
+      uint32_t done = 0;
+      for (uint32_t base = 0; base < c; base += kTopkThreads) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long u = (i < c) ? all_keys[i] : 0ull;
+        const bool win = (i < c) && (u >= kth);
+        uint32_t total;
+        const uint32_t pos = block_excl_scan(win ? 1u : 0u, scratch, &total) + done;
+        if (win) top_keys[pos] = u;
+        done += total;
+      }
+      to_sort = top_keys;
+      n_keep = (uint32_t)K;
     }
-    to_sort = top_keys;
-    n_keep = (uint32_t)K;
-  }
-  uint32_t n_sort = 1024;
-  while (n_sort < n_keep) n_sort <<= 1;
-  __syncthreads();
-  for (uint32_t i = n_keep + threadIdx.x; i < n_sort; i += kTopkThreads) to_sort[i] = 0ull;
-  __syncthreads();
-  switch (n_sort) {
-    case 1024: block_bitonic_sort_desc<1>(to_sort); break;
-    case 2048: block_bitonic_sort_desc<2>(to_sort); break;
-    case 4096: block_bitonic_sort_desc<4>(to_sort); break;
-    default: block_bitonic_sort_desc<8>(to_sort); break;
-  }
-  sort_keys = to_sort;
-  const int64_t N = src.N;
-  const uint32_t n_out = min(c, (uint32_t)K);
-  for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
-    uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
-    if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
-    const int64_t o = (int64_t)b * K_out + i;
-    out_score[o] = src.load1(b, idx);
-    if (out_flat) out_flat[o] = (int32_t)idx;
-    if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
-    if (out_token) out_token[o] = (int32_t)(idx % (uint32_t)V);
+    uint32_t n_sort = 1024;
+    while (n_sort < n_keep) n_sort <<= 1;
+    __syncthreads();
+    for (uint32_t i = n_keep + threadIdx.x; i < n_sort; i += kTopkThreads) to_sort[i] = 0ull;
+    __syncthreads();
+    switch (n_sort) {
+      case 1024: block_bitonic_sort_desc<1>(to_sort); break;
+      case 2048: block_bitonic_sort_desc<2>(to_sort); break;
+      case 4096: block_bitonic_sort_desc<4>(to_sort); break;
+      default: block_bitonic_sort_desc<8>(to_sort); break;
+    }
+    sort_keys = to_sort;
+    for (uint32_t i = threadIdx.x; i < n_out; i += kTopkThreads) {
+      uint32_t idx = 0xffffffffu - (uint32_t)(sort_keys[i] & 0xffffffffull);
+      if ((int64_t)idx >= N) { flag_status(d_status, GRACE_DEV_BAD_INDEX); idx = 0; }    // cannot happen; never fault
+      const int64_t o = (int64_t)b * K_out + i;
+      out_score[o] = src.load1(b, idx);
+      if (out_flat) out_flat[o] = (int32_t)idx;
+      if (out_parent) out_parent[o] = (int32_t)(idx / (uint32_t)V);
+      if (out_token) out_token[o] = (int32_t)(idx % (uint32_t)V);
+    }
   }
   if (c < (uint32_t)K) {
     // Threshold was -inf and the row has fewer than K candidates above it: the rest of the beam
@@ -702,7 +800,7 @@ grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, floa
   if ((int64_t)K > N) K = (int)N;                            // every candidate is selected, the rest is padding
   const uint32_t rank = sample_rank(N, K);
   static unsigned long long attrs_set_devices = 0;
-  const size_t final_smem = (size_t)(kCap + kMaxK) * sizeof(unsigned long long) + 4096 * sizeof(uint32_t);
+  const size_t final_smem = (size_t)(kCap + kMaxK + kBucketMax) * sizeof(unsigned long long) + 2 * 4096 * sizeof(uint32_t);
   static int collect_grid_of[kMaxDevices] = {0};
   DeviceSetup su(&attrs_set_devices);
   if (su) {
