@@ -149,28 +149,31 @@ topk_sample_kernel(const CandSrc src, uint32_t rank, TopkHeader* hdr) {
   __shared__ uint32_t red[64];
   const int b = blockIdx.x;
   const int64_t N = src.N;
-  const int64_t stratum = (N / kSamplePoints) & ~(int64_t)7;       // multiple of 8 elements
-  const uint32_t slots = (uint32_t)(stratum >> 3);
+  const uint32_t stratum = (uint32_t)(N / kSamplePoints) & ~7u;     // multiple of 8 elements (N < 2^31)
+  const uint32_t slots = stratum >> 3;
   float4 v[2 * (kSamplePoints / kTopkThreads)];
 #pragma unroll
   for (int q = 0; q < kSamplePoints / kTopkThreads; ++q) {
-    const int p = q * kTopkThreads + threadIdx.x;
-    const uint32_t h = (uint32_t)(mix64((uint64_t)p * 0x10001ull + (uint64_t)b) >> 33);
-    const int64_t at = (int64_t)p * stratum + (int64_t)(h % slots) * 8;
-    v[2 * q] = src.load4(b, at >> 2, false);
-    v[2 * q + 1] = src.load4(b, (at >> 2) + 1, false);
+    const uint32_t p = q * kTopkThreads + threadIdx.x;
+    uint32_t h = p * 0x9e3779b1u + (uint32_t)b * 0x85ebca77u;      // where in its stratum point p of request b lies
+    h ^= h >> 16; h *= 0x85ebca6bu; h ^= h >> 13; h *= 0xc2b2ae35u; h ^= h >> 16;
+    const uint32_t at4 = (p * stratum + __umulhi(h, slots) * 8u) >> 2;
+    v[2 * q] = src.load4(b, at4, false);
+    v[2 * q + 1] = src.load4(b, at4 + 1, false);
   }
-  uint32_t top1 = 0, top2 = 0;
+  // the two largest of the thread's 32 values, on the floats themselves (a NaN never wins a maximum, so it
+  // cannot become the threshold; the collecting pass reports it)
+  float m1 = __int_as_float(0xff800000), m2 = m1;
 #pragma unroll
   for (int q = 0; q < 2 * (kSamplePoints / kTopkThreads); ++q) {
     const float x[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const uint32_t u = ordered_key(x[j]);
-      if (u > top1) { top2 = top1; top1 = u; }
-      else if (u > top2) top2 = u;
+      m2 = fmaxf(m2, fminf(m1, x[j]));
+      m1 = fmaxf(m1, x[j]);
     }
   }
+  const uint32_t top1 = ordered_key(m1), top2 = ordered_key(m2);
   // The threshold need not be the r-th largest key itself: any value at or below it with few keys in
   // between will do.  So instead of a full radix selection, histogram the keys over 4096 equal ranges
   // between the smallest and the largest, take the lower edge of the range that holds rank r, and look
@@ -271,8 +274,6 @@ __device__ __forceinline__ bool collect_hits(const float4 v, bool mine, uint32_t
 
 __global__ void __launch_bounds__(kCollectThreads, 5)
 topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d_status) {
-  pdl_wait();
-  pdl_trigger();
   // grid (x, B): the CTAs of column b split request b's candidates into contiguous, equal chunks of whole
   // 256-float4 rows.  Hits are a fraction of a percent; each warp stages its own in shared memory (a
   // shared-memory atomic per hit, no scan) and appends them to the request's list with ONE global atomic
@@ -294,18 +295,38 @@ topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d
   uint32_t r = blockIdx.x * rows_per_cta;
   const uint32_t r_end = min(rows_total, r + rows_per_cta);
   const uint32_t r_full = min(r_end, n4 / kCollectThreads);      // rows below this one are wholly in bounds
+  const float ninf = __int_as_float(0xff800000);
+  // This kernel is scheduled while the sampling kernel still runs, and only the threshold depends on that
+  // kernel: the candidates were complete before it started (it waits for its own predecessors before it
+  // lets this kernel be scheduled).  So the first tile of the chunk is requested now, past the L1 (which
+  // may hold lines of an earlier call's candidates), and the memory system works under the sampling
+  // kernel instead of idling.  (Fetching further rows into shared memory at this point was measured
+  // slower: the shared-memory carve-out it needs shrinks the L1 the streaming loads pass through.)
+  const uint32_t i_first = r * kCollectThreads + threadIdx.x;
+  float4 v[kCollectUnroll];
+#pragma unroll
+  for (int u = 0; u < kCollectUnroll; ++u)
+    v[u] = (r + u < r_full) ? __ldcg(row + i_first + u * kCollectThreads) : make_float4(ninf, ninf, ninf, ninf);
+  pdl_wait();
+  pdl_trigger();
   const uint32_t t_excl = __ldcg(&hdr[b].t_excl);
   // the same threshold as a float: key(x) > t_excl  <=>  x > thr for every non-NaN x
   const float thr = __uint_as_float((t_excl & 0x80000000u) ? (t_excl ^ 0x80000000u) : ~t_excl);
   bool saw_nan = false, dead = false;
+#pragma unroll
+  for (int u = 0; u < kCollectUnroll; ++u) {
+    // !(x <= thr): above the threshold, or NaN
+    const bool mine = !(v[u].x <= thr) || !(v[u].y <= thr) || !(v[u].z <= thr) || !(v[u].w <= thr);
+    if (__any_sync(kFullMask, mine))
+      dead |= collect_hits(v[u], mine, i_first + u * kCollectThreads, thr, wstage, wcount, list_count, list, &saw_nan);
+  }
+  if (r < r_full) r = min(r + kCollectUnroll, r_full);
   for (; r + kCollectUnroll <= r_full && !dead; r += kCollectUnroll) {
     const uint32_t i0 = r * kCollectThreads + threadIdx.x;
-    float4 v[kCollectUnroll];
 #pragma unroll
     for (int u = 0; u < kCollectUnroll; ++u) v[u] = __ldcs(row + i0 + u * kCollectThreads);
 #pragma unroll
     for (int u = 0; u < kCollectUnroll; ++u) {
-      // !(x <= thr): above the threshold, or NaN
       const bool mine = !(v[u].x <= thr) || !(v[u].y <= thr) || !(v[u].z <= thr) || !(v[u].w <= thr);
       if (__any_sync(kFullMask, mine))
         dead |= collect_hits(v[u], mine, i0 + u * kCollectThreads, thr, wstage, wcount, list_count, list, &saw_nan);
@@ -313,11 +334,10 @@ topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d
   }
   for (; r < r_end && !dead; ++r) {
     const uint32_t i = r * kCollectThreads + threadIdx.x;
-    const float ninf = __int_as_float(0xff800000);
-    const float4 v = (i < n4) ? __ldcs(row + i) : make_float4(ninf, ninf, ninf, ninf);
-    const bool mine = !(v.x <= thr) || !(v.y <= thr) || !(v.z <= thr) || !(v.w <= thr);
+    const float4 x = (i < n4) ? __ldcs(row + i) : make_float4(ninf, ninf, ninf, ninf);
+    const bool mine = !(x.x <= thr) || !(x.y <= thr) || !(x.z <= thr) || !(x.w <= thr);
     if (__any_sync(kFullMask, mine))
-      dead |= collect_hits(v, mine, i, thr, wstage, wcount, list_count, list, &saw_nan);
+      dead |= collect_hits(x, mine, i, thr, wstage, wcount, list_count, list, &saw_nan);
   }
   warp_flush(wstage, wcount, list_count, list);
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);

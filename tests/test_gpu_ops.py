@@ -386,6 +386,29 @@ def test_topk_adversarial_inputs_take_the_exact_path_and_stay_exact(api):
     _check_topk(api, -ramp, K, V)
 
 
+def test_topk_outliers_clusters_and_tie_groups_on_the_sampled_path(api):
+    """Inputs that stress the range histograms of the sampled path: an outlier that stretches the key range of
+    the sample (the threshold search has to look closer), tie groups of tens of candidates around the K-th
+    value (ranked by index inside a bucket of the counting sort), values clustered on both sides of zero."""
+    B, M, V, K = 3, 300, 1024, 2048
+    rng = synth.rng_for(4, 302)
+    cand = (synth.normal_f32(rng, (B, M * V), 3.0) - 8.0).astype(np.float32)
+    wild = cand.copy()
+    wild[0, 12345] = 1e30
+    wild[1, 777] = np.inf
+    wild[2, 5] = 3e38
+    wild[2, 4096] = 1e-30
+    _check_topk(api, wild, K, V, expect_exact_path=False)
+    stepped = (np.round(cand * 64.0) / 64.0).astype(np.float32)
+    _check_topk(api, stepped, K, V, expect_exact_path=False)
+    _check_topk(api, stepped, 100, V)
+    near_zero = (synth.normal_f32(rng, (B, M * V), 1.0) * np.float32(1e-3)).astype(np.float32)
+    _check_topk(api, near_zero, K, V)
+    near_zero[:, ::3] = 0.0
+    near_zero[:, 1::3] = -0.0
+    _check_topk(api, near_zero, K, V)
+
+
 def test_topk_flags_nan(api):
     cand = synth.normal_f32(synth.rng_for(4, 301), (1, 4096))
     cand[0, 77] = np.nan
