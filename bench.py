@@ -265,6 +265,11 @@ def op_breakdown(dec, cfg, reps=3):
         """LayerNorm + the GEMM behind it, as the decode path runs them (two kernels, or folded)."""
         if folded:
             wf, cs, cb = fold
+            if dec.centre_stream and x.shape[0] >= 1024 and 256 <= wf.shape[0] <= 512:
+                # what the decode step launches here: one kernel, statistics from the GEMM's own operand tiles
+                timed("linear", lambda: api.grace_linear_layer_norm(x, wf, 1e-5, dec.row_affine[:x.shape[0]],
+                                                                    None, cb, y, relu, lse_part), fl)
+                return
             timed("row_stats", lambda: api.grace_row_stats_bf16(x, dec.row_affine[:x.shape[0]]))
             timed("linear", lambda: api.grace_linear_folded_ln(x, wf, dec.row_affine[:x.shape[0]],
                                                                None if dec.centre_stream else cs, cb, y, relu, lse_part), fl)

@@ -458,6 +458,18 @@ grace_status_t grace_linear_folded_ln(const uint16_t* x, int64_t ldx, const uint
                                       uint16_t* y_bf16, float* y_f32, int64_t ldy, float* lse_part,
                                       int M, int N, int K, int relu, void* stream);
 
+/* grace_row_stats_bf16 (over D = K, with eps) followed by grace_linear_folded_ln, as one call: the LayerNorm over
+ * the rows of x [M][K] (ldx == K) and the GEMM behind it.  For M >= 1024 and 256 <= N <= 512 with centred rows
+ * (col_sum NULL) it is ONE kernel: the row statistics are formed from the GEMM's own operand tiles in shared
+ * memory while the tensor cores work on them, so the residual stream is not read a second time; row_affine
+ * (device, fp32 [M][2], 8-byte aligned) is then not touched.  Otherwise (wider outputs, where forming the
+ * statistics once per 256-column tile costs more than reading the stream once) the statistics kernel runs
+ * first, into row_affine.  Other arguments and errors as grace_linear_folded_ln. */
+grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw, float eps,
+                                       float* row_affine, const float* col_sum, const float* col_bias,
+                                       uint16_t* y_bf16, float* y_f32, int64_t ldy, float* lse_part,
+                                       int M, int N, int K, int relu, void* stream);
+
 /* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
 grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
                                 uint16_t* out, int R, int D, float eps, void* stream);

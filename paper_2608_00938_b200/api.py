@@ -120,6 +120,8 @@ _gtm_mask_logits_parts = _sig("grace_gtm_mask_logits_parts", _i32,
 _row_stats_bf16 = _sig("grace_row_stats_bf16", _i32, [_vp, _i32, _i32, _f32, _vp, _vp])
 _linear_folded_ln = _sig("grace_linear_folded_ln", _i32, [_vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
                                                          _i32, _i32, _i32, _i32, _vp])
+_linear_layer_norm = _sig("grace_linear_layer_norm", _i32, [_vp, _i64, _vp, _i64, _f32, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
+                                                           _i32, _i32, _i32, _i32, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
 _stream_l2_persist = _sig("grace_stream_l2_persist", _i32, [_vp, _vp, C.c_size_t, C.c_float])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
@@ -391,6 +393,21 @@ def grace_linear_folded_ln(x, w_folded, row_affine, col_sum, col_bias, y, relu: 
     _check(_linear_folded_ln(x.data_ptr(), x.stride(0), w_folded.data_ptr(), w_folded.stride(0), _dp(row_affine),
                              _dp(col_sum), _dp(col_bias), None if f32 else _dp(y), _dp(y) if f32 else None, y.stride(0),
                              _dp(lse_part), M, N, K, int(relu), _stream()), "grace_linear_folded_ln")
+    return y
+
+
+def grace_linear_layer_norm(x, w_folded, eps: float, row_affine, col_sum, col_bias, y, relu: bool = False, lse_part=None):
+    """LayerNorm over the rows of x (statistics with eps) and the GEMM behind it in one call: the result of
+    grace_row_stats_bf16 + grace_linear_folded_ln.  row_affine: fp32 [M, 2] scratch (used only when the
+    statistics cannot be formed inside the GEMM kernel)."""
+    import torch
+    M, K = x.shape
+    N = w_folded.shape[0]
+    f32 = y.dtype == torch.float32
+    _check(_linear_layer_norm(x.data_ptr(), x.stride(0), w_folded.data_ptr(), w_folded.stride(0), float(eps),
+                              _dp(row_affine), _dp(col_sum), _dp(col_bias), None if f32 else _dp(y),
+                              _dp(y) if f32 else None, y.stride(0), _dp(lse_part), M, N, K, int(relu), _stream()),
+           "grace_linear_layer_norm")
     return y
 
 

@@ -88,12 +88,9 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   const bool folded = xb && d->row_affine != nullptr;
   auto ln_linear = [&](const float* g, const float* b, const uint16_t* w, const float* cs, const float* cb,
                        uint16_t* y_bf16, float* y_f32, int64_t ldy, int N, int relu, float* lse_part) -> grace_status_t {
-    if (folded) {
-      grace_status_t s1 = grace_row_stats_bf16(d->x_bf16, R, D, d->ln_eps, d->row_affine, stream);
-      if (s1 != GRACE_OK) return s1;
-      return grace_linear_folded_ln(d->x_bf16, D, w, D, d->row_affine, cs, cb, y_bf16, y_f32, ldy, lse_part, R, N, D, relu,
-                                    stream);
-    }
+    if (folded)
+      return grace_linear_layer_norm(d->x_bf16, D, w, D, d->ln_eps, d->row_affine, cs, cb, y_bf16, y_f32, ldy, lse_part, R,
+                                     N, D, relu, stream);
     grace_status_t s1 = layer_norm(g, b);
     if (s1 != GRACE_OK) return s1;
     if (lse_part != nullptr) return grace_linear_f32_lse(d->h, D, w, D, y_f32, ldy, lse_part, R, N, D, stream);

@@ -232,12 +232,19 @@ constexpr int kQAffBytes = 256 * 2 * 4;                   // the tile's 256 (col
 // checks it (six stages, the staging buffers and the column vectors leave less than 1 KB of the 227 KB)
 constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 256 + kQAffBytes;
 
-template <int OUT>
-__global__ void __launch_bounds__(192, 1)
+// STATS: the rows' LayerNorm statistics are not read from memory (aff_row is only a non-null marker then) but
+// formed inside the kernel: four more warps per CTA read every A tile out of the ring while the tensor cores
+// work on it (a row per thread, its sum and sum of squares over the whole K = the LayerNorm width), and hand
+// (rstd, -rstd * mean) of the CTA's 128 rows to the epilogue through 1 KB of shared memory.  A stage is
+// released by the MMAs' commit AND by these warps; the odd CTA, whose tiles are counted on the even CTA's
+// barrier, learns that a stage has landed from an arrive the even CTA forwards.  Centred rows only (aff_cs ==
+// nullptr): the second half of the column-vector buffer is what holds the statistics.
+template <int OUT, bool STATS>
+__global__ void __launch_bounds__(STATS ? 320 : 192, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part,
                    const float2* __restrict__ aff_row, const float* __restrict__ aff_cs,
-                   const float* __restrict__ aff_cb) {
+                   const float* __restrict__ aff_cb, float ln_eps) {
   extern __shared__ __align__(1024) uint8_t smem_pair[];
   uint8_t* tiles = smem_pair;
   if ((tc::smem_addr(tiles) & 1023u) != 0) {               // the swizzled tiles need it; same answer in every thread
@@ -251,7 +258,11 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   uint64_t* acc_empty = acc_full + 2;          // [2] even CTA only: 4 local + 4 remote epilogue warps
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* a_ready = acc_empty + 3;           // [kQStages] STATS, odd CTA: the stage has landed (forwarded by the even CTA)
+  uint64_t* stats_full = a_ready + kQStages;   // [1] STATS: the tile's row statistics are in shared memory
+  uint64_t* stats_empty = stats_full + 1;      // [1] STATS: the epilogue has taken them
   float4* aff_s = reinterpret_cast<float4*>(staging + 2 * kPStagingBytes + 256);   // [128]: (cs, cs, cb, cb) of 2 columns
+  float2* stats_s = reinterpret_cast<float2*>(staging + 2 * kPStagingBytes + 256 + kQAffBytes / 2);   // [128] STATS
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = tc::cluster_cta_rank();            // 0: issues the MMAs; 1: peer
@@ -261,8 +272,13 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
   const int total = n_tiles * m_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kQStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, 1); }
+    for (int s = 0; s < kQStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, STATS ? 5 : 1); }
     for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 8); }
+    if (STATS) {
+      for (int s = 0; s < kQStages; ++s) tc::mbar_init(a_ready + s, 1);
+      tc::mbar_init(stats_full, 4);
+      tc::mbar_init(stats_empty, 4);
+    }
     *abort_flag = 0;
     tc::fence_mbar_init();
     tc::tma_prefetch_desc(&map_x); tc::tma_prefetch_desc(&map_w); tc::tma_prefetch_desc(&map_y);
@@ -319,6 +335,51 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         tc::mma_commit_pair(acc_full + ab, 3);
       }
     }
+  } else if (STATS && warp >= 6) {
+    // ---- statistics warps 6..9 of both CTAs: row (warp - 6) * 32 + lane of this CTA's 128 ----
+    const int row = (warp - 6) * 32 + lane;
+    const float inv_k = 1.f / (float)K;
+    int it = 0, local = 0;
+    bool ok = true;
+    for (int tile = pair; tile < total && ok; tile += n_pairs, ++local) {
+      f32x2_t acc = f2_pack(0.f, 0.f), sq = f2_pack(0.f, 0.f);
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % kQStages;
+        const uint32_t ph = (it / kQStages) & 1;
+        if (rank == 0) {
+          ok = tc::mbar_wait_cluster(full + s, ph, abort_flag);
+          if (ok && warp == 6 && lane == 0) tc::mbar_arrive_remote(a_ready + s, 1);
+        } else {
+          ok = tc::mbar_wait_cluster(a_ready + s, ph, abort_flag);
+        }
+        ok = __all_sync(kFullMask, ok);
+        if (!ok) break;
+        // 128 bytes of the row, in the order that keeps eight neighbouring rows on different banks
+        const uint4* a_row = reinterpret_cast<const uint4*>(tiles + s * kQStageBytes + row * 128);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint4 t = a_row[j ^ (row & 7)];
+          const f32x2_t a = f2_from_bf16x2(t.x), b = f2_from_bf16x2(t.y), c = f2_from_bf16x2(t.z), d = f2_from_bf16x2(t.w);
+          acc = f2_add(acc, f2_add(f2_add(a, b), f2_add(c, d)));
+          sq = f2_fma(a, a, sq); sq = f2_fma(b, b, sq); sq = f2_fma(c, c, sq); sq = f2_fma(d, d, sq);
+        }
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(empty + s);
+      }
+      if (!ok) break;
+      float lo, hi, qlo, qhi;
+      f2_unpack(acc, lo, hi);
+      f2_unpack(sq, qlo, qhi);
+      const float mean = (lo + hi) * inv_k;
+      const float var = fmaxf((qlo + qhi) * inv_k - mean * mean, 0.f);
+      const float rstd = rsqrtf(var + ln_eps);
+      ok = tc::mbar_wait_cluster(stats_empty, (local & 1) ^ 1, abort_flag);   // the previous tile's were taken
+      ok = __all_sync(kFullMask, ok);
+      if (!ok) break;
+      stats_s[row] = make_float2(rstd, -rstd * mean);
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(stats_full);
+    }
   } else {
     // ---- epilogue warps 2..5 of both CTAs: TMEM lane quarter q = rows q*32 + lane of this CTA's 128 ----
     const int q = warp & 3;
@@ -338,7 +399,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       tile = min(tile, total - 1);
       const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
       const int col = min(n0 + 2 * row, N - 2);
-      ar_next = __ldg(aff_row + min(m0 + row, M - 1));
+      if (!STATS) ar_next = __ldg(aff_row + min(m0 + row, M - 1));
       cb_next = __ldg(reinterpret_cast<const float2*>(aff_cb + col));
       cs_next = __ldg(reinterpret_cast<const float2*>(cs_or_cb + col));
     };
@@ -346,13 +407,21 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     for (int tile = pair; tile < total; tile += n_pairs, ++local) {
       const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
       const int ab = local & 1;
-      const float2 ar = ar_next;                           // rows and columns past the edge: values never stored
+      float2 ar = ar_next;                                 // rows and columns past the edge: values never stored
       const float4 cv = aff_cs != nullptr ? make_float4(cs_next.x, cs_next.y, cb_next.x, cb_next.y)
                                           : make_float4(cb_next.x, cb_next.y, 0.f, 0.f);
       bool ok = tc::mbar_wait_cluster(acc_full + ab, (local >> 1) & 1, abort_flag);
       ok = __all_sync(kFullMask, ok);
       if (!ok) break;
       tc::tc_fence_after();
+      if (STATS) {
+        ok = tc::mbar_wait_cluster(stats_full, local & 1, abort_flag);
+        ok = __all_sync(kFullMask, ok);
+        if (!ok) break;
+        ar = stats_s[row];
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(stats_empty);
+      }
       const uint32_t t_acc = tmem_base + (uint32_t)(ab * 256) + ((uint32_t)(q * 32) << 16);
       float lse_m = -INFINITY, lse_s = 0.f;                // kOutF32Lse: running maximum and sum of 2^((v - max) log2 e)
       // read after the first chunk's barrier; the previous tile's readers are past its last barrier.
@@ -487,9 +556,11 @@ struct Affine {                                            // LayerNorm folded i
   const float2* row;
   const float* cs;
   const float* cb;
+  float eps = 0.f;                                         // in_kernel_stats only
+  bool in_kernel_stats = false;                            // the pair kernel forms (rstd, -rstd * mean) itself
 };
 
-template <int OUT>
+template <int OUT, bool STATS = false>
 static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
                                   int K, int relu, cudaStream_t s, float2* lse_part = nullptr,
                                   Affine aff = Affine{nullptr, nullptr, nullptr}) {
@@ -501,14 +572,14 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.blockDim = dim3(192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
+  cfg.blockDim = dim3(STATS ? 320 : 192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   DeviceSetup su(&attr_set_devices);
   if (su) {
-    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
+    GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
     int n_sm = 0, clusters = 0;
     GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, su.dev));
     cfg.gridDim = dim3(n_sm & ~1);
-    GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, linear_pair_kernel<OUT>, &cfg));
+    GRACE_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, linear_pair_kernel<OUT, STATS>, &cfg));
     if (clusters <= 0) return GRACE_CUDA_ERROR;
     if (clusters > n_sm / 2) clusters = n_sm / 2;
     max_clusters_of[su.dev] = clusters;
@@ -517,7 +588,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   const int max_clusters = max_clusters_of[su.dev];
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
-  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb));
+  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT, STATS>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb, aff.eps));
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -569,6 +640,12 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
         !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
       return GRACE_CUDA_ERROR;
     if (aff.row != nullptr && (add_into_bf16 || aliased)) return GRACE_INVALID_ARG;
+    if (aff.in_kernel_stats) {
+      if (f32) return lse_part != nullptr
+                          ? launch_pair<kOutF32Lse, true>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part), aff)
+                          : launch_pair<kOutF32, true>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
+      return launch_pair<kOutBf16, true>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
+    }
     if (!f32) return add_into_bf16 ? launch_pair<kOutBf16Add>(mx, mw, my, M, N, K, relu, s)
                                    : launch_pair<kOutBf16>(mx, mw, my, M, N, K, relu, s, nullptr, aff);
     if (lse_part != nullptr)
@@ -620,6 +697,33 @@ extern "C" grace_status_t grace_linear_folded_ln(const uint16_t* x, int64_t ldx,
     return GRACE_INVALID_ARG;
   if (lse_part != nullptr && (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
   grace::Affine aff = {reinterpret_cast<const float2*>(row_affine), col_sum, col_bias};
+  return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, nullptr, false, M, N, K, relu, stream, lse_part, aff);
+}
+
+extern "C" grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                                  float eps, float* row_affine, const float* col_sum,
+                                                  const float* col_bias, uint16_t* y_bf16, float* y_f32, int64_t ldy,
+                                                  float* lse_part, int M, int N, int K, int relu, void* stream) {
+  if (!row_affine || !col_bias || (reinterpret_cast<uintptr_t>(row_affine) & 7) ||
+      !grace_aligned16(col_sum) || !grace_aligned16(col_bias))
+    return GRACE_INVALID_ARG;
+  if (lse_part != nullptr && (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || ldx != K) return GRACE_INVALID_ARG;     // the LayerNorm is over the whole row of x
+  grace::Affine aff = {reinterpret_cast<const float2*>(row_affine), col_sum, col_bias};
+  // The statistics come out of the GEMM's own operand tiles where the CTA-pair kernel runs, the rows are centred
+  // (no col_sum) and the output is at most two tiles wide; otherwise the statistics kernel runs first, into
+  // row_affine.  Every n-tile forms the statistics of its rows again, and the shared-memory reads that takes
+  // (16 KB per k-block on top of the 32 KB the tensor cores read and the 32 KB TMA writes) slow the main loop by a
+  // fifth: measured at 65536 x 512 -> N, one kernel against two: N = 512: 36 us against 43; N = 1536: 99 against
+  // 95; N = 2048: 130 against 122.
+  const bool pair_kernel = (M >= 1024 && N >= 256);
+  if (pair_kernel && col_sum == nullptr && N <= 512) {
+    aff.eps = eps;
+    aff.in_kernel_stats = true;
+  } else {
+    const grace_status_t st = grace_row_stats_bf16(x, M, K, eps, row_affine, stream);
+    if (st != GRACE_OK) return st;
+  }
   return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, nullptr, false, M, N, K, relu, stream, lse_part, aff);
 }
 

@@ -830,7 +830,9 @@ def test_mask_kernel_merges_log_sum_exp_partials(api, kind, M):
                                                (2100, 1536, 512, False, False), (1500, 2048, 512, True, False),
                                                (1100, 512, 512, False, True), (33000, 2048, 512, False, True),
                                                # ragged last column tile in the pair kernel (clamped vector fetches)
-                                               (1500, 784, 512, True, False), (1300, 336, 512, False, True)])
+                                               (1500, 784, 512, True, False), (1300, 336, 512, False, True),
+                                               # one-kernel form of grace_linear_layer_norm (centred, N <= 512), bf16 out
+                                               (33000, 512, 512, True, False), (2100, 384, 512, False, False)])
 @pytest.mark.parametrize("centred", [False, True])
 def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
     """grace_row_stats_bf16 + grace_linear_folded_ln against LayerNorm(x) @ w^T in fp64: the GEMM reads the raw
@@ -875,6 +877,24 @@ def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
         lse = p[:, :, 0].max(1) + np.log((p[:, :, 1] * np.exp(p[:, :, 0] - p[:, :, 0].max(1, keepdims=True))).sum(1))
         want = np.log(np.exp(got - got.max(1, keepdims=True)).sum(1)) + got.max(1)
         np.testing.assert_allclose(lse, want, atol=1e-5, rtol=0)
+    # the same as ONE call (for large centred problems one kernel: statistics from the GEMM's own operand tiles)
+    y1 = torch.zeros_like(y)
+    part1 = torch.zeros_like(part) if part is not None else None
+    scratch = torch.full((M, 2), 7.0, device=DEV)
+    api.grace_linear_layer_norm(dev_bf16(x), dev_bf16(wf_bits), 1e-5, scratch, None if centred else dev(cs), dev(cb), y1,
+                                relu, part1)
+    torch.cuda.synchronize()
+    got1 = y1.float().cpu().numpy().astype(np.float64)
+    assert np.abs(got1 - ref).max() <= tol * max(1.0, np.abs(ref).max()), np.abs(got1 - ref).max()
+    assert np.sqrt(((got1 - ref) ** 2).sum() / (ref ** 2).sum()) <= 5e-3
+    # against the two-kernel form: the statistics agree to rounding (2e-6), so the outputs do to that times |y|
+    # plus, for bf16 outputs, a rounding that may fall the other way
+    slack = 1e-5 * np.abs(got) + (0 if f32out else 2.0 ** -7 * np.abs(got)) + 1e-6
+    assert (np.abs(got1 - got) <= slack).all(), np.abs(got1 - got).max()
+    if part1 is not None:
+        np.testing.assert_allclose(part1.cpu().numpy(), part.cpu().numpy(), rtol=2e-5, atol=2e-5)
+    in_kernel = centred and M >= 1024 and 256 <= N <= 512
+    assert bool((scratch == 7.0).all().item()) == in_kernel       # the scratch is touched only by the two-kernel form
 
 
 def test_l2_residency_window_is_a_hint_only(api):
