@@ -401,6 +401,39 @@ def _time_op(fn, n_sets, iters=200, warm=20):
     return ts[len(ts) // 2] * 1e3, ts[min(len(ts) - 1, int(len(ts) * 0.99))] * 1e3    # P50, P99 in us
 
 
+def library_gemm_same_shape(device, cfg):
+    """Context for the GEMM roofline: the decoder's widest projection (rows x d_ffn x d_model) through
+    grace_linear and through torch.matmul (cuBLAS) on the same random operands, back to back in this process.
+    The measured peak the fraction is quoted against is a square 8192^3 product; this is the library on the
+    kernel's own shape."""
+    import torch
+    from paper_2608_00938_b200 import api
+    M, N, K = cfg["B"] * max(cfg["schedule"]), cfg["d_ffn"], cfg["d_model"]
+    g = torch.Generator(device=device); g.manual_seed(synth.seed_for(6))
+    x = torch.randn(M, K, device=device, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, device=device, generator=g) * 0.05).to(torch.bfloat16)
+    y = torch.empty(M, N, device=device, dtype=torch.bfloat16)
+
+    def timed(fn, n=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / n
+    us_lib = timed(lambda: torch.matmul(x, w.t(), out=y))
+    us_own = timed(lambda: api.grace_linear(x, w, y))
+    fl = 2.0 * M * N * K
+    return dict(shape=[M, N, K], library="torch.matmul (cuBLAS), bf16, random normal operands",
+                library_us=us_lib, library_tflops=fl / us_lib / 1e6, grace_linear_us=us_own,
+                grace_linear_tflops=fl / us_own / 1e6,
+                note="20 launches back to back each; all-zero operands run 12-25 % faster in both (the tensor pipe is at "
+                     "its power limit), so only same-data figures compare")
+
+
 def op_rooflines(device, peaks):
     import torch
     from paper_2608_00938_b200 import api
@@ -690,10 +723,10 @@ def main():
         line["op_breakdown"] = bd
         top = max(bd, key=lambda k: bd[k]["ms_per_loop"])
         # DRAM bytes per flop of the dominant kernels, from the committed ncu captures under profiles/
-        # (linear_pair_kernel 32768x2048x512: 111.2 MB for 68.7 GFLOP; cross_attn_tc_kernel B16 M2048 T1024:
-        # 73.8 MB for 68.7 GFLOP); the bench's launches are larger than a capture may be, so the traffic is scaled
+        # (linear_pair_kernel 32768x2048x512: 111.2 MB for 68.7 GFLOP; cross_attn_ms_kernel B16 M2048 T1024:
+        # 73.2 MB for 68.7 GFLOP); the bench's launches are larger than a capture may be, so the traffic is scaled
         # by the flops of an average launch (it grows in proportion: every tile streams its operands once).
-        dram_bytes_per_flop = {"linear": 111.23e6 / 68.72e9, "cross_attn": 73.85e6 / 68.72e9}
+        dram_bytes_per_flop = {"linear": 111.23e6 / 68.72e9, "cross_attn": 73.19e6 / 68.72e9}
         line["whole_loop_tflops"] = sum(v["flops_per_loop"] for v in bd.values()) / (ms_loop * 1e-3) / 1e12
         if top in ("linear", "cross_attn") and not default_workload:
             ach = bd[top]["flops_per_loop"] / (bd[top]["ms_per_loop"] * 1e-3) / 1e12
@@ -716,6 +749,8 @@ def main():
                                     us_per_launch=bd[top]["ms_per_loop"] * 1e3 / bd[top]["calls_per_loop"],
                                     peak_source=f"{peaks['source']} (sustained: kernel timed inside a long step)",
                                     launches_per_loop=bd[top]["calls_per_loop"])
+            if top == "linear" and world == 1:
+                line["roofline"]["library_same_shape"] = library_gemm_same_shape(device, cfg)
         else:
             line["roofline"] = dict(kernel=top, bound="hbm", achieved=None, peak=peaks["hbm_gbs"], unit="GB/s", frac=None,
                                     traffic=None, peak_source=peaks["source"])
