@@ -86,7 +86,7 @@ def make_inputs(cfg, variant=0):
 
 
 def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, fold_layer_norm=None,
-                  persist_stream_l2=None, kv_in_place=True):
+                  persist_stream_l2=None, kv_in_place=True, logits_allowed_only=True, masked_from_step=None):
     from paper_2608_00938_b200 import api
     from paper_2608_00938_b200.decoder import Decoder
     bits, base, level_start = api.grace_trie_build_dense(inp["sids"], cfg["V"])
@@ -99,7 +99,8 @@ def build_decoder(cfg, inp, device, residual_bf16=False, materialize_cand=None, 
                   trie_base=base, num_nodes=num_nodes,
                   matcher=(api.MATCH_PREFIX_BLOOM, blooms, cfg["bloom_log2"], cfg["bloom_hashes"]), device=device,
                   residual_bf16=residual_bf16, level_start=level_start, materialize_cand=materialize_cand,
-                  fold_layer_norm=fold_layer_norm, persist_stream_l2=persist_stream_l2, kv_in_place=kv_in_place)
+                  fold_layer_norm=fold_layer_norm, persist_stream_l2=persist_stream_l2, kv_in_place=kv_in_place,
+                  logits_allowed_only=logits_allowed_only, masked_from_step=masked_from_step)
     return dec
 
 
@@ -320,10 +321,33 @@ def op_breakdown(dec, cfg, reps=3):
             logp = dec.logp[:R]
             parts = dec.lse_part is not None and R >= 1024   # the logits GEMM also leaves the rows' log-sum-exp partials
             lsep = dec.lse_part[:R] if parts else None
-            ln_linear(x, dec.lnf_g, dec.lnf_b, hD, dec.w_out, (dec.w_out, dec.cs_out, dec.cb_out) if folded else None,
-                      logp, 2.0 * R * D * V, lse_part=lsep)
             par = dec.parents[t + 1]
             masked = dec.allow_bits is not None and t >= dec.masked_from_step
+            allowed_only = masked and parts and dec.logits_allowed_only
+            if allowed_only:
+                # the constraint first, a logits GEMM that stores the allowed logits only, the merge of its
+                # log-sum-exp partials, the selection through the allow bits
+                bits = dec.allow_bits[:R]
+                timed("gtm_mask", lambda: api.grace_gtm_allow_bits(dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
+                                                                   bits, B, M, t, dec.d_status))
+                if folded:                          # (the call runs the row-statistics kernel itself: 12 us of its time)
+                    timed("linear", lambda: api.grace_linear_logits_allowed(
+                        x, dec.w_out, bits, logp, lsep, 1e-5, dec.row_affine[:R],
+                        None if dec.centre_stream else dec.cs_out, dec.cb_out), 2.0 * R * D * V)
+                else:
+                    timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))
+                    timed("linear", lambda: api.grace_linear_logits_allowed(hD, dec.w_out, bits, logp, lsep), 2.0 * R * D * V)
+                timed("gtm_mask", lambda: api.grace_row_lse_from_parts(lsep, dec.node[cur][:R], dec.trie, dec.row_lse[:R]))
+                timed("beam_topk", lambda: api.grace_beam_topk_masked(
+                    logp, bits, dec.score[cur][:R], dec.row_lse[:R], B, M, K, dec.score[nxt][:B * K].view(B, K),
+                    dec.out_flat[:B * K].view(B, K), par[:B * K].view(B, K), dec.token[nxt][:B * K].view(B, K),
+                    dec.topk_ws, dec.d_status))
+                timed("beam_update", lambda: api.grace_beam_update(
+                    par[:B * K], dec.token[nxt][:B * K], dec.score[nxt][:B * K], dec.node[cur][:R], dec.key[cur][:R], dec.trie,
+                    dec.node[nxt][:B * K], dec.key[nxt][:B * K], B, K, M, t, dec.d_status))
+                continue
+            ln_linear(x, dec.lnf_g, dec.lnf_b, hD, dec.w_out, (dec.w_out, dec.cs_out, dec.cb_out) if folded else None,
+                      logp, 2.0 * R * D * V, lse_part=lsep)
             if masked:                                  # candidates never materialised: allow bits + masked top-k
                 bits = dec.allow_bits[:R]
                 if parts:
@@ -642,6 +666,11 @@ def main():
                     help="keep the residual stream resident in L2 (access-policy window on the stream)")
     ap.add_argument("--layer-norm", default="folded", choices=["folded", "kernel"],
                     help="LayerNorms folded into the GEMMs behind them (bf16 stream), or run as kernels of their own")
+    ap.add_argument("--logits", default="allowed", choices=["allowed", "dense"],
+                    help="on the allow-bits steps: constraint first and a logits GEMM that stores the allowed logits only, "
+                         "or the whole fp32 logits tensor written and the constraint after it")
+    ap.add_argument("--masked-from-step", type=int, default=None,
+                    help="first step that selects through allow bits (default: chosen from the trie's fan-out per level)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -674,7 +703,8 @@ def main():
     dec = build_decoder(cfg, inp, device, residual_bf16=(args.residual == "bf16"),
                         fold_layer_norm=(None if args.layer_norm == "folded" else False),
                         persist_stream_l2=(None if args.l2_persist == "on" else False),
-                        kv_in_place=(args.kv_cache == "inplace"))
+                        kv_in_place=(args.kv_cache == "inplace"), logits_allowed_only=(args.logits == "allowed"),
+                        masked_from_step=args.masked_from_step)
     dec._layer_tensors = _layer_tensor_views(dec, inp)
     enc_dev = torch.from_numpy(inp["enc_bits"].view(np.int16).copy()).to(device).view(torch.bfloat16)
     dec.project_cross_kv(enc_dev)

@@ -268,6 +268,21 @@ grace_status_t grace_gtm_mask_logits_parts(const float* logits, float* row_lse, 
                                            int prefix_len, const float* lse_part, int n_parts,
                                            int32_t* d_status, void* stream);
 
+/* The constraint alone (Sections 3.1, 4.1): allow_bits[r][V / 64] = catalog-valid children of the row's node AND
+ * the request's matcher, exactly the bits grace_gtm_mask* leave, computed from the beam state only.  It needs
+ * no log-probabilities, so it can run BEFORE the logits GEMM of a decode step, which then stores only the
+ * allowed logits (grace_linear_logits_allowed): the [B*M][V] fp32 tensor is never written out.
+ * Arguments and errors as grace_gtm_mask. */
+grace_status_t grace_gtm_allow_bits(const int32_t* beam_node, const uint64_t* beam_key, const grace_trie_t* trie,
+                                    const grace_matcher_t* matcher, uint64_t* allow_bits, int B, int M, int V,
+                                    int prefix_len, int32_t* d_status, void* stream);
+
+/* row_lse[r] = log-sum-exp of row r from the per-tile partials lse_part [R][n_parts][2] of a logits GEMM
+ * (n_parts <= 32), 0 for dead rows (beam_node < 0 or a leaf): the merge grace_gtm_mask_logits_parts performs,
+ * bit for bit, as a kernel of its own for the order allow bits -> GEMM -> merge -> selection. */
+grace_status_t grace_row_lse_from_parts(const float* lse_part, int n_parts, const int32_t* beam_node,
+                                        const grace_trie_t* trie, float* row_lse, int R, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * The paper's own index form (Sections 4.2-4.4, 5.4, Appendix A): CSR child entries that carry
  * ids of deduplicated per-node matcher rows, tested against per-request attribute rows.
@@ -470,6 +485,17 @@ grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx, const uin
                                        uint16_t* y_bf16, float* y_f32, int64_t ldy, float* lse_part,
                                        int M, int N, int K, int relu, void* stream);
 
+/* The logits GEMM of a constrained decode step (Section 3.1: the constraint is known before the logits are):
+ * the products of grace_linear_f32_lse (row_affine NULL) or of grace_linear_layer_norm with lse_part (row_affine
+ * = fp32 [M][2] scratch, eps, col_sum / col_bias as there), with the same lse_part [M][N / 256][2] over ALL
+ * columns, but of the values only those whose bit is set in allow_bits (device, [M][N / 64] words, 16-byte
+ * aligned; bit v % 64 of word v / 64 = column v) are stored, at their place in y_f32 [M][ldy]; every other
+ * element of y_f32 is left as it was.  M >= 1024, N % 256 == 0, else GRACE_UNSUPPORTED_SHAPE. */
+grace_status_t grace_linear_logits_allowed(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw, float eps,
+                                           float* row_affine, const float* col_sum, const float* col_bias,
+                                           const uint64_t* allow_bits, float* y_f32, int64_t ldy, float* lse_part,
+                                           int M, int N, int K, void* stream);
+
 /* out bf16 [R][D] = LayerNorm(x fp32 [R][D]) * gamma + beta, eps inside the square root. */
 grace_status_t grace_layer_norm(const float* x, const float* gamma, const float* beta,
                                 uint16_t* out, int R, int D, float eps, void* stream);
@@ -548,7 +574,9 @@ typedef struct {
                                  them (cheaper where few tokens per row survive; where a fifth of the row
                                  survives, materialised candidates are faster); earlier steps use cand   */
   int32_t masked_from_step;   /* first step (0-based) that takes the allow-bits path                   */
-  int32_t reserved2;
+  int32_t logits_allowed_only; /* != 0 (needs allow_bits, row_lse, lse_part): on the allow-bits steps of large
+                                 width the constraint runs BEFORE the logits GEMM, which then stores only the
+                                 allowed logits; logp holds valid values only where a token is allowed */
   float *lse_part;            /* NULL, or [R_max][V/256][2] (needs row_lse, V % 256 == 0): the logits GEMM
                                  leaves per-tile log-sum-exp partials and the mask kernel merges them     */
   /* LayerNorms folded into the GEMMs behind them (bf16 residual stream only): NULL, or [R_max][2] scratch

@@ -69,7 +69,7 @@ class DecoderStruct(C.Structure):
         ("token", _vp * 2), ("score", _vp * 2), ("node", _vp * 2), ("key", _vp * 2),
         ("parents", _vp), ("out_flat", _vp),
         ("x", _vp), ("x_bf16", _vp), ("h", _vp), ("qkv", _vp), ("attn", _vp), ("logp", _vp), ("row_lse", _vp), ("cand", _vp), ("allow_bits", _vp), ("masked_from_step", C.c_int32),
-        ("reserved2", C.c_int32), ("lse_part", _vp), ("row_affine", _vp), ("cs_out", _vp), ("cb_out", _vp),
+        ("logits_allowed_only", C.c_int32), ("lse_part", _vp), ("row_affine", _vp), ("cs_out", _vp), ("cb_out", _vp),
         ("topk_ws", _vp), ("topk_ws_bytes", C.c_size_t),
         ("d_status", _vp),
     ]
@@ -122,6 +122,11 @@ _linear_folded_ln = _sig("grace_linear_folded_ln", _i32, [_vp, _i64, _vp, _i64, 
                                                          _i32, _i32, _i32, _i32, _vp])
 _linear_layer_norm = _sig("grace_linear_layer_norm", _i32, [_vp, _i64, _vp, _i64, _f32, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
                                                            _i32, _i32, _i32, _i32, _vp])
+_linear_logits_allowed = _sig("grace_linear_logits_allowed", _i32, [_vp, _i64, _vp, _i64, _f32, _vp, _vp, _vp, _vp, _vp, _i64,
+                                                                   _vp, _i32, _i32, _i32, _vp])
+_gtm_allow_bits = _sig("grace_gtm_allow_bits", _i32, [_vp, _vp, C.POINTER(TrieStruct), C.POINTER(MatcherStruct), _vp,
+                                                     _i32, _i32, _i32, _i32, _vp, _vp])
+_row_lse_from_parts = _sig("grace_row_lse_from_parts", _i32, [_vp, _i32, _vp, C.POINTER(TrieStruct), _vp, _i32, _vp])
 _wait_timeouts = _sig("grace_wait_timeouts", _i32, [])
 _stream_l2_persist = _sig("grace_stream_l2_persist", _i32, [_vp, _vp, C.c_size_t, C.c_float])
 _selftest_bounded_wait = _sig("grace_selftest_bounded_wait", _i32, [_vp])
@@ -409,6 +414,34 @@ def grace_linear_layer_norm(x, w_folded, eps: float, row_affine, col_sum, col_bi
                               _dp(y) if f32 else None, y.stride(0), _dp(lse_part), M, N, K, int(relu), _stream()),
            "grace_linear_layer_norm")
     return y
+
+
+def grace_linear_logits_allowed(x, w, allow_bits, y, lse_part, eps: float = 0.0, row_affine=None, col_sum=None,
+                                col_bias=None):
+    """fp32 logits GEMM that stores only the allowed elements of y (bits [M, N/64] int64) and the log-sum-exp
+    partials of all of them; row_affine (fp32 [M, 2] scratch) given: a LayerNorm with eps folded in front."""
+    M, K = x.shape
+    N = w.shape[0]
+    _check(_linear_logits_allowed(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), float(eps), _dp(row_affine),
+                                  _dp(col_sum), _dp(col_bias), _dp(allow_bits), _dp(y), y.stride(0), _dp(lse_part),
+                                  M, N, K, _stream()), "grace_linear_logits_allowed")
+    return y
+
+
+def grace_gtm_allow_bits(beam_node, beam_key, trie: TrieStruct, matcher: MatcherStruct, allow_bits, B: int, M: int,
+                         prefix_len: int, d_status=None):
+    """allow_bits [B*M, V/64] = catalog-valid children AND matcher, from the beam state alone."""
+    _check(_gtm_allow_bits(_dp(beam_node), _dp(beam_key), C.byref(trie), C.byref(matcher), _dp(allow_bits), B, M,
+                           trie.V, prefix_len, _dp(d_status), _stream()), "grace_gtm_allow_bits")
+    return allow_bits
+
+
+def grace_row_lse_from_parts(lse_part, beam_node, trie: TrieStruct, row_lse):
+    """row_lse [R] from the logits GEMM's per-tile partials [R, n_parts, 2]; 0 for dead rows."""
+    R, n_parts = lse_part.shape[0], lse_part.shape[1]
+    _check(_row_lse_from_parts(_dp(lse_part), n_parts, _dp(beam_node), C.byref(trie), _dp(row_lse), R, _stream()),
+           "grace_row_lse_from_parts")
+    return row_lse
 
 
 def grace_stream_l2_persist(t=None, fraction: float = 0.5) -> None:

@@ -36,6 +36,7 @@ extern "C" grace_status_t grace_decoder_validate(const grace_decoder_t* d) {
       if (!w.cb_qkv || !w.cb_qc || !w.cb_1) return GRACE_INVALID_ARG;
     }
   }
+  if (d->logits_allowed_only && (!d->allow_bits || !d->row_lse || !d->lse_part)) return GRACE_INVALID_ARG;
   for (int i = 0; i < 2; ++i)
     if (!d->token[i] || !d->score[i] || !d->node[i] || !d->key[i]) return GRACE_INVALID_ARG;
   if (d->trie.V != d->V || d->trie.L != d->L || !d->trie.child_bits || !d->trie.child_base) return GRACE_INVALID_ARG;
@@ -129,10 +130,31 @@ extern "C" grace_status_t grace_decode_step(const grace_decoder_t* d, int t, voi
   // the logits GEMM can leave the rows' log-sum-exp partials (large steps), the mask kernel then merges them
   const int n_parts = d->V / 256;
   const bool parts = d->lse_part != nullptr && d->row_lse != nullptr && R >= 1024 && (d->V % 256) == 0 && n_parts <= 32;
+  int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
+  if (parts && d->logits_allowed_only && d->allow_bits != nullptr && t >= d->masked_from_step) {
+    // The constraint first (it needs the beam state only), then a logits GEMM that stores only the allowed logits
+    // and the rows' log-sum-exp partials, their merge, and the selection through the allow bits: neither the
+    // logits tensor nor the candidates are written out.
+    GRACE_TRY(grace_gtm_allow_bits(d->node[cur], d->key[cur], &d->trie, &d->matcher, d->allow_bits, B, M, d->V, t, st,
+                                   stream));
+    if (folded)
+      GRACE_TRY(grace_linear_logits_allowed(d->x_bf16, D, d->w_out, D, d->ln_eps, d->row_affine, d->cs_out, d->cb_out,
+                                            d->allow_bits, d->logp, d->V, d->lse_part, R, d->V, D, stream));
+    else {
+      GRACE_TRY(layer_norm(d->lnf_g, d->lnf_b));
+      GRACE_TRY(grace_linear_logits_allowed(d->h, D, d->w_out, D, 0.f, nullptr, nullptr, nullptr, d->allow_bits, d->logp,
+                                            d->V, d->lse_part, R, d->V, D, stream));
+    }
+    GRACE_TRY(grace_row_lse_from_parts(d->lse_part, n_parts, d->node[cur], &d->trie, d->row_lse, R, stream));
+    GRACE_TRY(grace_beam_topk_masked(d->logp, d->allow_bits, d->score[cur], d->row_lse, B, M, d->V, K, d->score[nxt],
+                                     d->out_flat, parent_out, d->token[nxt], d->topk_ws, d->topk_ws_bytes, st, stream));
+    GRACE_TRY(grace_beam_update(parent_out, d->token[nxt], d->score[nxt], d->node[cur], d->key[cur], &d->trie,
+                                d->node[nxt], d->key[nxt], B, K, M, t, st, stream));
+    return GRACE_OK;
+  }
   GRACE_TRY(ln_linear(d->lnf_g, d->lnf_b, d->w_out, d->cs_out, d->cb_out, nullptr, d->logp, d->V, d->V, 0,
                       parts ? d->lse_part : nullptr));
   // log-softmax, CD + GTM mask and score add: one fused kernel when row_lse is provided
-  int32_t* parent_out = d->parents + (int64_t)(t + 1) * d->R_max;
   if (d->row_lse != nullptr && d->allow_bits != nullptr && t >= d->masked_from_step) {
     // candidates never materialised: the mask kernel leaves the allow bits and the rows' log-sum-exp, the
     // selection reads the logits through them (and only where a token is allowed)

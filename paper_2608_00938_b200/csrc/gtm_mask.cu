@@ -49,6 +49,19 @@ __device__ __forceinline__ int nth_set_bit64(uint64_t word, int n) {
 
 constexpr int kMaskWarpsPerBlock = 8;
 
+// The log-sum-exp of a row from per-lane (maximum, sum of e^(x - maximum)) pairs (lanes without a pair pass
+// (-inf, 0)): every lane returns the same value.  One definition, with the roundings spelled out, for the mask
+// kernel and the merge kernel below, so that both give the same bits.
+__device__ __forceinline__ float warp_merge_lse(float m_l, float s_l) {
+  float m_w = m_l;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
+  float s_w = (m_l > -INFINITY) ? __fmul_rn(s_l, expf(m_l - m_w)) : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s_w = __fadd_rn(s_w, __shfl_xor_sync(kFullMask, s_w, o));
+  return __fadd_rn(m_w, logf(s_w));
+}
+
 // One warp per beam row, two phases per chunk of 2048 tokens:
 //   1. the catalog-valid children (set bits of the node's child bitmask) are enumerated compactly,
 //      lane k takes the k-th, (k+32)-th, ... child, evaluates the request's matcher for it and ORs
@@ -85,7 +98,7 @@ gtm_mask_kernel(const MaskParams p) {
     if (node >= p.num_nodes && lane == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
     dead = true;
   }
-  const float score = __ldg(p.beam_score + r);
+  const float score = p.beam_score != nullptr ? __ldg(p.beam_score + r) : 0.f;    // not needed for allow bits alone
   const uint64_t row_key = (KIND == GRACE_MATCH_PREFIX_BLOOM) ? __ldg(p.beam_key + r) : 0ull;
   const uint64_t* req_bits = (KIND == GRACE_MATCH_NONE) ? nullptr : p.matcher_bits + (int64_t)b * p.words_per_request;
   const int32_t base = dead ? -1 : __ldg(p.child_base + node);
@@ -125,14 +138,17 @@ gtm_mask_kernel(const MaskParams p) {
         m_l = mx;
       }
     }
-    float m_w = m_l;
+    if (!SPLIT) {
+      lse = warp_merge_lse(m_l, s_l);
+    } else {
+      float m_w = m_l;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
-    float s_w = (m_l > -INFINITY) ? s_l * expf(m_l - m_w) : 0.f;
+      for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
+      float s_w = (m_l > -INFINITY) ? s_l * expf(m_l - m_w) : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s_w += __shfl_xor_sync(kFullMask, s_w, o);
-    if (!SPLIT) lse = m_w + logf(s_w);
-    else if (lane == 0) { s_lse[0][wib] = m_w; s_lse[1][wib] = s_w; }
+      for (int o = 16; o > 0; o >>= 1) s_w += __shfl_xor_sync(kFullMask, s_w, o);
+      if (lane == 0) { s_lse[0][wib] = m_w; s_lse[1][wib] = s_w; }
+    }
   }
   if (SPLIT && LOGITS) {                                 // merge the warps' (maximum, rescaled sum) pairs
     __syncthreads();
@@ -254,6 +270,29 @@ gtm_mask_kernel(const MaskParams p) {
     sync_row();
   }
   if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
+}
+
+// The rows' log-sum-exp from the partials a logits GEMM left per 256-column tile, when the mask ran BEFORE that
+// GEMM (allow bits first, so that the GEMM stores only allowed logits): one warp per row, the arithmetic of the
+// mask kernel's own merge; dead rows (no node, or a leaf) get 0 as there.
+__global__ void __launch_bounds__(256)
+row_lse_from_parts_kernel(const float2* __restrict__ lse_part, int n_parts, const int32_t* __restrict__ beam_node,
+                          int64_t num_internal, float* __restrict__ row_lse, int R) {
+  pdl_wait();
+  pdl_trigger();
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= R) return;
+  const int node = __ldg(beam_node + r);
+  const bool dead = node < 0 || node >= num_internal;
+  float m_l = -INFINITY, s_l = 0.f;
+  if (!dead && lane < n_parts) {
+    const float2 pr = __ldg(lse_part + (int64_t)r * n_parts + lane);
+    m_l = pr.x;
+    s_l = pr.y;
+  }
+  const float lse = dead ? 0.f : warp_merge_lse(m_l, s_l);
+  if (lane == 0) row_lse[r] = lse;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -482,7 +521,9 @@ static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse
                                   int V, int prefix_len, int32_t* d_status, void* stream,
                                   const float* lse_part = nullptr, int n_parts = 0) {
   using namespace grace;
-  if (!logp || !beam_score || !beam_node || !matcher || (!cand && !allow_bits)) return GRACE_INVALID_ARG;
+  const bool bits_only = (logp == nullptr);              // CD + matcher alone: no values in, allow bits out
+  if (bits_only && (logits || cand || !allow_bits)) return GRACE_INVALID_ARG;
+  if ((!bits_only && !beam_score) || !beam_node || !matcher || (!cand && !allow_bits)) return GRACE_INVALID_ARG;
   if (B <= 0 || M <= 0 || (int64_t)B * M > 0x7fffffff) return GRACE_INVALID_ARG;
   if (!trie_ok(trie, V)) return GRACE_INVALID_ARG;
   if (prefix_len < 0 || prefix_len >= trie->L) return GRACE_INVALID_ARG;
@@ -563,6 +604,25 @@ extern "C" grace_status_t grace_gtm_mask_logits_parts(const float* logits, float
                                                       void* stream) {
   return launch_mask(logits, true, row_lse, beam_score, beam_node, beam_key, trie, matcher, cand, allow_bits, B, M, V,
                      prefix_len, d_status, stream, lse_part, n_parts);
+}
+
+extern "C" grace_status_t grace_gtm_allow_bits(const int32_t* beam_node, const uint64_t* beam_key,
+                                               const grace_trie_t* trie, const grace_matcher_t* matcher,
+                                               uint64_t* allow_bits, int B, int M, int V, int prefix_len,
+                                               int32_t* d_status, void* stream) {
+  return launch_mask(nullptr, false, nullptr, nullptr, beam_node, beam_key, trie, matcher, nullptr, allow_bits, B, M, V,
+                     prefix_len, d_status, stream);
+}
+
+extern "C" grace_status_t grace_row_lse_from_parts(const float* lse_part, int n_parts, const int32_t* beam_node,
+                                                   const grace_trie_t* trie, float* row_lse, int R, void* stream) {
+  if (!lse_part || !beam_node || !trie || !row_lse || R <= 0 || n_parts < 1 || n_parts > 32 ||
+      (reinterpret_cast<uintptr_t>(lse_part) & 7))
+    return GRACE_INVALID_ARG;
+  grace::launch_pdl(grace::row_lse_from_parts_kernel, dim3((R + 7) / 8), dim3(256), 0, (cudaStream_t)stream,
+                    reinterpret_cast<const float2*>(lse_part), n_parts, beam_node, trie->num_internal, row_lse, R);
+  GRACE_LAUNCH_CHECK();
+  return GRACE_OK;
 }
 
 extern "C" grace_status_t grace_beam_update(const int32_t* parent, const int32_t* token, const float* score,

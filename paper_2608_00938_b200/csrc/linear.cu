@@ -221,7 +221,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 constexpr int kPBK = 64;
 constexpr int kPStagingBytes = 128 * 128;                 // 128 rows x 128 bytes
 
-enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3, kOutF32Lse = 4 };
+enum { kOutBf16 = 0, kOutF32 = 1, kOutF32Add = 2, kOutBf16Add = 3, kOutF32Lse = 4, kOutF32LseAllowed = 5 };
 
 constexpr int kQStages = 6;
 constexpr int kQABytes = 128 * kPBK * 2;                  // 16 KB: 128 rows of A
@@ -244,7 +244,12 @@ __global__ void __launch_bounds__(STATS ? 320 : 192, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part,
                    const float2* __restrict__ aff_row, const float* __restrict__ aff_cs,
-                   const float* __restrict__ aff_cb, float ln_eps) {
+                   const float* __restrict__ aff_cb, float ln_eps, const uint64_t* __restrict__ allow_bits,
+                   float* __restrict__ y_direct, int64_t ldy) {
+  // kOutF32LseAllowed: the log-sum-exp partials of every row and tile as in kOutF32Lse, but of the values
+  // themselves only those whose bit is set in allow_bits [M][N / 64] are stored, by the row's own thread at
+  // their place in y_direct [M][ldy] (no staging tile, no TMA store): with a constrained decode's allow bits
+  // the fp32 logits tensor is never written out.
   extern __shared__ __align__(1024) uint8_t smem_pair[];
   uint8_t* tiles = smem_pair;
   if ((tc::smem_addr(tiles) & 1023u) != 0) {               // the swizzled tiles need it; same answer in every thread
@@ -393,8 +398,18 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     // ahead, so their latency never sits between two tiles of an epilogue that is the pair's critical path.
     // (The loads are unconditional, from clamped addresses, so that nothing waits for them before their use.)
     float2 ar_next = make_float2(1.f, 0.f), cs_next = make_float2(0.f, 0.f), cb_next = make_float2(0.f, 0.f);
+    constexpr bool kAllowed = (OUT == kOutF32LseAllowed);
+    ulonglong2 aw_lo_next = make_ulonglong2(0ull, 0ull), aw_hi_next = aw_lo_next;      // the row's 256 allow bits of the tile
     const float* cs_or_cb = aff_cs != nullptr ? aff_cs : aff_cb;
     auto fetch_affine = [&](int tile) {
+      if (kAllowed) {
+        const int ta = min(tile, total - 1);
+        const int ma = (ta / n_tiles) * 256 + (int)rank * 128 + row, na = (ta % n_tiles) * 256;
+        const ulonglong2* aw = reinterpret_cast<const ulonglong2*>(allow_bits + (int64_t)min(ma, M - 1) * (N >> 6) + (na >> 6));
+        aw_lo_next = __ldg(aw);
+        aw_hi_next = __ldg(aw + 1);
+        if (ma >= M) aw_lo_next = aw_hi_next = make_ulonglong2(0ull, 0ull);
+      }
       if (aff_row == nullptr) return;
       tile = min(tile, total - 1);
       const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
@@ -408,6 +423,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       const int m0 = (tile / n_tiles) * 256 + (int)rank * 128, n0 = (tile % n_tiles) * 256;
       const int ab = local & 1;
       float2 ar = ar_next;                                 // rows and columns past the edge: values never stored
+      const ulonglong2 aw_lo = aw_lo_next, aw_hi = aw_hi_next;
       const float4 cv = aff_cs != nullptr ? make_float4(cs_next.x, cs_next.y, cb_next.x, cb_next.y)
                                           : make_float4(cb_next.x, cb_next.y, 0.f, 0.f);
       bool ok = tc::mbar_wait_cluster(acc_full + ab, (local >> 1) & 1, abort_flag);
@@ -459,6 +475,61 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       };
 #pragma unroll 1
       for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
+        if (kAllowed) {
+          uint32_t r[32];
+          tc::tmem_ld32(t_acc + (uint32_t)(c * 32), r);
+          // the tile's column vectors in shared memory: written by all four warps above, read by all in fold();
+          // without the staging barriers of the other epilogues this path orders the two itself, once per tile
+          if (c == 0) tc::named_bar_sync(1, 128);
+          tc::tmem_ld_wait();
+          fold(r, c * 32);
+          if (c == 256 / kColsPerChunk - 1) tc::named_bar_sync(1, 128);
+          {
+            float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
+#pragma unroll
+            for (int i = 4; i < 32; i += 4) {
+              m0c = fmaxf(m0c, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+              m1c = fmaxf(m1c, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
+            }
+            const float m_new = fmaxf(lse_m, fmaxf(m0c, m1c));
+            const float kLog2e = 1.4426950408889634f;
+            const float neg = -m_new * kLog2e;
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              s0 += fast_ex2(fmaf(__uint_as_float(r[i]), kLog2e, neg));
+              s1 += fast_ex2(fmaf(__uint_as_float(r[i + 1]), kLog2e, neg));
+            }
+            lse_s = lse_s * fast_ex2((lse_m - m_new) * kLog2e) + (s0 + s1);
+            lse_m = m_new;
+          }
+          const uint64_t aw = (c < 4) ? ((c < 2) ? aw_lo.x : aw_lo.y) : ((c < 6) ? aw_hi.x : aw_hi.y);
+          const uint32_t bits = (uint32_t)(aw >> ((c & 1) * 32));
+          if (bits != 0u) {
+            float* dst = y_direct + (int64_t)(m0 + row) * ldy + n0 + c * 32;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t nib = (bits >> (4 * j)) & 0xfu;
+              if (nib == 0xfu) {
+                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+              } else if (nib != 0u) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if ((nib >> e) & 1u) dst[4 * j + e] = __uint_as_float(r[4 * j + e]);
+              }
+            }
+          }
+          if (c == 256 / kColsPerChunk - 1) {
+            if (m0 + row < M) lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = make_float2(lse_m, lse_s);
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (rank == 0) tc::mbar_arrive(acc_empty + ab);
+              else tc::mbar_arrive_remote(acc_empty + ab, 0);
+            }
+          }
+          continue;
+        }
         uint8_t* buf = staging + (g & 1) * kPStagingBytes;
         uint32_t rr[kBf16Out ? 2 : 1][32];
         if (kBf16Out) {                                    // the chunk's loads fly while the staging buffer frees up
@@ -559,11 +630,16 @@ struct Affine {                                            // LayerNorm folded i
   float eps = 0.f;                                         // in_kernel_stats only
   bool in_kernel_stats = false;                            // the pair kernel forms (rstd, -rstd * mean) itself
 };
+struct AllowedStores {                                     // kOutF32LseAllowed
+  const uint64_t* bits = nullptr;
+  float* y = nullptr;
+  int64_t ldy = 0;
+};
 
 template <int OUT, bool STATS = false>
 static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, int M, int N,
                                   int K, int relu, cudaStream_t s, float2* lse_part = nullptr,
-                                  Affine aff = Affine{nullptr, nullptr, nullptr}) {
+                                  Affine aff = Affine{nullptr, nullptr, nullptr}, AllowedStores al = AllowedStores{}) {
   static unsigned long long attr_set_devices = 0;
   static int max_clusters_of[kMaxDevices] = {0};
   cudaLaunchConfig_t cfg = {};
@@ -588,7 +664,8 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   const int max_clusters = max_clusters_of[su.dev];
   const int total = ((N + 255) / 256) * ((M + 255) / 256);
   cfg.gridDim = dim3(2 * (total < max_clusters ? total : max_clusters));
-  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT, STATS>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb, aff.eps));
+  GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, linear_pair_kernel<OUT, STATS>, mx, mw, my, M, N, K, relu, lse_part, aff.row, aff.cs, aff.cb, aff.eps,
+                                    al.bits, al.y, al.ldy));
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }
@@ -614,7 +691,8 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
                                   uint16_t* y_bf16, float* y_f32, int64_t ldy, const float* residual,
                                   bool add_into_bf16, int M, int N, int K, int relu, void* stream,
                                   float* lse_part = nullptr,
-                                  grace::Affine aff = grace::Affine{nullptr, nullptr, nullptr}) {
+                                  grace::Affine aff = grace::Affine{nullptr, nullptr, nullptr},
+                                  const uint64_t* allow_bits = nullptr) {
   using namespace grace;
   if (!x || !w || ((y_bf16 == nullptr) == (y_f32 == nullptr))) return GRACE_INVALID_ARG;
   if (M <= 0 || N <= 0 || K <= 0) return GRACE_INVALID_ARG;
@@ -626,6 +704,8 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
   const bool aliased = (residual != nullptr) && (residual == y_f32);
   if (lse_part != nullptr && !(M >= 1024 && N >= 256 && (N % 256) == 0 && y_f32 != nullptr && residual == nullptr && !relu))
     return GRACE_UNSUPPORTED_SHAPE;
+  if (allow_bits != nullptr && (lse_part == nullptr || (reinterpret_cast<uintptr_t>(allow_bits) & 15)))
+    return GRACE_UNSUPPORTED_SHAPE;                          // allowed-only stores exist in the large-problem kernel only
   if (M >= 1024 && N >= 256 && (residual == nullptr || aliased)) {
     // large GEMM: persistent CTA-pair kernel, TMA-store epilogue (add-reduction when y is the residual stream)
     CUtensorMap mx, mw, my;
@@ -640,6 +720,9 @@ static grace_status_t linear_impl(const uint16_t* x, int64_t ldx, const uint16_t
         !tc::make_tmap(&my, f32 ? (const void*)y_f32 : (const void*)y_bf16, 2, dy, sy, by, f32))
       return GRACE_CUDA_ERROR;
     if (aff.row != nullptr && (add_into_bf16 || aliased)) return GRACE_INVALID_ARG;
+    if (allow_bits != nullptr)
+      return launch_pair<kOutF32LseAllowed>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part), aff,
+                                            AllowedStores{allow_bits, y_f32, ldy});
     if (aff.in_kernel_stats) {
       if (f32) return lse_part != nullptr
                           ? launch_pair<kOutF32Lse, true>(mx, mw, my, M, N, K, relu, s, reinterpret_cast<float2*>(lse_part), aff)
@@ -725,6 +808,24 @@ extern "C" grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx
     if (st != GRACE_OK) return st;
   }
   return linear_impl(x, ldx, w, ldw, y_bf16, y_f32, ldy, nullptr, false, M, N, K, relu, stream, lse_part, aff);
+}
+
+extern "C" grace_status_t grace_linear_logits_allowed(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,
+                                                      float eps, float* row_affine, const float* col_sum,
+                                                      const float* col_bias, const uint64_t* allow_bits, float* y_f32,
+                                                      int64_t ldy, float* lse_part, int M, int N, int K, void* stream) {
+  if (!allow_bits || !y_f32 || !lse_part || (reinterpret_cast<uintptr_t>(lse_part) & 7)) return GRACE_INVALID_ARG;
+  if (M < 1024 || N < 256 || (N % 256)) return GRACE_UNSUPPORTED_SHAPE;
+  grace::Affine aff = {nullptr, nullptr, nullptr};
+  if (row_affine != nullptr) {                              // a LayerNorm in front: statistics first, folded epilogue
+    if (!col_bias || (reinterpret_cast<uintptr_t>(row_affine) & 7) || !grace_aligned16(col_sum) ||
+        !grace_aligned16(col_bias) || ldx != K)
+      return GRACE_INVALID_ARG;
+    const grace_status_t st = grace_row_stats_bf16(x, M, K, eps, row_affine, stream);
+    if (st != GRACE_OK) return st;
+    aff = grace::Affine{reinterpret_cast<const float2*>(row_affine), col_sum, col_bias};
+  }
+  return linear_impl(x, ldx, w, ldw, nullptr, y_f32, ldy, nullptr, false, M, N, K, 0, stream, lse_part, aff, allow_bits);
 }
 
 extern "C" grace_status_t grace_linear_add_bf16(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw,

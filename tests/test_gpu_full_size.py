@@ -305,9 +305,14 @@ def test_bench_decode_path_equals_the_materialised_path_at_config5():
     enc = dev_bf16(inp["enc_bits"])
     B, K = cfg["B"], cfg["final_k"]
     outs = []
-    for materialize in (False, True):
-        dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True, materialize_cand=materialize)
-        if not materialize:
+    # bench's own form (the constraint before a logits GEMM that stores allowed logits only, on every step); the
+    # whole logits tensor written, candidates materialised on the dense trie level and read through allow bits on
+    # the sparse ones; everything materialised
+    for how in (dict(), dict(logits_allowed_only=False), dict(materialize_cand=True)):
+        dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True, **how)
+        if not how:
+            assert dec.allow_bits is not None and dec.logits_allowed_only and dec.masked_from_step == 0
+        elif "logits_allowed_only" in how:
             assert dec.allow_bits is not None and 0 < dec.masked_from_step < cfg["L"]      # a mixed schedule
         dec.project_cross_kv(enc)
         dec.reset(); dec.decode()
@@ -318,14 +323,16 @@ def test_bench_decode_path_equals_the_materialised_path_at_config5():
         del dec
         torch.cuda.empty_cache()
     assert torch.isfinite(outs[0][0]).sum() > B * K // 2
-    assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
-    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+    for other in outs[1:]:
+        assert torch.equal(outs[0][0].view(torch.int32), other[0].view(torch.int32))
+        assert torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
 
 
 def test_bench_decoder_teacher_forced_against_the_oracle_at_config5():
     """The decoder exactly as bench.py builds it (bf16 residual stream, LayerNorm folded into the GEMMs over a
-    centred stream, cache held in place, candidates materialised on the dense trie level and read through
-    allow bits on the sparse ones), teacher-forced on request 0 against the oracle's decode of that request:
+    centred stream, cache held in place, the constraint ahead of a logits GEMM that stores the allowed logits
+    only), and its form with the whole logits tensor written and candidates materialised on the dense trie
+    level, teacher-forced on request 0 against the oracle's decode of that request:
     at every step the allow bits / finite candidates equal the oracle's mask, the log-probabilities agree
     within the decoder tolerance, and the selection, parents, tokens, nodes and keys equal the oracle's
     top-k and state update run on the GPU's own candidates, bit for bit."""
@@ -341,8 +348,20 @@ def test_bench_decoder_teacher_forced_against_the_oracle_at_config5():
     record = []
     OD.beam_search(inp["weights"], inp["shp"], synth.bf16_bits_to_f32(inp["enc_bits"][:1]), trie,
                    OG.PrefixBloomMatcher([bloom0]), cfg["schedule"], cfg["final_k"], record=record)
-    dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True)
-    assert dec.allow_bits is not None and 0 < dec.masked_from_step < L          # both candidate paths are exercised
+    # bench's own form (constraint first, allowed logits only, every step through the allow bits) and the form that
+    # writes the whole logits tensor (dense trie level materialised, sparse levels through the allow bits)
+    for how in (dict(), dict(logits_allowed_only=False)):
+        dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True, **how)
+        if not how:
+            assert dec.allow_bits is not None and dec.logits_allowed_only and dec.masked_from_step == 0
+        else:
+            assert dec.allow_bits is not None and 0 < dec.masked_from_step < L   # both candidate paths are exercised
+        _teacher_force_bench_decoder(dec, record, trie, inp, sizes, V, L, api)
+        del dec
+        torch.cuda.empty_cache()
+
+
+def _teacher_force_bench_decoder(dec, record, trie, inp, sizes, V, L, api):
     dec.project_cross_kv(dev_bf16(inp["enc_bits"]))
     dec.reset()
     for t in range(L):
@@ -372,7 +391,10 @@ def test_bench_decoder_teacher_forced_against_the_oracle_at_config5():
             lse = dec.row_lse[:M].cpu().numpy()
             logp = logits - lse[:, None]
             cand = np.where(step["allow"], score[:, None] + logp, np.float32(-np.inf)).astype(np.float32)
-            got_logp, ref_logp = logp[live], step["logp"][live]
+            if dec.logits_allowed_only:          # the GEMM stored the allowed logits only: the rest of logp is stale
+                got_logp, ref_logp = logp[step["allow"]], step["logp"][step["allow"]]
+            else:
+                got_logp, ref_logp = logp[live], step["logp"][live]
         assert_log_probs_close(got_logp, ref_logp, f"bench decoder step {t}")
         sc, flat, par, tok = OT.beam_topk(cand.reshape(1, M * V), K, V)           # exact, on the GPU's own candidates
         assert np.array_equal(dec.out_flat[:K].cpu().numpy(), flat[0])

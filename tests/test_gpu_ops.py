@@ -897,6 +897,82 @@ def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
     assert bool((scratch == 7.0).all().item()) == in_kernel       # the scratch is touched only by the two-kernel form
 
 
+@pytest.mark.parametrize("M,N,K,density,folded", [(2100, 2048, 512, 0.2, True), (1100, 512, 512, 0.002, False),
+                                                  (1500, 1024, 256, 1.0, True), (1030, 256, 128, 0.0, False),
+                                                  (33000, 2048, 512, 0.0005, True)])
+def test_logits_gemm_stores_only_the_allowed_logits(api, M, N, K, density, folded):
+    """grace_linear_logits_allowed against the dense logits GEMM (grace_linear_f32_lse, or the folded-LayerNorm
+    form with partials): where a bit is set the stored value is the dense one bit for bit, everything else keeps
+    what the buffer held, and the log-sum-exp partials (over ALL columns) are the same bits."""
+    rng = synth.rng_for(5, 900 + M + N)
+    x = synth.normal_bf16(rng, (M, K), 1.5)
+    xc = synth.bf16_bits_to_f32(x).astype(np.float64)
+    x = synth.f32_to_bf16_bits((xc - xc.mean(1, keepdims=True)).astype(np.float32))       # centred rows (no col_sum)
+    w = synth.normal_bf16(rng, (N, K), 0.05)
+    cb = synth.normal_f32(rng, N) if folded else None
+    allow = rng.random((M, N)) < density
+    allow[M // 2] = True                                     # a full row and an empty one whatever the density
+    allow[M // 3] = False
+    bits = OG.pack_allow_bits(allow)
+    dense = torch.zeros((M, N), device=DEV)
+    part = torch.zeros((M, N // 256, 2), device=DEV)
+    aff = torch.zeros((M, 2), device=DEV)
+    if folded:
+        api.grace_linear_layer_norm(dev_bf16(x), dev_bf16(w), 1e-5, aff, None, dev(cb), dense, False, part)
+    else:
+        api.grace_linear_f32_lse(dev_bf16(x), dev_bf16(w), dense, part)
+    sentinel = np.float32(-123.25)
+    y = torch.full((M, N), float(sentinel), device=DEV)
+    part1 = torch.zeros_like(part)
+    api.grace_linear_logits_allowed(dev_bf16(x), dev_bf16(w), dev(bits.view(np.int64)), y, part1, 1e-5,
+                                    aff if folded else None, None, dev(cb) if folded else None)
+    torch.cuda.synchronize()
+    got, ref = y.cpu().numpy(), dense.cpu().numpy()
+    assert np.array_equal(got[allow].view(np.uint32), ref[allow].view(np.uint32))
+    assert (got[~allow] == sentinel).all()
+    assert np.array_equal(part1.cpu().numpy().view(np.uint32), part.cpu().numpy().view(np.uint32))
+
+
+def test_allow_bits_before_the_logits_and_the_merge_of_their_partials(api):
+    """grace_gtm_allow_bits leaves the bits the mask kernels leave (and the oracle's mask), from the beam state
+    alone; grace_row_lse_from_parts gives the rows' log-sum-exp the mask kernel gives from the same partials, bit
+    for bit, 0 on dead rows."""
+    V, L, B, M = 1024, 4, 3, 400
+    sids, trie, elig, node, key, score, logp = _mask_problem(12, V, L, 60000, B, M, 1)
+    node = node.copy()
+    node[5] = -1                                             # a dead row
+    bits, base, _ = api.grace_trie_build_dense(sids, V)
+    trie_s = api.make_trie(dev(bits), dev(base), V, L, trie.num_nodes)
+    for kind in ("bloom", "node"):
+        if kind == "bloom":
+            om = OG.PrefixBloomMatcher([OM.build_prefix_bloom(sids, e, 16, 3) for e in elig])
+            keep = dev(np.stack([api.grace_bloom_build(sids, V, e, 16, 3) for e in elig]))
+            matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, keep, 16, 3)
+        else:
+            om = OG.NodeBitmaskMatcher(np.stack([OM.node_eligibility(trie, sids, e) for e in elig]))
+            keep = dev(np.stack([api.grace_node_bitmask_build(sids, V, e, trie.num_nodes) for e in elig]))
+            matcher = api.make_matcher(api.MATCH_NODE_BITMASK, keep)
+        R = B * M
+        logits = (logp * 3.0).astype(np.float32)
+        d_logits = dev(logits)
+        part = torch.zeros((R, V // 256, 2), device=DEV)
+        lg = logits.reshape(R, V // 256, 256).astype(np.float64)
+        mx = lg.max(2)
+        part.copy_(dev(np.stack([mx, np.exp(lg - mx[:, :, None]).sum(2)], axis=2).astype(np.float32)))
+        lse_a, allow_a = torch.zeros(R, device=DEV), torch.zeros((R, V // 64), dtype=torch.int64, device=DEV)
+        api.grace_gtm_mask_logits_parts(d_logits, lse_a, dev(score), dev(node), dev(key), trie_s, matcher, None, allow_a,
+                                        B, M, 1, part)
+        lse_b, allow_b = torch.full((R,), 9.0, device=DEV), torch.full((R, V // 64), -1, dtype=torch.int64, device=DEV)
+        api.grace_gtm_allow_bits(dev(node), dev(key), trie_s, matcher, allow_b, B, M, 1)
+        api.grace_row_lse_from_parts(part, dev(node), trie_s, lse_b)
+        torch.cuda.synchronize()
+        assert torch.equal(allow_a, allow_b)
+        assert torch.equal(lse_a.view(torch.int32), lse_b.view(torch.int32))
+        assert lse_b[5].item() == 0.0
+        _, a_ref, _ = OG.gtm_mask(logp, score, node, key, 1, trie, om, B, M)
+        assert np.array_equal(allow_b.cpu().numpy().view(np.uint64), OG.pack_allow_bits(a_ref))
+
+
 def test_l2_residency_window_is_a_hint_only(api):
     """grace_stream_l2_persist changes where lines live, never what a kernel computes: the same GEMM into the
     same residual stream gives the same bits with the window set, with it cleared, and on another stream."""
