@@ -575,6 +575,15 @@ def mask_roofline(dec, cfg, inp, peaks):
                                                          matcher, cand, None, B, M, 1, dec.d_status), 1)
         out[name] = dict(p50_us=p50, p99_us=p99, gbs=nbytes / p50 / 1e3, bound="hbm",
                          frac=nbytes / p50 / 1e3 / peaks["hbm_gbs"], live_rows=live, rows=R, note=note)
+    # the form the decode loop runs: the constraint alone (allow bits from the beam state), ahead of the logits GEMM
+    bits = torch.empty((R, V // 64), dtype=torch.int64, device=dec.device)
+    p50, p99 = _time_op(lambda i: api.grace_gtm_allow_bits(dec.node[1][:R], dec.key[1][:R], dec.trie, dec.matcher, bits,
+                                                           B, M, 1, dec.d_status), 1)
+    out["gtm_allow_bits_depth1_B32_M2048_V2048"] = dict(
+        p50_us=p50, p99_us=p99, bound="l2/dsmem probes", frac=None, rows=R,
+        note="prefix Bloom 2^22 x 4, allow bits only (no values in or out): the request's filter sits in the shared "
+             "memory of a cluster of four CTAs and is probed with ld.shared::cluster; against the fused mask above "
+             "this is what the loop pays for the constraint at the dense trie level")
     return out
 
 

@@ -8,6 +8,7 @@
 // sectors in only where a token is allowed.  HBM-bound at the root levels (4 bytes out plus up to
 // 4 bytes in per candidate); with the Bloom matcher the random 8-byte probes into the request's
 // 512 KB filter (L2-resident) add a latency/L2-bandwidth term.
+#include <cstdlib>
 #include "common.cuh"
 
 namespace grace {
@@ -270,6 +271,118 @@ gtm_mask_kernel(const MaskParams p) {
     sync_row();
   }
   if (saw_nan) flag_status(p.d_status, GRACE_DEV_NAN);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The allow bits of the prefix-Bloom matcher with the request's filter in distributed shared memory.
+// The probes of the kernel above are random 8-byte reads in a 512 KB filter that lives in L2: the kernel is
+// bound by the 32-byte sectors it pulls from there.  Here a cluster of kBloomClusterCtas CTAs serves ONE
+// request: each CTA copies its share of the filter words into its shared memory once, and every probe is an
+// ld.shared::cluster from the CTA that owns the word.  Same hash, same positions, same bits.
+// grid (kBloomClusterCtas, B); the cluster's warps take the request's rows round-robin.
+// MEASURED SLOWER than the L2 form and therefore off unless GRACE_BLOOM_DSMEM is set in the environment: at 32
+// requests x 2048 rows x 2048 tokens (430 catalog children per row, filter 2^22 x 4) 796 us against 278 us;
+// with four probes in flight per lane instead of one at a time 1184 us.  Time follows the number of probes
+// (63 M and 113 M): random 8-byte loads from other SMs' shared memory run at about a third of a probe per
+// clock and SM, the L2 serves 2.4 times that.  Kept as the record of that measurement.
+// ---------------------------------------------------------------------------------------------
+constexpr int kBloomClusterCtas = 4;
+constexpr int kBloomClusterWarps = 16;                    // per CTA
+
+__device__ __forceinline__ uint32_t mask_cluster_rank() {
+  uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void mask_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint64_t ld_cluster_u64(uint32_t local_smem_addr, uint32_t rank) {
+  uint64_t v;
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %1, %2;\n\t"
+      "ld.shared::cluster.u64 %0, [ra];\n\t}"
+      : "=l"(v) : "r"(local_smem_addr), "r"(rank) : "memory");
+  return v;
+}
+
+__global__ void __launch_bounds__(kBloomClusterWarps * 32, 1)
+gtm_allow_bloom_cluster_kernel(const MaskParams p, int log2_words_per_cta) {
+  extern __shared__ __align__(16) uint64_t s_filter[];                         // this CTA's words of the request's filter
+  __shared__ uint64_t s_words[kBloomClusterWarps][32];
+  __shared__ unsigned long long s_allow[kBloomClusterWarps][32];
+  __shared__ int s_incl[kBloomClusterWarps][32];
+  pdl_wait();
+  pdl_trigger();
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const uint32_t rank = mask_cluster_rank();
+  const int b = blockIdx.y;
+  const int words_per_cta = 1 << log2_words_per_cta;
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(p.matcher_bits + (int64_t)b * p.words_per_request +
+                                                     (int64_t)rank * words_per_cta);
+    uint4* dst = reinterpret_cast<uint4*>(s_filter);
+    for (int i = threadIdx.x; i < words_per_cta / 2; i += blockDim.x) dst[i] = __ldg(src + i);
+  }
+  __syncthreads();
+  mask_cluster_sync();                                     // every share is in place before anyone probes
+  const uint32_t filter_base = (uint32_t)__cvta_generic_to_shared(s_filter);
+  const int V = p.V, W = V >> 6;
+  uint64_t* words = s_words[wib];
+  unsigned long long* allow = s_allow[wib];
+  int* incl = s_incl[wib];
+  for (int m = (int)rank * kBloomClusterWarps + wib; m < p.M; m += kBloomClusterCtas * kBloomClusterWarps) {
+    const int r = b * p.M + m;
+    int node = __ldg(p.beam_node + r);
+    bool dead = node < 0;
+    if (!dead && node >= p.num_internal) {
+      if (node >= p.num_nodes && lane == 0) flag_status(p.d_status, GRACE_DEV_BAD_INDEX);
+      dead = true;
+    }
+    const uint64_t row_key = __ldg(p.beam_key + r);
+    for (int w0 = 0; w0 < W; w0 += 32) {
+      uint64_t word = 0;
+      if (!dead && w0 + lane < W) word = __ldg(p.child_bits + (int64_t)node * W + w0 + lane);
+      const int pc = __popcll(word);
+      int inc = pc;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(kFullMask, inc, d);
+        if (lane >= d) inc += o;
+      }
+      const int total = __shfl_sync(kFullMask, inc, 31);
+      __syncwarp();
+      words[lane] = word;
+      incl[lane] = inc;
+      allow[lane] = 0ull;
+      __syncwarp();
+      for (int k0 = 0; k0 < total; k0 += 32) {
+        const int k = k0 + lane;
+        const bool have = k < total;
+        int lo = 0;
+#pragma unroll
+        for (int step = 16; step >= 1; step >>= 1)
+          if (have && incl[lo + step - 1] <= k) lo += step;
+        const uint64_t cw = have ? words[lo] : 1ull;
+        const int within = have ? k - (incl[lo] - __popcll(cw)) : 0;
+        const int bit = nth_set_bit64(cw, within);
+        const int v = (w0 << 6) + (lo << 6) + bit;
+        const uint64_t z = mix64(row_key | ((uint64_t)(v + 1) << (16 * p.prefix_len)));
+        const uint32_t h1 = (uint32_t)z, h2 = (uint32_t)(z >> 32) | 1u;
+        bool ok = have;
+        for (int i = 0; i < p.bloom_hashes && ok; ++i) {
+          const uint32_t pos = (h1 + (uint32_t)i * h2) & (uint32_t)p.bloom_mask_bits;
+          const uint32_t w = pos >> 6;
+          const uint64_t fw = ld_cluster_u64(filter_base + ((w & (uint32_t)(words_per_cta - 1)) << 3), w >> log2_words_per_cta);
+          ok = (fw >> (pos & 63)) & 1ull;
+        }
+        if (ok) atomicOr(&allow[lo], 1ull << bit);
+      }
+      __syncwarp();
+      if (w0 + lane < W) p.allow_bits[(int64_t)r * W + w0 + lane] = allow[lane];
+      __syncwarp();
+    }
+  }
+  mask_cluster_sync();                                     // no CTA leaves while its share may still be probed
 }
 
 // The rows' log-sum-exp from the partials a logits GEMM left per 256-column tile, when the mask ran BEFORE that
@@ -568,6 +681,30 @@ static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse
         return GRACE_INVALID_ARG;
       p.bloom_mask_bits = (int)(uint32_t)((1ull << matcher->bloom_log2_bits) - 1ull);
       p.bloom_hashes = matcher->bloom_hashes;
+      static const bool dsmem_filter = getenv("GRACE_BLOOM_DSMEM") != nullptr;    // measured slower: see the kernel
+      if (dsmem_filter && bits_only && matcher->bloom_log2_bits >= 10 && matcher->bloom_log2_bits <= 22 && M >= 256 &&
+          grace_aligned16(matcher->bits)) {
+        // the request's filter in the shared memory of a cluster of four CTAs (up to 128 KB each)
+        const int log2_words_per_cta = matcher->bloom_log2_bits - 6 - 2;
+        const size_t smem = (size_t)8 << log2_words_per_cta;
+        static unsigned long long attr_set_devices = 0;
+        DeviceSetup su(&attr_set_devices);
+        if (su) {
+          GRACE_CUDA_TRY(cudaFuncSetAttribute(gtm_allow_bloom_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              128 * 1024));
+          su.done();
+        }
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kBloomClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.gridDim = dim3(kBloomClusterCtas, B); cfg.blockDim = dim3(kBloomClusterWarps * 32);
+        cfg.dynamicSmemBytes = smem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
+        GRACE_CUDA_TRY(cudaLaunchKernelEx(&cfg, gtm_allow_bloom_cluster_kernel, p, log2_words_per_cta));
+        break;
+      }
       GRACE_MASK_LAUNCH(GRACE_MATCH_PREFIX_BLOOM);
       break;
     default:

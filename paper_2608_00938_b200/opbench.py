@@ -44,6 +44,7 @@ def main():
     ap.add_argument("--bf16stream", action="store_true", help="linear / layer_norm: bf16 residual stream")
     ap.add_argument("--kway", type=int, default=1, help="lookup: static k-way partitioned rows with this k at every level")
     ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
+    ap.add_argument("--allow-only", action="store_true", help="mask: the constraint alone (grace_gtm_allow_bits)")
     ap.add_argument("--inplace", action="store_true",
                     help="self_attn: the cache slabs are the steps' QKV projections (nothing written but the output)")
     ap.add_argument("--folded", action="store_true",
@@ -129,6 +130,13 @@ def main():
         node = torch.arange(R, device=dev, dtype=torch.int32)
         key = torch.randint(1, a.V, (R,), device=dev, dtype=torch.int64)
         cand = torch.empty_like(logp)
+        if a.allow_only:
+            # the constraint alone (allow bits from the beam state); GRACE_BLOOM_DSMEM=1 in the environment selects the
+            # variant that keeps the request's Bloom filter in the shared memory of a four-CTA cluster
+            allow = torch.empty(R, W, dtype=torch.int64, device=dev)
+            us = _time(lambda: api.grace_gtm_allow_bits(node, key, trie, matcher, allow, a.B, a.M, 1), a.iters)
+            print(f"allow_bits[{a.matcher}] R={R} V={a.V} density={a.density}: {us:.1f} us")
+            return
         if a.logits:
             lse = torch.empty(R, device=dev)
             us = _time(lambda: api.grace_gtm_mask_logits(logp, lse, score, node, key, trie, matcher, cand, None, a.B, a.M, 1),

@@ -999,3 +999,44 @@ def test_l2_residency_window_is_a_hint_only(api):
         api.grace_stream_l2_persist(base, 0.0)
     with pytest.raises(Exception):
         api.grace_stream_l2_persist(base, 1.5)
+
+
+_DSMEM_CHILD = r"""
+import sys, numpy as np, torch
+sys.path.insert(0, sys.argv[1])
+sys.path.insert(0, sys.argv[1] + "/tests")
+import synth
+from paper_2608_00938_b200 import api
+from test_gpu_ops import _mask_problem
+from gpu_util import dev
+V, L, B, M = 1024, 4, 2, 600
+sids, trie, elig, node, key, score, logp = _mask_problem(13, V, L, 60000, B, M, 1)
+bits, base, _ = api.grace_trie_build_dense(sids, V)
+trie_s = api.make_trie(dev(bits), dev(base), V, L, trie.num_nodes)
+keep = dev(np.stack([api.grace_bloom_build(sids, V, e, 16, 4) for e in elig]))
+matcher = api.make_matcher(api.MATCH_PREFIX_BLOOM, keep, 16, 4)
+allow = torch.zeros((B * M, V // 64), dtype=torch.int64, device="cuda:0")
+api.grace_gtm_allow_bits(dev(node), dev(key), trie_s, matcher, allow, B, M, 1)
+torch.cuda.synchronize()
+np.save(sys.argv[2], allow.cpu().numpy())
+"""
+
+
+def test_bloom_filter_in_cluster_shared_memory_gives_the_same_bits(api, tmp_path):
+    """The variant of grace_gtm_allow_bits that keeps each request's Bloom filter in the shared memory of a
+    four-CTA cluster (off by default: measured slower; GRACE_BLOOM_DSMEM selects it) leaves the same allow bits as
+    the default form.  The switch is read once per process, so each form runs in a process of its own."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for flag in (None, "1"):
+        env = dict(os.environ)
+        env.pop("GRACE_BLOOM_DSMEM", None)
+        if flag:
+            env["GRACE_BLOOM_DSMEM"] = flag
+        out = str(tmp_path / f"allow_{flag}.npy")
+        subprocess.run([sys.executable, "-c", _DSMEM_CHILD, root, out], check=True, env=env, timeout=600)
+        outs.append(np.load(out))
+    assert outs[0].any() and np.array_equal(outs[0], outs[1])
