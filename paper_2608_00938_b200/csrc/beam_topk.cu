@@ -230,7 +230,6 @@ constexpr int kCollectThreads = 256;
 constexpr int kCollectUnroll = 8;                         // float4 loads in flight per thread
 constexpr int kCollectWarps = kCollectThreads / 32;
 
-constexpr int kStage = 1024;                              // hits staged per CTA before a flush (masked pass)
 constexpr int kWarpStage = 256;                           // hits staged per warp before a flush (dense pass)
 
 // Appends the warp's staged hits to the request's list with one global atomic; returns true once the list
@@ -344,86 +343,100 @@ topk_collect_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d
 }
 
 // Collecting pass over candidates that are not materialised: the unit of work is one 64-bit allow word (64
-// tokens of one row).  A zero word costs one 8-byte load; otherwise the thread visits the word's non-empty
-// groups of four tokens, reads those 16 bytes of logits and tests the (up to four) allowed ones.  Hits are
-// appended one by one (they are rare) with the same staging and overflow rules as the dense pass.
+// tokens of one row).  A zero word costs one 8-byte load; otherwise the thread walks the word's set bits four at a
+// time: the four logits are requested together, then tested (work follows the allowed tokens, not the codebook:
+// a pass over 16-byte groups of four tokens spent most of its instructions on tokens that were not allowed).
+// Hits are rare and go to the warp's own staging list, as in the dense pass (a full stage: straight to the
+// request's list); no block-wide barrier in the loop.
 constexpr int kCollectWords = 8;                          // allow words in flight per thread
 
-__global__ void __launch_bounds__(kCollectThreads, 5)
+__global__ void __launch_bounds__(kCollectThreads, 4)
 topk_collect_masked_kernel(const CandSrc src, TopkHeader* hdr, uint2* lists, int32_t* d_status) {
   pdl_wait();
   pdl_trigger();
-  __shared__ uint2 stage[kStage];
-  __shared__ uint32_t stage_count, flush_base;
+  __shared__ uint2 stage[kCollectWarps][kWarpStage];
+  __shared__ uint32_t stage_count[kCollectWarps];
   const int b = blockIdx.y;
-  const int64_t n_words = src.N >> 6;
+  const int warp = threadIdx.x >> 5;
+  uint2* wstage = stage[warp];
+  uint32_t* wcount = &stage_count[warp];
+  if ((threadIdx.x & 31) == 0) *wcount = 0;
+  __syncwarp();
+  const uint32_t n_words = (uint32_t)(src.N >> 6);
   const uint64_t* words = src.allow + (((int64_t)b * src.N) >> 6);
   uint2* list = lists + (int64_t)b * kCap;
-  const int64_t tile = (int64_t)kCollectThreads * kCollectWords;
-  bool saw_nan = false;
-  if (threadIdx.x == 0) stage_count = 0;
-  __syncthreads();
+  uint32_t* list_count = &hdr[b].count;
+  const uint32_t rows_total = (n_words + kCollectThreads - 1) / kCollectThreads;      // rows of 256 words
+  const uint32_t rows_per_cta = (rows_total + gridDim.x - 1) / gridDim.x;
+  const uint32_t r_begin = blockIdx.x * rows_per_cta;
+  const uint32_t r_end = min(rows_total, r_begin + rows_per_cta);
   const uint32_t t_excl = __ldcg(&hdr[b].t_excl);
-  for (int64_t base = (int64_t)blockIdx.x * tile; base < n_words; base += (int64_t)gridDim.x * tile) {
+  const float thr = __uint_as_float((t_excl & 0x80000000u) ? (t_excl ^ 0x80000000u) : ~t_excl);
+  bool saw_nan = false, dead = false;
+  for (uint32_t r0 = r_begin; r0 < r_end && !dead; r0 += kCollectWords) {
     uint64_t w[kCollectWords];
 #pragma unroll
     for (int u = 0; u < kCollectWords; ++u) {
-      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
-      w[u] = (i < n_words) ? __ldcs(words + i) : 0ull;
+      const uint32_t i = (r0 + u) * kCollectThreads + threadIdx.x;
+      w[u] = (r0 + u < r_end && i < n_words) ? __ldcs(words + i) : 0ull;
     }
 #pragma unroll 1
     for (int u = 0; u < kCollectWords; ++u) {
-      uint64_t bits = w[u];
+      const uint64_t bits = w[u];
       if (bits == 0ull) continue;
-      const int64_t i = base + (int64_t)u * kCollectThreads + threadIdx.x;
-      const int64_t g0 = (int64_t)b * src.N + (i << 6);    // first token of the word, global element index
+      const uint32_t i = (r0 + u) * kCollectThreads + threadIdx.x;
+      const int64_t g0 = (int64_t)b * src.N + ((int64_t)i << 6);    // first token of the word, global element index
       const int64_t r = (src.log2_V >= 0) ? (g0 >> src.log2_V) : (g0 / src.V);
       const float lse = __ldg(src.row_lse + r), sc = __ldg(src.row_score + r);
-      while (bits != 0ull) {
-        const int q = (__ffsll((long long)bits) - 1) >> 2;  // group of four tokens holding the lowest set bit
-        const uint32_t nib = (uint32_t)(bits >> (4 * q)) & 0xfu;
-        bits &= ~(0xfull << (4 * q));
-        const float4 x = __ldg(reinterpret_cast<const float4*>(src.data + g0 + 4 * q));
-        const float xs[4] = {x.x, x.y, x.z, x.w};
+      const float* tok = src.data + g0;
+      uint64_t rest = bits;
+#pragma unroll 1
+      while (rest != 0ull) {
+        // the next (up to) four allowed tokens of the word: their logits are requested together
+        int pos[4];
+        float x[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if (!((nib >> j) & 1u)) continue;
-          const float val = sc + (xs[j] - lse);
+        for (int e = 0; e < 4; ++e) {
+          pos[e] = (rest != 0ull) ? __ffsll((long long)rest) - 1 : -1;
+          rest &= rest - 1ull;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[e] = (pos[e] >= 0) ? __ldg(tok + pos[e]) : 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (pos[e] < 0) continue;
+          const float val = sc + (x[e] - lse);
+          if (val <= thr) continue;                               // NaN falls through
           if (val != val) { saw_nan = true; continue; }
-          const uint32_t key = ordered_key(val);
-          if (key <= t_excl) continue;
-          const uint2 entry = make_uint2(key, (uint32_t)((i << 6) + 4 * q + j));
-          const uint32_t pos = atomicAdd(&stage_count, 1u);
-          if (pos < (uint32_t)kStage) {
-            stage[pos] = entry;
-          } else {                                          // stage full: straight to the request's list
-            const uint32_t gpos = atomicAdd(&hdr[b].count, 1u);
+          const uint2 entry = make_uint2(ordered_key(val), (i << 6) + (uint32_t)pos[e]);
+          const uint32_t at = atomicAdd(wcount, 1u);
+          if (at < (uint32_t)kWarpStage) {
+            wstage[at] = entry;
+          } else {                                                // stage full: straight to the request's list
+            const uint32_t gpos = atomicAdd(list_count, 1u);
             if (gpos < (uint32_t)kCap) list[gpos] = entry;
           }
         }
       }
     }
-    __syncthreads();
-    const uint32_t staged = min(stage_count, (uint32_t)kStage);
-    if (staged >= (uint32_t)kStage / 2) {
-      if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
-      __syncthreads();
-      const uint32_t dst = flush_base;
-      for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
-        if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
-      __syncthreads();
-      if (threadIdx.x == 0) stage_count = 0;
-      __syncthreads();
+    __syncwarp();
+    const uint32_t staged = *reinterpret_cast<volatile uint32_t*>(wcount);
+    if (staged >= (uint32_t)kWarpStage / 2) {                     // uniform over the warp
+      if (staged > (uint32_t)kWarpStage) {                        // the overhang went to the list already
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) *reinterpret_cast<volatile uint32_t*>(wcount) = (uint32_t)kWarpStage;
+      }
+      dead = warp_flush(wstage, wcount, list_count, list);
     }
   }
-  __syncthreads();
-  const uint32_t staged = min(stage_count, (uint32_t)kStage);
-  if (staged != 0) {
-    if (threadIdx.x == 0) flush_base = atomicAdd(&hdr[b].count, staged);
-    __syncthreads();
-    const uint32_t dst = flush_base;
-    for (uint32_t e = threadIdx.x; e < staged; e += kCollectThreads)
-      if (dst + e < (uint32_t)kCap) list[dst + e] = stage[e];
+  {
+    __syncwarp();
+    const uint32_t staged = *reinterpret_cast<volatile uint32_t*>(wcount);
+    if (staged > (uint32_t)kWarpStage) {
+      __syncwarp();
+      if ((threadIdx.x & 31) == 0) *reinterpret_cast<volatile uint32_t*>(wcount) = (uint32_t)kWarpStage;
+    }
+    warp_flush(wstage, wcount, list_count, list);
   }
   if (saw_nan) flag_status(d_status, GRACE_DEV_NAN);
 }
@@ -822,6 +835,7 @@ grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, floa
   static unsigned long long attrs_set_devices = 0;
   const size_t final_smem = (size_t)(kCap + kMaxK + kBucketMax) * sizeof(unsigned long long) + 2 * 4096 * sizeof(uint32_t);
   static int collect_grid_of[kMaxDevices] = {0};
+  static int collect_masked_grid_of[kMaxDevices] = {0};
   DeviceSetup su(&attrs_set_devices);
   if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(topk_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)final_smem));
@@ -829,6 +843,8 @@ grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, floa
     GRACE_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, su.dev));
     GRACE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_collect_kernel, kCollectThreads, 0));
     collect_grid_of[su.dev] = n_sm * (per_sm > 0 ? per_sm : 1);
+    GRACE_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topk_collect_masked_kernel, kCollectThreads, 0));
+    collect_masked_grid_of[su.dev] = n_sm * (per_sm > 0 ? per_sm : 1);
     su.done();
   }
   const int collect_grid = collect_grid_of[su.dev];
@@ -844,7 +860,7 @@ grace_status_t launch_beam_topk(const CandSrc& src_in, int B, int K, int V, floa
     if (src.allow != nullptr) {                              // masked: the tile is 256 x 8 allow words
       const int64_t wtile = (int64_t)kCollectThreads * kCollectWords;
       const int64_t wtiles = ((N >> 6) + wtile - 1) / wtile;
-      per_request = collect_grid / B;
+      per_request = collect_masked_grid_of[su.dev] / B;
       if (per_request < 1) per_request = 1;
       if (per_request > wtiles) per_request = wtiles;
       launch_pdl(topk_collect_masked_kernel, dim3((unsigned)per_request, (unsigned)B), dim3(kCollectThreads), 0, s, src, hdr,
