@@ -330,9 +330,10 @@ def op_breakdown(dec, cfg, reps=3):
                 bits = dec.allow_bits[:R]
                 timed("gtm_mask", lambda: api.grace_gtm_allow_bits(dec.node[cur][:R], dec.key[cur][:R], dec.trie, dec.matcher,
                                                                    bits, B, M, t, dec.d_status))
-                if folded:                          # (the call runs the row-statistics kernel itself: 12 us of its time)
+                if folded:                          # (timed apart: in the decode step one call launches both kernels)
+                    timed("row_stats", lambda: api.grace_row_stats_bf16(x, dec.row_affine[:R]))
                     timed("linear", lambda: api.grace_linear_logits_allowed(
-                        x, dec.w_out, bits, logp, lsep, 1e-5, dec.row_affine[:R],
+                        x, dec.w_out, bits, logp, lsep, -1.0, dec.row_affine[:R],
                         None if dec.centre_stream else dec.cs_out, dec.cb_out), 2.0 * R * D * V)
                 else:
                     timed("layer_norm", lambda: api.grace_layer_norm(x, dec.lnf_g, dec.lnf_b, hD))

@@ -487,7 +487,8 @@ grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx, const uin
 
 /* The logits GEMM of a constrained decode step (Section 3.1: the constraint is known before the logits are):
  * the products of grace_linear_f32_lse (row_affine NULL) or of grace_linear_layer_norm with lse_part (row_affine
- * = fp32 [M][2] scratch, eps, col_sum / col_bias as there), with the same lse_part [M][N / 256][2] over ALL
+ * = fp32 [M][2] scratch, eps, col_sum / col_bias as there; eps < 0: row_affine already holds the rows' statistics
+ * from grace_row_stats_bf16 and is only read), with the same lse_part [M][N / 256][2] over ALL
  * columns, but of the values only those whose bit is set in allow_bits (device, [M][N / 64] words, 16-byte
  * aligned; bit v % 64 of word v / 64 = column v) are stored, at their place in y_f32 [M][ldy]; every other
  * element of y_f32 is left as it was.  M >= 1024, N % 256 == 0, else GRACE_UNSUPPORTED_SHAPE. */

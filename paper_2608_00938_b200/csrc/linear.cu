@@ -822,8 +822,10 @@ extern "C" grace_status_t grace_linear_logits_allowed(const uint16_t* x, int64_t
     if (!col_bias || (reinterpret_cast<uintptr_t>(row_affine) & 7) || !grace_aligned16(col_sum) ||
         !grace_aligned16(col_bias) || ldx != K)
       return GRACE_INVALID_ARG;
-    const grace_status_t st = grace_row_stats_bf16(x, M, K, eps, row_affine, stream);
-    if (st != GRACE_OK) return st;
+    if (eps >= 0.f) {                                       // eps < 0: the caller has run grace_row_stats_bf16 into row_affine
+      const grace_status_t st = grace_row_stats_bf16(x, M, K, eps, row_affine, stream);
+      if (st != GRACE_OK) return st;
+    }
     aff = grace::Affine{reinterpret_cast<const float2*>(row_affine), col_sum, col_bias};
   }
   return linear_impl(x, ldx, w, ldw, nullptr, y_f32, ldy, nullptr, false, M, N, K, 0, stream, lse_part, aff, allow_bits);

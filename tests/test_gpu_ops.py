@@ -931,6 +931,12 @@ def test_logits_gemm_stores_only_the_allowed_logits(api, M, N, K, density, folde
     assert np.array_equal(got[allow].view(np.uint32), ref[allow].view(np.uint32))
     assert (got[~allow] == sentinel).all()
     assert np.array_equal(part1.cpu().numpy().view(np.uint32), part.cpu().numpy().view(np.uint32))
+    if folded:                                   # eps < 0: the statistics are the caller's (same kernel, same bits)
+        api.grace_row_stats_bf16(dev_bf16(x), aff, 1e-5)
+        y2 = torch.full((M, N), float(sentinel), device=DEV)
+        api.grace_linear_logits_allowed(dev_bf16(x), dev_bf16(w), dev(bits.view(np.int64)), y2, part1, -1.0, aff, None, dev(cb))
+        torch.cuda.synchronize()
+        assert torch.equal(y2.view(torch.int32), y.view(torch.int32))
 
 
 def test_allow_bits_before_the_logits_and_the_merge_of_their_partials(api):
