@@ -475,7 +475,7 @@ grace_status_t grace_linear_folded_ln(const uint16_t* x, int64_t ldx, const uint
 
 /* grace_row_stats_bf16 (over D = K, with eps) followed by grace_linear_folded_ln, as one call: the LayerNorm over
  * the rows of x [M][K] (ldx == K) and the GEMM behind it.  For M >= 1024 and 256 <= N <= 512 with centred rows
- * (col_sum NULL) it is ONE kernel: the row statistics are formed from the GEMM's own operand tiles in shared
+ * (col_sum NULL) and no lse_part it is ONE kernel: the row statistics are formed from the GEMM's own operand tiles in shared
  * memory while the tensor cores work on them, so the residual stream is not read a second time; row_affine
  * (device, fp32 [M][2], 8-byte aligned) is then not touched.  Otherwise (wider outputs, where forming the
  * statistics once per 256-column tile costs more than reading the stream once) the statistics kernel runs

@@ -801,7 +801,9 @@ extern "C" grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx
   // fifth: measured at 65536 x 512 -> N, one kernel against two: N = 512: 36 us against 43; N = 1536: 99 against
   // 95; N = 2048: 130 against 122.
   const bool pair_kernel = (M >= 1024 && N >= 256);
-  if (pair_kernel && col_sum == nullptr && N <= 512) {
+  // (not for a logits GEMM with log-sum-exp partials: grace_linear_logits_allowed takes its statistics from the
+  // statistics kernel, and the two forms of a decode step are to agree bit for bit)
+  if (pair_kernel && col_sum == nullptr && N <= 512 && lse_part == nullptr) {
     aff.eps = eps;
     aff.in_kernel_stats = true;
   } else {

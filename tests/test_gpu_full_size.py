@@ -295,12 +295,14 @@ def test_decode_step_full_size_teacher_forced_on_one_request(workload, schedule,
         torch.cuda.empty_cache()
 
 
-def test_bench_decode_path_equals_the_materialised_path_at_config5():
-    """The decoder exactly as bench.py builds it (bf16 residual stream; candidates written out on the dense trie
-    level, read through allow bits on the sparse ones) against the same decoder with every step materialised:
-    free-running over all 32 requests, the final beams must agree bit for bit."""
+@pytest.mark.parametrize("workload", ["cfg5", "paper"])
+def test_bench_decode_path_equals_the_materialised_path_at_config5(workload):
+    """The decoder exactly as bench.py builds it (bf16 residual stream; the constraint ahead of a logits GEMM that
+    stores the allowed logits only, every step selected through the allow bits) against the same decoder with the
+    whole logits tensor written, and with every step materialised: free-running over all requests, at serving
+    scale and at the paper's decoder shape (head size 128, V = 512), the final beams must agree bit for bit."""
     import bench
-    cfg = dict(bench.CFG5)
+    cfg = dict(bench.WORKLOADS[workload])
     inp = bench.make_inputs(cfg, 0)
     enc = dev_bf16(inp["enc_bits"])
     B, K = cfg["B"], cfg["final_k"]

@@ -893,7 +893,7 @@ def test_layer_norm_folded_into_the_gemm(api, M, N, K, relu, f32out, centred):
     assert (np.abs(got1 - got) <= slack).all(), np.abs(got1 - got).max()
     if part1 is not None:
         np.testing.assert_allclose(part1.cpu().numpy(), part.cpu().numpy(), rtol=2e-5, atol=2e-5)
-    in_kernel = centred and M >= 1024 and 256 <= N <= 512
+    in_kernel = centred and M >= 1024 and 256 <= N <= 512 and part is None
     assert bool((scratch == 7.0).all().item()) == in_kernel       # the scratch is touched only by the two-kernel form
 
 
