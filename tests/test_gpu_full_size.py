@@ -328,6 +328,23 @@ def test_bench_decode_path_equals_the_materialised_path_at_config5(workload):
     for other in outs[1:]:
         assert torch.equal(outs[0][0].view(torch.int32), other[0].view(torch.int32))
         assert torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
+    if workload != "cfg5":
+        return
+    # the same pair with the LayerNorms as kernels of their own (the logits GEMM then reads the normalised copy)
+    outs = []
+    for how in (dict(), dict(logits_allowed_only=False)):
+        dec = bench.build_decoder(cfg, inp, DEV, residual_bf16=True, fold_layer_norm=False, **how)
+        dec.project_cross_kv(enc)
+        dec.reset(); dec.decode()
+        torch.cuda.synchronize()
+        fin = dec.L & 1
+        assert dec.d_status.item() & ~8 == 0
+        outs.append((dec.score[fin][:B * K].clone(), dec.key[fin][:B * K].clone(), dec.node[fin][:B * K].clone()))
+        del dec
+        torch.cuda.empty_cache()
+    assert torch.isfinite(outs[0][0]).sum() > B * K // 2
+    assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
 
 
 def test_bench_decoder_teacher_forced_against_the_oracle_at_config5():
