@@ -491,7 +491,8 @@ grace_status_t grace_linear_layer_norm(const uint16_t* x, int64_t ldx, const uin
  * from grace_row_stats_bf16 and is only read), with the same lse_part [M][N / 256][2] over ALL
  * columns, but of the values only those whose bit is set in allow_bits (device, [M][N / 64] words, 16-byte
  * aligned; bit v % 64 of word v / 64 = column v) are stored, at their place in y_f32 [M][ldy]; every other
- * element of y_f32 is left as it was.  M >= 1024, N % 256 == 0, else GRACE_UNSUPPORTED_SHAPE. */
+ * element of y_f32 is left as it was or, if it shares an aligned group of 8 columns (one 32-byte sector) with an
+ * allowed one, set to its product as well.  M >= 1024, N % 256 == 0, else GRACE_UNSUPPORTED_SHAPE. */
 grace_status_t grace_linear_logits_allowed(const uint16_t* x, int64_t ldx, const uint16_t* w, int64_t ldw, float eps,
                                            float* row_affine, const float* col_sum, const float* col_bias,
                                            const uint64_t* allow_bits, float* y_f32, int64_t ldy, float* lse_part,

@@ -240,8 +240,39 @@ constexpr int kQSmem = kQStages * kQStageBytes + 2 * kPStagingBytes + 256 + kQAf
 // released by the MMAs' commit AND by these warps; the odd CTA, whose tiles are counted on the even CTA's
 // barrier, learns that a stage has landed from an arrive the even CTA forwards.  Centred rows only (aff_cs ==
 // nullptr): the second half of the column-vector buffer is what holds the statistics.
+// Log-sum-exp partial of a row over a 256-column tile, 32 columns at a time: running maximum and sum of
+// 2^((v - maximum) log2 e).  The tile is summed as TWO halves of 128 columns that are merged at the end: in the
+// allowed-only epilogue two threads (of two warp groups) take a half each, elsewhere one thread takes both, and
+// both forms give the same bits.
+__device__ __forceinline__ void lse_add_chunk(const uint32_t (&r)[32], float& lse_m, float& lse_s) {
+  float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
+#pragma unroll
+  for (int i = 4; i < 32; i += 4) {
+    m0c = fmaxf(m0c, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+    m1c = fmaxf(m1c, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
+  }
+  const float m_new = fmaxf(lse_m, fmaxf(m0c, m1c));
+  const float kLog2e = 1.4426950408889634f;
+  const float neg = __fmul_rn(-m_new, kLog2e);
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    s0 = __fadd_rn(s0, fast_ex2(__fmaf_rn(__uint_as_float(r[i]), kLog2e, neg)));
+    s1 = __fadd_rn(s1, fast_ex2(__fmaf_rn(__uint_as_float(r[i + 1]), kLog2e, neg)));
+  }
+  // first chunk: lse_s = 0 and the factor is 2^-inf = 0
+  lse_s = __fmaf_rn(lse_s, fast_ex2(__fmul_rn(__fsub_rn(lse_m, m_new), kLog2e)), __fadd_rn(s0, s1));
+  lse_m = m_new;
+}
+__device__ __forceinline__ float2 lse_merge_halves(float m_a, float s_a, float m_b, float s_b) {
+  const float kLog2e = 1.4426950408889634f;
+  const float m = fmaxf(m_a, m_b);
+  const float ea = fast_ex2(__fmul_rn(__fsub_rn(m_a, m), kLog2e)), eb = fast_ex2(__fmul_rn(__fsub_rn(m_b, m), kLog2e));
+  return make_float2(m, __fmaf_rn(s_a, ea, __fmul_rn(s_b, eb)));
+}
+
 template <int OUT, bool STATS>
-__global__ void __launch_bounds__(STATS ? 320 : 192, 1)
+__global__ void __launch_bounds__((STATS || OUT == kOutF32LseAllowed) ? 320 : 192, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const __grid_constant__ CUtensorMap map_y, int M, int N, int K, int relu, float2* lse_part,
                    const float2* __restrict__ aff_row, const float* __restrict__ aff_cs,
@@ -279,7 +310,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kQStages; ++s) { tc::mbar_init(full + s, 1); tc::mbar_init(empty + s, STATS ? 5 : 1); }
-    for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, 8); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(acc_full + a, 1); tc::mbar_init(acc_empty + a, OUT == kOutF32LseAllowed ? 16 : 8); }
     if (STATS) {
       for (int s = 0; s < kQStages; ++s) tc::mbar_init(a_ready + s, 1);
       tc::mbar_init(stats_full, 4);
@@ -388,7 +419,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
   } else {
     // ---- epilogue warps 2..5 of both CTAs: TMEM lane quarter q = rows q*32 + lane of this CTA's 128 ----
+    // (kOutF32LseAllowed: warps 6..9 as well; a row's two threads take 128 of the tile's 256 columns each)
     const int q = warp & 3;
+    const int half = (warp >= 6) ? 1 : 0;
     const int row = q * 32 + lane;
     const bool issuer = (warp == 2 && lane == 0);
     constexpr bool kBf16Out = (OUT == kOutBf16 || OUT == kOutBf16Add);
@@ -441,9 +474,10 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
       }
       const uint32_t t_acc = tmem_base + (uint32_t)(ab * 256) + ((uint32_t)(q * 32) << 16);
       float lse_m = -INFINITY, lse_s = 0.f;                // kOutF32Lse: running maximum and sum of 2^((v - max) log2 e)
+      float lse_m_a = -INFINITY, lse_s_a = 0.f;            //   of the tile's first 128 columns, once the second half has begun
       // read after the first chunk's barrier; the previous tile's readers are past its last barrier.
       // With col_sum: [128] x (cs, cs, cb, cb) of two columns; without: col_bias alone, [256] floats.
-      if (aff_row != nullptr) {
+      if (aff_row != nullptr && half == 0) {
         if (aff_cs != nullptr) aff_s[row] = cv;
         else reinterpret_cast<float2*>(aff_s)[row] = make_float2(cv.x, cv.y);
       }
@@ -474,63 +508,52 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           r[i + 1] = __float_as_uint(hi);
         }
       };
+      if (kAllowed) {
+        // Two threads per row, 128 columns each; no staging tile, no TMA store.  The tile's column vectors in
+        // shared memory (written above by the first warp group) are ordered against their readers by the two
+        // barriers, which also carry the second half's partial to the thread that merges and stores it.
+        tc::named_bar_sync(1, 256);
 #pragma unroll 1
-      for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
-        if (kAllowed) {
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = half * 4 + cc;
           uint32_t r[32];
           tc::tmem_ld32(t_acc + (uint32_t)(c * 32), r);
-          // the tile's column vectors in shared memory: written by all four warps above, read by all in fold();
-          // without the staging barriers of the other epilogues this path orders the two itself, once per tile
-          if (c == 0) tc::named_bar_sync(1, 128);
           tc::tmem_ld_wait();
           fold(r, c * 32);
-          if (c == 256 / kColsPerChunk - 1) tc::named_bar_sync(1, 128);
-          {
-            float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
-#pragma unroll
-            for (int i = 4; i < 32; i += 4) {
-              m0c = fmaxf(m0c, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
-              m1c = fmaxf(m1c, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
-            }
-            const float m_new = fmaxf(lse_m, fmaxf(m0c, m1c));
-            const float kLog2e = 1.4426950408889634f;
-            const float neg = -m_new * kLog2e;
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              s0 += fast_ex2(fmaf(__uint_as_float(r[i]), kLog2e, neg));
-              s1 += fast_ex2(fmaf(__uint_as_float(r[i + 1]), kLog2e, neg));
-            }
-            lse_s = lse_s * fast_ex2((lse_m - m_new) * kLog2e) + (s0 + s1);
-            lse_m = m_new;
-          }
-          const uint64_t aw = (c < 4) ? ((c < 2) ? aw_lo.x : aw_lo.y) : ((c < 6) ? aw_hi.x : aw_hi.y);
+          lse_add_chunk(r, lse_m, lse_s);
+          const uint64_t aw = half ? ((cc < 2) ? aw_hi.x : aw_hi.y) : ((cc < 2) ? aw_lo.x : aw_lo.y);
           const uint32_t bits = (uint32_t)(aw >> ((c & 1) * 32));
           if (bits != 0u) {
+            // whole 32-byte sectors (8 columns) that hold an allowed column: a sector written in full costs the
+            // memory system less than a few of its words (no merge with the old contents), and eight predicated
+            // stores per chunk instead of thirty-two (measured at 5 % allowed: 173 -> see the notes)
             float* dst = y_direct + (int64_t)(m0 + row) * ldy + n0 + c * 32;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const uint32_t nib = (bits >> (4 * j)) & 0xfu;
-              if (nib == 0xfu) {
-                *reinterpret_cast<uint4*>(dst + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-              } else if (nib != 0u) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if ((nib >> e) & 1u) dst[4 * j + e] = __uint_as_float(r[4 * j + e]);
+            for (int j = 0; j < 4; ++j) {
+              if ((bits >> (8 * j)) & 0xffu) {
+                *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3]);
+                *reinterpret_cast<uint4*>(dst + 8 * j + 4) = make_uint4(r[8 * j + 4], r[8 * j + 5], r[8 * j + 6], r[8 * j + 7]);
               }
             }
           }
-          if (c == 256 / kColsPerChunk - 1) {
-            if (m0 + row < M) lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = make_float2(lse_m, lse_s);
-            tc::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-              if (rank == 0) tc::mbar_arrive(acc_empty + ab);
-              else tc::mbar_arrive_remote(acc_empty + ab, 0);
-            }
-          }
-          continue;
         }
+        float2* part_s = reinterpret_cast<float2*>(staging);       // [128]: the staging tiles are unused here
+        if (half == 1) part_s[row] = make_float2(lse_m, lse_s);
+        tc::tc_fence_before();
+        tc::named_bar_sync(1, 256);
+        if (half == 0 && m0 + row < M) {
+          const float2 other = part_s[row];
+          lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = lse_merge_halves(lse_m, lse_s, other.x, other.y);
+        }
+        __syncwarp();
+        if (lane == 0) {
+          if (rank == 0) tc::mbar_arrive(acc_empty + ab);
+          else tc::mbar_arrive_remote(acc_empty + ab, 0);
+        }
+        continue;
+      }
+#pragma unroll 1
+      for (int c = 0; c < 256 / kColsPerChunk; ++c, ++g) {
         uint8_t* buf = staging + (g & 1) * kPStagingBytes;
         uint32_t rr[kBf16Out ? 2 : 1][32];
         if (kBf16Out) {                                    // the chunk's loads fly while the staging buffer frees up
@@ -565,24 +588,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
           uint32_t (&r)[32] = rr[0];
           fold(r, c * 32);
           if (OUT == kOutF32Lse) {
-            // the row's log-sum-exp over this tile's 256 columns, 32 at a time (the tiles of a row are merged later)
-            float m0c = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), m1c = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
-#pragma unroll
-            for (int i = 4; i < 32; i += 4) {
-              m0c = fmaxf(m0c, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
-              m1c = fmaxf(m1c, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
-            }
-            const float m_new = fmaxf(lse_m, fmaxf(m0c, m1c));
-            const float kLog2e = 1.4426950408889634f;
-            const float neg = -m_new * kLog2e;
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              s0 += fast_ex2(fmaf(__uint_as_float(r[i]), kLog2e, neg));
-              s1 += fast_ex2(fmaf(__uint_as_float(r[i + 1]), kLog2e, neg));
-            }
-            lse_s = lse_s * fast_ex2((lse_m - m_new) * kLog2e) + (s0 + s1);     // first chunk: lse_s = 0, factor 0
-            lse_m = m_new;
+            // the row's log-sum-exp over this tile's 256 columns, as two halves of 128 (the tiles of a row are merged later)
+            if (c == 4) { lse_m_a = lse_m; lse_s_a = lse_s; lse_m = -INFINITY; lse_s = 0.f; }
+            lse_add_chunk(r, lse_m, lse_s);
           }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -598,7 +606,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         }
         if (c == 256 / kColsPerChunk - 1) {                // accumulator fully read: hand it back to the issuer
           if (OUT == kOutF32Lse && m0 + row < M)
-            lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = make_float2(lse_m, lse_s);
+            lse_part[(int64_t)(m0 + row) * n_tiles + (tile % n_tiles)] = lse_merge_halves(lse_m_a, lse_s_a, lse_m, lse_s);
           tc::tc_fence_before();
           __syncwarp();
           if (lane == 0) {
@@ -649,7 +657,7 @@ static grace_status_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, 
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.blockDim = dim3(STATS ? 320 : 192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
+  cfg.blockDim = dim3((STATS || OUT == kOutF32LseAllowed) ? 320 : 192); cfg.dynamicSmemBytes = kQSmem; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
   DeviceSetup su(&attr_set_devices);
   if (su) {
     GRACE_CUDA_TRY(cudaFuncSetAttribute(linear_pair_kernel<OUT, STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem));
