@@ -45,6 +45,8 @@ def main():
     ap.add_argument("--kway", type=int, default=1, help="lookup: static k-way partitioned rows with this k at every level")
     ap.add_argument("--logits", action="store_true", help="mask: fused log-softmax form (input = logits, in place)")
     ap.add_argument("--allow-only", action="store_true", help="mask: the constraint alone (grace_gtm_allow_bits)")
+    ap.add_argument("--allowed", type=float, default=-1.0,
+                    help="linear: grace_linear_logits_allowed with this fraction of the columns allowed (folded LayerNorm)")
     ap.add_argument("--inplace", action="store_true",
                     help="self_attn: the cache slabs are the steps' QKV projections (nothing written but the output)")
     ap.add_argument("--folded", action="store_true",
@@ -57,7 +59,16 @@ def main():
         x, w = bf(a.M, a.K), bf(a.N, a.K) * 0.05
         y = torch.zeros(a.M, a.N, device=dev, dtype=torch.float32 if (a.f32out or a.residual) and not a.bf16stream
                         else torch.bfloat16)
-        if a.folded:
+        if a.allowed >= 0:
+            # logits GEMM that stores only the allowed logits (random allow bits of the given density) + partials
+            aff, cb = torch.ones(a.M, 2, device=dev), torch.zeros(a.N, device=dev)
+            bits = torch.zeros(a.M, a.N // 64, dtype=torch.int64, device=dev)
+            for bit in range(64):
+                bits |= (torch.rand(a.M, a.N // 64, device=dev) < a.allowed).to(torch.int64) << bit
+            y = torch.zeros(a.M, a.N, device=dev)
+            part = torch.zeros(a.M, a.N // 256, 2, device=dev)
+            us = _time(lambda: api.grace_linear_logits_allowed(x, w, bits, y, part, -1.0, aff, None, cb), a.iters)
+        elif a.folded:
             aff, cb = torch.ones(a.M, 2, device=dev), torch.zeros(a.N, device=dev)
             us = _time(lambda: api.grace_linear_folded_ln(x, w, aff, None, cb, y, a.relu), a.iters)
         elif a.bf16stream:
