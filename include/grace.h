@@ -574,7 +574,8 @@ typedef struct {
   uint64_t *allow_bits;       /* NULL, or [R_max][V/64] (needs row_lse): from step masked_from_step on the
                                  mask kernel writes only these bits and the top-k reads the logits through
                                  them (cheaper where few tokens per row survive; where a fifth of the row
-                                 survives, materialised candidates are faster); earlier steps use cand   */
+                                 survives and the whole logits tensor is written anyway, materialised
+                                 candidates are faster); earlier steps use cand                          */
   int32_t masked_from_step;   /* first step (0-based) that takes the allow-bits path                   */
   int32_t logits_allowed_only; /* != 0 (needs allow_bits, row_lse, lse_part): on the allow-bits steps of large
                                  width the constraint runs BEFORE the logits GEMM, which then stores only the
