@@ -53,13 +53,16 @@ constexpr int kMaskWarpsPerBlock = 8;
 // The log-sum-exp of a row from per-lane (maximum, sum of e^(x - maximum)) pairs (lanes without a pair pass
 // (-inf, 0)): every lane returns the same value.  One definition, with the roundings spelled out, for the mask
 // kernel and the merge kernel below, so that both give the same bits.
+// G: lanes that share a row (32, or fewer when the pairs of several rows sit side by side in a warp).  Lanes
+// without a pair contribute max(., -inf) and + 0, both exact, so the result does not depend on G.
+template <int G = 32>
 __device__ __forceinline__ float warp_merge_lse(float m_l, float s_l) {
   float m_w = m_l;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
+  for (int o = G / 2; o > 0; o >>= 1) m_w = fmaxf(m_w, __shfl_xor_sync(kFullMask, m_w, o));
   float s_w = (m_l > -INFINITY) ? __fmul_rn(s_l, expf(m_l - m_w)) : 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) s_w = __fadd_rn(s_w, __shfl_xor_sync(kFullMask, s_w, o));
+  for (int o = G / 2; o > 0; o >>= 1) s_w = __fadd_rn(s_w, __shfl_xor_sync(kFullMask, s_w, o));
   return __fadd_rn(m_w, logf(s_w));
 }
 
@@ -387,25 +390,27 @@ gtm_allow_bloom_cluster_kernel(const MaskParams p, int log2_words_per_cta) {
 
 // The rows' log-sum-exp from the partials a logits GEMM left per 256-column tile, when the mask ran BEFORE that
 // GEMM (allow bits first, so that the GEMM stores only allowed logits): one warp per row, the arithmetic of the
-// mask kernel's own merge; dead rows (no node, or a leaf) get 0 as there.
+// mask kernel's own merge; dead rows (no node, or a leaf) get 0 as there.  G lanes per row, 32 / G rows per warp.
+template <int G>
 __global__ void __launch_bounds__(256)
 row_lse_from_parts_kernel(const float2* __restrict__ lse_part, int n_parts, const int32_t* __restrict__ beam_node,
                           int64_t num_internal, float* __restrict__ row_lse, int R) {
   pdl_wait();
   pdl_trigger();
   const int lane = threadIdx.x & 31;
-  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (r >= R) return;
-  const int node = __ldg(beam_node + r);
+  const int part = lane % G;
+  const int r = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + lane / G;
+  const bool in_range = r < R;                             // (whole warps stay: the merge shuffles over all lanes)
+  const int node = in_range ? __ldg(beam_node + r) : -1;
   const bool dead = node < 0 || node >= num_internal;
   float m_l = -INFINITY, s_l = 0.f;
-  if (!dead && lane < n_parts) {
-    const float2 pr = __ldg(lse_part + (int64_t)r * n_parts + lane);
+  if (!dead && part < n_parts) {
+    const float2 pr = __ldg(lse_part + (int64_t)r * n_parts + part);
     m_l = pr.x;
     s_l = pr.y;
   }
-  const float lse = dead ? 0.f : warp_merge_lse(m_l, s_l);
-  if (lane == 0) row_lse[r] = lse;
+  const float merged = warp_merge_lse<G>(m_l, s_l);
+  if (in_range && part == 0) row_lse[r] = dead ? 0.f : merged;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -756,8 +761,15 @@ extern "C" grace_status_t grace_row_lse_from_parts(const float* lse_part, int n_
   if (!lse_part || !beam_node || !trie || !row_lse || R <= 0 || n_parts < 1 || n_parts > 32 ||
       (reinterpret_cast<uintptr_t>(lse_part) & 7))
     return GRACE_INVALID_ARG;
-  grace::launch_pdl(grace::row_lse_from_parts_kernel, dim3((R + 7) / 8), dim3(256), 0, (cudaStream_t)stream,
-                    reinterpret_cast<const float2*>(lse_part), n_parts, beam_node, trie->num_internal, row_lse, R);
+  const float2* parts = reinterpret_cast<const float2*>(lse_part);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int64_t ni = trie->num_internal;
+  if (n_parts <= 8)
+    grace::launch_pdl(grace::row_lse_from_parts_kernel<8>, dim3((R + 31) / 32), dim3(256), 0, s, parts, n_parts, beam_node, ni, row_lse, R);
+  else if (n_parts <= 16)
+    grace::launch_pdl(grace::row_lse_from_parts_kernel<16>, dim3((R + 15) / 16), dim3(256), 0, s, parts, n_parts, beam_node, ni, row_lse, R);
+  else
+    grace::launch_pdl(grace::row_lse_from_parts_kernel<32>, dim3((R + 7) / 8), dim3(256), 0, s, parts, n_parts, beam_node, ni, row_lse, R);
   GRACE_LAUNCH_CHECK();
   return GRACE_OK;
 }

@@ -982,6 +982,21 @@ def test_allow_bits_before_the_logits_and_the_merge_of_their_partials(api):
         assert lse_b[5].item() == 0.0
         _, a_ref, _ = OG.gtm_mask(logp, score, node, key, 1, trie, om, B, M)
         assert np.array_equal(allow_b.cpu().numpy().view(np.uint64), OG.pack_allow_bits(a_ref))
+    # other numbers of partials per row (the merge kernel packs 4, 2 or 1 rows into a warp): against the definition
+    rng = synth.rng_for(4, 1201)
+    for n_parts in (1, 2, 8, 12, 16, 17, 32):
+        R = B * M
+        mx = synth.normal_f32(rng, (R, n_parts), 4.0)
+        sm = (1.0 + rng.random((R, n_parts)) * 255.0).astype(np.float32)
+        part = dev(np.stack([mx, sm], axis=2).astype(np.float32))
+        out = torch.full((R,), 9.0, device=DEV)
+        api.grace_row_lse_from_parts(part, dev(node), trie_s, out)
+        torch.cuda.synchronize()
+        m64 = mx.astype(np.float64)
+        want = m64.max(1) + np.log((sm.astype(np.float64) * np.exp(m64 - m64.max(1, keepdims=True))).sum(1))
+        want[node < 0] = 0.0
+        leaf = node >= trie.num_internal_nodes()
+        np.testing.assert_allclose(out.cpu().numpy()[~leaf], want[~leaf], rtol=0, atol=2e-5)
 
 
 def test_l2_residency_window_is_a_hint_only(api):
