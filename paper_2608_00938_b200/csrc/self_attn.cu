@@ -173,8 +173,9 @@ static grace_status_t launch_np(const SelfAttnParams& p, int d_h, cudaStream_t s
     // thread halve and more warps fit (65536 rows x 512, T_self = 4: 103.7 -> 99.6 us, in place 89.4 -> 85.3;
     // T_self = 5: 124 -> 118); with fewer positions one warp per row is as fast or faster.
     case 2: return (T >= 4) ? launch_dh<T, 1>(p, d_h, s) : launch_dh<T, 2>(p, d_h, s);
-    case 3: case 4: return launch_dh<T, 4>(p, d_h, s);
-    default: return launch_dh<T, 4>(p, d_h, s);            // wider rows: segments of 4 x 32 pieces
+    // wider rows: segments of 4 x 32 pieces, one warp each; from three positions on segments of 32 pieces
+    // (16384 rows x 2048, in place: T_self = 3: 84.0 -> 80.4 us, T_self = 4: 107.7 -> 93.9 us)
+    default: return (T >= 3) ? launch_dh<T, 1>(p, d_h, s) : launch_dh<T, 4>(p, d_h, s);
   }
 }
 
