@@ -37,6 +37,12 @@ __device__ __forceinline__ uint32_t ordered_key(float x) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// One 32-byte store (a whole sector; the address must be 32-byte aligned).
+__device__ __forceinline__ void st_global_32B(void* p, const uint4& lo, const uint4& hi) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+}
+
 __device__ __forceinline__ void flag_status(int32_t* d_status, int bits) {
   if (d_status != nullptr) atomicOr(d_status, bits);
 }

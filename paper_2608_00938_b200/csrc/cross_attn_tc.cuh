@@ -42,8 +42,8 @@ template <int DH> struct CaCfg {
   static constexpr int kHalves = DH / 64;
   static constexpr int kTileBytes = kCaHalfBytes * kHalves;      // Q, K_blk or V_blk
   static constexpr int kSmemBytes = kTileBytes * (2 + 2 * kCaStages) + 1024 + kCaBarBytes + 2 * 2 * 128 * 4 + 2 * 2 * 128 * 4;
-  static constexpr uint32_t kTmemCols = DH == 64 ? 256 : 512;    // S: 0..127, O: 128..128+DH-1, P: the next 64
-  static constexpr int kCtasPerSm = DH == 64 ? 2 : 1;
+  static constexpr uint32_t kTmemCols = 512;                     // S: 0..127, O: 2 x DH (by item parity), P: 2 x 64 (by block parity)
+  static constexpr int kCtasPerSm = 1;
 };
 
 struct CrossTcParams {
@@ -91,8 +91,8 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   uint64_t* v_empty = v_full + kCaStages;     // [stages]
   uint64_t* s_full = v_empty + kCaStages;
   uint64_t* p_full = s_full + 1;
-  uint64_t* o_full = p_full + 1;
-  uint64_t* s_free = o_full + 1;
+  uint64_t* o_full = p_full + 1;              // [2] by block parity: P V of the block is complete
+  uint64_t* s_free = o_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_free + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* half_max = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + kCaBarBytes);   // [2][2][128]
@@ -110,6 +110,7 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     tc::mbar_init(s_full, 1);
     tc::mbar_init(p_full, kCaSoftmaxWarps);    // one arrival per softmax warp
     tc::mbar_init(o_full, 1);
+    tc::mbar_init(o_full + 1, 1);
     tc::mbar_init(s_free, kCaSoftmaxWarps);
     *abort_flag = 0;
     tc::fence_mbar_init();
@@ -122,8 +123,14 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   pdl_wait();                                  // barrier set-up and TMEM allocation overlapped the previous kernel's tail
   pdl_trigger();
   const uint32_t tmem_s = tmem_base;           // S fp32, 128 columns
-  const uint32_t tmem_o = tmem_base + 128;     // O fp32, DH columns
-  const uint32_t tmem_p = tmem_base + 128 + DH;   // P bf16 pairs, 64 columns
+  // O of an item lives in one of two accumulators (item parity) and P of a block in one of two column sets (block
+  // parity), so the softmax threads hand P(g) over and go straight on to block g + 1 (whose S is already there)
+  // while the tensor core runs P V of block g; an item's output is read and stored one block later, when its last
+  // P V has long finished.  With one K/V block per item (128 encoder positions) that takes the wait for P V and
+  // most of the output path out of the per-item chain.
+  static_assert(128 + 2 * DH + 2 * 64 <= 512, "TMEM columns");
+  const uint32_t tmem_o = tmem_base + 128;             // O fp32, 2 x DH columns
+  const uint32_t tmem_p = tmem_base + 128 + 2 * DH;    // P bf16 pairs, 2 x 64 columns
 
   if (warp == kCaSoftmaxWarps) {
     // ---------------- TMA producer ----------------
@@ -258,21 +265,22 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (!tc::mbar_wait(p_full, g & 1, abort_flag)) break;
         if (!tc::mbar_wait(v_full + s, (g >> 1) & 1, abort_flag)) break;
         tc::tc_fence_after();
+        const uint32_t o_acc = tmem_o + (uint32_t)((li & 1) * DH), p_cols = tmem_p + (uint32_t)((g & 1) * 64);
         if (s == 0) {
 #pragma unroll
           for (int hf = 0; hf < kHalves; ++hf)
 #pragma unroll
             for (int k = 0; k < kCaBN / 16; ++k)
-              tc::mma_ts(tmem_o + 64 * hf, tmem_p + 8 * k, v_desc[0][hf][k], idesc_o, (j | k) ? 1u : 0u);
+              tc::mma_ts(o_acc + 64 * hf, p_cols + 8 * k, v_desc[0][hf][k], idesc_o, (j | k) ? 1u : 0u);
         } else {
 #pragma unroll
           for (int hf = 0; hf < kHalves; ++hf)
 #pragma unroll
             for (int k = 0; k < kCaBN / 16; ++k)
-              tc::mma_ts(tmem_o + 64 * hf, tmem_p + 8 * k, v_desc[1][hf][k], idesc_o, (j | k) ? 1u : 0u);
+              tc::mma_ts(o_acc + 64 * hf, p_cols + 8 * k, v_desc[1][hf][k], idesc_o, (j | k) ? 1u : 0u);
         }
         tc::mma_commit(v_empty + s);                         // V of block g is consumed
-        tc::mma_commit(o_full);                              // O includes block g
+        tc::mma_commit(o_full + (g & 1));                    // O includes block g
         j = j1; li = li1;
       }
     }
@@ -288,10 +296,64 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int col_base = kCols * half;
     constexpr int kOutCols = DH / TPR;                     // output columns per thread
     bool ok = true;
-    int g = 0, n_done = 0;
-    for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
-      const int tile = item % p.tiles_m, bh = item / p.tiles_m;
+    int g = 0, n_done = 0, li = 0;
+    // the item whose output is still to be read from TMEM and stored (after the next block's P hand-over)
+    int pend_item = -1, pend_g = 0, pend_li = 0;
+    float pend_m = 0.f, pend_l = 0.f;
+    // wait for P V of global block gb (completion gb >> 1 of the barrier of its parity)
+    auto wait_pv = [&](int gb) -> bool {
+      bool w = tc::mbar_wait(o_full + (gb & 1), (gb >> 1) & 1, abort_flag);
+      return __all_sync(kFullMask, w);
+    };
+    auto store_item = [&](int item_e, int g_last, int li_e, float m_e, float l_e) -> bool {
+      const int tile = item_e % p.tiles_m, bh = item_e / p.tiles_m;
       const int h = bh % p.H, b = bh / p.H;
+      if (!wait_pv(g_last)) return false;
+      tc::tc_fence_after();
+      const uint32_t o_acc = tmem_o + (uint32_t)((li_e & 1) * DH);
+      uint32_t o[kOutCols];
+#pragma unroll
+      for (int c = 0; c < kOutCols; c += 32)
+        tc::tmem_ld32(o_acc + lane_addr + kOutCols * half + c, *reinterpret_cast<uint32_t(*)[32]>(&o[c]));
+      tc::tmem_ld_wait();
+      float l_tot = l_e;
+      if (TPR == 2) {
+        float* hs = half_sum + (n_done & 1) * 256;            // double-buffered by item parity
+        hs[half * 128 + row] = l_e;
+        tc::named_bar_sync(2 + quarter, 64);
+        l_tot += hs[(half ^ 1) * 128 + row];
+      }
+      ++n_done;
+      const int m = tile * kCaBM + row;
+      if (m < p.M) {
+        const float inv = 1.f / l_tot;
+        const int64_t r_out = (int64_t)b * p.M + m;
+        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * DH + kOutCols * half);
+        auto piece = [&](int i) {
+          return make_uint4(
+              pack_bf16x2(__uint_as_float(o[8 * i]) * inv, __uint_as_float(o[8 * i + 1]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv),
+              pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv));
+        };
+        // a thread owns a row: its stores are pieces at a row stride, so whole 32-byte sectors where the
+        // output's alignment allows (half the store transactions of 16-byte pieces)
+        if ((reinterpret_cast<uintptr_t>(dst) & 31) == 0) {
+#pragma unroll
+          for (int i = 0; i < kOutCols / 8; i += 2) st_global_32B(dst + i, piece(i), piece(i + 1));
+        } else {
+#pragma unroll
+          for (int i = 0; i < kOutCols / 8; ++i) dst[i] = piece(i);
+        }
+        if (p.lse != nullptr && half == 0) p.lse[r_out * p.H + h] = (m_e + log2f(l_tot)) * 0.6931471805599453f;
+      }
+      // the accumulator is free for the item after next: its first P V is issued only after these threads have
+      // arrived on p_full for that item's first block, which comes after this read in program order
+      tc::tc_fence_before();
+      return true;
+    };
+    for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x, ++li) {
+      const uint32_t o_acc = tmem_o + (uint32_t)((li & 1) * DH);
       float m_run = -INFINITY, l_run = 0.f;
       for (int j = 0; j < NB; ++j, ++g) {
         ok = ok && tc::mbar_wait(s_full, g & 1, abort_flag);
@@ -354,73 +416,51 @@ cross_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           r[2 * i + 1] = pack_bf16x2(e2, e3);
         }
         l_run = fmaf(l_run, alpha, (s0 + s1) + (s2 + s3));
-        if (j > 0) {
-          // P V of block j-1 reads the P columns and writes O: it must be complete before P of this
-          // block is stored and before O is rescaled.  (It was issued right after S of this block,
-          // so by now it has long finished.)
-          ok = tc::mbar_wait(o_full, (g - 1) & 1, abort_flag);
-          ok = __all_sync(kFullMask, ok);
+        if (g >= 2) {
+          // the P columns of this parity were read by P V of block g - 2: long finished, but it must be
+          ok = wait_pv(g - 2);
           if (!ok) break;
           tc::tc_fence_after();
         }
         {
 #pragma unroll
           for (int c = 0; c < kCols / 2; c += 16)
-            tc::tmem_st16(tmem_p + lane_addr + (kCols / 2) * half + c, *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
+            tc::tmem_st16(tmem_p + (uint32_t)((g & 1) * 64) + lane_addr + (kCols / 2) * half + c,
+                          *reinterpret_cast<uint32_t(*)[16]>(&r[c]));
         }
         if (j > 0 && __any_sync(kFullMask, grow)) {           // rare after the first blocks
+          // O changes under the tensor core only here: P V of block g - 1 (the same item) must be complete
+          ok = wait_pv(g - 1);
+          if (!ok) break;
+          tc::tc_fence_after();
 #pragma unroll
           for (int c = 0; c < kOutCols; c += 32) {
             uint32_t o[32];
-            tc::tmem_ld32(tmem_o + lane_addr + kOutCols * half + c, o);
+            tc::tmem_ld32(o_acc + lane_addr + kOutCols * half + c, o);
             tc::tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
             uint32_t (&o0)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[0]);
             uint32_t (&o1)[16] = *reinterpret_cast<uint32_t(*)[16]>(&o[16]);
-            tc::tmem_st16(tmem_o + lane_addr + kOutCols * half + c, o0);
-            tc::tmem_st16(tmem_o + lane_addr + kOutCols * half + c + 16, o1);
+            tc::tmem_st16(o_acc + lane_addr + kOutCols * half + c, o0);
+            tc::tmem_st16(o_acc + lane_addr + kOutCols * half + c + 16, o1);
           }
         }
         tc::tmem_st_wait();
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(p_full);
+        // the previous item's output, now that this block is with the tensor core
+        if (pend_item >= 0) {
+          ok = store_item(pend_item, pend_g, pend_li, pend_m, pend_l);
+          pend_item = -1;
+          if (!ok) break;
+        }
       }
       if (!ok) break;
-      // ---- epilogue of the item: O / l -> bf16 rows of out ----
-      ok = tc::mbar_wait(o_full, (g - 1) & 1, abort_flag);
-      ok = __all_sync(kFullMask, ok);
-      if (!ok) break;
-      tc::tc_fence_after();
-      uint32_t o[kOutCols];
-#pragma unroll
-      for (int c = 0; c < kOutCols; c += 32)
-        tc::tmem_ld32(tmem_o + lane_addr + kOutCols * half + c, *reinterpret_cast<uint32_t(*)[32]>(&o[c]));
-      tc::tmem_ld_wait();
-      float l_tot = l_run;
-      if (TPR == 2) {
-        float* hs = half_sum + (n_done & 1) * 256;            // double-buffered by item parity
-        hs[half * 128 + row] = l_run;
-        tc::named_bar_sync(2 + quarter, 64);
-        l_tot += hs[(half ^ 1) * 128 + row];
-      }
-      ++n_done;
-      const int m = tile * kCaBM + row;
-      if (m < p.M) {
-        const float inv = 1.f / l_tot;
-        const int64_t r_out = (int64_t)b * p.M + m;
-        uint4* dst = reinterpret_cast<uint4*>(p.out + r_out * p.out_row_stride + h * DH + kOutCols * half);
-#pragma unroll
-        for (int i = 0; i < kOutCols / 8; ++i)
-          dst[i] = make_uint4(
-              pack_bf16x2(__uint_as_float(o[8 * i]) * inv, __uint_as_float(o[8 * i + 1]) * inv),
-              pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv),
-              pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv),
-              pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv));
-        if (p.lse != nullptr && half == 0) p.lse[r_out * p.H + h] = (m_run + log2f(l_tot)) * 0.6931471805599453f;
-      }
+      pend_item = item; pend_g = g - 1; pend_li = li; pend_m = m_run; pend_l = l_run;
     }
+    if (ok && pend_item >= 0) store_item(pend_item, pend_g, pend_li, pend_m, pend_l);
   }
   tc::tc_fence_before();
   __syncthreads();

@@ -513,6 +513,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // shared memory (written above by the first warp group) are ordered against their readers by the two
         // barriers, which also carry the second half's partial to the thread that merges and stores it.
         tc::named_bar_sync(1, 256);
+        const bool sector_aligned = ((reinterpret_cast<uintptr_t>(y_direct) | (uintptr_t)(ldy * 4)) & 31) == 0;
 #pragma unroll 1
         for (int cc = 0; cc < 4; ++cc) {
           const int c = half * 4 + cc;
@@ -531,8 +532,14 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               if ((bits >> (8 * j)) & 0xffu) {
-                *reinterpret_cast<uint4*>(dst + 8 * j) = make_uint4(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3]);
-                *reinterpret_cast<uint4*>(dst + 8 * j + 4) = make_uint4(r[8 * j + 4], r[8 * j + 5], r[8 * j + 6], r[8 * j + 7]);
+                const uint4 lo = make_uint4(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3]);
+                const uint4 hi = make_uint4(r[8 * j + 4], r[8 * j + 5], r[8 * j + 6], r[8 * j + 7]);
+                if (sector_aligned) {
+                  st_global_32B(dst + 8 * j, lo, hi);
+                } else {
+                  *reinterpret_cast<uint4*>(dst + 8 * j) = lo;
+                  *reinterpret_cast<uint4*>(dst + 8 * j + 4) = hi;
+                }
               }
             }
           }
