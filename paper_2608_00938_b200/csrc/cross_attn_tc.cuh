@@ -6,8 +6,7 @@
 // blocks of 128:
 //   S   = Q K_blk^T        tcgen05.mma, A = Q (shared, K-major), B = K_blk (shared, K-major),
 //                          fp32 S[128 x 128] in TMEM
-//   P   = exp2(S*c - max)  softmax threads: TMEM lane = query row; head size 64: one thread per row
-//                          (128 threads); head size 128: two threads per row, half of the block's
+//   P   = exp2(S*c - max)  softmax threads: TMEM lane = query row; two threads per row, half of the block's
 //                          columns each (256 threads); P goes to its own TMEM columns as packed bf16
 //   O  += P V_blk          tcgen05.mma, A = P (TMEM), B = V_blk (shared, read MN-major, so V is
 //                          used as stored: no transpose anywhere); O stays in TMEM for the whole
@@ -17,12 +16,12 @@
 // permute / reshape chain of Section 5.1 costs nothing).  Ragged M and T are zero-filled by TMA
 // and masked in the softmax.  Warp roles: softmax + epilogue warps first, then the TMA producer warp, then
 // the MMA issuer warp.
-// The kernel is persistent (each CTA loops over work items; Q is double-buffered), so the next item's
-// loads and first S overlap the current item's epilogue.  Head size 64 runs two CTAs per SM (256 TMEM
-// columns each), so one CTA's MMAs run under the other's exponentials; head size 128 needs 320
-// columns (O is twice as wide) and 192 KB of tiles, so it runs one CTA per SM.  A 128-wide tile is
-// held as two 64-wide halves (the 128-byte swizzle spans 64 bf16), each with its own TMA box and its
-// own MMA k-steps (Q, K) or output-column half (V).
+// The kernel is persistent (each CTA loops over work items; Q is double-buffered), one CTA per SM with all
+// 512 TMEM columns: S (128), O twice (by item parity) and P twice (by block parity).  The softmax threads
+// therefore never wait for P V: they hand P of a block over and go on to the next block (whose S the tensor
+// core produced under their exponentials), and an item's output is read from TMEM and stored one block later.
+// A 128-wide tile is held as two 64-wide halves (the 128-byte swizzle spans 64 bf16), each with its own TMA
+// box and its own MMA k-steps (Q, K) or output-column half (V).
 #pragma once
 #include "common.cuh"
 #include "tc.cuh"
