@@ -25,23 +25,27 @@ def api():
 
 
 # ---- configuration 2: cross-attention op sweep ----------------------------------------------------
-@pytest.mark.parametrize("B,M,T", [(64, 256, 512), (64, 1024, 512), (64, 256, 1024), (64, 1024, 1024)])
-def test_cross_attn_config2_sampled_rows(api, B, M, T):
-    H, d = 8, 64
-    rng = synth.rng_for(2, M + T)
+@pytest.mark.parametrize("B,M,T,H,d", [(64, 256, 512, 8, 64), (64, 1024, 512, 8, 64), (64, 256, 1024, 8, 64),
+                                       (64, 1024, 1024, 8, 64),
+                                       # head size 128: several items per CTA (both O accumulators and both P column
+                                       # sets in turn), one K/V block per item (the paper's shape) and several, ragged T
+                                       (16, 1024, 128, 16, 128), (8, 1000, 300, 8, 128), (32, 2048, 1024, 4, 128)])
+def test_cross_attn_config2_sampled_rows(api, B, M, T, H, d):
+    rng = synth.rng_for(2, M + T + d)
     q = synth.normal_bf16(rng, (B * M, H, d))
     k = synth.normal_bf16(rng, (B, H, T, d))
     v = synth.normal_bf16(rng, (B, H, T, d))
     out = torch.zeros((B * M, H, d), dtype=torch.bfloat16, device=DEV)
     lse = torch.zeros((B * M, H), dtype=torch.float32, device=DEV)
-    api.grace_cross_attn(dev_bf16(q), dev_bf16(k), dev_bf16(v), out, 0.125, lse)
+    scale = float(d) ** -0.5
+    api.grace_cross_attn(dev_bf16(q), dev_bf16(k), dev_bf16(v), out, scale, lse)
     torch.cuda.synchronize()
     got = out.float().cpu().numpy()
     pick = np.random.default_rng(0)
     rows = pick.integers(0, B * M, size=4096)
     rows[:4] = [0, M - 1, M, B * M - 1]                        # tile and request boundaries
     heads = pick.integers(0, H, size=4096)
-    ref = np.stack([OA.cross_attn_row(f64(q[r, h]), f64(k[r // M, h]), f64(v[r // M, h]), 0.125)
+    ref = np.stack([OA.cross_attn_row(f64(q[r, h]), f64(k[r // M, h]), f64(v[r // M, h]), scale)
                     for r, h in zip(rows, heads)])
     assert_attention_close(got[rows, heads], ref, f"cross-attn B{B} M{M} T{T}")
     assert np.isfinite(got).all() and np.isfinite(lse.cpu().numpy()).all()

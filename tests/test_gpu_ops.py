@@ -612,19 +612,22 @@ def test_cross_attn_with_per_request_encoder_lengths(api, B, M, H, d, T):
     np.testing.assert_allclose(got_lse[~empty], lse_ref[~empty], atol=2e-3, rtol=0)
 
 
-def test_cross_attn_with_scores_that_keep_growing(api):
+@pytest.mark.parametrize("B,M,H,d,T", [(2, 300, 2, 64, 640),
+                                       # head size 128 (its own kernel and threshold, 2^8), several items per CTA so
+                                       # that both output accumulators are rescaled under way
+                                       (20, 300, 8, 128, 640)])
+def test_cross_attn_with_scores_that_keep_growing(api, B, M, H, d, T):
     """Keys whose scores rise along the encoder positions by far more than the lazy-rescaling threshold
     (2^16 between neighbouring blocks): the running maximum moves in almost every block and the output
     accumulator is rescaled under way; and rows whose maximum sits in the first block, where it never is."""
-    B, M, H, d, T = 2, 300, 2, 64, 640
-    rng = synth.rng_for(2, 950)
+    rng = synth.rng_for(2, 950 + d)
     q = np.abs(synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, M, H, d)))) + 0.5     # positive queries
     q[:, ::2] *= -1.0                                                                  # every second row: scores fall instead
     ramp = np.linspace(0.0, 9.0, T, dtype=np.float32)[None, None, :, None]
     k = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, H, T, d))) * 0.1 + ramp
     v = synth.bf16_bits_to_f32(synth.normal_bf16(rng, (B, H, T, d)))
     qb, kb, vb = synth.f32_to_bf16_bits(q), synth.f32_to_bf16_bits(k), synth.f32_to_bf16_bits(v)
-    scale = 0.125
+    scale = 0.125 if d == 64 else 0.125 * 0.5
     ref, _ = OA.cross_attn(f64(qb), f64(kb), f64(vb), scale)
     s_first = (f64(qb)[0, 1, 0] @ f64(kb)[0, 0].T) * scale * np.log2(np.e)
     assert s_first[-1] - s_first[63] > 100.0                    # several thresholds of growth for the rising rows
