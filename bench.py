@@ -251,11 +251,12 @@ def op_breakdown(dec, cfg, reps=3):
     scale = 1.0 / np.sqrt(dh)
     times, flops, counts = {}, {}, {}
     pending = []
+    rep_index = [0]
 
     def timed(name, fn, fl=0.0):
         a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
         a.record(); fn(); b.record()
-        pending.append((name, a, b))
+        pending.append((name, a, b, rep_index[0]))
         flops[name] = flops.get(name, 0.0) + fl
         counts[name] = counts.get(name, 0) + 1
 
@@ -285,7 +286,8 @@ def op_breakdown(dec, cfg, reps=3):
         add_into_x = lambda a, w, x: api.grace_linear_add_bf16(a, w, x)
     else:
         add_into_x = lambda a, w, x: api.grace_linear(a, w, x, x)
-    for _ in range(reps):
+    for rep_no in range(reps):
+        rep_index[0] = rep_no
         dec.reset()
         for t in range(L):
             M, K = sizes[t], sizes[t + 1]
@@ -386,8 +388,13 @@ def op_breakdown(dec, cfg, reps=3):
                                                                dec.node[nxt][:B * K], dec.key[nxt][:B * K], B, K, M, t,
                                                                dec.d_status))
     torch.cuda.synchronize()
-    for name, a, b in pending:
-        times[name] = times.get(name, 0.0) + a.elapsed_time(b)
+    # per op: the median over the passes of its time per loop (a host hiccup between an event and the launch behind
+    # it would otherwise count as kernel time); times[] holds that median times the number of passes
+    per_rep = {}
+    for name, a, b, rep_no in pending:
+        per_rep.setdefault(name, [0.0] * reps)[rep_no] += a.elapsed_time(b)
+    for name, vals in per_rep.items():
+        times[name] = sorted(vals)[len(vals) // 2] * reps
     total = sum(times.values())
     return {name: dict(ms_per_loop=times[name] / reps, share=times[name] / total, calls_per_loop=counts[name] // reps,
                        flops_per_loop=flops[name] / reps) for name in times}
