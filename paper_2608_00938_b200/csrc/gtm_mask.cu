@@ -49,6 +49,7 @@ __device__ __forceinline__ int nth_set_bit64(uint64_t word, int n) {
 }
 
 constexpr int kMaskWarpsPerBlock = 8;
+constexpr int kMaskSplitWarps = 32;      // SPLIT: warps that share one row (a CTA of 1024 threads)
 
 // The log-sum-exp of a row from per-lane (maximum, sum of e^(x - maximum)) pairs (lanes without a pair pass
 // (-inf, 0)): every lane returns the same value.  One definition, with the roundings spelled out, for the mask
@@ -75,23 +76,23 @@ __device__ __forceinline__ float warp_merge_lse(float m_l, float s_l) {
 //      log-probabilities is read only if one of its tokens is allowed.
 // LOGITS = true: `logp` holds raw logits; the row's log-sum-exp is taken in a first streaming pass
 // and cand = score + (logit - lse) for allowed tokens.
-// SPLIT = true (few rows, e.g. step 0 with one beam per request): the eight warps of a CTA share ONE
-// row: each takes every eighth group of 32 children in phase 1 and every eighth group of 128 tokens in
+// SPLIT = true (few rows, e.g. step 0 with one beam per request): the 32 warps of a 1024-thread CTA share ONE
+// row: each takes every 32nd group of 32 children in phase 1 and every 32nd group of 128 tokens in
 // the streaming passes; the warp-level synchronisation points become CTA barriers.
 template <int KIND, bool LOGITS, bool SPLIT>
-__global__ void __launch_bounds__(kMaskWarpsPerBlock * 32)
+__global__ void __launch_bounds__((SPLIT ? kMaskSplitWarps : kMaskWarpsPerBlock) * 32)
 gtm_mask_kernel(const MaskParams p) {
   __shared__ uint64_t s_words[kMaskWarpsPerBlock][32];
   __shared__ unsigned long long s_allow[kMaskWarpsPerBlock][32];
   __shared__ int s_incl[kMaskWarpsPerBlock][32];
-  __shared__ float s_lse[2][kMaskWarpsPerBlock];
+  __shared__ float s_lse[2][kMaskSplitWarps];
   pdl_wait();
   pdl_trigger();
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int r = SPLIT ? (int)blockIdx.x : (int)blockIdx.x * kMaskWarpsPerBlock + wib;
   if (r >= p.R) return;
   const int part = SPLIT ? wib : 0;                      // this warp's share of the row's work
-  constexpr int kParts = SPLIT ? kMaskWarpsPerBlock : 1;
+  constexpr int kParts = SPLIT ? kMaskSplitWarps : 1;
   auto sync_row = [&]() { if (SPLIT) __syncthreads(); else __syncwarp(); };
   const int V = p.V;
   const int W = V >> 6;
@@ -158,9 +159,9 @@ gtm_mask_kernel(const MaskParams p) {
     __syncthreads();
     if (!dead) {
       float m_c = -INFINITY;
-      for (int w = 0; w < kMaskWarpsPerBlock; ++w) m_c = fmaxf(m_c, s_lse[0][w]);
+      for (int w = 0; w < kParts; ++w) m_c = fmaxf(m_c, s_lse[0][w]);
       float s_c = 0.f;
-      for (int w = 0; w < kMaskWarpsPerBlock; ++w)
+      for (int w = 0; w < kParts; ++w)
         if (s_lse[0][w] > -INFINITY) s_c += s_lse[1][w] * expf(s_lse[0][w] - m_c);
       lse = m_c + logf(s_c);
     }
@@ -663,7 +664,7 @@ static grace_status_t launch_mask(const float* logp, bool logits, float* row_lse
   // few rows: a CTA per row, so that the row's matcher look-ups and its streaming passes use eight warps
   const bool split = p.R <= 2048;
   const int blocks = split ? p.R : (p.R + kMaskWarpsPerBlock - 1) / kMaskWarpsPerBlock;
-  const int threads = kMaskWarpsPerBlock * 32;
+  const int threads = (split ? kMaskSplitWarps : kMaskWarpsPerBlock) * 32;
 #define GRACE_MASK_LAUNCH(K)                                                      \
   do {                                                                            \
     if (logits && split) gtm_mask_kernel<K, true, true><<<blocks, threads, 0, s>>>(p);        \
